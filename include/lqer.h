@@ -1,0 +1,162 @@
+/*
+ * lqer.h - C ABI of the B200 (sm_100a) LQER / L2QER inference linear layer.
+ *
+ *   Y = X W_q + (X A_k) B_k                        (paper Section 3.1, Section 3.2)
+ *
+ * W_q is the MXINT4 weight (4-bit mantissas, one shared power-of-two exponent per
+ * block of 16 along K), X is quantised on the fly to MXINT8 (blocks of 16 along K),
+ * A_k [K,k] and B_k [k,N] are the rank-k factors in MXINT8 (Section 2.2, Section 4.1).
+ *
+ * Conventions
+ *  - Plain C.  Every function returns lqer_status_t (LQER_OK == 0) and never throws,
+ *    aborts or prints.
+ *  - Unless a parameter says "host", every data pointer is DEVICE memory owned by the
+ *    caller.  The library allocates no device memory (the one exception is stated at
+ *    its entry point) and never synchronises the stream except where stated.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *  - Matrices are dense row-major: X [M,K] fp32, W [K,N] fp32, A [K,k] fp32,
+ *    B [k,N] fp32, Y [M,N] fp32.  Pointers must be 16-byte aligned.
+ *  - Host-side argument checks run before any launch; on error nothing is launched
+ *    and outputs are untouched.  Conditions that only the device can see (a bounded
+ *    wait that ran out) are written to a status word at the head of `workspace` and
+ *    read back with lqer_poll_status.
+ *  - Element value convention: value = mantissa * 2^(e - (bits - 2)), e the block's
+ *    shared exponent = clamp(floor(log2(max|v|)), exp_min, exp_max); mantissas are
+ *    rounded half-to-even and clamped to +-(2^(bits-1) - 1).  Exponents are stored
+ *    as one byte e + 127.
+ */
+#ifndef LQER_H
+#define LQER_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LQER_OK = 0,
+  LQER_ERR_NULL = 1,             /* a required pointer is NULL */
+  LQER_ERR_SHAPE = 2,            /* M/K/N/k out of range, K % 16 != 0, N % 8 != 0 */
+  LQER_ERR_ALIGN = 3,            /* a pointer is not 16-byte aligned */
+  LQER_ERR_CONFIG = 4,           /* unsupported lqer_config_t */
+  LQER_ERR_BUFFER_TOO_SMALL = 5, /* packed / workspace buffer smaller than required */
+  LQER_ERR_BAD_PACKED = 6,       /* packed buffer unknown to the library or header corrupt */
+  LQER_ERR_ARCH = 7,             /* current device is not compute capability 10.x */
+  LQER_ERR_CUDA = 8,             /* a CUDA runtime / driver call failed */
+  LQER_ERR_TIMEOUT = 9,          /* device side: a bounded wait ran out */
+  LQER_ERR_BOUNDS = 10           /* device side: an index check failed */
+} lqer_status_t;
+
+/* Format parameters (Section 3.1: b_l, b_h; Section 4.1: block size, exponent width). */
+typedef struct {
+  int w_bits;        /* mantissa bits of W_q: 4 */
+  int a_bits;        /* mantissa bits of X and of T = X A_k: 8 */
+  int lr_bits;       /* mantissa bits of A_k, B_k: 8 */
+  int block;         /* block size along the contraction dimension: 16 */
+  int exp_min;       /* shared-exponent clamp window, default [-56, 55] */
+  int exp_max;
+  int deterministic; /* 1: fixed reduction order (the only mode implemented) */
+} lqer_config_t;
+
+/* One call of a batch (Section 4.3: layers are independent). */
+typedef struct {
+  const float* X;     /* [M,K] */
+  int M;
+  const void* packed; /* prepared weights of this layer */
+  float* Y;           /* [M,N] */
+} lqer_call_t;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* lqer_status_string(lqer_status_t status);
+
+/* Fill *cfg (host) with the defaults above. */
+lqer_status_t lqer_default_config(lqer_config_t* cfg);
+
+/* Size in bytes (host out) of the packed buffer for a [K,N] layer of rank k (k may be 0).
+ * Storage follows Section 4.1: 4-bit mantissas + one exponent byte per 16 for W_q,
+ * 8-bit mantissas + one exponent byte per 16 for A_k and B_k, plus a 256-byte header
+ * and tile padding (N to a multiple of 128, K to a multiple of 64, k to a multiple of 16). */
+lqer_status_t lqer_packed_bytes(int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
+
+/* Size in bytes (host out) of the scratch `workspace` lqer_linear* needs for up to M_max rows.
+ * The workspace holds a 256-byte status area and the quantised activations [X_q | T_q]. */
+lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
+
+/* Weight preparation (Section 3.1: W_q = q(W); Section 4.1 formats): quantise W to MXINT4
+ * (blocks of 16 along K), A and B to MXINT8 (A: blocks of 16 along K; B: blocks of 16 along
+ * the rank, zero-padded to a multiple of 16) on the GPU and write the kernel layout into
+ * `packed` (device, >= lqer_packed_bytes, 256-byte aligned).  A and B may be NULL iff k == 0.
+ * Asynchronous on `stream`.  The buffer is registered with the library under its address. */
+lqer_status_t lqer_prepare_weights(const float* W, const float* A, const float* B, int K, int N, int k,
+                                   const lqer_config_t* cfg, void* packed, size_t packed_bytes, void* stream);
+
+/* Register a packed buffer that was produced earlier and copied to a new address
+ * (save / restore).  Reads the header back from the device: synchronises `stream`. */
+lqer_status_t lqer_attach_packed(const void* packed, size_t packed_bytes, void* stream);
+
+/* Forget a packed buffer (call before freeing it).  Host only. */
+lqer_status_t lqer_release_packed(const void* packed);
+
+/* Shape of a registered packed buffer (host outs, any may be NULL). */
+lqer_status_t lqer_packed_shape(const void* packed, int* K, int* N, int* k, int* k_pad);
+
+/* Canonical read-back of the packed operands for bit-exact comparison: two's-complement
+ * mantissas and exponent bytes (e + 127).  Any output pair may be NULL.  Device outputs:
+ * Wm [K,N], We [K/16,N], Am [K,k], Ae [K/16,k], Bm [k_pad,N], Be [k_pad/16,N]. */
+lqer_status_t lqer_export_weights(const void* packed, int8_t* Wm, uint8_t* We, int8_t* Am, uint8_t* Ae,
+                                  int8_t* Bm, uint8_t* Be, void* stream);
+
+/* Activation quantisation alone (Section 4.1: X_q in MXINT8, blocks [1,16]) with the same
+ * device routine the layer uses.  Outputs Xm [M,K] int8, Xe [M,K/16] bytes. */
+lqer_status_t lqer_quantize_activations(const float* X, int M, int K, const lqer_config_t* cfg,
+                                        int8_t* Xm, uint8_t* Xe, void* stream);
+
+/* The low-rank projection alone (Section 3.1: X A_k), re-quantised to the activation
+ * format: T_q = q(X_q A_q), blocks of 16 along the rank.  Runs the layer's own prologue
+ * kernel.  Outputs Tm [M,k_pad] int8, Te [M,k_pad/16] bytes.  Needs the same workspace
+ * as lqer_linear. */
+lqer_status_t lqer_project_lowrank(const float* X, int M, const void* packed, int8_t* Tm, uint8_t* Te,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/* The layer (Section 3.1 last display, Section 3.2 last display):
+ *   Y[M,N] = X_q W_q + q(X_q A_q) B_q,  fp32 accumulation of exactly represented products.
+ * M <= 16 runs the fused split-K decode kernel; larger M runs the activation prologue and
+ * the tensor-core GEMM over the concatenated contraction [X_q | T_q] . [W_q ; B_q].
+ * lqer_linear uses the default stream. */
+lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y,
+                          void* workspace, size_t workspace_bytes);
+lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, float* Y,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* n_calls independent layers back to back on one stream (`calls` is a HOST array).
+ * The workspace is reused by consecutive calls (stream order makes that safe) and must
+ * fit the largest of them. */
+lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same layer with host buffers: copies X (host, [M,K]) to the device part of `workspace`,
+ * runs the layer and copies Y back to Y_host ([M,N]); synchronises `stream` before it
+ * returns.  workspace must be lqer_workspace_bytes + 4*M*(K+N) bytes. */
+lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, float* Y_host,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/* Clear the status area at the head of a fresh workspace (asynchronous on `stream`).
+ * Call once after allocating the workspace and after an error was polled. */
+lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Read the device-side status word of `workspace` (synchronises `stream`). */
+lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_t* device_status);
+
+/* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel,
+ * 2 decode kernel, 3 tensor-core kernel.  Host only, process wide. */
+lqer_status_t lqer_set_path(int path);
+
+/* Number of kernels launched by the library in this process so far (host). */
+unsigned long long lqer_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQER_H */

@@ -1,0 +1,27 @@
+"""B200 (sm_100a) implementation of the LQER / L2QER inference linear layer.
+
+The package is a thin ctypes binding over the C ABI declared in include/lqer.h;
+every step of the layer runs in the CUDA library.  There is no CPU fallback:
+loading fails loudly when the library has not been built.
+"""
+from .binding import (  # noqa: F401
+    LqerError,
+    Config,
+    PackedWeights,
+    lib,
+    lib_path,
+    default_config,
+    packed_bytes,
+    workspace_bytes,
+    prepare_weights,
+    export_weights,
+    quantize_activations,
+    project_lowrank,
+    new_workspace,
+    linear,
+    linear_batched,
+    linear_host,
+    poll_status,
+    set_path,
+    launch_count,
+)

@@ -1,0 +1,237 @@
+"""ctypes binding of include/lqer.h.  Argument marshalling only.
+
+torch is used for device memory and streams; tensors are passed to the library
+as raw device pointers.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "lib", "liblqer.so")
+_lib = None
+
+STATUS_NAMES = ["LQER_OK", "LQER_ERR_NULL", "LQER_ERR_SHAPE", "LQER_ERR_ALIGN", "LQER_ERR_CONFIG",
+                "LQER_ERR_BUFFER_TOO_SMALL", "LQER_ERR_BAD_PACKED", "LQER_ERR_ARCH", "LQER_ERR_CUDA",
+                "LQER_ERR_TIMEOUT", "LQER_ERR_BOUNDS"]
+
+PATH_AUTO, PATH_SIMT, PATH_DECODE, PATH_TENSOR = 0, 1, 2, 3
+
+
+class LqerError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{what}: {name} ({lib().lqer_status_string(status).decode()})")
+
+
+class Config(C.Structure):
+    _fields_ = [("w_bits", C.c_int), ("a_bits", C.c_int), ("lr_bits", C.c_int), ("block", C.c_int),
+                ("exp_min", C.c_int), ("exp_max", C.c_int), ("deterministic", C.c_int)]
+
+
+class Call(C.Structure):
+    _fields_ = [("X", C.c_void_p), ("M", C.c_int), ("packed", C.c_void_p), ("Y", C.c_void_p)]
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> C.CDLL:
+    """The loaded CUDA library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2402_02446_b200.build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(_LIB_PATH)
+        vp, sz, i = C.c_void_p, C.c_size_t, C.c_int
+        cfgp = C.POINTER(Config)
+        sig = {
+            "lqer_status_string": (C.c_char_p, [i]),
+            "lqer_default_config": (i, [cfgp]),
+            "lqer_packed_bytes": (i, [i, i, i, cfgp, C.POINTER(sz)]),
+            "lqer_workspace_bytes": (i, [i, i, i, i, cfgp, C.POINTER(sz)]),
+            "lqer_prepare_weights": (i, [vp, vp, vp, i, i, i, cfgp, vp, sz, vp]),
+            "lqer_attach_packed": (i, [vp, sz, vp]),
+            "lqer_release_packed": (i, [vp]),
+            "lqer_packed_shape": (i, [vp, C.POINTER(i), C.POINTER(i), C.POINTER(i), C.POINTER(i)]),
+            "lqer_export_weights": (i, [vp, vp, vp, vp, vp, vp, vp, vp]),
+            "lqer_quantize_activations": (i, [vp, i, i, cfgp, vp, vp, vp]),
+            "lqer_project_lowrank": (i, [vp, i, vp, vp, vp, vp, sz, vp]),
+            "lqer_linear": (i, [vp, i, vp, vp, vp, sz]),
+            "lqer_linear_stream": (i, [vp, i, vp, vp, vp, sz, vp]),
+            "lqer_linear_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
+            "lqer_linear_host": (i, [vp, i, vp, vp, vp, sz, vp]),
+            "lqer_workspace_init": (i, [vp, sz, vp]),
+            "lqer_poll_status": (i, [vp, vp, C.POINTER(i)]),
+            "lqer_set_path": (i, [i]),
+            "lqer_launch_count": (C.c_ulonglong, []),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        raise LqerError(status, what)
+
+
+def _stream(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype=None) -> int:
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def default_config() -> Config:
+    cfg = Config()
+    _check(lib().lqer_default_config(C.byref(cfg)), "lqer_default_config")
+    return cfg
+
+
+def packed_bytes(K: int, N: int, k: int, cfg: Config | None = None) -> int:
+    cfg = cfg or default_config()
+    out = C.c_size_t()
+    _check(lib().lqer_packed_bytes(K, N, k, C.byref(cfg), C.byref(out)), "lqer_packed_bytes")
+    return out.value
+
+
+def workspace_bytes(M_max: int, K: int, N: int, k: int, cfg: Config | None = None) -> int:
+    cfg = cfg or default_config()
+    out = C.c_size_t()
+    _check(lib().lqer_workspace_bytes(M_max, K, N, k, C.byref(cfg), C.byref(out)), "lqer_workspace_bytes")
+    return out.value
+
+
+@dataclass
+class PackedWeights:
+    buf: torch.Tensor   # uint8 device buffer in the kernel layout
+    K: int
+    N: int
+    k: int
+    k_pad: int
+
+    @property
+    def ptr(self) -> int:
+        return self.buf.data_ptr()
+
+    def release(self) -> None:
+        lib().lqer_release_packed(self.ptr)
+
+
+def prepare_weights(W: torch.Tensor, A: torch.Tensor | None, B: torch.Tensor | None,
+                    cfg: Config | None = None, stream=None) -> PackedWeights:
+    cfg = cfg or default_config()
+    K, N = W.shape
+    k = 0 if A is None else A.shape[1]
+    nbytes = packed_bytes(K, N, k, cfg)
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    _check(lib().lqer_prepare_weights(_dev(W, torch.float32), None if k == 0 else _dev(A, torch.float32),
+                                      None if k == 0 else _dev(B, torch.float32), K, N, k, C.byref(cfg),
+                                      buf.data_ptr(), nbytes, _stream(stream)), "lqer_prepare_weights")
+    return PackedWeights(buf, K, N, k, (k + 15) // 16 * 16)
+
+
+def export_weights(P: PackedWeights, stream=None) -> dict:
+    dev = P.buf.device
+    out = {"Wm": torch.empty((P.K, P.N), dtype=torch.int8, device=dev),
+           "We": torch.empty((P.K // 16, P.N), dtype=torch.uint8, device=dev)}
+    ptrs = [out["Wm"].data_ptr(), out["We"].data_ptr()]
+    if P.k > 0:
+        out["Am"] = torch.empty((P.K, P.k), dtype=torch.int8, device=dev)
+        out["Ae"] = torch.empty((P.K // 16, P.k), dtype=torch.uint8, device=dev)
+        out["Bm"] = torch.empty((P.k_pad, P.N), dtype=torch.int8, device=dev)
+        out["Be"] = torch.empty((P.k_pad // 16, P.N), dtype=torch.uint8, device=dev)
+        ptrs += [out[n].data_ptr() for n in ("Am", "Ae", "Bm", "Be")]
+    else:
+        ptrs += [None] * 4
+    _check(lib().lqer_export_weights(P.ptr, *ptrs, _stream(stream)), "lqer_export_weights")
+    return out
+
+
+def quantize_activations(X: torch.Tensor, cfg: Config | None = None, stream=None):
+    cfg = cfg or default_config()
+    M, K = X.shape
+    Xm = torch.empty((M, K), dtype=torch.int8, device=X.device)
+    Xe = torch.empty((M, K // 16), dtype=torch.uint8, device=X.device)
+    _check(lib().lqer_quantize_activations(_dev(X, torch.float32), M, K, C.byref(cfg), Xm.data_ptr(),
+                                           Xe.data_ptr(), _stream(stream)), "lqer_quantize_activations")
+    return Xm, Xe
+
+
+def new_workspace(M_max: int, P: PackedWeights, extra_bytes: int = 0, stream=None) -> torch.Tensor:
+    n = workspace_bytes(M_max, P.K, P.N, P.k) + extra_bytes
+    ws = torch.empty(n, dtype=torch.uint8, device=P.buf.device)
+    _check(lib().lqer_workspace_init(ws.data_ptr(), n, _stream(stream)), "lqer_workspace_init")
+    return ws
+
+
+def project_lowrank(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, stream=None):
+    M = X.shape[0]
+    Tm = torch.empty((M, P.k_pad), dtype=torch.int8, device=X.device)
+    Te = torch.empty((M, P.k_pad // 16), dtype=torch.uint8, device=X.device)
+    _check(lib().lqer_project_lowrank(_dev(X, torch.float32), M, P.ptr, Tm.data_ptr(), Te.data_ptr(),
+                                      ws.data_ptr(), ws.numel(), _stream(stream)), "lqer_project_lowrank")
+    return Tm, Te
+
+
+def linear(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y: torch.Tensor | None = None, stream=None):
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, P.N), dtype=torch.float32, device=X.device)
+    _check(lib().lqer_linear_stream(_dev(X, torch.float32), M, P.ptr, _dev(Y, torch.float32), ws.data_ptr(),
+                                    ws.numel(), _stream(stream)), "lqer_linear_stream")
+    return Y
+
+
+def make_calls(items) -> "C.Array":
+    """items: iterable of (X, PackedWeights, Y) -> a host array of lqer_call_t."""
+    items = list(items)
+    arr = (Call * len(items))()
+    for j, (X, P, Y) in enumerate(items):
+        arr[j] = Call(_dev(X, torch.float32), X.shape[0], P.ptr, _dev(Y, torch.float32))
+    return arr
+
+
+def linear_batched(calls, ws: torch.Tensor, stream=None) -> None:
+    arr = calls if isinstance(calls, C.Array) else make_calls(calls)
+    _check(lib().lqer_linear_batched(arr, len(arr), ws.data_ptr(), ws.numel(), _stream(stream)),
+           "lqer_linear_batched")
+
+
+def linear_host(X_host: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y_host: torch.Tensor, stream=None):
+    """X_host / Y_host are (pinned) CPU tensors; copies both ways happen inside the call."""
+    if X_host.is_cuda or Y_host.is_cuda or not X_host.is_contiguous() or not Y_host.is_contiguous():
+        raise ValueError("expected contiguous CPU tensors")
+    _check(lib().lqer_linear_host(X_host.data_ptr(), X_host.shape[0], P.ptr, Y_host.data_ptr(), ws.data_ptr(),
+                                  ws.numel(), _stream(stream)), "lqer_linear_host")
+    return Y_host
+
+
+def poll_status(ws: torch.Tensor, stream=None) -> int:
+    out = C.c_int()
+    _check(lib().lqer_poll_status(ws.data_ptr(), _stream(stream), C.byref(out)), "lqer_poll_status")
+    return out.value
+
+
+def set_path(path: int) -> None:
+    _check(lib().lqer_set_path(path), "lqer_set_path")
+
+
+def launch_count() -> int:
+    return int(lib().lqer_launch_count())

@@ -1,0 +1,347 @@
+// Host side of the C ABI: argument checks, the registry of packed buffers, path selection.
+#include <atomic>
+#include <cstring>
+#include <mutex>
+#include <unordered_map>
+
+#include "lqer_common.cuh"
+
+namespace lqer {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+static std::mutex g_mu;
+static std::unordered_map<const void*, PackedMeta> g_registry;
+static std::atomic<int> g_path{0};
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static lqer_status_t check_config(const lqer_config_t* cfg) {
+  if (cfg == nullptr) return LQER_ERR_NULL;
+  if (cfg->w_bits != 4 || cfg->a_bits != 8 || cfg->lr_bits != 8 || cfg->block != 16) return LQER_ERR_CONFIG;
+  // every dequantised value must be a normal bf16 and every product a normal fp32
+  if (cfg->exp_min < -56 || cfg->exp_max > 55 || cfg->exp_min > cfg->exp_max) return LQER_ERR_CONFIG;
+  if (cfg->deterministic != 0 && cfg->deterministic != 1) return LQER_ERR_CONFIG;
+  return LQER_OK;
+}
+
+static lqer_status_t check_shape(int K, int N, int k) {
+  if (K <= 0 || N <= 0 || k < 0) return LQER_ERR_SHAPE;
+  if (K % 16 != 0 || N % 8 != 0) return LQER_ERR_SHAPE;
+  if (k > 256 || k > K || k > N) return LQER_ERR_SHAPE;
+  if ((long long)K > (1 << 20) || (long long)N > (1 << 22)) return LQER_ERR_SHAPE;
+  return LQER_OK;
+}
+
+static void fill_meta(PackedMeta& m, int K, int N, int k, const lqer_config_t& c) {
+  std::memset(&m, 0, sizeof(m));
+  m.magic = kMagic; m.version = kVersion;
+  m.K = K; m.N = N; m.k = k; m.k_pad = (k + 15) / 16 * 16;
+  m.K64 = (K + 63) / 64 * 64;
+  m.n_tiles = (N + kTileN - 1) / kTileN;
+  m.k_slabs = m.K64 / kSlabK;
+  m.r_blocks = m.k_pad / 16;
+  m.w_bits = c.w_bits; m.a_bits = c.a_bits; m.lr_bits = c.lr_bits; m.block = c.block;
+  m.exp_min = c.exp_min; m.exp_max = c.exp_max; m.deterministic = 1;
+  m.off_w = kHeaderBytes;
+  m.off_b = align_up(m.off_w + (size_t)m.n_tiles * m.k_slabs * kWTileBytes, 256);
+  m.off_a = align_up(m.off_b + (size_t)m.n_tiles * b_tile_bytes(m), 256);
+  m.total_bytes = align_up(m.off_a + (size_t)(K / 16) * m.k_pad * 17, 256);
+  m.checksum = meta_checksum(m);
+}
+
+static bool meta_valid(const PackedMeta& m) {
+  if (m.magic != kMagic || m.version != kVersion || m.checksum != meta_checksum(m)) return false;
+  lqer_config_t c{m.w_bits, m.a_bits, m.lr_bits, m.block, m.exp_min, m.exp_max, m.deterministic};
+  if (check_config(&c) != LQER_OK || check_shape(m.K, m.N, m.k) != LQER_OK) return false;
+  PackedMeta ref;
+  fill_meta(ref, m.K, m.N, m.k, c);
+  return std::memcmp(&ref, &m, sizeof(m)) == 0;
+}
+
+static lqer_status_t lookup(const void* packed, PackedMeta& out) {
+  if (packed == nullptr) return LQER_ERR_NULL;
+  std::lock_guard<std::mutex> lock(g_mu);
+  auto it = g_registry.find(packed);
+  if (it == g_registry.end()) return LQER_ERR_BAD_PACKED;
+  out = it->second;
+  return LQER_OK;
+}
+
+static lqer_status_t check_arch() {
+  static std::mutex mu;
+  static std::unordered_map<int, int> major_of;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LQER_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  auto it = major_of.find(dev);
+  if (it == major_of.end()) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return LQER_ERR_CUDA;
+    it = major_of.emplace(dev, major).first;
+  }
+  return it->second == 10 ? LQER_OK : LQER_ERR_ARCH;
+}
+
+static size_t xcat_bytes(const PackedMeta& m, int M) { return align_up((size_t)M * xcat_cols(m) * 2, 256); }
+
+static lqer_status_t run_linear(const float* X, int M, const void* packed, float* Y, void* workspace,
+                                size_t workspace_bytes, cudaStream_t s, int8_t* Tm, uint8_t* Te, bool project_only) {
+  if (X == nullptr || packed == nullptr || workspace == nullptr || (Y == nullptr && !project_only)) return LQER_ERR_NULL;
+  if (M <= 0 || M > (1 << 24)) return LQER_ERR_SHAPE;
+  if (!aligned16(X) || (Y != nullptr && !aligned16(Y)) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return LQER_ERR_ALIGN;
+  PackedMeta m;
+  lqer_status_t st = lookup(packed, m);
+  if (st != LQER_OK) return st;
+  if (workspace_bytes < kStatusBytes + xcat_bytes(m, M)) return LQER_ERR_BUFFER_TOO_SMALL;
+  if ((st = check_arch()) != LQER_OK) return st;
+  DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
+  void* xcat = static_cast<uint8_t*>(workspace) + kStatusBytes;
+  int path = g_path.load();
+  if (project_only) path = 3;
+  if (path == 0) path = (M <= decode_max_m()) ? 2 : 3;
+  cudaError_t err;
+  if (path == 2) {
+    if (M > decode_max_m()) return LQER_ERR_SHAPE;
+    err = launch_decode(X, M, m, packed, Y, dst, s);
+  } else {
+    if (path == 1 && M > 65535) return LQER_ERR_SHAPE;
+    err = launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
+    if (err == cudaSuccess && !project_only)
+      err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, Y, s) : launch_gemm_tc(xcat, M, m, packed, Y, dst, s);
+  }
+  return err == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+}
+
+}  // namespace lqer
+
+using namespace lqer;
+
+extern "C" {
+
+const char* lqer_status_string(lqer_status_t status) {
+  switch (status) {
+    case LQER_OK: return "ok";
+    case LQER_ERR_NULL: return "null pointer";
+    case LQER_ERR_SHAPE: return "unsupported shape";
+    case LQER_ERR_ALIGN: return "misaligned pointer";
+    case LQER_ERR_CONFIG: return "unsupported configuration";
+    case LQER_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case LQER_ERR_BAD_PACKED: return "unknown or corrupt packed buffer";
+    case LQER_ERR_ARCH: return "device is not compute capability 10.x";
+    case LQER_ERR_CUDA: return "CUDA call failed";
+    case LQER_ERR_TIMEOUT: return "device-side wait timed out";
+    case LQER_ERR_BOUNDS: return "device-side bounds check failed";
+  }
+  return "unknown status";
+}
+
+lqer_status_t lqer_default_config(lqer_config_t* cfg) {
+  if (cfg == nullptr) return LQER_ERR_NULL;
+  *cfg = lqer_config_t{4, 8, 8, 16, -56, 55, 1};
+  return LQER_OK;
+}
+
+lqer_status_t lqer_packed_bytes(int K, int N, int k, const lqer_config_t* cfg, size_t* bytes) {
+  if (bytes == nullptr) return LQER_ERR_NULL;
+  lqer_status_t st = check_config(cfg);
+  if (st != LQER_OK) return st;
+  if ((st = check_shape(K, N, k)) != LQER_OK) return st;
+  PackedMeta m;
+  fill_meta(m, K, N, k, *cfg);
+  *bytes = (size_t)m.total_bytes;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes) {
+  if (bytes == nullptr) return LQER_ERR_NULL;
+  lqer_status_t st = check_config(cfg);
+  if (st != LQER_OK) return st;
+  if ((st = check_shape(K, N, k)) != LQER_OK) return st;
+  if (M_max <= 0 || M_max > (1 << 24)) return LQER_ERR_SHAPE;
+  PackedMeta m;
+  fill_meta(m, K, N, k, *cfg);
+  *bytes = kStatusBytes + xcat_bytes(m, M_max);
+  return LQER_OK;
+}
+
+lqer_status_t lqer_prepare_weights(const float* W, const float* A, const float* B, int K, int N, int k,
+                                   const lqer_config_t* cfg, void* packed, size_t packed_bytes, void* stream) {
+  if (W == nullptr || packed == nullptr) return LQER_ERR_NULL;
+  lqer_status_t st = check_config(cfg);
+  if (st != LQER_OK) return st;
+  if ((st = check_shape(K, N, k)) != LQER_OK) return st;
+  if (k > 0 && (A == nullptr || B == nullptr)) return LQER_ERR_NULL;
+  if (!aligned16(W) || (k > 0 && (!aligned16(A) || !aligned16(B))) || (reinterpret_cast<uintptr_t>(packed) & 255u) != 0)
+    return LQER_ERR_ALIGN;
+  PackedMeta m;
+  fill_meta(m, K, N, k, *cfg);
+  if (packed_bytes < m.total_bytes) return LQER_ERR_BUFFER_TOO_SMALL;
+  if ((st = check_arch()) != LQER_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  {
+    // the header travels with the buffer; the registry keeps a stable host copy for the async copy
+    std::lock_guard<std::mutex> lock(g_mu);
+    PackedMeta& slot = g_registry[packed];
+    slot = m;
+    if (cudaMemcpyAsync(packed, &slot, sizeof(PackedMeta), cudaMemcpyHostToDevice, s) != cudaSuccess) {
+      g_registry.erase(packed);
+      return LQER_ERR_CUDA;
+    }
+  }
+  if (launch_pack(W, A, B, m, packed, s) != cudaSuccess) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_registry.erase(packed);
+    return LQER_ERR_CUDA;
+  }
+  return LQER_OK;
+}
+
+lqer_status_t lqer_attach_packed(const void* packed, size_t packed_bytes, void* stream) {
+  if (packed == nullptr) return LQER_ERR_NULL;
+  if (packed_bytes < (size_t)kHeaderBytes) return LQER_ERR_BUFFER_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(packed) & 255u) != 0) return LQER_ERR_ALIGN;
+  PackedMeta m;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&m, packed, sizeof(m), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LQER_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return LQER_ERR_CUDA;
+  if (!meta_valid(m)) return LQER_ERR_BAD_PACKED;
+  if (packed_bytes < m.total_bytes) return LQER_ERR_BUFFER_TOO_SMALL;
+  std::lock_guard<std::mutex> lock(g_mu);
+  g_registry[packed] = m;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_release_packed(const void* packed) {
+  if (packed == nullptr) return LQER_ERR_NULL;
+  std::lock_guard<std::mutex> lock(g_mu);
+  return g_registry.erase(packed) ? LQER_OK : LQER_ERR_BAD_PACKED;
+}
+
+lqer_status_t lqer_packed_shape(const void* packed, int* K, int* N, int* k, int* k_pad) {
+  PackedMeta m;
+  lqer_status_t st = lookup(packed, m);
+  if (st != LQER_OK) return st;
+  if (K) *K = m.K;
+  if (N) *N = m.N;
+  if (k) *k = m.k;
+  if (k_pad) *k_pad = m.k_pad;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_export_weights(const void* packed, int8_t* Wm, uint8_t* We, int8_t* Am, uint8_t* Ae,
+                                  int8_t* Bm, uint8_t* Be, void* stream) {
+  PackedMeta m;
+  lqer_status_t st = lookup(packed, m);
+  if (st != LQER_OK) return st;
+  if ((st = check_arch()) != LQER_OK) return st;
+  return launch_export(m, packed, Wm, We, Am, Ae, Bm, Be, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LQER_OK : LQER_ERR_CUDA;
+}
+
+lqer_status_t lqer_quantize_activations(const float* X, int M, int K, const lqer_config_t* cfg, int8_t* Xm,
+                                        uint8_t* Xe, void* stream) {
+  if (X == nullptr || (Xm == nullptr && Xe == nullptr)) return LQER_ERR_NULL;
+  lqer_status_t st = check_config(cfg);
+  if (st != LQER_OK) return st;
+  if (M <= 0 || K <= 0 || K % 16 != 0 || M > (1 << 24) || K > (1 << 20)) return LQER_ERR_SHAPE;
+  if (!aligned16(X) || (Xm != nullptr && (reinterpret_cast<uintptr_t>(Xm) & 3u) != 0)) return LQER_ERR_ALIGN;
+  if ((st = check_arch()) != LQER_OK) return st;
+  return launch_quantize_x(X, M, K, cfg->a_bits, cfg->exp_min, cfg->exp_max, Xm, Xe,
+                           static_cast<cudaStream_t>(stream)) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+}
+
+lqer_status_t lqer_project_lowrank(const float* X, int M, const void* packed, int8_t* Tm, uint8_t* Te,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+  if (Tm == nullptr && Te == nullptr) return LQER_ERR_NULL;
+  PackedMeta m;
+  lqer_status_t st = lookup(packed, m);
+  if (st != LQER_OK) return st;
+  if (m.k == 0) return LQER_ERR_SHAPE;
+  return run_linear(X, M, packed, nullptr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), Tm, Te, true);
+}
+
+lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, float* Y, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  return run_linear(X, M, packed, Y, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), nullptr,
+                    nullptr, false);
+}
+
+lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y, void* workspace,
+                          size_t workspace_bytes) {
+  return lqer_linear_stream(X, M, packed, Y, workspace, workspace_bytes, nullptr);
+}
+
+lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+  if (calls == nullptr) return LQER_ERR_NULL;
+  if (n_calls < 0) return LQER_ERR_SHAPE;
+  // validate everything before the first launch
+  for (int i = 0; i < n_calls; ++i) {
+    const lqer_call_t& c = calls[i];
+    if (c.X == nullptr || c.packed == nullptr || c.Y == nullptr || workspace == nullptr) return LQER_ERR_NULL;
+    if (c.M <= 0 || c.M > (1 << 24)) return LQER_ERR_SHAPE;
+    if (!aligned16(c.X) || !aligned16(c.Y)) return LQER_ERR_ALIGN;
+    PackedMeta m;
+    lqer_status_t st = lookup(c.packed, m);
+    if (st != LQER_OK) return st;
+    if (workspace_bytes < kStatusBytes + xcat_bytes(m, c.M)) return LQER_ERR_BUFFER_TOO_SMALL;
+  }
+  for (int i = 0; i < n_calls; ++i) {
+    lqer_status_t st = lqer_linear_stream(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace,
+                                          workspace_bytes, stream);
+    if (st != LQER_OK) return st;
+  }
+  return LQER_OK;
+}
+
+lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, float* Y_host, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+  if (X_host == nullptr || Y_host == nullptr || workspace == nullptr) return LQER_ERR_NULL;
+  if (M <= 0 || M > (1 << 24)) return LQER_ERR_SHAPE;
+  PackedMeta m;
+  lqer_status_t st = lookup(packed, m);
+  if (st != LQER_OK) return st;
+  const size_t core = kStatusBytes + xcat_bytes(m, M);
+  const size_t xb = align_up((size_t)M * m.K * 4, 256), yb = align_up((size_t)M * m.N * 4, 256);
+  if (workspace_bytes < core + xb + yb) return LQER_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  float* Xd = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + core);
+  float* Yd = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + core + xb);
+  if (cudaMemcpyAsync(Xd, X_host, (size_t)M * m.K * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return LQER_ERR_CUDA;
+  if ((st = lqer_linear_stream(Xd, M, packed, Yd, workspace, core, stream)) != LQER_OK) return st;
+  if (cudaMemcpyAsync(Y_host, Yd, (size_t)M * m.N * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LQER_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return LQER_ERR_CUDA;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (workspace == nullptr) return LQER_ERR_NULL;
+  if (workspace_bytes < (size_t)kStatusBytes) return LQER_ERR_BUFFER_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
+  return cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LQER_OK : LQER_ERR_CUDA;
+}
+
+lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_t* device_status) {
+  if (workspace == nullptr || device_status == nullptr) return LQER_ERR_NULL;
+  DeviceStatus h;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LQER_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return LQER_ERR_CUDA;
+  *device_status = (h.code >= 0 && h.code <= LQER_ERR_BOUNDS) ? (lqer_status_t)h.code : LQER_ERR_CUDA;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_set_path(int path) {
+  if (path < 0 || path > 3) return LQER_ERR_CONFIG;
+  g_path.store(path);
+  return LQER_OK;
+}
+
+unsigned long long lqer_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

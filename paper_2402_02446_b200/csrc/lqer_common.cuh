@@ -1,0 +1,130 @@
+// Internal declarations shared by the translation units of the LQER library:
+// the packed weight layout, the MXINT quantisation device routines and the
+// launch wrappers of each kernel family.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lqer.h"
+
+namespace lqer {
+
+// ----------------------------------------------------------------------------
+// Packed weight layout
+// ----------------------------------------------------------------------------
+// header (256 B)
+// W section: tiles [n_tile][k_slab], one tile = 128 output columns x 64 K:
+//     nibbles [bp 2][n 128][16 B]   (bp = pair of 16-blocks; 16 B = 32 nibbles of one column)
+//     exps    [n 128][4 B]          (the slab's four block exponents of one column)
+//   Within a 32-bit word, nibble position p holds k_local = {0,2,4,6,1,3,5,7}[p] of the
+//   word's eight consecutive K, offset-binary (mantissa + 8), so that
+//   (w >> 4i) & 0x000F000F yields the adjacent pair (2i, 2i+1).
+// B section: per n_tile:  mantissas [rb][n 128][16 B int8]  then exps [rb][n 128]
+// A section: mantissas [K/16][k_pad][16 B int8]  then exps [K/16][k_pad]
+constexpr uint32_t kMagic = 0x5245514Cu;  // "LQER"
+constexpr uint32_t kVersion = 1;
+constexpr int kHeaderBytes = 256;
+constexpr int kTileN = 128;
+constexpr int kSlabK = 64;
+constexpr int kWTileBytes = kTileN * kSlabK / 2 + kTileN * 4;  // 4608
+constexpr int kWTileNibbleBytes = kTileN * kSlabK / 2;          // 4096
+constexpr int kStatusBytes = 256;
+
+struct PackedMeta {
+  uint32_t magic, version;
+  int32_t K, N, k, k_pad;
+  int32_t K64, n_tiles, k_slabs, r_blocks;
+  int32_t w_bits, a_bits, lr_bits, block, exp_min, exp_max, deterministic;
+  int32_t reserved0;
+  uint64_t off_w, off_b, off_a, total_bytes;
+  uint32_t checksum;
+  uint32_t pad_[64 - 27];
+};
+static_assert(sizeof(PackedMeta) == kHeaderBytes, "header must be 256 bytes");
+
+inline uint32_t meta_checksum(const PackedMeta& m) {
+  const uint32_t* w = reinterpret_cast<const uint32_t*>(&m);
+  uint32_t h = 2166136261u;
+  for (int i = 0; i < 26; ++i) { h ^= w[i]; h *= 16777619u; }
+  return h;
+}
+
+__host__ __device__ inline int b_tile_bytes(const PackedMeta& m) { return m.r_blocks * kTileN * 17; }
+__host__ __device__ inline size_t xcat_cols(const PackedMeta& m) { return (size_t)m.K64 + (size_t)m.k_pad; }
+
+// ----------------------------------------------------------------------------
+// MXINT quantisation (value = m * 2^(e - (bits-2)), round half to even, symmetric clamp)
+// ----------------------------------------------------------------------------
+__device__ __forceinline__ float abs_ignore_nan(float v) { return (v != v) ? 0.0f : fabsf(v); }
+
+// Shared exponent of a block from its maximum magnitude: the fp32 exponent field, clamped.
+__device__ __forceinline__ int block_exponent(float amax, int emin, int emax) {
+  int field = (int)((__float_as_uint(amax) >> 23) & 0xFFu);
+  return min(max(field - 127, emin), emax);
+}
+__device__ __forceinline__ int block_exponent(double amax, int emin, int emax) {
+  int field = (__double2hiint(amax) >> 20) & 0x7FF;
+  return min(max(field - 1023, emin), emax);
+}
+// 2^p as fp32 / fp64 (p inside the normal range).
+__device__ __forceinline__ float pow2f(int p) { return __uint_as_float((uint32_t)(p + 127) << 23); }
+__device__ __forceinline__ double pow2d(int p) { return __hiloint2double((p + 1023) << 20, 0); }
+
+__device__ __forceinline__ int quant_mantissa(float v, int e, int bits) {
+  const float qmax = (float)((1 << (bits - 1)) - 1);
+  float r = v * pow2f((bits - 2) - e);           // exact: power-of-two scaling
+  r = fminf(fmaxf(r, -qmax), qmax);              // clamp first; +-inf saturate
+  int m = __float2int_rn(r);                     // round half to even
+  return (v != v) ? 0 : m;
+}
+__device__ __forceinline__ int quant_mantissa(double v, int e, int bits) {
+  const double qmax = (double)((1 << (bits - 1)) - 1);
+  double r = v * pow2d((bits - 2) - e);
+  r = fmin(fmax(r, -qmax), qmax);
+  int m = __double2int_rn(r);
+  return (v != v) ? 0 : m;
+}
+// bf16 bit pattern of m * 2^p for |m| <= 127 (exact: at most 7 significant bits).
+__device__ __forceinline__ uint32_t bf16_bits_of(int m, int p) {
+  return __float_as_uint((float)m * pow2f(p)) >> 16;
+}
+
+// ----------------------------------------------------------------------------
+// Device status word (head of the workspace)
+// ----------------------------------------------------------------------------
+struct DeviceStatus {
+  int code;        // lqer_status_t, first error wins
+  int where;       // kernel-specific location id
+  int detail0, detail1;
+};
+__device__ __forceinline__ void report_error(DeviceStatus* st, int code, int where, int d0 = 0, int d1 = 0) {
+  if (st != nullptr && atomicCAS(&st->code, 0, code) == 0) {
+    st->where = where; st->detail0 = d0; st->detail1 = d1;
+  }
+}
+
+// ----------------------------------------------------------------------------
+// Launch wrappers (each returns the cudaError_t of its launches)
+// ----------------------------------------------------------------------------
+void count_launch(int n = 1);
+
+cudaError_t launch_pack(const float* W, const float* A, const float* B, const PackedMeta& m, void* packed,
+                        cudaStream_t s);
+cudaError_t launch_export(const PackedMeta& m, const void* packed, int8_t* Wm, uint8_t* We, int8_t* Am,
+                          uint8_t* Ae, int8_t* Bm, uint8_t* Be, cudaStream_t s);
+cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, int emax, int8_t* Xm,
+                              uint8_t* Xe, cudaStream_t s);
+// X -> Xcat[:, 0:K64] (bf16 of the dequantised MXINT8 value) and T_q -> Xcat[:, K64:K64+k_pad];
+// optional int8 / exponent exports of T_q.
+cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
+                            int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s);
+cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+                             cudaStream_t s);
+cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+                           DeviceStatus* st, cudaStream_t s);
+cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
+                          DeviceStatus* st, cudaStream_t s);
+int decode_max_m();
+
+}  // namespace lqer
