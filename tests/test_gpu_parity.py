@@ -114,3 +114,29 @@ def test_linear_reference_kernel(spec):
     assert worst_ratio(Y, ref) <= 1.0
     assert L.poll_status(ws) == 0
     Pg.release()
+
+
+MID_SPECS = [
+    gen.LayerSpec("mid_odd_tiles", M=300, K=1024, N=640, k=40, calib_rows=128, outlier_frac=0.01, outlier_scale=20.0, seed=31),
+    gen.LayerSpec("mid_k0", M=129, K=512, N=384, k=0, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=32),
+    gen.LayerSpec("mid_rank96", M=257, K=2048, N=512, k=96, calib_rows=128, outlier_frac=0.005, outlier_scale=50.0,
+                  weight_law="student_t4", seed=33),
+]
+
+
+@pytest.mark.parametrize("spec", SMALL_SPECS + MID_SPECS, ids=lambda s: s.name)
+def test_linear_tensor_core_kernel(spec):
+    W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
+    X = gen.make_activations(spec)
+    ref = olqer.forward(X, P)
+    ws = L.new_workspace(spec.M, Pg)
+    L.set_path(binding.PATH_TENSOR)
+    try:
+        Y = L.linear(_t(X), Pg, ws).cpu().numpy()
+        Y2 = L.linear(_t(X), Pg, ws).cpu().numpy()
+    finally:
+        L.set_path(binding.PATH_AUTO)
+    assert L.poll_status(ws) == 0
+    assert worst_ratio(Y, ref) <= 1.0
+    assert np.array_equal(Y, Y2)          # fixed reduction order: bit-identical run to run
+    Pg.release()
