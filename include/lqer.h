@@ -149,8 +149,9 @@ lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void*
 /* Read the device-side status word of `workspace` (synchronises `stream`). */
 lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_t* device_status);
 
-/* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel,
- * 2 decode kernel, 3 tensor-core kernel.  Host only, process wide. */
+/* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 decode kernel,
+ * 3 tensor-core kernel (one CTA per tile), 4 tensor-core kernel (CTA pair per tile).
+ * Host only, process wide. */
 lqer_status_t lqer_set_path(int path);
 
 /* Number of kernels launched by the library in this process so far (host). */

@@ -102,7 +102,7 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
   void* xcat = static_cast<uint8_t*>(workspace) + kStatusBytes;
   int path = g_path.load();
   if (project_only) path = 3;
-  if (path == 0) path = (M <= decode_max_m()) ? 2 : 3;
+  if (path == 0 && M <= decode_max_m()) path = 2;
   cudaError_t err;
   if (path == 2) {
     if (M > decode_max_m()) return LQER_ERR_SHAPE;
@@ -111,7 +111,9 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
     if (path == 1 && M > 65535) return LQER_ERR_SHAPE;
     err = launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
-      err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, Y, s) : launch_gemm_tc(xcat, M, m, packed, Y, dst, s);
+      err = (path == 1)   ? launch_gemm_simt(xcat, M, m, packed, Y, s)
+            : (path == 4 || (path == 0 && M > 128)) ? launch_gemm_tc2(xcat, M, m, packed, Y, dst, s)
+                          : launch_gemm_tc(xcat, M, m, packed, Y, dst, s);
   }
   return err == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
@@ -337,7 +339,7 @@ lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_
 }
 
 lqer_status_t lqer_set_path(int path) {
-  if (path < 0 || path > 3) return LQER_ERR_CONFIG;
+  if (path < 0 || path > 4) return LQER_ERR_CONFIG;
   g_path.store(path);
   return LQER_OK;
 }

@@ -123,6 +123,8 @@ cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const
                              cudaStream_t s);
 cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                            DeviceStatus* st, cudaStream_t s);
+cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+                            DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
                           DeviceStatus* st, cudaStream_t s);
 int decode_max_m();

@@ -1,0 +1,361 @@
+// CTA-pair form of the main GEMM (paper Section 3.1 / 3.2: Y = [X_q | T_q] . [W_q ; B_q]).
+//
+// Two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 output tile.  CTA r holds
+// token rows [128 r, 128 r + 128) of the tile (its own A operand and its own accumulator
+// lanes) and output columns [128 r, 128 r + 128) of the weight tile (its half of the B
+// operand).  Each CTA therefore fetches and converts only HALF of the 4-bit weights per
+// tensor-core stage, and reads half of B from its shared memory; tcgen05.mma.cta_group::2,
+// issued by CTA 0 alone, combines the halves.  Roles per CTA:
+//   warp 0      TMA producer (own activation tile + own packed weight half)
+//   warp 1      tensor memory allocation; in CTA 0 also the MMA issuer
+//   warps 2-5   epilogue (tcgen05.ld of the finished accumulator, fp32 stores to Y)
+//   warps 6-21  converters in four groups; a group converts every fourth stage (one weight
+//               column = 64 weights per thread), so that its fixed per-stage latencies
+//               (barrier wait, shared-memory round trip, proxy fence) overlap the other groups
+// One ring of six stages; a stage holds the activation tile, the packed weight tile and the
+// converted weight tile, so each role waits on one barrier and signals one per stage:
+//   loaded[s]   (per CTA)  TMA bytes have landed          -> converters
+//   ready[s]    (in CTA 0) both CTAs' converters are done -> MMA issuer; implies both
+//                          activation tiles have landed, since a converter waits for loaded[s]
+//   free[s]     (per CTA)  tcgen05.commit with a two-CTA mask: the MMAs that read the stage
+//                          have finished                   -> TMA producer
+// "accumulator full" is the same kind of commit; "accumulator free" lives in CTA 0 and
+// collects the epilogue warps of both CTAs.
+#include <cstdlib>
+
+#include "lqer_tc_ptx.cuh"
+
+namespace lqer {
+namespace tc2 {
+using namespace tc;
+
+constexpr int BM = 128;                    // token rows per CTA (256 per pair)
+constexpr int BN = 256;                    // output columns per pair tile
+constexpr int BNH = 128;                   // columns converted by one CTA
+constexpr int BK = 64;
+constexpr int STAGES = 6;
+constexpr int A_TILE_BYTES = BM * BK * 2;                     // 16384: activations (TMA, swizzled)
+constexpr int B_TILE_BYTES = BNH * BK * 2;                    // 16384: converted weights (swizzled)
+constexpr int PK_OFFSET = A_TILE_BYTES + B_TILE_BYTES;        // packed weight tile (4608) behind them
+constexpr int STAGE_BYTES = 37 * 1024;
+constexpr int RANK_PER_STAGE = 32;
+constexpr int NUM_BARRIERS = 3 * STAGES + 4;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;
+constexpr int CONVERTER_WARPS = 16;
+constexpr int CONVERTER_GROUPS = 4;          // group g converts the stages with index = g (mod 4)
+constexpr int WARPS_PER_GROUP = CONVERTER_WARPS / CONVERTER_GROUPS;
+constexpr int NUM_THREADS = (6 + CONVERTER_WARPS) * 32;
+static_assert(PK_OFFSET + kWTileBytes <= STAGE_BYTES && STAGE_BYTES % 1024 == 0, "stage layout");
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+struct Params {
+  const uint8_t* wsec;
+  const uint8_t* bsec;
+  float* Y;
+  DeviceStatus* status;
+  int M, N, K64;
+  int n_tiles, k_slabs, r_blocks;
+  int m_tiles, n256_tiles;     // pair tiles: 256 rows x 256 columns
+  int lr_shift;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage_base = smem;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARRIERS);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const uint32_t bar0 = smem_u32(bars);
+  auto loaded = [&](int s) { return bar0 + 8u * s; };                        // local
+  auto ready = [&](int s) { return bar0 + 8u * (STAGES + s); };              // used in CTA 0
+  auto freed = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };          // local, pair commit
+  auto acc_full = [&](int a) { return bar0 + 8u * (3 * STAGES + a); };       // local, pair commit
+  auto acc_empty = [&](int a) { return bar0 + 8u * (3 * STAGES + 2 + a); };  // used in CTA 0
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();          // 0 = leader (issues the MMAs)
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(loaded(s), 1);
+      mbar_init(ready(s), 2 * WARPS_PER_GROUP);
+      mbar_init(freed(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 8); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), 512);
+  tc_fence_before();
+  __syncthreads();
+  cluster_barrier();                             // both CTAs' barriers exist before any remote arrive
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int rank_stages = (p.r_blocks + 1) / 2;
+  const int stages_per_tile = p.k_slabs + rank_stages;
+  const int num_tiles = p.m_tiles * p.n256_tiles;
+  const int b_tile_stride = p.r_blocks * kTileN * 17;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (own halves)
+    if (lane == 0) {
+      int st = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int t = pair; t < num_tiles && ok; t += num_pairs) {
+        const int mt = t % p.m_tiles, nt = t / p.m_tiles;
+        const int my_ntile = 2 * nt + (int)rank;
+        const bool has_w = my_ntile < p.n_tiles;
+        const int row0 = mt * 2 * BM + (int)rank * BM;
+        for (int s = 0; s < stages_per_tile; ++s) {
+          if (!mbar_wait<true>(freed(st), ph ^ 1, abort_flag)) { ok = false; break; }
+          const uint32_t a_dst = smem_u32(stage_base + st * STAGE_BYTES);
+          if (s < p.k_slabs) {
+            mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? kWTileBytes : 0));
+            tma_load_2d(a_dst, &tmap_x, s * BK, row0, loaded(st));
+            if (has_w)
+              bulk_load(a_dst + PK_OFFSET, p.wsec + ((size_t)my_ntile * p.k_slabs + s) * kWTileBytes, kWTileBytes,
+                        loaded(st));
+          } else {
+            const int rs = s - p.k_slabs;
+            const int rb0 = rs * 2, nb = min(2, p.r_blocks - rb0);
+            mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? nb * (kTileN * 17) : 0));
+            tma_load_2d(a_dst, &tmap_x, p.K64 + rs * RANK_PER_STAGE, row0, loaded(st));
+            if (has_w) {
+              const uint8_t* tile = p.bsec + (size_t)my_ntile * b_tile_stride;
+              bulk_load(a_dst + PK_OFFSET, tile + (size_t)rb0 * kTileN * 16, nb * kTileN * 16, loaded(st));
+              bulk_load(a_dst + PK_OFFSET + 4096, tile + (size_t)p.r_blocks * kTileN * 16 + rb0 * kTileN,
+                        nb * kTileN, loaded(st));
+            }
+          }
+          if (++st == STAGES) { st = 0; ph ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      int st = 0;
+      uint32_t ph = 0, tile_it = 0;
+      const uint32_t idesc = make_idesc(2 * BM, BN);
+      const uint64_t a_desc0 = make_desc(smem_u32(stage_base));
+      const uint64_t b_desc0 = make_desc(smem_u32(stage_base + A_TILE_BYTES));
+      bool ok = true;
+      for (int t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
+        const int acc = tile_it & 1;
+        if (!mbar_wait(acc_empty(acc), ((tile_it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int s = 0; s < stages_per_tile; ++s) {
+          // everything that does not depend on the wait is computed before it
+          const uint64_t a_desc = a_desc0 + (uint64_t)(st * (STAGE_BYTES >> 4));
+          const uint64_t b_desc = b_desc0 + (uint64_t)(st * (STAGE_BYTES >> 4));
+          const uint32_t first = s > 0 ? 1u : 0u;
+          const uint32_t free_bar = freed(st);
+          if (!mbar_wait(ready(st), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          if (s < p.k_slabs) {           // 64 K = four MMAs; +2 in the address field = 32 bytes = 16 K
+            umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, first);
+            umma_bf16_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
+            umma_bf16_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
+            umma_bf16_pair(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+          } else {
+            const int nk = min(2, p.r_blocks - (s - p.k_slabs) * 2);
+            for (int j = 0; j < nk; ++j) umma_bf16_pair(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, 1u);
+          }
+          umma_commit_pair(free_bar);
+          if (++st == STAGES) { st = 0; ph ^= 1; }
+        }
+        if (ok) umma_commit_pair(acc_full(acc));
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ epilogue (own 128 rows)
+    const int q = warp & 3;
+    uint32_t tile_it = 0;
+    bool ok = true;
+    for (int t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
+      const int mt = t % p.m_tiles, nt = t / p.m_tiles;
+      const int acc = tile_it & 1;
+      if (!mbar_wait<true>(acc_full(acc), (tile_it >> 1) & 1, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = mt * 2 * BM + (int)rank * BM + q * 32 + lane;
+      const int ncols = min(BN, p.N - nt * BN);
+      float* yrow = p.Y + (size_t)row * p.N + (size_t)nt * BN;
+      for (int c = 0; c < BN; c += 32) {
+        if (c >= ncols) break;
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, r);
+        tmem_ld_wait();
+        if (row < p.M) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (c + 4 * j < ncols)
+              *reinterpret_cast<uint4*>(yrow + c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (rank == 0) mbar_arrive(acc_empty(acc)); else mbar_arrive_remote(acc_empty(acc), 0);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ converters (own weight half)
+    const int c = threadIdx.x - 6 * 32;          // 0..511
+    const int group = c >> 7, nl = c & 127;      // stage group; weight column of the half tile
+    const int sw = nl & 7;
+    uint32_t chunk[8];                           // the row's eight 16-byte chunks after the 128-byte swizzle
+#pragma unroll
+    for (int i = 0; i < 8; ++i) chunk[i] = (uint32_t)(nl * 128 + ((i ^ sw) << 4));
+    const int my_tiles = pair < num_tiles ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
+    const long long total = (long long)my_tiles * stages_per_tile;
+    int tile_i = 0, s = group;                   // s may run past the tile; normalised below
+    bool ok = true;
+    for (long long it = group; it < total && ok; it += CONVERTER_GROUPS, s += CONVERTER_GROUPS) {
+      while (s >= stages_per_tile) { s -= stages_per_tile; ++tile_i; }
+      const int nt = (pair + tile_i * num_pairs) / p.m_tiles;
+      const bool has_w = 2 * nt + (int)rank < p.n_tiles;
+      const int st = (int)(it % STAGES);
+      const uint32_t ph = (uint32_t)((it / STAGES) & 1);
+      if (!mbar_wait(loaded(st), ph, abort_flag)) { ok = false; break; }
+      const uint8_t* pk = stage_base + st * STAGE_BYTES + PK_OFFSET;
+      uint8_t* bt = stage_base + st * STAGE_BYTES + A_TILE_BYTES;
+      if (s < p.k_slabs) {
+        if (has_w) {
+          const uint4 wa = *reinterpret_cast<const uint4*>(pk + nl * 16);
+          const uint4 wb = *reinterpret_cast<const uint4*>(pk + (kTileN + nl) * 16);
+          const uint32_t eb = *reinterpret_cast<const uint32_t*>(pk + kWTileNibbleBytes + nl * 4);
+          uint32_t s2, c2;
+          w_scales(eb & 0xFFu, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[0]) = convert_word(wa.x, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[1]) = convert_word(wa.y, s2, c2);
+          w_scales((eb >> 8) & 0xFFu, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[2]) = convert_word(wa.z, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[3]) = convert_word(wa.w, s2, c2);
+          w_scales((eb >> 16) & 0xFFu, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[4]) = convert_word(wb.x, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[5]) = convert_word(wb.y, s2, c2);
+          w_scales(eb >> 24, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[6]) = convert_word(wb.z, s2, c2);
+          *reinterpret_cast<uint4*>(bt + chunk[7]) = convert_word(wb.w, s2, c2);
+        } else {                                 // columns beyond N: a zero operand half
+#pragma unroll
+          for (int i = 0; i < 8; ++i) *reinterpret_cast<uint4*>(bt + chunk[i]) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      } else {
+        const int nb = min(2, p.r_blocks - (s - p.k_slabs) * 2);
+        for (int rb = 0; rb < nb; ++rb) {
+          uint4 o0 = make_uint4(0u, 0u, 0u, 0u), o1 = o0;
+          if (has_w) {
+            const uint4 w = *reinterpret_cast<const uint4*>(pk + (rb * kTileN + nl) * 16);
+            const float scale = pow2f((int)pk[4096 + rb * kTileN + nl] - 127 - p.lr_shift);
+            o0 = convert_i8x8(w.x, w.y, scale);
+            o1 = convert_i8x8(w.z, w.w, scale);
+          }
+          *reinterpret_cast<uint4*>(bt + chunk[rb * 2]) = o0;
+          *reinterpret_cast<uint4*>(bt + chunk[rb * 2 + 1]) = o1;
+        }
+      }
+      fence_proxy_async_smem();        // generic-proxy writes -> visible to the MMA's async proxy
+      __syncwarp();
+      if (lane == 0) {
+        if (rank == 0) mbar_arrive(ready(st)); else mbar_arrive_remote(ready(st), 0);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (*abort_flag != 0) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 400000) { }
+    if (threadIdx.x == 0) report_error(p.status, LQER_ERR_TIMEOUT, 400, blockIdx.x);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_barrier();                    // the peer may still read this CTA's shared / tensor memory until here
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &f, 12000, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+}  // namespace tc2
+
+cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+                            DeviceStatus* st, cudaStream_t s) {
+  using namespace tc2;
+  EncodeTiledFn enc = encode_fn();
+  if (enc == nullptr) return cudaErrorNotSupported;
+  CUtensorMap tmap;
+  const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
+  const cuuint32_t box[2] = {BK, BM};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xcat), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+
+  static int sm_count = 0;
+  static bool attr_set = false;
+  if (!attr_set) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  Params p;
+  const uint8_t* base = static_cast<const uint8_t*>(packed);
+  p.wsec = base + m.off_w;
+  p.bsec = base + m.off_b;
+  p.Y = Y;
+  p.status = st;
+  p.M = M; p.N = m.N; p.K64 = m.K64;
+  p.n_tiles = m.n_tiles; p.k_slabs = m.k_slabs; p.r_blocks = m.r_blocks;
+  p.m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  p.n256_tiles = (m.n_tiles + 1) / 2;
+  p.lr_shift = m.lr_bits - 2;
+  const int num_tiles = p.m_tiles * p.n256_tiles;
+  const int max_pairs = sm_count / 2;
+  const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  count_launch();
+  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, tmap, p);
+}
+
+}  // namespace lqer

@@ -1,34 +1,48 @@
 // Activation prologue of the prefill path (paper Section 4.1: X_q in MXINT8, blocks [1,16];
-// Section 3.1: the small product X A_k):
+// Section 3.1: the small high-precision product X A_k):
 //   X fp32 -> per 16-block shared exponent + 8-bit mantissas (128-bit loads, 4 lanes per
 //   block, two shuffle steps for the maximum), written as the exactly representable bf16
 //   value m * 2^(e-6) into Xcat[:, 0:K64];
-//   T = X_q A_q by integer dot products per block (dp4a) scaled and summed in fp64, then
-//   re-quantised to MXINT8 along the rank and written into Xcat[:, K64:K64+k_pad].
+//   T = X_q A_q: one int8 tensor-core MMA (m16n8k16, exact int32) per 16-block, each block
+//   result scaled by 2^(e_x + e_a) and summed in fp64 (exact for any realistic exponent
+//   spread, so the re-quantisation below takes the same decisions as an fp64 reference);
+//   T -> MXINT8 along the rank, appended to Xcat[:, K64:K64+k_pad].
+// A CTA owns 16 rows of X and walks K in steps; the global loads of step s+1 are in flight
+// while the MMAs of step s run.
 #include "lqer_common.cuh"
 
 namespace lqer {
 
-constexpr int kRows = 8;        // rows of X per CTA
-constexpr int kChunk = 512;     // K columns per pass
+constexpr int kRows = 16;       // rows of X per CTA = one MMA M tile
 constexpr int kThreads = 256;
-constexpr int kMaxOut = 8;      // T outputs per thread: kRows * k_pad / kThreads <= 8  (k_pad <= 256)
+constexpr int kXqStride = 528;  // bytes per row of the int8 panel (512 + 16: conflict-free fragment loads)
+constexpr int kPanelBytes = 1024 * 17;   // A_q panel: PB blocks x k_pad columns x (16 mantissas + 1 exponent)
 
 // Quantise the four values a lane holds; the 16-block is spread over 4 adjacent lanes.
-__device__ __forceinline__ void quantize_quad(const float4 v, int bits, int emin, int emax, int& e, int (&q)[4]) {
+// Returns the four int8 mantissas packed in one word and the four exact bf16 values
+// m * 2^(e - (bits-2)) packed in two words.
+__device__ __forceinline__ void quantize_quad(const float4 v, int bits, int emin, int emax, int& e, uint32_t& m8,
+                                              uint2& bf) {
   float amax = fmaxf(fmaxf(abs_ignore_nan(v.x), abs_ignore_nan(v.y)), fmaxf(abs_ignore_nan(v.z), abs_ignore_nan(v.w)));
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
   e = block_exponent(amax, emin, emax);
-  q[0] = quant_mantissa(v.x, e, bits);
-  q[1] = quant_mantissa(v.y, e, bits);
-  q[2] = quant_mantissa(v.z, e, bits);
-  q[3] = quant_mantissa(v.w, e, bits);
-}
-
-__device__ __forceinline__ uint32_t pack4_i8(const int (&q)[4]) {
-  return ((uint32_t)q[0] & 0xFFu) | (((uint32_t)q[1] & 0xFFu) << 8) | (((uint32_t)q[2] & 0xFFu) << 16) |
-         (((uint32_t)q[3] & 0xFFu) << 24);
+  const float qmax = (float)((1 << (bits - 1)) - 1);
+  const float inv_step = pow2f((bits - 2) - e), step = pow2f(e - (bits - 2));
+  const float in[4] = {v.x, v.y, v.z, v.w};
+  float r[4];
+  int q[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float t = fminf(fmaxf(in[i] * inv_step, -qmax), qmax);   // exact scaling, clamp (+-inf saturate)
+    t = rintf(t);                                            // round half to even
+    r[i] = (in[i] != in[i]) ? 0.0f : t;                      // NaN -> 0
+    q[i] = (int)r[i];
+    r[i] *= step;                                            // exact: at most 7 significant bits
+  }
+  m8 = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
+  bf.x = __byte_perm(__float_as_uint(r[0]), __float_as_uint(r[1]), 0x7632);
+  bf.y = __byte_perm(__float_as_uint(r[2]), __float_as_uint(r[3]), 0x7632);
 }
 
 // Stand-alone activation quantiser (export for bit-exact comparison).  One lane per float4.
@@ -43,107 +57,214 @@ __global__ void __launch_bounds__(256) quantize_x_kernel(const float* __restrict
     const size_t idx = it * stride + (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool ok = idx < total4;
     const float4 v = ok ? reinterpret_cast<const float4*>(X)[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
-    int e, q[4];
-    quantize_quad(v, bits, emin, emax, e, q);
+    int e;
+    uint32_t m8;
+    uint2 bf;
+    quantize_quad(v, bits, emin, emax, e, m8, bf);
     if (ok) {
-      if (Xm != nullptr) reinterpret_cast<uint32_t*>(Xm)[idx] = pack4_i8(q);
+      if (Xm != nullptr) reinterpret_cast<uint32_t*>(Xm)[idx] = m8;
       if (Xe != nullptr && (idx & 3) == 0) Xe[idx >> 2] = (uint8_t)(e + 127);
     }
   }
 }
 
-__global__ void __launch_bounds__(kThreads) prologue_kernel(const float* __restrict__ X, int M, PackedMeta m,
-                                                            const uint8_t* __restrict__ asec,
-                                                            uint16_t* __restrict__ xcat,
-                                                            int8_t* __restrict__ Tm, uint8_t* __restrict__ Te) {
-  __shared__ __align__(16) uint32_t s_xq[kRows][kChunk / 4];   // int8 mantissas, 4 per word
-  __shared__ int s_xe[kRows][kChunk / 16];
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-  const int tid = threadIdx.x;
-  const int row0 = blockIdx.x * kRows;
+__device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
+               : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3]) : "r"(a0), "r"(a1), "r"(b0), "r"(0));
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Read a double from the same shared-memory offset in another CTA of the cluster.
+__device__ __forceinline__ double ld_dsmem_f64(const double* local, uint32_t cta) {
+  uint32_t remote;
+  double v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(cta));
+  asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(remote) : "memory");
+  return v;
+}
+
+// PB = 16-blocks of K per step; PB * k_pad <= 1024.  A cluster of CS CTAs shares 16 rows: CTA r
+// takes the K steps s = r, r + CS, ...; the partial T sums meet through distributed shared memory.
+template <int PB>
+__global__ void __launch_bounds__(kThreads, 2) prologue_kernel(const float* __restrict__ X, int M, PackedMeta m,
+                                                               const uint8_t* __restrict__ asec,
+                                                               uint16_t* __restrict__ xcat,
+                                                               int8_t* __restrict__ Tm, uint8_t* __restrict__ Te) {
+  constexpr int SW = PB * 16;                     // columns per step
+  constexpr int F4 = kRows * SW / 4 / kThreads;   // float4 per thread per step (PB / 4)
+  __shared__ __align__(16) uint8_t s_xq[kRows * kXqStride];
+  __shared__ int8_t s_xe[kRows][32];
+  __shared__ __align__(16) uint8_t s_panel[2][kPanelBytes];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, tig = lane & 3;
+  const int CS = (int)cluster_nctarank(), crank = (int)cluster_ctarank();
+  const int row0 = (blockIdx.x / CS) * kRows;
   const size_t ldx = xcat_cols(m);
-  const int n_out = kRows * m.k_pad;
-  const uint8_t* a_exp = asec + (size_t)(m.K / 16) * m.k_pad * 16;
+  const int kblocks = m.K / 16;
+  const int steps = (m.K64 + SW - 1) / SW;
+  const uint8_t* a_exp = asec + (size_t)kblocks * m.k_pad * 16;
+  const int NT = m.k_pad / 8;                     // 8-column rank tiles
+  const int WPN = NT >= 8 ? 1 : 8 / NT;           // warps that share one rank tile (they split the blocks)
+  const bool has_rank = m.k > 0;
+  const bool active = has_rank && (NT >= 8 || warp < NT * WPN);
 
-  double acc[kMaxOut];
+  double acc[4][4];
 #pragma unroll
-  for (int i = 0; i < kMaxOut; ++i) acc[i] = 0.0;
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
 
-  for (int c0 = 0; c0 < m.K64; c0 += kChunk) {
-    // ---- quantise a [kRows x kChunk] panel of X
+  float4 xr[F4];
+  auto load_x = [&](int s) {
 #pragma unroll
-    for (int i = 0; i < kRows * (kChunk / 4) / kThreads; ++i) {
-      const int idx = tid + i * kThreads;
-      const int r = idx / (kChunk / 4);
-      const int c4 = idx % (kChunk / 4);
-      const int col = c0 + c4 * 4;
-      const int row = row0 + r;
-      const bool in = (row < M) && (col < m.K);
-      const float4 v = in ? *reinterpret_cast<const float4*>(X + (size_t)row * m.K + col)
-                          : make_float4(0.f, 0.f, 0.f, 0.f);
-      int e, q[4];
-      quantize_quad(v, m.a_bits, m.exp_min, m.exp_max, e, q);
-      s_xq[r][c4] = pack4_i8(q);
-      if ((c4 & 3) == 0) s_xe[r][c4 >> 2] = e;
-      if (row < M && col < m.K64) {
-        const int p = e - (m.a_bits - 2);
-        uint2 o;
-        o.x = bf16_bits_of(q[0], p) | (bf16_bits_of(q[1], p) << 16);
-        o.y = bf16_bits_of(q[2], p) | (bf16_bits_of(q[3], p) << 16);
-        *reinterpret_cast<uint2*>(xcat + (size_t)row * ldx + col) = o;
-      }
+    for (int i = 0; i < F4; ++i) {
+      const int f = tid + i * kThreads;
+      const int r = f / (SW / 4), c4 = f % (SW / 4);
+      const int col = s * SW + c4 * 4, row = row0 + r;
+      xr[i] = (row < M && col < m.K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * m.K + col))
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    __syncthreads();
-    // ---- T += X_q A_q over this panel: exact integer dot per 16-block, fp64 scaling and sum
-    if (m.k > 0) {
-      const int kb_end = min(kChunk / 16, (m.K - c0) / 16);
+  };
+  auto load_panel = [&](int s, int buf) {
+    const int kb0 = s * PB;
+    const int nblk = min(PB, kblocks - kb0);
+    if (nblk > 0) {
+      const int mant16 = nblk * m.k_pad;          // 16-byte units of mantissas
+      const int exp16 = nblk * m.k_pad / 16;      // 16-byte units of exponents
+      const uint8_t* gm = asec + (size_t)kb0 * m.k_pad * 16;
+      const uint8_t* ge = a_exp + (size_t)kb0 * m.k_pad;
+      for (int u = tid; u < mant16; u += kThreads) cp_async16(&s_panel[buf][u * 16], gm + (size_t)u * 16);
+      for (int u = tid; u < exp16; u += kThreads) cp_async16(&s_panel[buf][PB * m.k_pad * 16 + u * 16], ge + (size_t)u * 16);
+    }
+  };
+
+  if (crank < steps) {
+    load_x(crank);
+    if (has_rank) load_panel(crank, 0);
+  }
+  cp_async_commit();
+
+  int buf = 0;
+  for (int s = crank; s < steps; s += CS, buf ^= 1) {
+    // ---- quantise the panel held in registers: Xcat (bf16) to global, int8 + exponents to shared
 #pragma unroll
-      for (int i = 0; i < kMaxOut; ++i) {
-        const int o = tid + i * kThreads;
-        if (o < n_out) {
-          const int r = o / m.k_pad, j = o % m.k_pad;
-          double a = acc[i];
-          for (int kb = 0; kb < kb_end; ++kb) {
-            const int kbg = c0 / 16 + kb;
-            const uint4 xa = *reinterpret_cast<const uint4*>(&s_xq[r][kb * 4]);
-            const uint4 aa = __ldg(reinterpret_cast<const uint4*>(asec + ((size_t)kbg * m.k_pad + j) * 16));
-            int d = __dp4a((int)xa.x, (int)aa.x, 0);
-            d = __dp4a((int)xa.y, (int)aa.y, d);
-            d = __dp4a((int)xa.z, (int)aa.z, d);
-            d = __dp4a((int)xa.w, (int)aa.w, d);
-            const int ea = (int)__ldg(a_exp + (size_t)kbg * m.k_pad + j) - 127;
-            a = fma((double)d, pow2d(s_xe[r][kb] + ea - (m.a_bits - 2) - (m.lr_bits - 2)), a);
+    for (int i = 0; i < F4; ++i) {
+      const int f = tid + i * kThreads;
+      const int r = f / (SW / 4), c4 = f % (SW / 4);
+      const int col = s * SW + c4 * 4, row = row0 + r;
+      int e;
+      uint32_t m8;
+      uint2 bf;
+      quantize_quad(xr[i], m.a_bits, m.exp_min, m.exp_max, e, m8, bf);
+      *reinterpret_cast<uint32_t*>(&s_xq[r * kXqStride + c4 * 4]) = m8;
+      if ((c4 & 3) == 0) s_xe[r][c4 >> 2] = (int8_t)e;
+      if (row < M && col < m.K64) *reinterpret_cast<uint2*>(xcat + (size_t)row * ldx + col) = bf;
+    }
+    // ---- next step's loads fly while this step's MMAs run
+    if (s + CS < steps) {
+      load_x(s + CS);
+      if (has_rank) load_panel(s + CS, buf ^ 1);
+    }
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+
+    if (active) {
+      const uint8_t* panel = s_panel[buf];
+      const uint8_t* pexp = panel + PB * m.k_pad * 16;
+      const int nblk = min(PB, kblocks - s * PB);
+      const int b_first = NT >= 8 ? 0 : warp / NT;
+      const int b_step = NT >= 8 ? 1 : WPN;
+      const int nt0 = NT >= 8 ? warp : warp % NT;
+      const int bias = -127 - (m.a_bits - 2) - (m.lr_bits - 2);   // exponent bytes carry +127
+      for (int b = b_first; b < nblk; b += b_step) {
+        const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s_xq[g * kXqStride + b * 16 + tig * 4]);
+        const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s_xq[(g + 8) * kXqStride + b * 16 + tig * 4]);
+        const int ex0 = s_xe[g][b] + bias, ex1 = s_xe[g + 8][b] + bias;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int nt = nt0 + 8 * i;
+          if (nt < NT) {
+            const int j = nt * 8 + g;
+            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(panel + ((size_t)(b * m.k_pad + j) * 16) + tig * 4);
+            const uint32_t ea2 = *reinterpret_cast<const uint16_t*>(pexp + b * m.k_pad + nt * 8 + tig * 2);
+            int c[4];
+            mma_s8(c, a0, a1, b0);
+            const int ea_lo = (int)(ea2 & 0xFFu), ea_hi = (int)(ea2 >> 8);
+            acc[i][0] = fma((double)c[0], pow2d(ex0 + ea_lo), acc[i][0]);
+            acc[i][1] = fma((double)c[1], pow2d(ex0 + ea_hi), acc[i][1]);
+            acc[i][2] = fma((double)c[2], pow2d(ex1 + ea_lo), acc[i][2]);
+            acc[i][3] = fma((double)c[3], pow2d(ex1 + ea_hi), acc[i][3]);
           }
-          acc[i] = a;
         }
       }
     }
     __syncthreads();
   }
 
-  // ---- re-quantise T along the rank (16 adjacent lanes hold one block) and append to Xcat
-  if (m.k > 0) {
+  if (!has_rank) return;       // uniform over the cluster: nobody reaches the cluster barriers below
+  // ---- partial sums of this CTA's warps -> shared memory
+  cp_async_wait<0>();
+  double* tpart = reinterpret_cast<double*>(&s_panel[0][0]);      // [WPN][16][k_pad]
+  const int n_out = kRows * m.k_pad;
+  if (active) {
+    const int slot = NT >= 8 ? 0 : warp / NT;
+    const int nt0 = NT >= 8 ? warp : warp % NT;
 #pragma unroll
-    for (int i = 0; i < kMaxOut; ++i) {
-      const int o = tid + i * kThreads;
-      if (i * kThreads < n_out) {          // uniform over the warp: n_out is a multiple of 128
-        const bool ok = o < n_out;
-        const double t = ok ? acc[i] : 0.0;
-        double amax = (t != t) ? 0.0 : fabs(t);
-#pragma unroll
-        for (int s = 1; s < 16; s <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, s));
-        const int e = block_exponent(amax, m.exp_min, m.exp_max);
-        const int q = quant_mantissa(t, e, m.a_bits);
-        const int r = o / m.k_pad, j = o % m.k_pad;
-        const int row = row0 + r;
-        if (ok && row < M) {
-          xcat[(size_t)row * ldx + m.K64 + j] = (uint16_t)bf16_bits_of(q, e - (m.a_bits - 2));
-          if (Tm != nullptr) Tm[(size_t)row * m.k_pad + j] = (int8_t)q;
-          if (Te != nullptr && (j & 15) == 0) Te[(size_t)row * (m.k_pad / 16) + (j >> 4)] = (uint8_t)(e + 127);
-        }
+    for (int i = 0; i < 4; ++i) {
+      const int nt = nt0 + 8 * i;
+      if (nt < NT) {
+        double* base = tpart + (size_t)slot * n_out;
+        base[g * m.k_pad + nt * 8 + tig * 2] = acc[i][0];
+        base[g * m.k_pad + nt * 8 + tig * 2 + 1] = acc[i][1];
+        base[(g + 8) * m.k_pad + nt * 8 + tig * 2] = acc[i][2];
+        base[(g + 8) * m.k_pad + nt * 8 + tig * 2 + 1] = acc[i][3];
       }
     }
   }
+  cluster_sync();
+  // ---- CTA r finishes rows [r * 16/CS, (r+1) * 16/CS): sum over CTAs and warps in a fixed order,
+  //      re-quantise along the rank (16 adjacent lanes hold one block), append to Xcat
+  const int rows_per = kRows / CS;
+  const int n_mine = rows_per * m.k_pad;           // multiple of 32
+  for (int o = tid; o < n_mine; o += kThreads) {
+    const int r = crank * rows_per + o / m.k_pad, j = o % m.k_pad;
+    double t = 0.0;
+    for (int c = 0; c < CS; ++c)
+      for (int w = 0; w < WPN; ++w) t += ld_dsmem_f64(tpart + (size_t)w * n_out + r * m.k_pad + j, (uint32_t)c);
+    double amax = (t != t) ? 0.0 : fabs(t);
+#pragma unroll
+    for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+    const int e = block_exponent(amax, m.exp_min, m.exp_max);
+    const int q = quant_mantissa(t, e, m.a_bits);
+    const int row = row0 + r;
+    if (row < M) {
+      xcat[(size_t)row * ldx + m.K64 + j] = (uint16_t)bf16_bits_of(q, e - (m.a_bits - 2));
+      if (Tm != nullptr) Tm[(size_t)row * m.k_pad + j] = (int8_t)q;
+      if (Te != nullptr && (j & 15) == 0) Te[(size_t)row * (m.k_pad / 16) + (j >> 4)] = (uint8_t)(e + 127);
+    }
+  }
+  cluster_sync();              // no CTA leaves while its shared memory may still be read
 }
 
 cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, int emax, int8_t* Xm,
@@ -157,13 +278,35 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
   return cudaGetLastError();
 }
 
+template <int PB>
+static cudaError_t launch_prologue_pb(const float* X, int M, const PackedMeta& m, const uint8_t* asec, uint16_t* xc,
+                                      int8_t* Tm, uint8_t* Te, cudaStream_t s) {
+  const int groups = (M + kRows - 1) / kRows;
+  const int steps = (m.K64 + PB * 16 - 1) / (PB * 16);
+  int cs = 1;
+  while (cs < 8 && groups * cs < 2 * 148 && cs * 2 <= steps) cs *= 2;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(groups * cs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  count_launch();
+  return cudaLaunchKernelEx(&cfg, prologue_kernel<PB>, X, M, m, asec, xc, Tm, Te);
+}
+
 cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s) {
   (void)st;
   const uint8_t* asec = static_cast<const uint8_t*>(packed) + m.off_a;
-  prologue_kernel<<<(M + kRows - 1) / kRows, kThreads, 0, s>>>(X, M, m, asec, static_cast<uint16_t*>(xcat), Tm, Te);
-  count_launch();
-  return cudaGetLastError();
+  uint16_t* xc = static_cast<uint16_t*>(xcat);
+  if (m.k_pad <= 64) return launch_prologue_pb<16>(X, M, m, asec, xc, Tm, Te, s);
+  if (m.k_pad <= 128) return launch_prologue_pb<8>(X, M, m, asec, xc, Tm, Te, s);
+  return launch_prologue_pb<4>(X, M, m, asec, xc, Tm, Te, s);
 }
 
 }  // namespace lqer

@@ -124,13 +124,14 @@ MID_SPECS = [
 ]
 
 
+@pytest.mark.parametrize("path", [binding.PATH_TENSOR, binding.PATH_TENSOR_PAIR], ids=["cta1", "cta2"])
 @pytest.mark.parametrize("spec", SMALL_SPECS + MID_SPECS, ids=lambda s: s.name)
-def test_linear_tensor_core_kernel(spec):
+def test_linear_tensor_core_kernel(spec, path):
     W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
     X = gen.make_activations(spec)
     ref = olqer.forward(X, P)
     ws = L.new_workspace(spec.M, Pg)
-    L.set_path(binding.PATH_TENSOR)
+    L.set_path(path)
     try:
         Y = L.linear(_t(X), Pg, ws).cpu().numpy()
         Y2 = L.linear(_t(X), Pg, ws).cpu().numpy()
