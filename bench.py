@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the LQER / L2QER inference linear layer on B200.
+
+One step = one pass of the whole hot path over the LLaMA-7B-shaped decoder linear stack
+(32 layers x {q,k,v,o: 4096x4096; gate,up: 4096x11008; down: 11008x4096}, MXINT4 weights,
+MXINT8 activations, block 16, rank 32): the 224 linears at M=1 (decode) and then at M=2048
+(prefill), back to back on one stream through lqer_linear_batched.  Weights, factors and
+activations are seeded synthetic draws of the paper's shapes and value structure.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--layers L]
+
+Prints ONE JSON line (rank 0).  `value` is the whole-job TFLOP/s of the timed steps
+(algorithmic flops 2 M [(K + k) N + K k] per linear); the decode and prefill legs of the same
+steps are reported separately, as are the end-to-end figure through host buffers, the
+roofline of the dominant kernel and the CPU oracle timed on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import lqer_inputs as gen
+
+METRIC = "fused W4A8+low-rank linear: prefill TOPS & % MMA peak; decode us/layer & HBM GB/s"
+WORKLOAD = ("LLaMA-7B-shaped decoder linear stack: 32 layers x {q,k,v,o 4096x4096; gate,up 4096x11008; "
+            "down 11008x4096}, MXINT4/MXINT8 block 16, rank 32, M=1 then M=2048 back to back on one stream")
+M_DECODE, M_PREFILL = 1, 2048
+
+# DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum
+# from an ncu capture) per shape, valid only for the kernel sources whose hash is given.
+TRAFFIC = {"sources_sha256": None, "bytes_per_launch": None, "note": None}
+DOMINANT_SOURCES = ["paper_2402_02446_b200/csrc/lqer_gemm_tc2.cu", "paper_2402_02446_b200/csrc/lqer_tc_ptx.cuh"]
+
+
+def sources_hash() -> str:
+    h = hashlib.sha256()
+    for rel in DOMINANT_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def layer_flops(M: int, K: int, N: int, k: int) -> float:
+    return 2.0 * M * ((K + k) * N + K * k)
+
+
+def layer_weight_bytes(K: int, N: int, k: int) -> float:
+    """Algorithmic bytes of the stored operands: 4-bit + 1 exponent byte per 16 for W_q,
+    8-bit + 1 exponent byte per 16 for A_k and B_k (rank padded to a multiple of 16)."""
+    k_pad = (k + 15) // 16 * 16
+    return 0.5625 * K * N + 1.0625 * (k * K + k_pad * N)
+
+
+def measured_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 100 ms while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device: int):
+        self.proc = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, pw = [], [], []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def oracle_sample(rows: int):
+    """The bounded sample the oracle is timed on: layer 0's q, gate and down linears, `rows` tokens
+    of the M=2048 batch.  Returns (callable running the sample once, flops of one run, description)."""
+    from oracle import lqer as olqer
+    work = []
+    flops = 0.0
+    for which in (0, 4, 6):
+        spec = gen.config_stack(0, which, M_PREFILL)
+        W = gen.make_weight(spec)
+        A, B = gen.make_random_factors(spec)
+        P = olqer.prepare_weights(W, A, B)
+        X = gen.make_activations(spec, M=rows)
+        work.append((X, P))
+        flops += layer_flops(rows, spec.K, spec.N, spec.k)
+    def run():
+        for X, P in work:
+            olqer.forward(X, P)
+    return run, flops, f"layer 0 q, gate, down linears, {rows} rows of the M={M_PREFILL} batch"
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [int(p.get("num_threads", 1)) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def time_oracle(steps: int, warmup: int, rows: int):
+    run, flops, what = oracle_sample(rows)
+    for _ in range(warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        run()
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    return flops / dt / 1e12, dt * 1e3, what
+
+
+def run_reference(args) -> None:
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    steps, warmup = max(args.steps, 1), max(args.warmup, 0)
+    tflops, ms, what = time_oracle(steps, warmup, rows=args.oracle_rows)
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": what},
+            "cpu_baseline": {"value": tflops, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def run_ours(args) -> None:
+    import paper_2402_02446_b200 as L
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- build the stack (untimed): one packed buffer per linear, its own activations
+    layers = args.layers
+    packed, shapes = [], []
+    for layer in range(layers):
+        for which in range(len(gen.STACK_LINEARS)):
+            spec = gen.config_stack(layer, which, M_PREFILL)
+            W = gen.make_weight_device(spec, dev)
+            A, B = gen.make_random_factors_device(spec, dev)
+            packed.append(L.prepare_weights(W, A, B))
+            shapes.append((spec.K, spec.N, spec.k, spec))
+            del W, A, B
+    torch.cuda.synchronize()
+    n_lin = len(packed)
+    Kmax = max(s[0] for s in shapes)
+    ws_bytes = max(L.workspace_bytes(M_PREFILL, K, N, k) for K, N, k, _ in shapes)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    L.lib().lqer_workspace_init(ws.data_ptr(), ws_bytes, int(torch.cuda.current_stream().cuda_stream))
+
+    X1 = [gen.make_activations_device(s[3], dev, M=M_DECODE) for s in shapes]
+    X2 = [gen.make_activations_device(s[3], dev, M=M_PREFILL) for s in shapes]
+    # outputs: one buffer per linear type and M (write-only; each is larger than a tile's reuse window)
+    Y1 = [torch.empty((M_DECODE, N), dtype=torch.float32, device=dev) for _, N, _, _ in shapes]
+    Y2_by_type = [torch.empty((M_PREFILL, gen.STACK_LINEARS[w][2]), dtype=torch.float32, device=dev)
+                  for w in range(len(gen.STACK_LINEARS))]
+    Y2 = [Y2_by_type[j % len(gen.STACK_LINEARS)] for j in range(n_lin)]
+    decode_calls = L.make_calls(zip(X1, packed, Y1))
+    prefill_calls = L.make_calls(zip(X2, packed, Y2))
+
+    flops_decode = sum(layer_flops(M_DECODE, K, N, k) for K, N, k, _ in shapes)
+    flops_prefill = sum(layer_flops(M_PREFILL, K, N, k) for K, N, k, _ in shapes)
+    bytes_decode = sum(layer_weight_bytes(K, N, k) + 4.0 * M_DECODE * (K + N) for K, N, k, _ in shapes)
+
+    stream = torch.cuda.current_stream()
+
+    def step(mid_event=None):
+        L.linear_batched(decode_calls, ws)
+        if mid_event is not None:
+            mid_event.record(stream)
+        L.linear_batched(prefill_calls, ws)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    if L.poll_status(ws) != 0:
+        raise SystemExit("device-side error during warm-up")
+
+    # ---- timed region: exactly K steps, events on the launching stream
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = L.launch_count()
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_stop = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for e0, e1, e2 in ev:
+        e0.record(stream)
+        step(e1)
+        e2.record(stream)
+    t_stop.record(stream)
+    barrier()
+    launches = L.launch_count() - launches0
+    clocks = sampler.stop() if sampler is not None else None
+    total_ms = t_start.elapsed_time(t_stop)
+    decode_ms = [e0.elapsed_time(e1) for e0, e1, _ in ev]
+    prefill_ms = [e1.elapsed_time(e2) for _, e1, e2 in ev]
+    if dist is not None:
+        t = torch.tensor([total_ms, statistics.median(decode_ms), statistics.median(prefill_ms)], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, dec_ms, pre_ms = (float(v) for v in t.tolist())
+    else:
+        dec_ms, pre_ms = statistics.median(decode_ms), statistics.median(prefill_ms)
+    if L.poll_status(ws) != 0:
+        raise SystemExit("device-side error during the timed region")
+    ms_per_step = total_ms / args.steps
+    value = world * (flops_decode + flops_prefill) / (ms_per_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel: one more step with an event pair around every launch
+    peaks = measured_peaks()
+    L.profile_enable(True)
+    step()
+    torch.cuda.synchronize()
+    fam = L.profile_collect()
+    L.profile_enable(False)
+    fam_total = sum(ms for _, ms in fam.values())
+    dominant = max(fam, key=lambda n: fam[n][1])
+    dom_launches, dom_ms = fam[dominant]
+    roofline = None
+    if dominant.startswith("gemm"):
+        # every M=2048 linear goes through this kernel; algorithmic flops per launch = stack mean
+        flops_per_launch = sum(2.0 * M_PREFILL * (K + k) * N for K, N, k, _ in shapes) / n_lin
+        achieved = flops_per_launch / (dom_ms / dom_launches * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        traffic = TRAFFIC["bytes_per_launch"] if TRAFFIC["sources_sha256"] == sources_hash() else None
+        roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "peak_source": f"bf16 cuBLAS sustained, {peaks['source']}",
+                    "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
+                    "traffic": traffic, "avg_launch_us": dom_ms / dom_launches * 1e3, "launches": dom_launches,
+                    "share_of_kernel_time": dom_ms / fam_total}
+    kernels = {n: {"launches": c, "ms": round(ms, 4), "share": round(ms / fam_total, 4)} for n, (c, ms) in fam.items()}
+
+    # ---- end to end through host buffers (pinned), copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        types = len(gen.STACK_LINEARS)
+        hx1 = [torch.randn((M_DECODE, gen.STACK_LINEARS[w][1])).pin_memory() for w in range(types)]
+        hx2 = [torch.randn((M_PREFILL, gen.STACK_LINEARS[w][1])).pin_memory() for w in range(types)]
+        hy1 = [torch.empty((M_DECODE, gen.STACK_LINEARS[w][2])).pin_memory() for w in range(types)]
+        hy2 = [torch.empty((M_PREFILL, gen.STACK_LINEARS[w][2])).pin_memory() for w in range(types)]
+        extra = 4 * M_PREFILL * (Kmax + max(s[1] for s in shapes)) + 1024
+        ws_h = torch.empty(ws_bytes + extra, dtype=torch.uint8, device=dev)
+        L.lib().lqer_workspace_init(ws_h.data_ptr(), ws_h.numel(), int(stream.cuda_stream))
+
+        def e2e_step():
+            for hx, hy in ((hx1, hy1), (hx2, hy2)):
+                for j in range(n_lin):
+                    L.linear_host(hx[j % types], packed[j], ws_h, hy[j % types])
+
+        e2e_step()
+        barrier()
+        e_steps = max(1, min(args.steps, 2))
+        t0 = time.perf_counter()
+        for _ in range(e_steps):
+            e2e_step()
+        barrier()
+        e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
+        if dist is not None:
+            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d = sum(4 * (M_DECODE + M_PREFILL) * K for K, _, _, _ in shapes)
+        d2h = sum(4 * (M_DECODE + M_PREFILL) * N for _, N, _, _ in shapes)
+        e2e = {"value": world * (flops_decode + flops_prefill) / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+               "ms_per_step": e_ms, "steps": e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "api": "lqer_linear_host per linear, pinned host X and Y"}
+
+    # ---- the oracle on the host cores (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        tflops, ms, what = time_oracle(1, 0, rows=args.oracle_rows)
+        cpu = {"value": tflops, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": what,
+               "seconds": ms / 1e3}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
+            "config": {"workload": WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]",
+                       "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32,
+                       "l2": "inputs larger than L2: every linear has its own packed weights and activations "
+                             f"({sum(p.buf.numel() for p in packed) / 1e9:.2f} GB of weights per step)",
+                       "parallelism": "replicas (independent token batches)" if world > 1 else "1 GPU"},
+            "prefill": {"tflops": world * flops_prefill / (pre_ms * 1e-3) / 1e12, "ms": pre_ms,
+                        "frac_of_measured_bf16_sustained": flops_prefill / (pre_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                        "us_per_linear": pre_ms * 1e3 / n_lin},
+            "decode": {"us_per_linear": dec_ms * 1e3 / n_lin, "us_per_decoder_layer": dec_ms * 1e3 / layers,
+                       "hbm_gbs": bytes_decode / (dec_ms * 1e-3) / 1e9,
+                       "frac_of_measured_hbm": bytes_decode / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": dec_ms},
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": int(launches), "clocks": clocks, "peaks": peaks,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--layers", type=int, default=32, help="decoder layers of the stack (32 = the full workload)")
+    ap.add_argument("--oracle-rows", type=int, default=128, help="token rows of the oracle's bounded sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

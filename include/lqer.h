@@ -157,6 +157,22 @@ lqer_status_t lqer_set_path(int path);
 /* Number of kernels launched by the library in this process so far (host). */
 unsigned long long lqer_launch_count(void);
 
+/* Per-kernel timing for benchmarks.  While enabled (host, process wide), every kernel launch of
+ * the library is bracketed by two CUDA events recorded on the launching stream; the events
+ * serialise nothing but they do keep consecutive kernels from overlapping, so leave it off
+ * when measuring end-to-end time.  lqer_profile_collect waits for the recorded launches,
+ * sums launches and elapsed milliseconds per kernel family into *out (host) and forgets them.
+ * Families: 0 weight pack, 1 export, 2 stand-alone activation quantiser, 3 activation prologue,
+ * 4 CUDA-core reference GEMM, 5 tensor-core GEMM (one CTA per tile), 6 tensor-core GEMM (CTA
+ * pair per tile), 7 decode kernel. */
+#define LQER_NUM_KERNEL_FAMILIES 8
+typedef struct {
+  unsigned long long launches[LQER_NUM_KERNEL_FAMILIES];
+  double milliseconds[LQER_NUM_KERNEL_FAMILIES];
+} lqer_kernel_times_t;
+lqer_status_t lqer_profile_enable(int on);
+lqer_status_t lqer_profile_collect(lqer_kernel_times_t* out);
+
 #ifdef __cplusplus
 }
 #endif

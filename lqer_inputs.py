@@ -146,3 +146,51 @@ def config_stack(layer: int, which: int, M: int) -> LayerSpec:
     name, K, N = STACK_LINEARS[which]
     return LayerSpec(f"stack_L{layer}_{name}_M{M}", M=M, K=K, N=N, k=32, calib_rows=512,
                      outlier_frac=0.01, outlier_scale=20.0, seed=5000 + layer * 7 + which)
+
+
+# ----------------------------------------------------------------------------
+# Device-side draws for full-size throughput runs
+# ----------------------------------------------------------------------------
+# A 224-matrix stack holds 6.5 G weights; drawing them with numpy on the host
+# would take minutes, so throughput runs draw directly on the device with
+# torch's seeded generator.  The law, the shapes and the outlier structure are
+# the ones above; the stream of numbers is a different one (kernel speed does
+# not depend on the values, and parity is always checked on the numpy draws).
+
+def _torch_gen(spec: LayerSpec, stream: int, device):
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(spec.seed * 8 + stream)
+    return g
+
+
+def make_weight_device(spec: LayerSpec, device):
+    import torch
+    g = _torch_gen(spec, 2, device)
+    if spec.weight_law == "normal":
+        return torch.randn((spec.K, spec.N), generator=g, device=device, dtype=torch.float32) * 0.02
+    if spec.weight_law == "student_t4":
+        z = torch.randn((spec.K, spec.N), generator=g, device=device, dtype=torch.float32)
+        c = torch.randn((4, spec.K, spec.N), generator=g, device=device, dtype=torch.float32).square_().sum(0)
+        return z / torch.sqrt(c / 4.0) * (0.02 / 2.0 ** 0.5)
+    raise ValueError(f"unknown weight law {spec.weight_law!r}")
+
+
+def make_activations_device(spec: LayerSpec, device, M: int | None = None):
+    import torch
+    g = _torch_gen(spec, 3, device)
+    x = torch.randn((spec.M if M is None else M, spec.K), generator=g, device=device, dtype=torch.float32)
+    ch = outlier_channels(spec)
+    if ch.size:
+        x[:, torch.from_numpy(ch).to(device)] *= spec.outlier_scale
+    return x
+
+
+def make_random_factors_device(spec: LayerSpec, device):
+    """Device-side twin of make_random_factors (same magnitudes)."""
+    import torch
+    g = _torch_gen(spec, 5, device)
+    a = torch.randn((spec.K, spec.k), generator=g, device=device, dtype=torch.float32) * (1.0 / spec.K ** 0.5)
+    sig = 0.004 * (spec.K ** 0.5 + spec.N ** 0.5)
+    b = torch.randn((spec.k, spec.N), generator=g, device=device, dtype=torch.float32) * (sig / spec.N ** 0.5)
+    return a, b

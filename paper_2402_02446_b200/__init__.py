@@ -24,4 +24,7 @@ from .binding import (  # noqa: F401
     poll_status,
     set_path,
     launch_count,
+    profile_enable,
+    profile_collect,
+    make_calls,
 )

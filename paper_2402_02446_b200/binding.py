@@ -34,6 +34,13 @@ class Config(C.Structure):
                 ("exp_min", C.c_int), ("exp_max", C.c_int), ("deterministic", C.c_int)]
 
 
+KERNEL_FAMILIES = ["pack", "export", "quantize", "prologue", "gemm_simt", "gemm_tc", "gemm_tc_pair", "decode"]
+
+
+class KernelTimes(C.Structure):
+    _fields_ = [("launches", C.c_ulonglong * len(KERNEL_FAMILIES)), ("milliseconds", C.c_double * len(KERNEL_FAMILIES))]
+
+
 class Call(C.Structure):
     _fields_ = [("X", C.c_void_p), ("M", C.c_int), ("packed", C.c_void_p), ("Y", C.c_void_p)]
 
@@ -72,6 +79,8 @@ def lib() -> C.CDLL:
             "lqer_poll_status": (i, [vp, vp, C.POINTER(i)]),
             "lqer_set_path": (i, [i]),
             "lqer_launch_count": (C.c_ulonglong, []),
+            "lqer_profile_enable": (i, [i]),
+            "lqer_profile_collect": (i, [C.POINTER(KernelTimes)]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -235,3 +244,15 @@ def set_path(path: int) -> None:
 
 def launch_count() -> int:
     return int(lib().lqer_launch_count())
+
+
+def profile_enable(on: bool) -> None:
+    _check(lib().lqer_profile_enable(1 if on else 0), "lqer_profile_enable")
+
+
+def profile_collect() -> dict:
+    """{family: (launches, milliseconds)} of the launches recorded since the last collect."""
+    out = KernelTimes()
+    _check(lib().lqer_profile_collect(C.byref(out)), "lqer_profile_collect")
+    return {name: (int(out.launches[j]), float(out.milliseconds[j])) for j, name in enumerate(KERNEL_FAMILIES)
+            if out.launches[j]}

@@ -3,13 +3,41 @@
 #include <cstring>
 #include <mutex>
 #include <unordered_map>
+#include <vector>
 
 #include "lqer_common.cuh"
 
 namespace lqer {
 
 static std::atomic<unsigned long long> g_launches{0};
-void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+// Optional per-family kernel timing: pairs of events recorded around each launch while enabled.
+struct TimedLaunch { int family; int n_kernels; cudaEvent_t start, stop; };
+static std::mutex g_prof_mu;
+static std::atomic<int> g_prof_on{0};
+static std::vector<TimedLaunch> g_prof_records;
+static std::vector<cudaEvent_t> g_prof_free;
+
+static cudaEvent_t prof_event() {
+  if (!g_prof_free.empty()) { cudaEvent_t e = g_prof_free.back(); g_prof_free.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+  return e;
+}
+
+LaunchScope::LaunchScope(int family, cudaStream_t s, int n_kernels) : stream_(s), stop_(nullptr) {
+  g_launches.fetch_add((unsigned long long)n_kernels, std::memory_order_relaxed);
+  if (g_prof_on.load(std::memory_order_relaxed) == 0) return;
+  std::lock_guard<std::mutex> lock(g_prof_mu);
+  TimedLaunch r{family, n_kernels, prof_event(), prof_event()};
+  if (r.start == nullptr || r.stop == nullptr) return;
+  cudaEventRecord(r.start, s);
+  stop_ = r.stop;
+  g_prof_records.push_back(r);
+}
+LaunchScope::~LaunchScope() {
+  if (stop_ != nullptr) cudaEventRecord(stop_, stream_);
+}
 
 static std::mutex g_mu;
 static std::unordered_map<const void*, PackedMeta> g_registry;
@@ -345,5 +373,31 @@ lqer_status_t lqer_set_path(int path) {
 }
 
 unsigned long long lqer_launch_count(void) { return g_launches.load(); }
+
+lqer_status_t lqer_profile_enable(int on) {
+  if (on != 0 && on != 1) return LQER_ERR_CONFIG;
+  g_prof_on.store(on);
+  return LQER_OK;
+}
+
+lqer_status_t lqer_profile_collect(lqer_kernel_times_t* out) {
+  if (out == nullptr) return LQER_ERR_NULL;
+  std::memset(out, 0, sizeof(*out));
+  std::lock_guard<std::mutex> lock(g_prof_mu);
+  lqer_status_t st = LQER_OK;
+  for (const TimedLaunch& r : g_prof_records) {
+    float ms = 0.0f;
+    if (cudaEventSynchronize(r.stop) != cudaSuccess || cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) {
+      st = LQER_ERR_CUDA;
+    } else if (r.family >= 0 && r.family < LQER_NUM_KERNEL_FAMILIES) {
+      out->launches[r.family] += (unsigned long long)r.n_kernels;
+      out->milliseconds[r.family] += (double)ms;
+    }
+    g_prof_free.push_back(r.start);
+    g_prof_free.push_back(r.stop);
+  }
+  g_prof_records.clear();
+  return st;
+}
 
 }  // extern "C"

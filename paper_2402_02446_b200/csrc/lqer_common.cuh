@@ -107,7 +107,23 @@ __device__ __forceinline__ void report_error(DeviceStatus* st, int code, int whe
 // ----------------------------------------------------------------------------
 // Launch wrappers (each returns the cudaError_t of its launches)
 // ----------------------------------------------------------------------------
-void count_launch(int n = 1);
+// Kernel families, as reported by lqer_profile_collect.
+enum KernelFamily {
+  kFamPack = 0, kFamExport, kFamQuantize, kFamPrologue, kFamGemmSimt, kFamGemmTc, kFamGemmTcPair, kFamDecode,
+  kNumFamilies
+};
+// Brackets the launches of one kernel family: counts them and, while profiling is enabled,
+// records a CUDA event on the stream before and after.
+class LaunchScope {
+ public:
+  LaunchScope(int family, cudaStream_t s, int n_kernels = 1);
+  ~LaunchScope();
+  LaunchScope(const LaunchScope&) = delete;
+  LaunchScope& operator=(const LaunchScope&) = delete;
+ private:
+  cudaStream_t stream_;
+  cudaEvent_t stop_;
+};
 
 cudaError_t launch_pack(const float* W, const float* A, const float* B, const PackedMeta& m, void* packed,
                         cudaStream_t s);

@@ -18,8 +18,6 @@
 //   warps 2-5   epilogue: tcgen05.ld of a finished accumulator, fp32 stores to Y, while the
 //               other accumulator (TMEM is double buffered: 2 x 256 columns) is being filled
 // The rank tiles of B_q are appended as the last K stages of the same loop.
-#include <cstdlib>
-
 #include "lqer_tc_ptx.cuh"
 
 namespace lqer {
@@ -39,8 +37,6 @@ constexpr int CONVERTER_WARPS = 8;
 static_assert(RAW_STAGE_BYTES % 1024 == 0 && B_STAGE_BYTES % 1024 == 0, "swizzle atoms need 1024-byte bases");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
-#define TRACE(slot, idx) do { if (p.trace != nullptr && blockIdx.x == 0 && (idx) < 512) p.trace[(slot) * 512 + (idx)] = clock64(); } while (0)
-
 struct Params {
   const uint8_t* wsec;
   const uint8_t* bsec;
@@ -52,8 +48,6 @@ struct Params {
   int r_blocks;       // 16-row rank blocks of B
   int m_tiles, n256_tiles;
   int lr_shift;       // lr_bits - 2
-  int dbg;
-  long long* trace;   // debug timeline (nullptr in normal use)
 };
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -106,13 +100,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
         for (int s = 0; s < stages_per_tile; ++s, ++it) {
           const int st = it % RAW_STAGES;
           if (!mbar_wait(raw_empty(st), ((it / RAW_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-          TRACE(0, it);
           uint8_t* stage = raw_base + st * RAW_STAGE_BYTES;
           const uint32_t a_dst = smem_u32(stage);
           if (s < p.k_slabs) {
-            mbar_expect_tx(raw_full(st), ((p.dbg & 8) ? 0 : A_TILE_BYTES) + ((p.dbg & 16) ? 0 : halves * PK_HALF_BYTES));
-            if (!(p.dbg & 8)) tma_load_2d(a_dst, &tmap_x, s * BK, mt * BM, raw_full(st));
-            if (!(p.dbg & 16)) for (int h = 0; h < halves; ++h)
+            mbar_expect_tx(raw_full(st), A_TILE_BYTES + halves * PK_HALF_BYTES);
+            tma_load_2d(a_dst, &tmap_x, s * BK, mt * BM, raw_full(st));
+            for (int h = 0; h < halves; ++h)
               bulk_load(a_dst + A_TILE_BYTES + h * PK_HALF_BYTES,
                         p.wsec + ((size_t)(2 * nt + h) * p.k_slabs + s) * kWTileBytes, kWTileBytes, raw_full(st));
           } else {
@@ -146,18 +139,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
         for (int s = 0; s < stages_per_tile; ++s, ++it) {
           const int st = it % RAW_STAGES, bst = it % B_STAGES;
           if (!mbar_wait(raw_full(st), (it / RAW_STAGES) & 1, abort_flag)) { ok = false; break; }
-          TRACE(1, it);
           if (!mbar_wait(b_full(bst), (it / B_STAGES) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          TRACE(2, it);
           const uint64_t a_desc = make_desc(smem_u32(raw_base + st * RAW_STAGE_BYTES));
           const uint64_t b_desc = make_desc(smem_u32(b_base + bst * B_STAGE_BYTES));
           const int nk = (s < p.k_slabs) ? BK / 16 : min(2, p.r_blocks - (s - p.k_slabs) * 2);
-          if (!(p.dbg & 2)) for (int j = 0; j < nk; ++j)     // 16 K = 32 bytes along the swizzled row: +2 in the address field
+          for (int j = 0; j < nk; ++j)     // 16 K = 32 bytes along the swizzled row: +2 in the address field
             umma_bf16(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (s > 0 || j > 0) ? 1u : 0u);
           umma_commit(raw_empty(st));
           umma_commit(b_empty(bst));
-          TRACE(3, it);
         }
         if (ok) umma_commit(acc_full(acc));
       }
@@ -180,7 +170,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, r);
         tmem_ld_wait();
-        if (row < p.M && !(p.dbg & 4)) {
+        if (row < p.M) {
 #pragma unroll
           for (int j = 0; j < 8; ++j)
             if (c + 4 * j < ncols)
@@ -202,7 +192,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
     for (int i = 0; i < 8; ++i) chunk[i] = (uint32_t)(c * 128 + ((i ^ sw) << 4));
     const uint32_t pk_off = A_TILE_BYTES + half * PK_HALF_BYTES;
     int st = 0, bst = 0;
-    uint32_t cit = 0;
     uint32_t ph = 0, bph = 0;            // phase parities of the two rings
     bool ok = true;
     for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
@@ -210,12 +199,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
       const bool mine = half < min(2, p.n_tiles - 2 * nt);
       for (int s = 0; s < stages_per_tile; ++s) {
         if (!mbar_wait(raw_full(st), ph, abort_flag)) { ok = false; break; }
-        if (c == 0) TRACE(4, cit);
         if (!mbar_wait(b_empty(bst), bph ^ 1, abort_flag)) { ok = false; break; }
-        if (c == 0) TRACE(5, cit);
         const uint8_t* pk = raw_base + st * RAW_STAGE_BYTES + pk_off;
         uint8_t* bt = b_base + bst * B_STAGE_BYTES;
-        if (mine && !(p.dbg & 1)) {
+        if (mine) {
           if (s < p.k_slabs) {
             const uint4 wa = *reinterpret_cast<const uint4*>(pk + nl * 16);
             const uint4 wb = *reinterpret_cast<const uint4*>(pk + (kTileN + nl) * 16);
@@ -245,9 +232,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
         }
         fence_proxy_async_smem();        // generic-proxy writes -> visible to the MMA's async proxy
         __syncwarp();
-        if (c == 0) TRACE(6, cit);
         if (lane == 0) { mbar_arrive(b_full(bst)); mbar_arrive(raw_empty(st)); }
-        ++cit;
         if (++st == RAW_STAGES) { st = 0; ph ^= 1; }
         if (++bst == B_STAGES) { bst = 0; bph ^= 1; }
       }
@@ -323,12 +308,10 @@ cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const v
   p.m_tiles = (M + BM - 1) / BM;
   p.n256_tiles = (m.n_tiles + 1) / 2;
   p.lr_shift = m.lr_bits - 2;
-  { const char* e = getenv("LQER_TC_DBG"); p.dbg = e ? atoi(e) : 0; }
-  { const char* e = getenv("LQER_TC_TRACE"); p.trace = e ? reinterpret_cast<long long*>(strtoull(e, nullptr, 16)) : nullptr; }
   const int num_tiles = p.m_tiles * p.n256_tiles;
   const int grid = num_tiles < sm_count ? num_tiles : sm_count;
+  LaunchScope scope(kFamGemmTc, s);
   gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmap, p);
-  count_launch();
   return cudaGetLastError();
 }
 

@@ -21,8 +21,6 @@
 //                          have finished                   -> TMA producer
 // "accumulator full" is the same kind of commit; "accumulator free" lives in CTA 0 and
 // collects the epilogue warps of both CTAs.
-#include <cstdlib>
-
 #include "lqer_tc_ptx.cuh"
 
 namespace lqer {
@@ -354,7 +352,7 @@ cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const 
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  count_launch();
+  LaunchScope scope(kFamGemmTcPair, s);
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, tmap, p);
 }
 

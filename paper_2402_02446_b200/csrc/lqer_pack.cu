@@ -127,12 +127,11 @@ __global__ void export_b_kernel(PackedMeta m, const uint8_t* __restrict__ bsec, 
 cudaError_t launch_pack(const float* W, const float* A, const float* B, const PackedMeta& m, void* packed,
                         cudaStream_t s) {
   uint8_t* base = static_cast<uint8_t*>(packed);
+  LaunchScope scope(kFamPack, s, m.k > 0 ? 3 : 1);
   pack_w_kernel<<<dim3(m.n_tiles, m.k_slabs), dim3(kTileN, 4), 0, s>>>(W, m, base + m.off_w);
-  count_launch();
   if (m.k > 0) {
     pack_a_kernel<<<dim3((m.k_pad + 63) / 64, m.K / 16), 64, 0, s>>>(A, m, base + m.off_a);
     pack_b_kernel<<<dim3(m.n_tiles, m.r_blocks), kTileN, 0, s>>>(B, m, base + m.off_b);
-    count_launch(2);
   }
   return cudaGetLastError();
 }
@@ -140,18 +139,14 @@ cudaError_t launch_pack(const float* W, const float* A, const float* B, const Pa
 cudaError_t launch_export(const PackedMeta& m, const void* packed, int8_t* Wm, uint8_t* We, int8_t* Am,
                           uint8_t* Ae, int8_t* Bm, uint8_t* Be, cudaStream_t s) {
   const uint8_t* base = static_cast<const uint8_t*>(packed);
-  if (Wm != nullptr || We != nullptr) {
-    export_w_kernel<<<dim3(m.n_tiles, m.k_slabs), dim3(kTileN, 4), 0, s>>>(m, base + m.off_w, Wm, We);
-    count_launch();
-  }
-  if (m.k > 0 && (Am != nullptr || Ae != nullptr)) {
-    export_a_kernel<<<dim3((m.k + 63) / 64, m.K / 16), 64, 0, s>>>(m, base + m.off_a, Am, Ae);
-    count_launch();
-  }
-  if (m.k > 0 && (Bm != nullptr || Be != nullptr)) {
-    export_b_kernel<<<dim3(m.n_tiles, m.r_blocks), kTileN, 0, s>>>(m, base + m.off_b, Bm, Be);
-    count_launch();
-  }
+  const bool do_w = Wm != nullptr || We != nullptr;
+  const bool do_a = m.k > 0 && (Am != nullptr || Ae != nullptr);
+  const bool do_b = m.k > 0 && (Bm != nullptr || Be != nullptr);
+  if (!do_w && !do_a && !do_b) return cudaSuccess;
+  LaunchScope scope(kFamExport, s, (int)do_w + (int)do_a + (int)do_b);
+  if (do_w) export_w_kernel<<<dim3(m.n_tiles, m.k_slabs), dim3(kTileN, 4), 0, s>>>(m, base + m.off_w, Wm, We);
+  if (do_a) export_a_kernel<<<dim3((m.k + 63) / 64, m.K / 16), 64, 0, s>>>(m, base + m.off_a, Am, Ae);
+  if (do_b) export_b_kernel<<<dim3(m.n_tiles, m.r_blocks), kTileN, 0, s>>>(m, base + m.off_b, Bm, Be);
   return cudaGetLastError();
 }
 

@@ -273,8 +273,8 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
   int blocks = (int)((total4 + 255) / 256);
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
+  LaunchScope scope(kFamQuantize, s);
   quantize_x_kernel<<<blocks, 256, 0, s>>>(X, M, K, bits, emin, emax, Xm, Xe);
-  count_launch();
   return cudaGetLastError();
 }
 
@@ -295,7 +295,7 @@ static cudaError_t launch_prologue_pb(const float* X, int M, const PackedMeta& m
   attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  count_launch();
+  LaunchScope scope(kFamPrologue, s);
   return cudaLaunchKernelEx(&cfg, prologue_kernel<PB>, X, M, m, asec, xc, Tm, Te);
 }
 

@@ -48,9 +48,9 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const uint16_t* __restri
 cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                              cudaStream_t s) {
   const uint8_t* base = static_cast<const uint8_t*>(packed);
+  LaunchScope scope(kFamGemmSimt, s);
   gemm_simt_kernel<<<dim3((m.N + 255) / 256, M), 256, 0, s>>>(static_cast<const uint16_t*>(xcat), M, m,
                                                               base + m.off_w, base + m.off_b, Y);
-  count_launch();
   return cudaGetLastError();
 }
 
