@@ -46,7 +46,8 @@ typedef enum {
   LQER_ERR_ARCH = 7,             /* current device is not compute capability 10.x */
   LQER_ERR_CUDA = 8,             /* a CUDA runtime / driver call failed */
   LQER_ERR_TIMEOUT = 9,          /* device side: a bounded wait ran out */
-  LQER_ERR_BOUNDS = 10           /* device side: an index check failed */
+  LQER_ERR_BOUNDS = 10,          /* device side: an index check failed */
+  LQER_ERR_STATIC_SCRATCH = 11   /* lqer_linear_static: the call needs more than LQER_STATIC_SCRATCH_BYTES */
 } lqer_status_t;
 
 /* Format parameters (Section 3.1: b_l, b_h; Section 4.1: block size, exponent width). */
@@ -129,6 +130,29 @@ lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y,
                           void* workspace, size_t workspace_bytes);
 lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, float* Y,
                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* The same layer for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a property of the library, not of the method).  It is meant for code that runs
+ * inside another component's memory plan - a plugin of a runtime that owns the whole device
+ * and exposes no allocator, a path on which cudaMalloc's device-wide synchronisation is not
+ * acceptable, a process whose memory budget was fixed before this library was loaded.  The
+ * scratch that lqer_linear_stream takes from the caller lives here in a fixed array of
+ * LQER_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds
+ * that much memory until the process exits.  The call itself allocates and frees nothing.
+ *  - X, Y, packed, stream: as for lqer_linear_stream (device pointers, caller owned).
+ *  - Limit: lqer_workspace_bytes(M, K, N, k) <= LQER_STATIC_SCRATCH_BYTES, otherwise
+ *    LQER_ERR_STATIC_SCRATCH is returned and nothing is launched (M = 256 at K = 4096 needs
+ *    about 2.1 MB; M = 16 fits for every supported K).
+ *  - The first call on a device looks up the array's device address (the device must be
+ *    current); make that first call before any stream capture begins.
+ *  - All calls on a device share the one array and it keeps the previous call's contents; the
+ *    status area at its head is cleared at the start of every call.  Two calls that overlap on
+ *    the GPU (different streams without an ordering between them) race on the array and give
+ *    undefined results: keep calls of this entry point on one stream, or order them.
+ *  - Device-side conditions (a bounded wait that ran out) cannot be polled for this variant;
+ *    use lqer_linear_stream with a workspace where that matters. */
+#define LQER_STATIC_SCRATCH_BYTES (8u << 20)
+lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, float* Y, void* stream);
 
 /* n_calls independent layers back to back on one stream (`calls` is a HOST array).
  * The workspace is reused by consecutive calls (stream order makes that safe) and must

@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     new_workspace,
     linear,
     linear_batched,
+    linear_static,
     linear_host,
     poll_status,
     set_path,

@@ -17,7 +17,7 @@ _lib = None
 
 STATUS_NAMES = ["LQER_OK", "LQER_ERR_NULL", "LQER_ERR_SHAPE", "LQER_ERR_ALIGN", "LQER_ERR_CONFIG",
                 "LQER_ERR_BUFFER_TOO_SMALL", "LQER_ERR_BAD_PACKED", "LQER_ERR_ARCH", "LQER_ERR_CUDA",
-                "LQER_ERR_TIMEOUT", "LQER_ERR_BOUNDS"]
+                "LQER_ERR_TIMEOUT", "LQER_ERR_BOUNDS", "LQER_ERR_STATIC_SCRATCH"]
 
 PATH_AUTO, PATH_SIMT, PATH_DECODE, PATH_TENSOR, PATH_TENSOR_PAIR = 0, 1, 2, 3, 4
 
@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
             "lqer_project_lowrank": (i, [vp, i, vp, vp, vp, vp, sz, vp]),
             "lqer_linear": (i, [vp, i, vp, vp, vp, sz]),
             "lqer_linear_stream": (i, [vp, i, vp, vp, vp, sz, vp]),
+            "lqer_linear_static": (i, [vp, i, vp, vp, vp]),
             "lqer_linear_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
             "lqer_linear_host": (i, [vp, i, vp, vp, vp, sz, vp]),
             "lqer_workspace_init": (i, [vp, sz, vp]),
@@ -206,6 +207,21 @@ def linear(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y: torch.Tensor 
     _check(lib().lqer_linear_stream(_dev(X, torch.float32), M, P.ptr, _dev(Y, torch.float32), ws.data_ptr(),
                                     ws.numel(), _stream(stream)), "lqer_linear_stream")
     return Y
+
+
+def linear_static(X: torch.Tensor, P: PackedWeights, Y: torch.Tensor | None = None, stream=None):
+    """The layer without a caller-provided workspace: the scratch is a fixed array inside the
+    library (STATIC_SCRATCH_BYTES); nothing is allocated by the call (Y must be given for that to
+    hold on the Python side too)."""
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, P.N), dtype=torch.float32, device=X.device)
+    _check(lib().lqer_linear_static(_dev(X, torch.float32), M, P.ptr, _dev(Y, torch.float32), _stream(stream)),
+           "lqer_linear_static")
+    return Y
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 def make_calls(items) -> "C.Array":

@@ -165,6 +165,7 @@ const char* lqer_status_string(lqer_status_t status) {
     case LQER_ERR_CUDA: return "CUDA call failed";
     case LQER_ERR_TIMEOUT: return "device-side wait timed out";
     case LQER_ERR_BOUNDS: return "device-side bounds check failed";
+    case LQER_ERR_STATIC_SCRATCH: return "problem too large for the library's fixed scratch array";
   }
   return "unknown status";
 }
