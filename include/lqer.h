@@ -81,8 +81,11 @@ lqer_status_t lqer_default_config(lqer_config_t* cfg);
  * and tile padding (N to a multiple of 128, K to a multiple of 64, k to a multiple of 16). */
 lqer_status_t lqer_packed_bytes(int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
 
-/* Size in bytes (host out) of the scratch `workspace` lqer_linear* needs for up to M_max rows.
- * The workspace holds a 256-byte status area and the quantised activations [X_q | T_q]. */
+/* Size in bytes (host out) of the scratch `workspace` lqer_linear* needs for any call of up to
+ * M_max rows.  The workspace holds a head that is all zero between calls (status area, the
+ * decode kernel's arrival counters and its fp64 accumulator of X A_k) followed by per-call
+ * scratch: the quantised activations [X_q | T_q] (bf16, M rows) or the decode kernel's
+ * partial sums.  One workspace may serve layers of different shapes if it fits the largest. */
 lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
 
 /* Weight preparation (Section 3.1: W_q = q(W); Section 4.1 formats): quantise W to MXINT4
@@ -162,12 +165,14 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
 
 /* Same layer with host buffers: copies X (host, [M,K]) to the device part of `workspace`,
  * runs the layer and copies Y back to Y_host ([M,N]); synchronises `stream` before it
- * returns.  workspace must be lqer_workspace_bytes + 4*M*(K+N) bytes. */
+ * returns.  workspace must hold lqer_workspace_bytes(M, ...) plus 4*M*K and 4*M*N, each rounded
+ * up to a multiple of 256. */
 lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, float* Y_host,
                                void* workspace, size_t workspace_bytes, void* stream);
 
-/* Clear the status area at the head of a fresh workspace (asynchronous on `stream`).
- * Call once after allocating the workspace and after an error was polled. */
+/* Zero the head of a fresh workspace (status area, counters, accumulator; at most 164096 bytes;
+ * asynchronous on `stream`).  Call once after allocating the workspace and again after
+ * lqer_poll_status reported a device-side error (an interrupted call may leave counters behind). */
 lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Read the device-side status word of `workspace` (synchronises `stream`). */

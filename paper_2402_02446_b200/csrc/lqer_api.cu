@@ -114,6 +114,15 @@ static lqer_status_t check_arch() {
 }
 
 static size_t xcat_bytes(const PackedMeta& m, int M) { return align_up((size_t)M * xcat_cols(m) * 2, 256); }
+// Bytes a call with M rows needs: the persistent head plus the scratch of the path it takes.
+static size_t call_bytes(const PackedMeta& m, int M, bool decode) {
+  return align_up(persist_bytes(m), 256) + (decode ? decode_scratch_bytes(m) : xcat_bytes(m, M));
+}
+// Bytes that fit every call of up to M_max rows, whichever path it takes.
+static size_t workspace_total(const PackedMeta& m, int M_max) {
+  const size_t a = xcat_bytes(m, M_max), b = decode_scratch_bytes(m);
+  return align_up(persist_bytes(m), 256) + (a > b ? a : b);
+}
 
 static lqer_status_t run_linear(const float* X, int M, const void* packed, float* Y, void* workspace,
                                 size_t workspace_bytes, cudaStream_t s, int8_t* Tm, uint8_t* Te, bool project_only) {
@@ -124,17 +133,17 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
   PackedMeta m;
   lqer_status_t st = lookup(packed, m);
   if (st != LQER_OK) return st;
-  if (workspace_bytes < kStatusBytes + xcat_bytes(m, M)) return LQER_ERR_BUFFER_TOO_SMALL;
-  if ((st = check_arch()) != LQER_OK) return st;
-  DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
-  void* xcat = static_cast<uint8_t*>(workspace) + kStatusBytes;
   int path = g_path.load();
   if (project_only) path = 3;
   if (path == 0 && M <= decode_max_m()) path = 2;
+  if (path == 2 && M > decode_max_m()) return LQER_ERR_SHAPE;
+  if (workspace_bytes < call_bytes(m, M, path == 2)) return LQER_ERR_BUFFER_TOO_SMALL;
+  if ((st = check_arch()) != LQER_OK) return st;
+  DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
+  void* xcat = static_cast<uint8_t*>(workspace) + align_up(persist_bytes(m), 256);
   cudaError_t err;
   if (path == 2) {
-    if (M > decode_max_m()) return LQER_ERR_SHAPE;
-    err = launch_decode(X, M, m, packed, Y, dst, s);
+    err = launch_decode(X, M, m, packed, Y, workspace, s);
   } else {
     if (path == 1 && M > 65535) return LQER_ERR_SHAPE;
     err = launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
@@ -195,7 +204,7 @@ lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_co
   if (M_max <= 0 || M_max > (1 << 24)) return LQER_ERR_SHAPE;
   PackedMeta m;
   fill_meta(m, K, N, k, *cfg);
-  *bytes = kStatusBytes + xcat_bytes(m, M_max);
+  *bytes = workspace_total(m, M_max);
   return LQER_OK;
 }
 
@@ -319,7 +328,9 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     PackedMeta m;
     lqer_status_t st = lookup(c.packed, m);
     if (st != LQER_OK) return st;
-    if (workspace_bytes < kStatusBytes + xcat_bytes(m, c.M)) return LQER_ERR_BUFFER_TOO_SMALL;
+    const int path = g_path.load();
+    const bool decode = path == 2 || (path == 0 && c.M <= decode_max_m());
+    if (workspace_bytes < call_bytes(m, c.M, decode)) return LQER_ERR_BUFFER_TOO_SMALL;
   }
   for (int i = 0; i < n_calls; ++i) {
     lqer_status_t st = lqer_linear_stream(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace,
@@ -336,7 +347,7 @@ lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, f
   PackedMeta m;
   lqer_status_t st = lookup(packed, m);
   if (st != LQER_OK) return st;
-  const size_t core = kStatusBytes + xcat_bytes(m, M);
+  const size_t core = workspace_total(m, M);
   const size_t xb = align_up((size_t)M * m.K * 4, 256), yb = align_up((size_t)M * m.N * 4, 256);
   if (workspace_bytes < core + xb + yb) return LQER_ERR_BUFFER_TOO_SMALL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -353,7 +364,8 @@ lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void*
   if (workspace == nullptr) return LQER_ERR_NULL;
   if (workspace_bytes < (size_t)kStatusBytes) return LQER_ERR_BUFFER_TOO_SMALL;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
-  return cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+  const size_t n = workspace_bytes < kPersistMaxBytes ? workspace_bytes : kPersistMaxBytes;
+  return cudaMemsetAsync(workspace, 0, n, static_cast<cudaStream_t>(stream)) == cudaSuccess
              ? LQER_OK : LQER_ERR_CUDA;
 }
 

@@ -50,6 +50,33 @@ inline uint32_t meta_checksum(const PackedMeta& m) {
   return h;
 }
 
+// Workspace layout: a persistent head that is all zero between calls
+//   [0, 256)   status area: DeviceStatus, the decode kernel's two T counters
+//   [256, ..)  per-column-tile arrival counters of the decode kernel, then its fp64 T accumulator
+// followed by per-call scratch: Xcat (bf16 [M, K64 + k_pad]) for the GEMM path, or the partial-sum
+// slots of the decode path.
+constexpr int kTCountOffset = 64, kTDoneOffset = 68;
+constexpr int kDecodeMaxCtas = 160;
+constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8;
+__host__ __device__ inline size_t tacc_offset(const PackedMeta& m) {
+  return (size_t)kStatusBytes + (((size_t)m.n_tiles * 4 + 255) & ~(size_t)255);
+}
+__host__ __device__ inline size_t persist_bytes(const PackedMeta& m) {
+  return tacc_offset(m) + (size_t)16 * m.k_pad * 8;
+}
+__host__ __device__ inline int decode_units(const PackedMeta& m) {
+  return m.n_tiles * (m.k_slabs + (m.r_blocks + 1) / 2);
+}
+inline int decode_ctas(const PackedMeta& m, int sm_count) {
+  int g = decode_units(m);
+  if (g > sm_count) g = sm_count;
+  if (g > kDecodeMaxCtas) g = kDecodeMaxCtas;
+  return g;
+}
+inline size_t decode_scratch_bytes(const PackedMeta& m) {
+  return (size_t)decode_ctas(m, kDecodeMaxCtas) * 2 * 16 * kTileN * 4;
+}
+
 __host__ __device__ inline int b_tile_bytes(const PackedMeta& m) { return m.r_blocks * kTileN * 17; }
 __host__ __device__ inline size_t xcat_cols(const PackedMeta& m) { return (size_t)m.K64 + (size_t)m.k_pad; }
 
@@ -88,6 +115,38 @@ __device__ __forceinline__ int quant_mantissa(double v, int e, int bits) {
 // bf16 bit pattern of m * 2^p for |m| <= 127 (exact: at most 7 significant bits).
 __device__ __forceinline__ uint32_t bf16_bits_of(int m, int p) {
   return __float_as_uint((float)m * pow2f(p)) >> 16;
+}
+
+// Quantise the four values a lane holds; the 16-block is spread over 4 adjacent lanes.
+// Returns the four int8 mantissas packed in one word and the four exact bf16 values
+// m * 2^(e - (bits-2)) packed in two words.
+__device__ __forceinline__ void quantize_quad(const float4 v, int bits, int emin, int emax, int& e, uint32_t& m8,
+                                              uint2& bf) {
+  float amax = fmaxf(fmaxf(abs_ignore_nan(v.x), abs_ignore_nan(v.y)), fmaxf(abs_ignore_nan(v.z), abs_ignore_nan(v.w)));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+  e = block_exponent(amax, emin, emax);
+  const float qmax = (float)((1 << (bits - 1)) - 1);
+  const float inv_step = pow2f((bits - 2) - e), step = pow2f(e - (bits - 2));
+  const float in[4] = {v.x, v.y, v.z, v.w};
+  float r[4];
+  int q[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float t = fminf(fmaxf(in[i] * inv_step, -qmax), qmax);   // exact scaling, clamp (+-inf saturate)
+    t = rintf(t);                                            // round half to even
+    r[i] = (in[i] != in[i]) ? 0.0f : t;                      // NaN -> 0
+    q[i] = (int)r[i];
+    r[i] *= step;                                            // exact: at most 7 significant bits
+  }
+  m8 = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
+  bf.x = __byte_perm(__float_as_uint(r[0]), __float_as_uint(r[1]), 0x7632);
+  bf.y = __byte_perm(__float_as_uint(r[2]), __float_as_uint(r[3]), 0x7632);
+}
+
+__device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
+               : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3]) : "r"(a0), "r"(a1), "r"(b0), "r"(0));
 }
 
 // ----------------------------------------------------------------------------
@@ -142,7 +201,7 @@ cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const v
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
-                          DeviceStatus* st, cudaStream_t s);
+                          void* workspace, cudaStream_t s);
 int decode_max_m();
 
 }  // namespace lqer

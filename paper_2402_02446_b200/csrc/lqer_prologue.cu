@@ -18,33 +18,6 @@ constexpr int kThreads = 256;
 constexpr int kXqStride = 528;  // bytes per row of the int8 panel (512 + 16: conflict-free fragment loads)
 constexpr int kPanelBytes = 1024 * 17;   // A_q panel: PB blocks x k_pad columns x (16 mantissas + 1 exponent)
 
-// Quantise the four values a lane holds; the 16-block is spread over 4 adjacent lanes.
-// Returns the four int8 mantissas packed in one word and the four exact bf16 values
-// m * 2^(e - (bits-2)) packed in two words.
-__device__ __forceinline__ void quantize_quad(const float4 v, int bits, int emin, int emax, int& e, uint32_t& m8,
-                                              uint2& bf) {
-  float amax = fmaxf(fmaxf(abs_ignore_nan(v.x), abs_ignore_nan(v.y)), fmaxf(abs_ignore_nan(v.z), abs_ignore_nan(v.w)));
-  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
-  e = block_exponent(amax, emin, emax);
-  const float qmax = (float)((1 << (bits - 1)) - 1);
-  const float inv_step = pow2f((bits - 2) - e), step = pow2f(e - (bits - 2));
-  const float in[4] = {v.x, v.y, v.z, v.w};
-  float r[4];
-  int q[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float t = fminf(fmaxf(in[i] * inv_step, -qmax), qmax);   // exact scaling, clamp (+-inf saturate)
-    t = rintf(t);                                            // round half to even
-    r[i] = (in[i] != in[i]) ? 0.0f : t;                      // NaN -> 0
-    q[i] = (int)r[i];
-    r[i] *= step;                                            // exact: at most 7 significant bits
-  }
-  m8 = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
-  bf.x = __byte_perm(__float_as_uint(r[0]), __float_as_uint(r[1]), 0x7632);
-  bf.y = __byte_perm(__float_as_uint(r[2]), __float_as_uint(r[3]), 0x7632);
-}
-
 // Stand-alone activation quantiser (export for bit-exact comparison).  One lane per float4.
 __global__ void __launch_bounds__(256) quantize_x_kernel(const float* __restrict__ X, int M, int K, int bits,
                                                          int emin, int emax, int8_t* __restrict__ Xm,
@@ -74,11 +47,6 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
-               : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3]) : "r"(a0), "r"(a1), "r"(b0), "r"(0));
-}
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;

@@ -50,7 +50,8 @@ extern "C" lqer_status_t lqer_linear_static(const float* X, int M, const void* p
   if (need > (size_t)LQER_STATIC_SCRATCH_BYTES) return LQER_ERR_STATIC_SCRATCH;   // M (K + k) too large for the fixed array
   void* scratch = nullptr;
   if ((st = lqer::static_scratch(&scratch)) != LQER_OK) return st;
-  // The array keeps whatever the previous call left: the status area must start at zero.
-  if (cudaMemsetAsync(scratch, 0, lqer::kStatusBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return LQER_ERR_CUDA;
+  // The array keeps whatever the previous call left: the head of the workspace (status area,
+  // arrival counters, accumulator) must start at zero.
+  if ((st = lqer_workspace_init(scratch, need, stream)) != LQER_OK) return st;
   return lqer_linear_stream(X, M, packed, Y, scratch, need, stream);
 }

@@ -141,3 +141,66 @@ def test_linear_tensor_core_kernel(spec, path):
     assert worst_ratio(Y, ref) <= 1.0
     assert np.array_equal(Y, Y2)          # fixed reduction order: bit-identical run to run
     Pg.release()
+
+
+# ---------------------------------------------------------------------------- decode kernel (M <= 16)
+DECODE_SPECS = SMALL_SPECS + MID_SPECS + [
+    gen.LayerSpec("dec_many_tiles", M=16, K=64, N=2048, k=24, calib_rows=32, outlier_frac=0.0, n_outliers=1,
+                  outlier_scale=20.0, seed=41),      # few units per column tile: CTAs span several tiles
+    gen.LayerSpec("dec_interior", M=16, K=64, N=65536, k=8, calib_rows=32, outlier_frac=0.0, n_outliers=1,
+                  outlier_scale=20.0, seed=43),      # CTAs that cover whole column tiles between two partial ones
+    gen.LayerSpec("dec_deep", M=16, K=4096, N=128, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=42),
+]
+
+
+@pytest.mark.parametrize("M", [1, 5, 16])
+@pytest.mark.parametrize("spec", DECODE_SPECS, ids=lambda s: s.name)
+def test_linear_decode_kernel(spec, M):
+    W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
+    X = gen.make_activations(spec, M=M)
+    ref = olqer.forward(X, P)
+    ws = L.new_workspace(M, Pg)
+    L.set_path(binding.PATH_DECODE)
+    try:
+        Y = L.linear(_t(X), Pg, ws).cpu().numpy()
+        Y2 = L.linear(_t(X), Pg, ws).cpu().numpy()      # same workspace again: the kernel left its counters at zero
+    finally:
+        L.set_path(binding.PATH_AUTO)
+    assert L.poll_status(ws) == 0
+    assert worst_ratio(Y, ref) <= 1.0
+    assert np.array_equal(Y, Y2)
+    Pg.release()
+
+
+def test_decode_chain_shares_one_workspace():
+    # layers of different shapes back to back on one stream (each launch may start while the previous drains)
+    specs = [DECODE_SPECS[0], MID_SPECS[0], DECODE_SPECS[3], MID_SPECS[2], DECODE_SPECS[-3]]
+    layers = [_prepare(s, "jacobi" if s.K <= 320 else "subspace") for s in specs]
+    M = 4
+    Xs = [gen.make_activations(s, M=M) for s in specs]
+    refs = [olqer.forward(X, lay[3]) for X, lay in zip(Xs, layers)]
+    n = max(L.workspace_bytes(M, s.K, s.N, s.k) for s in specs)
+    ws = torch.zeros(n, dtype=torch.uint8, device=DEV)
+    Xg = [_t(X) for X in Xs]
+    Yg = [torch.empty((M, s.N), dtype=torch.float32, device=DEV) for s in specs]
+    for _ in range(3):
+        L.linear_batched([(x, lay[4], y) for x, lay, y in zip(Xg, layers, Yg)] * 2, ws)
+    torch.cuda.synchronize()
+    assert L.poll_status(ws) == 0
+    for y, ref, s in zip(Yg, refs, specs):
+        assert worst_ratio(y.cpu().numpy(), ref) <= 1.0, s.name
+    for lay in layers:
+        lay[4].release()
+
+
+@pytest.mark.parametrize("M", [1, 16])
+def test_linear_decode_full_size(M):
+    spec = gen.config_decode(M)
+    W, A, B, P, Pg = _prepare(spec, "subspace")
+    X = gen.make_activations(spec)
+    ref = olqer.forward(X, P)
+    ws = L.new_workspace(M, Pg)
+    Y = L.linear(_t(X), Pg, ws).cpu().numpy()          # automatic path selection: decode for M <= 16
+    assert L.poll_status(ws) == 0
+    assert worst_ratio(Y, ref) <= 1.0
+    Pg.release()
