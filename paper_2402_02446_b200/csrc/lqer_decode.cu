@@ -17,29 +17,31 @@
 // kernel start and adds them to an accumulator in the workspace; the CTAs that own rank units
 // process those last and, before them, wait (bounded) until all G contributions have arrived.
 //
-// Roles in a CTA (16 warps, four per scheduler):
-//   warp 0       producer: bulk copies of weight tiles and of the matching X columns into a ring
-//   warps 1-3    quantisers: X fp32 -> MXINT8 -> exact bf16, one 16 x 64 tile per stage
-//   warps 4-7    T: partial X_q A_q, later T -> T_q (bf16) for the rank units
-//   warps 8-15   consumers: nibbles -> exact bf16 in registers, mma.sync m16n8k16 (tokens are
-//                the M side of the MMA, 16 output columns per warp), fp32 accumulation
-// Weight copies do not depend on earlier kernels of the stream, so they are issued before
-// griddepcontrol.wait: with programmatic dependent launch the next layer's weights are already
-// in flight while the previous layer finishes.
+// A kernel that lives for a few microseconds pays for every instruction-cache line it touches
+// and for every hand-over between warps, so all 16 warps run the same small loop.  Warp w owns
+// output columns [8 w, 8 w + 8) of the current column tile and walks all units of the CTA:
+//   * its share of a unit (8 columns x 64 K = 256 bytes of nibbles + 32 exponent bytes, or
+//     8 columns x 32 rank values) goes global -> shared memory by cp.async into a private ring,
+//     16 units ahead, so the whole share of the CTA is requested at once; these copies depend on
+//     no earlier kernel and are issued before griddepcontrol.wait (programmatic dependent launch);
+//   * X is quantised to MXINT8 once per CTA, cooperatively, into one exact-bf16 tile per unit;
+//   * nibbles -> exact bf16 in registers, mma.sync m16n8k16 with the tokens on the M side,
+//     fp32 accumulation; no partial sums cross warps.
 #include "lqer_tc_ptx.cuh"
 
 namespace lqer {
 namespace dec {
 using namespace tc;
 
-constexpr int kQuantWarps = 3, kTWarps = 4, kConsumerWarps = 8;
-constexpr int kThreads = (1 + kQuantWarps + kTWarps + kConsumerWarps) * 32;   // 512
+constexpr int kWarps = 16;
+constexpr int kThreads = kWarps * 32;
 constexpr int kXTileStride = 144;                    // bytes per row of the bf16 X tile (64 values + pad)
 constexpr int kXTileBytes = 16 * kXTileStride;       // 2304
-constexpr int kMaxStages = 32;
-constexpr int kAChunkBytes = 16 * 1024;              // staging of A_q blocks and their X columns
+constexpr int kPhaseUnits = 40;                      // units whose X tiles are resident at a time
+constexpr int kDepth = 16;                           // units a warp keeps in flight
+constexpr int kSlotBytes = 288;                      // a warp's share of one unit: 256 B mantissas + 32 B exponents
+constexpr int kTabUnits = kPhaseUnits + kDepth;      // window of the unit table
 constexpr int kSlotFloats = 16 * kTileN;             // one partial-sum slot: 16 rows x 128 columns
-constexpr int kSmemBudget = 225 * 1024;
 
 struct Params {
   const float* X;
@@ -56,7 +58,6 @@ struct Params {
   int M, K, N, k_pad;
   int n_tiles, k_slabs, r_blocks, U;   // U = units per column tile = k_slabs + rank units
   int total_units;
-  int stages, stage_bytes, xf_bytes, a_chunk_blocks;
   int a_bits, lr_bits, exp_min, exp_max;
 };
 
@@ -89,20 +90,6 @@ struct Seq {
   }
 };
 
-// Position in the walk: the current unit is slab / rank unit j of column tile nt.  Steps to the
-// next unit by incrementing; divides only where the order jumps.
-struct Walker {
-  int u, nt, j;
-  __device__ void set(const Seq& s, int uu) { u = uu; nt = uu / s.U; j = uu - nt * s.U; }
-  __device__ void start(const Seq& s) { if (s.n > 0) set(s, s.unit(0)); else { u = 0; nt = 0; j = 0; } }
-  __device__ void step(const Seq& s, int i_next) {
-    if (i_next >= s.n) return;
-    const int nu = s.unit(i_next);
-    if (nu == u + 1) { u = nu; if (++j == s.U) { j = 0; ++nt; } }
-    else set(s, nu);
-  }
-};
-
 // First unit of CTA c's range (the product may exceed 32 bits; used a few times per thread only).
 __device__ __forceinline__ int range_lo(int c, int total, int G) { return (int)((long long)c * total / G); }
 // The CTA whose range holds unit u.
@@ -112,7 +99,7 @@ __device__ __forceinline__ int cta_of(int u, int total, int G) {
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -124,417 +111,270 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   return v;
 }
 
-// Wait of a whole warp on an mbarrier phase.  Only lane 0 polls, sleeping between polls, so that
-// waiting warps leave the issue slots and the shared-memory pipe to the warps that have work;
-// afterwards every lane observes the completed phase itself (one poll that succeeds at once).
-// Bounded: gives up after WAIT_LIMIT_CYCLES or as soon as another role has given up.
-template <int kSleepNs>
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0 && !mbar_try_wait(bar, parity)) {
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// What every thread of the CTA needs to know about the CTA's range, computed once.
+struct Ctx {
+  int lo, hi, nt_first;
+  int part_first[2], part_last[2], part_slot0[2];   // contributors of the first / last column tile of the range
+  int tab_nt[kTabUnits], tab_j[kTabUnits];           // (column tile, slab or rank unit) of units [tab0, tab0 + kTabUnits)
+  int flags[4];                                      // [0] a bounded wait ran out, [1], [2] broadcast slots
+};
+
+// Hand the sums of column tile nt over (rare path, kept out of line so that the unit loop stays
+// small): straight to Y when this CTA covered the whole contraction of the tile, otherwise
+// through a slot; the last CTA to arrive adds the slots in CTA order.  Called by all threads.
+__device__ __noinline__ void flush_tile(const Params& p, Ctx* cx, int nt, float s0, float s1, float s2, float s3) {
+  const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int M = p.M, cta = blockIdx.x;
+  const bool complete = nt * p.U >= cx->lo && (nt + 1) * p.U <= cx->hi;
+  const int cl = (tid >> 5) * 8 + t * 2, col = nt * kTileN + cl;
+  if (complete) {
+    if (col < p.N) {
+      if (g < M) *reinterpret_cast<float2*>(p.Y + (size_t)g * p.N + col) = make_float2(s0, s1);
+      if (g + 8 < M) *reinterpret_cast<float2*>(p.Y + (size_t)(g + 8) * p.N + col) = make_float2(s2, s3);
+    }
+    return;
+  }
+  float* slot = p.slots + ((size_t)cta * 2 + (nt == cx->nt_first ? 0 : 1)) * kSlotFloats;
+  if (g < M) __stcg(reinterpret_cast<float2*>(slot + g * kTileN + cl), make_float2(s0, s1));
+  if (g + 8 < M) __stcg(reinterpret_cast<float2*>(slot + (g + 8) * kTileN + cl), make_float2(s2, s3));
+  __threadfence();
+  __syncthreads();
+  const int e = nt == cx->nt_first ? 0 : 1;
+  const int c_first = cx->part_first[e], c_last = cx->part_last[e];
+  if (tid == 0) cx->flags[2] = (atomicAdd(p.cnt + nt, 1) == c_last - c_first) ? 1 : 0;
+  __syncthreads();
+  if (cx->flags[2] != 0) {
+    __threadfence();
+    float2 lo = make_float2(0.f, 0.f), hi = lo;
+    for (int cc = c_first; cc <= c_last; ++cc) {
+      const float* src = p.slots + ((size_t)cc * 2 + (cc == c_first ? cx->part_slot0[e] : 0)) * kSlotFloats;
+      if (g < M) { const float2 v = __ldcg(reinterpret_cast<const float2*>(src + g * kTileN + cl)); lo.x += v.x; lo.y += v.y; }
+      if (g + 8 < M) { const float2 v = __ldcg(reinterpret_cast<const float2*>(src + (g + 8) * kTileN + cl)); hi.x += v.x; hi.y += v.y; }
+    }
+    if (col < p.N) {
+      if (g < M) *reinterpret_cast<float2*>(p.Y + (size_t)g * p.N + col) = lo;
+      if (g + 8 < M) *reinterpret_cast<float2*>(p.Y + (size_t)(g + 8) * p.N + col) = hi;
+    }
+    if (tid == 0) p.cnt[nt] = 0;                 // every contributor has arrived: ready for the next call
+  }
+  __syncthreads();                               // flags[2] may be rewritten after this
+}
+
+// The T accumulator is released by every CTA once; the last one leaves it zero for the next call.
+__device__ __noinline__ void release_tacc(const Params& p, Ctx* cx) {
+  const int tid = threadIdx.x, G = gridDim.x;
+  if (tid == 0) cx->flags[1] = (atomicAdd(p.tdone, 1) == G - 1) ? 1 : 0;
+  __syncthreads();
+  if (cx->flags[1] != 0) {
+    __threadfence();
+    for (int o = tid; o < 16 * p.k_pad; o += kThreads) p.tacc[o] = 0.0;
+    if (tid == 0) { *p.tcount = 0; *p.tdone = 0; }
+  }
+}
+
+// T -> T_q (exact bf16, [16][k_pad + 8]) in shared memory, once, before the first rank unit.
+__device__ __noinline__ void build_tq(const Params& p, Ctx* cx, uint8_t* tq) {
+  const int tid = threadIdx.x, G = gridDim.x, M = p.M;
+  const int tq_stride = (p.k_pad + 8) * 2;
+  if (tid == 0) {                                // bounded wait for the contributions of all CTAs
     const long long t0 = clock64();
-    int spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-      __nanosleep(kSleepNs);
-      if ((++spins & 63) == 0) {
-        if (*abort_flag != 0) { ok = 0; break; }
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; ok = 0; break; }
-      }
+    while (ld_acquire(p.tcount) < G) {
+      __nanosleep(64);
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) { cx->flags[0] = 1; break; }
     }
   }
-  ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-  if (ok == 0) return false;
-  if (!mbar_try_wait(bar, parity)) return mbar_wait<true>(bar, parity, abort_flag);
-  return true;
+  __syncthreads();
+  __threadfence();
+  const int total = M * p.k_pad;                 // MXINT8 along the rank: 16 adjacent lanes hold one block
+  for (int base = 0; base < total; base += kThreads) {
+    const int idx = base + tid;
+    const bool valid = idx < total;
+    const int row = valid ? idx / p.k_pad : 0, col = valid ? idx % p.k_pad : 0;
+    const double tv = valid ? __ldcg(p.tacc + (size_t)row * p.k_pad + col) : 0.0;
+    double amax = (tv != tv) ? 0.0 : fabs(tv);
+#pragma unroll
+    for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+    const int e = block_exponent(amax, p.exp_min, p.exp_max);
+    const int qv = quant_mantissa(tv, e, p.a_bits);
+    if (valid) *reinterpret_cast<uint16_t*>(tq + row * tq_stride + col * 2) = (uint16_t)bf16_bits_of(qv, e - (p.a_bits - 2));
+  }
+  __syncthreads();
+  release_tacc(p, cx);
 }
 
-// Rendezvous of the warps of one role on an mbarrier (count = number of warps), bounded like
-// every other wait of the kernel.  `use` counts the rendezvous of this role so far.
-__device__ __forceinline__ bool role_sync(uint32_t bar, uint32_t& use, volatile int* abort_flag) {
-  __syncwarp();
-  if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
-  const bool ok = warp_wait<32>(bar, use & 1u, abort_flag);
-  ++use;
-  return ok;
-}
-
-__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
-  uint8_t* stage0 = smem;
+  uint8_t* xs = smem;                                               // [kPhaseUnits] bf16 X tiles
+  uint8_t* ring = xs + (size_t)kPhaseUnits * kXTileBytes;           // [kWarps][kDepth][kSlotBytes]
   const int tq_stride = (p.k_pad + 8) * 2;
-  const int tq_bytes = (16 * tq_stride + 127) & ~127;
-  uint8_t* tq = stage0 + (size_t)p.stages * p.stage_bytes;
-  uint8_t* abuf = tq + tq_bytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(abuf + kAChunkBytes);
-  int* misc = reinterpret_cast<int*>(bars + 3 * kMaxStages + 4);
-  volatile int* abort_flag = misc;                 // misc[0]; misc[1], misc[2]: broadcast slots
-
-  const uint32_t bar0 = smem_u32(bars);
-  auto full = [&](int s) { return bar0 + 8u * s; };
-  auto xready = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
-  auto empty = [&](int s) { return bar0 + 8u * (2 * kMaxStages + s); };
-  const uint32_t afull = bar0 + 8u * (3 * kMaxStages);
-  const uint32_t tq_ready = afull + 8u, t_bar = afull + 16u, c_bar = afull + 24u;
+  uint8_t* tq = ring + (size_t)kWarps * kDepth * kSlotBytes;        // [16][k_pad + 8] bf16 T_q
+  Ctx* cx = reinterpret_cast<Ctx*>(tq + ((16 * tq_stride + 127) & ~127));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
   const int G = gridDim.x, cta = blockIdx.x;
-  const int S = p.stages;
   const int M = p.M;
+  const int col = warp * 8 + g;                                     // this lane's column within a tile
+  uint8_t* my_ring = ring + (size_t)warp * kDepth * kSlotBytes;
 
   Seq seq;
   seq.init(range_lo(cta, p.total_units, G), range_lo(cta + 1, p.total_units, G), p.U, p.k_slabs);
-  const int pre = min(seq.n, S);                   // units whose copies are issued before anything is consumed
-
-  // ---- producer helpers (used by warp 0 only)
-  Walker pw;
-  auto issue_weights = [&](int st) {
-    const uint32_t dst = smem_u32(stage0 + (size_t)st * p.stage_bytes);
-    if (pw.j < p.k_slabs) {
-      const int vc = min(kSlabK, p.K - pw.j * kSlabK);
-      mbar_expect_tx(full(st), kWTileBytes + M * vc * 4);
-      bulk_load(dst, p.wsec + ((size_t)pw.nt * p.k_slabs + pw.j) * kWTileBytes, kWTileBytes, full(st));
-    } else {
-      const int rb0 = (pw.j - p.k_slabs) * 2, nb = min(2, p.r_blocks - rb0);
-      const uint8_t* tile = p.bsec + (size_t)pw.nt * ((size_t)p.r_blocks * kTileN * 17);
-      mbar_expect_tx(full(st), nb * kTileN * 17);
-      bulk_load(dst, tile + (size_t)rb0 * kTileN * 16, nb * kTileN * 16, full(st));
-      bulk_load(dst + kWTileNibbleBytes, tile + (size_t)p.r_blocks * kTileN * 16 + rb0 * kTileN, nb * kTileN, full(st));
-    }
-  };
-  auto issue_x = [&](int st) {                     // lane r copies row r's 64 columns of this slab
-    if (pw.j < p.k_slabs && lane < M) {
-      const int vc = min(kSlabK, p.K - pw.j * kSlabK);
-      const uint32_t dst = smem_u32(stage0 + (size_t)st * p.stage_bytes + kWTileBytes + lane * 256);
-      bulk_load(dst, p.X + (size_t)lane * p.K + (size_t)pw.j * kSlabK, vc * 4, full(st));
-    }
-  };
+  const int n = seq.n;
 
   pdl_launch_dependents();
-  if (warp == 0) {
-    // The producer sets the barriers up and starts the weight copies at once (they depend on no
-    // earlier kernel); the other warps clear the tiles that must hold zeros meanwhile.
-    if (lane == 0) {
-      for (int s = 0; s < S; ++s) {
-        mbar_init(full(s), 1);
-        mbar_init(xready(s), kQuantWarps);
-        mbar_init(empty(s), kQuantWarps + kConsumerWarps);
-      }
-      mbar_init(afull, 1);
-      mbar_init(tq_ready, kTWarps);
-      mbar_init(t_bar, kTWarps);
-      mbar_init(c_bar, kConsumerWarps);
-      for (int i = 0; i < 8; ++i) misc[i] = 0;
-      fence_barrier_init();
-      fence_proxy_async_smem();
-      pw.start(seq);
-      for (int i = 0; i < pre; ++i) { issue_weights(i); pw.step(seq, i + 1); }
-    }
-  } else {
-    // rows >= M of every bf16 X tile and of T_q stay zero for the whole kernel
-    const int zt = tid - 32, zn = kThreads - 32;
-    for (int s = 0; s < S; ++s) {
-      uint8_t* xb = stage0 + (size_t)s * p.stage_bytes + kWTileBytes + p.xf_bytes;
-      for (int o = zt * 16; o < kXTileBytes; o += zn * 16) *reinterpret_cast<uint4*>(xb + o) = make_uint4(0u, 0u, 0u, 0u);
-    }
-    for (int o = zt * 16; o < tq_bytes; o += zn * 16) *reinterpret_cast<uint4*>(tq + o) = make_uint4(0u, 0u, 0u, 0u);
+  if (tid < 4) cx->flags[tid] = 0;
+  if (tid == 0) { cx->lo = seq.lo; cx->hi = seq.hi; cx->nt_first = seq.nt_first; }
+  if (tid >= 32 && tid < 34) {
+    // contributors of the first / last column tile: CTAs c_first..c_last; the first of them uses its
+    // slot 1 if the tile is not the first of its range (every later one starts inside the tile: slot 0)
+    const int e = tid - 32, nt = e == 0 ? seq.nt_first : seq.nt_last;
+    const int c_first = cta_of(nt * p.U, p.total_units, G);
+    cx->part_first[e] = c_first;
+    cx->part_last[e] = cta_of((nt + 1) * p.U - 1, p.total_units, G);
+    cx->part_slot0[e] = (range_lo(c_first, p.total_units, G) / p.U == nt) ? 0 : 1;
   }
-  __syncthreads();
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer
-    pdl_wait();                                                  // X may be an earlier kernel's output
-    pw.start(seq);
-    for (int i = 0; i < pre; ++i) { issue_x(i); pw.step(seq, i + 1); }
-    int st = 0;
-    uint32_t ph = 0;                                             // parity of the pass whose consumption is awaited
-    for (int i = pre; i < seq.n; ++i) {
-      if (!warp_wait<32>(empty(st), ph, abort_flag)) break;
-      if (lane == 0) issue_weights(st);
-      __syncwarp();
-      issue_x(st);
-      pw.step(seq, i + 1);
-      if (++st == S) { st = 0; ph ^= 1; }
-    }
-  } else if (warp <= kQuantWarps) {
-    // ------------------------------------------------------------------ quantisers
-    pdl_wait();
-    const int q = tid - 32;                    // 0..95
-    Walker wk;
-    wk.start(seq);
-    int st = 0;
-    uint32_t ph = 0;
-    for (int i = 0; i < seq.n; ++i) {
-      if (!warp_wait<32>(full(st), ph, abort_flag)) break;
-      if (wk.j < p.k_slabs) {
-        const int vc = min(kSlabK, p.K - wk.j * kSlabK);
-        const uint8_t* xf = stage0 + (size_t)st * p.stage_bytes + kWTileBytes;
-        uint8_t* xb = stage0 + (size_t)st * p.stage_bytes + kWTileBytes + p.xf_bytes;
-        // one float4 (a quarter of a 16-block) per lane and pass; every lane runs every pass
-        for (int f = q; f - q < M * 16; f += 32 * kQuantWarps) {
-          const int row = f >> 4, c4 = f & 15;
-          const bool ok = row < M;
-          const float4 v = (ok && c4 * 4 < vc) ? *reinterpret_cast<const float4*>(xf + row * 256 + c4 * 16)
-                                               : make_float4(0.f, 0.f, 0.f, 0.f);
-          int e;
-          uint32_t m8;
-          uint2 bf;
-          quantize_quad(v, p.a_bits, p.exp_min, p.exp_max, e, m8, bf);
-          if (ok) *reinterpret_cast<uint2*>(xb + row * kXTileStride + c4 * 8) = bf;
-        }
-      }
-      __syncwarp();
-      if (lane == 0) { mbar_arrive(xready(st)); mbar_arrive(empty(st)); }
-      wk.step(seq, i + 1);
-      if (++st == S) { st = 0; ph ^= 1; }
-    }
-  } else if (warp <= kQuantWarps + kTWarps) {
-    // ------------------------------------------------------------------ T = X_q A_q, then T_q
-    const int tw = warp - 1 - kQuantWarps;           // 0..3
-    const int tt = tid - 32 * (1 + kQuantWarps);     // 0..127
-    uint32_t sync_use = 0;
-    if (p.k_pad == 0) {
-      pdl_wait();
-    } else {
-      const int KB = p.K / 16;
-      const int kb_lo = (int)((long long)cta * KB / G), kb_hi = (int)((long long)(cta + 1) * KB / G);
-      const int CH = p.a_chunk_blocks;
-      const int NT = p.k_pad / 8;                    // 8-column rank tiles
-      uint8_t* amant = abuf;
-      uint8_t* aexp = abuf + (size_t)CH * p.k_pad * 16;
-      uint8_t* xa = aexp + (size_t)CH * p.k_pad;     // [M][CH * 16] fp32
-      const uint8_t* g_aexp = p.asec + (size_t)KB * p.k_pad * 16;
-      const int bias = -127 - (p.a_bits - 2) - (p.lr_bits - 2);   // exponent bytes carry +127
-      bool ok = true;
-      int ci = 0;                                    // chunk loads so far (buffer hand-over, barrier parity)
-      if (kb_lo >= kb_hi) pdl_wait();                // no share of K: still ordered behind earlier kernels
-      // 16 rank tiles per pass (4 per warp); ranks above 128 take a second pass over the same blocks
-      for (int pass = 0; pass * 16 < NT && ok && kb_lo < kb_hi; ++pass) {
-        double acc[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
-        for (int c0 = kb_lo; c0 < kb_hi && ok; c0 += CH, ++ci) {
-          const int nbc = min(CH, kb_hi - c0);
-          if (ci > 0) ok = role_sync(t_bar, sync_use, abort_flag);      // everybody is done with the buffer
-          if (tw == 0) {
-            if (lane == 0) {
-              mbar_expect_tx(afull, nbc * p.k_pad * 17 + M * nbc * 64);
-              bulk_load(smem_u32(amant), p.asec + (size_t)c0 * p.k_pad * 16, nbc * p.k_pad * 16, afull);
-              bulk_load(smem_u32(aexp), g_aexp + (size_t)c0 * p.k_pad, nbc * p.k_pad, afull);
-            }
-            __syncwarp();
-            if (ci == 0) pdl_wait();
-            if (lane < M) bulk_load(smem_u32(xa + (size_t)lane * CH * 64), p.X + (size_t)lane * p.K + (size_t)c0 * 16, nbc * 64, afull);
-          } else if (ci == 0) {
-            pdl_wait();
-          }
-          if (!warp_wait<32>(afull, ci & 1, abort_flag)) { ok = false; break; }
-          for (int b = 0; b < nbc; ++b) {
-            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            const float4 v0 = g < M ? *reinterpret_cast<const float4*>(xa + ((size_t)g * CH * 16 + b * 16 + t * 4) * 4) : z;
-            const float4 v1 = g + 8 < M ? *reinterpret_cast<const float4*>(xa + ((size_t)(g + 8) * CH * 16 + b * 16 + t * 4) * 4) : z;
-            int e0, e1;
-            uint32_t m0, m1;
-            uint2 unused;
-            quantize_quad(v0, p.a_bits, p.exp_min, p.exp_max, e0, m0, unused);
-            quantize_quad(v1, p.a_bits, p.exp_min, p.exp_max, e1, m1, unused);
-            const int ex0 = e0 + bias, ex1 = e1 + bias;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int nt = pass * 16 + tw + 4 * i;
-              if (nt < NT) {
-                const uint32_t b0 = *reinterpret_cast<const uint32_t*>(amant + ((size_t)(b * p.k_pad + nt * 8 + g) * 16) + t * 4);
-                const uint32_t ea2 = *reinterpret_cast<const uint16_t*>(aexp + b * p.k_pad + nt * 8 + t * 2);
-                int c[4];
-                mma_s8(c, m0, m1, b0);
-                const int ea_lo = (int)(ea2 & 0xFFu), ea_hi = (int)(ea2 >> 8);
-                acc[i][0] = fma((double)c[0], pow2d(ex0 + ea_lo), acc[i][0]);
-                acc[i][1] = fma((double)c[1], pow2d(ex0 + ea_hi), acc[i][1]);
-                acc[i][2] = fma((double)c[2], pow2d(ex1 + ea_lo), acc[i][2]);
-                acc[i][3] = fma((double)c[3], pow2d(ex1 + ea_hi), acc[i][3]);
-              }
-            }
-          }
-        }
-        // contribution of this CTA (exact partial sums; fp64 addition of them is exact as well
-        // unless the block exponents of one row spread over more than about 30 binades)
-        if (ok) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int nt = pass * 16 + tw + 4 * i;
-            if (nt < NT) {
-              const int col = nt * 8 + t * 2;
-              if (g < M) { atomicAdd(p.tacc + (size_t)g * p.k_pad + col, acc[i][0]); atomicAdd(p.tacc + (size_t)g * p.k_pad + col + 1, acc[i][1]); }
-              if (g + 8 < M) { atomicAdd(p.tacc + (size_t)(g + 8) * p.k_pad + col, acc[i][2]); atomicAdd(p.tacc + (size_t)(g + 8) * p.k_pad + col + 1, acc[i][3]); }
-            }
-          }
-        }
-      }
-      __threadfence();
-      role_sync(t_bar, sync_use, abort_flag);
-      if (tt == 0) atomicAdd(p.tcount, 1);
-
-      // does this CTA own rank units?
-      bool has_rank = false;
-      if (seq.n > 0) has_rank = seq.nt_first != seq.nt_last || seq.hi > seq.nt_first * p.U + p.k_slabs;
-      if (has_rank) {
-        if (tt == 0) {                                // bounded wait for the contributions of all CTAs
-          const long long t0 = clock64();
-          while (ld_acquire(p.tcount) < G) {
-            __nanosleep(100);
-            if (*abort_flag != 0) break;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 2; break; }
-          }
-        }
-        role_sync(t_bar, sync_use, abort_flag);
-        __threadfence();
-        // T -> MXINT8 along the rank (16 adjacent lanes hold one block) -> exact bf16 in shared memory
-        const int total = M * p.k_pad;
-        for (int base = 0; base < total; base += 32 * kTWarps) {
-          const int idx = base + tt;
-          const bool valid = idx < total;
-          const int row = valid ? idx / p.k_pad : 0, col = valid ? idx % p.k_pad : 0;
-          const double tv = valid ? __ldcg(p.tacc + (size_t)row * p.k_pad + col) : 0.0;
-          double amax = (tv != tv) ? 0.0 : fabs(tv);
-#pragma unroll
-          for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
-          const int e = block_exponent(amax, p.exp_min, p.exp_max);
-          const int qv = quant_mantissa(tv, e, p.a_bits);
-          if (valid) *reinterpret_cast<uint16_t*>(tq + row * tq_stride + col * 2) = (uint16_t)bf16_bits_of(qv, e - (p.a_bits - 2));
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(tq_ready);
-      }
-      // the last CTA that is done with the accumulator leaves it zero for the next call
-      role_sync(t_bar, sync_use, abort_flag);
-      if (tt == 0) misc[1] = (atomicAdd(p.tdone, 1) == G - 1) ? 1 : 0;
-      role_sync(t_bar, sync_use, abort_flag);
-      if (misc[1] != 0) {
-        __threadfence();
-        for (int o = tt; o < 16 * p.k_pad; o += 32 * kTWarps) p.tacc[o] = 0.0;
-        if (tt == 0) { *p.tcount = 0; *p.tdone = 0; }
+  // Copy of this warp's share of unit fi into its ring (nothing if the walk has ended); tab0 = first unit of the table.
+  auto issue = [&](int fi, int tab0) {
+    if (fi < n) {
+      const int nt = cx->tab_nt[fi - tab0], j = cx->tab_j[fi - tab0];
+      uint8_t* dst = my_ring + (fi % kDepth) * kSlotBytes;
+      if (j < p.k_slabs) {
+        // lane (g, t): block t of the slab for column g (16 nibbles); lanes t == 0: the column's four exponents
+        const uint8_t* tile = p.wsec + ((size_t)nt * p.k_slabs + j) * kWTileBytes;
+        cp_async8(dst + lane * 8, tile + (t >> 1) * (kTileN * 16) + col * 16 + (t & 1) * 8);
+        if (t == 0) cp_async4(dst + 256 + g * 4, tile + kWTileNibbleBytes + col * 4);
+      } else {
+        // lane (g, t): rank values 4t..4t+3 of two rank blocks for column g; lanes 0-3: exponent bytes
+        const int rb0 = (j - p.k_slabs) * 2;
+        const bool two = rb0 + 1 < p.r_blocks;
+        const uint8_t* tile = p.bsec + (size_t)nt * ((size_t)p.r_blocks * kTileN * 17);
+        const uint8_t* ex = tile + (size_t)p.r_blocks * kTileN * 16;
+        cp_async4(dst + lane * 8, tile + ((size_t)rb0 * kTileN + col) * 16 + t * 4);
+        if (two) cp_async4(dst + lane * 8 + 4, tile + ((size_t)(rb0 + 1) * kTileN + col) * 16 + t * 4);
+        if (lane < 2) cp_async4(dst + 256 + lane * 4, ex + rb0 * kTileN + warp * 8 + lane * 4);
+        if (two && lane >= 2 && lane < 4) cp_async4(dst + 264 + (lane - 2) * 4, ex + (rb0 + 1) * kTileN + warp * 8 + (lane - 2) * 4);
       }
     }
-  } else {
-    // ------------------------------------------------------------------ consumers
-    pdl_wait();
-    const int cw = warp - 1 - kQuantWarps - kTWarps;     // 0..7: columns [16 cw, 16 cw + 16) of the tile
-    const int ctid = tid - 32 * (1 + kQuantWarps + kTWarps);
-    uint32_t sync_use = 0;
-    float acc[2][4], acc_head[2][4];
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; acc_head[i][j] = 0.f; }
+    cp_async_commit();
+  };
 
-    // Contributors of the (at most two) column tiles this CTA covers only in part: CTAs
-    // c_first..c_last, and the slot the first of them uses (every later one starts inside the
-    // tile and uses its slot 0).  Computed once, while the first copies are in flight.
-    int part_first[2], part_last[2], part_slot0[2];
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int nt = e == 0 ? seq.nt_first : seq.nt_last;
-      part_first[e] = cta_of(nt * p.U, p.total_units, G);
-      part_last[e] = cta_of((nt + 1) * p.U - 1, p.total_units, G);
-      part_slot0[e] = (range_lo(part_first[e], p.total_units, G) / p.U == nt) ? 0 : 1;
+  float acc_a[4] = {0.f, 0.f, 0.f, 0.f}, acc_b[4] = {0.f, 0.f, 0.f, 0.f};   // two chains of MMAs, summed at the end
+  float acc_head[4] = {0.f, 0.f, 0.f, 0.f};
+  int cur_nt = -1;
+  bool tq_built = false;
+
+  for (int ph0 = 0; ph0 < n; ph0 += kPhaseUnits) {
+    // ---- unit table of this phase (and of the units that will be requested ahead of it)
+    __syncthreads();
+    if (tid < kTabUnits && ph0 + tid < n) {
+      const int u = seq.unit(ph0 + tid), nt = u / p.U;
+      cx->tab_nt[tid] = nt;
+      cx->tab_j[tid] = u - nt * p.U;
     }
+    __syncthreads();
+    if (ph0 == 0) {
+      // weights depend on no earlier kernel: request the first kDepth units before the dependency wait
+      for (int u = 0; u < kDepth; ++u) issue(u, 0);
+      pdl_wait();                                // X (and the workspace) may be an earlier kernel's output
+      // ---- this CTA's share of T = X_q A_q: exact int8 MMA per (16-block of K, 8 rank columns),
+      //      scaled in fp64 and added to the accumulator in the workspace
+      if (p.k_pad > 0) {
+        const int KB = p.K / 16, NT = p.k_pad / 8;
+        const int kb_lo = (int)((long long)cta * KB / G), kb_hi = (int)((long long)(cta + 1) * KB / G);
+        const uint8_t* a_exp = p.asec + (size_t)KB * p.k_pad * 16;
+        const int bias = -127 - (p.a_bits - 2) - (p.lr_bits - 2);   // exponent bytes carry +127
+        const int items = (kb_hi - kb_lo) * NT;
+        for (int it = warp; it < items; it += kWarps) {
+          const int kb = kb_lo + it / NT, nt = it % NT;
+          const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 v0 = g < M ? __ldg(reinterpret_cast<const float4*>(p.X + (size_t)g * p.K + kb * 16 + t * 4)) : z;
+          const float4 v1 = g + 8 < M ? __ldg(reinterpret_cast<const float4*>(p.X + (size_t)(g + 8) * p.K + kb * 16 + t * 4)) : z;
+          const uint32_t b0 = __ldg(reinterpret_cast<const uint32_t*>(p.asec + ((size_t)kb * p.k_pad + nt * 8 + g) * 16 + t * 4));
+          const uint32_t ea2 = __ldg(reinterpret_cast<const uint16_t*>(a_exp + (size_t)kb * p.k_pad + nt * 8 + t * 2));
+          int e0, e1;
+          uint32_t m0, m1;
+          uint2 unused;
+          quantize_quad(v0, p.a_bits, p.exp_min, p.exp_max, e0, m0, unused);
+          quantize_quad(v1, p.a_bits, p.exp_min, p.exp_max, e1, m1, unused);
+          int c[4];
+          mma_s8(c, m0, m1, b0);
+          const int ea_lo = (int)(ea2 & 0xFFu) + bias, ea_hi = (int)(ea2 >> 8) + bias;
+          const int tc = nt * 8 + t * 2;
+          // exact products; their fp64 sum is exact as well unless the block exponents of one row
+          // spread over more than about 30 binades, so the order of the additions does not matter
+          if (g < M) {
+            atomicAdd(p.tacc + (size_t)g * p.k_pad + tc, (double)c[0] * pow2d(e0 + ea_lo));
+            atomicAdd(p.tacc + (size_t)g * p.k_pad + tc + 1, (double)c[1] * pow2d(e0 + ea_hi));
+          }
+          if (g + 8 < M) {
+            atomicAdd(p.tacc + (size_t)(g + 8) * p.k_pad + tc, (double)c[2] * pow2d(e1 + ea_lo));
+            atomicAdd(p.tacc + (size_t)(g + 8) * p.k_pad + tc + 1, (double)c[3] * pow2d(e1 + ea_hi));
+          }
+        }
+      }
+    }
+    // ---- X -> MXINT8 -> exact bf16, one 16 x 64 tile per unit of the phase
+    const int cnt = min(kPhaseUnits, n - ph0);
+    {
+      const int per_unit = M * 16, total = cnt * per_unit;          // float4 items: (unit, row, quarter-block)
+      for (int base = 0; base < total; base += kThreads) {
+        const int item = base + tid;
+        const bool valid = item < total;
+        const int u = valid ? item / per_unit : 0, f = valid ? item % per_unit : 0;
+        const int row = f >> 4, c4 = f & 15;
+        const int slab = cx->tab_j[u] < p.k_slabs ? cx->tab_j[u] : -1;
+        const int xc = slab * kSlabK + c4 * 4;
+        const float4 v = (valid && slab >= 0 && xc < p.K) ? __ldg(reinterpret_cast<const float4*>(p.X + (size_t)row * p.K + xc))
+                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+        int e;
+        uint32_t m8;
+        uint2 bf;
+        quantize_quad(v, p.a_bits, p.exp_min, p.exp_max, e, m8, bf);
+        if (valid && slab >= 0) *reinterpret_cast<uint2*>(xs + (size_t)u * kXTileBytes + row * kXTileStride + c4 * 8) = bf;
+      }
+    }
+    if (ph0 == 0) __threadfence();               // the T contributions of this CTA are out
+    __syncthreads();
+    if (ph0 == 0 && tid == 0 && p.k_pad > 0) atomicAdd(p.tcount, 1);
 
-    // Hand the partial sums of column tile nt over: straight to Y when this CTA covered the whole
-    // contraction of the tile, otherwise through a slot; the last arriver adds the slots in CTA order.
-    auto flush = [&](int nt) {
-      const bool complete = nt * p.U >= seq.lo && (nt + 1) * p.U <= seq.hi;
-      const int cl = cw * 16 + t * 2;                    // + 8 cg: column within the tile
-      if (complete) {
-#pragma unroll
-        for (int cg = 0; cg < 2; ++cg) {
-          const int col = nt * kTileN + cl + 8 * cg;
-          if (col < p.N) {
-            if (g < M) *reinterpret_cast<float2*>(p.Y + (size_t)g * p.N + col) = make_float2(acc[cg][0], acc[cg][1]);
-            if (g + 8 < M) *reinterpret_cast<float2*>(p.Y + (size_t)(g + 8) * p.N + col) = make_float2(acc[cg][2], acc[cg][3]);
-          }
-        }
-        return;
-      }
-      float* slot = p.slots + ((size_t)cta * 2 + (nt == seq.nt_first ? 0 : 1)) * kSlotFloats;
-#pragma unroll
-      for (int cg = 0; cg < 2; ++cg) {
-        if (g < M) __stcg(reinterpret_cast<float2*>(slot + g * kTileN + cl + 8 * cg), make_float2(acc[cg][0], acc[cg][1]));
-        if (g + 8 < M) __stcg(reinterpret_cast<float2*>(slot + (g + 8) * kTileN + cl + 8 * cg), make_float2(acc[cg][2], acc[cg][3]));
-      }
-      __threadfence();
-      role_sync(c_bar, sync_use, abort_flag);
-      const int e = nt == seq.nt_first ? 0 : 1;
-      const int c_first = part_first[e], c_last = part_last[e];
-      if (ctid == 0) misc[2] = (atomicAdd(p.cnt + nt, 1) == c_last - c_first) ? 1 : 0;
-      role_sync(c_bar, sync_use, abort_flag);
-      if (misc[2] != 0) {
-        __threadfence();
-        float2 s[2][2];
-#pragma unroll
-        for (int cg = 0; cg < 2; ++cg) { s[cg][0] = make_float2(0.f, 0.f); s[cg][1] = make_float2(0.f, 0.f); }
-        for (int cc = c_first; cc <= c_last; ++cc) {
-          const float* src = p.slots + ((size_t)cc * 2 + (cc == c_first ? part_slot0[e] : 0)) * kSlotFloats;
-#pragma unroll
-          for (int cg = 0; cg < 2; ++cg) {
-            if (g < M) { const float2 v = __ldcg(reinterpret_cast<const float2*>(src + g * kTileN + cl + 8 * cg)); s[cg][0].x += v.x; s[cg][0].y += v.y; }
-            if (g + 8 < M) { const float2 v = __ldcg(reinterpret_cast<const float2*>(src + (g + 8) * kTileN + cl + 8 * cg)); s[cg][1].x += v.x; s[cg][1].y += v.y; }
-          }
-        }
-#pragma unroll
-        for (int cg = 0; cg < 2; ++cg) {
-          const int col = nt * kTileN + cl + 8 * cg;
-          if (col < p.N) {
-            if (g < M) *reinterpret_cast<float2*>(p.Y + (size_t)g * p.N + col) = s[cg][0];
-            if (g + 8 < M) *reinterpret_cast<float2*>(p.Y + (size_t)(g + 8) * p.N + col) = s[cg][1];
-          }
-        }
-        if (ctid == 0) p.cnt[nt] = 0;                  // every contributor has arrived: ready for the next call
-      }
-      role_sync(c_bar, sync_use, abort_flag);          // misc[2] may be rewritten after this
-    };
-
-    int cur_nt = -1;
-    bool tq_waited = false;
-    Walker wk;
-    wk.start(seq);
-    int st = 0;
-    uint32_t ph = 0;
-    for (int i = 0; i < seq.n; ++i) {
-      const int nt = wk.nt, j = wk.j;
-      if (seq.reordered && i == seq.n_before) {
-        // the deferred rank units of the first column tile: finish the current tile, resume the first
-        if (cur_nt >= 0) flush(cur_nt);
-#pragma unroll
-        for (int a = 0; a < 2; ++a)
-#pragma unroll
-          for (int b = 0; b < 4; ++b) acc[a][b] = acc_head[a][b];
-        cur_nt = nt;
-      } else if (nt != cur_nt) {
+    // ---- the units of the phase
+#pragma unroll 1
+    for (int i = ph0; i < ph0 + cnt; ++i) {
+      const int nt = cx->tab_nt[i - ph0], j = cx->tab_j[i - ph0];
+      const bool deferred_start = seq.reordered && i == seq.n_before;
+      if (nt != cur_nt || deferred_start) {
+        // column-tile boundary (uniform over the CTA): the first tile's sums are kept when its rank
+        // units are deferred, any other tile's sums are handed over
         if (cur_nt >= 0) {
-          if (seq.reordered && cur_nt == seq.nt_first) {
+          if (!deferred_start && seq.reordered && cur_nt == seq.nt_first) {
 #pragma unroll
-            for (int a = 0; a < 2; ++a)
-#pragma unroll
-              for (int b = 0; b < 4; ++b) acc_head[a][b] = acc[a][b];
+            for (int a = 0; a < 4; ++a) acc_head[a] = acc_a[a] + acc_b[a];
           } else {
-            flush(cur_nt);
+            flush_tile(p, cx, cur_nt, acc_a[0] + acc_b[0], acc_a[1] + acc_b[1], acc_a[2] + acc_b[2], acc_a[3] + acc_b[3]);
           }
+#pragma unroll
+          for (int a = 0; a < 4; ++a) { acc_a[a] = 0.f; acc_b[a] = 0.f; }
         }
-#pragma unroll
-        for (int a = 0; a < 2; ++a)
-#pragma unroll
-          for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
         cur_nt = nt;
       }
-      if (!warp_wait<20>(full(st), ph, abort_flag)) break;
-      if (!warp_wait<20>(xready(st), ph, abort_flag)) break;
-      const uint8_t* stage = stage0 + (size_t)st * p.stage_bytes;
+      cp_async_wait<kDepth - 1>();
+      __syncwarp();
+      const uint8_t* slot = my_ring + (i % kDepth) * kSlotBytes;
       if (j < p.k_slabs) {
         // ---- 64 K of W_q: lane (g, t) holds block t of the slab for row g (A side) and column g (B side)
-        const uint8_t* xb = stage + kWTileBytes + p.xf_bytes;
+        const uint8_t* xb = xs + (size_t)(i - ph0) * kXTileBytes;
         const uint4 q0 = *reinterpret_cast<const uint4*>(xb + g * kXTileStride + t * 32);
         const uint4 q1 = *reinterpret_cast<const uint4*>(xb + g * kXTileStride + t * 32 + 16);
         uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
@@ -542,57 +382,43 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const Params p) {
           r0 = *reinterpret_cast<const uint4*>(xb + (g + 8) * kXTileStride + t * 32);
           r1 = *reinterpret_cast<const uint4*>(xb + (g + 8) * kXTileStride + t * 32 + 16);
         }
-#pragma unroll
-        for (int cg = 0; cg < 2; ++cg) {
-          const int col = cw * 16 + cg * 8 + g;
-          const uint2 w = *reinterpret_cast<const uint2*>(stage + (t >> 1) * (kTileN * 16) + col * 16 + (t & 1) * 8);
-          const uint32_t eb = stage[kWTileNibbleBytes + col * 4 + t];
-          uint32_t s2, c2;
-          w_scales(eb, s2, c2);
-          const uint4 b0 = convert_word(w.x, s2, c2), b1 = convert_word(w.y, s2, c2);
-          mma_bf16(acc[cg], q0.x, r0.x, q0.y, r0.y, b0.x, b0.y);
-          mma_bf16(acc[cg], q0.z, r0.z, q0.w, r0.w, b0.z, b0.w);
-          mma_bf16(acc[cg], q1.x, r1.x, q1.y, r1.y, b1.x, b1.y);
-          mma_bf16(acc[cg], q1.z, r1.z, q1.w, r1.w, b1.z, b1.w);
-        }
+        const uint2 w = *reinterpret_cast<const uint2*>(slot + lane * 8);
+        uint32_t s2, c2;
+        w_scales(slot[256 + lane], s2, c2);
+        const uint4 b0 = convert_word(w.x, s2, c2), b1 = convert_word(w.y, s2, c2);
+        mma_bf16(acc_a, q0.x, r0.x, q0.y, r0.y, b0.x, b0.y);
+        mma_bf16(acc_b, q0.z, r0.z, q0.w, r0.w, b0.z, b0.w);
+        mma_bf16(acc_a, q1.x, r1.x, q1.y, r1.y, b1.x, b1.y);
+        mma_bf16(acc_b, q1.z, r1.z, q1.w, r1.w, b1.z, b1.w);
       } else {
-        // ---- 32 rank values of B_q against T_q
-        if (!tq_waited) {
-          if (!warp_wait<32>(tq_ready, 0u, abort_flag)) break;
-          tq_waited = true;
-        }
-        const int rb0 = (j - p.k_slabs) * 2, nb = min(2, p.r_blocks - rb0);
-        for (int rb = 0; rb < nb; ++rb) {
+        // ---- up to 32 rank values of B_q against T_q
+        if (!tq_built) { build_tq(p, cx, tq); tq_built = true; }
+        const int rb0 = (j - p.k_slabs) * 2;
+        const uint2 w = *reinterpret_cast<const uint2*>(slot + lane * 8);
+        for (int rb = 0; rb < 2 && rb0 + rb < p.r_blocks; ++rb) {
           const uint2 a_lo = *reinterpret_cast<const uint2*>(tq + g * tq_stride + ((rb0 + rb) * 16 + t * 4) * 2);
           uint2 a_hi = make_uint2(0u, 0u);
           if (M > 8) a_hi = *reinterpret_cast<const uint2*>(tq + (g + 8) * tq_stride + ((rb0 + rb) * 16 + t * 4) * 2);
-#pragma unroll
-          for (int cg = 0; cg < 2; ++cg) {
-            const int col = cw * 16 + cg * 8 + g;
-            const uint32_t wv = *reinterpret_cast<const uint32_t*>(stage + (rb * kTileN + col) * 16 + t * 4);
-            const float scale = pow2f((int)stage[kWTileNibbleBytes + rb * kTileN + col] - 127 - (p.lr_bits - 2));
-            const uint32_t b0 = pack_bf16x2((float)(int8_t)(wv) * scale, (float)(int8_t)(wv >> 8) * scale);
-            const uint32_t b1 = pack_bf16x2((float)(int8_t)(wv >> 16) * scale, (float)(int8_t)(wv >> 24) * scale);
-            mma_bf16(acc[cg], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b0, b1);
-          }
+          const uint32_t wv = rb == 0 ? w.x : w.y;
+          const float scale = pow2f((int)slot[256 + rb * 8 + g] - 127 - (p.lr_bits - 2));
+          const uint32_t b0 = pack_bf16x2((float)(int8_t)(wv) * scale, (float)(int8_t)(wv >> 8) * scale);
+          const uint32_t b1 = pack_bf16x2((float)(int8_t)(wv >> 16) * scale, (float)(int8_t)(wv >> 24) * scale);
+          mma_bf16(acc_a, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b0, b1);
         }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty(st));
-      wk.step(seq, i + 1);
-      if (++st == S) { st = 0; ph ^= 1; }
+      __syncwarp();                              // the slot is free: request the unit kDepth ahead into it
+      issue(i + kDepth, ph0);
     }
-    if (cur_nt >= 0 && *abort_flag == 0) flush(cur_nt);
   }
-
-  // ------------------------------------------------------------------ teardown
-  __syncthreads();
-  if (*abort_flag != 0) {
-    // a wait ran out: give copies that may still be in flight time to land before shared memory goes away
-    const long long t0 = clock64();
-    while (clock64() - t0 < 400000) { }
-    if (tid == 0) report_error(p.status, LQER_ERR_TIMEOUT, 500 + *abort_flag, cta);
+  if (cur_nt >= 0) {
+    // with a deferred part, the last segment belongs to the first tile
+    const float h0 = seq.reordered ? acc_head[0] : 0.f, h1 = seq.reordered ? acc_head[1] : 0.f;
+    const float h2 = seq.reordered ? acc_head[2] : 0.f, h3 = seq.reordered ? acc_head[3] : 0.f;
+    flush_tile(p, cx, cur_nt, acc_a[0] + acc_b[0] + h0, acc_a[1] + acc_b[1] + h1, acc_a[2] + acc_b[2] + h2, acc_a[3] + acc_b[3] + h3);
   }
+  if (p.k_pad > 0 && !tq_built) release_tacc(p, cx);
+  cp_async_wait<0>();
+  if (cx->flags[0] != 0 && tid == 0) report_error(p.status, LQER_ERR_TIMEOUT, 500, cta);
 }
 
 }  // namespace dec
@@ -604,11 +430,13 @@ cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void
   using namespace dec;
   static int sm_count = 0;
   static bool attr_set = false;
+  const size_t fixed = (size_t)kPhaseUnits * kXTileBytes + (size_t)kWarps * kDepth * kSlotBytes + sizeof(Ctx) + 256;
   if (!attr_set) {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(fixed + 16 * (256 + 8) * 2 + 128));
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -628,27 +456,8 @@ cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void
   p.U = m.k_slabs + (m.r_blocks + 1) / 2;
   p.total_units = decode_units(m);
   p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
-
   const int G = decode_ctas(m, sm_count);
-  p.xf_bytes = M * 256;
-  p.stage_bytes = kWTileBytes + p.xf_bytes + kXTileBytes;
-  const int tq_bytes = (16 * (m.k_pad + 8) * 2 + 127) & ~127;
-  const int fixed = tq_bytes + kAChunkBytes + (3 * kMaxStages + 4) * 8 + 64 + 128;
-  const int per_cta = (p.total_units + G - 1) / G;
-  int stages = (kSmemBudget - fixed) / p.stage_bytes;
-  if (stages > kMaxStages) stages = kMaxStages;
-  if (stages > per_cta) stages = per_cta;
-  if (stages < 1) return cudaErrorInvalidValue;
-  p.stages = stages;
-  p.a_chunk_blocks = 1;
-  if (m.k_pad > 0) {
-    const int KB = m.K / 16;
-    const int need = (KB + G - 1) / G;
-    const int fit = kAChunkBytes / (m.k_pad * 17 + M * 64);
-    if (fit < 1) return cudaErrorInvalidValue;
-    p.a_chunk_blocks = need < fit ? need : fit;
-  }
-  const size_t smem = (size_t)stages * p.stage_bytes + fixed;
+  const size_t smem = fixed + ((16 * (m.k_pad + 8) * 2 + 127) & ~127);
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(G);
