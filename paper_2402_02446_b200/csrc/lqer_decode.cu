@@ -90,11 +90,11 @@ struct Seq {
   }
 };
 
-// First unit of CTA c's range (the product may exceed 32 bits; used a few times per thread only).
-__device__ __forceinline__ int range_lo(int c, int total, int G) { return (int)((long long)c * total / G); }
+// First unit of CTA c's range.  32-bit arithmetic: the host refuses layers with total * G >= 2^32.
+__device__ __forceinline__ int range_lo(int c, int total, int G) { return (int)((uint32_t)c * (uint32_t)total / (uint32_t)G); }
 // The CTA whose range holds unit u.
 __device__ __forceinline__ int cta_of(int u, int total, int G) {
-  return (int)((((long long)u + 1) * G + total - 1) / total) - 1;
+  return (int)((((uint32_t)u + 1u) * (uint32_t)G + (uint32_t)total - 1u) / (uint32_t)total) - 1;
 }
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -126,13 +126,14 @@ struct Ctx {
   int lo, hi, nt_first;
   int part_first[2], part_last[2], part_slot0[2];   // contributors of the first / last column tile of the range
   int tab_nt[kTabUnits], tab_j[kTabUnits];           // (column tile, slab or rank unit) of units [tab0, tab0 + kTabUnits)
-  int flags[4];                                      // [0] a bounded wait ran out, [1], [2] broadcast slots
+  int pending[2];                                    // column tile + 1 whose sums sit in this CTA's slot 0 / 1
+  int flags[4];                                      // [0] a bounded wait ran out, [1], [2], [3] broadcast slots
 };
 
-// Hand the sums of column tile nt over (rare path, kept out of line so that the unit loop stays
-// small): straight to Y when this CTA covered the whole contraction of the tile, otherwise
-// through a slot; the last CTA to arrive adds the slots in CTA order.  Called by all threads.
-__device__ __noinline__ void flush_tile(const Params& p, Ctx* cx, int nt, float s0, float s1, float s2, float s3) {
+// Hand the sums of column tile nt over (rare path, out of line so that the unit loop stays small).
+// A tile whose whole contraction this CTA covered goes straight to Y.  Otherwise the sums go to
+// this CTA's slot for the tile and the tile is marked pending; nothing is waited for here.
+__device__ __noinline__ void store_partial(const Params& p, Ctx* cx, int nt, float s0, float s1, float s2, float s3) {
   const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int M = p.M, cta = blockIdx.x;
   const bool complete = nt * p.U >= cx->lo && (nt + 1) * p.U <= cx->hi;
@@ -144,19 +145,42 @@ __device__ __noinline__ void flush_tile(const Params& p, Ctx* cx, int nt, float 
     }
     return;
   }
-  float* slot = p.slots + ((size_t)cta * 2 + (nt == cx->nt_first ? 0 : 1)) * kSlotFloats;
+  const int e = nt == cx->nt_first ? 0 : 1;
+  float* slot = p.slots + ((size_t)cta * 2 + e) * kSlotFloats;
   if (g < M) __stcg(reinterpret_cast<float2*>(slot + g * kTileN + cl), make_float2(s0, s1));
   if (g + 8 < M) __stcg(reinterpret_cast<float2*>(slot + (g + 8) * kTileN + cl), make_float2(s2, s3));
-  __threadfence();
+  if (tid == 0) cx->pending[e] = nt + 1;
+}
+
+// End of the kernel: announce the pending slots (one release-acquire increment per tile, after a
+// CTA barrier that orders every thread's slot stores before it); whoever arrives last at a tile
+// adds the slots of all its contributors in CTA order and writes Y.
+__device__ __noinline__ void finish_tiles(const Params& p, Ctx* cx) {
+  const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int M = p.M;
   __syncthreads();
-  const int e = nt == cx->nt_first ? 0 : 1;
-  const int c_first = cx->part_first[e], c_last = cx->part_last[e];
-  if (tid == 0) cx->flags[2] = (atomicAdd(p.cnt + nt, 1) == c_last - c_first) ? 1 : 0;
+  if (tid < 2) {
+    int last = 0;
+    const int nt = cx->pending[tid] - 1;
+    if (nt >= 0) {
+      int old;
+      asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.cnt + nt) : "memory");
+      last = old == cx->part_last[tid] - cx->part_first[tid];
+      if (last) p.cnt[nt] = 0;                   // every contributor has arrived: ready for the next call
+    }
+    cx->flags[2 + tid] = last;
+  }
   __syncthreads();
-  if (cx->flags[2] != 0) {
+#pragma unroll 1
+  for (int e = 0; e < 2; ++e) {
+    if (cx->flags[2 + e] == 0) continue;
     __threadfence();
+    const int nt = cx->pending[e] - 1;
+    const int c_first = cx->part_first[e], c_last = cx->part_last[e];
+    const int cl = (tid >> 5) * 8 + t * 2, col = nt * kTileN + cl;
     float2 lo = make_float2(0.f, 0.f), hi = lo;
     for (int cc = c_first; cc <= c_last; ++cc) {
+      // a contributor's slot for the tile: slot 1 only if the tile is not the first of its range
       const float* src = p.slots + ((size_t)cc * 2 + (cc == c_first ? cx->part_slot0[e] : 0)) * kSlotFloats;
       if (g < M) { const float2 v = __ldcg(reinterpret_cast<const float2*>(src + g * kTileN + cl)); lo.x += v.x; lo.y += v.y; }
       if (g + 8 < M) { const float2 v = __ldcg(reinterpret_cast<const float2*>(src + (g + 8) * kTileN + cl)); hi.x += v.x; hi.y += v.y; }
@@ -165,9 +189,7 @@ __device__ __noinline__ void flush_tile(const Params& p, Ctx* cx, int nt, float 
       if (g < M) *reinterpret_cast<float2*>(p.Y + (size_t)g * p.N + col) = lo;
       if (g + 8 < M) *reinterpret_cast<float2*>(p.Y + (size_t)(g + 8) * p.N + col) = hi;
     }
-    if (tid == 0) p.cnt[nt] = 0;                 // every contributor has arrived: ready for the next call
   }
-  __syncthreads();                               // flags[2] may be rewritten after this
 }
 
 // The T accumulator is released by every CTA once; the last one leaves it zero for the next call.
@@ -234,6 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 
   pdl_launch_dependents();
   if (tid < 4) cx->flags[tid] = 0;
+  if (tid < 2) cx->pending[tid] = 0;
   if (tid == 0) { cx->lo = seq.lo; cx->hi = seq.hi; cx->nt_first = seq.nt_first; }
   if (tid >= 32 && tid < 34) {
     // contributors of the first / last column tile: CTAs c_first..c_last; the first of them uses its
@@ -286,13 +309,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     __syncthreads();
     if (ph0 == 0) {
       // weights depend on no earlier kernel: request the first kDepth units before the dependency wait
+#pragma unroll 4
       for (int u = 0; u < kDepth; ++u) issue(u, 0);
       pdl_wait();                                // X (and the workspace) may be an earlier kernel's output
       // ---- this CTA's share of T = X_q A_q: exact int8 MMA per (16-block of K, 8 rank columns),
       //      scaled in fp64 and added to the accumulator in the workspace
       if (p.k_pad > 0) {
         const int KB = p.K / 16, NT = p.k_pad / 8;
-        const int kb_lo = (int)((long long)cta * KB / G), kb_hi = (int)((long long)(cta + 1) * KB / G);
+        const int kb_lo = cta * KB / G, kb_hi = (cta + 1) * KB / G;
         const uint8_t* a_exp = p.asec + (size_t)KB * p.k_pad * 16;
         const int bias = -127 - (p.a_bits - 2) - (p.lr_bits - 2);   // exponent bytes carry +127
         const int items = (kb_hi - kb_lo) * NT;
@@ -345,13 +369,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         if (valid && slab >= 0) *reinterpret_cast<uint2*>(xs + (size_t)u * kXTileBytes + row * kXTileStride + c4 * 8) = bf;
       }
     }
-    if (ph0 == 0) __threadfence();               // the T contributions of this CTA are out
     __syncthreads();
-    if (ph0 == 0 && tid == 0 && p.k_pad > 0) atomicAdd(p.tcount, 1);
+    if (ph0 == 0 && tid == 0 && p.k_pad > 0)     // the T contributions of this CTA are out (ordered by the barrier)
+      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.tcount) : "memory");
 
-    // ---- the units of the phase
+    // ---- the units of the phase, in runs that share a column tile and a kind
+    int i = ph0;
+    const int ph_end = ph0 + cnt;
 #pragma unroll 1
-    for (int i = ph0; i < ph0 + cnt; ++i) {
+    while (i < ph_end) {
       const int nt = cx->tab_nt[i - ph0], j = cx->tab_j[i - ph0];
       const bool deferred_start = seq.reordered && i == seq.n_before;
       if (nt != cur_nt || deferred_start) {
@@ -362,37 +388,67 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 #pragma unroll
             for (int a = 0; a < 4; ++a) acc_head[a] = acc_a[a] + acc_b[a];
           } else {
-            flush_tile(p, cx, cur_nt, acc_a[0] + acc_b[0], acc_a[1] + acc_b[1], acc_a[2] + acc_b[2], acc_a[3] + acc_b[3]);
+            store_partial(p, cx, cur_nt, acc_a[0] + acc_b[0], acc_a[1] + acc_b[1], acc_a[2] + acc_b[2], acc_a[3] + acc_b[3]);
           }
 #pragma unroll
           for (int a = 0; a < 4; ++a) { acc_a[a] = 0.f; acc_b[a] = 0.f; }
         }
         cur_nt = nt;
       }
-      cp_async_wait<kDepth - 1>();
-      __syncwarp();
-      const uint8_t* slot = my_ring + (i % kDepth) * kSlotBytes;
       if (j < p.k_slabs) {
-        // ---- 64 K of W_q: lane (g, t) holds block t of the slab for row g (A side) and column g (B side)
-        const uint8_t* xb = xs + (size_t)(i - ph0) * kXTileBytes;
-        const uint4 q0 = *reinterpret_cast<const uint4*>(xb + g * kXTileStride + t * 32);
-        const uint4 q1 = *reinterpret_cast<const uint4*>(xb + g * kXTileStride + t * 32 + 16);
-        uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
-        if (M > 8) {
-          r0 = *reinterpret_cast<const uint4*>(xb + (g + 8) * kXTileStride + t * 32);
-          r1 = *reinterpret_cast<const uint4*>(xb + (g + 8) * kXTileStride + t * 32 + 16);
+        // ---- a run of slabs of W_q (consecutive units): four at a time, so that their chains of
+        //      shared-memory loads, conversions and MMAs overlap
+        int run_end = min(ph_end, i + (p.k_slabs - j));
+        if (seq.reordered && i < seq.n_before) run_end = min(run_end, seq.n_before);   // the deferred part starts there
+        // 64 K of W_q: lane (g, t) holds block t of the slab for row g (A side) and column g (B side)
+        auto slab = [&](int iu, float (&ca)[4], float (&cb)[4]) {
+          const uint8_t* slot = my_ring + (iu % kDepth) * kSlotBytes;
+          const uint8_t* xb = xs + (size_t)(iu - ph0) * kXTileBytes;
+          const uint4 q0 = *reinterpret_cast<const uint4*>(xb + g * kXTileStride + t * 32);
+          const uint4 q1 = *reinterpret_cast<const uint4*>(xb + g * kXTileStride + t * 32 + 16);
+          uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
+          if (M > 8) {
+            r0 = *reinterpret_cast<const uint4*>(xb + (g + 8) * kXTileStride + t * 32);
+            r1 = *reinterpret_cast<const uint4*>(xb + (g + 8) * kXTileStride + t * 32 + 16);
+          }
+          const uint2 w = *reinterpret_cast<const uint2*>(slot + lane * 8);
+          uint32_t s2, c2;
+          w_scales(slot[256 + lane], s2, c2);
+          const uint4 b0 = convert_word(w.x, s2, c2), b1 = convert_word(w.y, s2, c2);
+          mma_bf16(ca, q0.x, r0.x, q0.y, r0.y, b0.x, b0.y);
+          mma_bf16(cb, q0.z, r0.z, q0.w, r0.w, b0.z, b0.w);
+          mma_bf16(ca, q1.x, r1.x, q1.y, r1.y, b1.x, b1.y);
+          mma_bf16(cb, q1.z, r1.z, q1.w, r1.w, b1.z, b1.w);
+        };
+#pragma unroll 1
+        for (; i + 4 <= run_end; i += 4) {
+          cp_async_wait<kDepth - 4>();
+          __syncwarp();
+          float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+          slab(i, acc_a, acc_b);
+          slab(i + 1, c0, c1);
+          slab(i + 2, acc_a, acc_b);
+          slab(i + 3, c0, c1);
+#pragma unroll
+          for (int a = 0; a < 4; ++a) { acc_a[a] += c0[a]; acc_b[a] += c1[a]; }
+          __syncwarp();                          // the four slots are free: request the units kDepth ahead
+#pragma unroll 1
+          for (int u = 0; u < 4; ++u) issue(i + kDepth + u, ph0);
         }
-        const uint2 w = *reinterpret_cast<const uint2*>(slot + lane * 8);
-        uint32_t s2, c2;
-        w_scales(slot[256 + lane], s2, c2);
-        const uint4 b0 = convert_word(w.x, s2, c2), b1 = convert_word(w.y, s2, c2);
-        mma_bf16(acc_a, q0.x, r0.x, q0.y, r0.y, b0.x, b0.y);
-        mma_bf16(acc_b, q0.z, r0.z, q0.w, r0.w, b0.z, b0.w);
-        mma_bf16(acc_a, q1.x, r1.x, q1.y, r1.y, b1.x, b1.y);
-        mma_bf16(acc_b, q1.z, r1.z, q1.w, r1.w, b1.z, b1.w);
+#pragma unroll 1
+        for (; i < run_end; ++i) {
+          cp_async_wait<kDepth - 1>();
+          __syncwarp();
+          slab(i, acc_a, acc_b);
+          __syncwarp();
+          issue(i + kDepth, ph0);
+        }
       } else {
         // ---- up to 32 rank values of B_q against T_q
         if (!tq_built) { build_tq(p, cx, tq); tq_built = true; }
+        cp_async_wait<kDepth - 1>();
+        __syncwarp();
+        const uint8_t* slot = my_ring + (i % kDepth) * kSlotBytes;
         const int rb0 = (j - p.k_slabs) * 2;
         const uint2 w = *reinterpret_cast<const uint2*>(slot + lane * 8);
         for (int rb = 0; rb < 2 && rb0 + rb < p.r_blocks; ++rb) {
@@ -405,17 +461,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
           const uint32_t b1 = pack_bf16x2((float)(int8_t)(wv >> 16) * scale, (float)(int8_t)(wv >> 24) * scale);
           mma_bf16(acc_a, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b0, b1);
         }
+        __syncwarp();
+        issue(i + kDepth, ph0);
+        ++i;
       }
-      __syncwarp();                              // the slot is free: request the unit kDepth ahead into it
-      issue(i + kDepth, ph0);
     }
   }
   if (cur_nt >= 0) {
     // with a deferred part, the last segment belongs to the first tile
     const float h0 = seq.reordered ? acc_head[0] : 0.f, h1 = seq.reordered ? acc_head[1] : 0.f;
     const float h2 = seq.reordered ? acc_head[2] : 0.f, h3 = seq.reordered ? acc_head[3] : 0.f;
-    flush_tile(p, cx, cur_nt, acc_a[0] + acc_b[0] + h0, acc_a[1] + acc_b[1] + h1, acc_a[2] + acc_b[2] + h2, acc_a[3] + acc_b[3] + h3);
+    store_partial(p, cx, cur_nt, acc_a[0] + acc_b[0] + h0, acc_a[1] + acc_b[1] + h1, acc_a[2] + acc_b[2] + h2, acc_a[3] + acc_b[3] + h3);
   }
+  finish_tiles(p, cx);
   if (p.k_pad > 0 && !tq_built) release_tacc(p, cx);
   cp_async_wait<0>();
   if (cx->flags[0] != 0 && tid == 0) report_error(p.status, LQER_ERR_TIMEOUT, 500, cta);
@@ -457,6 +515,7 @@ cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void
   p.total_units = decode_units(m);
   p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
   const int G = decode_ctas(m, sm_count);
+  if ((unsigned long long)(p.total_units + 1) * (unsigned long long)(G + 1) >= (1ull << 32)) return cudaErrorInvalidValue;
   const size_t smem = fixed + ((16 * (m.k_pad + 8) * 2 + 127) & ~127);
 
   cudaLaunchConfig_t cfg = {};
