@@ -178,8 +178,9 @@ lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void*
 /* Read the device-side status word of `workspace` (synchronises `stream`). */
 lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_t* device_status);
 
-/* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 decode kernel,
- * 3 tensor-core kernel (one CTA per tile), 4 tensor-core kernel (CTA pair per tile).
+/* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 decode kernels
+ * (column-owner kernel for M <= 4, split-K kernel for M <= 16), 3 tensor-core kernel (one CTA per
+ * tile), 4 tensor-core kernel (CTA pair per tile), 5 split-K decode kernel for every M <= 16.
  * Host only, process wide. */
 lqer_status_t lqer_set_path(int path);
 

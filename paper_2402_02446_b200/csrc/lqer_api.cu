@@ -136,14 +136,15 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
   int path = g_path.load();
   if (project_only) path = 3;
   if (path == 0 && M <= decode_max_m()) path = 2;
-  if (path == 2 && M > decode_max_m()) return LQER_ERR_SHAPE;
-  if (workspace_bytes < call_bytes(m, M, path == 2)) return LQER_ERR_BUFFER_TOO_SMALL;
+  const bool decode = path == 2 || path == 5;
+  if (decode && M > decode_max_m()) return LQER_ERR_SHAPE;
+  if (workspace_bytes < call_bytes(m, M, decode)) return LQER_ERR_BUFFER_TOO_SMALL;
   if ((st = check_arch()) != LQER_OK) return st;
   DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
   void* xcat = static_cast<uint8_t*>(workspace) + align_up(persist_bytes(m), 256);
   cudaError_t err;
-  if (path == 2) {
-    err = launch_decode(X, M, m, packed, Y, workspace, s);
+  if (decode) {
+    err = launch_decode(X, M, m, packed, Y, workspace, s, path == 5);
   } else {
     if (path == 1 && M > 65535) return LQER_ERR_SHAPE;
     err = launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
@@ -329,7 +330,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     lqer_status_t st = lookup(c.packed, m);
     if (st != LQER_OK) return st;
     const int path = g_path.load();
-    const bool decode = path == 2 || (path == 0 && c.M <= decode_max_m());
+    const bool decode = path == 2 || path == 5 || (path == 0 && c.M <= decode_max_m());
     if (workspace_bytes < call_bytes(m, c.M, decode)) return LQER_ERR_BUFFER_TOO_SMALL;
   }
   for (int i = 0; i < n_calls; ++i) {
@@ -380,7 +381,7 @@ lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_
 }
 
 lqer_status_t lqer_set_path(int path) {
-  if (path < 0 || path > 4) return LQER_ERR_CONFIG;
+  if (path < 0 || path > 5) return LQER_ERR_CONFIG;
   g_path.store(path);
   return LQER_OK;
 }

@@ -200,8 +200,12 @@ cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const v
                            DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s);
+// M <= 4 goes to the column-owner kernel unless force_split_k (test hook: the split-K kernel serves every M <= 16).
 cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
-                          void* workspace, cudaStream_t s);
+                          void* workspace, cudaStream_t s, bool force_split_k = false);
+cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
+                               void* workspace, cudaStream_t s);
+bool decode_cols_fits(const PackedMeta& m, int M);
 int decode_max_m();
 
 }  // namespace lqer

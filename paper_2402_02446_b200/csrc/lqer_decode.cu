@@ -479,13 +479,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   if (cx->flags[0] != 0 && tid == 0) report_error(p.status, LQER_ERR_TIMEOUT, 500, cta);
 }
 
+
 }  // namespace dec
 
 int decode_max_m() { return 16; }
 
 cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void* packed, float* Y, void* workspace,
-                          cudaStream_t s) {
+                          cudaStream_t s, bool force_split_k) {
   using namespace dec;
+  if (decode_cols_fits(m, M) && !force_split_k) return launch_decode_cols(X, M, m, packed, Y, workspace, s);
   static int sm_count = 0;
   static bool attr_set = false;
   const size_t fixed = (size_t)kPhaseUnits * kXTileBytes + (size_t)kWarps * kDepth * kSlotBytes + sizeof(Ctx) + 256;

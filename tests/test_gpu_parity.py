@@ -153,14 +153,16 @@ DECODE_SPECS = SMALL_SPECS + MID_SPECS + [
 ]
 
 
-@pytest.mark.parametrize("M", [1, 5, 16])
+@pytest.mark.parametrize("M,path", [(1, binding.PATH_DECODE), (3, binding.PATH_DECODE), (4, binding.PATH_DECODE),
+                                    (1, binding.PATH_DECODE_SPLIT_K), (5, binding.PATH_DECODE), (16, binding.PATH_DECODE)],
+                         ids=["cols_M1", "cols_M3", "cols_M4", "splitk_M1", "splitk_M5", "splitk_M16"])
 @pytest.mark.parametrize("spec", DECODE_SPECS, ids=lambda s: s.name)
-def test_linear_decode_kernel(spec, M):
+def test_linear_decode_kernel(spec, M, path):
     W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
     X = gen.make_activations(spec, M=M)
     ref = olqer.forward(X, P)
     ws = L.new_workspace(M, Pg)
-    L.set_path(binding.PATH_DECODE)
+    L.set_path(path)
     try:
         Y = L.linear(_t(X), Pg, ws).cpu().numpy()
         Y2 = L.linear(_t(X), Pg, ws).cpu().numpy()      # same workspace again: the kernel left its counters at zero
