@@ -18,9 +18,11 @@
 // bytes of nibbles + 32 exponent bytes) goes global -> registers, four slabs (16 units) ahead;
 // these loads depend on no earlier kernel and are issued before griddepcontrol.wait.
 //
-// T = X_q A_q: every CTA adds the exact partial products of its share of K (int8 tensor-core MMA
-// per 16-block, scaled in fp64) to an accumulator in the workspace at kernel start; before its
-// rank part each CTA waits (bounded) until all G contributions have arrived and re-quantises T.
+// T = X_q A_q is needed by every CTA.  The CTAs of a cluster of four share the work: each takes a
+// quarter of K (exact int8 tensor-core MMA per 16-block on the X mantissas already in shared
+// memory, scaled and summed in fp64 in a fixed order), publishes its partial T in its own shared
+// memory, and after a cluster barrier (arrive early, wait just before the rank part) reads the
+// other three through distributed shared memory.  No global atomics, no workspace state.
 #include "lqer_common.cuh"
 
 namespace lqer {
@@ -31,7 +33,9 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kMaxM = 4;
 constexpr int kCg = 4;            // column groups (of 8 columns) per round
 constexpr int kSets = 4;          // slabs a warp keeps in flight (x kCg units each)
-constexpr long long kWaitLimitCycles = 4000000000LL;
+constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q
+constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
+constexpr int kAStageMax = 100 * 1024;   // a CTA's quarter of A_q is staged in shared memory if it fits in this
 
 struct Params {
   const float* X;
@@ -40,10 +44,8 @@ struct Params {
   const uint8_t* bsec;
   const uint8_t* asec;
   DeviceStatus* status;
-  int* tcount;          // CTAs whose T contribution has arrived
-  int* tdone;           // CTAs that no longer need the T accumulator
-  double* tacc;         // [16][k_pad] T accumulator (all zero between calls)
   int M, K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
+  int a_stage_bytes;    // shared memory reserved for staging A_q (0: read it from global memory)
   int a_bits, lr_bits, exp_min, exp_max;
 };
 
@@ -67,54 +69,25 @@ __device__ __forceinline__ uint32_t ld_stream_u8(const void* p) {
   asm volatile("ld.global.nc.L1::no_allocate.u8 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
 }
-__device__ __forceinline__ int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// Read a double from the same shared-memory offset in another CTA of the cluster.
+__device__ __forceinline__ double ld_dsmem_f64(const double* local, uint32_t cta) {
+  uint32_t remote;
+  double v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(cta));
+  asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(remote) : "memory");
   return v;
-}
-
-// The T accumulator is released by every CTA once; the last one leaves it zero for the next call.
-__device__ __noinline__ void release_tacc(const Params& p, int* flags) {
-  const int tid = threadIdx.x, G = gridDim.x;
-  if (tid == 0) flags[1] = (atomicAdd(p.tdone, 1) == G - 1) ? 1 : 0;
-  __syncthreads();
-  if (flags[1] != 0) {
-    __threadfence();
-    for (int o = tid; o < 16 * p.k_pad; o += kThreads) p.tacc[o] = 0.0;
-    if (tid == 0) { *p.tcount = 0; *p.tdone = 0; }
-  }
-}
-
-// T -> T_q as int8 mantissas [M][k_pad] and block scales 2^(e - 6) [M][k_pad / 16] in shared memory.
-__device__ __noinline__ void build_tq(const Params& p, int* flags, int8_t* tq8, float* tqs) {
-  const int tid = threadIdx.x, G = gridDim.x, M = p.M;
-  if (tid == 0) {                                // bounded wait for the contributions of all CTAs
-    const long long t0 = clock64();
-    while (ld_acquire(p.tcount) < G) {
-      __nanosleep(64);
-      if (clock64() - t0 > kWaitLimitCycles) { flags[0] = 1; break; }
-    }
-  }
-  __syncthreads();
-  __threadfence();
-  const int total = M * p.k_pad;                 // 16 adjacent lanes hold one block
-  for (int base = 0; base < total; base += kThreads) {
-    const int idx = base + tid;
-    const bool valid = idx < total;
-    const int row = valid ? idx / p.k_pad : 0, col = valid ? idx % p.k_pad : 0;
-    const double tv = valid ? __ldcg(p.tacc + (size_t)row * p.k_pad + col) : 0.0;
-    double amax = (tv != tv) ? 0.0 : fabs(tv);
-#pragma unroll
-    for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
-    const int e = block_exponent(amax, p.exp_min, p.exp_max);
-    const int qv = quant_mantissa(tv, e, p.a_bits);
-    if (valid) {
-      tq8[row * p.k_pad + col] = (int8_t)qv;
-      if ((col & 15) == 0) tqs[row * (p.k_pad / 16) + (col >> 4)] = pow2f(e - (p.a_bits - 2));
-    }
-  }
-  __syncthreads();
-  release_tacc(p, flags);
 }
 
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
@@ -125,9 +98,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   float* xsc = reinterpret_cast<float*>(xm + (size_t)M * p.K64);    // [M][KB] 2^(e_x - 6)
   int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);          // [M][KB] 8 * sum(x) of the block
   float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // [kWarps][kCg][8][kMaxM]
-  float* tqs = red + kWarps * kCg * 8 * kMaxM;                      // [M][k_pad / 16]
-  int* flags = reinterpret_cast<int*>(tqs + kMaxM * 16);            // [0] a bounded wait ran out, [1] broadcast
-  int8_t* tq8 = reinterpret_cast<int8_t*>(flags + 4);               // [M][k_pad]
+  double* tpart = reinterpret_cast<double*>(red + kWarps * kCg * 8 * kMaxM);   // [M][k_pad] this CTA's partial T
+  double* tsub = tpart + (size_t)kMaxM * p.k_pad;                   // [subsets][M][k_pad] per-warp-subset partials
+  float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * p.k_pad * kMaxSubsets);   // [M][k_pad / 16]
+  int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);        // [M][k_pad]
+  uint8_t* a_stage = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(tq8) + (size_t)kMaxM * (p.k_pad > 0 ? p.k_pad : 16) + 15) & ~(uintptr_t)15);   // staged A_q
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -147,45 +123,45 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   };
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (tid < 4) flags[tid] = 0;
+
+  // this lane's share of (column group cg, rank block warp) of B_q: rank values 4t..4t+3 and the exponent byte
+  auto fetch_rank = [&](uint32_t& wv, uint32_t& eb, int cg) {
+    wv = 0u;
+    eb = 127u;
+    if (cg < cg_hi && warp < p.r_blocks) {
+      const int col = (cg & 15) * 8 + g;
+      const uint8_t* tile = p.bsec + (size_t)(cg >> 4) * ((size_t)p.r_blocks * kTileN * 17);
+      wv = ld_stream_u32(tile + ((size_t)warp * kTileN + col) * 16 + t * 4);
+      eb = ld_stream_u8(tile + (size_t)p.r_blocks * kTileN * 16 + warp * kTileN + col);
+    }
+  };
 
   UnitRegs regs[kSets][kCg];
-  // weights depend on no earlier kernel: request the first slabs before the dependency wait
+  uint32_t rank_w[kCg], rank_e[kCg];
+  // weights depend on no earlier kernel: request the first slabs, the rank blocks and this CTA's
+  // quarter of A_q before the dependency wait
 #pragma unroll
   for (int s = 0; s < kSets; ++s)
 #pragma unroll
     for (int u = 0; u < kCg; ++u) fetch(regs[s][u], cg_lo + u, warp + kWarps * s);
+#pragma unroll
+  for (int u = 0; u < kCg; ++u) fetch_rank(rank_w[u], rank_e[u], cg_lo + u);
+  const int KBr = p.K / 16;
+  const int cs = (int)cluster_nctarank(), cr = (int)cluster_ctarank();
+  const int kb_lo = cr * KBr / cs, kb_hi = (cr + 1) * KBr / cs;      // this CTA's share of K for T
+  const bool a_staged = p.k_pad > 0 && (kb_hi - kb_lo) * p.k_pad * 17 <= p.a_stage_bytes;
+  if (a_staged) {
+    const int mant = (kb_hi - kb_lo) * p.k_pad * 16, ex = (kb_hi - kb_lo) * p.k_pad;
+    const uint8_t* gm = p.asec + (size_t)kb_lo * p.k_pad * 16;
+    const uint8_t* ge = p.asec + (size_t)KBr * p.k_pad * 16 + (size_t)kb_lo * p.k_pad;
+    for (int o = tid * 16; o < mant; o += kThreads * 16)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(a_stage + o)), "l"(gm + o) : "memory");
+    for (int o = tid * 16; o < ex; o += kThreads * 16)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(a_stage + mant + o)), "l"(ge + o) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
 
   asm volatile("griddepcontrol.wait;" ::: "memory");   // X (and the workspace) may be an earlier kernel's output
-
-  // ---- this CTA's share of T = X_q A_q: exact int8 MMA per (16-block of K, 8 rank columns), scaled in
-  //      fp64 and added to the accumulator in the workspace (exact products; their fp64 sum is exact as
-  //      well unless the block exponents of one row spread over more than about 30 binades)
-  if (p.k_pad > 0) {
-    const int KBr = p.K / 16, NT = p.k_pad / 8;
-    const int kb_lo = cta * KBr / G, kb_hi = (cta + 1) * KBr / G;
-    const uint8_t* a_exp = p.asec + (size_t)KBr * p.k_pad * 16;
-    const int bias = -127 - (p.a_bits - 2) - (p.lr_bits - 2);       // exponent bytes carry +127
-    const int items = (kb_hi - kb_lo) * NT;
-    for (int it = warp; it < items; it += kWarps) {
-      const int kb = kb_lo + it / NT, nt = it % NT;
-      const float4 v0 = g < M ? __ldg(reinterpret_cast<const float4*>(p.X + (size_t)g * p.K + kb * 16 + t * 4))
-                              : make_float4(0.f, 0.f, 0.f, 0.f);
-      const uint32_t b0 = __ldg(reinterpret_cast<const uint32_t*>(p.asec + ((size_t)kb * p.k_pad + nt * 8 + g) * 16 + t * 4));
-      const uint32_t ea2 = __ldg(reinterpret_cast<const uint16_t*>(a_exp + (size_t)kb * p.k_pad + nt * 8 + t * 2));
-      int e0;
-      uint32_t m0;
-      uint2 unused;
-      quantize_quad(v0, p.a_bits, p.exp_min, p.exp_max, e0, m0, unused);
-      int c[4];
-      mma_s8(c, m0, 0u, b0);
-      const int tc = nt * 8 + t * 2;
-      if (g < M) {
-        atomicAdd(p.tacc + (size_t)g * p.k_pad + tc, (double)c[0] * pow2d(e0 + (int)(ea2 & 0xFFu) + bias));
-        atomicAdd(p.tacc + (size_t)g * p.k_pad + tc + 1, (double)c[1] * pow2d(e0 + (int)(ea2 >> 8) + bias));
-      }
-    }
-  }
 
   // ---- X -> MXINT8 for the whole contraction: per row the mantissas in the byte order the nibbles
   //      unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales and the offsets 8 * sum(x)
@@ -215,20 +191,62 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       }
     }
   }
+  if (a_staged) asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
-  if (tid == 0 && p.k_pad > 0)                   // the T contributions of this CTA are out (ordered by the barrier)
-    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.tcount) : "memory");
+
+  // ---- this CTA's quarter of T = X_q A_q: exact int8 MMA per (16-block of K, 8 rank columns) on the
+  //      mantissas in shared memory, scaled in fp64.  The products are exact; their fp64 sums are exact
+  //      too unless the block exponents of one row spread over more than about 30 binades, and the
+  //      order of the additions is fixed in any case.
+  if (p.k_pad > 0) {
+    const int NT = p.k_pad / 8;
+    // A_q of blocks kb_lo..kb_hi: staged copy, or global memory
+    const uint8_t* a_mant = a_staged ? a_stage - (size_t)kb_lo * p.k_pad * 16 : p.asec;
+    const uint8_t* a_exp = a_staged ? a_stage + (size_t)(kb_hi - kb_lo) * p.k_pad * 16 - (size_t)kb_lo * p.k_pad
+                                    : p.asec + (size_t)KBr * p.k_pad * 16;
+    const int bias = -127 - (p.lr_bits - 2);                        // exponent bytes carry +127
+    const int tiles_w = NT < kWarps ? NT : kWarps;                  // warps side by side on different rank tiles
+    int subsets = kWarps / tiles_w;                                 // warps that split the K blocks of one tile
+    if (subsets > kMaxSubsets) subsets = kMaxSubsets;
+    const int sb = warp / tiles_w;
+    if (sb < subsets) {
+      for (int nt = warp % tiles_w; nt < NT; nt += tiles_w) {
+        double t0 = 0.0, t1 = 0.0;
+#pragma unroll 4
+        for (int kb = kb_lo + sb; kb < kb_hi; kb += subsets) {
+          // the X mantissas are stored as {0,4,1,5}, {2,6,3,7} within each 8: bring A_q into the same order
+          const uint4 q = *reinterpret_cast<const uint4*>(a_mant + ((size_t)kb * p.k_pad + nt * 8 + g) * 16);
+          const uint32_t lo = (t & 2) ? q.z : q.x, hi = (t & 2) ? q.w : q.y;
+          const uint32_t b0 = (t & 1) ? __byte_perm(lo, hi, 0x7362) : __byte_perm(lo, hi, 0x5140);
+          const uint32_t ea2 = *reinterpret_cast<const uint16_t*>(a_exp + (size_t)kb * p.k_pad + nt * 8 + t * 2);
+          const uint32_t a0 = g < M ? *reinterpret_cast<const uint32_t*>(xm + (size_t)g * p.K64 + kb * 16 + t * 4) : 0u;
+          const double sx = g < M ? (double)xsc[g * KB + kb] : 0.0;
+          int c[4];
+          mma_s8(c, a0, 0u, b0);
+          t0 = fma((double)c[0], sx * pow2d((int)(ea2 & 0xFFu) + bias), t0);
+          t1 = fma((double)c[1], sx * pow2d((int)(ea2 >> 8) + bias), t1);
+        }
+        if (g < M) {
+          tsub[((size_t)sb * kMaxM + g) * p.k_pad + nt * 8 + t * 2] = t0;
+          tsub[((size_t)sb * kMaxM + g) * p.k_pad + nt * 8 + t * 2 + 1] = t1;
+        }
+      }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < M * p.k_pad; idx += kThreads) {
+      const int row = idx / p.k_pad, col = idx % p.k_pad;
+      double v = 0.0;
+      for (int q = 0; q < subsets; ++q) v += tsub[((size_t)q * kMaxM + row) * p.k_pad + col];
+      tpart[row * p.k_pad + col] = v;
+    }
+    __syncthreads();
+    cluster_arrive();                            // this CTA's partial T is published; waited for before the rank part
+  }
 
   bool tq_built = false;
   const int slabs_mine = p.k_slabs > warp ? (p.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
 #pragma unroll 1
   for (int cg0 = cg_lo; cg0 < cg_hi; cg0 += kCg) {
-    if (cg0 != cg_lo) {
-#pragma unroll
-      for (int s = 0; s < kSets; ++s)
-#pragma unroll
-        for (int u = 0; u < kCg; ++u) fetch(regs[s][u], cg0 + u, warp + kWarps * s);
-    }
     float acc[kCg][kMaxM];
 #pragma unroll
     for (int u = 0; u < kCg; ++u)
@@ -261,35 +279,59 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
             }
           }
         }
+        // refill the set: the same groups four slabs on, or - past this warp's last slabs - the
+        // next round's groups from their first slabs, so that rounds follow each other without a bubble
+        const bool more = js + kSets < slabs_mine;
 #pragma unroll
-        for (int u = 0; u < kCg; ++u) fetch(regs[s][u], cg0 + u, j + kWarps * kSets);
+        for (int u = 0; u < kCg; ++u)
+          fetch(regs[s][u], more ? cg0 + u : cg0 + kCg + u, more ? j + kWarps * kSets : warp + kWarps * s);
       }
     }
 
     // ---- B_q against T_q: rank blocks warp, warp + 16, ...
     if (p.k_pad > 0) {
-      if (!tq_built) { build_tq(p, flags, tq8, tqs); tq_built = true; }
+      if (!tq_built) {
+        // T = sum of the cluster's partials (CTA order), then MXINT8 along the rank: 16 adjacent lanes hold one block
+        cluster_wait();
+        const int cs = (int)cluster_nctarank();
+        const int total = M * p.k_pad;
+        for (int base = 0; base < total; base += kThreads) {
+          const int idx = base + tid;
+          const bool valid = idx < total;
+          const int row = valid ? idx / p.k_pad : 0, col = valid ? idx % p.k_pad : 0;
+          double tv = 0.0;
+          if (valid)
+            for (int c = 0; c < cs; ++c) tv += ld_dsmem_f64(tpart + row * p.k_pad + col, (uint32_t)c);
+          double amax = (tv != tv) ? 0.0 : fabs(tv);
+#pragma unroll
+          for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+          const int e = block_exponent(amax, p.exp_min, p.exp_max);
+          const int qv = quant_mantissa(tv, e, p.a_bits);
+          if (valid) {
+            tq8[row * p.k_pad + col] = (int8_t)qv;
+            if ((col & 15) == 0) tqs[row * (p.k_pad / 16) + (col >> 4)] = pow2f(e - (p.a_bits - 2));
+          }
+        }
+        __syncthreads();
+        cluster_arrive();                        // done reading the peers' shared memory
+        tq_built = true;
+      }
       const int rbn = p.k_pad / 16;
-      for (int rb = warp; rb < p.r_blocks; rb += kWarps) {
+      if (warp < p.r_blocks) {                   // rank block `warp` (k <= 256: at most 16 blocks); data already in registers
 #pragma unroll
         for (int u = 0; u < kCg; ++u) {
-          const int cg = cg0 + u;
-          if (cg < cg_hi) {
-            const int col = (cg & 15) * 8 + g;
-            const uint8_t* tile = p.bsec + (size_t)(cg >> 4) * ((size_t)p.r_blocks * kTileN * 17);
-            const uint32_t wv = ld_stream_u32(tile + ((size_t)rb * kTileN + col) * 16 + t * 4);
-            const uint32_t eb = ld_stream_u8(tile + (size_t)p.r_blocks * kTileN * 16 + rb * kTileN + col);
-            const float sb = __uint_as_float((eb - (uint32_t)(p.lr_bits - 2)) << 23);            // 2^(e_b - 6)
+          const float sb = __uint_as_float((rank_e[u] - (uint32_t)(p.lr_bits - 2)) << 23);        // 2^(e_b - 6)
 #pragma unroll
-            for (int r = 0; r < kMaxM; ++r) {
-              if (r < M) {
-                const int tw = *reinterpret_cast<const int*>(tq8 + r * p.k_pad + rb * 16 + t * 4);
-                acc[u][r] = fmaf((float)__dp4a(tw, (int)wv, 0), tqs[r * rbn + rb] * sb, acc[u][r]);
-              }
+          for (int r = 0; r < kMaxM; ++r) {
+            if (r < M) {
+              const int tw = *reinterpret_cast<const int*>(tq8 + r * p.k_pad + warp * 16 + t * 4);
+              acc[u][r] = fmaf((float)__dp4a(tw, (int)rank_w[u], 0), tqs[r * rbn + warp] * sb, acc[u][r]);
             }
           }
         }
       }
+#pragma unroll
+      for (int u = 0; u < kCg; ++u) fetch_rank(rank_w[u], rank_e[u], cg0 + kCg + u);   // the next round's rank blocks
     }
 
     // ---- the four lanes of a column, then the 16 warps (fixed order), then Y
@@ -316,16 +358,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     }
     __syncthreads();                             // red is rewritten by the next round
   }
-  if (p.k_pad > 0 && !tq_built) release_tacc(p, flags);
-  if (flags[0] != 0 && tid == 0) report_error(p.status, LQER_ERR_TIMEOUT, 600, cta);
+  if (p.k_pad > 0) {
+    if (!tq_built) { cluster_wait(); cluster_arrive(); }   // a CTA without columns still serves its partial T
+    cluster_wait();                              // no CTA leaves while its shared memory may still be read
+  }
 }
 
 }  // namespace dcol
 
 static size_t cols_smem_bytes(const PackedMeta& m, int M) {
   using namespace dcol;
-  return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + kWarps * kCg * 8 * kMaxM * 4 + kMaxM * 16 * 4 + 16 +
-         (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
+  return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + kWarps * kCg * 8 * kMaxM * 4 +
+         (size_t)kMaxM * m.k_pad * 8 * (1 + kMaxSubsets) + kMaxM * 16 * 4 + (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
 }
 // The column-owner kernel serves M <= 4 as long as the quantised X of the whole contraction fits in shared memory.
 bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
@@ -349,16 +393,18 @@ cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const
   p.X = X; p.Y = Y;
   p.wsec = base + m.off_w; p.bsec = base + m.off_b; p.asec = base + m.off_a;
   p.status = reinterpret_cast<DeviceStatus*>(ws);
-  p.tcount = reinterpret_cast<int*>(ws + kTCountOffset);
-  p.tdone = reinterpret_cast<int*>(ws + kTDoneOffset);
-  p.tacc = reinterpret_cast<double*>(ws + tacc_offset(m));
   p.M = M; p.K = m.K; p.N = m.N; p.K64 = m.K64; p.k_pad = m.k_pad;
   p.k_slabs = m.k_slabs; p.r_blocks = m.r_blocks;
   p.n_cg = m.N / 8;
   p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
   int G = p.n_cg < sm_count ? p.n_cg : sm_count;
   if (G > kDecodeMaxCtas) G = kDecodeMaxCtas;
-  const size_t smem = cols_smem_bytes(m, M);
+  const int cs = G >= kClusterSize ? kClusterSize : 1;
+  G = G / cs * cs;
+  // stage this CTA's share of A_q in shared memory when it fits beside everything else
+  const size_t a_need = m.k_pad > 0 ? (size_t)((m.K / 16 + cs - 1) / cs) * m.k_pad * 17 + 16 : 0;
+  p.a_stage_bytes = (a_need <= (size_t)kAStageMax && cols_smem_bytes(m, M) + a_need <= 200 * 1024) ? (int)a_need : 0;
+  const size_t smem = cols_smem_bytes(m, M) + p.a_stage_bytes;
   if (!decode_cols_fits(m, M)) return cudaErrorInvalidValue;
 
   cudaLaunchConfig_t cfg = {};
@@ -366,11 +412,26 @@ cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the previous kernel drains
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cs; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
+  if (cs > 1) {
+    // all clusters must be resident at once: the CTAs are sized for one wave
+    static int max_clusters = -1;
+    if (max_clusters < 0) {
+      cudaLaunchConfig_t probe = cfg;
+      probe.dynamicSmemBytes = 200 * 1024;
+      probe.gridDim = dim3(sm_count / cs * cs);
+      int nc = 0;
+      if (cudaOccupancyMaxActiveClusters(&nc, decode_cols_kernel, &probe) != cudaSuccess || nc < 1) nc = 1;
+      max_clusters = nc;
+    }
+    if (G > max_clusters * cs) { G = max_clusters * cs; cfg.gridDim = dim3(G); }
+  }
   LaunchScope scope(kFamDecode, s);
   return cudaLaunchKernelEx(&cfg, decode_cols_kernel, p);
 }
