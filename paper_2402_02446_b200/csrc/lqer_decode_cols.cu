@@ -33,9 +33,9 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kMaxM = 4;
 constexpr int kCg = 4;            // column groups (of 8 columns) per round
 constexpr int kSets = 4;          // slabs a warp keeps in flight (x kCg units each)
-constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q
+constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q (pairs would fill all 148 SMs instead of 132, but the doubled share of T costs more than that gains)
 constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
-constexpr int kAStageMax = 100 * 1024;   // a CTA's quarter of A_q is staged in shared memory if it fits in this
+constexpr int kAStageMax = 100 * 1024;   // a CTA's share of A_q is staged in shared memory if it fits in this
 
 struct Params {
   const float* X;
@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   UnitRegs regs[kSets][kCg];
   uint32_t rank_w[kCg], rank_e[kCg];
   // weights depend on no earlier kernel: request the first slabs, the rank blocks and this CTA's
-  // quarter of A_q before the dependency wait
+  // share of A_q before the dependency wait
 #pragma unroll
   for (int s = 0; s < kSets; ++s)
 #pragma unroll
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   if (a_staged) asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
-  // ---- this CTA's quarter of T = X_q A_q: exact int8 MMA per (16-block of K, 8 rank columns) on the
+  // ---- this CTA's share of T = X_q A_q: exact int8 MMA per (16-block of K, 8 rank columns) on the
   //      mantissas in shared memory, scaled in fp64.  The products are exact; their fp64 sums are exact
   //      too unless the block exponents of one row spread over more than about 30 binades, and the
   //      order of the additions is fixed in any case.

@@ -72,8 +72,9 @@ __device__ __forceinline__ double ld_dsmem_f64(const double* local, uint32_t cta
 
 // PB = 16-blocks of K per step; PB * k_pad <= 1024.  A cluster of CS CTAs shares 16 rows: CTA r
 // takes the K steps s = r, r + CS, ...; the partial T sums meet through distributed shared memory.
-template <int PB>
-__global__ void __launch_bounds__(kThreads, 2) prologue_kernel(const float* __restrict__ X, int M, PackedMeta m,
+// TPW = rank tiles one warp can own (1 for ranks up to 64): fewer accumulators, more CTAs per SM.
+template <int PB, int TPW>
+__global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(const float* __restrict__ X, int M, PackedMeta m,
                                                                const uint8_t* __restrict__ asec,
                                                                uint16_t* __restrict__ xcat,
                                                                int8_t* __restrict__ Tm, uint8_t* __restrict__ Te) {
@@ -96,9 +97,9 @@ __global__ void __launch_bounds__(kThreads, 2) prologue_kernel(const float* __re
   const bool has_rank = m.k > 0;
   const bool active = has_rank && (NT >= 8 || warp < NT * WPN);
 
-  double acc[4][4];
+  double acc[TPW][4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < TPW; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
 
@@ -170,7 +171,7 @@ __global__ void __launch_bounds__(kThreads, 2) prologue_kernel(const float* __re
         const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s_xq[(g + 8) * kXqStride + b * 16 + tig * 4]);
         const int ex0 = s_xe[g][b] + bias, ex1 = s_xe[g + 8][b] + bias;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < TPW; ++i) {
           const int nt = nt0 + 8 * i;
           if (nt < NT) {
             const int j = nt * 8 + g;
@@ -199,7 +200,7 @@ __global__ void __launch_bounds__(kThreads, 2) prologue_kernel(const float* __re
     const int slot = NT >= 8 ? 0 : warp / NT;
     const int nt0 = NT >= 8 ? warp : warp % NT;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < TPW; ++i) {
       const int nt = nt0 + 8 * i;
       if (nt < NT) {
         double* base = tpart + (size_t)slot * n_out;
@@ -246,7 +247,7 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
   return cudaGetLastError();
 }
 
-template <int PB>
+template <int PB, int TPW>
 static cudaError_t launch_prologue_pb(const float* X, int M, const PackedMeta& m, const uint8_t* asec, uint16_t* xc,
                                       int8_t* Tm, uint8_t* Te, cudaStream_t s) {
   const int groups = (M + kRows - 1) / kRows;
@@ -264,7 +265,7 @@ static cudaError_t launch_prologue_pb(const float* X, int M, const PackedMeta& m
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   LaunchScope scope(kFamPrologue, s);
-  return cudaLaunchKernelEx(&cfg, prologue_kernel<PB>, X, M, m, asec, xc, Tm, Te);
+  return cudaLaunchKernelEx(&cfg, prologue_kernel<PB, TPW>, X, M, m, asec, xc, Tm, Te);
 }
 
 cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
@@ -272,9 +273,9 @@ cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const vo
   (void)st;
   const uint8_t* asec = static_cast<const uint8_t*>(packed) + m.off_a;
   uint16_t* xc = static_cast<uint16_t*>(xcat);
-  if (m.k_pad <= 64) return launch_prologue_pb<16>(X, M, m, asec, xc, Tm, Te, s);
-  if (m.k_pad <= 128) return launch_prologue_pb<8>(X, M, m, asec, xc, Tm, Te, s);
-  return launch_prologue_pb<4>(X, M, m, asec, xc, Tm, Te, s);
+  if (m.k_pad <= 64) return launch_prologue_pb<16, 1>(X, M, m, asec, xc, Tm, Te, s);
+  if (m.k_pad <= 128) return launch_prologue_pb<8, 2>(X, M, m, asec, xc, Tm, Te, s);
+  return launch_prologue_pb<4, 4>(X, M, m, asec, xc, Tm, Te, s);
 }
 
 }  // namespace lqer
