@@ -182,6 +182,21 @@ def run_reference(args) -> None:
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of per-rank timings over all ranks (the job is as slow as its slowest rank);
+    the values themselves when the job has one rank (dist is None)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_value(flops_per_rank_step: float, ms_per_step: float, world: int) -> float:
+    """TFLOP/s of the whole job: every rank runs its own replica of the step (weak scaling)."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------------------------ GPU arm
 def run_ours(args) -> None:
     import paper_2402_02446_b200 as L
@@ -268,16 +283,11 @@ def run_ours(args) -> None:
     total_ms = t_start.elapsed_time(t_stop)
     decode_ms = [e0.elapsed_time(e1) for e0, e1, _ in ev]
     prefill_ms = [e1.elapsed_time(e2) for _, e1, e2 in ev]
-    if dist is not None:
-        t = torch.tensor([total_ms, statistics.median(decode_ms), statistics.median(prefill_ms)], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, dec_ms, pre_ms = (float(v) for v in t.tolist())
-    else:
-        dec_ms, pre_ms = statistics.median(decode_ms), statistics.median(prefill_ms)
+    total_ms, dec_ms, pre_ms = max_over_ranks([total_ms, statistics.median(decode_ms), statistics.median(prefill_ms)], dist, dev)
     if L.poll_status(ws) != 0:
         raise SystemExit("device-side error during the timed region")
     ms_per_step = total_ms / args.steps
-    value = world * (flops_decode + flops_prefill) / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_value(flops_decode + flops_prefill, ms_per_step, world)
 
     # ---- roofline of the dominant kernel: one more step with an event pair around every launch
     peaks = measured_peaks()
@@ -328,10 +338,7 @@ def run_ours(args) -> None:
             e2e_step()
         barrier()
         e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
-        if dist is not None:
-            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        (e_ms,) = max_over_ranks([e_ms], dist, dev)
         h2d = sum(4 * (M_DECODE + M_PREFILL) * K for K, _, _, _ in shapes)
         d2h = sum(4 * (M_DECODE + M_PREFILL) * N for _, N, _, _ in shapes)
         e2e = {"value": world * (flops_decode + flops_prefill) / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
@@ -377,7 +384,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--layers", type=int, default=32, help="decoder layers of the stack (32 = the full workload)")
-    ap.add_argument("--oracle-rows", type=int, default=128, help="token rows of the oracle's bounded sample")
+    ap.add_argument("--oracle-rows", type=int, default=2048, help="token rows of the oracle's bounded sample")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

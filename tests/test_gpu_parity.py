@@ -206,3 +206,62 @@ def test_linear_decode_full_size(M):
     assert L.poll_status(ws) == 0
     assert worst_ratio(Y, ref) <= 1.0
     Pg.release()
+
+
+# ---------------------------------------------------------------------------- full-size layers, sampled rows
+def _random_factor_layer(spec):
+    """Full-size layer with seeded stand-in factors (the factors are inputs of the layer; deriving them by
+    SVD at this size would take minutes on the host)."""
+    W = gen.make_weight(spec)
+    A, B = gen.make_random_factors(spec)
+    P = olqer.prepare_weights(W, A, B)
+    Pg = L.prepare_weights(_t(W), _t(A), _t(B))
+    return P, Pg
+
+
+FULL_SPECS = [
+    gen.config_prefill(False),                       # M=2048, 4096 x 11008, rank 32
+    gen.config_prefill(True),                        # M=2048, 11008 x 4096
+    gen.config_sweep(13824, 512, 128),               # 13B-shaped: K=5120, N=13824, M=512, rank 128, Student-t weights
+    gen.config_sweep(5120, 64, 256),                 # M=64, rank 256
+]
+
+
+@pytest.mark.parametrize("spec", FULL_SPECS, ids=lambda s: s.name)
+def test_linear_full_size_sampled_rows(spec):
+    # Rows of Y depend only on the same rows of X, so the oracle computes a seeded sample of rows that
+    # touches every 128-row tile (and the first and last row); the GPU runs the whole layer as bench.py does.
+    P, Pg = _random_factor_layer(spec)
+    X = gen.make_activations(spec)
+    g = np.random.default_rng(spec.seed)
+    rows = sorted({0, spec.M - 1} | {int(t * 128 + g.integers(0, 128)) for t in range((spec.M + 127) // 128) if t * 128 + 127 < spec.M})
+    ref = olqer.forward(X[rows], P)
+    ws = L.new_workspace(spec.M, Pg)
+    Y = L.linear(_t(X), Pg, ws)
+    assert L.poll_status(ws) == 0
+    Ys = Y[torch.tensor(rows, device=DEV)].cpu().numpy()
+    assert worst_ratio(Ys, ref) <= 1.0
+    Pg.release()
+
+
+def test_stack_linears_batched_decode_and_prefill():
+    # the q, gate and down linears of one decoder layer of the 7B stack through lqer_linear_batched on one
+    # workspace: M = 1 (decode kernels) and then M = 2048 (prologue + GEMM), as bench.py runs them
+    specs = [gen.config_stack(0, w, 2048) for w in (0, 4, 6)]
+    layers = [_random_factor_layer(s) for s in specs]
+    X1 = [gen.make_activations(s, M=1) for s in specs]
+    X2 = [gen.make_activations(s, M=2048) for s in specs]
+    rows = [0, 777, 2047]
+    n = max(L.workspace_bytes(2048, s.K, s.N, s.k) for s in specs)
+    ws = torch.zeros(n, dtype=torch.uint8, device=DEV)
+    Y1 = [torch.empty((1, s.N), dtype=torch.float32, device=DEV) for s in specs]
+    Y2 = [torch.empty((2048, s.N), dtype=torch.float32, device=DEV) for s in specs]
+    L.linear_batched([(_t(x), lay[1], y) for x, lay, y in zip(X1, layers, Y1)], ws)
+    L.linear_batched([(_t(x), lay[1], y) for x, lay, y in zip(X2, layers, Y2)], ws)
+    torch.cuda.synchronize()
+    assert L.poll_status(ws) == 0
+    for s, lay, x1, x2, y1, y2 in zip(specs, layers, X1, X2, Y1, Y2):
+        assert worst_ratio(y1.cpu().numpy(), olqer.forward(x1, lay[0])) <= 1.0, s.name
+        assert worst_ratio(y2[torch.tensor(rows, device=DEV)].cpu().numpy(), olqer.forward(x2[rows], lay[0])) <= 1.0, s.name
+    for lay in layers:
+        lay[1].release()
