@@ -9,7 +9,7 @@
 //   warp 0      TMA producer (own activation tile + own packed weight half)
 //   warp 1      tensor memory allocation; in CTA 0 also the MMA issuer
 //   warps 2-5   epilogue (tcgen05.ld of the finished accumulator, fp32 stores to Y)
-//   warps 6-21  converters in four groups; a group converts every fourth stage (one weight
+//   warps 6-29  converters in six groups; a group converts every sixth stage (one weight
 //               column = 64 weights per thread), so that its fixed per-stage latencies
 //               (barrier wait, shared-memory round trip, proxy fence) overlap the other groups
 // One ring of six stages; a stage holds the activation tile, the packed weight tile and the
@@ -39,12 +39,15 @@ constexpr int STAGE_BYTES = 37 * 1024;
 constexpr int RANK_PER_STAGE = 32;
 constexpr int NUM_BARRIERS = 3 * STAGES + 4;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;
-constexpr int CONVERTER_WARPS = 16;
-constexpr int CONVERTER_GROUPS = 4;          // group g converts the stages with index = g (mod 4)
+constexpr int CONVERTER_WARPS = 24;
+constexpr int CONVERTER_GROUPS = 6;          // group g converts the stages with index = g (mod 6): with six ring
+                                             // slots a group meets one slot only, exactly one pass apart, so
+                                             // the parity of its wait can never alias an older pass
 constexpr int WARPS_PER_GROUP = CONVERTER_WARPS / CONVERTER_GROUPS;
 constexpr int NUM_THREADS = (6 + CONVERTER_WARPS) * 32;
 static_assert(PK_OFFSET + kWTileBytes <= STAGE_BYTES && STAGE_BYTES % 1024 == 0, "stage layout");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+static_assert(STAGES % CONVERTER_GROUPS == 0, "a converter group must revisit a ring slot exactly one pass later");
 
 struct Params {
   const uint8_t* wsec;
@@ -206,7 +209,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
     }
   } else {
     // ------------------------------------------------------------------ converters (own weight half)
-    const int c = threadIdx.x - 6 * 32;          // 0..511
+    const int c = threadIdx.x - 6 * 32;          // 0..767
     const int group = c >> 7, nl = c & 127;      // stage group; weight column of the half tile
     const int sw = nl & 7;
     uint32_t chunk[8];                           // the row's eight 16-byte chunks after the 128-byte swizzle
