@@ -170,7 +170,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
 lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, float* Y_host,
                                void* workspace, size_t workspace_bytes, void* stream);
 
-/* Zero the head of a fresh workspace (status area, counters, accumulator; at most 164096 bytes;
+/* Zero the head of a fresh workspace (status area, counters, accumulator; at most 166144 bytes;
  * asynchronous on `stream`).  Call once after allocating the workspace and again after
  * lqer_poll_status reported a device-side error (an interrupted call may leave counters behind). */
 lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
@@ -180,8 +180,9 @@ lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_
 
 /* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 decode kernels
  * (column-owner kernel for M <= 4, split-K kernel for M <= 16), 3 tensor-core kernel (one CTA per
- * tile), 4 tensor-core kernel (CTA pair per tile), 5 split-K decode kernel for every M <= 16.
- * Host only, process wide. */
+ * tile), 4 tensor-core kernel (CTA pair per tile), 5 split-K decode kernel for every M <= 16,
+ * 6 as 4 with the tensor-core activation prologue at every batch size (ranks up to 64; by default
+ * it serves M >= 1024, and paths 1 and 3 never use it).  Host only, process wide. */
 lqer_status_t lqer_set_path(int path);
 
 /* Number of kernels launched by the library in this process so far (host). */

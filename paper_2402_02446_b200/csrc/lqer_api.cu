@@ -116,11 +116,12 @@ static lqer_status_t check_arch() {
 static size_t xcat_bytes(const PackedMeta& m, int M) { return align_up((size_t)M * xcat_cols(m) * 2, 256); }
 // Bytes a call with M rows needs: the persistent head plus the scratch of the path it takes.
 static size_t call_bytes(const PackedMeta& m, int M, bool decode) {
-  return align_up(persist_bytes(m), 256) + (decode ? decode_scratch_bytes(m) : xcat_bytes(m, M));
+  return align_up(persist_bytes(m), 256) +
+         (decode ? decode_scratch_bytes(m) : xcat_bytes(m, M) + prologue_tc_scratch_bytes(m, M));
 }
 // Bytes that fit every call of up to M_max rows, whichever path it takes.
 static size_t workspace_total(const PackedMeta& m, int M_max) {
-  const size_t a = xcat_bytes(m, M_max), b = decode_scratch_bytes(m);
+  const size_t a = xcat_bytes(m, M_max) + prologue_tc_scratch_bound(m, M_max), b = decode_scratch_bytes(m);
   return align_up(persist_bytes(m), 256) + (a > b ? a : b);
 }
 
@@ -134,6 +135,9 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
   lqer_status_t st = lookup(packed, m);
   if (st != LQER_OK) return st;
   int path = g_path.load();
+  // Paths 1 and 3 keep the SIMT-style prologue at every batch size; the others take the tensor-core one where it fits.
+  const bool tc_prologue = path != 1 && path != 3 && prologue_tc_fits(m, M, X, path == 6);
+  if (path == 6) path = 4;
   if (project_only) path = 3;
   if (path == 0 && M <= decode_max_m()) path = 2;
   const bool decode = path == 2 || path == 5;
@@ -147,7 +151,11 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
     err = launch_decode(X, M, m, packed, Y, workspace, s, path == 5);
   } else {
     if (path == 1 && M > 65535) return LQER_ERR_SHAPE;
-    err = launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
+    uint8_t* wsb = static_cast<uint8_t*>(workspace);
+    err = tc_prologue ? launch_prologue_tc(X, M, m, packed, xcat, Tm, Te, dst,
+                                           reinterpret_cast<double*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M)),
+                                           reinterpret_cast<int*>(wsb + pcount_offset(m)), s)
+                      : launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
       err = (path == 1)   ? launch_gemm_simt(xcat, M, m, packed, Y, s)
             : (path == 4 || (path == 0 && M > 128)) ? launch_gemm_tc2(xcat, M, m, packed, Y, dst, s)
@@ -381,7 +389,7 @@ lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_
 }
 
 lqer_status_t lqer_set_path(int path) {
-  if (path < 0 || path > 5) return LQER_ERR_CONFIG;
+  if (path < 0 || path > 6) return LQER_ERR_CONFIG;
   g_path.store(path);
   return LQER_OK;
 }

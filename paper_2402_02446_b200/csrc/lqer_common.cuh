@@ -52,17 +52,43 @@ inline uint32_t meta_checksum(const PackedMeta& m) {
 
 // Workspace layout: a persistent head that is all zero between calls
 //   [0, 256)   status area: DeviceStatus, the decode kernel's two T counters
-//   [256, ..)  per-column-tile arrival counters of the decode kernel, then its fp64 T accumulator
-// followed by per-call scratch: Xcat (bf16 [M, K64 + k_pad]) for the GEMM path, or the partial-sum
-// slots of the decode path.
+//   [256, ..)  per-column-tile arrival counters of the decode kernel, its fp64 T accumulator, then the
+//              per-row-tile arrival counters of the tensor-core prologue
+// followed by per-call scratch: Xcat (bf16 [M, K64 + k_pad]) and the fp64 partial sums of the tensor-core
+// prologue for the GEMM path, or the partial-sum slots of the decode path.
 constexpr int kTCountOffset = 64, kTDoneOffset = 68;
 constexpr int kDecodeMaxCtas = 160;
-constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8;
+constexpr int kPrologueRowTiles = 512;               // arrival counters: batches up to 65536 rows
+constexpr int kPrologueMaxCtas = 148;
+constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8 + kPrologueRowTiles * 4;
 __host__ __device__ inline size_t tacc_offset(const PackedMeta& m) {
   return (size_t)kStatusBytes + (((size_t)m.n_tiles * 4 + 255) & ~(size_t)255);
 }
-__host__ __device__ inline size_t persist_bytes(const PackedMeta& m) {
+__host__ __device__ inline size_t pcount_offset(const PackedMeta& m) {
   return tacc_offset(m) + (size_t)16 * m.k_pad * 8;
+}
+__host__ __device__ inline size_t persist_bytes(const PackedMeta& m) {
+  return pcount_offset(m) + (size_t)kPrologueRowTiles * 4;
+}
+// Tensor-core prologue: a CTA owns 128 rows and one of `splits` ranges of K (in panels of 128 columns);
+// each CTA leaves a [128, k_pad] fp64 partial sum for the last CTA of its row tile to add up.
+inline bool prologue_tc_rank_ok(const PackedMeta& m) { return m.k > 0 && (m.k_pad == 16 || m.k_pad == 32 || m.k_pad == 64); }
+inline int prologue_tc_splits(const PackedMeta& m, int M) {
+  const int row_tiles = (M + 127) / 128, panels = (m.K64 + 127) / 128;
+  int s = kPrologueMaxCtas / row_tiles;
+  if (s > panels) s = panels;
+  return s < 1 ? 1 : s;
+}
+// Upper bound of prologue_tc_scratch_bytes over every batch of up to M_max rows.
+inline size_t prologue_tc_scratch_bound(const PackedMeta& m, int M_max) {
+  if (!prologue_tc_rank_ok(m)) return 0;
+  long long ctas = (long long)((M_max + 127) / 128) * ((m.K64 + 127) / 128);
+  if (ctas > kPrologueMaxCtas) ctas = kPrologueMaxCtas;
+  return (size_t)ctas * 128 * m.k_pad * 8;
+}
+inline size_t prologue_tc_scratch_bytes(const PackedMeta& m, int M) {
+  if (!prologue_tc_rank_ok(m) || (M + 127) / 128 > kPrologueRowTiles) return 0;
+  return (size_t)((M + 127) / 128) * prologue_tc_splits(m, M) * 128 * m.k_pad * 8;
 }
 __host__ __device__ inline int decode_units(const PackedMeta& m) {
   return m.n_tiles * (m.k_slabs + (m.r_blocks + 1) / 2);
@@ -120,26 +146,31 @@ __device__ __forceinline__ uint32_t bf16_bits_of(int m, int p) {
 // Quantise the four values a lane holds; the 16-block is spread over 4 adjacent lanes.
 // Returns the four int8 mantissas packed in one word and the four exact bf16 values
 // m * 2^(e - (bits-2)) packed in two words.
-__device__ __forceinline__ void quantize_quad(const float4 v, int bits, int emin, int emax, int& e, uint32_t& m8,
+__device__ __forceinline__ void quantize_quad(const float4 vin, int bits, int emin, int emax, int& e, uint32_t& m8,
                                               uint2& bf) {
-  float amax = fmaxf(fmaxf(abs_ignore_nan(v.x), abs_ignore_nan(v.y)), fmaxf(abs_ignore_nan(v.z), abs_ignore_nan(v.w)));
+  // NaN counts as zero, as a value and in the block maximum
+  const float v[4] = {(vin.x == vin.x) ? vin.x : 0.0f, (vin.y == vin.y) ? vin.y : 0.0f,
+                      (vin.z == vin.z) ? vin.z : 0.0f, (vin.w == vin.w) ? vin.w : 0.0f};
+  float amax = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
   e = block_exponent(amax, emin, emax);
   const float qmax = (float)((1 << (bits - 1)) - 1);
   const float inv_step = pow2f((bits - 2) - e), step = pow2f(e - (bits - 2));
-  const float in[4] = {v.x, v.y, v.z, v.w};
+  // Adding 1.5 * 2^23 rounds a value of magnitude below 2^22 to an integer, half to even, and leaves
+  // that integer (two's complement) in the low bits of the sum; (sum - 1.5 * 2^23) * step is exact.
+  const float kMagic = 12582912.0f;
+  const float back = -kMagic * step;
+  uint32_t rb[4];
   float r[4];
-  int q[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    float t = fminf(fmaxf(in[i] * inv_step, -qmax), qmax);   // exact scaling, clamp (+-inf saturate)
-    t = rintf(t);                                            // round half to even
-    r[i] = (in[i] != in[i]) ? 0.0f : t;                      // NaN -> 0
-    q[i] = (int)r[i];
-    r[i] *= step;                                            // exact: at most 7 significant bits
+    const float t = fminf(fmaxf(v[i] * inv_step, -qmax), qmax);   // exact scaling, clamp (+-inf saturate)
+    const float s = t + kMagic;
+    rb[i] = __float_as_uint(s);
+    r[i] = fmaf(s, step, back);                                    // exact: at most 7 significant bits
   }
-  m8 = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
+  m8 = __byte_perm(__byte_perm(rb[0], rb[1], 0x0040), __byte_perm(rb[2], rb[3], 0x0040), 0x5410);
   bf.x = __byte_perm(__float_as_uint(r[0]), __float_as_uint(r[1]), 0x7632);
   bf.y = __byte_perm(__float_as_uint(r[2]), __float_as_uint(r[3]), 0x7632);
 }
@@ -194,6 +225,12 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
 // optional int8 / exponent exports of T_q.
 cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s);
+// The same prologue with the projection on the tcgen05 int8 tensor cores: ranks up to 64, large batches.
+bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch);
+// `partials`: prologue_tc_scratch_bytes(m, M) of scratch; `counters`: the zeroed per-row-tile counters of the workspace head.
+cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
+                               int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
+                               cudaStream_t s);
 cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                              cudaStream_t s);
 cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,

@@ -1,0 +1,492 @@
+// Activation prologue of the prefill path for large batches, with the projection on the
+// 5th-generation tensor cores (paper Section 4.1: X_q in MXINT8, blocks [1,16]; Section 3.1:
+// the small high-precision product X A_k).
+//
+// Same results as prologue_kernel (bit for bit in X_q and T_q); what differs is where the work
+// runs.  A CTA owns 128 rows of X and one of `splits` ranges of K; the CTAs of a row tile leave
+// fp64 partial sums in global scratch and the last one to arrive adds them in a fixed order.
+//   scalers      read the int32 block products from tensor memory, scale each by 2^(e_x + e_a)
+//                and sum in fp64 (exact for any realistic exponent spread)
+//   quantisers   take fp32 X from a shared-memory ring that TMA fills, write the exact bf16
+//                values m * 2^(e-6) to Xcat, the int8 mantissas to shared memory in the K-major
+//                128-byte-swizzled layout the MMA reads, and the block exponents beside them
+//   panel warp   A_q panels: 16-byte asynchronous copies into a block-diagonal operand
+//   issuer warp  one lane issues tcgen05.mma kind::i8 (M=128, N=2*k_pad, K=32)
+//   TMA warp     one lane keeps the fp32 ring full (128 rows x 64 columns per stage)
+// Each 16-block needs its own integer product, because its scale differs from its neighbour's.
+// The int8 MMA contracts 32 values, so the B operand of a block pair is laid out as
+//     rows 0..k_pad-1:        [A_b | 0]        rows k_pad..2 k_pad-1:  [0 | A_{b+1}]
+// and one MMA yields X_b A_b in the first k_pad accumulator columns and X_{b+1} A_{b+1} in the
+// next k_pad.  The zero halves are written once; only the diagonal chunks change per panel.
+#include "lqer_tc_ptx.cuh"
+
+namespace lqer {
+namespace ptc {
+
+using namespace tc;
+
+constexpr int ROWS = 128;                    // rows of X per CTA = one MMA M tile
+constexpr int STAGE_COLS = 64;               // columns of X per stage: 4 blocks = 2 block pairs
+constexpr int RAW_SLOTS = 4;                 // fp32 ring
+constexpr int RAW_BYTES = ROWS * STAGE_COLS * 4;   // 32768
+constexpr int X_SLOTS = 4;                   // int8 ring of stages; two stages share one 128-byte-row buffer
+constexpr int XBUF_BYTES = ROWS * 128;       // 16384: 128 rows x 128 int8 (8 blocks), swizzled
+constexpr int PANELS = 3;                    // ring of A_q panels (8 blocks each)
+constexpr int WORK_WARPS = 24;               // scalers + quantisers
+constexpr int NUM_WARPS = WORK_WARPS + 3;
+constexpr int NUM_THREADS = NUM_WARPS * 32;  // 864
+constexpr int MAX_TMEM_SLOTS = 8;
+
+template <int KP>
+struct Cfg {
+  static constexpr int SCALER_WARPS = KP > 32 ? 16 : 8;      // four lane quarters x column groups
+  static constexpr int QUANT_WARPS = WORK_WARPS - SCALER_WARPS;
+  static constexpr int CPW = KP / (SCALER_WARPS / 4);        // rank columns per scaler warp
+  static constexpr int ROW_STEP = QUANT_WARPS * 2;           // rows one pass of the quantisers covers
+  static constexpr int QUADS = ROWS / ROW_STEP;              // float4 per quantiser per stage
+  static constexpr int SLOT_COLS = 2 * KP;                   // accumulator columns per block pair
+  static constexpr int TMEM_SLOTS = (512 / SLOT_COLS) < MAX_TMEM_SLOTS ? (512 / SLOT_COLS) : MAX_TMEM_SLOTS;
+  static constexpr int TMEM_COLS = 512;
+  // With 8 scaler and 16 quantiser warps (whole warpgroups each) the quantisers hand 8 registers per thread to the
+  // scalers: 8 x 88 + 16 x 64 + 3 x 72 registers per lane = the 27 x 72 the CTA was launched with.
+  static constexpr bool REG_SHIFT = SCALER_WARPS == 8;
+  static constexpr int PANEL_BYTES = 2 * KP * 128;           // 2 k_pad rows x 128 bytes
+  static constexpr int OFF_XQ = RAW_SLOTS * RAW_BYTES;
+  static constexpr int OFF_PANEL = OFF_XQ + (X_SLOTS / 2) * XBUF_BYTES;
+  static constexpr int OFF_XE = OFF_PANEL + PANELS * PANEL_BYTES;   // [X_SLOTS][ROWS][4] block exponents
+  static constexpr int OFF_HIA = OFF_XE + X_SLOTS * ROWS * 4;       // [PANELS][8][KP] high words of 2^(e_a + bias)
+  static constexpr int OFF_BARS = OFF_HIA + PANELS * 8 * KP * 4;
+  static constexpr int NUM_BARS = 2 * RAW_SLOTS + 2 * X_SLOTS + 2 * PANELS + 2 * MAX_TMEM_SLOTS;
+  static constexpr int SMEM_BYTES = OFF_BARS + NUM_BARS * 8 + 16 + 1024;
+  static_assert(CPW % 8 == 0 && CPW <= 16, "scaler registers");
+  static_assert(ROWS % ROW_STEP == 0, "quantiser passes");
+  static_assert(PANEL_BYTES % 1024 == 0, "swizzle atoms need 1024-byte bases");
+  static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+};
+
+struct Params {
+  const uint8_t* asec;      // A_q section of the packed buffer: mantissas then exponents
+  uint16_t* xcat;
+  int8_t* Tm;               // optional exports of T_q
+  uint8_t* Te;
+  DeviceStatus* status;
+  double* partials;         // [row tile][split][128][k_pad]
+  int* counters;            // [row tile], zero between calls
+  int M, K, K64;
+  int kblocks;              // K / 16
+  int panels;               // ceil(K64 / 128)
+  int splits;               // CTAs per row tile
+  int a_bits, lr_bits, exp_min, exp_max;
+  size_t ldx;               // columns of Xcat
+};
+
+// int8 x int8 -> int32, both operands K-major, M = m, N = n.
+__host__ __device__ constexpr uint32_t make_idesc_i8(int m, int n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+// D = A B (the accumulator is overwritten).
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, 0, 0;\n tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// try_wait with a suspend-time hint: the hardware parks the thread until the phase completes or the hint
+// (nanoseconds) runs out, so a waiting role takes few issue slots from the working ones.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
+  return ok != 0;
+}
+// Bounded like tc::mbar_wait: gives up after WAIT_LIMIT_CYCLES or as soon as another role has given up.
+__device__ __forceinline__ bool parked_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_parked(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait_parked(bar, parity)) {
+    if (*abort_flag != 0) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+  }
+  return true;
+}
+// A wait whose outcome every lane of the warp shares (the code after it shuffles or touches tensor memory as a warp).
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return __all_sync(0xFFFFFFFFu, parked_wait(bar, parity, abort_flag)) != 0;
+}
+
+template <int KP>
+__global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
+  using C = Cfg<KP>;
+  constexpr int SW = C::SCALER_WARPS, QW = C::QUANT_WARPS, CPW = C::CPW, QUADS = C::QUADS;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* raw_base = smem;
+  uint8_t* xq_base = smem + C::OFF_XQ;
+  uint8_t* panel_base = smem + C::OFF_PANEL;
+  int8_t* s_xe = reinterpret_cast<int8_t*>(smem + C::OFF_XE);
+  int* s_hia = reinterpret_cast<int*>(smem + C::OFF_HIA);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BARS);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* last_flag = reinterpret_cast<int*>(tmem_slot + 2);
+
+  const uint32_t bar0 = smem_u32(bars);
+  auto raw_full = [&](int s) { return bar0 + 8u * s; };
+  auto raw_empty = [&](int s) { return bar0 + 8u * (RAW_SLOTS + s); };
+  auto xq_full = [&](int s) { return bar0 + 8u * (2 * RAW_SLOTS + s); };
+  auto xq_empty = [&](int s) { return bar0 + 8u * (2 * RAW_SLOTS + X_SLOTS + s); };
+  auto panel_full = [&](int s) { return bar0 + 8u * (2 * RAW_SLOTS + 2 * X_SLOTS + s); };
+  auto panel_empty = [&](int s) { return bar0 + 8u * (2 * RAW_SLOTS + 2 * X_SLOTS + PANELS + s); };
+  auto slot_full = [&](int s) { return bar0 + 8u * (2 * RAW_SLOTS + 2 * X_SLOTS + 2 * PANELS + s); };
+  auto slot_empty = [&](int s) { return bar0 + 8u * (2 * RAW_SLOTS + 2 * X_SLOTS + 2 * PANELS + MAX_TMEM_SLOTS + s); };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row_tile = blockIdx.x / p.splits, split = blockIdx.x % p.splits;
+  const int row0 = row_tile * ROWS;
+  const int pan_lo = (int)((long long)split * p.panels / p.splits);
+  const int pan_hi = (int)((long long)(split + 1) * p.panels / p.splits);
+  const int n_stages = 2 * (pan_hi - pan_lo);
+  const uint8_t* a_exp = p.asec + (size_t)p.kblocks * KP * 16;
+
+  // zero halves of the block-diagonal panels (never written again)
+  for (int i = tid; i < PANELS * C::PANEL_BYTES / 16; i += NUM_THREADS)
+    reinterpret_cast<uint4*>(panel_base)[i] = make_uint4(0u, 0u, 0u, 0u);
+  if (tid == 0) {
+    for (int s = 0; s < RAW_SLOTS; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), QW); }
+    for (int s = 0; s < X_SLOTS; ++s) { mbar_init(xq_full(s), QW); mbar_init(xq_empty(s), SW + 1); }
+    for (int s = 0; s < PANELS; ++s) { mbar_init(panel_full(s), 1); mbar_init(panel_empty(s), SW + 1); }
+    for (int s = 0; s < MAX_TMEM_SLOTS; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), SW); }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  fence_proxy_async_smem();
+  if (warp == WORK_WARPS + 1) tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp < SW) {
+    // ------------------------------------------------------------------ scalers
+    if (C::REG_SHIFT) asm volatile("setmaxnreg.inc.sync.aligned.u32 88;" ::: "memory");   // registers the quantisers gave up
+    const int q = warp & 3, h = warp >> 2;
+    const int row = q * 32 + lane;
+    double acc[CPW];
+#pragma unroll
+    for (int i = 0; i < CPW; ++i) acc[i] = 0.0;
+    bool ok = true;
+    for (int s = 0; s < n_stages && ok; ++s) {
+      const int xs = s % X_SLOTS, pp = s >> 1, pb = pp % PANELS;
+      if ((s & 1) == 0 && !warp_wait(panel_full(pb), (pp / PANELS) & 1, abort_flag)) { ok = false; break; }
+      if (!warp_wait(xq_full(xs), (s / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
+      const uint32_t e4 = *reinterpret_cast<const uint32_t*>(s_xe + (xs * ROWS + row) * 4);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(xq_empty(xs));
+      const int* hia = s_hia + (pb * 8 + (s & 1) * 4) * KP;
+#pragma unroll 1
+      for (int j = 0; j < 2; ++j) {
+        const int u = 2 * s + j, slot = u % C::TMEM_SLOTS;
+        if (!warp_wait(slot_full(slot), (u / C::TMEM_SLOTS) & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk) {
+          const int bi = 2 * j + blk;                                   // block within the stage
+          const int ehi = (int)(int8_t)(e4 >> (8 * bi)) * (1 << 20);
+          const int* hrow = hia + bi * KP + h * CPW;
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + slot * C::SLOT_COLS + blk * KP + h * CPW;
+          const double kMagic = 4503601774854144.0;                     // 2^52 + 2^31
+#pragma unroll
+          for (int g8 = 0; g8 < CPW / 8; ++g8) {                        // eight columns at a time keeps the registers few
+            uint32_t c[8];
+            tmem_ld8(taddr + g8 * 8, c);
+            tmem_ld_wait();
+            if (blk == 1 && g8 == CPW / 8 - 1) {                        // the whole slot has been read
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(slot_empty(slot));
+            }
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+              const int4 hv = *reinterpret_cast<const int4*>(hrow + g8 * 8 + 4 * g);
+              double* a = acc + g8 * 8 + 4 * g;
+              // int32 -> fp64 without the conversion unit: 2^52 + 2^31 + c has the bits (0x43300000, c ^ 2^31)
+              a[0] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 0] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.x + ehi, 0), a[0]);
+              a[1] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 1] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.y + ehi, 0), a[1]);
+              a[2] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 2] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.z + ehi, 0), a[2]);
+              a[3] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 3] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.w + ehi, 0), a[3]);
+            }
+          }
+        }
+      }
+      if (ok && (s & 1)) {                                              // done with the panel's exponent table
+        __syncwarp();
+        if (lane == 0) mbar_arrive(panel_empty(pb));
+      }
+    }
+    // partial sums of this CTA's K range -> global scratch
+    double* dst = p.partials + ((size_t)blockIdx.x * ROWS + row) * KP + h * CPW;
+#pragma unroll
+    for (int i = 0; i < CPW; i += 2) *reinterpret_cast<double2*>(dst + i) = make_double2(acc[i], acc[i + 1]);
+  } else if (warp < WORK_WARPS) {
+    // ------------------------------------------------------------------ quantisers
+    if (C::REG_SHIFT) asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
+    const int tq = tid - SW * 32;
+    const int c4 = tq & 15, rb = tq >> 4;            // float4 within the 64-column stage; first row (then + ROW_STEP per quad)
+    const int col0 = pan_lo * 2 * STAGE_COLS + c4 * 4;
+    uint16_t* cp = p.xcat + (size_t)(row0 + rb) * p.ldx + col0;
+    const size_t c_step = (size_t)C::ROW_STEP * p.ldx;
+    const int rows_ok = p.M - (row0 + rb);            // quad i is a real row while ROW_STEP * i < rows_ok
+    const uint32_t off_row = (uint32_t)(rb * 128 + (c4 & 3) * 4);
+    int8_t* xe_dst = s_xe + rb * 4 + (c4 >> 2);
+    const bool xe_writer = (c4 & 3) == 0;
+    bool ok = true;
+    for (int s = 0; s < n_stages && ok; ++s) {
+      const int rs = s % RAW_SLOTS, xs = s % X_SLOTS;
+      if (!warp_wait(raw_full(rs), (s / RAW_SLOTS) & 1, abort_flag)) { ok = false; break; }
+      const float4* src = reinterpret_cast<const float4*>(raw_base + rs * RAW_BYTES) + rb * 16 + c4;
+      float4 xr[QUADS];
+#pragma unroll
+      for (int i = 0; i < QUADS; ++i) xr[i] = src[i * C::ROW_STEP * 16];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(raw_empty(rs));     // the values are in registers: the slot can be refilled
+      if (!warp_wait(xq_empty(xs), ((s / X_SLOTS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+      const int chunk = (xs & 1) * 4 + (c4 >> 2);    // 16-byte chunk of the 128-byte row
+      uint8_t* xdst = xq_base + (xs >> 1) * XBUF_BYTES + off_row + ((chunk ^ (rb & 7)) << 4);
+      const bool store_ok = col0 + s * STAGE_COLS < p.K64;
+      uint16_t* cd = cp + (size_t)s * STAGE_COLS;
+#pragma unroll
+      for (int i = 0; i < QUADS; ++i) {
+        uint32_t m8;
+        uint2 bf;
+        int e;
+        quantize_quad(xr[i], p.a_bits, p.exp_min, p.exp_max, e, m8, bf);
+        *reinterpret_cast<uint32_t*>(xdst + i * C::ROW_STEP * 128) = m8;
+        if (xe_writer) xe_dst[(xs * ROWS + C::ROW_STEP * i) * 4] = (int8_t)e;
+        if (store_ok && C::ROW_STEP * i < rows_ok) *reinterpret_cast<uint2*>(cd + i * c_step) = bf;
+      }
+      fence_proxy_async_smem();                      // generic-proxy writes -> visible to the MMA's async proxy
+      __syncwarp();
+      if (lane == 0) mbar_arrive(xq_full(xs));
+    }
+  } else if (warp == WORK_WARPS) {
+    // ------------------------------------------------------------------ A_q panels
+    const int n_pan = pan_hi - pan_lo;
+    const int cbias = -127 - (p.a_bits - 2) - (p.lr_bits - 2) + 1023;
+    constexpr int EPL = 8 * KP / 32;                  // table entries per lane and panel
+    bool ok = true;
+    // exponent bytes of a panel, one load ahead of their use
+    int eb[EPL];
+    auto load_exps = [&](int pp) {
+      const int b0 = (pan_lo + pp) * 8;
+#pragma unroll
+      for (int t = 0; t < EPL; ++t) {
+        const int i = lane + 32 * t;
+        eb[t] = (pp < n_pan && b0 + i / KP < p.kblocks) ? (int)__ldg(a_exp + (size_t)b0 * KP + i) : 1023 - cbias;
+      }
+    };
+    auto publish = [&](int pp) {
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(panel_full(pp % PANELS));
+    };
+    load_exps(0);
+    for (int pp = 0; pp < n_pan && ok; ++pp) {
+      const int pb = pp % PANELS;
+      if (!warp_wait(panel_empty(pb), ((pp / PANELS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+      const int b0 = (pan_lo + pp) * 8;
+      const uint32_t dst0 = smem_u32(panel_base + pb * C::PANEL_BYTES);
+      for (int i = lane; i < 8 * KP; i += 32) {
+        const int c = i / KP, j = i % KP;              // block within the panel, rank column
+        if (b0 + c < p.kblocks) {
+          const int prow = (c & 1) * KP + j;           // even blocks: first k_pad rows; odd: the rest
+          cp_async16(dst0 + prow * 128 + ((c ^ (prow & 7)) << 4), p.asec + ((size_t)(b0 + c) * KP + j) * 16);
+        }
+      }
+      cp_async_commit();
+      // high words of 2^(e_a - 127 - shifts) per block and rank column, for the scalers
+#pragma unroll
+      for (int t = 0; t < EPL; ++t) s_hia[pb * 8 * KP + lane + 32 * t] = (eb[t] + cbias) << 20;
+      load_exps(pp + 1);
+      // the first panel goes out as soon as it has landed; later ones one panel behind their copies
+      if (pp == 0) { cp_async_wait<0>(); publish(0); }
+      else if (pp >= 2) { cp_async_wait<1>(); publish(pp - 1); }
+    }
+    cp_async_wait<0>();
+    if (ok && n_pan > 1) publish(n_pan - 1);
+  } else if (warp == WORK_WARPS + 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_i8(ROWS, C::SLOT_COLS);
+      bool ok = true;
+      for (int s = 0; s < n_stages && ok; ++s) {
+        const int xs = s % X_SLOTS, pp = s >> 1, pb = pp % PANELS;
+        if (!parked_wait(xq_full(xs), (s / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
+        if ((s & 1) == 0 && !parked_wait(panel_full(pb), (pp / PANELS) & 1, abort_flag)) { ok = false; break; }
+        const uint64_t a_desc = make_desc(smem_u32(xq_base + (xs >> 1) * XBUF_BYTES));
+        const uint64_t b_desc = make_desc(smem_u32(panel_base + pb * C::PANEL_BYTES));
+        for (int j = 0; j < 2; ++j) {
+          const int u = 2 * s + j, slot = u % C::TMEM_SLOTS;
+          if (!parked_wait(slot_empty(slot), ((u / C::TMEM_SLOTS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const int kstep = (s & 1) * 2 + j;           // 32 bytes along the swizzled row: +2 in the address field
+          umma_i8(tmem_base + slot * C::SLOT_COLS, a_desc + 2 * kstep, b_desc + 2 * kstep, idesc);
+          umma_commit(slot_full(slot));
+        }
+        if (!ok) break;
+        umma_commit(xq_empty(xs));
+        if (s & 1) umma_commit(panel_empty(pb));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      for (int s = 0; s < n_stages; ++s) {
+        const int rs = s % RAW_SLOTS;
+        if (!parked_wait(raw_empty(rs), ((s / RAW_SLOTS) & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(raw_full(rs), RAW_BYTES);       // rows and columns outside X arrive as zeros
+        tma_load_2d(smem_u32(raw_base + rs * RAW_BYTES), &tmap_x, (pan_lo * 2 + s) * STAGE_COLS, row0, raw_full(rs));
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ the last CTA of the row tile finishes T
+  if (*abort_flag != 0) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 400000) { }
+    if (tid == 0) report_error(p.status, LQER_ERR_TIMEOUT, 400, blockIdx.x);
+  }
+  __threadfence();                 // this CTA's partial sums before its arrival
+  tc_fence_before();
+  __syncthreads();
+  if (warp == WORK_WARPS + 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+  if (tid == 0) {
+    const int arrived = atomicAdd(p.counters + row_tile, 1);
+    const int last = arrived == p.splits - 1;
+    if (last) p.counters[row_tile] = 0;                // zero again for the next call
+    *last_flag = last;
+  }
+  __syncthreads();
+  if (*last_flag == 0) return;
+  __threadfence();
+  // sum over the splits in a fixed order, re-quantise along the rank (16 adjacent lanes hold one block), append to Xcat
+  const double* part0 = p.partials + (size_t)row_tile * p.splits * ROWS * KP;
+  constexpr int OUTS = (ROWS * KP + NUM_THREADS - 1) / NUM_THREADS;     // outputs per thread
+  double t[OUTS];
+#pragma unroll
+  for (int i = 0; i < OUTS; ++i) t[i] = 0.0;
+#pragma unroll 4
+  for (int c = 0; c < p.splits; ++c) {
+    const double* pc = part0 + (size_t)c * ROWS * KP + tid;
+#pragma unroll
+    for (int i = 0; i < OUTS; ++i)
+      if (tid + i * NUM_THREADS < ROWS * KP) t[i] += __ldcg(pc + i * NUM_THREADS);
+  }
+#pragma unroll
+  for (int i = 0; i < OUTS; ++i) {
+    const int o = tid + i * NUM_THREADS;
+    if (o >= ROWS * KP) break;                     // uniform over the warp: ROWS * KP is a multiple of 32
+    const int r = o / KP, j = o % KP;
+    double amax = (t[i] != t[i]) ? 0.0 : fabs(t[i]);
+#pragma unroll
+    for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+    const int e = block_exponent(amax, p.exp_min, p.exp_max);
+    const int qv = quant_mantissa(t[i], e, p.a_bits);
+    const int row = row0 + r;
+    if (row < p.M) {
+      p.xcat[(size_t)row * p.ldx + p.K64 + j] = (uint16_t)bf16_bits_of(qv, e - (p.a_bits - 2));
+      if (p.Tm != nullptr) p.Tm[(size_t)row * KP + j] = (int8_t)qv;
+      if (p.Te != nullptr && (j & 15) == 0) p.Te[(size_t)row * (KP / 16) + (j >> 4)] = (uint8_t)(e + 127);
+    }
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &f, 12000, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+template <int KP>
+static cudaError_t launch_kp(const CUtensorMap& tmap, const Params& p, int ctas, cudaStream_t s) {
+  using C = Cfg<KP>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(prologue_tc_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  LaunchScope scope(kFamPrologue, s);
+  prologue_tc_kernel<KP><<<ctas, NUM_THREADS, C::SMEM_BYTES, s>>>(tmap, p);
+  return cudaGetLastError();
+}
+
+}  // namespace ptc
+
+// The tensor-core prologue serves ranks padded to 16, 32 or 64 and batches large enough to give most SMs a CTA.
+bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch) {
+  if (!prologue_tc_rank_ok(m) || (M + 127) / 128 > kPrologueRowTiles) return false;
+  if ((reinterpret_cast<uintptr_t>(X) & 15) != 0) return false;
+  return any_batch || M >= 1024;
+}
+
+cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
+                               int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
+                               cudaStream_t s) {
+  using namespace ptc;
+  EncodeTiledFn enc = encode_fn();
+  if (enc == nullptr) return cudaErrorNotSupported;
+  CUtensorMap tmap;
+  const cuuint64_t dims[2] = {(cuuint64_t)m.K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)m.K * 4};
+  const cuuint32_t box[2] = {STAGE_COLS, ROWS};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  Params p;
+  p.asec = static_cast<const uint8_t*>(packed) + m.off_a;
+  p.xcat = static_cast<uint16_t*>(xcat);
+  p.Tm = Tm; p.Te = Te; p.status = st;
+  p.partials = partials; p.counters = counters;
+  p.M = M; p.K = m.K; p.K64 = m.K64;
+  p.kblocks = m.K / 16;
+  p.panels = (m.K64 + 127) / 128;
+  p.splits = prologue_tc_splits(m, M);
+  p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
+  p.ldx = xcat_cols(m);
+  const int ctas = ((M + ROWS - 1) / ROWS) * p.splits;
+  switch (m.k_pad) {
+    case 16: return launch_kp<16>(tmap, p, ctas, s);
+    case 32: return launch_kp<32>(tmap, p, ctas, s);
+    case 64: return launch_kp<64>(tmap, p, ctas, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace lqer

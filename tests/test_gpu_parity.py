@@ -100,6 +100,36 @@ def test_project_lowrank_bit_exact(spec):
     Pg.release()
 
 
+TC_PROLOGUE_SPECS = [
+    gen.config_tiny(),
+    gen.LayerSpec("odd", M=37, K=80, N=136, k=5, calib_rows=48, outlier_frac=0, n_outliers=2, outlier_scale=20.0, seed=11),
+    gen.LayerSpec("tp_rank40", M=300, K=1024, N=640, k=40, calib_rows=128, outlier_frac=0.01, outlier_scale=20.0, seed=31),
+    gen.LayerSpec("tp_rank64_tail", M=1100, K=2112, N=256, k=64, calib_rows=128, outlier_frac=0.005, outlier_scale=50.0,
+                  weight_law="student_t4", seed=34),     # K = 16.5 panels of 128: a half panel at the end; nine row tiles
+    gen.LayerSpec("tp_rank32_k4096", M=260, K=4096, N=256, k=32, calib_rows=128, outlier_frac=0.01, outlier_scale=20.0, seed=35),
+]
+
+
+@pytest.mark.parametrize("spec", TC_PROLOGUE_SPECS, ids=lambda s: s.name)
+def test_project_lowrank_tensor_core_prologue_bit_exact(spec):
+    # the prologue whose projection runs on the int8 tensor cores, forced at every batch size
+    W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
+    X = gen.make_activations(spec)
+    ref = olqer.forward(X, P)
+    ws = L.new_workspace(spec.M, Pg)
+    L.set_path(binding.PATH_TENSOR_PROLOGUE)
+    try:
+        Tm, Te = L.project_lowrank(_t(X), Pg, ws)
+        Y = L.linear(_t(X), Pg, ws).cpu().numpy()
+    finally:
+        L.set_path(binding.PATH_AUTO)
+    assert L.poll_status(ws) == 0
+    assert np.array_equal(Tm.cpu().numpy(), ref.Tm)
+    assert np.array_equal(Te.cpu().numpy(), exp_bytes(ref.Te))
+    assert worst_ratio(Y, ref) <= 1.0
+    Pg.release()
+
+
 @pytest.mark.parametrize("spec", SMALL_SPECS, ids=lambda s: s.name)
 def test_linear_reference_kernel(spec):
     W, A, B, P, Pg = _prepare(spec)
@@ -124,7 +154,8 @@ MID_SPECS = [
 ]
 
 
-@pytest.mark.parametrize("path", [binding.PATH_TENSOR, binding.PATH_TENSOR_PAIR], ids=["cta1", "cta2"])
+@pytest.mark.parametrize("path", [binding.PATH_TENSOR, binding.PATH_TENSOR_PAIR, binding.PATH_TENSOR_PROLOGUE],
+                         ids=["cta1", "cta2", "cta2_tcprologue"])
 @pytest.mark.parametrize("spec", SMALL_SPECS + MID_SPECS, ids=lambda s: s.name)
 def test_linear_tensor_core_kernel(spec, path):
     W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
