@@ -98,6 +98,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
   cluster_barrier();                             // both CTAs' barriers exist before any remote arrive
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // barriers and tensor memory are set up: let the next kernel start its own setup, then wait for the
+  // prologue's Xcat (and for the previous user of Y and the workspace) before touching global memory
+  pdl_launch_dependents();
+  pdl_wait();
 
   const int rank_stages = (p.r_blocks + 1) / 2;
   const int stages_per_tile = p.k_slabs + rank_stages;
@@ -378,11 +382,13 @@ cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const 
   cfg.blockDim = dim3(NUM_THREADS);
   cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set up while the prologue drains
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   LaunchScope scope(kFamGemmTcPair, s);
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, tmap, p);
 }

@@ -177,6 +177,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // set up; the next kernel may start its own setup, and X, Xcat and the scratch may still be in use by an earlier one
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp < SW) {
     // ------------------------------------------------------------------ scalers
@@ -440,9 +443,18 @@ static cudaError_t launch_kp(const CUtensorMap& tmap, const Params& p, int ctas,
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ctas);
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set up while the previous kernel drains
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   LaunchScope scope(kFamPrologue, s);
-  prologue_tc_kernel<KP><<<ctas, NUM_THREADS, C::SMEM_BYTES, s>>>(tmap, p);
-  return cudaGetLastError();
+  return cudaLaunchKernelEx(&cfg, prologue_tc_kernel<KP>, tmap, p);
 }
 
 }  // namespace ptc
