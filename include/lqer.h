@@ -170,7 +170,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
 lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, float* Y_host,
                                void* workspace, size_t workspace_bytes, void* stream);
 
-/* Zero the head of a fresh workspace (status area, counters, accumulator; at most 166144 bytes;
+/* Zero the head of a fresh workspace (status area, counters, accumulator; at most 168192 bytes;
  * asynchronous on `stream`).  Call once after allocating the workspace and again after
  * lqer_poll_status reported a device-side error (an interrupted call may leave counters behind). */
 lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void* stream);

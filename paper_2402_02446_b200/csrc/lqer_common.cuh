@@ -58,9 +58,9 @@ inline uint32_t meta_checksum(const PackedMeta& m) {
 // prologue for the GEMM path, or the partial-sum slots of the decode path.
 constexpr int kTCountOffset = 64, kTDoneOffset = 68;
 constexpr int kDecodeMaxCtas = 160;
-constexpr int kPrologueRowTiles = 512;               // arrival counters: batches up to 65536 rows
+constexpr int kPrologueRowTiles = 512;               // an arrival and a departure counter each: batches up to 65536 rows
 constexpr int kPrologueMaxCtas = 148;
-constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8 + kPrologueRowTiles * 4;
+constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8 + kPrologueRowTiles * 8;
 __host__ __device__ inline size_t tacc_offset(const PackedMeta& m) {
   return (size_t)kStatusBytes + (((size_t)m.n_tiles * 4 + 255) & ~(size_t)255);
 }
@@ -68,10 +68,10 @@ __host__ __device__ inline size_t pcount_offset(const PackedMeta& m) {
   return tacc_offset(m) + (size_t)16 * m.k_pad * 8;
 }
 __host__ __device__ inline size_t persist_bytes(const PackedMeta& m) {
-  return pcount_offset(m) + (size_t)kPrologueRowTiles * 4;
+  return pcount_offset(m) + (size_t)kPrologueRowTiles * 8;
 }
 // Tensor-core prologue: a CTA owns 128 rows and one of `splits` ranges of K (in panels of 128 columns);
-// each CTA leaves a [128, k_pad] fp64 partial sum for the last CTA of its row tile to add up.
+// each CTA leaves a [128, k_pad] fp64 partial sum; once all CTAs of a row tile have arrived each adds up its share of rows.
 inline bool prologue_tc_rank_ok(const PackedMeta& m) { return m.k > 0 && (m.k_pad == 16 || m.k_pad == 32 || m.k_pad == 64); }
 inline int prologue_tc_splits(const PackedMeta& m, int M) {
   const int row_tiles = (M + 127) / 128, panels = (m.K64 + 127) / 128;
@@ -227,7 +227,7 @@ cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const vo
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s);
 // The same prologue with the projection on the tcgen05 int8 tensor cores: ranks up to 64, large batches.
 bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch);
-// `partials`: prologue_tc_scratch_bytes(m, M) of scratch; `counters`: the zeroed per-row-tile counters of the workspace head.
+// `partials`: prologue_tc_scratch_bytes(m, M) of scratch; `counters`: the zeroed counter pairs of the workspace head.
 cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                cudaStream_t s);

@@ -4,7 +4,8 @@
 //
 // Same results as prologue_kernel (bit for bit in X_q and T_q); what differs is where the work
 // runs.  A CTA owns 128 rows of X and one of `splits` ranges of K; the CTAs of a row tile leave
-// fp64 partial sums in global scratch and the last one to arrive adds them in a fixed order.
+// fp64 partial sums in global scratch and, once all have arrived, each adds up a share of the rows
+// in a fixed order.
 //   scalers      read the int32 block products from tensor memory, scale each by 2^(e_x + e_a)
 //                and sum in fp64 (exact for any realistic exponent spread)
 //   quantisers   take fp32 X from a shared-memory ring that TMA fills, write the exact bf16
@@ -71,7 +72,7 @@ struct Params {
   uint8_t* Te;
   DeviceStatus* status;
   double* partials;         // [row tile][split][128][k_pad]
-  int* counters;            // [row tile], zero between calls
+  int* counters;            // [row tile][arrivals, departures], zero between calls
   int M, K, K64;
   int kblocks;              // K / 16
   int panels;               // ceil(K64 / 128)
@@ -364,7 +365,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     }
   }
 
-  // ------------------------------------------------------------------ the last CTA of the row tile finishes T
+  // ------------------------------------------------------------------ the CTAs of a row tile finish T together
   if (*abort_flag != 0) {
     const long long t0 = clock64();
     while (clock64() - t0 < 400000) { }
@@ -377,44 +378,59 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     tc_fence_after();
     tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
+  // Every CTA of the row tile finishes a share of its rows once all partial sums are there.  The CTAs of a launch
+  // fit the GPU together (at most one per SM), so the wait below ends as soon as the last of them has run; it is
+  // bounded all the same.  Two counters per row tile: arrivals, and departures (the last to leave zeroes both).
+  int* arrive_cnt = p.counters + 2 * row_tile;
+  int* depart_cnt = arrive_cnt + 1;
   if (tid == 0) {
-    const int arrived = atomicAdd(p.counters + row_tile, 1);
-    const int last = arrived == p.splits - 1;
-    if (last) p.counters[row_tile] = 0;                // zero again for the next call
-    *last_flag = last;
+    atomicAdd(arrive_cnt, 1);
+    int seen = 1;
+    const long long t0 = clock64();
+    for (;;) {
+      int v;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(arrive_cnt) : "memory");
+      if (v >= p.splits) break;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) { seen = 0; break; }
+      __nanosleep(100);
+    }
+    if (!seen) report_error(p.status, LQER_ERR_TIMEOUT, 401, blockIdx.x);
+    *last_flag = seen;
   }
   __syncthreads();
-  if (*last_flag == 0) return;
-  __threadfence();
-  // sum over the splits in a fixed order, re-quantise along the rank (16 adjacent lanes hold one block), append to Xcat
-  const double* part0 = p.partials + (size_t)row_tile * p.splits * ROWS * KP;
-  constexpr int OUTS = (ROWS * KP + NUM_THREADS - 1) / NUM_THREADS;     // outputs per thread
-  double t[OUTS];
-#pragma unroll
-  for (int i = 0; i < OUTS; ++i) t[i] = 0.0;
+  if (*last_flag != 0) {
+    // rows [r_lo, r_hi) of the tile: sum over the K ranges in a fixed order, re-quantise along the rank (16 adjacent
+    // lanes hold one block), append to Xcat
+    const int r_lo = split * ROWS / p.splits, r_hi = (split + 1) * ROWS / p.splits;
+    const int n_out = (r_hi - r_lo) * KP;                                  // a multiple of 16
+    const double* part0 = p.partials + (size_t)row_tile * p.splits * ROWS * KP + (size_t)r_lo * KP;
+    for (int o0 = warp * 32; o0 < n_out; o0 += NUM_THREADS) {              // whole warps: the shuffles need every lane
+      const int o = o0 + lane;
+      const bool live = o < n_out;
+      double t = 0.0;
+      if (live) {
+        const double* pc = part0 + o;
 #pragma unroll 4
-  for (int c = 0; c < p.splits; ++c) {
-    const double* pc = part0 + (size_t)c * ROWS * KP + tid;
+        for (int c = 0; c < p.splits; ++c) t += __ldcg(pc + (size_t)c * ROWS * KP);
+      }
+      double amax = (t != t) ? 0.0 : fabs(t);
 #pragma unroll
-    for (int i = 0; i < OUTS; ++i)
-      if (tid + i * NUM_THREADS < ROWS * KP) t[i] += __ldcg(pc + i * NUM_THREADS);
-  }
-#pragma unroll
-  for (int i = 0; i < OUTS; ++i) {
-    const int o = tid + i * NUM_THREADS;
-    if (o >= ROWS * KP) break;                     // uniform over the warp: ROWS * KP is a multiple of 32
-    const int r = o / KP, j = o % KP;
-    double amax = (t[i] != t[i]) ? 0.0 : fabs(t[i]);
-#pragma unroll
-    for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
-    const int e = block_exponent(amax, p.exp_min, p.exp_max);
-    const int qv = quant_mantissa(t[i], e, p.a_bits);
-    const int row = row0 + r;
-    if (row < p.M) {
-      p.xcat[(size_t)row * p.ldx + p.K64 + j] = (uint16_t)bf16_bits_of(qv, e - (p.a_bits - 2));
-      if (p.Tm != nullptr) p.Tm[(size_t)row * KP + j] = (int8_t)qv;
-      if (p.Te != nullptr && (j & 15) == 0) p.Te[(size_t)row * (KP / 16) + (j >> 4)] = (uint8_t)(e + 127);
+      for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+      const int e = block_exponent(amax, p.exp_min, p.exp_max);
+      const int qv = quant_mantissa(t, e, p.a_bits);
+      const int r = r_lo + o / KP, j = o % KP;
+      const int row = row0 + r;
+      if (live && row < p.M) {
+        p.xcat[(size_t)row * p.ldx + p.K64 + j] = (uint16_t)bf16_bits_of(qv, e - (p.a_bits - 2));
+        if (p.Tm != nullptr) p.Tm[(size_t)row * KP + j] = (int8_t)qv;
+        if (p.Te != nullptr && (j & 15) == 0) p.Te[(size_t)row * (KP / 16) + (j >> 4)] = (uint8_t)(e + 127);
+      }
     }
+  }
+  __syncthreads();
+  if (tid == 0 && atomicAdd(depart_cnt, 1) == p.splits - 1) {              // everyone has read the counters: zero for the next call
+    *arrive_cnt = 0;
+    *depart_cnt = 0;
   }
 }
 
