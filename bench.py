@@ -359,6 +359,9 @@ def run_ours(args) -> None:
             "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
             "config": {"workload": WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]",
                        "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32,
+                       "decode_launches": "lqer_linear_batched runs consecutive independent same-shape decode calls "
+                                          "(q,k,v,o; gate,up) as one launch that divides the SMs among them: 3 launches "
+                                          "per decoder layer of 7 linears",
                        "l2": "inputs larger than L2: every linear has its own packed weights and activations "
                              f"({sum(p.buf.numel() for p in packed) / 1e9:.2f} GB of weights per step)",
                        "parallelism": "replicas (independent token batches)" if world > 1 else "1 GPU"},

@@ -159,7 +159,10 @@ lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, floa
 
 /* n_calls independent layers back to back on one stream (`calls` is a HOST array).
  * The workspace is reused by consecutive calls (stream order makes that safe) and must
- * fit the largest of them. */
+ * fit the largest of them.  Independent means that no call reads what another call of the
+ * same batch writes: with the path left at 0, up to four consecutive calls with M <= 4 and
+ * packed buffers of one shape (K, N, rank, formats) run as ONE launch that divides the SMs
+ * among them (the q, k, v or the gate and up projections of a decoder layer). */
 lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
                                   void* workspace, size_t workspace_bytes, void* stream);
 

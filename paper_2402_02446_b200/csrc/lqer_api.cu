@@ -43,6 +43,13 @@ static std::mutex g_mu;
 static std::unordered_map<const void*, PackedMeta> g_registry;
 static std::atomic<int> g_path{0};
 
+// Two packed buffers with the same sections, formats and sizes (their contents may differ).
+static bool same_shape(const PackedMeta& a, const PackedMeta& b) {
+  return a.K == b.K && a.N == b.N && a.k == b.k && a.k_pad == b.k_pad && a.w_bits == b.w_bits && a.a_bits == b.a_bits &&
+         a.lr_bits == b.lr_bits && a.exp_min == b.exp_min && a.exp_max == b.exp_max && a.off_w == b.off_w &&
+         a.off_b == b.off_b && a.off_a == b.off_a;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -341,10 +348,31 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     const bool decode = path == 2 || path == 5 || (path == 0 && c.M <= decode_max_m());
     if (workspace_bytes < call_bytes(m, c.M, decode)) return LQER_ERR_BUFFER_TOO_SMALL;
   }
-  for (int i = 0; i < n_calls; ++i) {
-    lqer_status_t st = lqer_linear_stream(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace,
-                                          workspace_bytes, stream);
-    if (st != LQER_OK) return st;
+  const bool may_group = g_path.load() == 0;   // a forced path runs every call on its own
+  for (int i = 0; i < n_calls;) {
+    // The calls are independent, so consecutive decode calls of one shape (the q, k, v projections of a layer, or
+    // its gate and up projections) share a launch: the column-owner decode kernel keeps nothing in the workspace.
+    int n = 1;
+    PackedMeta m0;
+    if (may_group && lookup(calls[i].packed, m0) == LQER_OK && decode_cols_fits(m0, calls[i].M)) {
+      while (i + n < n_calls && n < decode_cols_max_group()) {
+        PackedMeta m1;
+        if (calls[i + n].M != calls[i].M || lookup(calls[i + n].packed, m1) != LQER_OK || !same_shape(m0, m1)) break;
+        ++n;
+      }
+    }
+    if (n > 1) {
+      lqer_status_t st = check_arch();
+      if (st != LQER_OK) return st;
+      if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
+      if (launch_decode_cols_group(calls + i, n, m0, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return LQER_ERR_CUDA;
+    } else {
+      lqer_status_t st = lqer_linear_stream(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace,
+                                            workspace_bytes, stream);
+      if (st != LQER_OK) return st;
+    }
+    i += n;
   }
   return LQER_OK;
 }

@@ -37,12 +37,13 @@ constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q (pa
 constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
 constexpr int kAStageMax = 100 * 1024;   // a CTA's share of A_q is staged in shared memory if it fits in this
 
+constexpr int kMaxGroup = 4;   // independent layers of one shape that may share a launch (blockIdx.y picks one)
+
 struct Params {
-  const float* X;
-  float* Y;
-  const uint8_t* wsec;
-  const uint8_t* bsec;
-  const uint8_t* asec;
+  const float* X[kMaxGroup];
+  float* Y[kMaxGroup];
+  const uint8_t* packed[kMaxGroup];
+  size_t off_w, off_b, off_a;   // sections of a packed buffer (equal for equal shapes)
   DeviceStatus* status;
   int M, K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
   int a_stage_bytes;    // shared memory reserved for staging A_q (0: read it from global memory)
@@ -108,6 +109,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
   const int G = gridDim.x, cta = blockIdx.x;
+  const float* const X = p.X[blockIdx.y];
+  float* const Y = p.Y[blockIdx.y];
+  const uint8_t* const wsec = p.packed[blockIdx.y] + p.off_w;
+  const uint8_t* const bsec = p.packed[blockIdx.y] + p.off_b;
+  const uint8_t* const asec = p.packed[blockIdx.y] + p.off_a;
   const int cg_lo = cta * p.n_cg / G, cg_hi = (cta + 1) * p.n_cg / G;
 
   // this lane's share of (column group cg, slab j): global -> registers
@@ -116,7 +122,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     d.e = 127u;
     if (cg < cg_hi && j < p.k_slabs) {
       const int col = (cg & 15) * 8 + g;
-      const uint8_t* tile = p.wsec + ((size_t)(cg >> 4) * p.k_slabs + j) * kWTileBytes;
+      const uint8_t* tile = wsec + ((size_t)(cg >> 4) * p.k_slabs + j) * kWTileBytes;
       d.w = ld_stream_u64(tile + (t >> 1) * (kTileN * 16) + col * 16 + (t & 1) * 8);
       d.e = ld_stream_u8(tile + kWTileNibbleBytes + col * 4 + t);
     }
@@ -130,7 +136,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     eb = 127u;
     if (cg < cg_hi && warp < p.r_blocks) {
       const int col = (cg & 15) * 8 + g;
-      const uint8_t* tile = p.bsec + (size_t)(cg >> 4) * ((size_t)p.r_blocks * kTileN * 17);
+      const uint8_t* tile = bsec + (size_t)(cg >> 4) * ((size_t)p.r_blocks * kTileN * 17);
       wv = ld_stream_u32(tile + ((size_t)warp * kTileN + col) * 16 + t * 4);
       eb = ld_stream_u8(tile + (size_t)p.r_blocks * kTileN * 16 + warp * kTileN + col);
     }
@@ -152,8 +158,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const bool a_staged = p.k_pad > 0 && (kb_hi - kb_lo) * p.k_pad * 17 <= p.a_stage_bytes;
   if (a_staged) {
     const int mant = (kb_hi - kb_lo) * p.k_pad * 16, ex = (kb_hi - kb_lo) * p.k_pad;
-    const uint8_t* gm = p.asec + (size_t)kb_lo * p.k_pad * 16;
-    const uint8_t* ge = p.asec + (size_t)KBr * p.k_pad * 16 + (size_t)kb_lo * p.k_pad;
+    const uint8_t* gm = asec + (size_t)kb_lo * p.k_pad * 16;
+    const uint8_t* ge = asec + (size_t)KBr * p.k_pad * 16 + (size_t)kb_lo * p.k_pad;
     for (int o = tid * 16; o < mant; o += kThreads * 16)
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(a_stage + o)), "l"(gm + o) : "memory");
     for (int o = tid * 16; o < ex; o += kThreads * 16)
@@ -171,7 +177,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       const int item = base + tid;
       const bool valid = item < total;
       const int row = valid ? item / per_row : 0, c4 = valid ? item % per_row : 0;
-      const float4 v = (valid && c4 * 4 < p.K) ? __ldg(reinterpret_cast<const float4*>(p.X + (size_t)row * p.K + c4 * 4))
+      const float4 v = (valid && c4 * 4 < p.K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * p.K + c4 * 4))
                                                : make_float4(0.f, 0.f, 0.f, 0.f);
       int e;
       uint32_t m8;
@@ -201,9 +207,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   if (p.k_pad > 0) {
     const int NT = p.k_pad / 8;
     // A_q of blocks kb_lo..kb_hi: staged copy, or global memory
-    const uint8_t* a_mant = a_staged ? a_stage - (size_t)kb_lo * p.k_pad * 16 : p.asec;
+    const uint8_t* a_mant = a_staged ? a_stage - (size_t)kb_lo * p.k_pad * 16 : asec;
     const uint8_t* a_exp = a_staged ? a_stage + (size_t)(kb_hi - kb_lo) * p.k_pad * 16 - (size_t)kb_lo * p.k_pad
-                                    : p.asec + (size_t)KBr * p.k_pad * 16;
+                                    : asec + (size_t)KBr * p.k_pad * 16;
     const int bias = -127 - (p.lr_bits - 2);                        // exponent bytes carry +127
     const int tiles_w = NT < kWarps ? NT : kWarps;                  // warps side by side on different rank tiles
     int subsets = kWarps / tiles_w;                                 // warps that split the K blocks of one tile
@@ -354,7 +360,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) v += red[((w * kCg + u) * 8 + gg) * kMaxM + r];
       const int cg = cg0 + u;
-      if (cg < cg_hi && r < M) p.Y[(size_t)r * p.N + cg * 8 + gg] = v;
+      if (cg < cg_hi && r < M) Y[(size_t)r * p.N + cg * 8 + gg] = v;
     }
     __syncthreads();                             // red is rewritten by the next round
   }
@@ -376,6 +382,16 @@ bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && c
 
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y, void* workspace,
                                cudaStream_t s) {
+  const lqer_call_t one = {X, M, packed, Y};
+  return launch_decode_cols_group(&one, 1, m, workspace, s);
+}
+
+int decode_cols_max_group() { return dcol::kMaxGroup; }
+
+// n independent layers of one shape (same K, N, rank, formats) and one M in a single launch: the SMs are divided
+// among them, so the layers' fixed latencies (dependency wait, X quantisation, the T exchange, the final
+// reduction) overlap instead of following one another.
+cudaError_t launch_decode_cols_group(const lqer_call_t* calls, int n, const PackedMeta& m, void* workspace, cudaStream_t s) {
   using namespace dcol;
   static int sm_count = 0;
   static bool attr_set = false;
@@ -387,17 +403,22 @@ cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
+  if (n < 1 || n > kMaxGroup) return cudaErrorInvalidValue;
+  const int M = calls[0].M;
   Params p;
-  const uint8_t* base = static_cast<const uint8_t*>(packed);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  p.X = X; p.Y = Y;
-  p.wsec = base + m.off_w; p.bsec = base + m.off_b; p.asec = base + m.off_a;
+  for (int i = 0; i < kMaxGroup; ++i) {
+    const lqer_call_t& c = calls[i < n ? i : 0];
+    p.X[i] = c.X; p.Y[i] = c.Y; p.packed[i] = static_cast<const uint8_t*>(c.packed);
+  }
+  p.off_w = m.off_w; p.off_b = m.off_b; p.off_a = m.off_a;
   p.status = reinterpret_cast<DeviceStatus*>(ws);
   p.M = M; p.K = m.K; p.N = m.N; p.K64 = m.K64; p.k_pad = m.k_pad;
   p.k_slabs = m.k_slabs; p.r_blocks = m.r_blocks;
   p.n_cg = m.N / 8;
   p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
-  int G = p.n_cg < sm_count ? p.n_cg : sm_count;
+  int G = sm_count / n;                         // CTAs per layer
+  if (G > p.n_cg) G = p.n_cg;
   if (G > kDecodeMaxCtas) G = kDecodeMaxCtas;
   const int cs = G >= kClusterSize ? kClusterSize : 1;
   G = G / cs * cs;
@@ -408,7 +429,7 @@ cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const
   if (!decode_cols_fits(m, M)) return cudaErrorInvalidValue;
 
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(G);
+  cfg.gridDim = dim3(G, n);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
@@ -430,7 +451,8 @@ cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const
       if (cudaOccupancyMaxActiveClusters(&nc, decode_cols_kernel, &probe) != cudaSuccess || nc < 1) nc = 1;
       max_clusters = nc;
     }
-    if (G > max_clusters * cs) { G = max_clusters * cs; cfg.gridDim = dim3(G); }
+    if (G * n > max_clusters * cs) { G = max_clusters / n * cs; cfg.gridDim = dim3(G, n); }
+    if (G < cs) return cudaErrorInvalidConfiguration;
   }
   LaunchScope scope(kFamDecode, s);
   return cudaLaunchKernelEx(&cfg, decode_cols_kernel, p);

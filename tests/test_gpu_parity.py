@@ -226,6 +226,34 @@ def test_decode_chain_shares_one_workspace():
         lay[4].release()
 
 
+@pytest.mark.parametrize("M", [1, 3])
+def test_batched_decode_groups_same_shape_calls(M):
+    # seven independent calls: five layers of one shape (a group of four and a fifth), then two of another shape;
+    # the batched entry point runs same-shape neighbours in shared launches and must give what single calls give
+    spec_a = gen.LayerSpec("grp_a", M=M, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=51)
+    spec_b = gen.LayerSpec("grp_b", M=M, K=512, N=2048, k=8, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=52)
+    layers = []
+    for i, spec in enumerate([spec_a] * 5 + [spec_b] * 2):
+        sp = gen.LayerSpec(f"{spec.name}{i}", M=M, K=spec.K, N=spec.N, k=spec.k, calib_rows=spec.calib_rows,
+                           outlier_frac=spec.outlier_frac, outlier_scale=spec.outlier_scale, seed=spec.seed + i)
+        layers.append((sp,) + _random_factor_layer(sp))
+    Xs = [_t(gen.make_activations(sp, M=M)) for sp, _, _ in layers]
+    n = max(L.workspace_bytes(M, sp.K, sp.N, sp.k) for sp, _, _ in layers)
+    ws = torch.zeros(n, dtype=torch.uint8, device=DEV)
+    launches = L.launch_count()
+    Yb = [torch.full((M, sp.N), float("nan"), dtype=torch.float32, device=DEV) for sp, _, _ in layers]
+    L.linear_batched([(x, lay[2], y) for x, lay, y in zip(Xs, layers, Yb)], ws)
+    torch.cuda.synchronize()
+    assert L.poll_status(ws) == 0
+    assert L.launch_count() - launches == 3            # 4 + 1 of the first shape, 2 of the second
+    for x, (sp, P, Pg), yb in zip(Xs, layers, Yb):
+        ys = L.linear(x, Pg, ws)
+        assert torch.equal(ys, yb), sp.name             # same arithmetic, same order: bit-identical
+        assert worst_ratio(yb.cpu().numpy(), olqer.forward(x.cpu().numpy(), P)) <= 1.0, sp.name
+    for _, _, Pg in layers:
+        Pg.release()
+
+
 @pytest.mark.parametrize("M", [1, 16])
 def test_linear_decode_full_size(M):
     spec = gen.config_decode(M)
