@@ -91,6 +91,8 @@ __device__ __forceinline__ double ld_dsmem_f64(const double* local, uint32_t cta
   return v;
 }
 
+// MT: rows the accumulators are compiled for (1 for the single-token call, kMaxM otherwise); M <= MT.
+template <int MT>
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -116,16 +118,25 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const uint8_t* const asec = p.packed[blockIdx.y] + p.off_a;
   const int cg_lo = cta * p.n_cg / G, cg_hi = (cta + 1) * p.n_cg / G;
 
-  // this lane's share of (column group cg, slab j): global -> registers
-  auto fetch = [&](UnitRegs& d, int cg, int j) {
-    d.w = make_uint2(0x88888888u, 0x88888888u);  // mantissa 0 in offset binary
-    d.e = 127u;
-    if (cg < cg_hi && j < p.k_slabs) {
-      const int col = (cg & 15) * 8 + g;
-      const uint8_t* tile = wsec + ((size_t)(cg >> 4) * p.k_slabs + j) * kWTileBytes;
-      d.w = ld_stream_u64(tile + (t >> 1) * (kTileN * 16) + col * 16 + (t & 1) * 8);
-      d.e = ld_stream_u8(tile + kWTileNibbleBytes + col * 4 + t);
-    }
+  // This lane's share of (column group cg, slab j): global -> registers.  Byte offsets into the W section are kept
+  // per column group (32 bits: the section is far below 4 GB); a load then costs two adds.  Column groups past the
+  // CTA's range are clamped to its last one and slabs past K to the last slab: such loads stay inside the section
+  // and what they return is never used (the sums of those slabs are skipped, those columns are not stored).
+  const uint32_t lane_w = (uint32_t)((t >> 1) * (kTileN * 16) + g * 16 + (t & 1) * 8);
+  const uint32_t lane_e = (uint32_t)(kWTileNibbleBytes + g * 4 + t);
+  struct GroupOff { uint32_t w, e; };
+  auto group_off = [&](int cg) -> GroupOff {
+    cg = max(min(cg, cg_hi - 1), 0);
+    const uint32_t tile = (uint32_t)(cg >> 4) * (uint32_t)p.k_slabs * (uint32_t)kWTileBytes;
+    GroupOff o;
+    o.w = tile + (uint32_t)(cg & 15) * 128u + lane_w;
+    o.e = tile + (uint32_t)(cg & 15) * 32u + lane_e;
+    return o;
+  };
+  auto fetch = [&](UnitRegs& d, const GroupOff& o, int j) {
+    const uint32_t jo = (uint32_t)min(j, p.k_slabs - 1) * (uint32_t)kWTileBytes;
+    d.w = ld_stream_u64(wsec + (o.w + jo));
+    d.e = ld_stream_u8(wsec + (o.e + jo));
   };
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -146,10 +157,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   uint32_t rank_w[kCg], rank_e[kCg];
   // weights depend on no earlier kernel: request the first slabs, the rank blocks and this CTA's
   // share of A_q before the dependency wait
+  GroupOff o_cur[kCg], o_nxt[kCg];               // offsets of this round's and the next round's column groups
+#pragma unroll
+  for (int u = 0; u < kCg; ++u) o_cur[u] = group_off(cg_lo + u);
 #pragma unroll
   for (int s = 0; s < kSets; ++s)
 #pragma unroll
-    for (int u = 0; u < kCg; ++u) fetch(regs[s][u], cg_lo + u, warp + kWarps * s);
+    for (int u = 0; u < kCg; ++u) fetch(regs[s][u], o_cur[u], warp + kWarps * s);
 #pragma unroll
   for (int u = 0; u < kCg; ++u) fetch_rank(rank_w[u], rank_e[u], cg_lo + u);
   const int KBr = p.K / 16;
@@ -253,11 +267,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const int slabs_mine = p.k_slabs > warp ? (p.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
 #pragma unroll 1
   for (int cg0 = cg_lo; cg0 < cg_hi; cg0 += kCg) {
-    float acc[kCg][kMaxM];
+    float acc[kCg][MT];
 #pragma unroll
     for (int u = 0; u < kCg; ++u)
 #pragma unroll
-      for (int r = 0; r < kMaxM; ++r) acc[u][r] = 0.f;
+      for (int r = 0; r < MT; ++r) acc[u][r] = 0.f;
+
+#pragma unroll
+    for (int u = 0; u < kCg; ++u) o_nxt[u] = group_off(cg0 + kCg + u);
 
     // ---- W_q: this warp's slabs of the round's column groups
 #pragma unroll 1
@@ -267,7 +284,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
         const int j = warp + kWarps * (js + s);
         if (j < p.k_slabs) {
 #pragma unroll
-          for (int r = 0; r < kMaxM; ++r) {
+          for (int r = 0; r < MT; ++r) {
             if (r < M) {
               const uint4 x = *reinterpret_cast<const uint4*>(xm + (size_t)r * p.K64 + j * 64 + t * 16);
               const float sx = xsc[r * KB + j * 4 + t];
@@ -288,11 +305,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
         // refill the set: the same groups four slabs on, or - past this warp's last slabs - the
         // next round's groups from their first slabs, so that rounds follow each other without a bubble
         const bool more = js + kSets < slabs_mine;
+        const int jn = more ? j + kWarps * kSets : warp + kWarps * s;
 #pragma unroll
-        for (int u = 0; u < kCg; ++u)
-          fetch(regs[s][u], more ? cg0 + u : cg0 + kCg + u, more ? j + kWarps * kSets : warp + kWarps * s);
+        for (int u = 0; u < kCg; ++u) {
+          GroupOff o;
+          o.w = more ? o_cur[u].w : o_nxt[u].w;
+          o.e = more ? o_cur[u].e : o_nxt[u].e;
+          fetch(regs[s][u], o, jn);
+        }
       }
     }
+#pragma unroll
+    for (int u = 0; u < kCg; ++u) o_cur[u] = o_nxt[u];
 
     // ---- B_q against T_q: rank blocks warp, warp + 16, ...
     if (p.k_pad > 0) {
@@ -328,7 +352,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
         for (int u = 0; u < kCg; ++u) {
           const float sb = __uint_as_float((rank_e[u] - (uint32_t)(p.lr_bits - 2)) << 23);        // 2^(e_b - 6)
 #pragma unroll
-          for (int r = 0; r < kMaxM; ++r) {
+          for (int r = 0; r < MT; ++r) {
             if (r < M) {
               const int tw = *reinterpret_cast<const int*>(tq8 + r * p.k_pad + warp * 16 + t * 4);
               acc[u][r] = fmaf((float)__dp4a(tw, (int)rank_w[u], 0), tqs[r * rbn + warp] * sb, acc[u][r]);
@@ -345,7 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     for (int u = 0; u < kCg; ++u) {
       float mine = 0.f;
 #pragma unroll
-      for (int r = 0; r < kMaxM; ++r) {
+      for (int r = 0; r < MT; ++r) {
         float v = acc[u][r];
         v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
         v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
@@ -399,7 +423,9 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, int n, const Pack
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(decode_cols_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(decode_cols_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(decode_cols_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -448,14 +474,14 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, int n, const Pack
       probe.dynamicSmemBytes = 200 * 1024;
       probe.gridDim = dim3(sm_count / cs * cs);
       int nc = 0;
-      if (cudaOccupancyMaxActiveClusters(&nc, decode_cols_kernel, &probe) != cudaSuccess || nc < 1) nc = 1;
+      if (cudaOccupancyMaxActiveClusters(&nc, decode_cols_kernel<kMaxM>, &probe) != cudaSuccess || nc < 1) nc = 1;
       max_clusters = nc;
     }
     if (G * n > max_clusters * cs) { G = max_clusters / n * cs; cfg.gridDim = dim3(G, n); }
     if (G < cs) return cudaErrorInvalidConfiguration;
   }
   LaunchScope scope(kFamDecode, s);
-  return cudaLaunchKernelEx(&cfg, decode_cols_kernel, p);
+  return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM>, p);
 }
 
 }  // namespace lqer
