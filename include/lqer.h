@@ -144,8 +144,8 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * that much memory until the process exits.  The call itself allocates and frees nothing.
  *  - X, Y, packed, stream: as for lqer_linear_stream (device pointers, caller owned).
  *  - Limit: lqer_workspace_bytes(M, K, N, k) <= LQER_STATIC_SCRATCH_BYTES, otherwise
- *    LQER_ERR_STATIC_SCRATCH is returned and nothing is launched (M = 256 at K = 4096 needs
- *    about 2.1 MB; M = 16 fits for every supported K).
+ *    LQER_ERR_STATIC_SCRATCH is returned and nothing is launched (M = 256 at K = N = 4096, rank 32 needs
+ *    about 4.2 MB; M = 16 fits for every supported K).
  *  - The first call on a device looks up the array's device address (the device must be
  *    current); make that first call before any stream capture begins.
  *  - All calls on a device share the one array and it keeps the previous call's contents; the
