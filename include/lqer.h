@@ -173,6 +173,16 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
 lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, float* Y_host,
                                void* workspace, size_t workspace_bytes, void* stream);
 
+/* n_calls independent layers with HOST buffers (calls[i].X and calls[i].Y are host pointers; pinned
+ * memory gives full copy speed; `calls` is a host array).  Copies in, layers and copies out are
+ * pipelined: while layer i runs on `stream`, X of layer i+1 is on its way in and Y of layer i-1 on
+ * its way out, on two internal streams made at the first call on a device.  Returns when every Y
+ * is on the host.  workspace must hold lqer_linear_host_batched_bytes(calls, n_calls) bytes: the
+ * largest lqer_workspace_bytes of the calls plus two X and two Y buffers of the largest sizes. */
+lqer_status_t lqer_linear_host_batched_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes);
+lqer_status_t lqer_linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace,
+                                       size_t workspace_bytes, void* stream);
+
 /* Zero the head of a fresh workspace (status area, counters, accumulator; at most 168192 bytes;
  * asynchronous on `stream`).  Call once after allocating the workspace and again after
  * lqer_poll_status reported a device-side error (an interrupted call may leave counters behind). */

@@ -22,6 +22,9 @@ from .binding import (  # noqa: F401
     linear_batched,
     linear_static,
     linear_host,
+    linear_host_batched,
+    linear_host_batched_bytes,
+    make_host_calls,
     poll_status,
     set_path,
     launch_count,

@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
             "lqer_linear_static": (i, [vp, i, vp, vp, vp]),
             "lqer_linear_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
             "lqer_linear_host": (i, [vp, i, vp, vp, vp, sz, vp]),
+            "lqer_linear_host_batched_bytes": (i, [C.POINTER(Call), i, C.POINTER(sz)]),
+            "lqer_linear_host_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
             "lqer_workspace_init": (i, [vp, sz, vp]),
             "lqer_poll_status": (i, [vp, vp, C.POINTER(i)]),
             "lqer_set_path": (i, [i]),
@@ -246,6 +248,32 @@ def linear_host(X_host: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y_host
     _check(lib().lqer_linear_host(X_host.data_ptr(), X_host.shape[0], P.ptr, Y_host.data_ptr(), ws.data_ptr(),
                                   ws.numel(), _stream(stream)), "lqer_linear_host")
     return Y_host
+
+
+def make_host_calls(items) -> "C.Array":
+    """items: iterable of (X_cpu, PackedWeights, Y_cpu), contiguous fp32 CPU tensors -> a host array of lqer_call_t."""
+    items = list(items)
+    arr = (Call * len(items))()
+    for j, (X, P, Y) in enumerate(items):
+        for t in (X, Y):
+            if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
+                raise ValueError("expected contiguous fp32 CPU tensors")
+        arr[j] = Call(X.data_ptr(), X.shape[0], P.ptr, Y.data_ptr())
+    return arr
+
+
+def linear_host_batched_bytes(calls) -> int:
+    arr = calls if isinstance(calls, C.Array) else make_host_calls(calls)
+    out = C.c_size_t()
+    _check(lib().lqer_linear_host_batched_bytes(arr, len(arr), C.byref(out)), "lqer_linear_host_batched_bytes")
+    return out.value
+
+
+def linear_host_batched(calls, ws: torch.Tensor, stream=None) -> None:
+    """Independent layers with host buffers; copies in, layers and copies out overlap.  Returns when all Y are on the host."""
+    arr = calls if isinstance(calls, C.Array) else make_host_calls(calls)
+    _check(lib().lqer_linear_host_batched(arr, len(arr), ws.data_ptr(), ws.numel(), _stream(stream)),
+           "lqer_linear_host_batched")
 
 
 def poll_status(ws: torch.Tensor, stream=None) -> int:

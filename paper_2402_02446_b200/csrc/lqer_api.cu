@@ -1,4 +1,5 @@
 // Host side of the C ABI: argument checks, the registry of packed buffers, path selection.
+#include <algorithm>
 #include <atomic>
 #include <cstring>
 #include <mutex>
@@ -395,6 +396,112 @@ lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, f
   if (cudaMemcpyAsync(Y_host, Yd, (size_t)M * m.N * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LQER_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return LQER_ERR_CUDA;
   return LQER_OK;
+}
+
+// Streams and events of lqer_linear_host_batched, made once per device.
+namespace {
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, in_done[2] = {}, comp_done[2] = {}, out_done[2] = {};
+};
+HostPipe g_pipes[64];
+
+HostPipe* host_pipe() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_mu);
+  HostPipe& hp = g_pipes[dev];
+  if (!hp.ready) {
+    bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess;
+    for (int b = 0; b < 2 && ok; ++b)
+      ok = cudaEventCreateWithFlags(&hp.in_done[b], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.comp_done[b], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.out_done[b], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    hp.ready = true;
+  }
+  return &hp;
+}
+}  // namespace
+
+lqer_status_t lqer_linear_host_batched_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes) {
+  if (calls == nullptr || bytes == nullptr) return LQER_ERR_NULL;
+  if (n_calls < 0) return LQER_ERR_SHAPE;
+  size_t core = kStatusBytes, xb = 0, yb = 0;
+  for (int i = 0; i < n_calls; ++i) {
+    const lqer_call_t& c = calls[i];
+    if (c.packed == nullptr) return LQER_ERR_NULL;
+    if (c.M <= 0 || c.M > (1 << 24)) return LQER_ERR_SHAPE;
+    PackedMeta m;
+    lqer_status_t st = lookup(c.packed, m);
+    if (st != LQER_OK) return st;
+    core = std::max(core, workspace_total(m, c.M));
+    xb = std::max(xb, align_up((size_t)c.M * m.K * 4, 256));
+    yb = std::max(yb, align_up((size_t)c.M * m.N * 4, 256));
+  }
+  *bytes = align_up(core, 256) + 2 * xb + 2 * yb;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+  if (calls == nullptr || workspace == nullptr) return LQER_ERR_NULL;
+  if (n_calls < 0) return LQER_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
+  size_t core = kStatusBytes, xb = 0, yb = 0;
+  for (int i = 0; i < n_calls; ++i) {
+    const lqer_call_t& c = calls[i];
+    if (c.X == nullptr || c.Y == nullptr || c.packed == nullptr) return LQER_ERR_NULL;
+    if (c.M <= 0 || c.M > (1 << 24)) return LQER_ERR_SHAPE;
+    PackedMeta m;
+    lqer_status_t st = lookup(c.packed, m);
+    if (st != LQER_OK) return st;
+    core = std::max(core, workspace_total(m, c.M));
+    xb = std::max(xb, align_up((size_t)c.M * m.K * 4, 256));
+    yb = std::max(yb, align_up((size_t)c.M * m.N * 4, 256));
+  }
+  core = align_up(core, 256);
+  if (workspace_bytes < core + 2 * xb + 2 * yb) return LQER_ERR_BUFFER_TOO_SMALL;
+  if (n_calls == 0) return LQER_OK;
+  HostPipe* hp = host_pipe();
+  if (hp == nullptr) return LQER_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* Xd[2] = {reinterpret_cast<float*>(ws + core), reinterpret_cast<float*>(ws + core + xb)};
+  float* Yd[2] = {reinterpret_cast<float*>(ws + core + 2 * xb), reinterpret_cast<float*>(ws + core + 2 * xb + yb)};
+  bool ok = cudaEventRecord(hp->start, s) == cudaSuccess &&          // earlier work on `stream` may still use the workspace
+            cudaStreamWaitEvent(hp->in, hp->start, 0) == cudaSuccess &&
+            cudaStreamWaitEvent(hp->out, hp->start, 0) == cudaSuccess;
+  lqer_status_t result = ok ? LQER_OK : LQER_ERR_CUDA;
+  for (int i = 0; i < n_calls && result == LQER_OK; ++i) {
+    const lqer_call_t& c = calls[i];
+    const int b = i & 1;
+    PackedMeta m;
+    lookup(c.packed, m);
+    // copy in: the buffer is free once the layer two calls back has run
+    ok = (i < 2 || cudaStreamWaitEvent(hp->in, hp->comp_done[b], 0) == cudaSuccess) &&
+         cudaMemcpyAsync(Xd[b], c.X, (size_t)c.M * m.K * 4, cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
+         cudaEventRecord(hp->in_done[b], hp->in) == cudaSuccess &&
+         // the layer: after its X has landed and after the Y buffer's previous contents have left
+         cudaStreamWaitEvent(s, hp->in_done[b], 0) == cudaSuccess &&
+         (i < 2 || cudaStreamWaitEvent(s, hp->out_done[b], 0) == cudaSuccess);
+    if (!ok) { result = LQER_ERR_CUDA; break; }
+    result = lqer_linear_stream(Xd[b], c.M, c.packed, Yd[b], workspace, core, stream);
+    if (result != LQER_OK) break;
+    ok = cudaEventRecord(hp->comp_done[b], s) == cudaSuccess &&
+         cudaStreamWaitEvent(hp->out, hp->comp_done[b], 0) == cudaSuccess &&
+         cudaMemcpyAsync(c.Y, Yd[b], (size_t)c.M * m.N * 4, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess &&
+         cudaEventRecord(hp->out_done[b], hp->out) == cudaSuccess;
+    if (!ok) result = LQER_ERR_CUDA;
+  }
+  // nothing of this call is in flight when it returns, whatever happened
+  const bool drained = cudaStreamSynchronize(hp->in) == cudaSuccess && cudaStreamSynchronize(s) == cudaSuccess &&
+                       cudaStreamSynchronize(hp->out) == cudaSuccess;
+  if (result == LQER_OK && !drained) result = LQER_ERR_CUDA;
+  return result;
 }
 
 lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {

@@ -303,6 +303,31 @@ def test_linear_full_size_sampled_rows(spec):
     Pg.release()
 
 
+def test_host_buffer_entry_points_match_device_calls():
+    # lqer_linear_host (one layer) and lqer_linear_host_batched (copies and layers pipelined, buffers alternate)
+    # against the device entry point on the same inputs; five calls so that every buffer is reused
+    specs = [MID_SPECS[0], MID_SPECS[2], SMALL_SPECS[1], MID_SPECS[0], MID_SPECS[1]]
+    Ms = [300, 3, 37, 1, 129]
+    layers = [_prepare(s, "jacobi" if s.K <= 320 else "subspace") for s in specs]
+    Xs = [torch.from_numpy(gen.make_activations(s, M=M)).pin_memory() for s, M in zip(specs, Ms)]
+    Ys = [torch.full((M, s.N), float("nan")).pin_memory() for s, M in zip(specs, Ms)]
+    calls = L.make_host_calls([(x, lay[4], y) for x, lay, y in zip(Xs, layers, Ys)])
+    ws = torch.zeros(L.linear_host_batched_bytes(calls), dtype=torch.uint8, device=DEV)
+    L.linear_host_batched(calls, ws)
+    assert L.poll_status(ws) == 0
+    for s, M, lay, x, y in zip(specs, Ms, layers, Xs, Ys):
+        wd = L.new_workspace(M, lay[4])
+        yd = L.linear(x.to(DEV), lay[4], wd).cpu()
+        assert torch.equal(y, yd), s.name
+        y1 = torch.empty_like(y)
+        wh = L.new_workspace(M, lay[4], extra_bytes=4 * M * (s.K + s.N) + 1024)
+        L.linear_host(x, lay[4], wh, y1)
+        assert torch.equal(y1, yd), s.name
+    assert worst_ratio(Ys[0].numpy(), olqer.forward(Xs[0].numpy(), layers[0][3])) <= 1.0
+    for lay in layers:
+        lay[4].release()
+
+
 def test_stack_linears_batched_decode_and_prefill():
     # the q, gate and down linears of one decoder layer of the 7B stack through lqer_linear_batched on one
     # workspace: M = 1 (decode kernels) and then M = 2048 (prologue + GEMM), as bench.py runs them
