@@ -303,6 +303,25 @@ def test_linear_full_size_sampled_rows(spec):
     Pg.release()
 
 
+@pytest.mark.parametrize("which", [0, 6], ids=["q_4096x4096", "down_11008x4096"])
+def test_full_size_projection_bit_exact_on_sampled_rows(which):
+    # the bench's prefill configuration (M = 2048, rank 32): T_q of the tensor-core prologue, bit for bit, on one
+    # seeded row of every 128-row tile plus the first and last row (a row of T depends only on the same row of X)
+    spec = gen.config_stack(0, which, 2048)
+    P, Pg = _random_factor_layer(spec)
+    X = gen.make_activations(spec)
+    g = np.random.default_rng(spec.seed)
+    rows = sorted({0, spec.M - 1} | {int(t * 128 + g.integers(0, 128)) for t in range(spec.M // 128)})
+    ref = olqer.forward(X[rows], P)
+    ws = L.new_workspace(spec.M, Pg)
+    Tm, Te = L.project_lowrank(_t(X), Pg, ws)
+    assert L.poll_status(ws) == 0
+    idx = torch.tensor(rows, device=DEV)
+    assert np.array_equal(Tm[idx].cpu().numpy(), ref.Tm)
+    assert np.array_equal(Te[idx].cpu().numpy(), exp_bytes(ref.Te))
+    Pg.release()
+
+
 def test_host_buffer_entry_points_match_device_calls():
     # lqer_linear_host (one layer) and lqer_linear_host_batched (copies and layers pipelined, buffers alternate)
     # against the device entry point on the same inputs; five calls so that every buffer is reused
