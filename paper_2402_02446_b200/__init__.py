@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     new_workspace,
     linear,
     linear_batched,
+    batched_workspace_bytes,
     linear_static,
     linear_host,
     linear_host_batched,

@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
             "lqer_linear_stream": (i, [vp, i, vp, vp, vp, sz, vp]),
             "lqer_linear_static": (i, [vp, i, vp, vp, vp]),
             "lqer_linear_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
+            "lqer_batched_workspace_bytes": (i, [C.POINTER(Call), i, C.POINTER(sz)]),
             "lqer_linear_host": (i, [vp, i, vp, vp, vp, sz, vp]),
             "lqer_linear_host_batched_bytes": (i, [C.POINTER(Call), i, C.POINTER(sz)]),
             "lqer_linear_host_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
@@ -233,6 +234,14 @@ def make_calls(items) -> "C.Array":
     for j, (X, P, Y) in enumerate(items):
         arr[j] = Call(_dev(X, torch.float32), X.shape[0], P.ptr, _dev(Y, torch.float32))
     return arr
+
+
+def batched_workspace_bytes(calls) -> int:
+    """Workspace size with which lqer_linear_batched can run same-shape neighbours in shared launches."""
+    arr = calls if isinstance(calls, C.Array) else make_calls(calls)
+    out = C.c_size_t()
+    _check(lib().lqer_batched_workspace_bytes(arr, len(arr), C.byref(out)), "lqer_batched_workspace_bytes")
+    return out.value
 
 
 def linear_batched(calls, ws: torch.Tensor, stream=None) -> None:

@@ -172,6 +172,45 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
   return err == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
 
+// Scratch one layer of a grouped prefill launch needs: its own Xcat and its own prologue partial sums.
+static size_t group_slice_bytes(const PackedMeta& m, int M) {
+  return xcat_bytes(m, M) + align_up(prologue_tc_scratch_bytes(m, M), 256);
+}
+// Consecutive calls from `first` on that may share launches with it (auto path only): same M, same shape,
+// at most `limit` of them.
+static int same_shape_run(const lqer_call_t* calls, int first, int n_calls, const PackedMeta& m0, int limit) {
+  int n = 1;
+  while (first + n < n_calls && n < limit) {
+    PackedMeta m1;
+    if (calls[first + n].M != calls[first].M || lookup(calls[first + n].packed, m1) != LQER_OK || !same_shape(m0, m1)) break;
+    ++n;
+  }
+  return n;
+}
+// n prefill layers of one shape: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
+// the tiles of all of them.
+static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const PackedMeta& m, void* workspace, cudaStream_t s) {
+  const int M = calls[0].M;
+  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
+  const size_t slice = group_slice_bytes(m, M);
+  const void* xcats[8];
+  const void* packed[8];
+  float* Ys[8];
+  for (int g = 0; g < n; ++g) {
+    uint8_t* xcat = wsb + align_up(persist_bytes(m), 256) + (size_t)g * slice;
+    const float* X = calls[g].X;
+    cudaError_t err = prologue_tc_fits(m, M, X, false)
+                          ? launch_prologue_tc(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
+                                               reinterpret_cast<double*>(xcat + xcat_bytes(m, M)),
+                                               reinterpret_cast<int*>(wsb + pcount_offset(m)), s)
+                          : launch_prologue(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
+    if (err != cudaSuccess) return LQER_ERR_CUDA;
+    xcats[g] = xcat; packed[g] = calls[g].packed; Ys[g] = calls[g].Y;
+  }
+  return launch_gemm_tc2_group(xcats, packed, Ys, n, M, m, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+}
+
 }  // namespace lqer
 
 using namespace lqer;
@@ -351,23 +390,31 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
   }
   const bool may_group = g_path.load() == 0;   // a forced path runs every call on its own
   for (int i = 0; i < n_calls;) {
-    // The calls are independent, so consecutive decode calls of one shape (the q, k, v projections of a layer, or
-    // its gate and up projections) share a launch: the column-owner decode kernel keeps nothing in the workspace.
+    // The calls are independent, so consecutive calls of one shape (the q, k, v projections of a layer, or its gate
+    // and up projections) share launches: decode calls one launch of the column-owner kernel (it keeps nothing in the
+    // workspace), prefill calls one GEMM launch after their prologues, if the workspace has a slice for each.
     int n = 1;
     PackedMeta m0;
-    if (may_group && lookup(calls[i].packed, m0) == LQER_OK && decode_cols_fits(m0, calls[i].M)) {
-      while (i + n < n_calls && n < decode_cols_max_group()) {
-        PackedMeta m1;
-        if (calls[i + n].M != calls[i].M || lookup(calls[i + n].packed, m1) != LQER_OK || !same_shape(m0, m1)) break;
-        ++n;
+    bool decode_group = false;
+    if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
+      if (decode_cols_fits(m0, calls[i].M)) {
+        n = same_shape_run(calls, i, n_calls, m0, decode_cols_max_group());
+        decode_group = n > 1;
+      } else if (calls[i].M > 128) {
+        n = same_shape_run(calls, i, n_calls, m0, gemm_tc2_max_group());
+        while (n > 1 && workspace_bytes < align_up(persist_bytes(m0), 256) + (size_t)n * group_slice_bytes(m0, calls[i].M)) --n;
       }
     }
     if (n > 1) {
       lqer_status_t st = check_arch();
       if (st != LQER_OK) return st;
       if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
-      if (launch_decode_cols_group(calls + i, n, m0, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-        return LQER_ERR_CUDA;
+      if (decode_group) {
+        if (launch_decode_cols_group(calls + i, n, m0, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+          return LQER_ERR_CUDA;
+      } else if ((st = run_prefill_group(calls + i, n, m0, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) {
+        return st;
+      }
     } else {
       lqer_status_t st = lqer_linear_stream(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace,
                                             workspace_bytes, stream);
@@ -375,6 +422,29 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     }
     i += n;
   }
+  return LQER_OK;
+}
+
+lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes) {
+  if (calls == nullptr || bytes == nullptr) return LQER_ERR_NULL;
+  if (n_calls < 0) return LQER_ERR_SHAPE;
+  size_t need = kStatusBytes;
+  for (int i = 0; i < n_calls;) {
+    const lqer_call_t& c = calls[i];
+    if (c.packed == nullptr) return LQER_ERR_NULL;
+    if (c.M <= 0 || c.M > (1 << 24)) return LQER_ERR_SHAPE;
+    PackedMeta m;
+    lqer_status_t st = lookup(c.packed, m);
+    if (st != LQER_OK) return st;
+    need = std::max(need, workspace_total(m, c.M));
+    int n = 1;
+    if (c.M > 128 && !decode_cols_fits(m, c.M)) {
+      n = same_shape_run(calls, i, n_calls, m, gemm_tc2_max_group());
+      need = std::max(need, align_up(persist_bytes(m), 256) + (size_t)n * group_slice_bytes(m, c.M));
+    }
+    i += n;
+  }
+  *bytes = need;
   return LQER_OK;
 }
 

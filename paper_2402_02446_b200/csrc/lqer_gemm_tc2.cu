@@ -50,10 +50,17 @@ static_assert(PK_OFFSET + kWTileBytes <= STAGE_BYTES && STAGE_BYTES % 1024 == 0,
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 static_assert(STAGES % CONVERTER_GROUPS == 0, "a converter group must revisit a ring slot exactly one pass later");
 
+constexpr int MAX_GROUP = 4;               // independent layers of one shape and one M that may share a launch
+
+struct TensorMaps {                        // one activation map per layer of the group
+  CUtensorMap m[MAX_GROUP];
+};
+
 struct Params {
-  const uint8_t* wsec;
-  const uint8_t* bsec;
-  float* Y;
+  const uint8_t* wsec[MAX_GROUP];
+  const uint8_t* bsec[MAX_GROUP];
+  float* Y[MAX_GROUP];
+  int group;                   // layers in this launch; the tiles of layer g are g * tiles_per_layer ...
   DeviceStatus* status;
   int M, N, K64;
   int n_tiles, k_slabs, r_blocks;
@@ -62,7 +69,7 @@ struct Params {
 };
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
+gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stage_base = smem;
@@ -105,7 +112,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
 
   const int rank_stages = (p.r_blocks + 1) / 2;
   const int stages_per_tile = p.k_slabs + rank_stages;
-  const int num_tiles = p.m_tiles * p.n256_tiles;
+  const int tiles_per_layer = p.m_tiles * p.n256_tiles;
+  const int num_tiles = p.group * tiles_per_layer;
   const int b_tile_stride = p.r_blocks * kTileN * 17;
 
   if (warp == 0) {
@@ -115,7 +123,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
       uint32_t ph = 0;
       bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs) {
-        const int mt = t % p.m_tiles, nt = t / p.m_tiles;
+        const int layer = t / tiles_per_layer, tl = t - layer * tiles_per_layer;
+        const int mt = tl % p.m_tiles, nt = tl / p.m_tiles;
+        const CUtensorMap* tmap_x = &tmaps.m[layer];
+        const uint8_t* wsec = p.wsec[layer];
+        const uint8_t* bsec = p.bsec[layer];
         const int my_ntile = 2 * nt + (int)rank;
         const bool has_w = my_ntile < p.n_tiles;
         const int row0 = mt * 2 * BM + (int)rank * BM;
@@ -124,17 +136,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
           const uint32_t a_dst = smem_u32(stage_base + st * STAGE_BYTES);
           if (s < p.k_slabs) {
             mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? kWTileBytes : 0));
-            tma_load_2d(a_dst, &tmap_x, s * BK, row0, loaded(st));
+            tma_load_2d(a_dst, tmap_x, s * BK, row0, loaded(st));
             if (has_w)
-              bulk_load(a_dst + PK_OFFSET, p.wsec + ((size_t)my_ntile * p.k_slabs + s) * kWTileBytes, kWTileBytes,
+              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * p.k_slabs + s) * kWTileBytes, kWTileBytes,
                         loaded(st));
           } else {
             const int rs = s - p.k_slabs;
             const int rb0 = rs * 2, nb = min(2, p.r_blocks - rb0);
             mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? nb * (kTileN * 17) : 0));
-            tma_load_2d(a_dst, &tmap_x, p.K64 + rs * RANK_PER_STAGE, row0, loaded(st));
+            tma_load_2d(a_dst, tmap_x, p.K64 + rs * RANK_PER_STAGE, row0, loaded(st));
             if (has_w) {
-              const uint8_t* tile = p.bsec + (size_t)my_ntile * b_tile_stride;
+              const uint8_t* tile = bsec + (size_t)my_ntile * b_tile_stride;
               bulk_load(a_dst + PK_OFFSET, tile + (size_t)rb0 * kTileN * 16, nb * kTileN * 16, loaded(st));
               bulk_load(a_dst + PK_OFFSET + 4096, tile + (size_t)p.r_blocks * kTileN * 16 + rb0 * kTileN,
                         nb * kTileN, loaded(st));
@@ -214,13 +226,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
     uint32_t tile_it = 0;
     bool ok = true;
     for (int t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
-      const int mt = t % p.m_tiles, nt = t / p.m_tiles;
+      const int layer = t / tiles_per_layer, tl = t - layer * tiles_per_layer;
+      const int mt = tl % p.m_tiles, nt = tl / p.m_tiles;
       const int acc = tile_it & 1;
       if (!mbar_wait<true>(acc_full(acc), (tile_it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row = mt * 2 * BM + (int)rank * BM + q * 32 + lane;
       const int ncols = min(BN, p.N - nt * BN);
-      float* yrow = p.Y + (size_t)row * p.N + (size_t)nt * BN;
+      float* yrow = p.Y[layer] + (size_t)row * p.N + (size_t)nt * BN;
       for (int c = 0; c < BN; c += 32) {
         if (c >= ncols) break;
         uint32_t r[32];
@@ -253,7 +266,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
     bool ok = true;
     for (long long it = group; it < total && ok; it += CONVERTER_GROUPS, s += CONVERTER_GROUPS) {
       while (s >= stages_per_tile) { s -= stages_per_tile; ++tile_i; }
-      const int nt = (pair + tile_i * num_pairs) / p.m_tiles;
+      const int nt = ((pair + tile_i * num_pairs) % tiles_per_layer) / p.m_tiles;
       const bool has_w = 2 * nt + (int)rank < p.n_tiles;
       const int st = (int)(it % STAGES);
       const uint32_t ph = (uint32_t)((it / STAGES) & 1);
@@ -339,18 +352,30 @@ static EncodeTiledFn encode_fn() {
 
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s) {
+  return launch_gemm_tc2_group(&xcat, &packed, &Y, 1, M, m, st, s);
+}
+
+int gemm_tc2_max_group() { return tc2::MAX_GROUP; }
+
+// n layers of one shape (same K, N, rank, formats) and one M as ONE launch: the tiles of all layers form one list
+// that the CTA pairs walk, so the pairs idle only at the end of the whole list, and set-up and the last epilogue
+// are paid once.
+cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys, int n, int M,
+                                  const PackedMeta& m, DeviceStatus* st, cudaStream_t s) {
   using namespace tc2;
+  if (n < 1 || n > MAX_GROUP) return cudaErrorInvalidValue;
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
-  CUtensorMap tmap;
+  TensorMaps tmaps;
   const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
   const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
   const cuuint32_t box[2] = {BK, BM};
   const cuuint32_t estr[2] = {1, 1};
-  if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xcat), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorInvalidValue;
+  for (int g = 0; g < MAX_GROUP; ++g)
+    if (enc(&tmaps.m[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xcats[g < n ? g : 0]), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
 
   static int sm_count = 0;
   static bool attr_set = false;
@@ -363,17 +388,20 @@ cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const 
     attr_set = true;
   }
   Params p;
-  const uint8_t* base = static_cast<const uint8_t*>(packed);
-  p.wsec = base + m.off_w;
-  p.bsec = base + m.off_b;
-  p.Y = Y;
+  for (int g = 0; g < MAX_GROUP; ++g) {
+    const uint8_t* base = static_cast<const uint8_t*>(packed[g < n ? g : 0]);
+    p.wsec[g] = base + m.off_w;
+    p.bsec[g] = base + m.off_b;
+    p.Y[g] = Ys[g < n ? g : 0];
+  }
+  p.group = n;
   p.status = st;
   p.M = M; p.N = m.N; p.K64 = m.K64;
   p.n_tiles = m.n_tiles; p.k_slabs = m.k_slabs; p.r_blocks = m.r_blocks;
   p.m_tiles = (M + 2 * BM - 1) / (2 * BM);
   p.n256_tiles = (m.n_tiles + 1) / 2;
   p.lr_shift = m.lr_bits - 2;
-  const int num_tiles = p.m_tiles * p.n256_tiles;
+  const int num_tiles = n * p.m_tiles * p.n256_tiles;
   const int max_pairs = sm_count / 2;
   const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
 
@@ -390,7 +418,7 @@ cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const 
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   LaunchScope scope(kFamGemmTcPair, s);
-  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, tmap, p);
+  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, tmaps, p);
 }
 
 }  // namespace lqer

@@ -322,6 +322,40 @@ def test_full_size_projection_bit_exact_on_sampled_rows(which):
     Pg.release()
 
 
+def test_batched_prefill_groups_same_shape_calls():
+    # five independent prefill calls of one shape (a group of four and a fifth) and two of another: with a workspace
+    # of lqer_batched_workspace_bytes the groups share GEMM launches; every tile is computed as in a single call
+    spec_a = gen.LayerSpec("pgrp_a", M=300, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=61)
+    spec_b = gen.LayerSpec("pgrp_b", M=1100, K=512, N=1280, k=32, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=62)
+    layers = []
+    for i, spec in enumerate([spec_a] * 5 + [spec_b] * 2):
+        sp = gen.LayerSpec(f"{spec.name}{i}", M=spec.M, K=spec.K, N=spec.N, k=spec.k, calib_rows=spec.calib_rows,
+                           outlier_frac=spec.outlier_frac, outlier_scale=spec.outlier_scale, seed=spec.seed + i)
+        layers.append((sp,) + _random_factor_layer(sp))
+    Xs = [_t(gen.make_activations(sp)) for sp, _, _ in layers]
+    Yb = [torch.full((sp.M, sp.N), float("nan"), dtype=torch.float32, device=DEV) for sp, _, _ in layers]
+    calls = L.make_calls([(x, lay[2], y) for x, lay, y in zip(Xs, layers, Yb)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    launches = L.launch_count()
+    L.linear_batched(calls, ws)
+    torch.cuda.synchronize()
+    assert L.poll_status(ws) == 0
+    assert L.launch_count() - launches == 7 + 3         # seven prologues; GEMMs: 4 + 1 of the first shape, 2 of the second
+    for x, (sp, P, Pg), yb in zip(Xs, layers, Yb):
+        ys = L.linear(x, Pg, ws)
+        assert torch.equal(ys, yb), sp.name              # same tiles, same arithmetic
+    sp, P, Pg = layers[5]
+    assert worst_ratio(Yb[5].cpu().numpy(), olqer.forward(Xs[5].cpu().numpy(), P)) <= 1.0
+    # a workspace that only fits single calls: no sharing, same results
+    ws1 = torch.zeros(max(L.workspace_bytes(sp.M, sp.K, sp.N, sp.k) for sp, _, _ in layers), dtype=torch.uint8, device=DEV)
+    Y1 = [torch.empty_like(y) for y in Yb]
+    L.linear_batched([(x, lay[2], y) for x, lay, y in zip(Xs, layers, Y1)], ws1)
+    for y1, yb in zip(Y1, Yb):
+        assert torch.equal(y1, yb)
+    for _, _, Pg in layers:
+        Pg.release()
+
+
 def test_host_buffer_entry_points_match_device_calls():
     # lqer_linear_host (one layer) and lqer_linear_host_batched (copies and layers pipelined, buffers alternate)
     # against the device entry point on the same inputs; five calls so that every buffer is reused
