@@ -305,7 +305,7 @@ def run_ours(args) -> None:
     dom_launches, dom_ms = fam[dominant]
     roofline = None
     if dominant.startswith("gemm"):
-        # every M=2048 linear goes through this kernel, same-shape neighbours (q,k,v,o; gate,up) in one launch;
+        # every M=2048 linear goes through this kernel, up to eight neighbours in one launch;
         # algorithmic flops per launch = all of them / the launches counted
         flops_per_launch = sum(2.0 * M_PREFILL * (K + k) * N for K, N, k, _ in shapes) / dom_launches
         achieved = flops_per_launch / (dom_ms / dom_launches * 1e-3) / 1e12
@@ -368,10 +368,10 @@ def run_ours(args) -> None:
             "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
             "config": {"workload": WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]",
                        "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32,
-                       "shared_launches": "lqer_linear_batched runs consecutive independent same-shape calls (q,k,v,o; "
-                                          "gate,up) together: decode as one launch that divides the SMs among the layers "
-                                          "(3 launches per decoder layer of 7 linears), prefill as one prologue per layer "
-                                          "and one GEMM launch over the tiles of the group",
+                       "shared_launches": "lqer_linear_batched runs consecutive independent calls together: decode calls "
+                                          "of one shape (q,k,v,o; gate,up) as one launch that divides the SMs among the "
+                                          "layers (3 launches per decoder layer of 7 linears), prefill calls as one "
+                                          "prologue per layer and one GEMM launch over the tiles of up to 8 layers",
                        "l2": "inputs larger than L2: every linear has its own packed weights and activations "
                              f"({sum(p.buf.numel() for p in packed) / 1e9:.2f} GB of weights per step)",
                        "parallelism": "replicas (independent token batches)" if world > 1 else "1 GPU"},

@@ -162,9 +162,10 @@ lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, floa
  * fit the largest of them.  Independent means that no call reads what another call of the
  * same batch writes: with the path left at 0, up to four consecutive calls with M <= 4 and
  * packed buffers of one shape (K, N, rank, formats) run as ONE launch that divides the SMs
- * among them (the q, k, v or the gate and up projections of a decoder layer), and up to four
- * consecutive calls with one M > 128 and one shape run their prologues into separate slices of
- * the workspace and then ONE GEMM launch over the tiles of all of them - if the workspace holds
+ * among them (the q, k, v or the gate and up projections of a decoder layer), and up to eight
+ * consecutive calls with one M > 128 (any shapes, one set of formats) run their prologues into
+ * separate slices of the workspace and then ONE GEMM launch over the tiles of all of them - if
+ * the workspace holds
  * lqer_batched_workspace_bytes(calls, n_calls); with a smaller workspace (at least the largest
  * lqer_workspace_bytes of the calls) they run one after the other. */
 lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes);

@@ -187,18 +187,47 @@ static int same_shape_run(const lqer_call_t* calls, int first, int n_calls, cons
   }
   return n;
 }
-// n prefill layers of one shape: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
+// Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M > 128,
+// the same formats, any shapes; at most `limit`, and only as many as the workspace has slices for.
+static bool same_formats(const PackedMeta& a, const PackedMeta& b) {
+  return a.w_bits == b.w_bits && a.a_bits == b.a_bits && a.lr_bits == b.lr_bits && a.exp_min == b.exp_min &&
+         a.exp_max == b.exp_max && a.block == b.block;
+}
+static int prefill_run(const lqer_call_t* calls, int first, int n_calls, int limit, size_t workspace_bytes,
+                       PackedMeta* metas, size_t* need) {
+  const int M = calls[first].M;
+  size_t head = 0, slices = 0;
+  int n = 0;
+  while (first + n < n_calls && n < limit) {
+    PackedMeta m;
+    if (calls[first + n].M != M || lookup(calls[first + n].packed, m) != LQER_OK) break;
+    if (n > 0 && !same_formats(metas[0], m)) break;
+    const size_t h = std::max(head, align_up(persist_bytes(m), 256));
+    const size_t sl = slices + group_slice_bytes(m, M);
+    if (n > 0 && h + sl > workspace_bytes) break;
+    metas[n] = m; head = h; slices = sl;
+    ++n;
+  }
+  if (need != nullptr) *need = head + slices;
+  return n;
+}
+// n prefill layers with one M: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
 // the tiles of all of them.
-static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const PackedMeta& m, void* workspace, cudaStream_t s) {
+static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace,
+                                       cudaStream_t s) {
   const int M = calls[0].M;
   uint8_t* wsb = static_cast<uint8_t*>(workspace);
   DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
-  const size_t slice = group_slice_bytes(m, M);
+  size_t head = 0;
+  for (int g = 0; g < n; ++g) head = std::max(head, align_up(persist_bytes(metas[g]), 256));
   const void* xcats[8];
   const void* packed[8];
   float* Ys[8];
+  size_t off = head;
   for (int g = 0; g < n; ++g) {
-    uint8_t* xcat = wsb + align_up(persist_bytes(m), 256) + (size_t)g * slice;
+    const PackedMeta& m = metas[g];
+    uint8_t* xcat = wsb + off;
+    off += group_slice_bytes(m, M);
     const float* X = calls[g].X;
     cudaError_t err = prologue_tc_fits(m, M, X, false)
                           ? launch_prologue_tc(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
@@ -208,7 +237,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
     if (err != cudaSuccess) return LQER_ERR_CUDA;
     xcats[g] = xcat; packed[g] = calls[g].packed; Ys[g] = calls[g].Y;
   }
-  return launch_gemm_tc2_group(xcats, packed, Ys, n, M, m, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+  return launch_gemm_tc2_group(xcats, packed, Ys, metas, n, M, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
 
 }  // namespace lqer
@@ -394,15 +423,15 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     // and up projections) share launches: decode calls one launch of the column-owner kernel (it keeps nothing in the
     // workspace), prefill calls one GEMM launch after their prologues, if the workspace has a slice for each.
     int n = 1;
-    PackedMeta m0;
+    PackedMeta m0, metas[8];
     bool decode_group = false;
     if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
       if (decode_cols_fits(m0, calls[i].M)) {
         n = same_shape_run(calls, i, n_calls, m0, decode_cols_max_group());
         decode_group = n > 1;
       } else if (calls[i].M > 128) {
-        n = same_shape_run(calls, i, n_calls, m0, gemm_tc2_max_group());
-        while (n > 1 && workspace_bytes < align_up(persist_bytes(m0), 256) + (size_t)n * group_slice_bytes(m0, calls[i].M)) --n;
+        n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), workspace_bytes, metas, nullptr);
+        if (n < 1) n = 1;
       }
     }
     if (n > 1) {
@@ -412,7 +441,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
       if (decode_group) {
         if (launch_decode_cols_group(calls + i, n, m0, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
           return LQER_ERR_CUDA;
-      } else if ((st = run_prefill_group(calls + i, n, m0, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) {
+      } else if ((st = run_prefill_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) {
         return st;
       }
     } else {
@@ -439,8 +468,11 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
     need = std::max(need, workspace_total(m, c.M));
     int n = 1;
     if (c.M > 128 && !decode_cols_fits(m, c.M)) {
-      n = same_shape_run(calls, i, n_calls, m, gemm_tc2_max_group());
-      need = std::max(need, align_up(persist_bytes(m), 256) + (size_t)n * group_slice_bytes(m, c.M));
+      PackedMeta metas[8];
+      size_t group_need = 0;
+      n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), ~(size_t)0, metas, &group_need);
+      if (n < 1) n = 1;
+      need = std::max(need, group_need);
     }
     i += n;
   }

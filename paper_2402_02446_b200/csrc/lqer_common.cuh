@@ -237,10 +237,10 @@ cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const v
                            DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s);
-// Up to gemm_tc2_max_group() layers of one shape and one M in one launch (xcats, packed, Ys: host arrays of n pointers).
+// Up to gemm_tc2_max_group() layers with one M in one launch (xcats, packed, Ys, metas: host arrays of n entries).
 int gemm_tc2_max_group();
-cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys, int n, int M,
-                                  const PackedMeta& m, DeviceStatus* st, cudaStream_t s);
+cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys,
+                                  const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s);
 // M <= 4 goes to the column-owner kernel unless force_split_k (test hook: the split-K kernel serves every M <= 16).
 cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
                           void* workspace, cudaStream_t s, bool force_split_k = false);

@@ -50,23 +50,38 @@ static_assert(PK_OFFSET + kWTileBytes <= STAGE_BYTES && STAGE_BYTES % 1024 == 0,
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 static_assert(STAGES % CONVERTER_GROUPS == 0, "a converter group must revisit a ring slot exactly one pass later");
 
-constexpr int MAX_GROUP = 4;               // independent layers of one shape and one M that may share a launch
+constexpr int MAX_GROUP = 8;               // independent layers with one M that may share a launch
 
 struct TensorMaps {                        // one activation map per layer of the group
   CUtensorMap m[MAX_GROUP];
 };
 
-struct Params {
-  const uint8_t* wsec[MAX_GROUP];
-  const uint8_t* bsec[MAX_GROUP];
-  float* Y[MAX_GROUP];
-  int group;                   // layers in this launch; the tiles of layer g are g * tiles_per_layer ...
-  DeviceStatus* status;
-  int M, N, K64;
+struct Layer {
+  const uint8_t* wsec;
+  const uint8_t* bsec;
+  float* Y;
+  int N, K64;
   int n_tiles, k_slabs, r_blocks;
-  int m_tiles, n256_tiles;     // pair tiles: 256 rows x 256 columns
+  int spt;                     // K stages per tile: k_slabs + rank stages
+  int tile_begin;              // first tile of this layer in the launch's list (256 x 256 tiles, row tile fastest)
+};
+
+struct Params {
+  Layer L[MAX_GROUP];          // ordered by falling spt: the long tiles run first, the short ones fill the end
+  int group;                   // layers in this launch
+  int num_tiles;               // tiles of all layers
+  DeviceStatus* status;
+  int M, m_tiles;              // row tiles of 256 (the same M for every layer)
   int lr_shift;
 };
+
+__device__ __forceinline__ int layer_of(const Params& p, int t) {
+  int l = 0;
+#pragma unroll
+  for (int i = 1; i < MAX_GROUP; ++i)
+    if (i < p.group && t >= p.L[i].tile_begin) l = i;
+  return l;
+}
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
@@ -110,11 +125,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
   pdl_launch_dependents();
   pdl_wait();
 
-  const int rank_stages = (p.r_blocks + 1) / 2;
-  const int stages_per_tile = p.k_slabs + rank_stages;
-  const int tiles_per_layer = p.m_tiles * p.n256_tiles;
-  const int num_tiles = p.group * tiles_per_layer;
-  const int b_tile_stride = p.r_blocks * kTileN * 17;
+  const int num_tiles = p.num_tiles;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (own halves)
@@ -123,32 +134,35 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       uint32_t ph = 0;
       bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs) {
-        const int layer = t / tiles_per_layer, tl = t - layer * tiles_per_layer;
+        const int layer = layer_of(p, t), tl = t - p.L[layer].tile_begin;
         const int mt = tl % p.m_tiles, nt = tl / p.m_tiles;
         const CUtensorMap* tmap_x = &tmaps.m[layer];
-        const uint8_t* wsec = p.wsec[layer];
-        const uint8_t* bsec = p.bsec[layer];
+        const uint8_t* wsec = p.L[layer].wsec;
+        const uint8_t* bsec = p.L[layer].bsec;
+        const int k_slabs = p.L[layer].k_slabs, r_blocks = p.L[layer].r_blocks, K64 = p.L[layer].K64;
+        const int stages_per_tile = p.L[layer].spt, n_tiles = p.L[layer].n_tiles;
+        const int b_tile_stride = r_blocks * kTileN * 17;
         const int my_ntile = 2 * nt + (int)rank;
-        const bool has_w = my_ntile < p.n_tiles;
+        const bool has_w = my_ntile < n_tiles;
         const int row0 = mt * 2 * BM + (int)rank * BM;
         for (int s = 0; s < stages_per_tile; ++s) {
           if (!mbar_wait<true>(freed(st), ph ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = smem_u32(stage_base + st * STAGE_BYTES);
-          if (s < p.k_slabs) {
+          if (s < k_slabs) {
             mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? kWTileBytes : 0));
             tma_load_2d(a_dst, tmap_x, s * BK, row0, loaded(st));
             if (has_w)
-              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * p.k_slabs + s) * kWTileBytes, kWTileBytes,
+              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * k_slabs + s) * kWTileBytes, kWTileBytes,
                         loaded(st));
           } else {
-            const int rs = s - p.k_slabs;
-            const int rb0 = rs * 2, nb = min(2, p.r_blocks - rb0);
+            const int rs = s - k_slabs;
+            const int rb0 = rs * 2, nb = min(2, r_blocks - rb0);
             mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? nb * (kTileN * 17) : 0));
-            tma_load_2d(a_dst, tmap_x, p.K64 + rs * RANK_PER_STAGE, row0, loaded(st));
+            tma_load_2d(a_dst, tmap_x, K64 + rs * RANK_PER_STAGE, row0, loaded(st));
             if (has_w) {
               const uint8_t* tile = bsec + (size_t)my_ntile * b_tile_stride;
               bulk_load(a_dst + PK_OFFSET, tile + (size_t)rb0 * kTileN * 16, nb * kTileN * 16, loaded(st));
-              bulk_load(a_dst + PK_OFFSET + 4096, tile + (size_t)p.r_blocks * kTileN * 16 + rb0 * kTileN,
+              bulk_load(a_dst + PK_OFFSET + 4096, tile + (size_t)r_blocks * kTileN * 16 + rb0 * kTileN,
                         nb * kTileN, loaded(st));
             }
           }
@@ -166,6 +180,8 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       const uint64_t b_desc0 = make_desc(smem_u32(stage_base + A_TILE_BYTES));
       bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
+        const int layer = layer_of(p, t);
+        const int k_slabs = p.L[layer].k_slabs, r_blocks = p.L[layer].r_blocks, stages_per_tile = p.L[layer].spt;
         const int acc = tile_it & 1;
         if (!mbar_wait(acc_empty(acc), ((tile_it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -176,7 +192,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           const uint64_t b_desc = b_desc0 + (uint64_t)(st * (STAGE_BYTES >> 4));
           const uint32_t first = s > 0 ? 1u : 0u;
           const uint32_t free_bar = freed(st);
-          if (s + ROUND <= p.k_slabs) {
+          if (s + ROUND <= k_slabs) {
             // ROUND 64-K stages per round of the issuing thread: the poll of a barrier and the loop cost
             // about as much as one MMA takes the tensor pipe, so they are paid once per 4 * ROUND MMAs.
             int sr = st;
@@ -204,13 +220,13 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           }
           if (!mbar_wait(ready(st), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          if (s < p.k_slabs) {           // 64 K = four MMAs
+          if (s < k_slabs) {           // 64 K = four MMAs
             umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, first);
             umma_bf16_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
             umma_bf16_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
             umma_bf16_pair(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
           } else {
-            const int nk = min(2, p.r_blocks - (s - p.k_slabs) * 2);
+            const int nk = min(2, r_blocks - (s - k_slabs) * 2);
             for (int j = 0; j < nk; ++j) umma_bf16_pair(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, 1u);
           }
           umma_commit_pair(free_bar);
@@ -226,14 +242,15 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
     uint32_t tile_it = 0;
     bool ok = true;
     for (int t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
-      const int layer = t / tiles_per_layer, tl = t - layer * tiles_per_layer;
+      const int layer = layer_of(p, t), tl = t - p.L[layer].tile_begin;
       const int mt = tl % p.m_tiles, nt = tl / p.m_tiles;
+      const int Nl = p.L[layer].N;
       const int acc = tile_it & 1;
       if (!mbar_wait<true>(acc_full(acc), (tile_it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row = mt * 2 * BM + (int)rank * BM + q * 32 + lane;
-      const int ncols = min(BN, p.N - nt * BN);
-      float* yrow = p.Y[layer] + (size_t)row * p.N + (size_t)nt * BN;
+      const int ncols = min(BN, Nl - nt * BN);
+      float* yrow = p.L[layer].Y + (size_t)row * Nl + (size_t)nt * BN;
       for (int c = 0; c < BN; c += 32) {
         if (c >= ncols) break;
         uint32_t r[32];
@@ -260,20 +277,29 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
     uint32_t chunk[8];                           // the row's eight 16-byte chunks after the 128-byte swizzle
 #pragma unroll
     for (int i = 0; i < 8; ++i) chunk[i] = (uint32_t)(nl * 128 + ((i ^ sw) << 4));
-    const int my_tiles = pair < num_tiles ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
-    const long long total = (long long)my_tiles * stages_per_tile;
-    int tile_i = 0, s = group;                   // s may run past the tile; normalised below
+    // the pair's tiles one after the other; their K stages form one sequence of which this group takes every sixth
+    int tile = pair, s = group;                  // s may run past the tile; normalised below
+    int stages_per_tile = 0, k_slabs = 0, r_blocks = 0;
+    bool has_w = false;
+    auto enter_tile = [&]() {
+      if (tile < num_tiles) {
+        const int layer = layer_of(p, tile);
+        stages_per_tile = p.L[layer].spt; k_slabs = p.L[layer].k_slabs; r_blocks = p.L[layer].r_blocks;
+        const int nt = (tile - p.L[layer].tile_begin) / p.m_tiles;
+        has_w = 2 * nt + (int)rank < p.L[layer].n_tiles;
+      }
+    };
+    enter_tile();
     bool ok = true;
-    for (long long it = group; it < total && ok; it += CONVERTER_GROUPS, s += CONVERTER_GROUPS) {
-      while (s >= stages_per_tile) { s -= stages_per_tile; ++tile_i; }
-      const int nt = ((pair + tile_i * num_pairs) % tiles_per_layer) / p.m_tiles;
-      const bool has_w = 2 * nt + (int)rank < p.n_tiles;
-      const int st = (int)(it % STAGES);
+    for (int it = group; tile < num_tiles && ok; it += CONVERTER_GROUPS, s += CONVERTER_GROUPS) {
+      while (tile < num_tiles && s >= stages_per_tile) { s -= stages_per_tile; tile += num_pairs; enter_tile(); }
+      if (tile >= num_tiles) break;
+      const int st = it % STAGES;
       const uint32_t ph = (uint32_t)((it / STAGES) & 1);
       if (!mbar_wait(loaded(st), ph, abort_flag)) { ok = false; break; }
       const uint8_t* pk = stage_base + st * STAGE_BYTES + PK_OFFSET;
       uint8_t* bt = stage_base + st * STAGE_BYTES + A_TILE_BYTES;
-      if (s < p.k_slabs) {
+      if (s < k_slabs) {
         if (has_w) {
           const uint4 wa = *reinterpret_cast<const uint4*>(pk + nl * 16);
           const uint4 wb = *reinterpret_cast<const uint4*>(pk + (kTileN + nl) * 16);
@@ -296,7 +322,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           for (int i = 0; i < 8; ++i) *reinterpret_cast<uint4*>(bt + chunk[i]) = make_uint4(0u, 0u, 0u, 0u);
         }
       } else {
-        const int nb = min(2, p.r_blocks - (s - p.k_slabs) * 2);
+        const int nb = min(2, r_blocks - (s - k_slabs) * 2);
         for (int rb = 0; rb < nb; ++rb) {
           uint4 o0 = make_uint4(0u, 0u, 0u, 0u), o1 = o0;
           if (has_w) {
@@ -352,31 +378,20 @@ static EncodeTiledFn encode_fn() {
 
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s) {
-  return launch_gemm_tc2_group(&xcat, &packed, &Y, 1, M, m, st, s);
+  return launch_gemm_tc2_group(&xcat, &packed, &Y, &m, 1, M, st, s);
 }
 
 int gemm_tc2_max_group() { return tc2::MAX_GROUP; }
 
-// n layers of one shape (same K, N, rank, formats) and one M as ONE launch: the tiles of all layers form one list
-// that the CTA pairs walk, so the pairs idle only at the end of the whole list, and set-up and the last epilogue
-// are paid once.
-cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys, int n, int M,
-                                  const PackedMeta& m, DeviceStatus* st, cudaStream_t s) {
+// n layers with one M (shapes may differ, formats must not) as ONE launch: the tiles of all layers form one list that
+// the CTA pairs walk, so the pairs idle only at the end of the whole list, and set-up and the last epilogue are paid
+// once.  Layers with more K stages per tile come first in the list.
+cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys,
+                                  const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s) {
   using namespace tc2;
   if (n < 1 || n > MAX_GROUP) return cudaErrorInvalidValue;
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
-  TensorMaps tmaps;
-  const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
-  const cuuint32_t box[2] = {BK, BM};
-  const cuuint32_t estr[2] = {1, 1};
-  for (int g = 0; g < MAX_GROUP; ++g)
-    if (enc(&tmaps.m[g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xcats[g < n ? g : 0]), dims, strides, box,
-            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorInvalidValue;
-
   static int sm_count = 0;
   static bool attr_set = false;
   if (!attr_set) {
@@ -387,21 +402,46 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
+  // order: falling number of K stages per tile (stable, so equal layers keep the caller's order)
+  int order[MAX_GROUP];
+  for (int g = 0; g < n; ++g) order[g] = g;
+  auto spt_of = [&](int g) { return metas[g].k_slabs + (metas[g].r_blocks + 1) / 2; };
+  for (int a = 1; a < n; ++a)
+    for (int b = a; b > 0 && spt_of(order[b]) > spt_of(order[b - 1]); --b) { const int t = order[b]; order[b] = order[b - 1]; order[b - 1] = t; }
+
+  TensorMaps tmaps;
   Params p;
-  for (int g = 0; g < MAX_GROUP; ++g) {
-    const uint8_t* base = static_cast<const uint8_t*>(packed[g < n ? g : 0]);
-    p.wsec[g] = base + m.off_w;
-    p.bsec[g] = base + m.off_b;
-    p.Y[g] = Ys[g < n ? g : 0];
+  p.m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  int tile_begin = 0;
+  for (int slot = 0; slot < MAX_GROUP; ++slot) {
+    const int g = order[slot < n ? slot : 0];
+    const PackedMeta& m = metas[g];
+    if (m.lr_bits != metas[0].lr_bits) return cudaErrorInvalidValue;
+    const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
+    const cuuint32_t box[2] = {BK, BM};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmaps.m[slot], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xcats[g]), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    const uint8_t* base = static_cast<const uint8_t*>(packed[g]);
+    Layer& ly = p.L[slot];
+    ly.wsec = base + m.off_w;
+    ly.bsec = base + m.off_b;
+    ly.Y = Ys[g];
+    ly.N = m.N; ly.K64 = m.K64;
+    ly.n_tiles = m.n_tiles; ly.k_slabs = m.k_slabs; ly.r_blocks = m.r_blocks;
+    ly.spt = m.k_slabs + (m.r_blocks + 1) / 2;
+    ly.tile_begin = tile_begin;
+    if (slot < n) tile_begin += p.m_tiles * ((m.n_tiles + 1) / 2);
   }
   p.group = n;
+  p.num_tiles = tile_begin;
   p.status = st;
-  p.M = M; p.N = m.N; p.K64 = m.K64;
-  p.n_tiles = m.n_tiles; p.k_slabs = m.k_slabs; p.r_blocks = m.r_blocks;
-  p.m_tiles = (M + 2 * BM - 1) / (2 * BM);
-  p.n256_tiles = (m.n_tiles + 1) / 2;
-  p.lr_shift = m.lr_bits - 2;
-  const int num_tiles = n * p.m_tiles * p.n256_tiles;
+  p.M = M;
+  p.lr_shift = metas[0].lr_bits - 2;
+  const int num_tiles = p.num_tiles;
   const int max_pairs = sm_count / 2;
   const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
 
