@@ -427,7 +427,15 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     bool decode_group = false;
     if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
       if (decode_cols_fits(m0, calls[i].M)) {
-        n = same_shape_run(calls, i, n_calls, m0, decode_cols_max_group());
+        // decode calls with one M and one set of formats, each served by the column-owner kernel
+        metas[0] = m0;
+        while (i + n < n_calls && n < decode_cols_max_group()) {
+          PackedMeta m1;
+          if (calls[i + n].M != calls[i].M || lookup(calls[i + n].packed, m1) != LQER_OK || !same_formats(m0, m1) ||
+              !decode_cols_fits(m1, calls[i].M) || m1.N < 32 || m0.N < 32)
+            break;
+          metas[n++] = m1;
+        }
         decode_group = n > 1;
       } else if (calls[i].M > 128) {
         n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), workspace_bytes, metas, nullptr);
@@ -439,7 +447,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
       if (st != LQER_OK) return st;
       if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
       if (decode_group) {
-        if (launch_decode_cols_group(calls + i, n, m0, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        if (launch_decode_cols_group(calls + i, metas, n, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
           return LQER_ERR_CUDA;
       } else if ((st = run_prefill_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) {
         return st;

@@ -247,9 +247,10 @@ cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);
-// Up to decode_cols_max_group() independent layers of one shape and one M (all fitting decode_cols_fits) in one launch.
+// Up to decode_cols_max_group() independent layers with one M (all fitting decode_cols_fits, N >= 32) in one launch.
 int decode_cols_max_group();
-cudaError_t launch_decode_cols_group(const lqer_call_t* calls, int n, const PackedMeta& m, void* workspace, cudaStream_t s);
+cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
+                                     cudaStream_t s);
 int decode_max_m();
 
 }  // namespace lqer

@@ -37,16 +37,23 @@ constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q (pa
 constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
 constexpr int kAStageMax = 100 * 1024;   // a CTA's share of A_q is staged in shared memory if it fits in this
 
-constexpr int kMaxGroup = 4;   // independent layers of one shape that may share a launch (blockIdx.y picks one)
+constexpr int kMaxGroup = 8;   // independent layers with one M that may share a launch
+
+struct Layer {
+  const float* X;
+  float* Y;
+  const uint8_t* packed;
+  size_t off_w, off_b, off_a;   // sections of the packed buffer
+  int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
+  int a_stage_bytes;            // shared memory reserved for staging A_q (0: read it from global memory)
+  int cta_begin, ctas;          // this layer's CTAs in the launch: whole clusters, in proportion to its weight bytes
+};
 
 struct Params {
-  const float* X[kMaxGroup];
-  float* Y[kMaxGroup];
-  const uint8_t* packed[kMaxGroup];
-  size_t off_w, off_b, off_a;   // sections of a packed buffer (equal for equal shapes)
+  Layer L[kMaxGroup];
+  int group;                    // layers in this launch
   DeviceStatus* status;
-  int M, K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
-  int a_stage_bytes;    // shared memory reserved for staging A_q (0: read it from global memory)
+  int M;
   int a_bits, lr_bits, exp_min, exp_max;
 };
 
@@ -96,27 +103,32 @@ template <int MT>
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
-  const int M = p.M, KB = p.K64 / 16;
+  int layer = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxGroup; ++i)
+    if (i < p.group && (int)blockIdx.x >= p.L[i].cta_begin) layer = i;
+  const Layer& ly = p.L[layer];
+  const int M = p.M, KB = ly.K64 / 16;
   uint8_t* xm = smem;                                               // [M][K64] int8 mantissas, permuted within 8
-  float* xsc = reinterpret_cast<float*>(xm + (size_t)M * p.K64);    // [M][KB] 2^(e_x - 6)
+  float* xsc = reinterpret_cast<float*>(xm + (size_t)M * ly.K64);    // [M][KB] 2^(e_x - 6)
   int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);          // [M][KB] 8 * sum(x) of the block
   float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // [kWarps][kCg][8][kMaxM]
   double* tpart = reinterpret_cast<double*>(red + kWarps * kCg * 8 * kMaxM);   // [M][k_pad] this CTA's partial T
-  double* tsub = tpart + (size_t)kMaxM * p.k_pad;                   // [subsets][M][k_pad] per-warp-subset partials
-  float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * p.k_pad * kMaxSubsets);   // [M][k_pad / 16]
+  double* tsub = tpart + (size_t)kMaxM * ly.k_pad;                   // [subsets][M][k_pad] per-warp-subset partials
+  float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * kMaxSubsets);   // [M][k_pad / 16]
   int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);        // [M][k_pad]
   uint8_t* a_stage = reinterpret_cast<uint8_t*>(
-      (reinterpret_cast<uintptr_t>(tq8) + (size_t)kMaxM * (p.k_pad > 0 ? p.k_pad : 16) + 15) & ~(uintptr_t)15);   // staged A_q
+      (reinterpret_cast<uintptr_t>(tq8) + (size_t)kMaxM * (ly.k_pad > 0 ? ly.k_pad : 16) + 15) & ~(uintptr_t)15);   // staged A_q
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int G = gridDim.x, cta = blockIdx.x;
-  const float* const X = p.X[blockIdx.y];
-  float* const Y = p.Y[blockIdx.y];
-  const uint8_t* const wsec = p.packed[blockIdx.y] + p.off_w;
-  const uint8_t* const bsec = p.packed[blockIdx.y] + p.off_b;
-  const uint8_t* const asec = p.packed[blockIdx.y] + p.off_a;
-  const int cg_lo = cta * p.n_cg / G, cg_hi = (cta + 1) * p.n_cg / G;
+  const int G = ly.ctas, cta = (int)blockIdx.x - ly.cta_begin;
+  const float* const X = ly.X;
+  float* const Y = ly.Y;
+  const uint8_t* const wsec = ly.packed + ly.off_w;
+  const uint8_t* const bsec = ly.packed + ly.off_b;
+  const uint8_t* const asec = ly.packed + ly.off_a;
+  const int cg_lo = cta * ly.n_cg / G, cg_hi = (cta + 1) * ly.n_cg / G;
 
   // This lane's share of (column group cg, slab j): global -> registers.  Byte offsets into the W section are kept
   // per column group (32 bits: the section is far below 4 GB); a load then costs two adds.  Column groups past the
@@ -127,14 +139,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   struct GroupOff { uint32_t w, e; };
   auto group_off = [&](int cg) -> GroupOff {
     cg = max(min(cg, cg_hi - 1), 0);
-    const uint32_t tile = (uint32_t)(cg >> 4) * (uint32_t)p.k_slabs * (uint32_t)kWTileBytes;
+    const uint32_t tile = (uint32_t)(cg >> 4) * (uint32_t)ly.k_slabs * (uint32_t)kWTileBytes;
     GroupOff o;
     o.w = tile + (uint32_t)(cg & 15) * 128u + lane_w;
     o.e = tile + (uint32_t)(cg & 15) * 32u + lane_e;
     return o;
   };
   auto fetch = [&](UnitRegs& d, const GroupOff& o, int j) {
-    const uint32_t jo = (uint32_t)min(j, p.k_slabs - 1) * (uint32_t)kWTileBytes;
+    const uint32_t jo = (uint32_t)min(j, ly.k_slabs - 1) * (uint32_t)kWTileBytes;
     d.w = ld_stream_u64(wsec + (o.w + jo));
     d.e = ld_stream_u8(wsec + (o.e + jo));
   };
@@ -145,11 +157,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   auto fetch_rank = [&](uint32_t& wv, uint32_t& eb, int cg) {
     wv = 0u;
     eb = 127u;
-    if (cg < cg_hi && warp < p.r_blocks) {
+    if (cg < cg_hi && warp < ly.r_blocks) {
       const int col = (cg & 15) * 8 + g;
-      const uint8_t* tile = bsec + (size_t)(cg >> 4) * ((size_t)p.r_blocks * kTileN * 17);
+      const uint8_t* tile = bsec + (size_t)(cg >> 4) * ((size_t)ly.r_blocks * kTileN * 17);
       wv = ld_stream_u32(tile + ((size_t)warp * kTileN + col) * 16 + t * 4);
-      eb = ld_stream_u8(tile + (size_t)p.r_blocks * kTileN * 16 + warp * kTileN + col);
+      eb = ld_stream_u8(tile + (size_t)ly.r_blocks * kTileN * 16 + warp * kTileN + col);
     }
   };
 
@@ -166,14 +178,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     for (int u = 0; u < kCg; ++u) fetch(regs[s][u], o_cur[u], warp + kWarps * s);
 #pragma unroll
   for (int u = 0; u < kCg; ++u) fetch_rank(rank_w[u], rank_e[u], cg_lo + u);
-  const int KBr = p.K / 16;
+  const int KBr = ly.K / 16;
   const int cs = (int)cluster_nctarank(), cr = (int)cluster_ctarank();
   const int kb_lo = cr * KBr / cs, kb_hi = (cr + 1) * KBr / cs;      // this CTA's share of K for T
-  const bool a_staged = p.k_pad > 0 && (kb_hi - kb_lo) * p.k_pad * 17 <= p.a_stage_bytes;
+  const bool a_staged = ly.k_pad > 0 && (kb_hi - kb_lo) * ly.k_pad * 17 <= ly.a_stage_bytes;
   if (a_staged) {
-    const int mant = (kb_hi - kb_lo) * p.k_pad * 16, ex = (kb_hi - kb_lo) * p.k_pad;
-    const uint8_t* gm = asec + (size_t)kb_lo * p.k_pad * 16;
-    const uint8_t* ge = asec + (size_t)KBr * p.k_pad * 16 + (size_t)kb_lo * p.k_pad;
+    const int mant = (kb_hi - kb_lo) * ly.k_pad * 16, ex = (kb_hi - kb_lo) * ly.k_pad;
+    const uint8_t* gm = asec + (size_t)kb_lo * ly.k_pad * 16;
+    const uint8_t* ge = asec + (size_t)KBr * ly.k_pad * 16 + (size_t)kb_lo * ly.k_pad;
     for (int o = tid * 16; o < mant; o += kThreads * 16)
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(a_stage + o)), "l"(gm + o) : "memory");
     for (int o = tid * 16; o < ex; o += kThreads * 16)
@@ -186,12 +198,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   // ---- X -> MXINT8 for the whole contraction: per row the mantissas in the byte order the nibbles
   //      unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales and the offsets 8 * sum(x)
   {
-    const int per_row = p.K64 / 4, total = M * per_row;             // float4 items: (row, quarter-block)
+    const int per_row = ly.K64 / 4, total = M * per_row;             // float4 items: (row, quarter-block)
     for (int base = 0; base < total; base += kThreads) {
       const int item = base + tid;
       const bool valid = item < total;
       const int row = valid ? item / per_row : 0, c4 = valid ? item % per_row : 0;
-      const float4 v = (valid && c4 * 4 < p.K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * p.K + c4 * 4))
+      const float4 v = (valid && c4 * 4 < ly.K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * ly.K + c4 * 4))
                                                : make_float4(0.f, 0.f, 0.f, 0.f);
       int e;
       uint32_t m8;
@@ -203,7 +215,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
       sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
       if (valid) {
-        *reinterpret_cast<uint32_t*>(xm + (size_t)row * p.K64 + c4 * 4) = perm;
+        *reinterpret_cast<uint32_t*>(xm + (size_t)row * ly.K64 + c4 * 4) = perm;
         if ((c4 & 3) == 0) {
           xsc[row * KB + (c4 >> 2)] = pow2f(e - (p.a_bits - 2));
           xof[row * KB + (c4 >> 2)] = 8 * sum;
@@ -218,12 +230,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   //      mantissas in shared memory, scaled in fp64.  The products are exact; their fp64 sums are exact
   //      too unless the block exponents of one row spread over more than about 30 binades, and the
   //      order of the additions is fixed in any case.
-  if (p.k_pad > 0) {
-    const int NT = p.k_pad / 8;
+  if (ly.k_pad > 0) {
+    const int NT = ly.k_pad / 8;
     // A_q of blocks kb_lo..kb_hi: staged copy, or global memory
-    const uint8_t* a_mant = a_staged ? a_stage - (size_t)kb_lo * p.k_pad * 16 : asec;
-    const uint8_t* a_exp = a_staged ? a_stage + (size_t)(kb_hi - kb_lo) * p.k_pad * 16 - (size_t)kb_lo * p.k_pad
-                                    : asec + (size_t)KBr * p.k_pad * 16;
+    const uint8_t* a_mant = a_staged ? a_stage - (size_t)kb_lo * ly.k_pad * 16 : asec;
+    const uint8_t* a_exp = a_staged ? a_stage + (size_t)(kb_hi - kb_lo) * ly.k_pad * 16 - (size_t)kb_lo * ly.k_pad
+                                    : asec + (size_t)KBr * ly.k_pad * 16;
     const int bias = -127 - (p.lr_bits - 2);                        // exponent bytes carry +127
     const int tiles_w = NT < kWarps ? NT : kWarps;                  // warps side by side on different rank tiles
     int subsets = kWarps / tiles_w;                                 // warps that split the K blocks of one tile
@@ -235,11 +247,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 #pragma unroll 4
         for (int kb = kb_lo + sb; kb < kb_hi; kb += subsets) {
           // the X mantissas are stored as {0,4,1,5}, {2,6,3,7} within each 8: bring A_q into the same order
-          const uint4 q = *reinterpret_cast<const uint4*>(a_mant + ((size_t)kb * p.k_pad + nt * 8 + g) * 16);
+          const uint4 q = *reinterpret_cast<const uint4*>(a_mant + ((size_t)kb * ly.k_pad + nt * 8 + g) * 16);
           const uint32_t lo = (t & 2) ? q.z : q.x, hi = (t & 2) ? q.w : q.y;
           const uint32_t b0 = (t & 1) ? __byte_perm(lo, hi, 0x7362) : __byte_perm(lo, hi, 0x5140);
-          const uint32_t ea2 = *reinterpret_cast<const uint16_t*>(a_exp + (size_t)kb * p.k_pad + nt * 8 + t * 2);
-          const uint32_t a0 = g < M ? *reinterpret_cast<const uint32_t*>(xm + (size_t)g * p.K64 + kb * 16 + t * 4) : 0u;
+          const uint32_t ea2 = *reinterpret_cast<const uint16_t*>(a_exp + (size_t)kb * ly.k_pad + nt * 8 + t * 2);
+          const uint32_t a0 = g < M ? *reinterpret_cast<const uint32_t*>(xm + (size_t)g * ly.K64 + kb * 16 + t * 4) : 0u;
           const double sx = g < M ? (double)xsc[g * KB + kb] : 0.0;
           int c[4];
           mma_s8(c, a0, 0u, b0);
@@ -247,24 +259,24 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
           t1 = fma((double)c[1], sx * pow2d((int)(ea2 >> 8) + bias), t1);
         }
         if (g < M) {
-          tsub[((size_t)sb * kMaxM + g) * p.k_pad + nt * 8 + t * 2] = t0;
-          tsub[((size_t)sb * kMaxM + g) * p.k_pad + nt * 8 + t * 2 + 1] = t1;
+          tsub[((size_t)sb * kMaxM + g) * ly.k_pad + nt * 8 + t * 2] = t0;
+          tsub[((size_t)sb * kMaxM + g) * ly.k_pad + nt * 8 + t * 2 + 1] = t1;
         }
       }
     }
     __syncthreads();
-    for (int idx = tid; idx < M * p.k_pad; idx += kThreads) {
-      const int row = idx / p.k_pad, col = idx % p.k_pad;
+    for (int idx = tid; idx < M * ly.k_pad; idx += kThreads) {
+      const int row = idx / ly.k_pad, col = idx % ly.k_pad;
       double v = 0.0;
-      for (int q = 0; q < subsets; ++q) v += tsub[((size_t)q * kMaxM + row) * p.k_pad + col];
-      tpart[row * p.k_pad + col] = v;
+      for (int q = 0; q < subsets; ++q) v += tsub[((size_t)q * kMaxM + row) * ly.k_pad + col];
+      tpart[row * ly.k_pad + col] = v;
     }
     __syncthreads();
     cluster_arrive();                            // this CTA's partial T is published; waited for before the rank part
   }
 
   bool tq_built = false;
-  const int slabs_mine = p.k_slabs > warp ? (p.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
+  const int slabs_mine = ly.k_slabs > warp ? (ly.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
 #pragma unroll 1
   for (int cg0 = cg_lo; cg0 < cg_hi; cg0 += kCg) {
     float acc[kCg][MT];
@@ -282,11 +294,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 #pragma unroll
       for (int s = 0; s < kSets; ++s) {
         const int j = warp + kWarps * (js + s);
-        if (j < p.k_slabs) {
+        if (j < ly.k_slabs) {
 #pragma unroll
           for (int r = 0; r < MT; ++r) {
             if (r < M) {
-              const uint4 x = *reinterpret_cast<const uint4*>(xm + (size_t)r * p.K64 + j * 64 + t * 16);
+              const uint4 x = *reinterpret_cast<const uint4*>(xm + (size_t)r * ly.K64 + j * 64 + t * 16);
               const float sx = xsc[r * KB + j * 4 + t];
               const int off = xof[r * KB + j * 4 + t];
 #pragma unroll
@@ -319,42 +331,42 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     for (int u = 0; u < kCg; ++u) o_cur[u] = o_nxt[u];
 
     // ---- B_q against T_q: rank blocks warp, warp + 16, ...
-    if (p.k_pad > 0) {
+    if (ly.k_pad > 0) {
       if (!tq_built) {
         // T = sum of the cluster's partials (CTA order), then MXINT8 along the rank: 16 adjacent lanes hold one block
         cluster_wait();
         const int cs = (int)cluster_nctarank();
-        const int total = M * p.k_pad;
+        const int total = M * ly.k_pad;
         for (int base = 0; base < total; base += kThreads) {
           const int idx = base + tid;
           const bool valid = idx < total;
-          const int row = valid ? idx / p.k_pad : 0, col = valid ? idx % p.k_pad : 0;
+          const int row = valid ? idx / ly.k_pad : 0, col = valid ? idx % ly.k_pad : 0;
           double tv = 0.0;
           if (valid)
-            for (int c = 0; c < cs; ++c) tv += ld_dsmem_f64(tpart + row * p.k_pad + col, (uint32_t)c);
+            for (int c = 0; c < cs; ++c) tv += ld_dsmem_f64(tpart + row * ly.k_pad + col, (uint32_t)c);
           double amax = (tv != tv) ? 0.0 : fabs(tv);
 #pragma unroll
           for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
           const int e = block_exponent(amax, p.exp_min, p.exp_max);
           const int qv = quant_mantissa(tv, e, p.a_bits);
           if (valid) {
-            tq8[row * p.k_pad + col] = (int8_t)qv;
-            if ((col & 15) == 0) tqs[row * (p.k_pad / 16) + (col >> 4)] = pow2f(e - (p.a_bits - 2));
+            tq8[row * ly.k_pad + col] = (int8_t)qv;
+            if ((col & 15) == 0) tqs[row * (ly.k_pad / 16) + (col >> 4)] = pow2f(e - (p.a_bits - 2));
           }
         }
         __syncthreads();
         cluster_arrive();                        // done reading the peers' shared memory
         tq_built = true;
       }
-      const int rbn = p.k_pad / 16;
-      if (warp < p.r_blocks) {                   // rank block `warp` (k <= 256: at most 16 blocks); data already in registers
+      const int rbn = ly.k_pad / 16;
+      if (warp < ly.r_blocks) {                   // rank block `warp` (k <= 256: at most 16 blocks); data already in registers
 #pragma unroll
         for (int u = 0; u < kCg; ++u) {
           const float sb = __uint_as_float((rank_e[u] - (uint32_t)(p.lr_bits - 2)) << 23);        // 2^(e_b - 6)
 #pragma unroll
           for (int r = 0; r < MT; ++r) {
             if (r < M) {
-              const int tw = *reinterpret_cast<const int*>(tq8 + r * p.k_pad + warp * 16 + t * 4);
+              const int tw = *reinterpret_cast<const int*>(tq8 + r * ly.k_pad + warp * 16 + t * 4);
               acc[u][r] = fmaf((float)__dp4a(tw, (int)rank_w[u], 0), tqs[r * rbn + warp] * sb, acc[u][r]);
             }
           }
@@ -384,11 +396,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) v += red[((w * kCg + u) * 8 + gg) * kMaxM + r];
       const int cg = cg0 + u;
-      if (cg < cg_hi && r < M) Y[(size_t)r * p.N + cg * 8 + gg] = v;
+      if (cg < cg_hi && r < M) Y[(size_t)r * ly.N + cg * 8 + gg] = v;
     }
     __syncthreads();                             // red is rewritten by the next round
   }
-  if (p.k_pad > 0) {
+  if (ly.k_pad > 0) {
     if (!tq_built) { cluster_wait(); cluster_arrive(); }   // a CTA without columns still serves its partial T
     cluster_wait();                              // no CTA leaves while its shared memory may still be read
   }
@@ -407,19 +419,21 @@ bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && c
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y, void* workspace,
                                cudaStream_t s) {
   const lqer_call_t one = {X, M, packed, Y};
-  return launch_decode_cols_group(&one, 1, m, workspace, s);
+  return launch_decode_cols_group(&one, &m, 1, workspace, s);
 }
 
 int decode_cols_max_group() { return dcol::kMaxGroup; }
 
-// n independent layers of one shape (same K, N, rank, formats) and one M in a single launch: the SMs are divided
-// among them, so the layers' fixed latencies (dependency wait, X quantisation, the T exchange, the final
-// reduction) overlap instead of following one another.
-cudaError_t launch_decode_cols_group(const lqer_call_t* calls, int n, const PackedMeta& m, void* workspace, cudaStream_t s) {
+// n independent layers with one M (shapes may differ) in a single launch: the SMs are divided among them in proportion
+// to their weight bytes, so the layers' fixed latencies (dependency wait, X quantisation, the T exchange, the final
+// reduction) overlap instead of following one another.  Every layer must fit decode_cols_fits and, for n > 1, have
+// at least one cluster's worth of column groups.
+cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
+                                     cudaStream_t s) {
   using namespace dcol;
   static int sm_count = 0;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static int max_clusters = -1;
+  if (max_clusters < 0) {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
@@ -427,35 +441,86 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, int n, const Pack
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(decode_cols_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    // all clusters must be resident at once: the CTAs are sized for one wave
+    cudaLaunchConfig_t probe = {};
+    probe.gridDim = dim3(sm_count / kClusterSize * kClusterSize);
+    probe.blockDim = dim3(kThreads);
+    probe.dynamicSmemBytes = 200 * 1024;
+    cudaLaunchAttribute pa[1];
+    pa[0].id = cudaLaunchAttributeClusterDimension;
+    pa[0].val.clusterDim.x = kClusterSize; pa[0].val.clusterDim.y = 1; pa[0].val.clusterDim.z = 1;
+    probe.attrs = pa;
+    probe.numAttrs = 1;
+    int nc = 0;
+    if (cudaOccupancyMaxActiveClusters(&nc, decode_cols_kernel<kMaxM>, &probe) != cudaSuccess || nc < 1) nc = 1;
+    max_clusters = nc;
   }
   if (n < 1 || n > kMaxGroup) return cudaErrorInvalidValue;
   const int M = calls[0].M;
   Params p;
-  uint8_t* ws = static_cast<uint8_t*>(workspace);
-  for (int i = 0; i < kMaxGroup; ++i) {
-    const lqer_call_t& c = calls[i < n ? i : 0];
-    p.X[i] = c.X; p.Y[i] = c.Y; p.packed[i] = static_cast<const uint8_t*>(c.packed);
+  p.group = n;
+  p.status = reinterpret_cast<DeviceStatus*>(workspace);
+  p.M = M;
+  p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
+
+  // CTAs per layer: a single layer takes what it can use; several share the resident clusters by weight bytes
+  int ctas[kMaxGroup];
+  int cs = kClusterSize;
+  if (n == 1) {
+    int G = metas[0].N / 8 < sm_count ? metas[0].N / 8 : sm_count;
+    if (G > kDecodeMaxCtas) G = kDecodeMaxCtas;
+    cs = G >= kClusterSize ? kClusterSize : 1;
+    G = G / cs * cs;
+    if (cs > 1 && G > max_clusters * cs) G = max_clusters * cs;
+    ctas[0] = G;
+  } else {
+    double total_w = 0.0;
+    for (int g = 0; g < n; ++g) {
+      if (metas[g].N / 8 < kClusterSize) return cudaErrorInvalidValue;
+      total_w += (double)metas[g].K * metas[g].N;
+    }
+    int left = max_clusters;
+    for (int g = 0; g < n; ++g) {                     // at least one cluster each, the rest by weight
+      int c = (int)((double)max_clusters * ((double)metas[g].K * metas[g].N / total_w));
+      if (c < 1) c = 1;
+      const int cap = metas[g].N / 8 / kClusterSize;
+      if (c > cap) c = cap;
+      ctas[g] = c;
+      left -= c;
+    }
+    if (left < 0) return cudaErrorInvalidConfiguration;   // more layers than clusters
+    for (int g = 0; left > 0 && g < n; ++g)              // hand out what rounding left over
+      if (ctas[g] < metas[g].N / 8 / kClusterSize) { ++ctas[g]; --left; }
+    for (int g = 0; g < n; ++g) ctas[g] *= kClusterSize;
   }
-  p.off_w = m.off_w; p.off_b = m.off_b; p.off_a = m.off_a;
-  p.status = reinterpret_cast<DeviceStatus*>(ws);
-  p.M = M; p.K = m.K; p.N = m.N; p.K64 = m.K64; p.k_pad = m.k_pad;
-  p.k_slabs = m.k_slabs; p.r_blocks = m.r_blocks;
-  p.n_cg = m.N / 8;
-  p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
-  int G = sm_count / n;                         // CTAs per layer
-  if (G > p.n_cg) G = p.n_cg;
-  if (G > kDecodeMaxCtas) G = kDecodeMaxCtas;
-  const int cs = G >= kClusterSize ? kClusterSize : 1;
-  G = G / cs * cs;
-  // stage this CTA's share of A_q in shared memory when it fits beside everything else
-  const size_t a_need = m.k_pad > 0 ? (size_t)((m.K / 16 + cs - 1) / cs) * m.k_pad * 17 + 16 : 0;
-  p.a_stage_bytes = (a_need <= (size_t)kAStageMax && cols_smem_bytes(m, M) + a_need <= 200 * 1024) ? (int)a_need : 0;
-  const size_t smem = cols_smem_bytes(m, M) + p.a_stage_bytes;
-  if (!decode_cols_fits(m, M)) return cudaErrorInvalidValue;
+
+  size_t smem = 0;
+  int begin = 0;
+  for (int i = 0; i < kMaxGroup; ++i) {
+    const int g = i < n ? i : 0;
+    const PackedMeta& m = metas[g];
+    if (!decode_cols_fits(m, M) || !(m.a_bits == p.a_bits && m.lr_bits == p.lr_bits && m.exp_min == p.exp_min && m.exp_max == p.exp_max))
+      return cudaErrorInvalidValue;
+    Layer& ly = p.L[i];
+    ly.X = calls[g].X; ly.Y = calls[g].Y; ly.packed = static_cast<const uint8_t*>(calls[g].packed);
+    ly.off_w = m.off_w; ly.off_b = m.off_b; ly.off_a = m.off_a;
+    ly.K = m.K; ly.N = m.N; ly.K64 = m.K64; ly.k_pad = m.k_pad;
+    ly.k_slabs = m.k_slabs; ly.r_blocks = m.r_blocks;
+    ly.n_cg = m.N / 8;
+    // stage this CTA's share of A_q in shared memory when it fits beside everything else
+    const size_t a_need = m.k_pad > 0 ? (size_t)((m.K / 16 + cs - 1) / cs) * m.k_pad * 17 + 16 : 0;
+    ly.a_stage_bytes = (a_need <= (size_t)kAStageMax && cols_smem_bytes(m, M) + a_need <= 200 * 1024) ? (int)a_need : 0;
+    ly.cta_begin = begin;
+    ly.ctas = ctas[g];
+    if (i < n) {
+      begin += ctas[g];
+      const size_t need = cols_smem_bytes(m, M) + ly.a_stage_bytes;
+      if (need > smem) smem = need;
+    }
+  }
 
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(G, n);
+  cfg.gridDim = dim3(begin);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
@@ -466,20 +531,6 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, int n, const Pack
   attr[1].val.clusterDim.x = cs; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  if (cs > 1) {
-    // all clusters must be resident at once: the CTAs are sized for one wave
-    static int max_clusters = -1;
-    if (max_clusters < 0) {
-      cudaLaunchConfig_t probe = cfg;
-      probe.dynamicSmemBytes = 200 * 1024;
-      probe.gridDim = dim3(sm_count / cs * cs);
-      int nc = 0;
-      if (cudaOccupancyMaxActiveClusters(&nc, decode_cols_kernel<kMaxM>, &probe) != cudaSuccess || nc < 1) nc = 1;
-      max_clusters = nc;
-    }
-    if (G * n > max_clusters * cs) { G = max_clusters / n * cs; cfg.gridDim = dim3(G, n); }
-    if (G < cs) return cudaErrorInvalidConfiguration;
-  }
   LaunchScope scope(kFamDecode, s);
   return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM>, p);
 }

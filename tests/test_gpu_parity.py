@@ -228,8 +228,8 @@ def test_decode_chain_shares_one_workspace():
 
 @pytest.mark.parametrize("M", [1, 3])
 def test_batched_decode_groups_same_shape_calls(M):
-    # seven independent calls: five layers of one shape (a group of four and a fifth), then two of another shape;
-    # the batched entry point runs same-shape neighbours in shared launches and must give what single calls give
+    # seven independent calls: five layers of one shape, then two of another; the batched entry point runs them in
+    # one launch that divides the SMs among the layers by weight bytes, and must give what single calls give
     spec_a = gen.LayerSpec("grp_a", M=M, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=51)
     spec_b = gen.LayerSpec("grp_b", M=M, K=512, N=2048, k=8, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=52)
     layers = []
@@ -245,7 +245,7 @@ def test_batched_decode_groups_same_shape_calls(M):
     L.linear_batched([(x, lay[2], y) for x, lay, y in zip(Xs, layers, Yb)], ws)
     torch.cuda.synchronize()
     assert L.poll_status(ws) == 0
-    assert L.launch_count() - launches == 3            # 4 + 1 of the first shape, 2 of the second
+    assert L.launch_count() - launches == 1            # seven layers with one M: one launch
     for x, (sp, P, Pg), yb in zip(Xs, layers, Yb):
         ys = L.linear(x, Pg, ws)
         assert torch.equal(ys, yb), sp.name             # same arithmetic, same order: bit-identical
