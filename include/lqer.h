@@ -160,14 +160,15 @@ lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, floa
 /* n_calls independent layers back to back on one stream (`calls` is a HOST array).
  * The workspace is reused by consecutive calls (stream order makes that safe) and must
  * fit the largest of them.  Independent means that no call reads what another call of the
- * same batch writes: with the path left at 0, up to four consecutive calls with M <= 4 and
- * packed buffers of one shape (K, N, rank, formats) run as ONE launch that divides the SMs
- * among them (the q, k, v or the gate and up projections of a decoder layer), and up to eight
- * consecutive calls with one M > 128 (any shapes, one set of formats) run their prologues into
- * separate slices of the workspace and then ONE GEMM launch over the tiles of all of them - if
- * the workspace holds
- * lqer_batched_workspace_bytes(calls, n_calls); with a smaller workspace (at least the largest
- * lqer_workspace_bytes of the calls) they run one after the other. */
+ * same batch writes; the library uses that, with the path left at 0, to share launches:
+ *  - up to 16 consecutive calls with one M <= 4 (any shapes with N >= 32, one set of formats)
+ *    run as ONE launch of the decode kernel that divides the SMs among them by weight bytes;
+ *  - up to 8 consecutive calls with one M > 128 (any shapes, one set of formats) run their
+ *    prologues into separate slices of the workspace and then ONE GEMM launch over the tiles of
+ *    all of them - if the workspace holds lqer_batched_workspace_bytes(calls, n_calls); with a
+ *    smaller workspace (at least the largest lqer_workspace_bytes of the calls) fewer calls, or
+ *    none, share a launch.
+ * Results do not depend on the sharing. */
 lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes);
 lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
                                   void* workspace, size_t workspace_bytes, void* stream);

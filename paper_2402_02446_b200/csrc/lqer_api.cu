@@ -423,7 +423,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     // and up projections) share launches: decode calls one launch of the column-owner kernel (it keeps nothing in the
     // workspace), prefill calls one GEMM launch after their prologues, if the workspace has a slice for each.
     int n = 1;
-    PackedMeta m0, metas[8];
+    PackedMeta m0, metas[16];
     bool decode_group = false;
     if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
       if (decode_cols_fits(m0, calls[i].M)) {

@@ -37,7 +37,7 @@ constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q (pa
 constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
 constexpr int kAStageMax = 100 * 1024;   // a CTA's share of A_q is staged in shared memory if it fits in this
 
-constexpr int kMaxGroup = 8;   // independent layers with one M that may share a launch
+constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
 
 struct Layer {
   const float* X;
