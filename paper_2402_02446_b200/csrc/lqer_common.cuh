@@ -148,12 +148,11 @@ __device__ __forceinline__ uint32_t bf16_bits_of(int m, int p) {
 // m * 2^(e - (bits-2)) packed in two words.
 __device__ __forceinline__ void quantize_quad(const float4 vin, int bits, int emin, int emax, int& e, uint32_t& m8,
                                               uint2& bf) {
-  // NaN counts as zero, as a value and in the block maximum
-  const float v[4] = {(vin.x == vin.x) ? vin.x : 0.0f, (vin.y == vin.y) ? vin.y : 0.0f,
-                      (vin.z == vin.z) ? vin.z : 0.0f, (vin.w == vin.w) ? vin.w : 0.0f};
-  float amax = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+  // block maximum: fmaxf drops a NaN operand, so NaN counts as zero here; a block of NaNs only ends as zero too
+  float amax = fmaxf(fmaxf(fabsf(vin.x), fabsf(vin.y)), fmaxf(fabsf(vin.z), fabsf(vin.w)));
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+  amax = fmaxf(amax, 0.0f);
   e = block_exponent(amax, emin, emax);
   const float qmax = (float)((1 << (bits - 1)) - 1);
   const float inv_step = pow2f((bits - 2) - e), step = pow2f(e - (bits - 2));
@@ -161,14 +160,29 @@ __device__ __forceinline__ void quantize_quad(const float4 vin, int bits, int em
   // that integer (two's complement) in the low bits of the sum; (sum - 1.5 * 2^23) * step is exact.
   const float kMagic = 12582912.0f;
   const float back = -kMagic * step;
+  const float v[4] = {vin.x, vin.y, vin.z, vin.w};
   uint32_t rb[4];
   float r[4];
+  // The common case needs neither the clamp nor the NaN test: the lane's four values are numbers (their sum is
+  // not NaN; inf - inf only sends the lane the long way round) and the block's largest scaled magnitude stays
+  // below qmax + 1/2, so no element rounds past qmax (an infinite or clamped-exponent block fails this test).
+  const float lane_sum = (vin.x + vin.y) + (vin.z + vin.w);
+  if (lane_sum == lane_sum && amax * inv_step < qmax + 0.5f) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float t = fminf(fmaxf(v[i] * inv_step, -qmax), qmax);   // exact scaling, clamp (+-inf saturate)
-    const float s = t + kMagic;
-    rb[i] = __float_as_uint(s);
-    r[i] = fmaf(s, step, back);                                    // exact: at most 7 significant bits
+    for (int i = 0; i < 4; ++i) {
+      const float s = fmaf(v[i], inv_step, kMagic);                  // exact scaling, one rounding: to the integer
+      rb[i] = __float_as_uint(s);
+      r[i] = fmaf(s, step, back);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float x = (v[i] == v[i]) ? v[i] : 0.0f;                  // NaN -> 0
+      const float t = fminf(fmaxf(x * inv_step, -qmax), qmax);       // exact scaling, clamp (+-inf saturate)
+      const float s = t + kMagic;
+      rb[i] = __float_as_uint(s);
+      r[i] = fmaf(s, step, back);                                    // exact: at most 7 significant bits
+    }
   }
   m8 = __byte_perm(__byte_perm(rb[0], rb[1], 0x0040), __byte_perm(rb[2], rb[3], 0x0040), 0x5410);
   bf.x = __byte_perm(__float_as_uint(r[0]), __float_as_uint(r[1]), 0x7632);
