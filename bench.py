@@ -41,7 +41,7 @@ M_DECODE, M_PREFILL = 1, 2048
 
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # from an ncu capture) per shape, valid only for the kernel sources whose hash is given.
-TRAFFIC = {"sources_sha256": "88a3f91a59039cc2", "bytes_per_launch": 739e6,
+TRAFFIC = {"sources_sha256": "d730580d1107dc3f", "bytes_per_launch": 739e6,
            "note": "646.5 MB measured on one launch of the seven linears of a decoder layer, scaled to the eight linears "
                    "of a bench launch (profiles/gemm_tc2_kernel_7b_layer.md)"}
 DOMINANT_SOURCES = ["paper_2402_02446_b200/csrc/lqer_gemm_tc2.cu", "paper_2402_02446_b200/csrc/lqer_tc_ptx.cuh"]

@@ -83,9 +83,10 @@ lqer_status_t lqer_packed_bytes(int K, int N, int k, const lqer_config_t* cfg, s
 
 /* Size in bytes (host out) of the scratch `workspace` lqer_linear* needs for any call of up to
  * M_max rows.  The workspace holds a head that is all zero between calls (status area, the
- * decode kernel's arrival counters and its fp64 accumulator of X A_k) followed by per-call
- * scratch: the quantised activations [X_q | T_q] (bf16, M rows) or the decode kernel's
- * partial sums.  One workspace may serve layers of different shapes if it fits the largest. */
+ * kernels' arrival counters, the decode kernel's fp64 accumulator of X A_k) followed by per-call
+ * scratch: the quantised activations [X_q | T_q] (bf16, M rows) with the prologue's fp64
+ * partial sums of X A_k, or the decode kernel's partial sums.  One workspace may serve layers
+ * of different shapes if it fits the largest. */
 lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
 
 /* Weight preparation (Section 3.1: W_q = q(W); Section 4.1 formats): quantise W to MXINT4
@@ -126,8 +127,9 @@ lqer_status_t lqer_project_lowrank(const float* X, int M, const void* packed, in
 
 /* The layer (Section 3.1 last display, Section 3.2 last display):
  *   Y[M,N] = X_q W_q + q(X_q A_q) B_q,  fp32 accumulation of exactly represented products.
- * M <= 16 runs the fused split-K decode kernel; larger M runs the activation prologue and
- * the tensor-core GEMM over the concatenated contraction [X_q | T_q] . [W_q ; B_q].
+ * M <= 16 runs a fused decode kernel (M <= 4: a kernel whose CTAs own output columns; up to
+ * 16: a split-K kernel); larger M runs the activation prologue and the tensor-core GEMM over
+ * the concatenated contraction [X_q | T_q] . [W_q ; B_q].
  * lqer_linear uses the default stream. */
 lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y,
                           void* workspace, size_t workspace_bytes);

@@ -21,6 +21,9 @@
 //                          have finished                   -> TMA producer
 // "accumulator full" is the same kind of commit; "accumulator free" lives in CTA 0 and
 // collects the epilogue warps of both CTAs.
+// A launch may serve several layers with one M: their tiles form one list (layers with more K
+// stages per tile first) that the pairs walk round robin, so pairs idle only at the end of the
+// list and set-up and the last epilogue are paid once per launch.
 #include "lqer_tc_ptx.cuh"
 
 namespace lqer {
