@@ -166,7 +166,7 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
                       : launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
       err = (path == 1)   ? launch_gemm_simt(xcat, M, m, packed, Y, s)
-            : (path == 4 || (path == 0 && M > 128)) ? launch_gemm_tc2(xcat, M, m, packed, Y, dst, s)
+            : (path == 4 || path == 0) ? launch_gemm_tc2(xcat, M, m, packed, Y, dst, s)   // the pair kernel is the faster one at every M above the decode range
                           : launch_gemm_tc(xcat, M, m, packed, Y, dst, s);
   }
   return err == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
@@ -187,7 +187,7 @@ static int same_shape_run(const lqer_call_t* calls, int first, int n_calls, cons
   }
   return n;
 }
-// Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M > 128,
+// Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M above the decode range,
 // the same formats, any shapes; at most `limit`, and only as many as the workspace has slices for.
 static bool same_formats(const PackedMeta& a, const PackedMeta& b) {
   return a.w_bits == b.w_bits && a.a_bits == b.a_bits && a.lr_bits == b.lr_bits && a.exp_min == b.exp_min &&
@@ -437,7 +437,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
           metas[n++] = m1;
         }
         decode_group = n > 1;
-      } else if (calls[i].M > 128) {
+      } else if (calls[i].M > decode_max_m()) {
         n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), workspace_bytes, metas, nullptr);
         if (n < 1) n = 1;
       }
@@ -475,7 +475,7 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
     if (st != LQER_OK) return st;
     need = std::max(need, workspace_total(m, c.M));
     int n = 1;
-    if (c.M > 128 && !decode_cols_fits(m, c.M)) {
+    if (c.M > decode_max_m() && !decode_cols_fits(m, c.M)) {
       PackedMeta metas[8];
       size_t group_need = 0;
       n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), ~(size_t)0, metas, &group_need);
