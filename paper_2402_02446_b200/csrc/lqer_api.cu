@@ -125,11 +125,13 @@ static size_t xcat_bytes(const PackedMeta& m, int M) { return align_up((size_t)M
 // Bytes a call with M rows needs: the persistent head plus the scratch of the path it takes.
 static size_t call_bytes(const PackedMeta& m, int M, bool decode) {
   return align_up(persist_bytes(m), 256) +
-         (decode ? decode_scratch_bytes(m) : xcat_bytes(m, M) + prologue_tc_scratch_bytes(m, M));
+         (decode ? decode_scratch_bytes(m)
+                 : xcat_bytes(m, M) + align_up(prologue_tc_scratch_bytes(m, M), 256) + gemm_splitk_bytes(m, M));
 }
 // Bytes that fit every call of up to M_max rows, whichever path it takes.
 static size_t workspace_total(const PackedMeta& m, int M_max) {
-  const size_t a = xcat_bytes(m, M_max) + prologue_tc_scratch_bound(m, M_max), b = decode_scratch_bytes(m);
+  const size_t a = xcat_bytes(m, M_max) + align_up(prologue_tc_scratch_bound(m, M_max), 256) + gemm_splitk_bound(m, M_max);
+  const size_t b = decode_scratch_bytes(m);
   return align_up(persist_bytes(m), 256) + (a > b ? a : b);
 }
 
@@ -166,7 +168,11 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
                       : launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
       err = (path == 1)   ? launch_gemm_simt(xcat, M, m, packed, Y, s)
-            : (path == 4 || path == 0) ? launch_gemm_tc2(xcat, M, m, packed, Y, dst, s)   // the pair kernel is the faster one at every M above the decode range
+            : (path == 4 || path == 0)   // the pair kernel is the faster one at every M above the decode range
+                ? launch_gemm_tc2_splitk(xcat, M, m, packed, Y,
+                                         reinterpret_cast<float*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M) +
+                                                                  align_up(prologue_tc_scratch_bytes(m, M), 256)),
+                                         dst, s)
                           : launch_gemm_tc(xcat, M, m, packed, Y, dst, s);
   }
   return err == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
@@ -187,7 +193,7 @@ static int same_shape_run(const lqer_call_t* calls, int first, int n_calls, cons
   }
   return n;
 }
-// Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M above the decode range,
+// Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M > 128,
 // the same formats, any shapes; at most `limit`, and only as many as the workspace has slices for.
 static bool same_formats(const PackedMeta& a, const PackedMeta& b) {
   return a.w_bits == b.w_bits && a.a_bits == b.a_bits && a.lr_bits == b.lr_bits && a.exp_min == b.exp_min &&
@@ -437,7 +443,7 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
           metas[n++] = m1;
         }
         decode_group = n > 1;
-      } else if (calls[i].M > decode_max_m()) {
+      } else if (calls[i].M > kGemmSplitMaxM) {   // smaller batches run split K, each on its own
         n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), workspace_bytes, metas, nullptr);
         if (n < 1) n = 1;
       }
@@ -475,7 +481,7 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
     if (st != LQER_OK) return st;
     need = std::max(need, workspace_total(m, c.M));
     int n = 1;
-    if (c.M > decode_max_m() && !decode_cols_fits(m, c.M)) {
+    if (c.M > kGemmSplitMaxM && !decode_cols_fits(m, c.M)) {
       PackedMeta metas[8];
       size_t group_need = 0;
       n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), ~(size_t)0, metas, &group_need);

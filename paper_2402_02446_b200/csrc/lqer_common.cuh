@@ -60,6 +60,8 @@ constexpr int kTCountOffset = 64, kTDoneOffset = 68;
 constexpr int kDecodeMaxCtas = 160;
 constexpr int kPrologueRowTiles = 512;               // an arrival and a departure counter each: batches up to 65536 rows
 constexpr int kPrologueMaxCtas = 148;
+constexpr int kGemmMaxPairs = 74;                    // CTA pairs of the pair GEMM (one per two SMs)
+constexpr int kGemmSplitMaxM = 128;                  // batches up to this many rows (one row tile) may have their K range cut
 constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8 + kPrologueRowTiles * 8;
 __host__ __device__ inline size_t tacc_offset(const PackedMeta& m) {
   return (size_t)kStatusBytes + (((size_t)m.n_tiles * 4 + 255) & ~(size_t)255);
@@ -69,6 +71,21 @@ __host__ __device__ inline size_t pcount_offset(const PackedMeta& m) {
 }
 __host__ __device__ inline size_t persist_bytes(const PackedMeta& m) {
   return pcount_offset(m) + (size_t)kPrologueRowTiles * 8;
+}
+// Split-K form of the pair GEMM for small batches (one row tile, so few tiles): the number of K ranges, the scratch
+// for a batch of M rows, and a bound over all batches up to M_max.
+inline int gemm_splitk_ranges(const PackedMeta& m, int M) {
+  if (M > kGemmSplitMaxM) return 1;
+  int c = kGemmMaxPairs / ((m.n_tiles + 1) / 2);
+  if (c > 8) c = 8;
+  if (c > m.k_slabs / 8) c = m.k_slabs / 8;      // at least eight K stages per range
+  return c < 2 ? 1 : c;
+}
+inline size_t gemm_splitk_bytes(const PackedMeta& m, int M) {
+  return ((size_t)(gemm_splitk_ranges(m, M) - 1) * M * m.N * 4 + 255) & ~(size_t)255;
+}
+inline size_t gemm_splitk_bound(const PackedMeta& m, int M_max) {
+  return gemm_splitk_bytes(m, M_max < kGemmSplitMaxM ? M_max : kGemmSplitMaxM);
 }
 // Tensor-core prologue: a CTA owns 128 rows and one of `splits` ranges of K (in panels of 128 columns);
 // each CTA leaves a [128, k_pad] fp64 partial sum; once all CTAs of a row tile have arrived each adds up its share of rows.
@@ -251,6 +268,10 @@ cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const v
                            DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s);
+// Small batches: the layer's K range cut into gemm_splitk_ranges(m, M) ranges that run as layers of one launch;
+// `partials` holds (ranges - 1) * M * N floats (gemm_splitk_bytes).
+cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+                                   float* partials, DeviceStatus* st, cudaStream_t s);
 // Up to gemm_tc2_max_group() layers with one M in one launch (xcats, packed, Ys, metas: host arrays of n entries).
 int gemm_tc2_max_group();
 cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys,

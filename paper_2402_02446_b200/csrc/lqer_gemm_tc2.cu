@@ -65,6 +65,8 @@ struct Layer {
   float* Y;
   int N, K64;
   int n_tiles, k_slabs, r_blocks;
+  int slab0, slab_stride;      // a layer may be a K range of a real layer (split K): its first weight slab, and the
+                               // real layer's slab count (the stride between column tiles of the packed weights)
   int spt;                     // K stages per tile: k_slabs + rank stages
   int tile_begin;              // first tile of this layer in the launch's list (256 x 256 tiles, row tile fastest)
 };
@@ -144,6 +146,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
         const uint8_t* bsec = p.L[layer].bsec;
         const int k_slabs = p.L[layer].k_slabs, r_blocks = p.L[layer].r_blocks, K64 = p.L[layer].K64;
         const int stages_per_tile = p.L[layer].spt, n_tiles = p.L[layer].n_tiles;
+        const int slab0 = p.L[layer].slab0, slab_stride = p.L[layer].slab_stride;
         const int b_tile_stride = r_blocks * kTileN * 17;
         const int my_ntile = 2 * nt + (int)rank;
         const bool has_w = my_ntile < n_tiles;
@@ -153,9 +156,9 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           const uint32_t a_dst = smem_u32(stage_base + st * STAGE_BYTES);
           if (s < k_slabs) {
             mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? kWTileBytes : 0));
-            tma_load_2d(a_dst, tmap_x, s * BK, row0, loaded(st));
+            tma_load_2d(a_dst, tmap_x, (slab0 + s) * BK, row0, loaded(st));
             if (has_w)
-              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * k_slabs + s) * kWTileBytes, kWTileBytes,
+              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * slab_stride + slab0 + s) * kWTileBytes, kWTileBytes,
                         loaded(st));
           } else {
             const int rs = s - k_slabs;
@@ -379,6 +382,104 @@ static EncodeTiledFn encode_fn() {
 
 }  // namespace tc2
 
+namespace tc2 {
+
+static cudaError_t launch_params(const TensorMaps& tmaps, const Params& p, int sm_count, cudaStream_t s) {
+  const int max_pairs = sm_count / 2;
+  const int pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set up while the prologue drains
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  LaunchScope scope(kFamGemmTcPair, s);
+  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, tmaps, p);
+}
+
+// Y += P_0 + P_1 + ... in that order: the K ranges of a split layer other than the first.
+__global__ void __launch_bounds__(256) splitk_sum_kernel(float4* __restrict__ Y, const float4* __restrict__ P, int parts,
+                                                         size_t quads) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < quads; i += (size_t)gridDim.x * blockDim.x) {
+    float4 y = Y[i];
+    for (int c = 0; c < parts; ++c) {
+      const float4 v = __ldcs(P + (size_t)c * quads + i);
+      y.x += v.x; y.y += v.y; y.z += v.z; y.w += v.w;
+    }
+    Y[i] = y;
+  }
+}
+
+}  // namespace tc2
+
+// Small batches have few tiles; their K range is cut into ranges that run as layers of one launch, the first into Y,
+// the others into scratch that a second kernel adds to Y in a fixed order.
+cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+                                   float* partials, DeviceStatus* st, cudaStream_t s) {
+  using namespace tc2;
+  const int C = gemm_splitk_ranges(m, M);
+  if (C < 2) return launch_gemm_tc2(xcat, M, m, packed, Y, st, s);
+  if ((m.N & 3) != 0) return cudaErrorInvalidValue;
+  EncodeTiledFn enc = encode_fn();
+  if (enc == nullptr) return cudaErrorNotSupported;
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+  }
+  TensorMaps tmaps;
+  const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
+  const cuuint32_t box[2] = {BK, BM};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&tmaps.m[0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xcat), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  for (int g = 1; g < MAX_GROUP; ++g) tmaps.m[g] = tmaps.m[0];
+  Params p;
+  p.m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  const uint8_t* base = static_cast<const uint8_t*>(packed);
+  const int per_layer = p.m_tiles * ((m.n_tiles + 1) / 2);
+  // the last range (it carries the rank stages and is the longest) first
+  for (int slot = 0; slot < MAX_GROUP; ++slot) {
+    const int c = slot < C ? C - 1 - slot : C - 1;
+    const int lo = (int)((long long)c * m.k_slabs / C), hi = (int)((long long)(c + 1) * m.k_slabs / C);
+    Layer& ly = p.L[slot];
+    ly.wsec = base + m.off_w;
+    ly.bsec = base + m.off_b;
+    ly.Y = c == 0 ? Y : partials + (size_t)(c - 1) * M * m.N;
+    ly.N = m.N; ly.K64 = m.K64;
+    ly.n_tiles = m.n_tiles; ly.k_slabs = hi - lo;
+    ly.r_blocks = c == C - 1 ? m.r_blocks : 0;
+    ly.slab0 = lo; ly.slab_stride = m.k_slabs;
+    ly.spt = ly.k_slabs + (ly.r_blocks + 1) / 2;
+    ly.tile_begin = slot * per_layer;
+  }
+  p.group = C;
+  p.num_tiles = C * per_layer;
+  p.status = st;
+  p.M = M;
+  p.lr_shift = m.lr_bits - 2;
+  cudaError_t e = launch_params(tmaps, p, sm_count, s);
+  if (e != cudaSuccess) return e;
+  const size_t quads = (size_t)M * m.N / 4;
+  int blocks = (int)((quads + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  LaunchScope scope(kFamGemmTcPair, s);
+  splitk_sum_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<float4*>(Y), reinterpret_cast<const float4*>(partials), C - 1, quads);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s) {
   return launch_gemm_tc2_group(&xcat, &packed, &Y, &m, 1, M, st, s);
@@ -435,6 +536,7 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
     ly.Y = Ys[g];
     ly.N = m.N; ly.K64 = m.K64;
     ly.n_tiles = m.n_tiles; ly.k_slabs = m.k_slabs; ly.r_blocks = m.r_blocks;
+    ly.slab0 = 0; ly.slab_stride = m.k_slabs;
     ly.spt = m.k_slabs + (m.r_blocks + 1) / 2;
     ly.tile_begin = tile_begin;
     if (slot < n) tile_begin += p.m_tiles * ((m.n_tiles + 1) / 2);
@@ -444,24 +546,7 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
   p.status = st;
   p.M = M;
   p.lr_shift = metas[0].lr_bits - 2;
-  const int num_tiles = p.num_tiles;
-  const int max_pairs = sm_count / 2;
-  const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
-
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * pairs);
-  cfg.blockDim = dim3(NUM_THREADS);
-  cfg.dynamicSmemBytes = SMEM_BYTES;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may set up while the prologue drains
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 2;
-  LaunchScope scope(kFamGemmTcPair, s);
-  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel, tmaps, p);
+  return launch_params(tmaps, p, sm_count, s);
 }
 
 }  // namespace lqer
