@@ -165,7 +165,7 @@ lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, floa
  * same batch writes; the library uses that, with the path left at 0, to share launches:
  *  - up to 16 consecutive calls with one M <= 4 (any shapes with N >= 32, one set of formats)
  *    run as ONE launch of the decode kernel that divides the SMs among them by weight bytes;
- *  - up to 8 consecutive calls with one M > 128 (any shapes, one set of formats) run their
+ *  - up to 8 consecutive calls with one M > 256 (any shapes, one set of formats) run their
  *    prologues into separate slices of the workspace and then ONE GEMM launch over the tiles of
  *    all of them - if the workspace holds lqer_batched_workspace_bytes(calls, n_calls); with a
  *    smaller workspace (at least the largest lqer_workspace_bytes of the calls) fewer calls, or

@@ -193,7 +193,7 @@ static int same_shape_run(const lqer_call_t* calls, int first, int n_calls, cons
   }
   return n;
 }
-// Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M > 128,
+// Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M > 256,
 // the same formats, any shapes; at most `limit`, and only as many as the workspace has slices for.
 static bool same_formats(const PackedMeta& a, const PackedMeta& b) {
   return a.w_bits == b.w_bits && a.a_bits == b.a_bits && a.lr_bits == b.lr_bits && a.exp_min == b.exp_min &&

@@ -61,7 +61,7 @@ constexpr int kDecodeMaxCtas = 160;
 constexpr int kPrologueRowTiles = 512;               // an arrival and a departure counter each: batches up to 65536 rows
 constexpr int kPrologueMaxCtas = 148;
 constexpr int kGemmMaxPairs = 74;                    // CTA pairs of the pair GEMM (one per two SMs)
-constexpr int kGemmSplitMaxM = 128;                  // batches up to this many rows (one row tile) may have their K range cut
+constexpr int kGemmSplitMaxM = 256;                  // batches up to this many rows (one row tile) may have their K range cut
 constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8 + kPrologueRowTiles * 8;
 __host__ __device__ inline size_t tacc_offset(const PackedMeta& m) {
   return (size_t)kStatusBytes + (((size_t)m.n_tiles * 4 + 255) & ~(size_t)255);
