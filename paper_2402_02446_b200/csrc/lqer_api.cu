@@ -164,7 +164,7 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
     uint8_t* wsb = static_cast<uint8_t*>(workspace);
     err = tc_prologue ? launch_prologue_tc(X, M, m, packed, xcat, Tm, Te, dst,
                                            reinterpret_cast<double*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M)),
-                                           reinterpret_cast<int*>(wsb + pcount_offset(m)), s)
+                                           reinterpret_cast<int*>(wsb + pcount_offset(m)), kPrologueAlone, s)
                       : launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
       err = (path == 1)   ? launch_gemm_simt(xcat, M, m, packed, Y, s)
@@ -229,16 +229,23 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
   const void* xcats[8];
   const void* packed[8];
   float* Ys[8];
+  // The prologues of the group share nothing but the status word: each has its slice of the workspace, and, while the
+  // counter pairs last, its own range of them, so that each may overlap the tail of the one before.
+  size_t count_base = 0;
+  for (int g = 0; g < n; ++g) count_base = std::max(count_base, pcount_offset(metas[g]));
+  const int row_tiles = (M + 127) / 128;
+  const bool own_counters = (long long)row_tiles * n <= kPrologueRowTiles;
   size_t off = head;
   for (int g = 0; g < n; ++g) {
     const PackedMeta& m = metas[g];
     uint8_t* xcat = wsb + off;
     off += group_slice_bytes(m, M);
     const float* X = calls[g].X;
+    int* counters = reinterpret_cast<int*>(wsb + count_base) + (own_counters ? (size_t)g * row_tiles * 2 : 0);
+    const int order = !own_counters ? kPrologueAlone : g == 0 ? kPrologueGroupFirst : kPrologueGroupLater;
     cudaError_t err = prologue_tc_fits(m, M, X, false)
                           ? launch_prologue_tc(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
-                                               reinterpret_cast<double*>(xcat + xcat_bytes(m, M)),
-                                               reinterpret_cast<int*>(wsb + pcount_offset(m)), s)
+                                               reinterpret_cast<double*>(xcat + xcat_bytes(m, M)), counters, order, s)
                           : launch_prologue(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
     if (err != cudaSuccess) return LQER_ERR_CUDA;
     xcats[g] = xcat; packed[g] = calls[g].packed; Ys[g] = calls[g].Y;

@@ -258,10 +258,13 @@ cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const vo
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s);
 // The same prologue with the projection on the tcgen05 int8 tensor cores: ranks up to 64, large batches.
 bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch);
-// `partials`: prologue_tc_scratch_bytes(m, M) of scratch; `counters`: the zeroed counter pairs of the workspace head.
+// `partials`: prologue_tc_scratch_bytes(m, M) of scratch; `counters`: zeroed counter pairs of the workspace head,
+// one per row tile.  `order`: kPrologueAlone, or the place in a run of prologues that share no buffer or counter
+// (each later one overlaps the tail of the one before; the kernel after the run still finds all of them complete).
+enum PrologueOrder { kPrologueAlone = 0, kPrologueGroupFirst = 1, kPrologueGroupLater = 2 };
 cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
-                               cudaStream_t s);
+                               int order, cudaStream_t s);
 cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                              cudaStream_t s);
 cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,

@@ -78,6 +78,7 @@ struct Params {
   int panels;               // ceil(K64 / 128)
   int splits;               // CTAs per row tile
   int a_bits, lr_bits, exp_min, exp_max;
+  int order;                // PrologueOrder: where the wait for the previous kernel sits
   size_t ldx;               // columns of Xcat
 };
 
@@ -178,9 +179,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // set up; the next kernel may start its own setup, and X, Xcat and the scratch may still be in use by an earlier one
-  pdl_launch_dependents();
-  pdl_wait();
+  // Set up.  Alone: the next kernel may start its own setup at once; X, Xcat and the scratch may still be in use by
+  // an earlier kernel, so the work waits for it.  First of a group of independent prologues: the next one starts
+  // only once the earlier kernels are done, since it does not wait before it works.  Later in a group: nothing here
+  // is shared with the prologue before, so the work starts at once and only the exit waits for it (a kernel after
+  // the group then finds all of them complete).
+  if (p.order == kPrologueGroupFirst) {
+    pdl_wait();
+    pdl_launch_dependents();
+  } else {
+    pdl_launch_dependents();
+    if (p.order == kPrologueAlone) pdl_wait();
+  }
 
   if (warp < SW) {
     // ------------------------------------------------------------------ scalers
@@ -432,6 +442,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     *arrive_cnt = 0;
     *depart_cnt = 0;
   }
+  if (p.order == kPrologueGroupLater) pdl_wait();
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -484,7 +495,7 @@ bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch
 
 cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
-                               cudaStream_t s) {
+                               int order, cudaStream_t s) {
   using namespace ptc;
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
@@ -507,6 +518,7 @@ cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const
   p.panels = (m.K64 + 127) / 128;
   p.splits = prologue_tc_splits(m, M);
   p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
+  p.order = order;
   p.ldx = xcat_cols(m);
   const int ctas = ((M + ROWS - 1) / ROWS) * p.splits;
   switch (m.k_pad) {
