@@ -11,12 +11,13 @@
 // those groups, and the 16 warps' sums meet once in shared memory and are added in warp order.
 // Y is written once, by one thread per element, with no global synchronisation.
 //
-// Lane (g, t) of a warp keeps, for column g of a group, the exact integer dot product of block t
-// of the slab: four dp4a on the raw nibbles against the int8 mantissas of X (stored in the byte
-// order the nibbles unpack to), minus 8 * sum(x) for the offset-binary nibbles; the block result
-// is scaled by 2^(e_x + e_w) in fp32 and accumulated per token.  A warp's share of a unit (256
-// bytes of nibbles + 32 exponent bytes) goes global -> registers, four slabs (16 units) ahead;
-// these loads depend on no earlier kernel and are issued before griddepcontrol.wait.
+// A lane of a warp owns one of the round's 32 columns and takes a whole slab of it at a time: the
+// four 16-blocks of the slab as two 16-byte loads plus the four exponent bytes as one word.  Per
+// block: four dp4a on the raw nibbles against the int8 mantissas of X (stored in the byte order the
+// nibbles unpack to), started from 1.5 * 2^23 - 8 * sum(x) (the offset-binary nibbles; the constant
+// makes the integer sum the bit pattern of a float, so one subtraction converts it), scaled by
+// 2^(e_x + e_w) in fp32 and accumulated per token.  The loads run four slabs ahead; they depend on
+// no earlier kernel and are issued before griddepcontrol.wait.
 //
 // T = X_q A_q is needed by every CTA.  The CTAs of a cluster of four share the work: each takes a
 // quarter of K (exact int8 tensor-core MMA per 16-block on the X mantissas already in shared
@@ -31,8 +32,8 @@ namespace dcol {
 constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 constexpr int kMaxM = 4;
-constexpr int kCg = 4;            // column groups (of 8 columns) per round
-constexpr int kSets = 4;          // slabs a warp keeps in flight (x kCg units each)
+constexpr int kCg = 4;            // column groups (of 8 columns) per round: one column per lane
+constexpr int kSets = 4;          // slabs a warp keeps in flight
 constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q (pairs would fill all 148 SMs instead of 132, but the doubled share of T costs more than that gains)
 constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
 constexpr int kAStageMax = 100 * 1024;   // a CTA's share of A_q is staged in shared memory if it fits in this
@@ -57,19 +58,21 @@ struct Params {
   int a_bits, lr_bits, exp_min, exp_max;
 };
 
-struct UnitRegs {
-  uint2 w;      // block t of the slab for column g: 16 nibbles
-  uint32_t e;   // its exponent byte
+struct SlabRegs {
+  uint4 h0, h1;   // one column of a slab: blocks 0, 1 and blocks 2, 3 (16 nibbles = two words each)
+  uint32_t e;     // the four exponent bytes
 };
+constexpr float kIntMagic = 12582912.f;          // 1.5 * 2^23: int v (|v| < 2^22) + 0x4B400000 is the bit pattern of kIntMagic + v
+constexpr int kIntMagicBits = 0x4B400000;
 
 __device__ __forceinline__ uint32_t ld_stream_u32(const void* p) {
   uint32_t v;
   asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
 }
-__device__ __forceinline__ uint2 ld_stream_u64(const void* p) {
-  uint2 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+__device__ __forceinline__ uint4 ld_stream_u128(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
 __device__ __forceinline__ uint32_t ld_stream_u8(const void* p) {
@@ -111,8 +114,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const int M = p.M, KB = ly.K64 / 16;
   uint8_t* xm = smem;                                               // [M][K64] int8 mantissas, permuted within 8
   float* xsc = reinterpret_cast<float*>(xm + (size_t)M * ly.K64);    // [M][KB] 2^(e_x - 6)
-  int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);          // [M][KB] 8 * sum(x) of the block
-  float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // [kWarps][kCg][8][kMaxM]
+  int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);          // [M][KB] bits of 1.5 * 2^23, minus 8 * sum(x) of the block
+  float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // [kWarps][32 columns][kMaxM]
   double* tpart = reinterpret_cast<double*>(red + kWarps * kCg * 8 * kMaxM);   // [M][k_pad] this CTA's partial T
   double* tsub = tpart + (size_t)kMaxM * ly.k_pad;                   // [subsets][M][k_pad] per-warp-subset partials
   float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * kMaxSubsets);   // [M][k_pad / 16]
@@ -121,7 +124,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       (reinterpret_cast<uintptr_t>(tq8) + (size_t)kMaxM * (ly.k_pad > 0 ? ly.k_pad : 16) + 15) & ~(uintptr_t)15);   // staged A_q
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;
+  const int g = lane >> 2, t = lane & 3;             // fragment coordinates of the T part's MMA
   const int G = ly.ctas, cta = (int)blockIdx.x - ly.cta_begin;
   const float* const X = ly.X;
   float* const Y = ly.Y;
@@ -130,54 +133,52 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const uint8_t* const asec = ly.packed + ly.off_a;
   const int cg_lo = cta * ly.n_cg / G, cg_hi = (cta + 1) * ly.n_cg / G;
 
-  // This lane's share of (column group cg, slab j): global -> registers.  Byte offsets into the W section are kept
-  // per column group (32 bits: the section is far below 4 GB); a load then costs two adds.  Column groups past the
+  // This lane's column of a round (the 32 columns from column group cg0 on) and slab j: global -> registers.  Byte
+  // offsets into the W section are kept per round (32 bits: the section is far below 4 GB).  Column groups past the
   // CTA's range are clamped to its last one and slabs past K to the last slab: such loads stay inside the section
   // and what they return is never used (the sums of those slabs are skipped, those columns are not stored).
-  const uint32_t lane_w = (uint32_t)((t >> 1) * (kTileN * 16) + g * 16 + (t & 1) * 8);
-  const uint32_t lane_e = (uint32_t)(kWTileNibbleBytes + g * 4 + t);
-  struct GroupOff { uint32_t w, e; };
-  auto group_off = [&](int cg) -> GroupOff {
-    cg = max(min(cg, cg_hi - 1), 0);
+  const uint32_t lane_w = (uint32_t)((lane & 7) * 16);
+  const uint32_t lane_e = (uint32_t)(kWTileNibbleBytes + (lane & 7) * 4);
+  struct ColOff { uint32_t w, e; };
+  auto col_off = [&](int cg0) -> ColOff {
+    const int cg = max(min(cg0 + (lane >> 3), cg_hi - 1), 0);
     const uint32_t tile = (uint32_t)(cg >> 4) * (uint32_t)ly.k_slabs * (uint32_t)kWTileBytes;
-    GroupOff o;
+    ColOff o;
     o.w = tile + (uint32_t)(cg & 15) * 128u + lane_w;
     o.e = tile + (uint32_t)(cg & 15) * 32u + lane_e;
     return o;
   };
-  auto fetch = [&](UnitRegs& d, const GroupOff& o, int j) {
+  auto fetch = [&](SlabRegs& d, const ColOff& o, int j) {
     const uint32_t jo = (uint32_t)min(j, ly.k_slabs - 1) * (uint32_t)kWTileBytes;
-    d.w = ld_stream_u64(wsec + (o.w + jo));
-    d.e = ld_stream_u8(wsec + (o.e + jo));
+    d.h0 = ld_stream_u128(wsec + (o.w + jo));
+    d.h1 = ld_stream_u128(wsec + (o.w + jo + (uint32_t)(kTileN * 16)));
+    d.e = ld_stream_u32(wsec + (o.e + jo));
   };
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  // this lane's share of (column group cg, rank block warp) of B_q: rank values 4t..4t+3 and the exponent byte
-  auto fetch_rank = [&](uint32_t& wv, uint32_t& eb, int cg) {
-    wv = 0u;
+  // this lane's column of rank block `warp` of B_q: its 16 rank values and the exponent byte
+  auto fetch_rank = [&](uint4& wv, uint32_t& eb, int cg0) {
+    wv = make_uint4(0u, 0u, 0u, 0u);
     eb = 127u;
+    const int cg = cg0 + (lane >> 3);
     if (cg < cg_hi && warp < ly.r_blocks) {
-      const int col = (cg & 15) * 8 + g;
+      const int col = (cg & 15) * 8 + (lane & 7);
       const uint8_t* tile = bsec + (size_t)(cg >> 4) * ((size_t)ly.r_blocks * kTileN * 17);
-      wv = ld_stream_u32(tile + ((size_t)warp * kTileN + col) * 16 + t * 4);
+      wv = ld_stream_u128(tile + ((size_t)warp * kTileN + col) * 16);
       eb = ld_stream_u8(tile + (size_t)ly.r_blocks * kTileN * 16 + warp * kTileN + col);
     }
   };
 
-  UnitRegs regs[kSets][kCg];
-  uint32_t rank_w[kCg], rank_e[kCg];
+  SlabRegs regs[kSets];
+  uint4 rank_w;
+  uint32_t rank_e;
   // weights depend on no earlier kernel: request the first slabs, the rank blocks and this CTA's
   // share of A_q before the dependency wait
-  GroupOff o_cur[kCg], o_nxt[kCg];               // offsets of this round's and the next round's column groups
+  ColOff o_cur = col_off(cg_lo), o_nxt;          // offsets of this round's and the next round's columns
 #pragma unroll
-  for (int u = 0; u < kCg; ++u) o_cur[u] = group_off(cg_lo + u);
-#pragma unroll
-  for (int s = 0; s < kSets; ++s)
-#pragma unroll
-    for (int u = 0; u < kCg; ++u) fetch(regs[s][u], o_cur[u], warp + kWarps * s);
-#pragma unroll
-  for (int u = 0; u < kCg; ++u) fetch_rank(rank_w[u], rank_e[u], cg_lo + u);
+  for (int s = 0; s < kSets; ++s) fetch(regs[s], o_cur, warp + kWarps * s);
+  fetch_rank(rank_w, rank_e, cg_lo);
   const int KBr = ly.K / 16;
   const int cs = (int)cluster_nctarank(), cr = (int)cluster_ctarank();
   const int kb_lo = cr * KBr / cs, kb_hi = (cr + 1) * KBr / cs;      // this CTA's share of K for T
@@ -218,7 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
         *reinterpret_cast<uint32_t*>(xm + (size_t)row * ly.K64 + c4 * 4) = perm;
         if ((c4 & 3) == 0) {
           xsc[row * KB + (c4 >> 2)] = pow2f(e - (p.a_bits - 2));
-          xof[row * KB + (c4 >> 2)] = 8 * sum;
+          xof[row * KB + (c4 >> 2)] = kIntMagicBits - 8 * sum;
         }
       }
     }
@@ -279,56 +280,61 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const int slabs_mine = ly.k_slabs > warp ? (ly.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
 #pragma unroll 1
   for (int cg0 = cg_lo; cg0 < cg_hi; cg0 += kCg) {
-    float acc[kCg][MT];
+    float acc[MT];
 #pragma unroll
-    for (int u = 0; u < kCg; ++u)
-#pragma unroll
-      for (int r = 0; r < MT; ++r) acc[u][r] = 0.f;
+    for (int r = 0; r < MT; ++r) acc[r] = 0.f;
+    o_nxt = col_off(cg0 + kCg);
 
-#pragma unroll
-    for (int u = 0; u < kCg; ++u) o_nxt[u] = group_off(cg0 + kCg + u);
-
-    // ---- W_q: this warp's slabs of the round's column groups
+    // ---- W_q: this warp's slabs of the round's columns
 #pragma unroll 1
     for (int js = 0; js < slabs_mine; js += kSets) {
 #pragma unroll
       for (int s = 0; s < kSets; ++s) {
         const int j = warp + kWarps * (js + s);
         if (j < ly.k_slabs) {
+          const SlabRegs d = regs[s];
+          // nibbles as bytes: k {0,4,1,5}, {2,6,3,7}, {8,12,9,13}, {10,14,11,15} of each block
+          const uint32_t wd[8] = {d.h0.x, d.h0.y, d.h0.z, d.h0.w, d.h1.x, d.h1.y, d.h1.z, d.h1.w};
+          uint32_t nib[16];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            nib[2 * i] = wd[i] & 0x0F0F0F0Fu;
+            nib[2 * i + 1] = (wd[i] >> 4) & 0x0F0F0F0Fu;
+          }
+          float sw[4];                                               // 2^(e_w - 2) of the four blocks
+#pragma unroll
+          for (int b = 0; b < 4; ++b) sw[b] = __uint_as_float((((d.e >> (8 * b)) & 0xFFu) - 2u) << 23);
 #pragma unroll
           for (int r = 0; r < MT; ++r) {
             if (r < M) {
-              const uint4 x = *reinterpret_cast<const uint4*>(xm + (size_t)r * ly.K64 + j * 64 + t * 16);
-              const float sx = xsc[r * KB + j * 4 + t];
-              const int off = xof[r * KB + j * 4 + t];
+              const uint4* xp = reinterpret_cast<const uint4*>(xm + (size_t)r * ly.K64 + j * 64);
+              const float4 sx = *reinterpret_cast<const float4*>(xsc + r * KB + j * 4);      // 2^(e_x - 6)
+              const int4 seed = *reinterpret_cast<const int4*>(xof + r * KB + j * 4);
+              const float sxa[4] = {sx.x, sx.y, sx.z, sx.w};
+              const int seeda[4] = {seed.x, seed.y, seed.z, seed.w};
 #pragma unroll
-              for (int u = 0; u < kCg; ++u) {
-                const UnitRegs d = regs[s][u];
-                // nibbles as bytes: k {0,4,1,5}, {2,6,3,7}, {8,12,9,13}, {10,14,11,15} of the block
-                int sm = __dp4a((int)x.x, (int)(d.w.x & 0x0F0F0F0Fu), -off);
-                sm = __dp4a((int)x.y, (int)((d.w.x >> 4) & 0x0F0F0F0Fu), sm);
-                sm = __dp4a((int)x.z, (int)(d.w.y & 0x0F0F0F0Fu), sm);
-                sm = __dp4a((int)x.w, (int)((d.w.y >> 4) & 0x0F0F0F0Fu), sm);
-                acc[u][r] = fmaf((float)sm, sx * __uint_as_float((d.e - 2u) << 23), acc[u][r]);   // 2^(e_x - 6) 2^(e_w - 2)
+              for (int b = 0; b < 4; ++b) {
+                const uint4 x = xp[b];
+                int sm = __dp4a((int)x.x, (int)nib[4 * b], seeda[b]);
+                sm = __dp4a((int)x.y, (int)nib[4 * b + 1], sm);
+                sm = __dp4a((int)x.z, (int)nib[4 * b + 2], sm);
+                sm = __dp4a((int)x.w, (int)nib[4 * b + 3], sm);
+                acc[r] = fmaf(__int_as_float(sm) - kIntMagic, sxa[b] * sw[b], acc[r]);
               }
             }
           }
         }
-        // refill the set: the same groups four slabs on, or - past this warp's last slabs - the
-        // next round's groups from their first slabs, so that rounds follow each other without a bubble
+        // refill the set: the same columns four slabs on, or - past this warp's last slabs - the
+        // next round's columns from their first slabs, so that rounds follow each other without a bubble
         const bool more = js + kSets < slabs_mine;
         const int jn = more ? j + kWarps * kSets : warp + kWarps * s;
-#pragma unroll
-        for (int u = 0; u < kCg; ++u) {
-          GroupOff o;
-          o.w = more ? o_cur[u].w : o_nxt[u].w;
-          o.e = more ? o_cur[u].e : o_nxt[u].e;
-          fetch(regs[s][u], o, jn);
-        }
+        ColOff o;
+        o.w = more ? o_cur.w : o_nxt.w;
+        o.e = more ? o_cur.e : o_nxt.e;
+        fetch(regs[s], o, jn);
       }
     }
-#pragma unroll
-    for (int u = 0; u < kCg; ++u) o_cur[u] = o_nxt[u];
+    o_cur = o_nxt;
 
     // ---- B_q against T_q: rank blocks warp, warp + 16, ...
     if (ly.k_pad > 0) {
@@ -360,43 +366,34 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       }
       const int rbn = ly.k_pad / 16;
       if (warp < ly.r_blocks) {                   // rank block `warp` (k <= 256: at most 16 blocks); data already in registers
+        const float sb = __uint_as_float((rank_e - (uint32_t)(p.lr_bits - 2)) << 23);           // 2^(e_b - 6)
 #pragma unroll
-        for (int u = 0; u < kCg; ++u) {
-          const float sb = __uint_as_float((rank_e[u] - (uint32_t)(p.lr_bits - 2)) << 23);        // 2^(e_b - 6)
-#pragma unroll
-          for (int r = 0; r < MT; ++r) {
-            if (r < M) {
-              const int tw = *reinterpret_cast<const int*>(tq8 + r * ly.k_pad + warp * 16 + t * 4);
-              acc[u][r] = fmaf((float)__dp4a(tw, (int)rank_w[u], 0), tqs[r * rbn + warp] * sb, acc[u][r]);
-            }
+        for (int r = 0; r < MT; ++r) {
+          if (r < M) {
+            const uint4 tw = *reinterpret_cast<const uint4*>(tq8 + r * ly.k_pad + warp * 16);
+            int sm = __dp4a((int)tw.x, (int)rank_w.x, 0);
+            sm = __dp4a((int)tw.y, (int)rank_w.y, sm);
+            sm = __dp4a((int)tw.z, (int)rank_w.z, sm);
+            sm = __dp4a((int)tw.w, (int)rank_w.w, sm);
+            acc[r] = fmaf((float)sm, tqs[r * rbn + warp] * sb, acc[r]);
           }
         }
       }
-#pragma unroll
-      for (int u = 0; u < kCg; ++u) fetch_rank(rank_w[u], rank_e[u], cg0 + kCg + u);   // the next round's rank blocks
+      fetch_rank(rank_w, rank_e, cg0 + kCg);     // the next round's rank blocks
     }
 
-    // ---- the four lanes of a column, then the 16 warps (fixed order), then Y
+    // ---- the 16 warps' sums of a column (fixed order), then Y
 #pragma unroll
-    for (int u = 0; u < kCg; ++u) {
-      float mine = 0.f;
-#pragma unroll
-      for (int r = 0; r < MT; ++r) {
-        float v = acc[u][r];
-        v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-        v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-        if (r == t) mine = v;
-      }
-      red[((warp * kCg + u) * 8 + g) * kMaxM + t] = mine;          // lane t hands row t over
-    }
+    for (int r = 0; r < MT; ++r) red[(warp * 32 + lane) * kMaxM + r] = acc[r];
     __syncthreads();
-    if (tid < kCg * 8 * kMaxM) {
-      const int u = tid >> 5, gg = (tid >> 2) & 7, r = tid & 3;
-      float v = 0.f;
+    if (tid < 32 * kMaxM) {
+      const int col = tid >> 2, r = tid & 3;
+      if (cg0 + (col >> 3) < cg_hi && r < M) {
+        float v = 0.f;
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) v += red[((w * kCg + u) * 8 + gg) * kMaxM + r];
-      const int cg = cg0 + u;
-      if (cg < cg_hi && r < M) Y[(size_t)r * ly.N + cg * 8 + gg] = v;
+        for (int w = 0; w < kWarps; ++w) v += red[(w * 32 + col) * kMaxM + r];
+        Y[(size_t)r * ly.N + cg0 * 8 + col] = v;
+      }
     }
     __syncthreads();                             // red is rewritten by the next round
   }
