@@ -217,6 +217,29 @@ static int prefill_run(const lqer_call_t* calls, int first, int n_calls, int lim
   if (need != nullptr) *need = head + slices;
   return n;
 }
+// The run of decode calls from calls[first] on that may share one launch of the column-owner kernel: one M, one set of
+// formats, each fitting the kernel, at least 32 columns, and a slot for each layer's partial sums of T in the workspace.
+static int decode_run(const lqer_call_t* calls, int first, int n_calls, int max_group, size_t workspace_bytes,
+                      PackedMeta* metas, size_t* need) {
+  PackedMeta m0;
+  if (lookup(calls[first].packed, m0) != LQER_OK || !decode_cols_fits(m0, calls[first].M)) return 0;
+  metas[0] = m0;
+  size_t head = align_up(persist_bytes(m0), 256), slots = decode_cols_slot_bytes(m0);
+  int n = 1;
+  while (first + n < n_calls && n < max_group) {
+    PackedMeta m1;
+    if (calls[first + n].M != calls[first].M || lookup(calls[first + n].packed, m1) != LQER_OK ||
+        !same_formats(m0, m1) || !decode_cols_fits(m1, calls[first].M) || m1.N < 32 || m0.N < 32)
+      break;
+    const size_t h = std::max(head, align_up(persist_bytes(m1), 256));
+    if (h + slots + decode_cols_slot_bytes(m1) > workspace_bytes) break;
+    head = h;
+    slots += decode_cols_slot_bytes(m1);
+    metas[n++] = m1;
+  }
+  if (need != nullptr) *need = head + slots;
+  return n;
+}
 // n prefill layers with one M: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
 // the tiles of all of them.
 static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace,
@@ -433,22 +456,16 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
   const bool may_group = g_path.load() == 0;   // a forced path runs every call on its own
   for (int i = 0; i < n_calls;) {
     // The calls are independent, so consecutive calls of one shape (the q, k, v projections of a layer, or its gate
-    // and up projections) share launches: decode calls one launch of the column-owner kernel (it keeps nothing in the
-    // workspace), prefill calls one GEMM launch after their prologues, if the workspace has a slice for each.
+    // and up projections) share launches: decode calls one launch of the column-owner kernel (a slot of the workspace per
+    // layer for the partial sums of T), prefill calls one GEMM launch after their prologues, if the workspace has a
+    // slice for each.
     int n = 1;
     PackedMeta m0, metas[16];
     bool decode_group = false;
     if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
       if (decode_cols_fits(m0, calls[i].M)) {
-        // decode calls with one M and one set of formats, each served by the column-owner kernel
-        metas[0] = m0;
-        while (i + n < n_calls && n < decode_cols_max_group()) {
-          PackedMeta m1;
-          if (calls[i + n].M != calls[i].M || lookup(calls[i + n].packed, m1) != LQER_OK || !same_formats(m0, m1) ||
-              !decode_cols_fits(m1, calls[i].M) || m1.N < 32 || m0.N < 32)
-            break;
-          metas[n++] = m1;
-        }
+        n = decode_run(calls, i, n_calls, decode_cols_max_group(), workspace_bytes, metas, nullptr);
+        if (n < 1) n = 1;
         decode_group = n > 1;
       } else if (calls[i].M > kGemmSplitMaxM) {   // smaller batches run split K, each on its own
         n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), workspace_bytes, metas, nullptr);
@@ -488,7 +505,13 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
     if (st != LQER_OK) return st;
     need = std::max(need, workspace_total(m, c.M));
     int n = 1;
-    if (c.M > kGemmSplitMaxM && !decode_cols_fits(m, c.M)) {
+    if (decode_cols_fits(m, c.M)) {
+      PackedMeta metas[16];
+      size_t group_need = 0;
+      n = decode_run(calls, i, n_calls, decode_cols_max_group(), ~(size_t)0, metas, &group_need);
+      if (n < 1) n = 1;
+      need = std::max(need, group_need);
+    } else if (c.M > kGemmSplitMaxM) {
       PackedMeta metas[8];
       size_t group_need = 0;
       n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), ~(size_t)0, metas, &group_need);

@@ -116,8 +116,11 @@ inline int decode_ctas(const PackedMeta& m, int sm_count) {
   if (g > kDecodeMaxCtas) g = kDecodeMaxCtas;
   return g;
 }
+// Scratch of the column-owner decode kernel: fp64 partial sums of T, [16 ranges of K][4 rows][k_pad].
+inline size_t decode_cols_slot_bytes(const PackedMeta& m) { return (size_t)16 * 4 * m.k_pad * 8; }
 inline size_t decode_scratch_bytes(const PackedMeta& m) {
-  return (size_t)decode_ctas(m, kDecodeMaxCtas) * 2 * 16 * kTileN * 4;
+  const size_t a = (size_t)decode_ctas(m, kDecodeMaxCtas) * 2 * 16 * kTileN * 4, b = decode_cols_slot_bytes(m);
+  return a > b ? a : b;
 }
 
 __host__ __device__ inline int b_tile_bytes(const PackedMeta& m) { return m.r_blocks * kTileN * 17; }

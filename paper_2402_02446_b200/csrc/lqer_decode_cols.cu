@@ -19,11 +19,14 @@
 // 2^(e_x + e_w) in fp32 and accumulated per token.  The loads run four slabs ahead; they depend on
 // no earlier kernel and are issued before griddepcontrol.wait.
 //
-// T = X_q A_q is needed by every CTA.  The CTAs of a cluster of four share the work: each takes a
-// quarter of K (exact int8 tensor-core MMA per 16-block on the X mantissas already in shared
-// memory, scaled and summed in fp64 in a fixed order), publishes its partial T in its own shared
-// memory, and after a cluster barrier (arrive early, wait just before the rank part) reads the
-// other three through distributed shared memory.  No global atomics, no workspace state.
+// T = X_q A_q is needed by every CTA of a layer, but only after the first round's W_q part.  Up to 16
+// CTAs of the layer take a range of K each (exact int8 tensor-core MMA per 16-block on the X
+// mantissas already in shared memory, scaled and summed in fp64 in a fixed order), leave their
+// partial T in a scratch slot of the workspace and count themselves in; every CTA streams its
+// first round of weights, then waits (bounded) for the count, adds the slots in range order and
+// quantises T.  All CTAs of a launch are resident together (at most one per SM), so the count is
+// reached while the weights stream; a second counter lets the last CTA to have read the slots zero
+// both for the next call.
 #include "lqer_common.cuh"
 
 namespace lqer {
@@ -34,11 +37,12 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kMaxM = 4;
 constexpr int kCg = 4;            // column groups (of 8 columns) per round: one column per lane
 constexpr int kSets = 4;          // slabs a warp keeps in flight
-constexpr int kClusterSize = 4;   // CTAs that share the work of T = X_q A_q (pairs would fill all 148 SMs instead of 132, but the doubled share of T costs more than that gains)
+constexpr int kTRanges = 16;      // CTAs of a layer that share the work of T = X_q A_q (ranges of K), at most
 constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
 constexpr int kAStageMax = 100 * 1024;   // a CTA's share of A_q is staged in shared memory if it fits in this
 
 constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
+constexpr long long kSpinLimitCycles = 4000000000LL;   // about two seconds
 
 struct Layer {
   const float* X;
@@ -47,7 +51,10 @@ struct Layer {
   size_t off_w, off_b, off_a;   // sections of the packed buffer
   int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
   int a_stage_bytes;            // shared memory reserved for staging A_q (0: read it from global memory)
-  int cta_begin, ctas;          // this layer's CTAs in the launch: whole clusters, in proportion to its weight bytes
+  int cta_begin, ctas;          // this layer's CTAs in the launch, in proportion to its weight bytes
+  int t_ranges;                 // the first t_ranges of them compute T, a range of K each
+  double* tslot;                // [t_ranges][M][k_pad] partial sums of T (workspace scratch)
+  int* tcount;                  // arrivals, departures: zero between calls
 };
 
 struct Params {
@@ -80,27 +87,6 @@ __device__ __forceinline__ uint32_t ld_stream_u8(const void* p) {
   asm volatile("ld.global.nc.L1::no_allocate.u8 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
 }
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t cluster_nctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
-// Read a double from the same shared-memory offset in another CTA of the cluster.
-__device__ __forceinline__ double ld_dsmem_f64(const double* local, uint32_t cta) {
-  uint32_t remote;
-  double v;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(cta));
-  asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(remote) : "memory");
-  return v;
-}
-
 // MT: rows the accumulators are compiled for (1 for the single-token call, kMaxM otherwise); M <= MT.
 template <int MT>
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
@@ -116,8 +102,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   float* xsc = reinterpret_cast<float*>(xm + (size_t)M * ly.K64);    // [M][KB] 2^(e_x - 6)
   int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);          // [M][KB] bits of 1.5 * 2^23, minus 8 * sum(x) of the block
   float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // [kWarps][32 columns][kMaxM]
-  double* tpart = reinterpret_cast<double*>(red + kWarps * kCg * 8 * kMaxM);   // [M][k_pad] this CTA's partial T
-  double* tsub = tpart + (size_t)kMaxM * ly.k_pad;                   // [subsets][M][k_pad] per-warp-subset partials
+  double* tsub = reinterpret_cast<double*>(red + kWarps * kCg * 8 * kMaxM);   // [subsets][M][k_pad] per-warp-subset partials of T
+  int* wait_ok = reinterpret_cast<int*>(tsub);                       // reused once T's partial sums have left: outcome of the wait
   float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * kMaxSubsets);   // [M][k_pad / 16]
   int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);        // [M][k_pad]
   uint8_t* a_stage = reinterpret_cast<uint8_t*>(
@@ -180,9 +166,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   for (int s = 0; s < kSets; ++s) fetch(regs[s], o_cur, warp + kWarps * s);
   fetch_rank(rank_w, rank_e, cg_lo);
   const int KBr = ly.K / 16;
-  const int cs = (int)cluster_nctarank(), cr = (int)cluster_ctarank();
-  const int kb_lo = cr * KBr / cs, kb_hi = (cr + 1) * KBr / cs;      // this CTA's share of K for T
-  const bool a_staged = ly.k_pad > 0 && (kb_hi - kb_lo) * ly.k_pad * 17 <= ly.a_stage_bytes;
+  const bool t_worker = ly.k_pad > 0 && cta < ly.t_ranges;
+  const int kb_lo = t_worker ? cta * KBr / ly.t_ranges : 0;          // this CTA's share of K for T
+  const int kb_hi = t_worker ? (cta + 1) * KBr / ly.t_ranges : 0;
+  const bool a_staged = t_worker && (kb_hi - kb_lo) * ly.k_pad * 17 <= ly.a_stage_bytes;
   if (a_staged) {
     const int mant = (kb_hi - kb_lo) * ly.k_pad * 16, ex = (kb_hi - kb_lo) * ly.k_pad;
     const uint8_t* gm = asec + (size_t)kb_lo * ly.k_pad * 16;
@@ -231,7 +218,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   //      mantissas in shared memory, scaled in fp64.  The products are exact; their fp64 sums are exact
   //      too unless the block exponents of one row spread over more than about 30 binades, and the
   //      order of the additions is fixed in any case.
-  if (ly.k_pad > 0) {
+  if (t_worker) {
     const int NT = ly.k_pad / 8;
     // A_q of blocks kb_lo..kb_hi: staged copy, or global memory
     const uint8_t* a_mant = a_staged ? a_stage - (size_t)kb_lo * ly.k_pad * 16 : asec;
@@ -270,12 +257,58 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       const int row = idx / ly.k_pad, col = idx % ly.k_pad;
       double v = 0.0;
       for (int q = 0; q < subsets; ++q) v += tsub[((size_t)q * kMaxM + row) * ly.k_pad + col];
-      tpart[row * ly.k_pad + col] = v;
+      ly.tslot[((size_t)cta * M + row) * ly.k_pad + col] = v;
     }
+    __threadfence();                             // the slot before the count
     __syncthreads();
-    cluster_arrive();                            // this CTA's partial T is published; waited for before the rank part
+    if (tid == 0) atomicAdd(ly.tcount, 1);       // this range of T is published; waited for before the first rank part
   }
 
+  // T = sum of the ranges' partial sums (range order), then MXINT8 along the rank: 16 adjacent lanes hold one block.
+  // The ranges belong to CTAs of this launch, all resident; the wait is bounded all the same.
+  auto build_tq = [&]() {
+    if (tid == 0) {
+      int seen = 1;
+      const long long t0 = clock64();
+      for (;;) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ly.tcount) : "memory");
+        if (v >= ly.t_ranges) break;
+        if (clock64() - t0 > kSpinLimitCycles) { seen = 0; break; }
+        __nanosleep(100);
+      }
+      if (!seen) report_error(p.status, LQER_ERR_TIMEOUT, 500, blockIdx.x);
+      *wait_ok = seen;
+    }
+    __syncthreads();
+    const bool ok = *wait_ok != 0;
+    const int total = M * ly.k_pad;
+    for (int base = 0; base < total; base += kThreads) {
+      const int idx = base + tid;
+      const bool valid = idx < total;
+      const int row = valid ? idx / ly.k_pad : 0, col = valid ? idx % ly.k_pad : 0;
+      double tv = 0.0;
+      if (valid && ok) {
+        const double* sp = ly.tslot + (size_t)row * ly.k_pad + col;
+#pragma unroll 4
+        for (int c = 0; c < ly.t_ranges; ++c) tv += __ldcg(sp + (size_t)c * M * ly.k_pad);
+      }
+      double amax = (tv != tv) ? 0.0 : fabs(tv);
+#pragma unroll
+      for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+      const int e = block_exponent(amax, p.exp_min, p.exp_max);
+      const int qv = quant_mantissa(tv, e, p.a_bits);
+      if (valid) {
+        tq8[row * ly.k_pad + col] = (int8_t)qv;
+        if ((col & 15) == 0) tqs[row * (ly.k_pad / 16) + (col >> 4)] = pow2f(e - (p.a_bits - 2));
+      }
+    }
+    __syncthreads();
+    if (tid == 0 && atomicAdd(ly.tcount + 1, 1) == G - 1) {   // every CTA of the layer has read the slots: zero for the next call
+      ly.tcount[0] = 0;
+      ly.tcount[1] = 0;
+    }
+  };
   bool tq_built = false;
   const int slabs_mine = ly.k_slabs > warp ? (ly.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
 #pragma unroll 1
@@ -339,29 +372,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     // ---- B_q against T_q: rank blocks warp, warp + 16, ...
     if (ly.k_pad > 0) {
       if (!tq_built) {
-        // T = sum of the cluster's partials (CTA order), then MXINT8 along the rank: 16 adjacent lanes hold one block
-        cluster_wait();
-        const int cs = (int)cluster_nctarank();
-        const int total = M * ly.k_pad;
-        for (int base = 0; base < total; base += kThreads) {
-          const int idx = base + tid;
-          const bool valid = idx < total;
-          const int row = valid ? idx / ly.k_pad : 0, col = valid ? idx % ly.k_pad : 0;
-          double tv = 0.0;
-          if (valid)
-            for (int c = 0; c < cs; ++c) tv += ld_dsmem_f64(tpart + row * ly.k_pad + col, (uint32_t)c);
-          double amax = (tv != tv) ? 0.0 : fabs(tv);
-#pragma unroll
-          for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
-          const int e = block_exponent(amax, p.exp_min, p.exp_max);
-          const int qv = quant_mantissa(tv, e, p.a_bits);
-          if (valid) {
-            tq8[row * ly.k_pad + col] = (int8_t)qv;
-            if ((col & 15) == 0) tqs[row * (ly.k_pad / 16) + (col >> 4)] = pow2f(e - (p.a_bits - 2));
-          }
-        }
-        __syncthreads();
-        cluster_arrive();                        // done reading the peers' shared memory
+        build_tq();
         tq_built = true;
       }
       const int rbn = ly.k_pad / 16;
@@ -397,10 +408,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     }
     __syncthreads();                             // red is rewritten by the next round
   }
-  if (ly.k_pad > 0) {
-    if (!tq_built) { cluster_wait(); cluster_arrive(); }   // a CTA without columns still serves its partial T
-    cluster_wait();                              // no CTA leaves while its shared memory may still be read
-  }
+  if (ly.k_pad > 0 && !tq_built) build_tq();     // a CTA without columns still takes part in the counts
 }
 
 }  // namespace dcol
@@ -429,28 +437,15 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
                                      cudaStream_t s) {
   using namespace dcol;
   static int sm_count = 0;
-  static int max_clusters = -1;
-  if (max_clusters < 0) {
-    int dev = 0;
+  if (sm_count == 0) {
+    int dev = 0, sms = 0;
     cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaError_t e = cudaFuncSetAttribute(decode_cols_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(decode_cols_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    // all clusters must be resident at once: the CTAs are sized for one wave
-    cudaLaunchConfig_t probe = {};
-    probe.gridDim = dim3(sm_count / kClusterSize * kClusterSize);
-    probe.blockDim = dim3(kThreads);
-    probe.dynamicSmemBytes = 200 * 1024;
-    cudaLaunchAttribute pa[1];
-    pa[0].id = cudaLaunchAttributeClusterDimension;
-    pa[0].val.clusterDim.x = kClusterSize; pa[0].val.clusterDim.y = 1; pa[0].val.clusterDim.z = 1;
-    probe.attrs = pa;
-    probe.numAttrs = 1;
-    int nc = 0;
-    if (cudaOccupancyMaxActiveClusters(&nc, decode_cols_kernel<kMaxM>, &probe) != cudaSuccess || nc < 1) nc = 1;
-    max_clusters = nc;
+    sm_count = sms > 0 ? sms : 1;
   }
   if (n < 1 || n > kMaxGroup) return cudaErrorInvalidValue;
   const int M = calls[0].M;
@@ -460,36 +455,44 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   p.M = M;
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
 
-  // CTAs per layer: a single layer takes what it can use; several share the resident clusters by weight bytes
+  // CTAs per layer (one per SM at most, so that all of a launch are resident together): a single layer takes what
+  // it can use; several share the SMs by weight bytes, and what rounding leaves over goes where the load per CTA is
+  // largest
+  const int max_ctas = sm_count < kDecodeMaxCtas ? sm_count : kDecodeMaxCtas;
   int ctas[kMaxGroup];
-  int cs = kClusterSize;
   if (n == 1) {
-    int G = metas[0].N / 8 < sm_count ? metas[0].N / 8 : sm_count;
-    if (G > kDecodeMaxCtas) G = kDecodeMaxCtas;
-    cs = G >= kClusterSize ? kClusterSize : 1;
-    G = G / cs * cs;
-    if (cs > 1 && G > max_clusters * cs) G = max_clusters * cs;
-    ctas[0] = G;
+    ctas[0] = metas[0].N / 8 < max_ctas ? metas[0].N / 8 : max_ctas;
   } else {
     double total_w = 0.0;
+    for (int g = 0; g < n; ++g) total_w += (double)metas[g].K * metas[g].N;
+    int left = max_ctas;
     for (int g = 0; g < n; ++g) {
-      if (metas[g].N / 8 < kClusterSize) return cudaErrorInvalidValue;
-      total_w += (double)metas[g].K * metas[g].N;
-    }
-    int left = max_clusters;
-    for (int g = 0; g < n; ++g) {                     // at least one cluster each, the rest by weight
-      int c = (int)((double)max_clusters * ((double)metas[g].K * metas[g].N / total_w));
+      int c = (int)((double)max_ctas * ((double)metas[g].K * metas[g].N / total_w));
       if (c < 1) c = 1;
-      const int cap = metas[g].N / 8 / kClusterSize;
-      if (c > cap) c = cap;
+      if (c > metas[g].N / 8) c = metas[g].N / 8;
       ctas[g] = c;
       left -= c;
     }
-    if (left < 0) return cudaErrorInvalidConfiguration;   // more layers than clusters
-    for (int g = 0; left > 0 && g < n; ++g)              // hand out what rounding left over
-      if (ctas[g] < metas[g].N / 8 / kClusterSize) { ++ctas[g]; --left; }
-    for (int g = 0; g < n; ++g) ctas[g] *= kClusterSize;
+    if (left < 0) return cudaErrorInvalidConfiguration;   // more layers than SMs
+    while (left > 0) {
+      int best = -1;
+      double load = 0.0;
+      for (int g = 0; g < n; ++g) {
+        const double l = (double)metas[g].K * metas[g].N / ctas[g];
+        if (ctas[g] < metas[g].N / 8 && l > load) { load = l; best = g; }
+      }
+      if (best < 0) break;
+      ++ctas[best];
+      --left;
+    }
   }
+  size_t head = 0;
+  for (int g = 0; g < n; ++g) {
+    const size_t h = (persist_bytes(metas[g]) + 255) & ~(size_t)255;
+    if (h > head) head = h;
+  }
+  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  size_t slot_off = head;
 
   size_t smem = 0;
   int begin = 0;
@@ -504,8 +507,14 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     ly.K = m.K; ly.N = m.N; ly.K64 = m.K64; ly.k_pad = m.k_pad;
     ly.k_slabs = m.k_slabs; ly.r_blocks = m.r_blocks;
     ly.n_cg = m.N / 8;
+    int ranges = ctas[g] < kTRanges ? ctas[g] : kTRanges;
+    if (ranges > m.K / 16) ranges = m.K / 16;
+    ly.t_ranges = ranges;
+    ly.tslot = reinterpret_cast<double*>(wsb + slot_off);
+    ly.tcount = reinterpret_cast<int*>(wsb + kStatusBytes) + 2 * g;
+    if (i < n) slot_off += decode_cols_slot_bytes(m);
     // stage this CTA's share of A_q in shared memory when it fits beside everything else
-    const size_t a_need = m.k_pad > 0 ? (size_t)((m.K / 16 + cs - 1) / cs) * m.k_pad * 17 + 16 : 0;
+    const size_t a_need = m.k_pad > 0 ? (size_t)((m.K / 16 + ranges - 1) / ranges) * m.k_pad * 17 + 16 : 0;
     ly.a_stage_bytes = (a_need <= (size_t)kAStageMax && cols_smem_bytes(m, M) + a_need <= 200 * 1024) ? (int)a_need : 0;
     ly.cta_begin = begin;
     ly.ctas = ctas[g];
@@ -521,13 +530,11 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
-  cudaLaunchAttribute attr[2];
+  cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the previous kernel drains
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  attr[1].id = cudaLaunchAttributeClusterDimension;
-  attr[1].val.clusterDim.x = cs; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 2;
+  cfg.numAttrs = 1;
   LaunchScope scope(kFamDecode, s);
   return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM>, p);
 }
