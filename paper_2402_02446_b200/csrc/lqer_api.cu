@@ -164,7 +164,7 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
     uint8_t* wsb = static_cast<uint8_t*>(workspace);
     err = tc_prologue ? launch_prologue_tc(X, M, m, packed, xcat, Tm, Te, dst,
                                            reinterpret_cast<double*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M)),
-                                           reinterpret_cast<int*>(wsb + pcount_offset(m)), kPrologueAlone, s)
+                                           reinterpret_cast<int*>(wsb + pcount_offset(m)), kChainAlone, s)
                       : launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
       err = (path == 1)   ? launch_gemm_simt(xcat, M, m, packed, Y, s)
@@ -224,20 +224,19 @@ static int decode_run(const lqer_call_t* calls, int first, int n_calls, int max_
   PackedMeta m0;
   if (lookup(calls[first].packed, m0) != LQER_OK || !decode_cols_fits(m0, calls[first].M)) return 0;
   metas[0] = m0;
-  size_t head = align_up(persist_bytes(m0), 256), slots = decode_cols_slot_bytes(m0);
+  const size_t head = align_up(kPersistMaxBytes, 256);   // one bound for all layers, so that consecutive groups agree on it
+  size_t slots = decode_cols_slot_bytes(m0);
   int n = 1;
   while (first + n < n_calls && n < max_group) {
     PackedMeta m1;
     if (calls[first + n].M != calls[first].M || lookup(calls[first + n].packed, m1) != LQER_OK ||
         !same_formats(m0, m1) || !decode_cols_fits(m1, calls[first].M) || m1.N < 32 || m0.N < 32)
       break;
-    const size_t h = std::max(head, align_up(persist_bytes(m1), 256));
-    if (h + slots + decode_cols_slot_bytes(m1) > workspace_bytes) break;
-    head = h;
+    if (head + 2 * (slots + decode_cols_slot_bytes(m1)) > workspace_bytes) break;   // two sets: see launch_decode_cols_group
     slots += decode_cols_slot_bytes(m1);
     metas[n++] = m1;
   }
-  if (need != nullptr) *need = head + slots;
+  if (need != nullptr) *need = head + 2 * slots;
   return n;
 }
 // n prefill layers with one M: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
@@ -265,7 +264,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
     off += group_slice_bytes(m, M);
     const float* X = calls[g].X;
     int* counters = reinterpret_cast<int*>(wsb + count_base) + (own_counters ? (size_t)g * row_tiles * 2 : 0);
-    const int order = !own_counters ? kPrologueAlone : g == 0 ? kPrologueGroupFirst : kPrologueGroupLater;
+    const int order = !own_counters ? kChainAlone : g == 0 ? kChainFirst : kChainLater;
     cudaError_t err = prologue_tc_fits(m, M, X, false)
                           ? launch_prologue_tc(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
                                                reinterpret_cast<double*>(xcat + xcat_bytes(m, M)), counters, order, s)
@@ -454,6 +453,10 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     if (workspace_bytes < call_bytes(m, c.M, decode)) return LQER_ERR_BUFFER_TOO_SMALL;
   }
   const bool may_group = g_path.load() == 0;   // a forced path runs every call on its own
+  // Decode launches that follow one another are independent too (no buffer in common: two sets of slots and counters
+  // in turn), so a launch need not wait for the one before it, as long as that one had a CTA on every SM.
+  bool chain_open = false;
+  int chain_set = 0;
   for (int i = 0; i < n_calls;) {
     // The calls are independent, so consecutive calls of one shape (the q, k, v projections of a layer, or its gate
     // and up projections) share launches: decode calls one launch of the column-owner kernel (a slot of the workspace per
@@ -477,12 +480,19 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
       if (st != LQER_OK) return st;
       if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
       if (decode_group) {
-        if (launch_decode_cols_group(calls + i, metas, n, workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        const int set = chain_open ? 1 - chain_set : 0;
+        bool fills = false;
+        if (launch_decode_cols_group(calls + i, metas, n, workspace, workspace_bytes, chain_open ? kChainLater : kChainFirst,
+                                     set, &fills, static_cast<cudaStream_t>(stream)) != cudaSuccess)
           return LQER_ERR_CUDA;
-      } else if ((st = run_prefill_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) {
-        return st;
+        chain_open = fills;
+        chain_set = set;
+      } else {
+        chain_open = false;
+        if ((st = run_prefill_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) return st;
       }
     } else {
+      chain_open = false;
       lqer_status_t st = lqer_linear_stream(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace,
                                             workspace_bytes, stream);
       if (st != LQER_OK) return st;

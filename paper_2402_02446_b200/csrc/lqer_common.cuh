@@ -262,9 +262,9 @@ cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const vo
 // The same prologue with the projection on the tcgen05 int8 tensor cores: ranks up to 64, large batches.
 bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch);
 // `partials`: prologue_tc_scratch_bytes(m, M) of scratch; `counters`: zeroed counter pairs of the workspace head,
-// one per row tile.  `order`: kPrologueAlone, or the place in a run of prologues that share no buffer or counter
+// one per row tile.  `order`: kChainAlone, or the place in a run of prologues that share no buffer or counter
 // (each later one overlaps the tail of the one before; the kernel after the run still finds all of them complete).
-enum PrologueOrder { kPrologueAlone = 0, kPrologueGroupFirst = 1, kPrologueGroupLater = 2 };
+enum ChainOrder { kChainAlone = 0, kChainFirst = 1, kChainLater = 2 };
 cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                int order, cudaStream_t s);
@@ -289,9 +289,13 @@ cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);
 // Up to decode_cols_max_group() independent layers with one M (all fitting decode_cols_fits, N >= 32) in one launch.
+// `order`, `set`: consecutive launches of a chain (ChainOrder) alternate between two sets of slots and counters: set 0
+// behind the head of the workspace, set 1 at its end (`workspace_bytes`, read for set 1 only), so a chain needs
+// align_up(kPersistMaxBytes, 256) plus twice the largest group's decode_cols_slot_bytes.  A launch may be chained to
+// the one before only if that one reported `fills_gpu` (one CTA on every SM: at most two launches are alive then).
 int decode_cols_max_group();
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
-                                     cudaStream_t s);
+                                     size_t workspace_bytes, int order, int set, bool* fills_gpu, cudaStream_t s);
 int decode_max_m();
 
 }  // namespace lqer

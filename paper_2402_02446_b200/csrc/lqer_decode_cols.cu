@@ -38,8 +38,6 @@ constexpr int kMaxM = 4;
 constexpr int kCg = 4;            // column groups (of 8 columns) per round: one column per lane
 constexpr int kSets = 4;          // slabs a warp keeps in flight
 constexpr int kTRanges = 16;      // CTAs of a layer that share the work of T = X_q A_q (ranges of K), at most
-constexpr int kMaxSubsets = 8;    // warps that split the K blocks of one rank tile
-constexpr int kAStageMax = 100 * 1024;   // a CTA's share of A_q is staged in shared memory if it fits in this
 
 constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
 constexpr long long kSpinLimitCycles = 4000000000LL;   // about two seconds
@@ -50,7 +48,6 @@ struct Layer {
   const uint8_t* packed;
   size_t off_w, off_b, off_a;   // sections of the packed buffer
   int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
-  int a_stage_bytes;            // shared memory reserved for staging A_q (0: read it from global memory)
   int cta_begin, ctas;          // this layer's CTAs in the launch, in proportion to its weight bytes
   int t_ranges;                 // the first t_ranges of them compute T, a range of K each
   double* tslot;                // [t_ranges][M][k_pad] partial sums of T (workspace scratch)
@@ -58,8 +55,10 @@ struct Layer {
 };
 
 struct Params {
+  int cta_begin[kMaxGroup];     // first CTA of each layer (a copy, side by side: a CTA finds its layer in one cache line)
   Layer L[kMaxGroup];
   int group;                    // layers in this launch
+  int order;                    // ChainOrder: where the wait for the previous kernel sits
   DeviceStatus* status;
   int M;
   int a_bits, lr_bits, exp_min, exp_max;
@@ -87,6 +86,13 @@ __device__ __forceinline__ uint32_t ld_stream_u8(const void* p) {
   asm volatile("ld.global.nc.L1::no_allocate.u8 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
 }
+// T = X_q A_q: a warp takes 32 rank columns (a lane each) of some K blocks; these many warps split the K blocks of
+// one such tile of columns.
+__host__ __device__ inline int t_subsets(int k_pad) {
+  const int tiles = k_pad > 32 ? (k_pad + 31) / 32 : 1;
+  return tiles < kWarps ? kWarps / tiles : 1;
+}
+
 // MT: rows the accumulators are compiled for (1 for the single-token call, kMaxM otherwise); M <= MT.
 template <int MT>
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
@@ -95,7 +101,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   int layer = 0;
 #pragma unroll
   for (int i = 1; i < kMaxGroup; ++i)
-    if (i < p.group && (int)blockIdx.x >= p.L[i].cta_begin) layer = i;
+    if (i < p.group && (int)blockIdx.x >= p.cta_begin[i]) layer = i;
   const Layer& ly = p.L[layer];
   const int M = p.M, KB = ly.K64 / 16;
   uint8_t* xm = smem;                                               // [M][K64] int8 mantissas, permuted within 8
@@ -104,13 +110,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // [kWarps][32 columns][kMaxM]
   double* tsub = reinterpret_cast<double*>(red + kWarps * kCg * 8 * kMaxM);   // [subsets][M][k_pad] per-warp-subset partials of T
   int* wait_ok = reinterpret_cast<int*>(tsub);                       // reused once T's partial sums have left: outcome of the wait
-  float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * kMaxSubsets);   // [M][k_pad / 16]
+  float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * t_subsets(ly.k_pad));   // [M][k_pad / 16]
   int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);        // [M][k_pad]
-  uint8_t* a_stage = reinterpret_cast<uint8_t*>(
-      (reinterpret_cast<uintptr_t>(tq8) + (size_t)kMaxM * (ly.k_pad > 0 ? ly.k_pad : 16) + 15) & ~(uintptr_t)15);   // staged A_q
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;             // fragment coordinates of the T part's MMA
   const int G = ly.ctas, cta = (int)blockIdx.x - ly.cta_begin;
   const float* const X = ly.X;
   float* const Y = ly.Y;
@@ -141,7 +144,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     d.e = ld_stream_u32(wsec + (o.e + jo));
   };
 
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Alone: the next kernel may set up at once, and this one waits for the previous one before it reads X.  In a chain
+  // of launches that share no buffer (independent layers, scratch and counters of their own): the first lets its
+  // successor start only after its own wait, the later ones do not wait before they work but before they exit, so that
+  // a launch fills the SMs as the one before leaves them and the kernel after the chain finds all of it complete.
+  if (p.order != kChainFirst) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // this lane's column of rank block `warp` of B_q: its 16 rank values and the exponent byte
   auto fetch_rank = [&](uint4& wv, uint32_t& eb, int cg0) {
@@ -169,86 +176,97 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const bool t_worker = ly.k_pad > 0 && cta < ly.t_ranges;
   const int kb_lo = t_worker ? cta * KBr / ly.t_ranges : 0;          // this CTA's share of K for T
   const int kb_hi = t_worker ? (cta + 1) * KBr / ly.t_ranges : 0;
-  const bool a_staged = t_worker && (kb_hi - kb_lo) * ly.k_pad * 17 <= ly.a_stage_bytes;
-  if (a_staged) {
-    const int mant = (kb_hi - kb_lo) * ly.k_pad * 16, ex = (kb_hi - kb_lo) * ly.k_pad;
+  if (t_worker) {                                  // this CTA's share of A_q: towards L2 while X is quantised
     const uint8_t* gm = asec + (size_t)kb_lo * ly.k_pad * 16;
     const uint8_t* ge = asec + (size_t)KBr * ly.k_pad * 16 + (size_t)kb_lo * ly.k_pad;
-    for (int o = tid * 16; o < mant; o += kThreads * 16)
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(a_stage + o)), "l"(gm + o) : "memory");
-    for (int o = tid * 16; o < ex; o += kThreads * 16)
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(a_stage + mant + o)), "l"(ge + o) : "memory");
-    asm volatile("cp.async.commit_group;" ::: "memory");
+    const int mant = (kb_hi - kb_lo) * ly.k_pad * 16, ex = (kb_hi - kb_lo) * ly.k_pad;
+    for (int o = tid * 128; o < mant; o += kThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(gm + o));
+    for (int o = tid * 128; o < ex; o += kThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(ge + o));
   }
 
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // X (and the workspace) may be an earlier kernel's output
+  if (p.order != kChainLater) asm volatile("griddepcontrol.wait;" ::: "memory");   // X (and the workspace) may be an earlier kernel's output
+  if (p.order == kChainFirst) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // ---- X -> MXINT8 for the whole contraction: per row the mantissas in the byte order the nibbles
   //      unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales and the offsets 8 * sum(x)
   {
     const int per_row = ly.K64 / 4, total = M * per_row;             // float4 items: (row, quarter-block)
-    for (int base = 0; base < total; base += kThreads) {
-      const int item = base + tid;
-      const bool valid = item < total;
-      const int row = valid ? item / per_row : 0, c4 = valid ? item % per_row : 0;
-      const float4 v = (valid && c4 * 4 < ly.K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * ly.K + c4 * 4))
+    constexpr int U = 4;                                             // loads in flight per thread
+    for (int base = 0; base < total; base += kThreads * U) {
+      float4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int item = base + u * kThreads + tid;
+        const int row = item / per_row, c4 = item % per_row;
+        v[u] = (item < total && c4 * 4 < ly.K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * ly.K + c4 * 4))
                                                : make_float4(0.f, 0.f, 0.f, 0.f);
-      int e;
-      uint32_t m8;
-      uint2 unused;
-      quantize_quad(v, p.a_bits, p.exp_min, p.exp_max, e, m8, unused);
-      const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, m8, 1);
-      const uint32_t perm = (c4 & 1) ? __byte_perm(other, m8, 0x7362) : __byte_perm(m8, other, 0x5140);
-      int sum = __dp4a((int)m8, 0x01010101, 0);
-      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-      if (valid) {
-        *reinterpret_cast<uint32_t*>(xm + (size_t)row * ly.K64 + c4 * 4) = perm;
-        if ((c4 & 3) == 0) {
-          xsc[row * KB + (c4 >> 2)] = pow2f(e - (p.a_bits - 2));
-          xof[row * KB + (c4 >> 2)] = kIntMagicBits - 8 * sum;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int item = base + u * kThreads + tid;
+        if (base + u * kThreads + (tid & ~31) >= total) continue;      // a whole warp past the end (the shuffles need whole warps)
+        const bool valid = item < total;
+        const int row = valid ? item / per_row : 0, c4 = valid ? item % per_row : 0;
+        int e;
+        uint32_t m8;
+        uint2 unused;
+        quantize_quad(v[u], p.a_bits, p.exp_min, p.exp_max, e, m8, unused);
+        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, m8, 1);
+        const uint32_t perm = (c4 & 1) ? __byte_perm(other, m8, 0x7362) : __byte_perm(m8, other, 0x5140);
+        int sum = __dp4a((int)m8, 0x01010101, 0);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+        if (valid) {
+          *reinterpret_cast<uint32_t*>(xm + (size_t)row * ly.K64 + c4 * 4) = perm;
+          if ((c4 & 3) == 0) {
+            xsc[row * KB + (c4 >> 2)] = pow2f(e - (p.a_bits - 2));
+            xof[row * KB + (c4 >> 2)] = kIntMagicBits - 8 * sum;
+          }
         }
       }
     }
   }
-  if (a_staged) asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
-  // ---- this CTA's share of T = X_q A_q: exact int8 MMA per (16-block of K, 8 rank columns) on the
-  //      mantissas in shared memory, scaled in fp64.  The products are exact; their fp64 sums are exact
-  //      too unless the block exponents of one row spread over more than about 30 binades, and the
-  //      order of the additions is fixed in any case.
+  // ---- this CTA's share of T = X_q A_q: per (16-block of K, rank column) an exact integer dot product (dp4a) of
+  //      the mantissas, scaled in fp64.  The fp64 sums are exact too unless the block exponents of one row spread
+  //      over more than about 30 binades, and the order of the additions is fixed in any case.
   if (t_worker) {
-    const int NT = ly.k_pad / 8;
-    // A_q of blocks kb_lo..kb_hi: staged copy, or global memory
-    const uint8_t* a_mant = a_staged ? a_stage - (size_t)kb_lo * ly.k_pad * 16 : asec;
-    const uint8_t* a_exp = a_staged ? a_stage + (size_t)(kb_hi - kb_lo) * ly.k_pad * 16 - (size_t)kb_lo * ly.k_pad
-                                    : asec + (size_t)KBr * ly.k_pad * 16;
+    const int NT = (ly.k_pad + 31) / 32;                            // tiles of 32 rank columns, a lane each
+    const uint8_t* a_exp = asec + (size_t)KBr * ly.k_pad * 16;
     const int bias = -127 - (p.lr_bits - 2);                        // exponent bytes carry +127
-    const int tiles_w = NT < kWarps ? NT : kWarps;                  // warps side by side on different rank tiles
-    int subsets = kWarps / tiles_w;                                 // warps that split the K blocks of one tile
-    if (subsets > kMaxSubsets) subsets = kMaxSubsets;
+    const int tiles_w = NT < kWarps ? NT : kWarps;                  // warps side by side on different tiles
+    const int subsets = t_subsets(ly.k_pad);                        // warps that split the K blocks of one tile
     const int sb = warp / tiles_w;
     if (sb < subsets) {
       for (int nt = warp % tiles_w; nt < NT; nt += tiles_w) {
-        double t0 = 0.0, t1 = 0.0;
+        const int j = nt * 32 + lane;
+        const bool live = j < ly.k_pad;
+        const int jc = live ? j : 0;
+        double tacc[MT];
+#pragma unroll
+        for (int r = 0; r < MT; ++r) tacc[r] = 0.0;
 #pragma unroll 4
         for (int kb = kb_lo + sb; kb < kb_hi; kb += subsets) {
-          // the X mantissas are stored as {0,4,1,5}, {2,6,3,7} within each 8: bring A_q into the same order
-          const uint4 q = *reinterpret_cast<const uint4*>(a_mant + ((size_t)kb * ly.k_pad + nt * 8 + g) * 16);
-          const uint32_t lo = (t & 2) ? q.z : q.x, hi = (t & 2) ? q.w : q.y;
-          const uint32_t b0 = (t & 1) ? __byte_perm(lo, hi, 0x7362) : __byte_perm(lo, hi, 0x5140);
-          const uint32_t ea2 = *reinterpret_cast<const uint16_t*>(a_exp + (size_t)kb * ly.k_pad + nt * 8 + t * 2);
-          const uint32_t a0 = g < M ? *reinterpret_cast<const uint32_t*>(xm + (size_t)g * ly.K64 + kb * 16 + t * 4) : 0u;
-          const double sx = g < M ? (double)xsc[g * KB + kb] : 0.0;
-          int c[4];
-          mma_s8(c, a0, 0u, b0);
-          t0 = fma((double)c[0], sx * pow2d((int)(ea2 & 0xFFu) + bias), t0);
-          t1 = fma((double)c[1], sx * pow2d((int)(ea2 >> 8) + bias), t1);
+          const uint4 a = __ldg(reinterpret_cast<const uint4*>(asec + ((size_t)kb * ly.k_pad + jc) * 16));
+          const double sa = pow2d((int)__ldg(a_exp + (size_t)kb * ly.k_pad + jc) + bias);
+#pragma unroll
+          for (int r = 0; r < MT; ++r) {
+            if (r < M) {
+              // the X mantissas are stored as {0,4,1,5}, {2,6,3,7} within each 8: back to the order of A_q
+              const uint4 x = *reinterpret_cast<const uint4*>(xm + (size_t)r * ly.K64 + kb * 16);
+              int sm = __dp4a((int)__byte_perm(x.x, x.y, 0x6420), (int)a.x, 0);
+              sm = __dp4a((int)__byte_perm(x.x, x.y, 0x7531), (int)a.y, sm);
+              sm = __dp4a((int)__byte_perm(x.z, x.w, 0x6420), (int)a.z, sm);
+              sm = __dp4a((int)__byte_perm(x.z, x.w, 0x7531), (int)a.w, sm);
+              tacc[r] = fma((double)sm, (double)xsc[r * KB + kb] * sa, tacc[r]);
+            }
+          }
         }
-        if (g < M) {
-          tsub[((size_t)sb * kMaxM + g) * ly.k_pad + nt * 8 + t * 2] = t0;
-          tsub[((size_t)sb * kMaxM + g) * ly.k_pad + nt * 8 + t * 2 + 1] = t1;
+        if (live) {
+#pragma unroll
+          for (int r = 0; r < MT; ++r)
+            if (r < M) tsub[((size_t)sb * kMaxM + r) * ly.k_pad + j] = tacc[r];
         }
       }
     }
@@ -259,9 +277,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       for (int q = 0; q < subsets; ++q) v += tsub[((size_t)q * kMaxM + row) * ly.k_pad + col];
       ly.tslot[((size_t)cta * M + row) * ly.k_pad + col] = v;
     }
-    __threadfence();                             // the slot before the count
     __syncthreads();
-    if (tid == 0) atomicAdd(ly.tcount, 1);       // this range of T is published; waited for before the first rank part
+    if (tid == 0) {                              // this range of T is published; waited for before the first rank part
+      __threadfence();                           // the slot (ordered before by the barrier) before the count
+      atomicAdd(ly.tcount, 1);
+    }
   }
 
   // T = sum of the ranges' partial sums (range order), then MXINT8 along the rank: 16 adjacent lanes hold one block.
@@ -409,6 +429,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     __syncthreads();                             // red is rewritten by the next round
   }
   if (ly.k_pad > 0 && !tq_built) build_tq();     // a CTA without columns still takes part in the counts
+  if (p.order == kChainLater) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace dcol
@@ -416,7 +437,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 static size_t cols_smem_bytes(const PackedMeta& m, int M) {
   using namespace dcol;
   return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + kWarps * kCg * 8 * kMaxM * 4 +
-         (size_t)kMaxM * m.k_pad * 8 * (1 + kMaxSubsets) + kMaxM * 16 * 4 + (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
+         (size_t)kMaxM * m.k_pad * 8 * t_subsets(m.k_pad) + kMaxM * 16 * 4 + (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
 }
 // The column-owner kernel serves M <= 4 as long as the quantised X of the whole contraction fits in shared memory.
 bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
@@ -424,7 +445,7 @@ bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && c
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y, void* workspace,
                                cudaStream_t s) {
   const lqer_call_t one = {X, M, packed, Y};
-  return launch_decode_cols_group(&one, &m, 1, workspace, s);
+  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, s);
 }
 
 int decode_cols_max_group() { return dcol::kMaxGroup; }
@@ -434,7 +455,7 @@ int decode_cols_max_group() { return dcol::kMaxGroup; }
 // reduction) overlap instead of following one another.  Every layer must fit decode_cols_fits and, for n > 1, have
 // at least one cluster's worth of column groups.
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
-                                     cudaStream_t s) {
+                                     size_t workspace_bytes, int order, int set, bool* fills_gpu, cudaStream_t s) {
   using namespace dcol;
   static int sm_count = 0;
   if (sm_count == 0) {
@@ -451,6 +472,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   const int M = calls[0].M;
   Params p;
   p.group = n;
+  p.order = order;
   p.status = reinterpret_cast<DeviceStatus*>(workspace);
   p.M = M;
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
@@ -493,6 +515,12 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   }
   uint8_t* wsb = static_cast<uint8_t*>(workspace);
   size_t slot_off = head;
+  if (set != 0) {                                       // the second set of slots lies at the end of the workspace
+    size_t slots = 0;
+    for (int g = 0; g < n; ++g) slots += decode_cols_slot_bytes(metas[g]);
+    if (workspace_bytes < head + 2 * slots) return cudaErrorInvalidValue;
+    slot_off = (workspace_bytes - slots) & ~(size_t)255;
+  }
 
   size_t smem = 0;
   int begin = 0;
@@ -511,16 +539,14 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     if (ranges > m.K / 16) ranges = m.K / 16;
     ly.t_ranges = ranges;
     ly.tslot = reinterpret_cast<double*>(wsb + slot_off);
-    ly.tcount = reinterpret_cast<int*>(wsb + kStatusBytes) + 2 * g;
+    ly.tcount = reinterpret_cast<int*>(wsb + kStatusBytes) + 2 * (g + (set != 0 ? kMaxGroup : 0));
     if (i < n) slot_off += decode_cols_slot_bytes(m);
-    // stage this CTA's share of A_q in shared memory when it fits beside everything else
-    const size_t a_need = m.k_pad > 0 ? (size_t)((m.K / 16 + ranges - 1) / ranges) * m.k_pad * 17 + 16 : 0;
-    ly.a_stage_bytes = (a_need <= (size_t)kAStageMax && cols_smem_bytes(m, M) + a_need <= 200 * 1024) ? (int)a_need : 0;
     ly.cta_begin = begin;
+    p.cta_begin[i] = begin;
     ly.ctas = ctas[g];
     if (i < n) {
       begin += ctas[g];
-      const size_t need = cols_smem_bytes(m, M) + ly.a_stage_bytes;
+      const size_t need = cols_smem_bytes(m, M);
       if (need > smem) smem = need;
     }
   }
@@ -535,6 +561,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (fills_gpu != nullptr) *fills_gpu = begin == sm_count;
   LaunchScope scope(kFamDecode, s);
   return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM>, p);
 }

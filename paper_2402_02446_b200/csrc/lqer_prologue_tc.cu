@@ -78,7 +78,7 @@ struct Params {
   int panels;               // ceil(K64 / 128)
   int splits;               // CTAs per row tile
   int a_bits, lr_bits, exp_min, exp_max;
-  int order;                // PrologueOrder: where the wait for the previous kernel sits
+  int order;                // ChainOrder: where the wait for the previous kernel sits
   size_t ldx;               // columns of Xcat
 };
 
@@ -184,12 +184,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   // only once the earlier kernels are done, since it does not wait before it works.  Later in a group: nothing here
   // is shared with the prologue before, so the work starts at once and only the exit waits for it (a kernel after
   // the group then finds all of them complete).
-  if (p.order == kPrologueGroupFirst) {
+  if (p.order == kChainFirst) {
     pdl_wait();
     pdl_launch_dependents();
   } else {
     pdl_launch_dependents();
-    if (p.order == kPrologueAlone) pdl_wait();
+    if (p.order == kChainAlone) pdl_wait();
   }
 
   if (warp < SW) {
@@ -442,7 +442,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     *arrive_cnt = 0;
     *depart_cnt = 0;
   }
-  if (p.order == kPrologueGroupLater) pdl_wait();
+  if (p.order == kChainLater) pdl_wait();
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
