@@ -239,6 +239,27 @@ static int decode_run(const lqer_call_t* calls, int first, int n_calls, int max_
   if (need != nullptr) *need = head + 2 * slots;
   return n;
 }
+// The stretch of calls from calls[first] on that run as shared decode launches (decode_run after decode_run), and the
+// bytes that their quantised activations and T_q take when computed ahead; offsets[i - first] is call i's place
+// behind `base`.
+static int decode_stretch(const lqer_call_t* calls, int first, int n_calls, size_t workspace_bytes,
+                          std::vector<PackedMeta>* metas_out, std::vector<size_t>* offsets, size_t* bytes) {
+  int j = first;
+  size_t total = 0;
+  while (j < n_calls) {
+    PackedMeta metas[16];
+    const int n = decode_run(calls, j, n_calls, decode_cols_max_group(), workspace_bytes, metas, nullptr);
+    if (n < 2) break;
+    for (int g = 0; g < n; ++g) {
+      if (metas_out != nullptr) metas_out->push_back(metas[g]);
+      if (offsets != nullptr) offsets->push_back(total);
+      total += decode_pre_bytes(metas[g], calls[j + g].M);
+    }
+    j += n;
+  }
+  if (bytes != nullptr) *bytes = total;
+  return j - first;
+}
 // n prefill layers with one M: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
 // the tiles of all of them.
 static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace,
@@ -457,6 +478,12 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
   // in turn), so a launch need not wait for the one before it, as long as that one had a CTA on every SM.
   bool chain_open = false;
   int chain_set = 0;
+  // The quantised activations and T_q of a stretch of several decode launches are computed ahead, one CTA per call, if
+  // the workspace has room for them behind its head: the decode launches then stream weights from their first
+  // instruction.
+  const size_t pre_base = align_up(kPersistMaxBytes, 256);
+  int pre_first = 0, pre_end = 0;               // calls [pre_first, pre_end): the stretch looked at last
+  std::vector<size_t> pre_off;                  // its offsets behind pre_base; empty: nothing computed ahead
   for (int i = 0; i < n_calls;) {
     // The calls are independent, so consecutive calls of one shape (the q, k, v projections of a layer, or its gate
     // and up projections) share launches: decode calls one launch of the column-owner kernel (a slot of the workspace per
@@ -480,10 +507,35 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
       if (st != LQER_OK) return st;
       if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
       if (decode_group) {
+        cudaStream_t cs = static_cast<cudaStream_t>(stream);
+        if (i >= pre_end) {
+          std::vector<PackedMeta> pm;
+          size_t bytes = 0;
+          pre_off.clear();
+          pre_first = i;
+          pre_end = i + decode_stretch(calls, i, n_calls, workspace_bytes, &pm, &pre_off, &bytes);
+          if (pre_base + bytes > workspace_bytes || pre_end - i <= decode_cols_max_group()) {   // no room, or a single launch: it does the work itself
+            pre_off.clear();
+          } else {
+            std::vector<uint8_t*> outs(pm.size());
+            for (size_t q = 0; q < pm.size(); ++q) outs[q] = static_cast<uint8_t*>(workspace) + pre_base + pre_off[q];
+            const int step = decode_pre_max_calls();
+            for (int q = 0; q < (int)pm.size(); q += step) {
+              const int cnt = std::min(step, (int)pm.size() - q);
+              if (launch_decode_pre(calls + i + q, pm.data() + q, outs.data() + q, cnt, q == 0 ? kChainFirst : kChainLater,
+                                    cs) != cudaSuccess)
+                return LQER_ERR_CUDA;
+            }
+          }
+        }
+        const uint8_t* pres[16];
+        const bool ahead = !pre_off.empty();
+        for (int g = 0; g < n; ++g)
+          pres[g] = ahead ? static_cast<const uint8_t*>(workspace) + pre_base + pre_off[i + g - pre_first] : nullptr;
         const int set = chain_open ? 1 - chain_set : 0;
         bool fills = false;
         if (launch_decode_cols_group(calls + i, metas, n, workspace, workspace_bytes, chain_open ? kChainLater : kChainFirst,
-                                     set, &fills, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+                                     set, &fills, ahead ? pres : nullptr, cs) != cudaSuccess)
           return LQER_ERR_CUDA;
         chain_open = fills;
         chain_set = set;
@@ -505,8 +557,9 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
 lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes) {
   if (calls == nullptr || bytes == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
+  int stretch_end = 0;
   size_t need = kStatusBytes;
-  for (int i = 0; i < n_calls;) {
+  for (int i = 0; i < n_calls; ++i) {           // every call on its own
     const lqer_call_t& c = calls[i];
     if (c.packed == nullptr) return LQER_ERR_NULL;
     if (c.M <= 0 || c.M > (1 << 24)) return LQER_ERR_SHAPE;
@@ -514,13 +567,22 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
     lqer_status_t st = lookup(c.packed, m);
     if (st != LQER_OK) return st;
     need = std::max(need, workspace_total(m, c.M));
+  }
+  for (int i = 0; i < n_calls;) {               // the launches that calls may share
+    const lqer_call_t& c = calls[i];
+    PackedMeta m;
+    lookup(c.packed, m);
     int n = 1;
     if (decode_cols_fits(m, c.M)) {
       PackedMeta metas[16];
-      size_t group_need = 0;
+      size_t group_need = 0, ahead = 0;
       n = decode_run(calls, i, n_calls, decode_cols_max_group(), ~(size_t)0, metas, &group_need);
       if (n < 1) n = 1;
       need = std::max(need, group_need);
+      if (n > 1 && i >= stretch_end) {          // room to compute a whole stretch's activations ahead
+        stretch_end = i + decode_stretch(calls, i, n_calls, ~(size_t)0, nullptr, nullptr, &ahead);
+        need = std::max(need, align_up(kPersistMaxBytes, 256) + ahead);
+      }
     } else if (c.M > kGemmSplitMaxM) {
       PackedMeta metas[8];
       size_t group_need = 0;

@@ -295,7 +295,18 @@ bool decode_cols_fits(const PackedMeta& m, int M);
 // the one before only if that one reported `fills_gpu` (one CTA on every SM: at most two launches are alive then).
 int decode_cols_max_group();
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
-                                     size_t workspace_bytes, int order, int set, bool* fills_gpu, cudaStream_t s);
+                                     size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
+                                     cudaStream_t s);
+// The quantised activations and T_q of up to decode_pre_max_calls() independent decode calls, computed ahead (one CTA
+// per call) into outs[i] (decode_pre_bytes each, 256-byte aligned); launch_decode_cols_group takes them as `pres` and
+// then has no X to quantise, no T to compute and nothing to exchange.  `order` as above.
+inline size_t decode_pre_bytes(const PackedMeta& m, int M) {
+  const size_t b = (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + 4 * 16 * 4 + (size_t)4 * (m.k_pad > 0 ? m.k_pad : 16);
+  return (b + 255) & ~(size_t)255;
+}
+int decode_pre_max_calls();
+cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas, uint8_t* const* outs, int n, int order,
+                              cudaStream_t s);
 int decode_max_m();
 
 }  // namespace lqer

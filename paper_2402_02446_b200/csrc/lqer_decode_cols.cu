@@ -50,6 +50,7 @@ struct Layer {
   int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
   int cta_begin, ctas;          // this layer's CTAs in the launch, in proportion to its weight bytes
   int t_ranges;                 // the first t_ranges of them compute T, a range of K each
+  const uint8_t* pre;           // X_q and T_q computed ahead (decode_pre_kernel), or null: this launch computes them
   double* tslot;                // [t_ranges][M][k_pad] partial sums of T (workspace scratch)
   int* tcount;                  // arrivals, departures: zero between calls
 };
@@ -93,6 +94,173 @@ __host__ __device__ inline int t_subsets(int k_pad) {
   return tiles < kWarps ? kWarps / tiles : 1;
 }
 
+struct Formats { int a_bits, lr_bits, exp_min, exp_max; };
+
+// X -> MXINT8 for the whole contraction, by all threads of the CTA: per row the mantissas in the byte order the nibbles
+// unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales 2^(e_x - 6) and the dp4a seeds (bits of
+// 1.5 * 2^23, minus 8 * sum(x) of the block).
+__device__ __forceinline__ void quantize_x_rows(const float* X, int M, int K, int K64, const Formats& f, uint8_t* xm,
+                                                float* xsc, int* xof) {
+  const int tid = threadIdx.x, KB = K64 / 16;
+  const int per_row = K64 / 4, total = M * per_row;             // float4 items: (row, quarter-block)
+  constexpr int U = 4;                                             // loads in flight per thread
+  for (int base = 0; base < total; base += kThreads * U) {
+    float4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int item = base + u * kThreads + tid;
+      const int row = item / per_row, c4 = item % per_row;
+      v[u] = (item < total && c4 * 4 < K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * K + c4 * 4))
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int item = base + u * kThreads + tid;
+      if (base + u * kThreads + (tid & ~31) >= total) continue;      // a whole warp past the end (the shuffles need whole warps)
+      const bool valid = item < total;
+      const int row = valid ? item / per_row : 0, c4 = valid ? item % per_row : 0;
+      int e;
+      uint32_t m8;
+      uint2 unused;
+      quantize_quad(v[u], f.a_bits, f.exp_min, f.exp_max, e, m8, unused);
+      const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, m8, 1);
+      const uint32_t perm = (c4 & 1) ? __byte_perm(other, m8, 0x7362) : __byte_perm(m8, other, 0x5140);
+      int sum = __dp4a((int)m8, 0x01010101, 0);
+      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+      if (valid) {
+        *reinterpret_cast<uint32_t*>(xm + (size_t)row * K64 + c4 * 4) = perm;
+        if ((c4 & 3) == 0) {
+          xsc[row * KB + (c4 >> 2)] = pow2f(e - (f.a_bits - 2));
+          xof[row * KB + (c4 >> 2)] = kIntMagicBits - 8 * sum;
+        }
+      }
+    }
+  }
+}
+
+// Partial sums of T = X_q A_q over the K blocks [kb_lo, kb_hi), by all warps of the CTA: per (16-block of K, rank column)
+// an exact integer dot product (dp4a) of the mantissas, scaled in fp64.  The fp64 sums are exact too unless the block
+// exponents of one row spread over more than about 30 binades, and the order of the additions is fixed in any case.
+// Leaves tsub[t_subsets(k_pad)][kMaxM][k_pad]; the caller adds the subsets in order after a barrier.
+template <int MT>
+__device__ __forceinline__ void t_partial(const uint8_t* asec, int K, int K64, int k_pad, int kb_lo, int kb_hi, int M,
+                                          const Formats& f, const uint8_t* xm, const float* xsc, double* tsub) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KBr = K / 16, KB = K64 / 16;
+  const int NT = (k_pad + 31) / 32;                            // tiles of 32 rank columns, a lane each
+  const uint8_t* a_exp = asec + (size_t)KBr * k_pad * 16;
+  const int bias = -127 - (f.lr_bits - 2);                        // exponent bytes carry +127
+  const int tiles_w = NT < kWarps ? NT : kWarps;                  // warps side by side on different tiles
+  const int subsets = t_subsets(k_pad);                        // warps that split the K blocks of one tile
+  const int sb = warp / tiles_w;
+  if (sb < subsets) {
+    for (int nt = warp % tiles_w; nt < NT; nt += tiles_w) {
+      const int j = nt * 32 + lane;
+      const bool live = j < k_pad;
+      const int jc = live ? j : 0;
+      double tacc[MT];
+#pragma unroll
+      for (int r = 0; r < MT; ++r) tacc[r] = 0.0;
+#pragma unroll 4
+      for (int kb = kb_lo + sb; kb < kb_hi; kb += subsets) {
+        const uint4 a = __ldg(reinterpret_cast<const uint4*>(asec + ((size_t)kb * k_pad + jc) * 16));
+        const double sa = pow2d((int)__ldg(a_exp + (size_t)kb * k_pad + jc) + bias);
+#pragma unroll
+        for (int r = 0; r < MT; ++r) {
+          if (r < M) {
+            // the X mantissas are stored as {0,4,1,5}, {2,6,3,7} within each 8: back to the order of A_q
+            const uint4 x = *reinterpret_cast<const uint4*>(xm + (size_t)r * K64 + kb * 16);
+            int sm = __dp4a((int)__byte_perm(x.x, x.y, 0x6420), (int)a.x, 0);
+            sm = __dp4a((int)__byte_perm(x.x, x.y, 0x7531), (int)a.y, sm);
+            sm = __dp4a((int)__byte_perm(x.z, x.w, 0x6420), (int)a.z, sm);
+            sm = __dp4a((int)__byte_perm(x.z, x.w, 0x7531), (int)a.w, sm);
+            tacc[r] = fma((double)sm, (double)xsc[r * KB + kb] * sa, tacc[r]);
+          }
+        }
+      }
+      if (live) {
+#pragma unroll
+        for (int r = 0; r < MT; ++r)
+          if (r < M) tsub[((size_t)sb * kMaxM + r) * k_pad + j] = tacc[r];
+      }
+    }
+  }
+}
+
+// One value of T -> MXINT8 along the rank (16 adjacent lanes hold one block; every lane of the warp calls this).
+__device__ __forceinline__ void store_tq(double tv, bool valid, int row, int col, int k_pad, const Formats& f,
+                                         int8_t* tq8, float* tqs) {
+  double amax = (tv != tv) ? 0.0 : fabs(tv);
+#pragma unroll
+  for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+  const int e = block_exponent(amax, f.exp_min, f.exp_max);
+  const int qv = quant_mantissa(tv, e, f.a_bits);
+  if (valid) {
+    tq8[row * k_pad + col] = (int8_t)qv;
+    if ((col & 15) == 0) tqs[row * (k_pad / 16) + (col >> 4)] = pow2f(e - (f.a_bits - 2));
+  }
+}
+
+// What the decode kernel needs of a layer's activations, computed ahead for many layers at once (independent calls
+// of one batch): the quantised X and T_q, in the layout the decode kernel keeps them in shared memory:
+//   [M][K64] mantissas, [M][K64/16] scales, [M][K64/16] dp4a seeds, [kMaxM][16] scales of T_q, [kMaxM][k_pad] T_q.
+constexpr int kPreMaxCalls = 64;
+struct PreCall {
+  const float* X;
+  const uint8_t* asec;          // A_q section of the packed buffer
+  uint8_t* out;
+  int M, K, K64, k_pad;
+  Formats f;
+};
+struct PreParams {
+  PreCall c[kPreMaxCalls];
+  int order;                    // ChainOrder, as for the decode kernel
+};
+__host__ __device__ inline size_t pre_x_bytes(int M, int K64) { return (size_t)M * K64 + (size_t)M * (K64 / 16) * 8; }
+__host__ __device__ inline size_t pre_t_bytes(int k_pad) { return (size_t)kMaxM * 16 * 4 + (size_t)kMaxM * (k_pad > 0 ? k_pad : 16); }
+
+template <int MT>
+__global__ void __launch_bounds__(kThreads, 1) decode_pre_kernel(const __grid_constant__ PreParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+  const PreCall& c = p.c[blockIdx.x];
+  const int M = c.M, KB = c.K64 / 16, tid = threadIdx.x;
+  uint8_t* xm = smem;
+  float* xsc = reinterpret_cast<float*>(xm + (size_t)M * c.K64);
+  int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);
+  float* tqs = reinterpret_cast<float*>(xof + (size_t)M * KB);
+  int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);
+  const size_t out_bytes = pre_x_bytes(M, c.K64) + pre_t_bytes(c.k_pad);
+  double* tsub = reinterpret_cast<double*>(smem + ((out_bytes + 15) & ~(size_t)15));
+
+  if (p.order != kChainFirst) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (p.order != kChainLater) asm volatile("griddepcontrol.wait;" ::: "memory");   // X may be an earlier kernel's output
+  if (p.order == kChainFirst) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  quantize_x_rows(c.X, M, c.K, c.K64, c.f, xm, xsc, xof);
+  for (int i = tid; i < (int)pre_t_bytes(c.k_pad) / 4; i += kThreads) reinterpret_cast<uint32_t*>(tqs)[i] = 0u;
+  __syncthreads();
+  if (c.k_pad > 0) {
+    t_partial<MT>(c.asec, c.K, c.K64, c.k_pad, 0, c.K / 16, M, c.f, xm, xsc, tsub);
+    __syncthreads();
+    const int subsets = t_subsets(c.k_pad), total = M * c.k_pad;
+    for (int base = 0; base < total; base += kThreads) {
+      const int idx = base + tid;
+      const bool valid = idx < total;
+      const int row = valid ? idx / c.k_pad : 0, col = valid ? idx % c.k_pad : 0;
+      double tv = 0.0;
+      if (valid)
+        for (int q = 0; q < subsets; ++q) tv += tsub[((size_t)q * kMaxM + row) * c.k_pad + col];
+      store_tq(tv, valid, row, col, c.k_pad, c.f, tq8, tqs);
+    }
+    __syncthreads();
+  }
+  for (size_t o = (size_t)tid * 16; o < out_bytes; o += (size_t)kThreads * 16)
+    *reinterpret_cast<uint4*>(c.out + o) = *reinterpret_cast<const uint4*>(smem + o);
+  if (p.order == kChainLater) asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // MT: rows the accumulators are compiled for (1 for the single-token call, kMaxM otherwise); M <= MT.
 template <int MT>
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
@@ -107,8 +275,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   uint8_t* xm = smem;                                               // [M][K64] int8 mantissas, permuted within 8
   float* xsc = reinterpret_cast<float*>(xm + (size_t)M * ly.K64);    // [M][KB] 2^(e_x - 6)
   int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);          // [M][KB] bits of 1.5 * 2^23, minus 8 * sum(x) of the block
-  float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // [kWarps][32 columns][kMaxM]
-  double* tsub = reinterpret_cast<double*>(red + kWarps * kCg * 8 * kMaxM);   // [subsets][M][k_pad] per-warp-subset partials of T
+  float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // two of [kWarps][32 columns][kMaxM], used in turn
+  double* tsub = reinterpret_cast<double*>(red + 2 * kWarps * kCg * 8 * kMaxM);   // [subsets][M][k_pad] per-warp-subset partials of T
   int* wait_ok = reinterpret_cast<int*>(tsub);                       // reused once T's partial sums have left: outcome of the wait
   float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * t_subsets(ly.k_pad));   // [M][k_pad / 16]
   int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);        // [M][k_pad]
@@ -173,7 +341,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   for (int s = 0; s < kSets; ++s) fetch(regs[s], o_cur, warp + kWarps * s);
   fetch_rank(rank_w, rank_e, cg_lo);
   const int KBr = ly.K / 16;
-  const bool t_worker = ly.k_pad > 0 && cta < ly.t_ranges;
+  const bool pre = ly.pre != nullptr;
+  const bool t_worker = !pre && ly.k_pad > 0 && cta < ly.t_ranges;
   const int kb_lo = t_worker ? cta * KBr / ly.t_ranges : 0;          // this CTA's share of K for T
   const int kb_hi = t_worker ? (cta + 1) * KBr / ly.t_ranges : 0;
   if (t_worker) {                                  // this CTA's share of A_q: towards L2 while X is quantised
@@ -189,87 +358,24 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 
   // ---- X -> MXINT8 for the whole contraction: per row the mantissas in the byte order the nibbles
   //      unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales and the offsets 8 * sum(x)
-  {
-    const int per_row = ly.K64 / 4, total = M * per_row;             // float4 items: (row, quarter-block)
-    constexpr int U = 4;                                             // loads in flight per thread
-    for (int base = 0; base < total; base += kThreads * U) {
-      float4 v[U];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int item = base + u * kThreads + tid;
-        const int row = item / per_row, c4 = item % per_row;
-        v[u] = (item < total && c4 * 4 < ly.K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * ly.K + c4 * 4))
-                                               : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int item = base + u * kThreads + tid;
-        if (base + u * kThreads + (tid & ~31) >= total) continue;      // a whole warp past the end (the shuffles need whole warps)
-        const bool valid = item < total;
-        const int row = valid ? item / per_row : 0, c4 = valid ? item % per_row : 0;
-        int e;
-        uint32_t m8;
-        uint2 unused;
-        quantize_quad(v[u], p.a_bits, p.exp_min, p.exp_max, e, m8, unused);
-        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, m8, 1);
-        const uint32_t perm = (c4 & 1) ? __byte_perm(other, m8, 0x7362) : __byte_perm(m8, other, 0x5140);
-        int sum = __dp4a((int)m8, 0x01010101, 0);
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-        if (valid) {
-          *reinterpret_cast<uint32_t*>(xm + (size_t)row * ly.K64 + c4 * 4) = perm;
-          if ((c4 & 3) == 0) {
-            xsc[row * KB + (c4 >> 2)] = pow2f(e - (p.a_bits - 2));
-            xof[row * KB + (c4 >> 2)] = kIntMagicBits - 8 * sum;
-          }
-        }
-      }
-    }
+  const Formats fmt = {p.a_bits, p.lr_bits, p.exp_min, p.exp_max};
+  if (pre) {                                       // quantised X and T_q are there already: straight into shared memory
+    const int xb = (int)pre_x_bytes(M, ly.K64), tb = (int)pre_t_bytes(ly.k_pad);
+    for (int o = tid * 16; o < xb; o += kThreads * 16)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(xm + o)), "l"(ly.pre + o) : "memory");
+    for (int o = tid * 16; o < tb; o += kThreads * 16)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(reinterpret_cast<uint8_t*>(tqs) + o)), "l"(ly.pre + xb + o) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else {
+    quantize_x_rows(X, M, ly.K, ly.K64, fmt, xm, xsc, xof);
   }
   __syncthreads();
 
-  // ---- this CTA's share of T = X_q A_q: per (16-block of K, rank column) an exact integer dot product (dp4a) of
-  //      the mantissas, scaled in fp64.  The fp64 sums are exact too unless the block exponents of one row spread
-  //      over more than about 30 binades, and the order of the additions is fixed in any case.
+  // ---- this CTA's share of T = X_q A_q
   if (t_worker) {
-    const int NT = (ly.k_pad + 31) / 32;                            // tiles of 32 rank columns, a lane each
-    const uint8_t* a_exp = asec + (size_t)KBr * ly.k_pad * 16;
-    const int bias = -127 - (p.lr_bits - 2);                        // exponent bytes carry +127
-    const int tiles_w = NT < kWarps ? NT : kWarps;                  // warps side by side on different tiles
-    const int subsets = t_subsets(ly.k_pad);                        // warps that split the K blocks of one tile
-    const int sb = warp / tiles_w;
-    if (sb < subsets) {
-      for (int nt = warp % tiles_w; nt < NT; nt += tiles_w) {
-        const int j = nt * 32 + lane;
-        const bool live = j < ly.k_pad;
-        const int jc = live ? j : 0;
-        double tacc[MT];
-#pragma unroll
-        for (int r = 0; r < MT; ++r) tacc[r] = 0.0;
-#pragma unroll 4
-        for (int kb = kb_lo + sb; kb < kb_hi; kb += subsets) {
-          const uint4 a = __ldg(reinterpret_cast<const uint4*>(asec + ((size_t)kb * ly.k_pad + jc) * 16));
-          const double sa = pow2d((int)__ldg(a_exp + (size_t)kb * ly.k_pad + jc) + bias);
-#pragma unroll
-          for (int r = 0; r < MT; ++r) {
-            if (r < M) {
-              // the X mantissas are stored as {0,4,1,5}, {2,6,3,7} within each 8: back to the order of A_q
-              const uint4 x = *reinterpret_cast<const uint4*>(xm + (size_t)r * ly.K64 + kb * 16);
-              int sm = __dp4a((int)__byte_perm(x.x, x.y, 0x6420), (int)a.x, 0);
-              sm = __dp4a((int)__byte_perm(x.x, x.y, 0x7531), (int)a.y, sm);
-              sm = __dp4a((int)__byte_perm(x.z, x.w, 0x6420), (int)a.z, sm);
-              sm = __dp4a((int)__byte_perm(x.z, x.w, 0x7531), (int)a.w, sm);
-              tacc[r] = fma((double)sm, (double)xsc[r * KB + kb] * sa, tacc[r]);
-            }
-          }
-        }
-        if (live) {
-#pragma unroll
-          for (int r = 0; r < MT; ++r)
-            if (r < M) tsub[((size_t)sb * kMaxM + r) * ly.k_pad + j] = tacc[r];
-        }
-      }
-    }
+    const int subsets = t_subsets(ly.k_pad);
+    t_partial<MT>(asec, ly.K, ly.K64, ly.k_pad, kb_lo, kb_hi, M, fmt, xm, xsc, tsub);
     __syncthreads();
     for (int idx = tid; idx < M * ly.k_pad; idx += kThreads) {
       const int row = idx / ly.k_pad, col = idx % ly.k_pad;
@@ -313,15 +419,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 #pragma unroll 4
         for (int c = 0; c < ly.t_ranges; ++c) tv += __ldcg(sp + (size_t)c * M * ly.k_pad);
       }
-      double amax = (tv != tv) ? 0.0 : fabs(tv);
-#pragma unroll
-      for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
-      const int e = block_exponent(amax, p.exp_min, p.exp_max);
-      const int qv = quant_mantissa(tv, e, p.a_bits);
-      if (valid) {
-        tq8[row * ly.k_pad + col] = (int8_t)qv;
-        if ((col & 15) == 0) tqs[row * (ly.k_pad / 16) + (col >> 4)] = pow2f(e - (p.a_bits - 2));
-      }
+      store_tq(tv, valid, row, col, ly.k_pad, fmt, tq8, tqs);
     }
     __syncthreads();
     if (tid == 0 && atomicAdd(ly.tcount + 1, 1) == G - 1) {   // every CTA of the layer has read the slots: zero for the next call
@@ -329,7 +427,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       ly.tcount[1] = 0;
     }
   };
-  bool tq_built = false;
+  bool tq_built = pre;
+  int round_no = 0;
   const int slabs_mine = ly.k_slabs > warp ? (ly.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
 #pragma unroll 1
   for (int cg0 = cg_lo; cg0 < cg_hi; cg0 += kCg) {
@@ -413,20 +512,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       fetch_rank(rank_w, rank_e, cg0 + kCg);     // the next round's rank blocks
     }
 
-    // ---- the 16 warps' sums of a column (fixed order), then Y
+    // ---- the 16 warps' sums of a column (fixed order), then Y.  Two buffers in turn: the warps that add a round's
+    //      sums (the first four) do so while the others stream the next round; the barrier of that round keeps a
+    //      buffer from being rewritten before it has been read.
+    float* red_now = red + (round_no & 1) * (kWarps * 32 * kMaxM);
+    ++round_no;
 #pragma unroll
-    for (int r = 0; r < MT; ++r) red[(warp * 32 + lane) * kMaxM + r] = acc[r];
+    for (int r = 0; r < MT; ++r) red_now[(warp * 32 + lane) * kMaxM + r] = acc[r];
     __syncthreads();
     if (tid < 32 * kMaxM) {
       const int col = tid >> 2, r = tid & 3;
       if (cg0 + (col >> 3) < cg_hi && r < M) {
         float v = 0.f;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) v += red[(w * 32 + col) * kMaxM + r];
+        for (int w = 0; w < kWarps; ++w) v += red_now[(w * 32 + col) * kMaxM + r];
         Y[(size_t)r * ly.N + cg0 * 8 + col] = v;
       }
     }
-    __syncthreads();                             // red is rewritten by the next round
   }
   if (ly.k_pad > 0 && !tq_built) build_tq();     // a CTA without columns still takes part in the counts
   if (p.order == kChainLater) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -436,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 
 static size_t cols_smem_bytes(const PackedMeta& m, int M) {
   using namespace dcol;
-  return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + kWarps * kCg * 8 * kMaxM * 4 +
+  return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + 2 * kWarps * kCg * 8 * kMaxM * 4 +
          (size_t)kMaxM * m.k_pad * 8 * t_subsets(m.k_pad) + kMaxM * 16 * 4 + (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
 }
 // The column-owner kernel serves M <= 4 as long as the quantised X of the whole contraction fits in shared memory.
@@ -445,7 +547,7 @@ bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && c
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y, void* workspace,
                                cudaStream_t s) {
   const lqer_call_t one = {X, M, packed, Y};
-  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, s);
+  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, nullptr, s);
 }
 
 int decode_cols_max_group() { return dcol::kMaxGroup; }
@@ -455,7 +557,8 @@ int decode_cols_max_group() { return dcol::kMaxGroup; }
 // reduction) overlap instead of following one another.  Every layer must fit decode_cols_fits and, for n > 1, have
 // at least one cluster's worth of column groups.
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
-                                     size_t workspace_bytes, int order, int set, bool* fills_gpu, cudaStream_t s) {
+                                     size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
+                                     cudaStream_t s) {
   using namespace dcol;
   static int sm_count = 0;
   if (sm_count == 0) {
@@ -478,34 +581,29 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
 
   // CTAs per layer (one per SM at most, so that all of a launch are resident together): a single layer takes what
-  // it can use; several share the SMs by weight bytes, and what rounding leaves over goes where the load per CTA is
-  // largest
+  // it can use; several share the SMs by the time their columns take
   const int max_ctas = sm_count < kDecodeMaxCtas ? sm_count : kDecodeMaxCtas;
   int ctas[kMaxGroup];
   if (n == 1) {
     ctas[0] = metas[0].N / 8 < max_ctas ? metas[0].N / 8 : max_ctas;
   } else {
-    double total_w = 0.0;
-    for (int g = 0; g < n; ++g) total_w += (double)metas[g].K * metas[g].N;
-    int left = max_ctas;
+    // a CTA's time is its rounds (32 columns each) times the slabs a warp streams per round plus a fixed cost per
+    // round of about two slabs (measured); every layer gets one CTA, the rest go one by one where that time is largest
+    if (n > max_ctas) return cudaErrorInvalidConfiguration;   // more layers than SMs
+    double per_round[kMaxGroup];
     for (int g = 0; g < n; ++g) {
-      int c = (int)((double)max_ctas * ((double)metas[g].K * metas[g].N / total_w));
-      if (c < 1) c = 1;
-      if (c > metas[g].N / 8) c = metas[g].N / 8;
-      ctas[g] = c;
-      left -= c;
+      ctas[g] = 1;
+      per_round[g] = 2.0 + (double)((metas[g].k_slabs + kWarps - 1) / kWarps);
     }
-    if (left < 0) return cudaErrorInvalidConfiguration;   // more layers than SMs
-    while (left > 0) {
+    for (int left = max_ctas - n; left > 0; --left) {
       int best = -1;
-      double load = 0.0;
+      double worst = 0.0;
       for (int g = 0; g < n; ++g) {
-        const double l = (double)metas[g].K * metas[g].N / ctas[g];
-        if (ctas[g] < metas[g].N / 8 && l > load) { load = l; best = g; }
+        const double t = (double)(metas[g].N / 8) / (kCg * ctas[g]) * per_round[g];
+        if (ctas[g] < metas[g].N / 8 && t > worst) { worst = t; best = g; }
       }
       if (best < 0) break;
       ++ctas[best];
-      --left;
     }
   }
   size_t head = 0;
@@ -538,6 +636,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     int ranges = ctas[g] < kTRanges ? ctas[g] : kTRanges;
     if (ranges > m.K / 16) ranges = m.K / 16;
     ly.t_ranges = ranges;
+    ly.pre = pres != nullptr ? pres[g] : nullptr;
     ly.tslot = reinterpret_cast<double*>(wsb + slot_off);
     ly.tcount = reinterpret_cast<int*>(wsb + kStatusBytes) + 2 * (g + (set != 0 ? kMaxGroup : 0));
     if (i < n) slot_off += decode_cols_slot_bytes(m);
@@ -564,6 +663,56 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   if (fills_gpu != nullptr) *fills_gpu = begin == sm_count;
   LaunchScope scope(kFamDecode, s);
   return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM>, p);
+}
+
+int decode_pre_max_calls() { return dcol::kPreMaxCalls; }
+
+// X_q and T_q of n independent decode calls (M <= 4 each, every layer fitting decode_cols_fits), one CTA per call, into
+// outs[i] (decode_pre_bytes each, 256-byte aligned).
+cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas, uint8_t* const* outs, int n, int order,
+                              cudaStream_t s) {
+  using namespace dcol;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(decode_pre_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(decode_pre_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  if (n < 1 || n > kPreMaxCalls) return cudaErrorInvalidValue;
+  PreParams p;
+  p.order = order;
+  size_t smem = 0;
+  bool single = true;
+  for (int i = 0; i < kPreMaxCalls; ++i) {
+    const int g = i < n ? i : 0;
+    const PackedMeta& m = metas[g];
+    PreCall& c = p.c[i];
+    c.X = calls[g].X;
+    c.asec = static_cast<const uint8_t*>(calls[g].packed) + m.off_a;
+    c.out = outs[g];
+    c.M = calls[g].M; c.K = m.K; c.K64 = m.K64; c.k_pad = m.k_pad;
+    c.f = Formats{m.a_bits, m.lr_bits, m.exp_min, m.exp_max};
+    if (c.M < 1 || c.M > kMaxM) return cudaErrorInvalidValue;
+    if (c.M > 1) single = false;
+    const size_t need = pre_x_bytes(c.M, c.K64) + pre_t_bytes(c.k_pad) + 16 +
+                        (size_t)t_subsets(c.k_pad) * kMaxM * c.k_pad * 8 + 128;
+    if (need > smem) smem = need;
+  }
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  LaunchScope scope(kFamDecode, s);
+  return single ? cudaLaunchKernelEx(&cfg, decode_pre_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_pre_kernel<kMaxM>, p);
 }
 
 }  // namespace lqer

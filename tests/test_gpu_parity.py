@@ -229,7 +229,7 @@ def test_decode_chain_shares_one_workspace():
 @pytest.mark.parametrize("M", [1, 3])
 def test_batched_decode_groups_same_shape_calls(M):
     # seven independent calls: five layers of one shape, then two of another; the batched entry point runs them in
-    # one launch that divides the SMs among the layers by weight bytes, and must give what single calls give
+    # one launch that divides the SMs among the layers, and must give what single calls give
     spec_a = gen.LayerSpec("grp_a", M=M, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=51)
     spec_b = gen.LayerSpec("grp_b", M=M, K=512, N=2048, k=8, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=52)
     layers = []
@@ -251,6 +251,53 @@ def test_batched_decode_groups_same_shape_calls(M):
         assert torch.equal(ys, yb), sp.name             # same arithmetic, same order: bit-identical
         assert worst_ratio(yb.cpu().numpy(), olqer.forward(x.cpu().numpy(), P)) <= 1.0, sp.name
     for _, _, Pg in layers:
+        Pg.release()
+
+
+@pytest.mark.parametrize("M", [1, 4])
+def test_batched_decode_stretch_quantises_activations_ahead(M):
+    # 37 independent decode calls of three shapes (one with no low-rank part): more than one shared launch, so the
+    # batched entry point first computes every call's quantised activations and T_q in one launch, then runs the layers
+    # in launches of up to 16 that do not wait for one another; it must give what single calls give, bit for bit.
+    # With a workspace that has no room for the activations the launches compute them themselves: same results.
+    shapes = [gen.LayerSpec("st_a", M=M, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=71),
+              gen.LayerSpec("st_b", M=M, K=2112, N=264, k=16, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=72),
+              gen.LayerSpec("st_c", M=M, K=512, N=1032, k=0, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=73)]
+    base = []
+    for sp in shapes:
+        if sp.k:
+            base.append((sp,) + _random_factor_layer(sp))
+        else:
+            W = gen.make_weight(sp)
+            base.append((sp, olqer.prepare_weights(W, None, None), L.prepare_weights(_t(W), None, None)))
+    order = [0, 1, 0, 2, 1] * 7 + [0, 2]
+    Xs = [_t(gen.make_activations(base[j][0], M=M)) + 0.125 * i for i, j in enumerate(order)]
+    Yb = [torch.full((M, base[j][0].N), float("nan"), dtype=torch.float32, device=DEV) for j in order]
+    calls = L.make_calls([(x, base[j][2], y) for x, j, y in zip(Xs, order, Yb)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    launches = L.launch_count()
+    L.linear_batched(calls, ws)
+    torch.cuda.synchronize()
+    assert L.poll_status(ws) == 0
+    assert L.launch_count() - launches == 1 + 3         # activations ahead, then 16 + 16 + 5 layers
+    ws1 = torch.zeros(max(L.workspace_bytes(M, sp.K, sp.N, sp.k) for sp, _, _ in base), dtype=torch.uint8, device=DEV)
+    singles = []
+    for x, j, yb in zip(Xs, order, Yb):
+        ys = L.linear(x, base[j][2], ws1)
+        assert torch.equal(ys, yb), base[j][0].name
+        singles.append(ys)
+    for i in (0, 1, 3, 36):
+        sp, P, _ = base[order[i]]
+        assert worst_ratio(Yb[i].cpu().numpy(), olqer.forward(Xs[i].cpu().numpy(), P)) <= 1.0, sp.name
+    small = torch.zeros(ws1.numel(), dtype=torch.uint8, device=DEV)
+    Y2 = [torch.full_like(y, float("nan")) for y in Yb]
+    launches = L.launch_count()
+    L.linear_batched([(x, base[j][2], y) for x, j, y in zip(Xs, order, Y2)], small)
+    torch.cuda.synchronize()
+    assert L.poll_status(small) == 0
+    for y2, ys in zip(Y2, singles):
+        assert torch.equal(y2, ys)
+    for _, _, Pg in base:
         Pg.release()
 
 
