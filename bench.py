@@ -369,10 +369,11 @@ def run_ours(args) -> None:
             "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
             "config": {"workload": WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]",
                        "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32,
-                       "shared_launches": "lqer_linear_batched runs up to 8 consecutive independent calls together: "
-                                          "decode calls as one launch that divides the SMs among the layers by weight "
-                                          "bytes, prefill calls as one prologue per layer and one GEMM launch over the "
-                                          "tiles of all of them",
+                       "shared_launches": "lqer_linear_batched runs consecutive independent calls together: up to 16 "
+                                          "decode calls as one launch that divides the SMs among the layers (their "
+                                          "activations quantised ahead by one kernel per 64 calls), up to 8 prefill "
+                                          "calls as one prologue per layer and one GEMM launch over the tiles of all "
+                                          "of them",
                        "l2": "inputs larger than L2: every linear has its own packed weights and activations "
                              f"({sum(p.buf.numel() for p in packed) / 1e9:.2f} GB of weights per step)",
                        "parallelism": "replicas (independent token batches)" if world > 1 else "1 GPU"},

@@ -164,7 +164,9 @@ lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, floa
  * fit the largest of them.  Independent means that no call reads what another call of the
  * same batch writes; the library uses that, with the path left at 0, to share launches:
  *  - up to 16 consecutive calls with one M <= 4 (any shapes with N >= 32, one set of formats)
- *    run as ONE launch of the decode kernel that divides the SMs among them by weight bytes;
+ *    run as ONE launch of the decode kernel that divides the SMs among them; consecutive such
+ *    launches do not wait for one another, and a stretch of more than one launch first has the
+ *    quantised activations and T_q of all its calls computed by one kernel, into the workspace;
  *  - up to 8 consecutive calls with one M > 256 (any shapes, one set of formats) run their
  *    prologues into separate slices of the workspace and then ONE GEMM launch over the tiles of
  *    all of them - if the workspace holds lqer_batched_workspace_bytes(calls, n_calls); with a
