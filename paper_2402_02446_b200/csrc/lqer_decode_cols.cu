@@ -37,6 +37,7 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kMaxM = 4;
 constexpr int kCg = 4;            // column groups (of 8 columns) per round: one column per lane
 constexpr int kSets = 4;          // slabs a warp keeps in flight
+constexpr int kHoldMax = 2;       // rounds whose sums share one barrier and one pass through shared memory, at most
 constexpr int kTRanges = 16;      // CTAs of a layer that share the work of T = X_q A_q (ranges of K), at most
 
 constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
@@ -275,8 +276,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   uint8_t* xm = smem;                                               // [M][K64] int8 mantissas, permuted within 8
   float* xsc = reinterpret_cast<float*>(xm + (size_t)M * ly.K64);    // [M][KB] 2^(e_x - 6)
   int* xof = reinterpret_cast<int*>(xsc + (size_t)M * KB);          // [M][KB] bits of 1.5 * 2^23, minus 8 * sum(x) of the block
-  float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // two of [kWarps][32 columns][kMaxM], used in turn
-  double* tsub = reinterpret_cast<double*>(red + 2 * kWarps * kCg * 8 * kMaxM);   // [subsets][M][k_pad] per-warp-subset partials of T
+  float* red = reinterpret_cast<float*>(xof + (size_t)M * KB);      // two of [kHoldMax rounds][kWarps][32 columns][kMaxM], used in turn
+  double* tsub = reinterpret_cast<double*>(red + 2 * kHoldMax * kWarps * kCg * 8 * kMaxM);   // [subsets][M][k_pad] per-warp-subset partials of T
   int* wait_ok = reinterpret_cast<int*>(tsub);                       // reused once T's partial sums have left: outcome of the wait
   float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * t_subsets(ly.k_pad));   // [M][k_pad / 16]
   int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);        // [M][k_pad]
@@ -428,7 +429,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
     }
   };
   bool tq_built = pre;
-  int round_no = 0;
+  constexpr int kHold = MT == 1 ? kHoldMax : 1;  // rounds per barrier (their sums wait in registers; four were no faster)
+  constexpr int kHeld = kHold > 1 ? kHold - 1 : 1;
+  int meet_no = 0, n_held = 0;
+  int held_cg0[kHeld];
+  float held[kHeld][MT];
+#pragma unroll
+  for (int h = 0; h < kHold - 1; ++h) {
+    held_cg0[h] = 0;
+#pragma unroll
+    for (int r = 0; r < MT; ++r) held[h][r] = 0.f;
+  }
   const int slabs_mine = ly.k_slabs > warp ? (ly.k_slabs - warp + kWarps - 1) / kWarps : 0;   // slabs warp, warp + 16, ...
 #pragma unroll 1
   for (int cg0 = cg_lo; cg0 < cg_hi; cg0 += kCg) {
@@ -512,23 +523,51 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       fetch_rank(rank_w, rank_e, cg0 + kCg);     // the next round's rank blocks
     }
 
-    // ---- the 16 warps' sums of a column (fixed order), then Y.  Two buffers in turn: the warps that add a round's
-    //      sums (the first four) do so while the others stream the next round; the barrier of that round keeps a
-    //      buffer from being rewritten before it has been read.
-    float* red_now = red + (round_no & 1) * (kWarps * 32 * kMaxM);
-    ++round_no;
+    // ---- the 16 warps' sums of a column (fixed order), then Y.  Rounds meet kHold at a time: the earlier ones keep
+    //      their sums in registers and the last brings all to shared memory, so kHold rounds cost one barrier.  Two
+    //      buffers in turn: the warps that add the sums (the first four) do so while the others stream the next round;
+    //      the barrier of the next meeting keeps a buffer from being rewritten before it has been read.
+    if (n_held < kHold - 1 && cg0 + kCg < cg_hi) {
 #pragma unroll
-    for (int r = 0; r < MT; ++r) red_now[(warp * 32 + lane) * kMaxM + r] = acc[r];
+      for (int h = 0; h < kHold - 1; ++h)
+        if (h == n_held) {
+#pragma unroll
+          for (int r = 0; r < MT; ++r) held[h][r] = acc[r];
+          held_cg0[h] = cg0;
+        }
+      ++n_held;
+      continue;
+    }
+    float* red_now = red + (meet_no & 1) * (kHoldMax * kWarps * 32 * kMaxM);
+    ++meet_no;
+#pragma unroll
+    for (int h = 0; h < kHold - 1; ++h)
+      if (h < n_held) {
+#pragma unroll
+        for (int r = 0; r < MT; ++r) red_now[((h * kWarps + warp) * 32 + lane) * kMaxM + r] = held[h][r];
+      }
+#pragma unroll
+    for (int r = 0; r < MT; ++r) red_now[((n_held * kWarps + warp) * 32 + lane) * kMaxM + r] = acc[r];
     __syncthreads();
     if (tid < 32 * kMaxM) {
       const int col = tid >> 2, r = tid & 3;
-      if (cg0 + (col >> 3) < cg_hi && r < M) {
-        float v = 0.f;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) v += red_now[(w * 32 + col) * kMaxM + r];
-        Y[(size_t)r * ly.N + cg0 * 8 + col] = v;
+      for (int h = 0; h < kHold; ++h) {
+        if (h <= n_held) {
+          int c0 = cg0;
+#pragma unroll
+          for (int q = 0; q < kHold - 1; ++q)
+            if (q == h && h < n_held) c0 = held_cg0[q];
+          if (c0 + (col >> 3) < cg_hi && r < M) {
+            float v = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) v += red_now[((h * kWarps + w) * 32 + col) * kMaxM + r];
+            Y[(size_t)r * ly.N + c0 * 8 + col] = v;
+          }
+        }
       }
     }
+    n_held = 0;
   }
   if (ly.k_pad > 0 && !tq_built) build_tq();     // a CTA without columns still takes part in the counts
   if (p.order == kChainLater) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -538,7 +577,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 
 static size_t cols_smem_bytes(const PackedMeta& m, int M) {
   using namespace dcol;
-  return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + 2 * kWarps * kCg * 8 * kMaxM * 4 +
+  return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + 2 * kHoldMax * kWarps * kCg * 8 * kMaxM * 4 +
          (size_t)kMaxM * m.k_pad * 8 * t_subsets(m.k_pad) + kMaxM * 16 * 4 + (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
 }
 // The column-owner kernel serves M <= 4 as long as the quantised X of the whole contraction fits in shared memory.
@@ -561,6 +600,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
                                      cudaStream_t s) {
   using namespace dcol;
   static int sm_count = 0;
+  static bool one_cta_per_sm = false;
   if (sm_count == 0) {
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
@@ -569,6 +609,11 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(decode_cols_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
+    // chaining launches relies on one CTA per SM (registers): a launch on every SM then leaves room for no other
+    int o1 = 2, o4 = 2;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o1, decode_cols_kernel<1>, kThreads, 0) != cudaSuccess) o1 = 2;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o4, decode_cols_kernel<kMaxM>, kThreads, 0) != cudaSuccess) o4 = 2;
+    one_cta_per_sm = o1 == 1 && o4 == 1;
     sm_count = sms > 0 ? sms : 1;
   }
   if (n < 1 || n > kMaxGroup) return cudaErrorInvalidValue;
@@ -588,12 +633,12 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     ctas[0] = metas[0].N / 8 < max_ctas ? metas[0].N / 8 : max_ctas;
   } else {
     // a CTA's time is its rounds (32 columns each) times the slabs a warp streams per round plus a fixed cost per
-    // round of about two slabs (measured); every layer gets one CTA, the rest go one by one where that time is largest
+    // round of about 1.3 slabs (measured); every layer gets one CTA, the rest go one by one where that time is largest
     if (n > max_ctas) return cudaErrorInvalidConfiguration;   // more layers than SMs
     double per_round[kMaxGroup];
     for (int g = 0; g < n; ++g) {
       ctas[g] = 1;
-      per_round[g] = 2.0 + (double)((metas[g].k_slabs + kWarps - 1) / kWarps);
+      per_round[g] = 1.3 + (double)((metas[g].k_slabs + kWarps - 1) / kWarps);
     }
     for (int left = max_ctas - n; left > 0; --left) {
       int best = -1;
@@ -660,7 +705,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (fills_gpu != nullptr) *fills_gpu = begin == sm_count;
+  if (fills_gpu != nullptr) *fills_gpu = one_cta_per_sm && begin == sm_count;
   LaunchScope scope(kFamDecode, s);
   return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM>, p);
 }
