@@ -125,7 +125,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ reference arm
-def oracle_sample(rows: int):
+def oracle_sample(rows: int, a_bits: int = 8):
     """The bounded sample the oracle is timed on: layer 0's q, gate and down linears, `rows` tokens
     of the M=2048 batch.  Returns (callable running the sample once, flops of one run, description)."""
     from oracle import lqer as olqer
@@ -141,7 +141,7 @@ def oracle_sample(rows: int):
         flops += layer_flops(rows, spec.K, spec.N, spec.k)
     def run():
         for X, P in work:
-            olqer.forward(X, P)
+            olqer.forward(X, P, a_bits=a_bits)
     return run, flops, f"layer 0 q, gate, down linears, {rows} rows of the M={M_PREFILL} batch"
 
 
@@ -156,8 +156,8 @@ def blas_threads() -> int:
     return os.cpu_count() or 1
 
 
-def time_oracle(steps: int, warmup: int, rows: int):
-    run, flops, what = oracle_sample(rows)
+def time_oracle(steps: int, warmup: int, rows: int, a_bits: int = 8):
+    run, flops, what = oracle_sample(rows, a_bits)
     for _ in range(warmup):
         run()
     t0 = time.perf_counter()
@@ -171,7 +171,7 @@ def run_reference(args) -> None:
     if int(os.environ.get("RANK", "0")) != 0:
         return
     steps, warmup = max(args.steps, 1), max(args.warmup, 0)
-    tflops, ms, what = time_oracle(steps, warmup, rows=args.oracle_rows)
+    tflops, ms, what = time_oracle(steps, warmup, rows=args.oracle_rows, a_bits=args.a_bits)
     cores = blas_threads()
     line = {"impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -216,13 +216,15 @@ def run_ours(args) -> None:
 
     # ---- build the stack (untimed): one packed buffer per linear, its own activations
     layers = args.layers
+    cfg = L.default_config()
+    cfg.a_bits = args.a_bits
     packed, shapes = [], []
     for layer in range(layers):
         for which in range(len(gen.STACK_LINEARS)):
             spec = gen.config_stack(layer, which, M_PREFILL)
             W = gen.make_weight_device(spec, dev)
             A, B = gen.make_random_factors_device(spec, dev)
-            packed.append(L.prepare_weights(W, A, B))
+            packed.append(L.prepare_weights(W, A, B, cfg))
             shapes.append((spec.K, spec.N, spec.k, spec))
             del W, A, B
     torch.cuda.synchronize()
@@ -358,7 +360,7 @@ def run_ours(args) -> None:
     # ---- the oracle on the host cores (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        tflops, ms, what = time_oracle(1, 0, rows=args.oracle_rows)
+        tflops, ms, what = time_oracle(1, 0, rows=args.oracle_rows, a_bits=args.a_bits)
         cpu = {"value": tflops, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": what,
                "seconds": ms / 1e3}
 
@@ -367,8 +369,9 @@ def run_ours(args) -> None:
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
-            "config": {"workload": WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]",
-                       "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32,
+            "config": {"workload": (WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]") +
+                                   ("" if args.a_bits == 8 else f" [activations MXINT{args.a_bits}]"),
+                       "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32, "a_bits": args.a_bits,
                        "shared_launches": "lqer_linear_batched runs consecutive independent calls together: up to 16 "
                                           "decode calls as one launch that divides the SMs among the layers (their "
                                           "activations quantised ahead by one kernel per 64 calls), up to 8 prefill "
@@ -400,6 +403,7 @@ def main() -> None:
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--layers", type=int, default=32, help="decoder layers of the stack (32 = the full workload)")
     ap.add_argument("--oracle-rows", type=int, default=2048, help="token rows of the oracle's bounded sample")
+    ap.add_argument("--a-bits", type=int, default=8, help="mantissa bits of the activations: 8 (W4A8, the workload) or 6 (W4A6)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

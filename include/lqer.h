@@ -53,12 +53,14 @@ typedef enum {
 /* Format parameters (Section 3.1: b_l, b_h; Section 4.1: block size, exponent width). */
 typedef struct {
   int w_bits;        /* mantissa bits of W_q: 4 */
-  int a_bits;        /* mantissa bits of X and of T = X A_k: 8 */
+  int a_bits;        /* mantissa bits of X and of T = X A_k: 3..8, default 8 (W4A8; 6 gives the W4A6 of Section 4.3) */
   int lr_bits;       /* mantissa bits of A_k, B_k: 8 */
   int block;         /* block size along the contraction dimension: 16 */
-  int exp_min;       /* shared-exponent clamp window, default [-56, 55] */
+  int exp_min;       /* shared-exponent clamp window of X and T, default [-56, 55] */
   int exp_max;
   int deterministic; /* 1: fixed reduction order (the only mode implemented) */
+  int w_exp_min;     /* shared-exponent clamp window of W_q, A_k, B_k, default [-56, 55]; Section 4.1 gives these a */
+  int w_exp_max;     /* 4-bit shared exponent (16 values, e.g. [-12, 3]) and the activations an 8-bit one */
 } lqer_config_t;
 
 /* One call of a batch (Section 4.3: layers are independent). */

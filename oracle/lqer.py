@@ -219,16 +219,20 @@ def quantize_weight(W: np.ndarray, w_bits: int = 4) -> tuple[np.ndarray, np.ndar
 
 
 def prepare_weights(W: np.ndarray, A: np.ndarray | None, B: np.ndarray | None,
-                    w_bits: int = 4, lr_bits: int = 8) -> PreparedWeights:
+                    w_bits: int = 4, lr_bits: int = 8,
+                    exp_min: int = mxint.EXP_MIN, exp_max: int = mxint.EXP_MAX) -> PreparedWeights:
     """Quantise W, A_k, B_k as the layer stores them (Section 3.1, Section 4.1).
 
     The layer's interface carries fp32 tensors, so A and B are rounded to fp32
     first.  B's rank dimension is zero-padded to a multiple of 16 so that its
-    [16, 1] blocks are whole.
+    [16, 1] blocks are whole.  [exp_min, exp_max] is the shared-exponent window
+    of the three matrices (Section 4.1 gives them a 4-bit shared exponent, i.e.
+    16 values, against 8 bits for the activations; where the window sits is left
+    to the caller).
     """
     W = np.asarray(W, dtype=np.float32)
     K, N = W.shape
-    Wm, We = mxint.quantize(W, w_bits, axis=0)
+    Wm, We = mxint.quantize(W, w_bits, axis=0, exp_min=exp_min, exp_max=exp_max)
     k = 0 if A is None else A.shape[1]
     if k == 0:
         z8 = np.zeros((0, 0), np.int8)
@@ -236,8 +240,8 @@ def prepare_weights(W: np.ndarray, A: np.ndarray | None, B: np.ndarray | None,
                                np.zeros((0, N), np.int8), np.zeros((0, N), np.int16))
     A32 = np.asarray(A, dtype=np.float32)
     B32 = mxint.pad_axis(np.asarray(B, dtype=np.float32), axis=0)
-    Am, Ae = mxint.quantize(A32, lr_bits, axis=0)
-    Bm, Be = mxint.quantize(B32, lr_bits, axis=0)
+    Am, Ae = mxint.quantize(A32, lr_bits, axis=0, exp_min=exp_min, exp_max=exp_max)
+    Bm, Be = mxint.quantize(B32, lr_bits, axis=0, exp_min=exp_min, exp_max=exp_max)
     return PreparedWeights(K, N, k, B32.shape[0], Wm, We, Am, Ae, Bm, Be)
 
 

@@ -31,7 +31,8 @@ class LqerError(RuntimeError):
 
 class Config(C.Structure):
     _fields_ = [("w_bits", C.c_int), ("a_bits", C.c_int), ("lr_bits", C.c_int), ("block", C.c_int),
-                ("exp_min", C.c_int), ("exp_max", C.c_int), ("deterministic", C.c_int)]
+                ("exp_min", C.c_int), ("exp_max", C.c_int), ("deterministic", C.c_int),
+                ("w_exp_min", C.c_int), ("w_exp_max", C.c_int)]
 
 
 KERNEL_FAMILIES = ["pack", "export", "quantize", "prologue", "gemm_simt", "gemm_tc", "gemm_tc_pair", "decode"]

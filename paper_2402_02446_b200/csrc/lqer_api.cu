@@ -56,9 +56,11 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 static lqer_status_t check_config(const lqer_config_t* cfg) {
   if (cfg == nullptr) return LQER_ERR_NULL;
-  if (cfg->w_bits != 4 || cfg->a_bits != 8 || cfg->lr_bits != 8 || cfg->block != 16) return LQER_ERR_CONFIG;
+  // activations (and T) take 3 to 8 mantissa bits (Section 4.3 compares W4A8 and W4A6); weights and factors are fixed
+  if (cfg->w_bits != 4 || cfg->a_bits < 3 || cfg->a_bits > 8 || cfg->lr_bits != 8 || cfg->block != 16) return LQER_ERR_CONFIG;
   // every dequantised value must be a normal bf16 and every product a normal fp32
   if (cfg->exp_min < -56 || cfg->exp_max > 55 || cfg->exp_min > cfg->exp_max) return LQER_ERR_CONFIG;
+  if (cfg->w_exp_min < -56 || cfg->w_exp_max > 55 || cfg->w_exp_min > cfg->w_exp_max) return LQER_ERR_CONFIG;
   if (cfg->deterministic != 0 && cfg->deterministic != 1) return LQER_ERR_CONFIG;
   return LQER_OK;
 }
@@ -81,6 +83,7 @@ static void fill_meta(PackedMeta& m, int K, int N, int k, const lqer_config_t& c
   m.r_blocks = m.k_pad / 16;
   m.w_bits = c.w_bits; m.a_bits = c.a_bits; m.lr_bits = c.lr_bits; m.block = c.block;
   m.exp_min = c.exp_min; m.exp_max = c.exp_max; m.deterministic = 1;
+  m.w_exp_min = c.w_exp_min; m.w_exp_max = c.w_exp_max;
   m.off_w = kHeaderBytes;
   m.off_b = align_up(m.off_w + (size_t)m.n_tiles * m.k_slabs * kWTileBytes, 256);
   m.off_a = align_up(m.off_b + (size_t)m.n_tiles * b_tile_bytes(m), 256);
@@ -90,7 +93,7 @@ static void fill_meta(PackedMeta& m, int K, int N, int k, const lqer_config_t& c
 
 static bool meta_valid(const PackedMeta& m) {
   if (m.magic != kMagic || m.version != kVersion || m.checksum != meta_checksum(m)) return false;
-  lqer_config_t c{m.w_bits, m.a_bits, m.lr_bits, m.block, m.exp_min, m.exp_max, m.deterministic};
+  lqer_config_t c{m.w_bits, m.a_bits, m.lr_bits, m.block, m.exp_min, m.exp_max, m.deterministic, m.w_exp_min, m.w_exp_max};
   if (check_config(&c) != LQER_OK || check_shape(m.K, m.N, m.k) != LQER_OK) return false;
   PackedMeta ref;
   fill_meta(ref, m.K, m.N, m.k, c);
@@ -322,7 +325,7 @@ const char* lqer_status_string(lqer_status_t status) {
 
 lqer_status_t lqer_default_config(lqer_config_t* cfg) {
   if (cfg == nullptr) return LQER_ERR_NULL;
-  *cfg = lqer_config_t{4, 8, 8, 16, -56, 55, 1};
+  *cfg = lqer_config_t{4, 8, 8, 16, -56, 55, 1, -56, 55};
   return LQER_OK;
 }
 

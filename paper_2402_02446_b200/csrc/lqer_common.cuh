@@ -23,7 +23,7 @@ namespace lqer {
 // B section: per n_tile:  mantissas [rb][n 128][16 B int8]  then exps [rb][n 128]
 // A section: mantissas [K/16][k_pad][16 B int8]  then exps [K/16][k_pad]
 constexpr uint32_t kMagic = 0x5245514Cu;  // "LQER"
-constexpr uint32_t kVersion = 1;
+constexpr uint32_t kVersion = 2;
 constexpr int kHeaderBytes = 256;
 constexpr int kTileN = 128;
 constexpr int kSlabK = 64;
@@ -36,17 +36,17 @@ struct PackedMeta {
   int32_t K, N, k, k_pad;
   int32_t K64, n_tiles, k_slabs, r_blocks;
   int32_t w_bits, a_bits, lr_bits, block, exp_min, exp_max, deterministic;
-  int32_t reserved0;
+  int32_t w_exp_min, w_exp_max, reserved0;      // exp_min/max: window of X and T; w_exp_min/max: of W_q, A_k, B_k
   uint64_t off_w, off_b, off_a, total_bytes;
   uint32_t checksum;
-  uint32_t pad_[64 - 27];
+  uint32_t pad_[64 - 29];
 };
 static_assert(sizeof(PackedMeta) == kHeaderBytes, "header must be 256 bytes");
 
 inline uint32_t meta_checksum(const PackedMeta& m) {
   const uint32_t* w = reinterpret_cast<const uint32_t*>(&m);
   uint32_t h = 2166136261u;
-  for (int i = 0; i < 26; ++i) { h ^= w[i]; h *= 16777619u; }
+  for (int i = 0; i < 28; ++i) { h ^= w[i]; h *= 16777619u; }
   return h;
 }
 

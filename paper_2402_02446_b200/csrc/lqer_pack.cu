@@ -23,7 +23,7 @@ __global__ void __launch_bounds__(512) pack_w_kernel(const float* __restrict__ W
     v[i] = (n < m.N && k < m.K) ? W[(size_t)k * m.N + n] : 0.0f;
     amax = fmaxf(amax, abs_ignore_nan(v[i]));
   }
-  const int e = block_exponent(amax, m.exp_min, m.exp_max);
+  const int e = block_exponent(amax, m.w_exp_min, m.w_exp_max);
   uint32_t w[2] = {0u, 0u};
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
@@ -49,7 +49,7 @@ __global__ void pack_a_kernel(const float* __restrict__ A, PackedMeta m, uint8_t
     v[i] = (j < m.k) ? A[(size_t)(kb * 16 + i) * m.k + j] : 0.0f;
     amax = fmaxf(amax, abs_ignore_nan(v[i]));
   }
-  const int e = block_exponent(amax, m.exp_min, m.exp_max);
+  const int e = block_exponent(amax, m.w_exp_min, m.w_exp_max);
   uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
   for (int i = 0; i < 16; ++i)
@@ -71,7 +71,7 @@ __global__ void pack_b_kernel(const float* __restrict__ B, PackedMeta m, uint8_t
     v[i] = (n < m.N && r < m.k) ? B[(size_t)r * m.N + n] : 0.0f;
     amax = fmaxf(amax, abs_ignore_nan(v[i]));
   }
-  const int e = block_exponent(amax, m.exp_min, m.exp_max);
+  const int e = block_exponent(amax, m.w_exp_min, m.w_exp_max);
   uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
   for (int i = 0; i < 16; ++i)

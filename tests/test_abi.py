@@ -43,6 +43,7 @@ def test_status_strings_and_defaults():
     assert len(seen) == 11 and lib.lqer_status_string(0) == b"ok"
     cfg = L.default_config()
     assert (cfg.w_bits, cfg.a_bits, cfg.lr_bits, cfg.block, cfg.exp_min, cfg.exp_max) == (4, 8, 8, 16, -56, 55)
+    assert (cfg.w_exp_min, cfg.w_exp_max, cfg.deterministic) == (-56, 55, 1)
 
 
 def test_size_queries_follow_the_format():
@@ -76,6 +77,14 @@ def test_host_side_argument_errors():
     assert lib.lqer_packed_bytes(256, 256, 8, C.byref(bad), C.byref(out)) == E("LQER_ERR_CONFIG")
     bad = L.default_config(); bad.exp_min = -100
     assert lib.lqer_packed_bytes(256, 256, 8, C.byref(bad), C.byref(out)) == E("LQER_ERR_CONFIG")
+    bad = L.default_config(); bad.w_exp_max = 56
+    assert lib.lqer_packed_bytes(256, 256, 8, C.byref(bad), C.byref(out)) == E("LQER_ERR_CONFIG")
+    bad = L.default_config(); bad.w_exp_min, bad.w_exp_max = 4, 3
+    assert lib.lqer_packed_bytes(256, 256, 8, C.byref(bad), C.byref(out)) == E("LQER_ERR_CONFIG")
+    for a_bits, ok in ((2, False), (3, True), (6, True), (8, True), (9, False)):   # activation mantissa width
+        c6 = L.default_config(); c6.a_bits = a_bits
+        want = E("LQER_OK") if ok else E("LQER_ERR_CONFIG")
+        assert lib.lqer_packed_bytes(256, 256, 8, C.byref(c6), C.byref(out)) == want
     # null / unknown buffers are refused before anything is launched
     assert lib.lqer_linear(None, 1, None, None, None, 0) == E("LQER_ERR_NULL")
     assert lib.lqer_linear_stream(4096, 1, 8192, 4096, 4096, 1 << 20, None) == E("LQER_ERR_BAD_PACKED")

@@ -130,6 +130,87 @@ def test_project_lowrank_tensor_core_prologue_bit_exact(spec):
     Pg.release()
 
 
+@pytest.mark.parametrize("a_bits", [6, 4])
+def test_activation_mantissa_width_option(a_bits):
+    # W4A6 (Section 4.3) and a narrower width: X and T = X_q A_q take a_bits mantissa bits, everything else as before.
+    # Every path: the decode kernels (M = 1, 3 and 9), the GEMM with either prologue (M = 37, 300), and a stretch of
+    # batched decode calls whose activations are quantised ahead.
+    cfg = L.default_config()
+    cfg.a_bits = a_bits
+    for X in (_adversarial_x(), gen.make_activations(gen.config_tiny())):
+        Xm, Xe = L.quantize_activations(_t(X), cfg)
+        om, oe = mxint.quantize(X, a_bits, axis=1)
+        assert np.array_equal(Xm.cpu().numpy(), om)
+        assert np.array_equal(Xe.cpu().numpy(), exp_bytes(oe))
+    for spec, Ms in ((SMALL_SPECS[1], (2, 37)), (TC_PROLOGUE_SPECS[2], (1, 3, 9, 300))):
+        W, A, B, P = oracle_layer(spec, "jacobi" if spec.K <= 320 else "subspace")
+        Pg = L.prepare_weights(_t(W), _t(A), _t(B), cfg)
+        ws = L.new_workspace(max(Ms), Pg)
+        for M in Ms:
+            X = gen.make_activations(spec, M=M)
+            ref = olqer.forward(X, P, a_bits=a_bits)
+            for path in (binding.PATH_AUTO, binding.PATH_TENSOR_PROLOGUE):
+                if path != binding.PATH_AUTO and M <= 16:
+                    continue
+                L.set_path(path)
+                try:
+                    Tm, Te = L.project_lowrank(_t(X), Pg, ws)
+                    Y = L.linear(_t(X), Pg, ws).cpu().numpy()
+                finally:
+                    L.set_path(binding.PATH_AUTO)
+                assert L.poll_status(ws) == 0
+                assert np.array_equal(Tm.cpu().numpy(), ref.Tm), (spec.name, M, path)
+                assert np.array_equal(Te.cpu().numpy(), exp_bytes(ref.Te)), (spec.name, M, path)
+                assert worst_ratio(Y, ref) <= 1.0, (spec.name, M, path)
+        if spec.N >= 32 and 1 in Ms:
+            Xs = [_t(gen.make_activations(spec, M=1)) + 0.25 * i for i in range(20)]
+            Yb = [torch.full((1, spec.N), float("nan"), dtype=torch.float32, device=DEV) for _ in Xs]
+            calls = L.make_calls([(x, Pg, y) for x, y in zip(Xs, Yb)])
+            wsb = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+            L.linear_batched(calls, wsb)
+            torch.cuda.synchronize()
+            assert L.poll_status(wsb) == 0
+            for i, (x, yb) in enumerate(zip(Xs, Yb)):
+                assert torch.equal(L.linear(x, Pg, ws), yb)
+                if i in (0, 19):
+                    assert worst_ratio(yb.cpu().numpy(), olqer.forward(x.cpu().numpy(), P, a_bits=a_bits)) <= 1.0
+        Pg.release()
+
+
+def test_weight_exponent_window_option():
+    # W_q, A_k and B_k with a 4-bit shared exponent (Section 4.1): a window of 16 values, here [-12, 3], while X and T
+    # keep the wide one.  Some blocks lie below the window, some above; packing must match the oracle bit for bit and
+    # the layer (decode kernels and GEMM) must stay within the tolerance.
+    spec = gen.LayerSpec("win", M=40, K=256, N=264, k=24, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=81)
+    W = gen.make_weight(spec)
+    W[:, :8] *= np.float32(2.0 ** -12)
+    W[:, 8:16] *= np.float32(2.0 ** 9)
+    A, B = gen.make_random_factors(spec)
+    B[:, 16:24] *= np.float32(2.0 ** 12)
+    A[:, :2] *= np.float32(2.0 ** -14)
+    cfg = L.default_config()
+    cfg.w_exp_min, cfg.w_exp_max = -12, 3
+    P = olqer.prepare_weights(W, A, B, exp_min=-12, exp_max=3)
+    assert P.We.min() == -12 and P.We.max() == 3 and P.Be.max() == 3 and P.Ae.min() == -12
+    Pg = L.prepare_weights(_t(W), _t(A), _t(B), cfg)
+    ex = L.export_weights(Pg)
+    torch.cuda.synchronize()
+    for name in ("Wm", "Am", "Bm"):
+        assert np.array_equal(ex[name].cpu().numpy(), getattr(P, name)), name
+    for name in ("We", "Ae", "Be"):
+        assert np.array_equal(ex[name].cpu().numpy(), exp_bytes(getattr(P, name))), name
+    ws = L.new_workspace(spec.M, Pg)
+    for M in (1, 5, 40):
+        X = gen.make_activations(spec, M=M)
+        ref = olqer.forward(X, P)
+        Tm, Te = L.project_lowrank(_t(X), Pg, ws)
+        Y = L.linear(_t(X), Pg, ws).cpu().numpy()
+        assert L.poll_status(ws) == 0
+        assert np.array_equal(Tm.cpu().numpy(), ref.Tm) and np.array_equal(Te.cpu().numpy(), exp_bytes(ref.Te)), M
+        assert worst_ratio(Y, ref) <= 1.0, M
+    Pg.release()
+
+
 @pytest.mark.parametrize("spec", SMALL_SPECS, ids=lambda s: s.name)
 def test_linear_reference_kernel(spec):
     W, A, B, P, Pg = _prepare(spec)

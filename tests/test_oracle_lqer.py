@@ -208,6 +208,36 @@ def test_exact_integer_regime():
     assert np.array_equal(out.Y * 256.0, want.astype(np.float64))
 
 
+def test_prepare_weights_exponent_window():
+    # the window of W_q, A_k, B_k is passed through to every one of the three quantisers and nowhere else
+    g = np.random.default_rng(5)
+    W = (g.standard_normal((64, 24)) * 0.02).astype(np.float32)
+    W[:16, 0] = 2.0 ** -20           # a block below the window [-12, 3]
+    A = (g.standard_normal((64, 8)) * 0.1).astype(np.float32)
+    B = (g.standard_normal((8, 24)) * 0.05).astype(np.float32)
+    B[:, 1] = 300.0                   # a block above it
+    wide = lqer.prepare_weights(W, A, B)
+    narrow = lqer.prepare_weights(W, A, B, exp_min=-12, exp_max=3)
+    for name, bits, axis in (("W", 4, 0), ("A", 8, 0), ("B", 8, 0)):
+        src = {"W": W, "A": A, "B": mxint.pad_axis(B, axis=0)}[name]
+        m, e = mxint.quantize(src, bits, axis=axis, exp_min=-12, exp_max=3)
+        assert np.array_equal(getattr(narrow, name + "m"), m) and np.array_equal(getattr(narrow, name + "e"), e)
+    assert narrow.We.min() == -12 and narrow.We[0, 0] == -12 and wide.We[0, 0] == -20
+    assert narrow.Be.max() == 3 and narrow.Be[0, 1] == 3 and wide.Be[0, 1] == 8
+    # blocks inside the window are untouched
+    inside = (wide.We >= -12) & (wide.We <= 3)
+    assert np.array_equal(np.repeat(inside, 16, axis=0) * narrow.Wm, np.repeat(inside, 16, axis=0) * wide.Wm)
+    # the forward pass reads the stored exponents: X keeps its own, wide window
+    X = (g.standard_normal((3, 64)) * np.exp2(g.integers(-30, 20, size=(3, 1)))).astype(np.float32)
+    ref = lqer.forward(X, narrow)
+    assert ref.Xe.min() < -12 or ref.Xe.max() > 3
+    Xdq = mxint.dequantize(ref.Xm, ref.Xe, 8, axis=1)
+    Wdq = mxint.dequantize(narrow.Wm, narrow.We, 4, axis=0)
+    Tdq = mxint.dequantize(ref.Tm, ref.Te, 8, axis=1)
+    Bdq = mxint.dequantize(narrow.Bm, narrow.Be, 8, axis=0)
+    assert np.allclose(ref.Y, Xdq @ Wdq + Tdq @ Bdq, rtol=1e-13, atol=0)
+
+
 def test_tiny_config_end_to_end():
     # Config 1 end to end on the oracle alone: the factors come out of the full Jacobi SVD.
     spec = gen.config_tiny()

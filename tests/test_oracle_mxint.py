@@ -117,6 +117,23 @@ def test_window_and_specials():
     assert mxint.exponent_bytes(e)[:, 0].tolist() == [71, 182, 182, 126]
 
 
+def test_four_bit_exponent_window():
+    # A 4-bit shared exponent holds 16 values (Section 4.1: weights and low-rank matrices); with the window [-12, 3]:
+    # a block max of 0.05 (e = -5) is inside and quantises as in the wide window; 2^-20 is below it and takes
+    # e = -12, step 2^-14 (4-bit), so 2^-13 = 2 steps -> 2 and 2^-20 -> 0; 100 (e = 6) is above it and takes e = 3,
+    # step 2: 100 / 2 = 50 -> clamped to 7, 5 -> 2.5 steps -> 2 (half to even), 7 -> 3.5 steps -> 4.
+    v = np.zeros((3, 16), np.float32)
+    v[0, :4] = [0.02, -0.013, 0.05, 0.0039]
+    v[1, :2] = [2.0 ** -13, 2.0 ** -20]
+    v[2, :3] = [100.0, 5.0, 7.0]
+    m, e = mxint.quantize(v, 4, axis=1, exp_min=-12, exp_max=3)
+    assert e[:, 0].tolist() == [-5, -12, 3]
+    assert m[0, :4].tolist() == [3, -2, 6, 0]
+    assert m[1, :2].tolist() == [2, 0]
+    assert m[2, :3].tolist() == [7, 2, 4]
+    assert mxint.exponent_bytes(e)[:, 0].tolist() == [122, 115, 130]
+
+
 def test_padding_is_neutral():
     g = np.random.default_rng(9)
     b = g.standard_normal((8, 5)).astype(np.float32)
