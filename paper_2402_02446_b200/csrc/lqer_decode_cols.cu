@@ -144,7 +144,7 @@ __device__ __forceinline__ void quantize_x_rows(const float* X, int M, int K, in
 // an exact integer dot product (dp4a) of the mantissas, scaled in fp64.  The fp64 sums are exact too unless the block
 // exponents of one row spread over more than about 30 binades, and the order of the additions is fixed in any case.
 // Leaves tsub[t_subsets(k_pad)][kMaxM][k_pad]; the caller adds the subsets in order after a barrier.
-template <int MT>
+template <int MT, int UNROLL>
 __device__ __forceinline__ void t_partial(const uint8_t* asec, int K, int K64, int k_pad, int kb_lo, int kb_hi, int M,
                                           const Formats& f, const uint8_t* xm, const float* xsc, double* tsub) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -163,7 +163,7 @@ __device__ __forceinline__ void t_partial(const uint8_t* asec, int K, int K64, i
       double tacc[MT];
 #pragma unroll
       for (int r = 0; r < MT; ++r) tacc[r] = 0.0;
-#pragma unroll 4
+#pragma unroll UNROLL
       for (int kb = kb_lo + sb; kb < kb_hi; kb += subsets) {
         const uint4 a = __ldg(reinterpret_cast<const uint4*>(asec + ((size_t)kb * k_pad + jc) * 16));
         const double sa = pow2d((int)__ldg(a_exp + (size_t)kb * k_pad + jc) + bias);
@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_pre_kernel(const __grid_co
   for (int i = tid; i < (int)pre_t_bytes(c.k_pad) / 4; i += kThreads) reinterpret_cast<uint32_t*>(tqs)[i] = 0u;
   __syncthreads();
   if (c.k_pad > 0) {
-    t_partial<MT>(c.asec, c.K, c.K64, c.k_pad, 0, c.K / 16, M, c.f, xm, xsc, tsub);
+    t_partial<MT, 8>(c.asec, c.K, c.K64, c.k_pad, 0, c.K / 16, M, c.f, xm, xsc, tsub);   // the whole of K: many loads in flight
     __syncthreads();
     const int subsets = t_subsets(c.k_pad), total = M * c.k_pad;
     for (int base = 0; base < total; base += kThreads) {
@@ -376,7 +376,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   // ---- this CTA's share of T = X_q A_q
   if (t_worker) {
     const int subsets = t_subsets(ly.k_pad);
-    t_partial<MT>(asec, ly.K, ly.K64, ly.k_pad, kb_lo, kb_hi, M, fmt, xm, xsc, tsub);
+    t_partial<MT, 4>(asec, ly.K, ly.K64, ly.k_pad, kb_lo, kb_hi, M, fmt, xm, xsc, tsub);
     __syncthreads();
     for (int idx = tid; idx < M * ly.k_pad; idx += kThreads) {
       const int row = idx / ly.k_pad, col = idx % ly.k_pad;
