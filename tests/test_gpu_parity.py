@@ -382,6 +382,33 @@ def test_batched_decode_stretch_quantises_activations_ahead(M):
         Pg.release()
 
 
+def test_batched_mixed_stretches_and_prefill():
+    # one batched call: a stretch of 18 decode calls with M = 1, three prefill calls (M = 300), then a stretch of 20
+    # decode calls with M = 2 that is followed by a lone M = 9 call.  The stretches quantise their activations ahead into
+    # the part of the workspace that the prefill group uses in between; every call must give what it gives alone.
+    sd = gen.LayerSpec("mx_d", M=1, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=91)
+    se = gen.LayerSpec("mx_e", M=1, K=512, N=2048, k=8, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=92)
+    Pd, Pe = _random_factor_layer(sd)[1], _random_factor_layer(se)[1]
+    plan = [(1, Pd if i % 3 else Pe) for i in range(18)] + [(300, Pd), (300, Pe), (300, Pd)] + \
+           [(2, Pe if i % 4 else Pd) for i in range(20)] + [(9, Pd)]
+    Xs, Ys = [], []
+    for i, (M, P) in enumerate(plan):
+        spec = sd if P is Pd else se
+        Xs.append(_t(gen.make_activations(spec, M=M)) + 0.0625 * i)
+        Ys.append(torch.full((M, spec.N), float("nan"), dtype=torch.float32, device=DEV))
+    calls = L.make_calls([(x, P, y) for x, (_, P), y in zip(Xs, plan, Ys)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    for _ in range(2):                                  # twice: the counters and slots must be left clean
+        L.linear_batched(calls, ws)
+    torch.cuda.synchronize()
+    assert L.poll_status(ws) == 0
+    ws1 = torch.zeros(max(L.workspace_bytes(300, sp.K, sp.N, sp.k) for sp in (sd, se)), dtype=torch.uint8, device=DEV)
+    for x, (M, P), y in zip(Xs, plan, Ys):
+        assert torch.equal(L.linear(x, P, ws1), y), M
+    Pd.release()
+    Pe.release()
+
+
 @pytest.mark.parametrize("M", [1, 16])
 def test_linear_decode_full_size(M):
     spec = gen.config_decode(M)
