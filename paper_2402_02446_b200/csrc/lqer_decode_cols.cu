@@ -38,6 +38,8 @@ constexpr int kMaxM = 4;
 constexpr int kCg = 4;            // column groups (of 8 columns) per round: one column per lane
 constexpr int kSets = 4;          // slabs a warp keeps in flight
 constexpr int kHoldMax = 2;       // rounds whose sums share one barrier and one pass through shared memory, at most
+constexpr int kLocalTMinCtas = 24; // ... if the layer has at least this many CTAs (launches of few layers)
+constexpr int kLocalTUnits = 256; // up to this many (K block, 32 rank columns) units every CTA computes T for itself
 constexpr int kTRanges = 16;      // CTAs of a layer that share the work of T = X_q A_q (ranges of K), at most
 
 constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
@@ -50,7 +52,8 @@ struct Layer {
   size_t off_w, off_b, off_a;   // sections of the packed buffer
   int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
   int cta_begin, ctas;          // this layer's CTAs in the launch, in proportion to its weight bytes
-  int t_ranges;                 // the first t_ranges of them compute T, a range of K each
+  int a_stage_bytes;            // shared memory for a copy of A_q (every CTA computes all of T from it), or 0
+  int t_ranges;                 // the first t_ranges of them compute T, a range of K each; 0: every CTA computes all of T itself
   const uint8_t* pre;           // X_q and T_q computed ahead (decode_pre_kernel), or null: this launch computes them
   double* tslot;                // [t_ranges][M][k_pad] partial sums of T (workspace scratch)
   int* tcount;                  // arrivals, departures: zero between calls
@@ -144,7 +147,7 @@ __device__ __forceinline__ void quantize_x_rows(const float* X, int M, int K, in
 // an exact integer dot product (dp4a) of the mantissas, scaled in fp64.  The fp64 sums are exact too unless the block
 // exponents of one row spread over more than about 30 binades, and the order of the additions is fixed in any case.
 // Leaves tsub[t_subsets(k_pad)][kMaxM][k_pad]; the caller adds the subsets in order after a barrier.
-template <int MT, int UNROLL>
+template <int MT, int UNROLL, bool STAGED>
 __device__ __forceinline__ void t_partial(const uint8_t* asec, int K, int K64, int k_pad, int kb_lo, int kb_hi, int M,
                                           const Formats& f, const uint8_t* xm, const float* xsc, double* tsub) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -165,8 +168,10 @@ __device__ __forceinline__ void t_partial(const uint8_t* asec, int K, int K64, i
       for (int r = 0; r < MT; ++r) tacc[r] = 0.0;
 #pragma unroll UNROLL
       for (int kb = kb_lo + sb; kb < kb_hi; kb += subsets) {
-        const uint4 a = __ldg(reinterpret_cast<const uint4*>(asec + ((size_t)kb * k_pad + jc) * 16));
-        const double sa = pow2d((int)__ldg(a_exp + (size_t)kb * k_pad + jc) + bias);
+        // `asec` is the A_q section in global memory, or (STAGED) a copy of it in shared memory
+        const uint4 a = STAGED ? *reinterpret_cast<const uint4*>(asec + ((size_t)kb * k_pad + jc) * 16)
+                               : __ldg(reinterpret_cast<const uint4*>(asec + ((size_t)kb * k_pad + jc) * 16));
+        const double sa = pow2d((int)(STAGED ? a_exp[(size_t)kb * k_pad + jc] : __ldg(a_exp + (size_t)kb * k_pad + jc)) + bias);
 #pragma unroll
         for (int r = 0; r < MT; ++r) {
           if (r < M) {
@@ -243,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_pre_kernel(const __grid_co
   for (int i = tid; i < (int)pre_t_bytes(c.k_pad) / 4; i += kThreads) reinterpret_cast<uint32_t*>(tqs)[i] = 0u;
   __syncthreads();
   if (c.k_pad > 0) {
-    t_partial<MT, 8>(c.asec, c.K, c.K64, c.k_pad, 0, c.K / 16, M, c.f, xm, xsc, tsub);   // the whole of K: many loads in flight
+    t_partial<MT, 8, false>(c.asec, c.K, c.K64, c.k_pad, 0, c.K / 16, M, c.f, xm, xsc, tsub);   // the whole of K: many loads in flight
     __syncthreads();
     const int subsets = t_subsets(c.k_pad), total = M * c.k_pad;
     for (int base = 0; base < total; base += kThreads) {
@@ -281,6 +286,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   int* wait_ok = reinterpret_cast<int*>(tsub);                       // reused once T's partial sums have left: outcome of the wait
   float* tqs = reinterpret_cast<float*>(tsub + (size_t)kMaxM * ly.k_pad * t_subsets(ly.k_pad));   // [M][k_pad / 16]
   int8_t* tq8 = reinterpret_cast<int8_t*>(tqs + kMaxM * 16);        // [M][k_pad]
+  uint8_t* a_stage = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(tq8) + (size_t)kMaxM * (ly.k_pad > 0 ? ly.k_pad : 16) + 15) & ~(uintptr_t)15);   // a copy of A_q
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = ly.ctas, cta = (int)blockIdx.x - ly.cta_begin;
@@ -343,10 +350,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   fetch_rank(rank_w, rank_e, cg_lo);
   const int KBr = ly.K / 16;
   const bool pre = ly.pre != nullptr;
-  const bool t_worker = !pre && ly.k_pad > 0 && cta < ly.t_ranges;
-  const int kb_lo = t_worker ? cta * KBr / ly.t_ranges : 0;          // this CTA's share of K for T
-  const int kb_hi = t_worker ? (cta + 1) * KBr / ly.t_ranges : 0;
-  if (t_worker) {                                  // this CTA's share of A_q: towards L2 while X is quantised
+  const bool t_local = !pre && ly.k_pad > 0 && ly.t_ranges == 0;     // a small projection: cheaper to repeat than to exchange
+  const bool t_worker = !pre && ly.k_pad > 0 && (t_local || cta < ly.t_ranges);
+  const int kb_lo = t_worker && !t_local ? cta * KBr / ly.t_ranges : 0;          // this CTA's share of K for T
+  const int kb_hi = t_local ? KBr : t_worker ? (cta + 1) * KBr / ly.t_ranges : 0;
+  const bool a_staged = t_local && ly.a_stage_bytes >= KBr * ly.k_pad * 17;
+  if (a_staged) {                                  // all of A_q into shared memory: on its way while the kernel before drains
+    const int bytes = KBr * ly.k_pad * 17;         // mantissas, then exponents: one contiguous range
+    for (int o = tid * 16; o < bytes; o += kThreads * 16)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(a_stage + o)), "l"(asec + o) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  } else if (t_worker) {                           // this CTA's share of A_q: towards L2 while X is quantised
     const uint8_t* gm = asec + (size_t)kb_lo * ly.k_pad * 16;
     const uint8_t* ge = asec + (size_t)KBr * ly.k_pad * 16 + (size_t)kb_lo * ly.k_pad;
     const int mant = (kb_hi - kb_lo) * ly.k_pad * 16, ex = (kb_hi - kb_lo) * ly.k_pad;
@@ -376,17 +390,36 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   // ---- this CTA's share of T = X_q A_q
   if (t_worker) {
     const int subsets = t_subsets(ly.k_pad);
-    t_partial<MT, 4>(asec, ly.K, ly.K64, ly.k_pad, kb_lo, kb_hi, M, fmt, xm, xsc, tsub);
-    __syncthreads();
-    for (int idx = tid; idx < M * ly.k_pad; idx += kThreads) {
-      const int row = idx / ly.k_pad, col = idx % ly.k_pad;
-      double v = 0.0;
-      for (int q = 0; q < subsets; ++q) v += tsub[((size_t)q * kMaxM + row) * ly.k_pad + col];
-      ly.tslot[((size_t)cta * M + row) * ly.k_pad + col] = v;
+    if (a_staged) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncthreads();
+      t_partial<MT, 4, true>(a_stage, ly.K, ly.K64, ly.k_pad, kb_lo, kb_hi, M, fmt, xm, xsc, tsub);
+    } else {
+      t_partial<MT, 4, false>(asec, ly.K, ly.K64, ly.k_pad, kb_lo, kb_hi, M, fmt, xm, xsc, tsub);
     }
     __syncthreads();
-    if (tid == 0) {                              // this range of T is published; waited for before the first rank part
-      __threadfence();                           // the slot (ordered before by the barrier) before the count
+    if (t_local) {                                 // all of T is here: quantise it
+      const int total = M * ly.k_pad;
+      for (int base = 0; base < total; base += kThreads) {
+        const int idx = base + tid;
+        const bool valid = idx < total;
+        const int row = valid ? idx / ly.k_pad : 0, col = valid ? idx % ly.k_pad : 0;
+        double tv = 0.0;
+        if (valid)
+          for (int q = 0; q < subsets; ++q) tv += tsub[((size_t)q * kMaxM + row) * ly.k_pad + col];
+        store_tq(tv, valid, row, col, ly.k_pad, fmt, tq8, tqs);
+      }
+    } else {
+      for (int idx = tid; idx < M * ly.k_pad; idx += kThreads) {
+        const int row = idx / ly.k_pad, col = idx % ly.k_pad;
+        double v = 0.0;
+        for (int q = 0; q < subsets; ++q) v += tsub[((size_t)q * kMaxM + row) * ly.k_pad + col];
+        ly.tslot[((size_t)cta * M + row) * ly.k_pad + col] = v;
+      }
+    }
+    __syncthreads();
+    if (!t_local && tid == 0) {                    // this range of T is published; waited for before the first rank part
+      __threadfence();                             // the slot (ordered before by the barrier) before the count
       atomicAdd(ly.tcount, 1);
     }
   }
@@ -428,7 +461,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       ly.tcount[1] = 0;
     }
   };
-  bool tq_built = pre;
+  bool tq_built = pre || t_local;
   constexpr int kHold = MT == 1 ? kHoldMax : 1;  // rounds per barrier (their sums wait in registers; four were no faster)
   constexpr int kHeld = kHold > 1 ? kHold - 1 : 1;
   int meet_no = 0, n_held = 0;
@@ -680,8 +713,13 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     ly.n_cg = m.N / 8;
     int ranges = ctas[g] < kTRanges ? ctas[g] : kTRanges;
     if (ranges > m.K / 16) ranges = m.K / 16;
+    // a projection of few (K block, 32 rank columns) units costs a CTA less than the exchange of partial sums would,
+    // when the layer has so many CTAs that each streams little else
+    if ((long long)(m.K / 16) * ((m.k_pad + 31) / 32) <= kLocalTUnits && ctas[g] >= kLocalTMinCtas) ranges = 0;
     ly.t_ranges = ranges;
     ly.pre = pres != nullptr ? pres[g] : nullptr;
+    const size_t a_need = (size_t)(m.K / 16) * m.k_pad * 17 + 16;
+    ly.a_stage_bytes = (ranges == 0 && ly.pre == nullptr && m.k_pad > 0 && cols_smem_bytes(m, M) + a_need <= 200 * 1024) ? (int)a_need : 0;
     ly.tslot = reinterpret_cast<double*>(wsb + slot_off);
     ly.tcount = reinterpret_cast<int*>(wsb + kStatusBytes) + 2 * (g + (set != 0 ? kMaxGroup : 0));
     if (i < n) slot_off += decode_cols_slot_bytes(m);
@@ -690,7 +728,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     ly.ctas = ctas[g];
     if (i < n) {
       begin += ctas[g];
-      const size_t need = cols_smem_bytes(m, M);
+      const size_t need = cols_smem_bytes(m, M) + ly.a_stage_bytes;
       if (need > smem) smem = need;
     }
   }
