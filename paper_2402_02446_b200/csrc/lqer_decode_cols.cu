@@ -4,12 +4,12 @@
 //     Y[M,N] = X_q W_q + q(X_q A_q) B_q
 //
 // With so few tokens a tensor-core MMA would spend 16 rows of work on at most 4, and a split of K
-// across CTAs would end in a round trip through global memory (slots, a fence, an arrival
-// counter) that costs more than streaming the weights.  So here a CTA owns output columns and
+// across CTAs would end in cross-CTA partial sums of Y.  So here a CTA owns output columns and
 // the whole contraction for them: groups of 8 columns are dealt out to the CTAs in contiguous
-// ranges, four groups per round; within a round warp w takes the slabs (64 K) w, w + 16, ... of
-// those groups, and the 16 warps' sums meet once in shared memory and are added in warp order.
-// Y is written once, by one thread per element, with no global synchronisation.
+// ranges, four groups (32 columns) per round; within a round warp w takes the slabs (64 K) w,
+// w + 16, ... of those columns, and the 16 warps' sums meet in shared memory and are added in warp
+// order (at one token two rounds share a barrier: the first keeps its sums in registers).  Y is
+// written once, by one thread per element.
 //
 // A lane of a warp owns one of the round's 32 columns and takes a whole slab of it at a time: the
 // four 16-blocks of the slab as two 16-byte loads plus the four exponent bytes as one word.  Per
@@ -19,14 +19,21 @@
 // 2^(e_x + e_w) in fp32 and accumulated per token.  The loads run four slabs ahead; they depend on
 // no earlier kernel and are issued before griddepcontrol.wait.
 //
-// T = X_q A_q is needed by every CTA of a layer, but only after the first round's W_q part.  Up to 16
-// CTAs of the layer take a range of K each (exact int8 tensor-core MMA per 16-block on the X
-// mantissas already in shared memory, scaled and summed in fp64 in a fixed order), leave their
-// partial T in a scratch slot of the workspace and count themselves in; every CTA streams its
-// first round of weights, then waits (bounded) for the count, adds the slots in range order and
-// quantises T.  All CTAs of a launch are resident together (at most one per SM), so the count is
-// reached while the weights stream; a second counter lets the last CTA to have read the slots zero
-// both for the next call.
+// X_q and T_q = q(X_q A_q) (exact dp4a block products, scaled and summed in fp64 in a fixed order)
+// reach a CTA in one of three ways:
+//  - computed ahead by decode_pre_kernel for a whole stretch of independent calls and copied into
+//    shared memory (the batched entry point, more than one launch);
+//  - a small projection in a launch of few layers: every CTA quantises X and computes all of T
+//    from a copy of A_q that cp.async stages in shared memory while the kernel before drains;
+//  - otherwise up to 16 CTAs of the layer take a range of K each, leave their partial T in a
+//    scratch slot of the workspace and count themselves in; every CTA streams its first round of
+//    weights, then waits (bounded) for the count, adds the slots in range order and quantises T.
+//    All CTAs of a launch are resident together (at most one per SM), so the count is reached
+//    while the weights stream; a second counter lets the last CTA to have read the slots zero
+//    both for the next call.
+//
+// Launches of one batched call that follow one another share no buffer and need not wait for one
+// another (ChainOrder): a launch fills the SMs as the one before leaves them.
 #include "lqer_common.cuh"
 
 namespace lqer {
@@ -51,7 +58,7 @@ struct Layer {
   const uint8_t* packed;
   size_t off_w, off_b, off_a;   // sections of the packed buffer
   int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
-  int cta_begin, ctas;          // this layer's CTAs in the launch, in proportion to its weight bytes
+  int cta_begin, ctas;          // this layer's CTAs in the launch (dealt out by a time model)
   int a_stage_bytes;            // shared memory for a copy of A_q (every CTA computes all of T from it), or 0
   int t_ranges;                 // the first t_ranges of them compute T, a range of K each; 0: every CTA computes all of T itself
   const uint8_t* pre;           // X_q and T_q computed ahead (decode_pre_kernel), or null: this launch computes them
