@@ -283,18 +283,87 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
   const bool own_counters = (long long)row_tiles * n <= kPrologueRowTiles;
   size_t off = head;
   for (int g = 0; g < n; ++g) {
-    const PackedMeta& m = metas[g];
-    uint8_t* xcat = wsb + off;
-    off += group_slice_bytes(m, M);
-    const float* X = calls[g].X;
-    int* counters = reinterpret_cast<int*>(wsb + count_base) + (own_counters ? (size_t)g * row_tiles * 2 : 0);
-    const int order = !own_counters ? kChainAlone : g == 0 ? kChainFirst : kChainLater;
-    cudaError_t err = prologue_tc_fits(m, M, X, false)
-                          ? launch_prologue_tc(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
-                                               reinterpret_cast<double*>(xcat + xcat_bytes(m, M)), counters, order, s)
-                          : launch_prologue(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
-    if (err != cudaSuccess) return LQER_ERR_CUDA;
-    xcats[g] = xcat; packed[g] = calls[g].packed; Ys[g] = calls[g].Y;
+    xcats[g] = wsb + off;
+    off += group_slice_bytes(metas[g], M);
+    packed[g] = calls[g].packed; Ys[g] = calls[g].Y;
+  }
+  // One launch for the prologues of all layers, if every one takes the tensor-core prologue with the same rank padding:
+  // a CTA then carries a whole row tile of a layer, or a long K range of it, instead of a ninth.
+  bool together = own_counters && n > 1;
+  for (int g = 0; g < n && together; ++g)
+    together = prologue_tc_fits(metas[g], M, calls[g].X, false) && metas[g].k_pad == metas[0].k_pad;
+  if (together) {
+    // Layers whose K is so long that the CTAs of the whole group would carry unequal work get a launch of their own
+    // (as many K ranges as fit the SMs); the launches share no buffer, so a later one overlaps the tail of the one before.
+    bool alone[8] = {false, false, false, false, false, false, false, false};
+    int splits[8];
+    const long long row_tiles_ll = row_tiles;
+    for (;;) {
+      PackedMeta sub[8];
+      int idx[8], ns = 0;
+      for (int g = 0; g < n; ++g)
+        if (!alone[g]) { sub[ns] = metas[g]; idx[ns++] = g; }
+      if (ns == 0) break;
+      int sp[8];
+      const bool squeezed = prologue_tc_group_splits(sub, ns, M, kPrologueMaxCtas, sp);
+      long long total = 0;
+      double longest = 0.0;
+      int worst = 0;
+      for (int q = 0; q < ns; ++q) {
+        const int panels = (sub[q].K64 + 127) / 128;
+        total += row_tiles_ll * panels;
+        const double len = (double)panels / sp[q];
+        if (len > longest) { longest = len; worst = q; }
+      }
+      for (int q = 0; q < ns; ++q) splits[idx[q]] = sp[q];
+      if (ns == 1 || !squeezed || longest <= 1.35 * (double)total / kPrologueMaxCtas) break;
+      alone[idx[worst]] = true;
+    }
+    const float* Xs[8];
+    const void* pk[8];
+    void* xc[8];
+    double* parts[8];
+    int* counts[8];
+    PackedMeta ms[8];
+    int sp[8];
+    int launches = 0, planned = 0;
+    for (int g = 0, rest = 0; g < n; ++g) {
+      if (alone[g]) ++planned;
+      else if (rest++ == 0) ++planned;
+    }
+    for (int pass = 0; pass < 1 + n; ++pass) {                  // pass 0: the layers that stay together; then each loner
+      int cnt = 0;
+      for (int g = 0; g < n; ++g) {
+        const bool take = pass == 0 ? !alone[g] : (alone[g] && g == pass - 1);
+        if (!take) continue;
+        Xs[cnt] = calls[g].X;
+        pk[cnt] = packed[g];
+        xc[cnt] = const_cast<void*>(xcats[g]);
+        parts[cnt] = reinterpret_cast<double*>(static_cast<uint8_t*>(xc[cnt]) + xcat_bytes(metas[g], M));
+        counts[cnt] = reinterpret_cast<int*>(wsb + count_base) + (size_t)g * row_tiles * 2;
+        ms[cnt] = metas[g];
+        sp[cnt] = pass == 0 ? splits[g] : prologue_tc_splits(metas[g], M);
+        ++cnt;
+      }
+      if (cnt == 0) continue;
+      const int order = planned == 1 ? kChainAlone : launches == 0 ? kChainFirst : kChainLater;
+      if (launch_prologue_tc_group(Xs, M, ms, pk, xc, parts, counts, sp, cnt, nullptr, nullptr, dst, order, s) != cudaSuccess)
+        return LQER_ERR_CUDA;
+      ++launches;
+    }
+  } else {
+    for (int g = 0; g < n; ++g) {
+      const PackedMeta& m = metas[g];
+      uint8_t* xcat = static_cast<uint8_t*>(const_cast<void*>(xcats[g]));
+      const float* X = calls[g].X;
+      int* counters = reinterpret_cast<int*>(wsb + count_base) + (own_counters ? (size_t)g * row_tiles * 2 : 0);
+      const int order = !own_counters ? kChainAlone : g == 0 ? kChainFirst : kChainLater;
+      cudaError_t err = prologue_tc_fits(m, M, X, false)
+                            ? launch_prologue_tc(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
+                                                 reinterpret_cast<double*>(xcat + xcat_bytes(m, M)), counters, order, s)
+                            : launch_prologue(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
+      if (err != cudaSuccess) return LQER_ERR_CUDA;
+    }
   }
   return launch_gemm_tc2_group(xcats, packed, Ys, metas, n, M, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }

@@ -268,6 +268,14 @@ enum ChainOrder { kChainAlone = 0, kChainFirst = 1, kChainLater = 2 };
 cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                int order, cudaStream_t s);
+// The same for up to 8 layers with one M, one k_pad and one set of formats in ONE launch (a CTA per row tile and K range
+// of a layer, found by its index); prologue_tc_group_splits picks the K ranges per row tile so that the CTAs carry
+// about equal work and stay within one per SM.
+bool prologue_tc_group_splits(const PackedMeta* metas, int n, int M, int max_ctas, int* splits);
+cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const PackedMeta* metas, const void* const* packed,
+                                     void* const* xcats, double* const* partials, int* const* counters,
+                                     const int* splits, int n, int8_t* Tm, uint8_t* Te, DeviceStatus* st, int order,
+                                     cudaStream_t s);
 cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                              cudaStream_t s);
 cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,

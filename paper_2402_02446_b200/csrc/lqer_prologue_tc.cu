@@ -82,6 +82,18 @@ struct Params {
   size_t ldx;               // columns of Xcat
 };
 
+// Up to kMaxLayers independent layers with one M, one rank padding and one set of formats may share a launch: a
+// CTA finds its layer by its index (cta_begin) and then works as in a launch of that layer alone.
+constexpr int kMaxLayers = 8;
+struct GroupParams {
+  Params L[kMaxLayers];
+  int cta_begin[kMaxLayers];
+  int n;
+};
+struct TensorMaps {
+  CUtensorMap m[kMaxLayers];   // X of each layer: fp32 [M, K], box 64 x 128
+};
+
 // int8 x int8 -> int32, both operands K-major, M = m, N = n.
 __host__ __device__ constexpr uint32_t make_idesc_i8(int m, int n) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
@@ -129,8 +141,16 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 template <int KP>
-__global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
+__global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __grid_constant__ TensorMaps tmaps,
+                                                                     const __grid_constant__ GroupParams gp) {
   using C = Cfg<KP>;
+  int layer = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxLayers; ++i)
+    if (i < gp.n && (int)blockIdx.x >= gp.cta_begin[i]) layer = i;
+  const Params& p = gp.L[layer];
+  const CUtensorMap* const tmap_x = &tmaps.m[layer];
+  const int bid = (int)blockIdx.x - gp.cta_begin[layer];          // index within the layer's CTAs
   constexpr int SW = C::SCALER_WARPS, QW = C::QUANT_WARPS, CPW = C::CPW, QUADS = C::QUADS;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -155,7 +175,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   auto slot_empty = [&](int s) { return bar0 + 8u * (2 * RAW_SLOTS + 2 * X_SLOTS + 2 * PANELS + MAX_TMEM_SLOTS + s); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int row_tile = blockIdx.x / p.splits, split = blockIdx.x % p.splits;
+  const int row_tile = bid / p.splits, split = bid % p.splits;
   const int row0 = row_tile * ROWS;
   const int pan_lo = (int)((long long)split * p.panels / p.splits);
   const int pan_hi = (int)((long long)(split + 1) * p.panels / p.splits);
@@ -250,7 +270,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
       }
     }
     // partial sums of this CTA's K range -> global scratch
-    double* dst = p.partials + ((size_t)blockIdx.x * ROWS + row) * KP + h * CPW;
+    double* dst = p.partials + ((size_t)bid * ROWS + row) * KP + h * CPW;
 #pragma unroll
     for (int i = 0; i < CPW; i += 2) *reinterpret_cast<double2*>(dst + i) = make_double2(acc[i], acc[i + 1]);
   } else if (warp < WORK_WARPS) {
@@ -370,7 +390,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
         const int rs = s % RAW_SLOTS;
         if (!parked_wait(raw_empty(rs), ((s / RAW_SLOTS) & 1) ^ 1, abort_flag)) break;
         mbar_expect_tx(raw_full(rs), RAW_BYTES);       // rows and columns outside X arrive as zeros
-        tma_load_2d(smem_u32(raw_base + rs * RAW_BYTES), &tmap_x, (pan_lo * 2 + s) * STAGE_COLS, row0, raw_full(rs));
+        tma_load_2d(smem_u32(raw_base + rs * RAW_BYTES), tmap_x, (pan_lo * 2 + s) * STAGE_COLS, row0, raw_full(rs));
       }
     }
   }
@@ -462,7 +482,7 @@ static EncodeTiledFn encode_fn() {
 }
 
 template <int KP>
-static cudaError_t launch_kp(const CUtensorMap& tmap, const Params& p, int ctas, cudaStream_t s) {
+static cudaError_t launch_kp(const TensorMaps& tmaps, const GroupParams& gp, int ctas, cudaStream_t s) {
   using C = Cfg<KP>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -481,7 +501,7 @@ static cudaError_t launch_kp(const CUtensorMap& tmap, const Params& p, int ctas,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   LaunchScope scope(kFamPrologue, s);
-  return cudaLaunchKernelEx(&cfg, prologue_tc_kernel<KP>, tmap, p);
+  return cudaLaunchKernelEx(&cfg, prologue_tc_kernel<KP>, tmaps, gp);
 }
 
 }  // namespace ptc
@@ -493,40 +513,98 @@ bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch
   return any_batch || M >= 1024;
 }
 
-cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
-                               int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
-                               int order, cudaStream_t s) {
+// K ranges per row tile for each of n layers that share a launch: about as many panels (128 columns of X) per CTA
+// everywhere, at most max_ctas CTAs in all (one per SM: the CTAs of a row tile wait for one another).  Returns whether
+// ranges had to be taken away to stay within max_ctas (the work per CTA may then be unequal).
+bool prologue_tc_group_splits(const PackedMeta* metas, int n, int M, int max_ctas, int* splits) {
+  const int row_tiles = (M + 127) / 128;
+  long long total = 0;
+  int panels[ptc::kMaxLayers];
+  for (int g = 0; g < n; ++g) {
+    panels[g] = (metas[g].K64 + 127) / 128;
+    total += (long long)row_tiles * panels[g];
+  }
+  const double per = (double)total / max_ctas;
+  int ctas = 0;
+  for (int g = 0; g < n; ++g) {
+    int sp = (int)((double)panels[g] / per + 0.5);
+    const int cap = prologue_tc_splits(metas[g], M);              // what the scratch is sized for
+    if (sp > cap) sp = cap;
+    if (sp > panels[g]) sp = panels[g];
+    if (sp < 1) sp = 1;
+    splits[g] = sp;
+    ctas += row_tiles * sp;
+  }
+  bool squeezed = false;
+  while (ctas > max_ctas) {                                       // take a range away where the ranges are shortest
+    squeezed = true;
+    int best = -1;
+    double shortest = 0.0;
+    for (int g = 0; g < n; ++g) {
+      const double len = (double)panels[g] / splits[g];
+      if (splits[g] > 1 && (best < 0 || len < shortest)) { best = g; shortest = len; }
+    }
+    if (best < 0) break;
+    --splits[best];
+    ctas -= row_tiles;
+  }
+  return squeezed;
+}
+
+// n layers (one M, one k_pad, one set of formats) in ONE launch.  splits[g] K ranges per row tile of layer g; the
+// caller sees to it that the CTAs (row tiles x splits, summed) are at most one per SM.  Tm / Te: for n == 1 only.
+cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const PackedMeta* metas, const void* const* packed,
+                                     void* const* xcats, double* const* partials, int* const* counters,
+                                     const int* splits, int n, int8_t* Tm, uint8_t* Te, DeviceStatus* st, int order,
+                                     cudaStream_t s) {
   using namespace ptc;
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
-  CUtensorMap tmap;
-  const cuuint64_t dims[2] = {(cuuint64_t)m.K, (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)m.K * 4};
-  const cuuint32_t box[2] = {STAGE_COLS, ROWS};
-  const cuuint32_t estr[2] = {1, 1};
-  if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorInvalidValue;
-  Params p;
-  p.asec = static_cast<const uint8_t*>(packed) + m.off_a;
-  p.xcat = static_cast<uint16_t*>(xcat);
-  p.Tm = Tm; p.Te = Te; p.status = st;
-  p.partials = partials; p.counters = counters;
-  p.M = M; p.K = m.K; p.K64 = m.K64;
-  p.kblocks = m.K / 16;
-  p.panels = (m.K64 + 127) / 128;
-  p.splits = prologue_tc_splits(m, M);
-  p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
-  p.order = order;
-  p.ldx = xcat_cols(m);
-  const int ctas = ((M + ROWS - 1) / ROWS) * p.splits;
-  switch (m.k_pad) {
-    case 16: return launch_kp<16>(tmap, p, ctas, s);
-    case 32: return launch_kp<32>(tmap, p, ctas, s);
-    case 64: return launch_kp<64>(tmap, p, ctas, s);
+  if (n < 1 || n > kMaxLayers) return cudaErrorInvalidValue;
+  TensorMaps tmaps;
+  GroupParams gp;
+  gp.n = n;
+  int begin = 0;
+  for (int i = 0; i < kMaxLayers; ++i) {
+    const int g = i < n ? i : 0;
+    const PackedMeta& m = metas[g];
+    if (m.k_pad != metas[0].k_pad) return cudaErrorInvalidValue;
+    const cuuint64_t dims[2] = {(cuuint64_t)m.K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)m.K * 4};
+    const cuuint32_t box[2] = {STAGE_COLS, ROWS};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmaps.m[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(Xs[g]), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    Params& p = gp.L[i];
+    p.asec = static_cast<const uint8_t*>(packed[g]) + m.off_a;
+    p.xcat = static_cast<uint16_t*>(xcats[g]);
+    p.Tm = n == 1 ? Tm : nullptr; p.Te = n == 1 ? Te : nullptr; p.status = st;
+    p.partials = partials[g]; p.counters = counters[g];
+    p.M = M; p.K = m.K; p.K64 = m.K64;
+    p.kblocks = m.K / 16;
+    p.panels = (m.K64 + 127) / 128;
+    p.splits = splits[g];
+    p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
+    p.order = order;
+    p.ldx = xcat_cols(m);
+    gp.cta_begin[i] = begin;
+    if (i < n) begin += ((M + ROWS - 1) / ROWS) * p.splits;
+  }
+  switch (metas[0].k_pad) {
+    case 16: return launch_kp<16>(tmaps, gp, begin, s);
+    case 32: return launch_kp<32>(tmaps, gp, begin, s);
+    case 64: return launch_kp<64>(tmaps, gp, begin, s);
     default: return cudaErrorInvalidValue;
   }
+}
+
+cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
+                               int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
+                               int order, cudaStream_t s) {
+  const int splits = prologue_tc_splits(m, M);
+  return launch_prologue_tc_group(&X, M, &m, &packed, &xcat, &partials, &counters, &splits, 1, Tm, Te, st, order, s);
 }
 
 }  // namespace lqer
