@@ -515,6 +515,40 @@ def test_batched_prefill_calls_share_gemm_launches():
         Pg.release()
 
 
+def test_batched_prefill_group_with_long_and_short_layers():
+    # four prefill calls with M = 4096 (32 row tiles): two short layers (K = 512) and two long ones (K = 4096).  One
+    # prologue launch for all of them would leave the long layers a whole row tile per CTA and the CTAs unequal work,
+    # so the long layers get launches of their own; T_q and Y must be what single calls give, and within the oracle's
+    # tolerance.
+    M = 4096
+    short = gen.LayerSpec("lg_s", M=M, K=512, N=264, k=32, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=95)
+    long_ = gen.LayerSpec("lg_l", M=M, K=4096, N=136, k=32, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=96)
+    layers = []
+    for i, spec in enumerate([short, long_, short, long_]):
+        sp = gen.LayerSpec(f"{spec.name}{i}", M=M, K=spec.K, N=spec.N, k=spec.k, calib_rows=spec.calib_rows,
+                           outlier_frac=spec.outlier_frac, outlier_scale=spec.outlier_scale, seed=spec.seed + 10 * i)
+        layers.append((sp,) + _random_factor_layer(sp))
+    Xs = [_t(gen.make_activations(sp)) for sp, _, _ in layers]
+    Yb = [torch.full((M, sp.N), float("nan"), dtype=torch.float32, device=DEV) for sp, _, _ in layers]
+    calls = L.make_calls([(x, lay[2], y) for x, lay, y in zip(Xs, layers, Yb)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    launches = L.launch_count()
+    for _ in range(2):
+        L.linear_batched(calls, ws)
+    torch.cuda.synchronize()
+    assert L.poll_status(ws) == 0
+    assert L.launch_count() - launches == 2 * (3 + 1)    # the short layers together, each long one alone, one GEMM launch
+    for x, (sp, P, Pg), yb in zip(Xs, layers, Yb):
+        assert torch.equal(L.linear(x, Pg, ws), yb), sp.name
+    for j in (0, 1):
+        sp, P, Pg = layers[j]
+        rows = np.arange(0, M, 37)
+        ref = olqer.forward(Xs[j].cpu().numpy()[rows], P)
+        assert worst_ratio(Yb[j].cpu().numpy()[rows], ref) <= 1.0, sp.name
+    for _, _, Pg in layers:
+        Pg.release()
+
+
 def test_host_buffer_entry_points_match_device_calls():
     # lqer_linear_host (one layer) and lqer_linear_host_batched (copies and layers pipelined, buffers alternate)
     # against the device entry point on the same inputs; five calls so that every buffer is reused
