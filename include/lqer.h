@@ -42,7 +42,7 @@ typedef enum {
   LQER_ERR_ALIGN = 3,            /* a pointer is not 16-byte aligned */
   LQER_ERR_CONFIG = 4,           /* unsupported lqer_config_t */
   LQER_ERR_BUFFER_TOO_SMALL = 5, /* packed / workspace buffer smaller than required */
-  LQER_ERR_BAD_PACKED = 6,       /* packed buffer unknown to the library or header corrupt */
+  LQER_ERR_BAD_PACKED = 6,       /* not a packed buffer: no valid header at that (256-byte aligned, device) address */
   LQER_ERR_ARCH = 7,             /* current device is not compute capability 10.x */
   LQER_ERR_CUDA = 8,             /* a CUDA runtime / driver call failed */
   LQER_ERR_TIMEOUT = 9,          /* device side: a bounded wait ran out */
@@ -91,6 +91,12 @@ lqer_status_t lqer_packed_bytes(int K, int N, int k, const lqer_config_t* cfg, s
  * of different shapes if it fits the largest. */
 lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
 
+/* Size in bytes (host out) that one call with exactly M rows uses of its workspace on the path the library
+ * picks for it (decode kernels up to 16 rows, prologue + GEMM above): never more than
+ * lqer_workspace_bytes(M_max, ...) for any M_max >= M.  This is the figure lqer_linear_static holds against
+ * LQER_STATIC_SCRATCH_BYTES. */
+lqer_status_t lqer_call_workspace_bytes(int M, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
+
 /* Weight preparation (Section 3.1: W_q = q(W); Section 4.1 formats): quantise W to MXINT4
  * (blocks of 16 along K), A and B to MXINT8 (A: blocks of 16 along K; B: blocks of 16 along
  * the rank, zero-padded to a multiple of 16) on the GPU and write the kernel layout into
@@ -100,7 +106,9 @@ lqer_status_t lqer_prepare_weights(const float* W, const float* A, const float* 
                                    const lqer_config_t* cfg, void* packed, size_t packed_bytes, void* stream);
 
 /* Register a packed buffer that was produced earlier and copied to a new address
- * (save / restore).  Reads the header back from the device: synchronises `stream`. */
+ * (save / restore).  Reads the header back from the device: synchronises `stream`.
+ * Optional: every entry point that takes `packed` does the same on its own the first
+ * time it meets an address it has not seen (one blocking 256-byte read, then cached). */
 lqer_status_t lqer_attach_packed(const void* packed, size_t packed_bytes, void* stream);
 
 /* Forget a packed buffer (call before freeing it).  Host only. */
@@ -147,9 +155,12 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * LQER_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds
  * that much memory until the process exits.  The call itself allocates and frees nothing.
  *  - X, Y, packed, stream: as for lqer_linear_stream (device pointers, caller owned).
- *  - Limit: lqer_workspace_bytes(M, K, N, k) <= LQER_STATIC_SCRATCH_BYTES, otherwise
- *    LQER_ERR_STATIC_SCRATCH is returned and nothing is launched (M = 256 at K = N = 4096, rank 32 needs
- *    about 4.2 MB; M = 16 fits for every supported K).
+ *  - Limit: what this call itself needs on the path it takes must fit LQER_STATIC_SCRATCH_BYTES, otherwise
+ *    LQER_ERR_STATIC_SCRATCH is returned and nothing is launched.  The need is smaller than
+ *    lqer_workspace_bytes(M, ...), which covers every batch up to M: M <= 16 (the decode kernels: at most
+ *    2.8 MB) fits for every supported shape; larger batches need 2 M (K + k) bytes for [X_q | T_q], the
+ *    prologue's partial sums and, up to M = 256, the partial sums of the GEMM's K ranges (up to 7 M N 4
+ *    bytes).  At K = N = 4096, rank 32 that admits M <= 127 and 257 <= M <= 506, and refuses the rest.
  *  - The first call on a device looks up the array's device address (the device must be
  *    current); make that first call before any stream capture begins.
  *  - All calls on a device share the one array and it keeps the previous call's contents; the
@@ -205,11 +216,24 @@ lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void*
 lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_t* device_status);
 
 /* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 decode kernels
- * (column-owner kernel for M <= 4, split-K kernel for M <= 16), 3 tensor-core kernel (one CTA per
- * tile), 4 tensor-core kernel (CTA pair per tile), 5 split-K decode kernel for every M <= 16,
- * 6 as 4 with the tensor-core activation prologue at every batch size (ranks up to 64; by default
- * it serves M >= 1024, and paths 1 and 3 never use it).  Host only, process wide. */
+ * (column-owner kernel for M <= 4, split-K kernel for M <= 16), 3 tensor-core GEMM behind the
+ * activation prologue that runs the projection on int8 mma.sync (at every batch size), 4 tensor-core
+ * GEMM with the prologue chosen as in 0, 5 split-K decode kernel for every M <= 16, 6 as 4 with the
+ * tcgen05 activation prologue at every batch size (ranks up to 64; by default it serves M >= 1024,
+ * and paths 1 and 3 never use it).  Host only, process wide. */
 lqer_status_t lqer_set_path(int path);
+
+/* Test hooks for the device-side error path (host only, process wide; the paper has no counterpart: this is a
+ * property of the library).  Every wait of a kernel on another CTA, warp or copy is bounded; a wait that runs out makes
+ * the kernel give up, write LQER_ERR_TIMEOUT to the status word and return, so the context stays usable.
+ *  - lqer_set_wait_limit_cycles: the bound in SM clock cycles (default 4e9, about two seconds; 1e3 .. 2^40).
+ *  - lqer_inject_stall(family): the next launch of that kernel family (numbering of lqer_kernel_times_t:
+ *    3 activation prologue, 6 tensor-core GEMM pair kernel, 7 decode kernels) is told to expect one arrival
+ *    more than will ever come (3, 7) or has its last stage of operands withheld (6), so that its waits run
+ *    out; no memory is touched that an ordinary launch would not touch.  -1 disarms.  After such a launch
+ *    the outputs are undefined and the workspace needs lqer_workspace_init before its next use. */
+lqer_status_t lqer_set_wait_limit_cycles(long long cycles);
+lqer_status_t lqer_inject_stall(int kernel_family);
 
 /* Number of kernels launched by the library in this process so far (host). */
 unsigned long long lqer_launch_count(void);
@@ -220,8 +244,8 @@ unsigned long long lqer_launch_count(void);
  * when measuring end-to-end time.  lqer_profile_collect waits for the recorded launches,
  * sums launches and elapsed milliseconds per kernel family into *out (host) and forgets them.
  * Families: 0 weight pack, 1 export, 2 stand-alone activation quantiser, 3 activation prologue,
- * 4 CUDA-core reference GEMM, 5 tensor-core GEMM (one CTA per tile), 6 tensor-core GEMM (CTA
- * pair per tile), 7 decode kernel. */
+ * 4 CUDA-core reference GEMM, 5 factor preparation (calibration statistics, subspace iteration),
+ * 6 tensor-core GEMM (CTA pair per tile), 7 decode kernels. */
 #define LQER_NUM_KERNEL_FAMILIES 8
 typedef struct {
   unsigned long long launches[LQER_NUM_KERNEL_FAMILIES];

@@ -13,6 +13,9 @@ from .binding import (  # noqa: F401
     default_config,
     packed_bytes,
     workspace_bytes,
+    call_workspace_bytes,
+    set_wait_limit_cycles,
+    inject_stall,
     prepare_weights,
     export_weights,
     quantize_activations,

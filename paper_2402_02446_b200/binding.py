@@ -35,7 +35,7 @@ class Config(C.Structure):
                 ("w_exp_min", C.c_int), ("w_exp_max", C.c_int)]
 
 
-KERNEL_FAMILIES = ["pack", "export", "quantize", "prologue", "gemm_simt", "gemm_tc", "gemm_tc_pair", "decode"]
+KERNEL_FAMILIES = ["pack", "export", "quantize", "prologue", "gemm_simt", "prepare", "gemm_tc_pair", "decode"]
 
 
 class KernelTimes(C.Structure):
@@ -65,6 +65,9 @@ def lib() -> C.CDLL:
             "lqer_default_config": (i, [cfgp]),
             "lqer_packed_bytes": (i, [i, i, i, cfgp, C.POINTER(sz)]),
             "lqer_workspace_bytes": (i, [i, i, i, i, cfgp, C.POINTER(sz)]),
+            "lqer_call_workspace_bytes": (i, [i, i, i, i, cfgp, C.POINTER(sz)]),
+            "lqer_set_wait_limit_cycles": (i, [C.c_longlong]),
+            "lqer_inject_stall": (i, [i]),
             "lqer_prepare_weights": (i, [vp, vp, vp, i, i, i, cfgp, vp, sz, vp]),
             "lqer_attach_packed": (i, [vp, sz, vp]),
             "lqer_release_packed": (i, [vp]),
@@ -129,6 +132,13 @@ def workspace_bytes(M_max: int, K: int, N: int, k: int, cfg: Config | None = Non
     cfg = cfg or default_config()
     out = C.c_size_t()
     _check(lib().lqer_workspace_bytes(M_max, K, N, k, C.byref(cfg), C.byref(out)), "lqer_workspace_bytes")
+    return out.value
+
+
+def call_workspace_bytes(M: int, K: int, N: int, k: int, cfg: Config | None = None) -> int:
+    cfg = cfg or default_config()
+    out = C.c_size_t()
+    _check(lib().lqer_call_workspace_bytes(M, K, N, k, C.byref(cfg), C.byref(out)), "lqer_call_workspace_bytes")
     return out.value
 
 
@@ -294,6 +304,15 @@ def poll_status(ws: torch.Tensor, stream=None) -> int:
 
 def set_path(path: int) -> None:
     _check(lib().lqer_set_path(path), "lqer_set_path")
+
+
+def set_wait_limit_cycles(cycles: int) -> None:
+    _check(lib().lqer_set_wait_limit_cycles(cycles), "lqer_set_wait_limit_cycles")
+
+
+def inject_stall(kernel_family: int) -> None:
+    """Test hook: the next launch of that kernel family waits for something that never comes (-1 disarms)."""
+    _check(lib().lqer_inject_stall(kernel_family), "lqer_inject_stall")
 
 
 def launch_count() -> int:

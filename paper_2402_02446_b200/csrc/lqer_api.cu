@@ -43,6 +43,29 @@ LaunchScope::~LaunchScope() {
 static std::mutex g_mu;
 static std::unordered_map<const void*, PackedMeta> g_registry;
 static std::atomic<int> g_path{0};
+static std::atomic<long long> g_wait_limit{4000000000LL};      // about two seconds of SM clock
+static std::atomic<int> g_stall_family{-1};
+
+long long wait_limit_cycles() { return g_wait_limit.load(std::memory_order_relaxed); }
+
+bool take_stall(int family) {
+  int want = family;
+  return g_stall_family.compare_exchange_strong(want, -1);
+}
+
+int sm_count() {
+  static std::mutex mu;
+  static int count_of[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  std::lock_guard<std::mutex> lock(mu);
+  if (count_of[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    count_of[dev] = n;
+  }
+  return count_of[dev];
+}
 
 // Two packed buffers with the same sections, formats and sizes (their contents may differ).
 static bool same_shape(const PackedMeta& a, const PackedMeta& b) {
@@ -100,12 +123,27 @@ static bool meta_valid(const PackedMeta& m) {
   return std::memcmp(&ref, &m, sizeof(m)) == 0;
 }
 
+// The shape and formats of a packed buffer live in its 256-byte header.  The host keeps a copy per buffer address so
+// that a call costs no device read; a buffer the host has not seen yet (one that was copied to a new address, or
+// loaded from a file) has its header read back from the device once, checked, and remembered.  That first call
+// synchronises with the device (cudaMemcpy); lqer_attach_packed does the same ahead of time.
 static lqer_status_t lookup(const void* packed, PackedMeta& out) {
   if (packed == nullptr) return LQER_ERR_NULL;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    auto it = g_registry.find(packed);
+    if (it != g_registry.end()) { out = it->second; return LQER_OK; }
+  }
+  if ((reinterpret_cast<uintptr_t>(packed) & 255u) != 0) return LQER_ERR_BAD_PACKED;
+  cudaPointerAttributes pa;
+  if (cudaPointerGetAttributes(&pa, packed) != cudaSuccess) { cudaGetLastError(); return LQER_ERR_BAD_PACKED; }
+  if (pa.type != cudaMemoryTypeDevice && pa.type != cudaMemoryTypeManaged) return LQER_ERR_BAD_PACKED;
+  PackedMeta m;
+  if (cudaMemcpy(&m, packed, sizeof(m), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return LQER_ERR_BAD_PACKED; }
+  if (!meta_valid(m)) return LQER_ERR_BAD_PACKED;
   std::lock_guard<std::mutex> lock(g_mu);
-  auto it = g_registry.find(packed);
-  if (it == g_registry.end()) return LQER_ERR_BAD_PACKED;
-  out = it->second;
+  g_registry[packed] = m;
+  out = m;
   return LQER_OK;
 }
 
@@ -130,6 +168,17 @@ static size_t call_bytes(const PackedMeta& m, int M, bool decode) {
   return align_up(persist_bytes(m), 256) +
          (decode ? decode_scratch_bytes(m)
                  : xcat_bytes(m, M) + align_up(prologue_tc_scratch_bytes(m, M), 256) + gemm_splitk_bytes(m, M));
+}
+// The same for a registered packed buffer, on the path lqer_linear_stream takes for M rows right now.
+lqer_status_t call_workspace_bytes(const void* packed, int M, size_t* bytes) {
+  PackedMeta m;
+  lqer_status_t st = lookup(packed, m);
+  if (st != LQER_OK) return st;
+  if (M <= 0 || M > (1 << 24)) return LQER_ERR_SHAPE;
+  const int path = g_path.load();
+  const bool decode = path == 2 || path == 5 || (path == 0 && M <= decode_max_m());
+  *bytes = call_bytes(m, M, decode);
+  return LQER_OK;
 }
 // Bytes that fit every call of up to M_max rows, whichever path it takes.
 static size_t workspace_total(const PackedMeta& m, int M_max) {
@@ -170,13 +219,11 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
                                            reinterpret_cast<int*>(wsb + pcount_offset(m)), kChainAlone, s)
                       : launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
-      err = (path == 1)   ? launch_gemm_simt(xcat, M, m, packed, Y, s)
-            : (path == 4 || path == 0)   // the pair kernel is the faster one at every M above the decode range
-                ? launch_gemm_tc2_splitk(xcat, M, m, packed, Y,
-                                         reinterpret_cast<float*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M) +
-                                                                  align_up(prologue_tc_scratch_bytes(m, M), 256)),
-                                         dst, s)
-                          : launch_gemm_tc(xcat, M, m, packed, Y, dst, s);
+      err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, Y, s)
+                        : launch_gemm_tc2_splitk(xcat, M, m, packed, Y,
+                                                 reinterpret_cast<float*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M) +
+                                                                          align_up(prologue_tc_scratch_bytes(m, M), 256)),
+                                                 dst, s);
   }
   return err == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
@@ -263,6 +310,11 @@ static int decode_stretch(const lqer_call_t* calls, int first, int n_calls, size
   if (bytes != nullptr) *bytes = total;
   return j - first;
 }
+// CTAs a tensor-core prologue launch may have: one per SM (its CTAs wait for one another), within what the scratch is sized for.
+static int prologue_max_ctas() {
+  const int sms = sm_count();
+  return sms > 0 && sms < kPrologueMaxCtas ? sms : kPrologueMaxCtas;
+}
 // n prefill layers with one M: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
 // the tiles of all of them.
 static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace,
@@ -305,7 +357,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
         if (!alone[g]) { sub[ns] = metas[g]; idx[ns++] = g; }
       if (ns == 0) break;
       int sp[8];
-      const bool squeezed = prologue_tc_group_splits(sub, ns, M, kPrologueMaxCtas, sp);
+      const bool squeezed = prologue_tc_group_splits(sub, ns, M, prologue_max_ctas(), sp);
       long long total = 0;
       double longest = 0.0;
       int worst = 0;
@@ -316,7 +368,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
         if (len > longest) { longest = len; worst = q; }
       }
       for (int q = 0; q < ns; ++q) splits[idx[q]] = sp[q];
-      if (ns == 1 || !squeezed || longest <= 1.35 * (double)total / kPrologueMaxCtas) break;
+      if (ns == 1 || !squeezed || longest <= 1.35 * (double)total / prologue_max_ctas()) break;
       alone[idx[worst]] = true;
     }
     const float* Xs[8];
@@ -342,7 +394,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
         parts[cnt] = reinterpret_cast<double*>(static_cast<uint8_t*>(xc[cnt]) + xcat_bytes(metas[g], M));
         counts[cnt] = reinterpret_cast<int*>(wsb + count_base) + (size_t)g * row_tiles * 2;
         ms[cnt] = metas[g];
-        sp[cnt] = pass == 0 ? splits[g] : prologue_tc_splits(metas[g], M);
+        sp[cnt] = pass == 0 ? splits[g] : prologue_tc_splits(metas[g], M, prologue_max_ctas());
         ++cnt;
       }
       if (cnt == 0) continue;
@@ -418,6 +470,18 @@ lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_co
   PackedMeta m;
   fill_meta(m, K, N, k, *cfg);
   *bytes = workspace_total(m, M_max);
+  return LQER_OK;
+}
+
+lqer_status_t lqer_call_workspace_bytes(int M, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes) {
+  if (bytes == nullptr) return LQER_ERR_NULL;
+  lqer_status_t st = check_config(cfg);
+  if (st != LQER_OK) return st;
+  if ((st = check_shape(K, N, k)) != LQER_OK) return st;
+  if (M <= 0 || M > (1 << 24)) return LQER_ERR_SHAPE;
+  PackedMeta m;
+  fill_meta(m, K, N, k, *cfg);
+  *bytes = call_bytes(m, M, M <= decode_max_m());
   return LQER_OK;
 }
 
@@ -810,6 +874,18 @@ lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_
   if (cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LQER_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return LQER_ERR_CUDA;
   *device_status = (h.code >= 0 && h.code <= LQER_ERR_BOUNDS) ? (lqer_status_t)h.code : LQER_ERR_CUDA;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_set_wait_limit_cycles(long long cycles) {
+  if (cycles < 1000 || cycles > (1LL << 40)) return LQER_ERR_CONFIG;
+  g_wait_limit.store(cycles);
+  return LQER_OK;
+}
+
+lqer_status_t lqer_inject_stall(int kernel_family) {
+  if (kernel_family < -1 || kernel_family >= LQER_NUM_KERNEL_FAMILIES) return LQER_ERR_CONFIG;
+  g_stall_family.store(kernel_family);
   return LQER_OK;
 }
 

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "lqer.h"
 
 namespace lqer {
@@ -59,7 +61,7 @@ inline uint32_t meta_checksum(const PackedMeta& m) {
 constexpr int kTCountOffset = 64, kTDoneOffset = 68;
 constexpr int kDecodeMaxCtas = 160;
 constexpr int kPrologueRowTiles = 512;               // an arrival and a departure counter each: batches up to 65536 rows
-constexpr int kPrologueMaxCtas = 148;
+constexpr int kPrologueMaxCtas = 148;               // CTAs of one tensor-core prologue launch the scratch is sized for (launches use min(this, SMs))
 constexpr int kGemmMaxPairs = 74;                    // CTA pairs of the pair GEMM (one per two SMs)
 constexpr int kGemmSplitMaxM = 256;                  // batches up to this many rows (one row tile) may have their K range cut
 constexpr size_t kPersistMaxBytes = 256 + 32768 * 4 + 16 * 256 * 8 + kPrologueRowTiles * 8;
@@ -90,17 +92,23 @@ inline size_t gemm_splitk_bound(const PackedMeta& m, int M_max) {
 // Tensor-core prologue: a CTA owns 128 rows and one of `splits` ranges of K (in panels of 128 columns);
 // each CTA leaves a [128, k_pad] fp64 partial sum; once all CTAs of a row tile have arrived each adds up its share of rows.
 inline bool prologue_tc_rank_ok(const PackedMeta& m) { return m.k > 0 && (m.k_pad == 16 || m.k_pad == 32 || m.k_pad == 64); }
-inline int prologue_tc_splits(const PackedMeta& m, int M) {
+inline int prologue_tc_splits(const PackedMeta& m, int M, int max_ctas = kPrologueMaxCtas) {
   const int row_tiles = (M + 127) / 128, panels = (m.K64 + 127) / 128;
-  int s = kPrologueMaxCtas / row_tiles;
+  int s = max_ctas / row_tiles;
   if (s > panels) s = panels;
   return s < 1 ? 1 : s;
 }
-// Upper bound of prologue_tc_scratch_bytes over every batch of up to M_max rows.
+// Upper bound of prologue_tc_scratch_bytes over every batch of up to M_max rows: the largest number of CTAs any
+// such batch launches (row tiles x K ranges; beyond kPrologueMaxCtas row tiles every row tile is one CTA).
 inline size_t prologue_tc_scratch_bound(const PackedMeta& m, int M_max) {
   if (!prologue_tc_rank_ok(m)) return 0;
-  long long ctas = (long long)((M_max + 127) / 128) * ((m.K64 + 127) / 128);
-  if (ctas > kPrologueMaxCtas) ctas = kPrologueMaxCtas;
+  int rt_max = (M_max + 127) / 128;
+  if (rt_max > kPrologueRowTiles) rt_max = kPrologueRowTiles;
+  long long ctas = 0;
+  for (int rt = 1; rt <= rt_max; ++rt) {
+    const long long c = (long long)rt * prologue_tc_splits(m, rt * 128);
+    if (c > ctas) ctas = c;
+  }
   return (size_t)ctas * 128 * m.k_pad * 8;
 }
 inline size_t prologue_tc_scratch_bytes(const PackedMeta& m, int M) {
@@ -229,11 +237,45 @@ __device__ __forceinline__ void report_error(DeviceStatus* st, int code, int whe
 }
 
 // ----------------------------------------------------------------------------
+// Per-device host state
+// ----------------------------------------------------------------------------
+// Number of SMs of the current device (cached per device; 0 if the query fails).
+int sm_count();
+// Runs `set` the first time it is called with a given device current: kernel attributes such as the
+// dynamic shared-memory limit belong to a device, so a process that drives several GPUs sets them on each.
+class OncePerDevice {
+ public:
+  template <class F>
+  cudaError_t run(F&& set) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu_);
+    if (((done_ >> dev) & 1ull) == 0) {
+      if ((e = set()) != cudaSuccess) return e;
+      done_ |= 1ull << dev;
+    }
+    return cudaSuccess;
+  }
+ private:
+  std::mutex mu_;
+  unsigned long long done_ = 0;
+};
+// Bound, in SM clock cycles, of every device-side wait (lqer_set_wait_limit_cycles; default about two seconds).
+long long wait_limit_cycles();
+// Workspace bytes the call lqer_linear_stream(X, M, packed, ...) needs on the path it would take now.
+lqer_status_t call_workspace_bytes(const void* packed, int M, size_t* bytes);
+// Test hook (lqer_inject_stall): true once for the next launch of `family` after it was armed; that launch then
+// waits for one arrival more than will ever come, so its waits run out and it reports LQER_ERR_TIMEOUT.
+bool take_stall(int family);
+
+// ----------------------------------------------------------------------------
 // Launch wrappers (each returns the cudaError_t of its launches)
 // ----------------------------------------------------------------------------
 // Kernel families, as reported by lqer_profile_collect.
 enum KernelFamily {
-  kFamPack = 0, kFamExport, kFamQuantize, kFamPrologue, kFamGemmSimt, kFamGemmTc, kFamGemmTcPair, kFamDecode,
+  kFamPack = 0, kFamExport, kFamQuantize, kFamPrologue, kFamGemmSimt, kFamPrepare, kFamGemmTcPair, kFamDecode,
   kNumFamilies
 };
 // Brackets the launches of one kernel family: counts them and, while profiling is enabled,
@@ -278,8 +320,6 @@ cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const Packed
                                      cudaStream_t s);
 cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                              cudaStream_t s);
-cudaError_t launch_gemm_tc(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
-                           DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                             DeviceStatus* st, cudaStream_t s);
 // Small batches: the layer's K range cut into gemm_splitk_ranges(m, M) ranges that run as layers of one launch;

@@ -59,6 +59,8 @@ struct Params {
   int n_tiles, k_slabs, r_blocks, U;   // U = units per column tile = k_slabs + rank units
   int total_units;
   int a_bits, lr_bits, exp_min, exp_max;
+  long long wait_limit; // bound of the wait for the other CTAs' contributions to T, in clock cycles
+  int stall;            // test hook: wait for one contribution more than will come
 };
 
 // The order in which a CTA walks its units: memory order, except that the rank units of the
@@ -210,9 +212,9 @@ __device__ __noinline__ void build_tq(const Params& p, Ctx* cx, uint8_t* tq) {
   const int tq_stride = (p.k_pad + 8) * 2;
   if (tid == 0) {                                // bounded wait for the contributions of all CTAs
     const long long t0 = clock64();
-    while (ld_acquire(p.tcount) < G) {
+    while (ld_acquire(p.tcount) < G + p.stall) {
       __nanosleep(64);
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) { cx->flags[0] = 1; break; }
+      if (clock64() - t0 > p.wait_limit) { cx->flags[0] = 1; break; }
     }
   }
   __syncthreads();
@@ -488,18 +490,15 @@ cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void
                           cudaStream_t s, bool force_split_k) {
   using namespace dec;
   if (decode_cols_fits(m, M) && !force_split_k) return launch_decode_cols(X, M, m, packed, Y, workspace, s);
-  static int sm_count = 0;
-  static bool attr_set = false;
   const size_t fixed = (size_t)kPhaseUnits * kXTileBytes + (size_t)kWarps * kDepth * kSlotBytes + sizeof(Ctx) + 256;
-  if (!attr_set) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(fixed + 16 * (256 + 8) * 2 + 128));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static OncePerDevice once;
+  cudaError_t e0 = once.run([fixed] {
+    return cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)(fixed + 16 * (256 + 8) * 2 + 128));
+  });
+  if (e0 != cudaSuccess) return e0;
+  const int sm_count = lqer::sm_count();
+  if (sm_count < 1) return cudaErrorInvalidDevice;
   Params p;
   const uint8_t* base = static_cast<const uint8_t*>(packed);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -516,6 +515,8 @@ cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void
   p.U = m.k_slabs + (m.r_blocks + 1) / 2;
   p.total_units = decode_units(m);
   p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
+  p.wait_limit = wait_limit_cycles();
+  p.stall = take_stall(kFamDecode) ? 1 : 0;
   const int G = decode_ctas(m, sm_count);
   if ((unsigned long long)(p.total_units + 1) * (unsigned long long)(G + 1) >= (1ull << 32)) return cudaErrorInvalidValue;
   const size_t smem = fixed + ((16 * (m.k_pad + 8) * 2 + 127) & ~127);

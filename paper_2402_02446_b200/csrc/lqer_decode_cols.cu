@@ -50,7 +50,6 @@ constexpr int kLocalTUnits = 256; // up to this many (K block, 32 rank columns) 
 constexpr int kTRanges = 16;      // CTAs of a layer that share the work of T = X_q A_q (ranges of K), at most
 
 constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
-constexpr long long kSpinLimitCycles = 4000000000LL;   // about two seconds
 
 struct Layer {
   const float* X;
@@ -61,6 +60,7 @@ struct Layer {
   int cta_begin, ctas;          // this layer's CTAs in the launch (dealt out by a time model)
   int a_stage_bytes;            // shared memory for a copy of A_q (every CTA computes all of T from it), or 0
   int t_ranges;                 // the first t_ranges of them compute T, a range of K each; 0: every CTA computes all of T itself
+  int t_expect;                 // arrivals the CTAs wait for: t_ranges (one more under the stall test hook)
   const uint8_t* pre;           // X_q and T_q computed ahead (decode_pre_kernel), or null: this launch computes them
   double* tslot;                // [t_ranges][M][k_pad] partial sums of T (workspace scratch)
   int* tcount;                  // arrivals, departures: zero between calls
@@ -74,6 +74,7 @@ struct Params {
   DeviceStatus* status;
   int M;
   int a_bits, lr_bits, exp_min, exp_max;
+  long long wait_limit;         // bound of the wait for the other CTAs' partial sums, in clock cycles
 };
 
 struct SlabRegs {
@@ -440,8 +441,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
       for (;;) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ly.tcount) : "memory");
-        if (v >= ly.t_ranges) break;
-        if (clock64() - t0 > kSpinLimitCycles) { seen = 0; break; }
+        if (v >= ly.t_expect) break;
+        if (clock64() - t0 > p.wait_limit) { seen = 0; break; }
         __nanosleep(100);
       }
       if (!seen) report_error(p.status, LQER_ERR_TIMEOUT, 500, blockIdx.x);
@@ -639,12 +640,9 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
                                      size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
                                      cudaStream_t s) {
   using namespace dcol;
-  static int sm_count = 0;
-  static bool one_cta_per_sm = false;
-  if (sm_count == 0) {
-    int dev = 0, sms = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  static OncePerDevice once;
+  static bool one_cta_per_sm = true;               // false if any device could hold two CTAs of the kernel on one SM
+  cudaError_t e0 = once.run([] {
     cudaError_t e = cudaFuncSetAttribute(decode_cols_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(decode_cols_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -653,9 +651,11 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     int o1 = 2, o4 = 2;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o1, decode_cols_kernel<1>, kThreads, 0) != cudaSuccess) o1 = 2;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o4, decode_cols_kernel<kMaxM>, kThreads, 0) != cudaSuccess) o4 = 2;
-    one_cta_per_sm = o1 == 1 && o4 == 1;
-    sm_count = sms > 0 ? sms : 1;
-  }
+    if (!(o1 == 1 && o4 == 1)) one_cta_per_sm = false;
+    return cudaSuccess;
+  });
+  if (e0 != cudaSuccess) return e0;
+  const int sm_count = lqer::sm_count() > 0 ? lqer::sm_count() : 1;
   if (n < 1 || n > kMaxGroup) return cudaErrorInvalidValue;
   const int M = calls[0].M;
   Params p;
@@ -664,6 +664,8 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   p.status = reinterpret_cast<DeviceStatus*>(workspace);
   p.M = M;
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
+  p.wait_limit = wait_limit_cycles();
+  const int stall = take_stall(kFamDecode) ? 1 : 0;
 
   // CTAs per layer (one per SM at most, so that all of a launch are resident together): a single layer takes what
   // it can use; several share the SMs by the time their columns take
@@ -724,6 +726,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
     // when the layer has so many CTAs that each streams little else
     if ((long long)(m.K / 16) * ((m.k_pad + 31) / 32) <= kLocalTUnits && ctas[g] >= kLocalTMinCtas) ranges = 0;
     ly.t_ranges = ranges;
+    ly.t_expect = ranges + stall;
     ly.pre = pres != nullptr ? pres[g] : nullptr;
     const size_t a_need = (size_t)(m.K / 16) * m.k_pad * 17 + 16;
     ly.a_stage_bytes = (ranges == 0 && ly.pre == nullptr && m.k_pad > 0 && cols_smem_bytes(m, M) + a_need <= 200 * 1024) ? (int)a_need : 0;
@@ -762,14 +765,14 @@ int decode_pre_max_calls() { return dcol::kPreMaxCalls; }
 cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas, uint8_t* const* outs, int n, int order,
                               cudaStream_t s) {
   using namespace dcol;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static OncePerDevice once;
+  cudaError_t e0 = once.run([] {
     cudaError_t e = cudaFuncSetAttribute(decode_pre_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(decode_pre_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+    return e;
+  });
+  if (e0 != cudaSuccess) return e0;
   if (n < 1 || n > kPreMaxCalls) return cudaErrorInvalidValue;
   PreParams p;
   p.order = order;

@@ -78,6 +78,8 @@ struct Params {
   DeviceStatus* status;
   int M, m_tiles;              // row tiles of 256 (the same M for every layer)
   int lr_shift;
+  long long wait_limit;        // bound of every wait, in clock cycles
+  int stall;                   // test hook: the producers withhold the last stage of their last tile, so the waits run out
 };
 
 __device__ __forceinline__ int layer_of(const Params& p, int t) {
@@ -95,7 +97,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
   uint8_t* stage_base = smem;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARRIERS);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile WaitState* abort_flag = reinterpret_cast<volatile WaitState*>(tmem_slot + 2);
 
   const uint32_t bar0 = smem_u32(bars);
   auto loaded = [&](int s) { return bar0 + 8u * s; };                        // local
@@ -115,7 +117,8 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       mbar_init(freed(s), 1);
     }
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 8); }
-    *abort_flag = 0;
+    abort_flag->abort = 0;
+    abort_flag->limit = p.wait_limit;
     fence_barrier_init();
     fence_proxy_async_smem();
   }
@@ -152,6 +155,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
         const bool has_w = my_ntile < n_tiles;
         const int row0 = mt * 2 * BM + (int)rank * BM;
         for (int s = 0; s < stages_per_tile; ++s) {
+          if (p.stall != 0 && s == stages_per_tile - 1 && t + num_pairs >= num_tiles) { ok = false; break; }
           if (!mbar_wait<true>(freed(st), ph ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = smem_u32(stage_base + st * STAGE_BYTES);
           if (s < k_slabs) {
@@ -350,7 +354,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
   }
 
   // ------------------------------------------------------------------ teardown
-  if (*abort_flag != 0) {
+  if (abort_flag->abort != 0) {
     const long long t0 = clock64();
     while (clock64() - t0 < 400000) { }
     if (threadIdx.x == 0) report_error(p.status, LQER_ERR_TIMEOUT, 400, blockIdx.x);
@@ -384,8 +388,16 @@ static EncodeTiledFn encode_fn() {
 
 namespace tc2 {
 
-static cudaError_t launch_params(const TensorMaps& tmaps, const Params& p, int sm_count, cudaStream_t s) {
-  const int max_pairs = sm_count / 2;
+static cudaError_t launch_params(const TensorMaps& tmaps, Params& p, cudaStream_t s) {
+  static OncePerDevice once;
+  cudaError_t e = once.run([] {
+    return cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  });
+  if (e != cudaSuccess) return e;
+  const int max_pairs = sm_count() / 2;
+  if (max_pairs < 1) return cudaErrorInvalidDevice;
+  p.wait_limit = wait_limit_cycles();
+  p.stall = take_stall(kFamGemmTcPair) ? 1 : 0;
   const int pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
@@ -428,14 +440,6 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
   if ((m.N & 3) != 0) return cudaErrorInvalidValue;
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
-  static int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-  }
   TensorMaps tmaps;
   const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
   const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
@@ -470,11 +474,11 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
   p.status = st;
   p.M = M;
   p.lr_shift = m.lr_bits - 2;
-  cudaError_t e = launch_params(tmaps, p, sm_count, s);
+  cudaError_t e = launch_params(tmaps, p, s);
   if (e != cudaSuccess) return e;
   const size_t quads = (size_t)M * m.N / 4;
   int blocks = (int)((quads + 255) / 256);
-  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks > sm_count() * 8) blocks = sm_count() * 8;
   LaunchScope scope(kFamGemmTcPair, s);
   splitk_sum_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<float4*>(Y), reinterpret_cast<const float4*>(partials), C - 1, quads);
   return cudaGetLastError();
@@ -496,16 +500,6 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
   if (n < 1 || n > MAX_GROUP) return cudaErrorInvalidValue;
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
-  static int sm_count = 0;
-  static bool attr_set = false;
-  if (!attr_set) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
   // order: falling number of K stages per tile (stable, so equal layers keep the caller's order)
   int order[MAX_GROUP];
   for (int g = 0; g < n; ++g) order[g] = g;
@@ -546,7 +540,7 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
   p.status = st;
   p.M = M;
   p.lr_shift = metas[0].lr_bits - 2;
-  return launch_params(tmaps, p, sm_count, s);
+  return launch_params(tmaps, p, s);
 }
 
 }  // namespace lqer

@@ -240,7 +240,7 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
                               uint8_t* Xe, cudaStream_t s) {
   const size_t total4 = (size_t)M * (K / 4);
   int blocks = (int)((total4 + 255) / 256);
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   if (blocks < 1) blocks = 1;
   LaunchScope scope(kFamQuantize, s);
   quantize_x_kernel<<<blocks, 256, 0, s>>>(X, M, K, bits, emin, emax, Xm, Xe);
@@ -253,7 +253,7 @@ static cudaError_t launch_prologue_pb(const float* X, int M, const PackedMeta& m
   const int groups = (M + kRows - 1) / kRows;
   const int steps = (m.K64 + PB * 16 - 1) / (PB * 16);
   int cs = 1;
-  while (cs < 8 && groups * cs < 2 * 148 && cs * 2 <= steps) cs *= 2;
+  while (cs < 8 && groups * cs < 2 * sm_count() && cs * 2 <= steps) cs *= 2;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(groups * cs);
   cfg.blockDim = dim3(kThreads);

@@ -58,7 +58,7 @@ struct Cfg {
   static constexpr int OFF_HIA = OFF_XE + X_SLOTS * ROWS * 4;       // [PANELS][8][KP] high words of 2^(e_a + bias)
   static constexpr int OFF_BARS = OFF_HIA + PANELS * 8 * KP * 4;
   static constexpr int NUM_BARS = 2 * RAW_SLOTS + 2 * X_SLOTS + 2 * PANELS + 2 * MAX_TMEM_SLOTS;
-  static constexpr int SMEM_BYTES = OFF_BARS + NUM_BARS * 8 + 16 + 1024;
+  static constexpr int SMEM_BYTES = OFF_BARS + NUM_BARS * 8 + 32 + 1024;
   static_assert(CPW % 8 == 0 && CPW <= 16, "scaler registers");
   static_assert(ROWS % ROW_STEP == 0, "quantiser passes");
   static_assert(PANEL_BYTES % 1024 == 0, "swizzle atoms need 1024-byte bases");
@@ -77,6 +77,8 @@ struct Params {
   int kblocks;              // K / 16
   int panels;               // ceil(K64 / 128)
   int splits;               // CTAs per row tile
+  int expect;               // arrivals a row tile waits for: splits (one more under the stall test hook)
+  long long wait_limit;     // bound of every wait, in clock cycles
   int a_bits, lr_bits, exp_min, exp_max;
   int order;                // ChainOrder: where the wait for the previous kernel sits
   size_t ldx;               // columns of Xcat
@@ -125,18 +127,18 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t pari
       : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
   return ok != 0;
 }
-// Bounded like tc::mbar_wait: gives up after WAIT_LIMIT_CYCLES or as soon as another role has given up.
-__device__ __forceinline__ bool parked_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded like tc::mbar_wait: gives up after the launch's wait limit or as soon as another role has given up.
+__device__ __forceinline__ bool parked_wait(uint32_t bar, uint32_t parity, volatile WaitState* abort_flag) {
   if (mbar_try_wait_parked(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait_parked(bar, parity)) {
-    if (*abort_flag != 0) return false;
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+    if (abort_flag->abort != 0) return false;
+    if (clock64() - t0 > abort_flag->limit) { abort_flag->abort = 1; return false; }
   }
   return true;
 }
 // A wait whose outcome every lane of the warp shares (the code after it shuffles or touches tensor memory as a warp).
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile WaitState* abort_flag) {
   return __all_sync(0xFFFFFFFFu, parked_wait(bar, parity, abort_flag)) != 0;
 }
 
@@ -161,8 +163,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   int* s_hia = reinterpret_cast<int*>(smem + C::OFF_HIA);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BARS);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* last_flag = reinterpret_cast<int*>(tmem_slot + 2);
+  int* last_flag = reinterpret_cast<int*>(tmem_slot + 1);
+  volatile WaitState* abort_flag = reinterpret_cast<volatile WaitState*>(tmem_slot + 2);
 
   const uint32_t bar0 = smem_u32(bars);
   auto raw_full = [&](int s) { return bar0 + 8u * s; };
@@ -190,7 +192,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     for (int s = 0; s < X_SLOTS; ++s) { mbar_init(xq_full(s), QW); mbar_init(xq_empty(s), SW + 1); }
     for (int s = 0; s < PANELS; ++s) { mbar_init(panel_full(s), 1); mbar_init(panel_empty(s), SW + 1); }
     for (int s = 0; s < MAX_TMEM_SLOTS; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), SW); }
-    *abort_flag = 0;
+    abort_flag->abort = 0;
+    abort_flag->limit = p.wait_limit;
     fence_barrier_init();
   }
   fence_proxy_async_smem();
@@ -396,7 +399,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   }
 
   // ------------------------------------------------------------------ the CTAs of a row tile finish T together
-  if (*abort_flag != 0) {
+  if (abort_flag->abort != 0) {
     const long long t0 = clock64();
     while (clock64() - t0 < 400000) { }
     if (tid == 0) report_error(p.status, LQER_ERR_TIMEOUT, 400, blockIdx.x);
@@ -420,8 +423,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     for (;;) {
       int v;
       asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(arrive_cnt) : "memory");
-      if (v >= p.splits) break;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) { seen = 0; break; }
+      if (v >= p.expect) break;
+      if (clock64() - t0 > p.wait_limit) { seen = 0; break; }
       __nanosleep(100);
     }
     if (!seen) report_error(p.status, LQER_ERR_TIMEOUT, 401, blockIdx.x);
@@ -484,12 +487,11 @@ static EncodeTiledFn encode_fn() {
 template <int KP>
 static cudaError_t launch_kp(const TensorMaps& tmaps, const GroupParams& gp, int ctas, cudaStream_t s) {
   using C = Cfg<KP>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(prologue_tc_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static OncePerDevice once;
+  cudaError_t e = once.run([] {
+    return cudaFuncSetAttribute(prologue_tc_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+  });
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(ctas);
   cfg.blockDim = dim3(NUM_THREADS);
@@ -565,6 +567,8 @@ cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const Packed
   GroupParams gp;
   gp.n = n;
   int begin = 0;
+  const long long limit = wait_limit_cycles();
+  const int stall = take_stall(kFamPrologue) ? 1 : 0;
   for (int i = 0; i < kMaxLayers; ++i) {
     const int g = i < n ? i : 0;
     const PackedMeta& m = metas[g];
@@ -586,6 +590,8 @@ cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const Packed
     p.kblocks = m.K / 16;
     p.panels = (m.K64 + 127) / 128;
     p.splits = splits[g];
+    p.expect = splits[g] + stall;
+    p.wait_limit = limit;
     p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
     p.order = order;
     p.ldx = xcat_cols(m);
@@ -603,7 +609,8 @@ cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const Packed
 cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                int order, cudaStream_t s) {
-  const int splits = prologue_tc_splits(m, M);
+  const int sms = sm_count();
+  const int splits = prologue_tc_splits(m, M, sms > 0 && sms < kPrologueMaxCtas ? sms : kPrologueMaxCtas);
   return launch_prologue_tc_group(&X, M, &m, &packed, &xcat, &partials, &counters, &splits, 1, Tm, Te, st, order, s);
 }
 

@@ -40,14 +40,12 @@ static lqer_status_t static_scratch(void** out) {
 
 extern "C" lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, float* Y, void* stream) {
   if (X == nullptr || packed == nullptr || Y == nullptr) return LQER_ERR_NULL;
-  int K = 0, N = 0, k = 0;
-  lqer_status_t st = lqer_packed_shape(packed, &K, &N, &k, nullptr);
-  if (st != LQER_OK) return st;
-  lqer_config_t cfg;
-  lqer_default_config(&cfg);
+  // what this call needs on the path it takes (decode kernels, or prologue + GEMM with its split-K partial sums):
+  // less than lqer_workspace_bytes(M, ...), which covers every batch up to M
   size_t need = 0;
-  if ((st = lqer_workspace_bytes(M, K, N, k, &cfg, &need)) != LQER_OK) return st;
-  if (need > (size_t)LQER_STATIC_SCRATCH_BYTES) return LQER_ERR_STATIC_SCRATCH;   // M (K + k) too large for the fixed array
+  lqer_status_t st = lqer::call_workspace_bytes(packed, M, &need);
+  if (st != LQER_OK) return st;
+  if (need > (size_t)LQER_STATIC_SCRATCH_BYTES) return LQER_ERR_STATIC_SCRATCH;   // the fixed array is too small for this shape
   void* scratch = nullptr;
   if ((st = lqer::static_scratch(&scratch)) != LQER_OK) return st;
   // The array keeps whatever the previous call left: the head of the workspace (status area,

@@ -10,7 +10,13 @@
 namespace lqer {
 namespace tc {
 
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;        // about two seconds
+// What the bounded waits of a CTA share (shared memory): a flag that any role sets when it gives up, and the bound
+// in clock cycles (a launch parameter: wait_limit_cycles()).
+struct WaitState {
+  int abort;
+  int unused;
+  long long limit;
+};
 constexpr int UMMA_M = 128;                                  // rows of the MMA tile per CTA
 
 // ---------------------------------------------------------------------------- PTX wrappers
@@ -32,19 +38,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after WAIT_LIMIT_CYCLES or as soon as another role has given up.
+// Bounded wait: gives up after ws->limit cycles or as soon as another role has given up.
 // kBackoff: sleep between polls (for roles that are not on the critical path, so that their
 // polling does not take issue slots from the MMA issuer).
 template <bool kBackoff = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile WaitState* ws) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   int spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if (kBackoff) __nanosleep(64);
     if ((++spins & 255) == 0) {
-      if (*abort_flag != 0) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+      if (ws->abort != 0) return false;
+      if (clock64() - t0 > ws->limit) { ws->abort = 1; return false; }
     }
   }
   return true;

@@ -25,3 +25,22 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+# Observed max |Y_gpu - Y_oracle| / tol per named case, printed after the run: how close each case comes to the bound.
+_RATIOS = {}
+
+
+@pytest.fixture
+def ratio_log():
+    def log(name, ratio):
+        _RATIOS[name] = max(float(ratio), _RATIOS.get(name, 0.0))
+        return ratio
+    return log
+
+
+def pytest_terminal_summary(terminalreporter):
+    if _RATIOS:
+        terminalreporter.write_line("max |dY| / tol per case (bound 1.0):")
+        for name in sorted(_RATIOS):
+            terminalreporter.write_line(f"  {name}: {_RATIOS[name]:.4g}")

@@ -109,3 +109,27 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "_LIB_PATH", "/nonexistent/liblqer.so")
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_workspace_bound_covers_every_smaller_batch():
+    # lqer_workspace_bytes(M_max) must fit the call with any M <= M_max, whichever path that call takes: decode
+    # kernels (M <= 16), split-K GEMM (M <= 256), the tensor-core prologue's partial sums (row tiles x K ranges,
+    # which grows past one CTA per SM once there are more than 148 row tiles)
+    Ms = [1, 4, 16, 17, 64, 127, 128, 129, 255, 256, 257, 300, 511, 512, 1023, 1024, 2048, 4096, 18944, 19072,
+          32768, 65536]
+    for K, N, k in [(4096, 256, 64), (4096, 4096, 32), (11008, 4096, 32), (5120, 13824, 256), (256, 256, 8),
+                    (2112, 264, 16), (4096, 4096, 0), (1024, 640, 40)]:
+        need = [L.call_workspace_bytes(M, K, N, k) for M in Ms]
+        for i, M_max in enumerate(Ms):
+            total = L.workspace_bytes(M_max, K, N, k)
+            assert total >= max(need[: i + 1]), (K, N, k, M_max)
+
+
+def test_static_scratch_limits_follow_the_call_need():
+    # the figures the header states for lqer_linear_static at K = N = 4096, rank 32
+    fits = lambda M: L.call_workspace_bytes(M, 4096, 4096, 32) <= binding.STATIC_SCRATCH_BYTES
+    assert all(fits(M) for M in (1, 16, 17, 127, 257, 506))
+    assert not fits(128) and not fits(256) and not fits(507)
+    # decode-sized calls fit whatever the shape
+    assert L.call_workspace_bytes(16, 1 << 20, 4096, 256) <= binding.STATIC_SCRATCH_BYTES
+    assert L.call_workspace_bytes(16, 4096, 1 << 22, 256) <= binding.STATIC_SCRATCH_BYTES

@@ -255,3 +255,31 @@ def test_tiny_config_end_to_end():
     e_corr = np.linalg.norm(out.Y - ref)
     e_plain = np.linalg.norm(lqer.forward(X, lqer.prepare_weights(W, None, None)).Y - ref)
     assert e_corr < 0.8 * e_plain
+
+
+def test_forward_requantises_t_per_rank_block_hand_worked():
+    # T = X_q A_q has 20 rank columns -> two blocks of 16 after zero padding, each with its own shared exponent.
+    # Worked by hand: X = e_0 (quantises to exactly 1), A's row 0 = a (every entry a multiple of 2^(e-6) of its own
+    # block, so A_q = A), hence T row = a.
+    #   block 0: a = 0.75, -0.5, 0.3125, 2^-7, 0...   max 0.75 -> e = -1, step 2^-7: m = 96, -64, 40, 1
+    #   block 1: a = 40, -3.25, 0.25, 10.75, pad 0... max 40   -> e = 5,  step 2^-1: m = 80, -6 (6.5 -> even), 0 (0.5 -> even), 22 (21.5 -> even)
+    # One exponent for the whole padded row (e = 5) would turn block 0 into 1, -1, 1 (0.3125 / 0.5 = 0.625), 0.
+    K, N, k = 16, 8, 20
+    X = np.zeros((1, K), np.float32); X[0, 0] = 1.0
+    A = np.zeros((K, k), np.float32)
+    A[0, :4] = [0.75, -0.5, 0.3125, 2.0 ** -7]
+    A[0, 16:20] = [40.0, -3.25, 0.25, 10.75]
+    B = np.zeros((k, N), np.float32)
+    B[:, 0] = 1.0            # sums both blocks
+    B[16:, 1] = 1.0          # the second block alone
+    B[:16, 2] = 1.0          # the first block alone
+    P = lqer.prepare_weights(np.zeros((K, N), np.float32), A, B)
+    assert P.k_pad == 32
+    r = lqer.forward(X, P)
+    assert r.Tm.shape == (1, 32) and r.Te.shape == (1, 2)
+    assert r.Te.tolist() == [[-1, 5]]
+    assert r.Tm[0, :4].tolist() == [96, -64, 40, 1] and not r.Tm[0, 4:16].any()
+    assert r.Tm[0, 16:20].tolist() == [80, -6, 0, 22] and not r.Tm[0, 20:].any()
+    first, second = 73.0 / 128.0, 48.0
+    assert r.Y[0, 0] == first + second and r.Y[0, 1] == second and r.Y[0, 2] == first
+    assert not r.Y[0, 3:].any()

@@ -63,3 +63,31 @@ def test_static_scratch_rejects_what_does_not_fit():
     assert L.launch_count() == launches          # refused on the host, nothing was launched
     assert L.lib().lqer_linear_static(None, 1, P.ptr, Y.data_ptr(), None) == binding.STATUS_NAMES.index("LQER_ERR_NULL")
     P.release()
+
+
+def test_static_scratch_boundary_on_a_4096_layer_and_no_allocation():
+    # K = N = 4096, rank 32: the call's own need decides.  M = 127 is the largest small batch that fits (the split-K
+    # GEMM's partial sums grow with M), M = 128 is the first that is refused, and M = 300 fits again (no split K
+    # above 256 rows).  The calls that run must not change the amount of device memory in use.
+    spec = gen.LayerSpec("static_4096", M=300, K=4096, N=4096, k=32, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=94)
+    P = _layer(spec)
+    Xall = torch.from_numpy(gen.make_activations(spec)).to(DEV)
+    ws = L.new_workspace(spec.M, P)
+    refused = binding.STATUS_NAMES.index("LQER_ERR_STATIC_SCRATCH")
+    for M, fits in ((127, True), (128, False), (300, True), (16, True)):
+        assert (L.call_workspace_bytes(M, spec.K, spec.N, spec.k) <= binding.STATIC_SCRATCH_BYTES) == fits
+        X = Xall[:M].contiguous()
+        Y = torch.full((M, spec.N), float("nan"), dtype=torch.float32, device=DEV)
+        if not fits:
+            assert L.lib().lqer_linear_static(X.data_ptr(), M, P.ptr, Y.data_ptr(), None) == refused
+            continue
+        Y_ref = L.linear(X, P, ws)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        held0 = torch.cuda.memory_allocated()
+        L.linear_static(X, P, Y)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert torch.cuda.memory_allocated() == held0 and free1 == free0      # nothing was allocated, by torch or by the library
+        assert torch.equal(Y, Y_ref), M
+    P.release()
