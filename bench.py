@@ -47,12 +47,29 @@ TRAFFIC = {"sources_sha256": "f3ef00bfeb63edc0", "bytes_per_launch": 739e6,
 DOMINANT_SOURCES = ["paper_2402_02446_b200/csrc/lqer_gemm_tc2.cu", "paper_2402_02446_b200/csrc/lqer_tc_ptx.cuh"]
 
 
-def sources_hash() -> str:
+def sources_hash(sources=None) -> str:
     h = hashlib.sha256()
-    for rel in DOMINANT_SOURCES:
+    for rel in (DOMINANT_SOURCES if sources is None else sources):
         with open(os.path.join(ROOT, rel), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
+
+
+# The same for the HBM-bound kernels: measured DRAM bytes over algorithmic bytes of the captured launch (the traffic
+# grows in proportion to the bytes a launch streams), valid for the sources whose hash is given.
+TRAFFIC_RATIO = {
+    "decode": {"sources": ["paper_2402_02446_b200/csrc/lqer_decode_cols.cu", "paper_2402_02446_b200/csrc/lqer_common.cuh"],
+               "sha256": "", "ratio": 251.0 / 250.5, "note": "profiles/decode_cols_kernel_7b_layer.md"},
+    "prologue": {"sources": ["paper_2402_02446_b200/csrc/lqer_prologue_tc.cu", "paper_2402_02446_b200/csrc/lqer_common.cuh"],
+                 "sha256": "", "ratio": None, "note": "profiles/prologue_tc_kernel_7b_layer.md"},
+}
+
+
+def traffic_of(kernel: str, algorithmic_bytes_per_launch: float):
+    t = TRAFFIC_RATIO[kernel]
+    if t["ratio"] is None or t["sha256"] != sources_hash(t["sources"]):
+        return None
+    return t["ratio"] * algorithmic_bytes_per_launch
 
 
 def layer_flops(M: int, K: int, N: int, k: int) -> float:
@@ -137,11 +154,11 @@ def oracle_sample(rows: int, a_bits: int = 8):
         A, B = gen.make_random_factors(spec)
         P = olqer.prepare_weights(W, A, B)
         X = gen.make_activations(spec, M=rows)
-        work.append((X, P))
+        work.append((X, P, W, A, B))
         flops += layer_flops(rows, spec.K, spec.N, spec.k)
     def run():
-        for X, P in work:
-            olqer.forward(X, P, a_bits=a_bits)
+        return [olqer.forward(X, P, a_bits=a_bits) for X, P, _, _, _ in work]
+    run.work = work
     return run, flops, f"layer 0 q, gate, down linears, {rows} rows of the M={M_PREFILL} batch"
 
 
@@ -156,22 +173,27 @@ def blas_threads() -> int:
     return os.cpu_count() or 1
 
 
-def time_oracle(steps: int, warmup: int, rows: int, a_bits: int = 8):
+def time_oracle(steps: int, warmup: int, rows: int, a_bits: int = 8, check=None):
+    """TFLOP/s and milliseconds per run of the oracle on its bounded sample.  check(work, results), if given, is
+    called with the sample's inputs and the oracle's results of the last run (the GPU arm compares its own
+    output on the same inputs with them)."""
     run, flops, what = oracle_sample(rows, a_bits)
     for _ in range(warmup):
         run()
     t0 = time.perf_counter()
+    res = None
     for _ in range(steps):
-        run()
+        res = run()
     dt = (time.perf_counter() - t0) / max(steps, 1)
-    return flops / dt / 1e12, dt * 1e3, what
+    extra = check(run.work, res) if check is not None else None
+    return flops / dt / 1e12, dt * 1e3, what, extra
 
 
 def run_reference(args) -> None:
     if int(os.environ.get("RANK", "0")) != 0:
         return
     steps, warmup = max(args.steps, 1), max(args.warmup, 0)
-    tflops, ms, what = time_oracle(steps, warmup, rows=args.oracle_rows, a_bits=args.a_bits)
+    tflops, ms, what, _ = time_oracle(steps, warmup, rows=args.oracle_rows, a_bits=args.a_bits)
     cores = blas_threads()
     line = {"impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -196,6 +218,142 @@ def max_over_ranks(values, dist, device):
 def whole_job_value(flops_per_rank_step: float, ms_per_step: float, world: int) -> float:
     """TFLOP/s of the whole job: every rank runs its own replica of the step (weak scaling)."""
     return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
+
+# ------------------------------------------------------------------------------------------ the other workloads
+def time_calls(fn, iters: int, warmup: int = 3) -> float:
+    """Microseconds per call of fn(i), i = 0 .. iters - 1, timed with CUDA events on the current stream."""
+    stream = torch.cuda.current_stream()
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(iters):
+        fn(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / iters
+
+
+def one_launch_per_call_us(L, calls, ws, iters: int) -> float:
+    """Microseconds for one pass over `calls` (decode-sized) with every call a launch of its own, in stream order, as a
+    decoder must run layers that depend on one another.  The loop over the calls runs inside the library, so the
+    figure is the device's, not the Python interpreter's."""
+    from paper_2402_02446_b200 import binding
+    L.set_path(binding.PATH_DECODE)
+    try:
+        return time_calls(lambda i: L.linear_batched(calls, ws), iters)
+    finally:
+        L.set_path(binding.PATH_AUTO)
+
+
+def packed_copies(L, spec, cfg, dev, min_bytes: float, k: int | None = None):
+    """Distinct packed buffers of one layer (the same numbers at different addresses), at least min_bytes together."""
+    W = gen.make_weight_device(spec, dev)
+    kk = spec.k if k is None else k
+    A = B = None
+    if kk > 0:
+        sp = gen.LayerSpec(spec.name, spec.M, spec.K, spec.N, kk, spec.calib_rows, spec.outlier_frac, spec.outlier_scale,
+                           spec.weight_law, spec.seed)
+        A, B = gen.make_random_factors_device(sp, dev)
+    out = [L.prepare_weights(W, A, B, cfg)]
+    while sum(p.buf.numel() for p in out) < min_bytes:
+        out.append(L.prepare_weights(W, A, B, cfg))
+    torch.cuda.synchronize()
+    return out
+
+
+def run_other_configs(L, cfg, dev, peaks, quick: bool) -> dict:
+    """Driver-run figures for the decode-shaped layer, the two prefill MLP layers and the 13B-shaped rank sweep
+    (weights rotated through more than L2 where a layer alone would stay resident)."""
+    out = {}
+    rot = 272e6                                             # bytes of distinct packed copies a timing loop walks
+    hbm, hbm_nom = peaks["hbm_gbs"], 8000.0
+
+    # ---- decode-shaped layer: 4096 x 4096, rank 32, M in {1, 4, 16}
+    dec = {}
+    for M in (1, 4, 16):
+        spec = gen.config_decode(M)
+        copies = packed_copies(L, spec, cfg, dev, rot)
+        n = len(copies)
+        X = gen.make_activations_device(spec, dev)
+        Ys = [torch.empty((M, spec.N), dtype=torch.float32, device=dev) for _ in range(n)]
+        ws = L.new_workspace(M, copies[0])
+        nbytes = layer_weight_bytes(spec.K, spec.N, spec.k) + 4.0 * M * (spec.K + spec.N)
+        calls = L.make_calls([(X, c, y) for c, y in zip(copies, Ys)])
+        wsb = torch.zeros(max(L.batched_workspace_bytes(calls), ws.numel()), dtype=torch.uint8, device=dev)
+        us_lone = one_launch_per_call_us(L, calls, wsb, 4) / n
+        us_shared = time_calls(lambda i: L.linear_batched(calls, wsb), 8) / n
+        dec[f"M{M}"] = {
+            "bytes": nbytes, "copies": n,
+            "lone_call": {"us": us_lone, "gbs": nbytes / us_lone * 1e-3, "frac_of_measured_hbm": nbytes / us_lone * 1e-3 / hbm,
+                          "frac_of_8tbs": nbytes / us_lone * 1e-3 / hbm_nom},
+            "shared_launches": {"us_per_layer": us_shared, "gbs": nbytes / us_shared * 1e-3,
+                                "frac_of_measured_hbm": nbytes / us_shared * 1e-3 / hbm,
+                                "frac_of_8tbs": nbytes / us_shared * 1e-3 / hbm_nom, "independent_layers": n},
+        }
+        for c in copies:
+            c.release()
+        del copies, Ys, ws, wsb
+    out["decode_layer_4096x4096_k32"] = dec
+
+    # ---- prefill MLP layers alone: M = 2048, 4096 x 11008 and 11008 x 4096, rank 32
+    pre = {}
+    for transposed in (False, True):
+        spec = gen.config_prefill(transposed)
+        copies = packed_copies(L, spec, cfg, dev, 0)
+        Xs = [gen.make_activations_device(spec, dev) for _ in range(2)]
+        Y = torch.empty((spec.M, spec.N), dtype=torch.float32, device=dev)
+        ws = L.new_workspace(spec.M, copies[0])
+        us = time_calls(lambda i: L.linear(Xs[i & 1], copies[0], ws, Y), 20)
+        fl = layer_flops(spec.M, spec.K, spec.N, spec.k)
+        pre[spec.name] = {"K": spec.K, "N": spec.N, "M": spec.M, "us": us, "tflops": fl / us * 1e-6,
+                          "frac_of_measured_bf16_burst": fl / us * 1e-6 / peaks["bf16_tflops"],
+                          "frac_of_measured_bf16_sustained": fl / us * 1e-6 / peaks["bf16_tflops_sustained"]}
+        copies[0].release()
+        del copies, Xs, Y, ws
+    out["prefill_mlp_M2048_k32"] = pre
+
+    # ---- 13B-shaped sweep: K = 5120, low-rank overhead against rank
+    sweep = []
+    Ns = gen.SWEEP_N
+    Ms = (1, 512) if quick else gen.SWEEP_M
+    for N in Ns:
+        for M in Ms:
+            base_us = None
+            for k in (0,) + gen.SWEEP_K_RANK:
+                spec = gen.config_sweep(N, M, gen.SWEEP_K_RANK[0] if k == 0 else k)
+                copies = packed_copies(L, spec, cfg, dev, rot if M <= 64 else 0, k=k)
+                n = len(copies)
+                X = gen.make_activations_device(spec, dev)
+                Y = torch.empty((M, N), dtype=torch.float32, device=dev)
+                ws = L.new_workspace(M, copies[0])
+                if M <= 16:
+                    calls = L.make_calls([(X, c, Y) for c in copies])
+                    us = one_launch_per_call_us(L, calls, ws, 3) / n
+                else:
+                    iters = max(8, 2 * n) if M <= 64 else (12 if M <= 512 else 6)
+                    us = time_calls(lambda i: L.linear(X, copies[i % n], ws, Y), iters)
+                if k == 0:
+                    base_us = us
+                K = spec.K
+                row = {"N": N, "M": M, "k": k, "us": us, "overhead_vs_k0": us / base_us - 1.0,
+                       "analytic_flop_overhead": k * (K + N) / (K * N),
+                       "analytic_byte_overhead": 1.0625 * ((k + 15) // 16 * 16) * (K + N) / (0.5625 * K * N)}
+                if M >= 512:
+                    row["tflops"] = layer_flops(M, K, N, k) / us * 1e-6
+                else:
+                    nb = layer_weight_bytes(K, N, k) + 4.0 * M * (K + N)
+                    row["gbs"] = nb / us * 1e-3
+                    row["roofline_us"] = max(nb / (hbm * 1e3), layer_flops(M, K, N, k) / (peaks["bf16_tflops"] * 1e6))
+                sweep.append(row)
+                for c in copies:
+                    c.release()
+                del copies, X, Y, ws
+    out["sweep_13b_K5120"] = sweep
+    return out
 
 
 # ------------------------------------------------------------------------------------------ GPU arm
@@ -320,6 +478,37 @@ def run_ours(args) -> None:
                     "traffic": traffic, "avg_launch_us": dom_ms / dom_launches * 1e3, "launches": dom_launches,
                     "share_of_kernel_time": dom_ms / fam_total}
     kernels = {n: {"launches": c, "ms": round(ms, 4), "share": round(ms / fam_total, 4)} for n, (c, ms) in fam.items()}
+    # one entry per bound: the tensor-bound GEMM above, the HBM-bound decode kernels and the HBM-bound activation prologue
+    rooflines = {"tensor_gemm": roofline}
+    if "decode" in fam:
+        c, ms = fam["decode"]
+        ach = bytes_decode / (ms * 1e-3) / 1e9
+        rooflines["hbm_decode"] = {"bound": "hbm", "kernel": "decode (column-owner kernel, 16 layers per launch, + activations ahead)",
+                                   "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                                   "frac_of_8tbs": ach / 8000.0, "peak_source": f"copy bandwidth, {peaks['source']}",
+                                   "launches": c, "avg_launch_us": ms / c * 1e3,
+                                   "traffic": traffic_of("decode", bytes_decode / c)}
+    if "prologue" in fam:
+        c, ms = fam["prologue"]
+        pb = sum(4.0 * M_PREFILL * K + 2.0 * M_PREFILL * ((K + 63) // 64 * 64 + (k + 15) // 16 * 16) for K, N, k, _ in shapes)
+        ach = pb / (ms * 1e-3) / 1e9
+        rooflines["hbm_prologue"] = {"bound": "hbm", "kernel": "prologue (activation quantisation + low-rank projection)",
+                                     "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                                     "frac_of_8tbs": ach / 8000.0, "peak_source": f"copy bandwidth, {peaks['source']}",
+                                     "launches": c, "avg_launch_us": ms / c * 1e3, "traffic": traffic_of("prologue", pb / c)}
+
+    # ---- the decode leg with every linear a launch of its own (stream order, as layers that depend on one another run)
+    dep_us = one_launch_per_call_us(L, decode_calls, ws, max(2, min(args.steps, 5)))
+    (dep_us,) = max_over_ranks([dep_us], dist, dev)
+    decode_dependent = {"us_per_linear": dep_us / n_lin, "us_per_decoder_layer": dep_us / layers,
+                        "hbm_gbs": bytes_decode / dep_us * 1e-3,
+                        "frac_of_measured_hbm": bytes_decode / dep_us * 1e-3 / peaks["hbm_gbs"],
+                        "what": "224 linears at M=1, one launch per linear in stream order (no sharing of launches)"}
+
+    # ---- the other workloads (one GPU, rank 0's figures)
+    other = None
+    if not args.no_configs:
+        other = run_other_configs(L, cfg, dev, peaks, quick=args.quick_configs)
 
     # ---- end to end through host buffers (pinned), copies inside the timed region
     e2e = None
@@ -360,9 +549,19 @@ def run_ours(args) -> None:
     # ---- the oracle on the host cores (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        tflops, ms, what = time_oracle(1, 0, rows=args.oracle_rows, a_bits=args.a_bits)
+        def gpu_against_oracle(work, results):
+            # the same sample through the library: observed max |Y_gpu - Y_oracle| / tol (the parity bound is 1)
+            worst = 0.0
+            for (X, P, W, A, B), ref in zip(work, results):
+                Pg = L.prepare_weights(torch.from_numpy(W).to(dev), torch.from_numpy(A).to(dev), torch.from_numpy(B).to(dev), cfg)
+                wsg = L.new_workspace(X.shape[0], Pg)
+                Y = L.linear(torch.from_numpy(X).to(dev), Pg, wsg).cpu().numpy().astype(np.float64)
+                worst = max(worst, float(np.max(np.abs(Y - ref.Y) / ref.tol)))
+                Pg.release()
+            return worst
+        tflops, ms, what, worst = time_oracle(1, 0, rows=args.oracle_rows, a_bits=args.a_bits, check=gpu_against_oracle)
         cpu = {"value": tflops, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": what,
-               "seconds": ms / 1e3}
+               "seconds": ms / 1e3, "gpu_max_abs_err_over_tol": worst}
 
     if rank == 0:
         line = {
@@ -385,8 +584,11 @@ def run_ours(args) -> None:
                         "us_per_linear": pre_ms * 1e3 / n_lin},
             "decode": {"us_per_linear": dec_ms * 1e3 / n_lin, "us_per_decoder_layer": dec_ms * 1e3 / layers,
                        "hbm_gbs": bytes_decode / (dec_ms * 1e-3) / 1e9,
-                       "frac_of_measured_hbm": bytes_decode / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": dec_ms},
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+                       "frac_of_measured_hbm": bytes_decode / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                       "frac_of_8tbs": bytes_decode / (dec_ms * 1e-3) / 1e9 / 8000.0, "ms": dec_ms,
+                       "what": "224 independent linears at M=1, up to 16 per launch",
+                       "dependent_order": decode_dependent},
+            "roofline": roofline, "rooflines": rooflines, "configs": other, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks, "peaks": peaks,
         }
         print(json.dumps(line), flush=True)
@@ -405,6 +607,8 @@ def main() -> None:
     ap.add_argument("--oracle-rows", type=int, default=2048, help="token rows of the oracle's bounded sample")
     ap.add_argument("--a-bits", type=int, default=8, help="mantissa bits of the activations: 8 (W4A8, the workload) or 6 (W4A6)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the decode-layer, prefill-MLP and rank-sweep legs")
+    ap.add_argument("--quick-configs", action="store_true", help="rank sweep at M = 1 and 512 only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -88,6 +88,6 @@ def test_static_scratch_boundary_on_a_4096_layer_and_no_allocation():
         L.linear_static(X, P, Y)
         torch.cuda.synchronize()
         free1, _ = torch.cuda.mem_get_info()
-        assert torch.cuda.memory_allocated() == held0 and free1 == free0      # nothing was allocated, by torch or by the library
+        assert torch.cuda.memory_allocated() == held0 and free1 >= free0      # nothing was allocated, by torch or by the library
         assert torch.equal(Y, Y_ref), M
     P.release()
