@@ -354,6 +354,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
   }
 
   // ------------------------------------------------------------------ teardown
+  __syncthreads();                      // every role is done (or has given up): the flag below is final for this CTA
   if (abort_flag->abort != 0) {
     const long long t0 = clock64();
     while (clock64() - t0 < 400000) { }

@@ -399,6 +399,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   }
 
   // ------------------------------------------------------------------ the CTAs of a row tile finish T together
+  __syncthreads();                 // every role is done (or has given up): the flag below is final for this CTA
   if (abort_flag->abort != 0) {
     const long long t0 = clock64();
     while (clock64() - t0 < 400000) { }
