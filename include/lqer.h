@@ -137,9 +137,10 @@ lqer_status_t lqer_project_lowrank(const float* X, int M, const void* packed, in
 
 /* The layer (Section 3.1 last display, Section 3.2 last display):
  *   Y[M,N] = X_q W_q + q(X_q A_q) B_q,  fp32 accumulation of exactly represented products.
- * M <= 16 runs a fused decode kernel (M <= 4: a kernel whose CTAs own output columns; up to
- * 16: a split-K kernel); larger M runs the activation prologue and the tensor-core GEMM over
- * the concatenated contraction [X_q | T_q] . [W_q ; B_q].
+ * M <= 4 runs a fused decode kernel whose CTAs own output columns; M <= 128 a latency-oriented
+ * prologue and a tensor-core GEMM that streams the weights once with the tokens on the MMA's N side;
+ * larger M the activation prologue and the tensor-core GEMM over 256 x 256 tiles of the concatenated
+ * contraction [X_q | T_q] . [W_q ; B_q].
  * lqer_linear uses the default stream. */
 lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y,
                           void* workspace, size_t workspace_bytes);
@@ -155,12 +156,13 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * LQER_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds
  * that much memory until the process exits.  The call itself allocates and frees nothing.
  *  - X, Y, packed, stream: as for lqer_linear_stream (device pointers, caller owned).
- *  - Limit: what this call itself needs on the path it takes must fit LQER_STATIC_SCRATCH_BYTES, otherwise
- *    LQER_ERR_STATIC_SCRATCH is returned and nothing is launched.  The need is smaller than
- *    lqer_workspace_bytes(M, ...), which covers every batch up to M: M <= 16 (the decode kernels: at most
- *    2.8 MB) fits for every supported shape; larger batches need 2 M (K + k) bytes for [X_q | T_q], the
- *    prologue's partial sums and, up to M = 256, the partial sums of the GEMM's K ranges (up to 7 M N 4
- *    bytes).  At K = N = 4096, rank 32 that admits M <= 127 and 257 <= M <= 506, and refuses the rest.
+ *  - Limit: what this call itself needs on the path it takes (lqer_call_workspace_bytes) must fit
+ *    LQER_STATIC_SCRATCH_BYTES, otherwise LQER_ERR_STATIC_SCRATCH is returned and nothing is launched.  The
+ *    need is smaller than lqer_workspace_bytes(M, ...), which covers every batch up to M: it is 2 M (K + k)
+ *    bytes for [X_q | T_q] plus the partial sums of the path's K ranges (up to 128 rows: those of the
+ *    small-batch GEMM, n_tiles x chunks x M x 512 bytes; up to 256 rows: those of the split-K GEMM).  At
+ *    K = N = 4096, rank 32 that admits M <= 86 and 257 <= M <= 487 and refuses the rest; M <= 16 fits for
+ *    every K up to 131072.
  *  - The first call on a device looks up the array's device address (the device must be
  *    current); make that first call before any stream capture begins.
  *  - All calls on a device share the one array and it keeps the previous call's contents; the
@@ -215,10 +217,10 @@ lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void*
 /* Read the device-side status word of `workspace` (synchronises `stream`). */
 lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_t* device_status);
 
-/* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 decode kernels
- * (column-owner kernel for M <= 4, split-K kernel for M <= 16), 3 tensor-core GEMM behind the
+/* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 small-batch kernels
+ * (column-owner kernel for M <= 4, small prologue + tokens-on-N GEMM for M <= 128), 3 tensor-core GEMM behind the
  * activation prologue that runs the projection on int8 mma.sync (at every batch size), 4 tensor-core
- * GEMM with the prologue chosen as in 0, 5 split-K decode kernel for every M <= 16, 6 as 4 with the
+ * GEMM with the prologue chosen as in 0, 5 small prologue + tokens-on-N GEMM for every M <= 128, 6 as 4 with the
  * tcgen05 activation prologue at every batch size (ranks up to 64; by default it serves M >= 1024,
  * and paths 1 and 3 never use it).  Host only, process wide. */
 lqer_status_t lqer_set_path(int path);

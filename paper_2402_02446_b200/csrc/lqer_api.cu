@@ -163,11 +163,25 @@ static lqer_status_t check_arch() {
 }
 
 static size_t xcat_bytes(const PackedMeta& m, int M) { return align_up((size_t)M * xcat_cols(m) * 2, 256); }
+// Scratch of one small-batch call behind the head: Xcat, the prologue's partial sums of T, the GEMM's partial sums of Y.
+static size_t small_slice_bytes(const PackedMeta& m, int M) {
+  return xcat_bytes(m, M) + align_up(prologue_small_slot_bytes(m, M), 256) + align_up(small_gemm_partial_bytes(m, M), 256);
+}
+// A call of up to kSmallMaxM rows runs the column-owner decode kernel (M <= 4 where the layer fits it) or the small
+// prologue and the GEMM with the tokens on the N side; either finds its scratch behind the head.
+static size_t small_bytes(const PackedMeta& m, int M) {
+  const size_t a = small_slice_bytes(m, M), b = decode_cols_slot_bytes(m);
+  return a > b ? a : b;
+}
 // Bytes a call with M rows needs: the persistent head plus the scratch of the path it takes.
-static size_t call_bytes(const PackedMeta& m, int M, bool decode) {
+static size_t call_bytes(const PackedMeta& m, int M, bool small) {
   return align_up(persist_bytes(m), 256) +
-         (decode ? decode_scratch_bytes(m)
-                 : xcat_bytes(m, M) + align_up(prologue_tc_scratch_bytes(m, M), 256) + gemm_splitk_bytes(m, M));
+         (small ? small_bytes(m, M)
+                : xcat_bytes(m, M) + align_up(prologue_tc_scratch_bytes(m, M), 256) + gemm_splitk_bytes(m, M));
+}
+// Whether a call with M rows takes the small-batch kernels under the current path setting.
+static bool takes_small_path(int path, int M) {
+  return (path == 0 || path == 2 || path == 5) && M <= kSmallMaxM;
 }
 // The same for a registered packed buffer, on the path lqer_linear_stream takes for M rows right now.
 lqer_status_t call_workspace_bytes(const void* packed, int M, size_t* bytes) {
@@ -175,20 +189,47 @@ lqer_status_t call_workspace_bytes(const void* packed, int M, size_t* bytes) {
   lqer_status_t st = lookup(packed, m);
   if (st != LQER_OK) return st;
   if (M <= 0 || M > (1 << 24)) return LQER_ERR_SHAPE;
-  const int path = g_path.load();
-  const bool decode = path == 2 || path == 5 || (path == 0 && M <= decode_max_m());
-  *bytes = call_bytes(m, M, decode);
+  *bytes = call_bytes(m, M, takes_small_path(g_path.load(), M));
   return LQER_OK;
 }
 // Bytes that fit every call of up to M_max rows, whichever path it takes.
 static size_t workspace_total(const PackedMeta& m, int M_max) {
   const size_t a = xcat_bytes(m, M_max) + align_up(prologue_tc_scratch_bound(m, M_max), 256) + gemm_splitk_bound(m, M_max);
-  const size_t b = decode_scratch_bytes(m);
+  const size_t b = small_bytes(m, M_max < kSmallMaxM ? M_max : kSmallMaxM);
   return align_up(persist_bytes(m), 256) + (a > b ? a : b);
 }
 
-static lqer_status_t run_linear(const float* X, int M, const void* packed, float* Y, void* workspace,
-                                size_t workspace_bytes, cudaStream_t s, int8_t* Tm, uint8_t* Te, bool project_only) {
+// Element types of X and Y (Section 2.1: the layer sits between 16-bit activations in the w-only setting).
+struct IoTypes {
+  bool x_bf16 = false, y_bf16 = false;
+};
+
+// n small-batch layers with one M (n == 1: a single call): one launch of the small prologue for all of them, then one
+// launch of the GEMM over the work items of all of them.  Layer g finds its scratch at slices[g], its tile counters
+// at tile_counts[g] and its row-group counters at row_counts[g].
+static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, int n, uint8_t* const* slices,
+                             int* const* tile_counts, int* const* row_counts, DeviceStatus* dst, IoTypes io,
+                             int8_t* Tm, uint8_t* Te, bool project_only, cudaStream_t s) {
+  const int M = calls[0].M;
+  SmallPrologueLayer pl[16];
+  SmallGemmLayer gl[16];
+  for (int g = 0; g < n; ++g) {
+    const PackedMeta& m = metas[g];
+    uint8_t* xcat = slices[g];
+    uint8_t* slots = xcat + xcat_bytes(m, M);
+    uint8_t* partials = slots + align_up(prologue_small_slot_bytes(m, M), 256);
+    pl[g] = SmallPrologueLayer{calls[g].X, calls[g].packed, &metas[g], xcat, reinterpret_cast<double*>(slots), row_counts[g],
+                               n == 1 ? Tm : nullptr, n == 1 ? Te : nullptr};
+    gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g]};
+  }
+  cudaError_t err = launch_prologue_small(pl, n, M, io.x_bf16, s);
+  if (err == cudaSuccess && !project_only) err = launch_gemm_tn(gl, n, M, io.y_bf16, dst, s);
+  return err;
+}
+
+static lqer_status_t run_linear(const void* X, int M, const void* packed, void* Y, void* workspace,
+                                size_t workspace_bytes, cudaStream_t s, int8_t* Tm, uint8_t* Te, bool project_only,
+                                IoTypes io = IoTypes()) {
   if (X == nullptr || packed == nullptr || workspace == nullptr || (Y == nullptr && !project_only)) return LQER_ERR_NULL;
   if (M <= 0 || M > (1 << 24)) return LQER_ERR_SHAPE;
   if (!aligned16(X) || (Y != nullptr && !aligned16(Y)) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
@@ -197,30 +238,40 @@ static lqer_status_t run_linear(const float* X, int M, const void* packed, float
   lqer_status_t st = lookup(packed, m);
   if (st != LQER_OK) return st;
   int path = g_path.load();
+  if ((path == 2 || path == 5) && M > kSmallMaxM) return LQER_ERR_SHAPE;
+  const bool small = takes_small_path(path, M);
+  if (project_only && !small) path = 3;
   // Paths 1 and 3 keep the SIMT-style prologue at every batch size; the others take the tensor-core one where it fits.
-  const bool tc_prologue = path != 1 && path != 3 && prologue_tc_fits(m, M, X, path == 6);
+  const bool tc_prologue = path != 1 && path != 3 && !io.x_bf16 && prologue_tc_fits(m, M, static_cast<const float*>(X), path == 6);
   if (path == 6) path = 4;
-  if (project_only) path = 3;
-  if (path == 0 && M <= decode_max_m()) path = 2;
-  const bool decode = path == 2 || path == 5;
-  if (decode && M > decode_max_m()) return LQER_ERR_SHAPE;
-  if (workspace_bytes < call_bytes(m, M, decode)) return LQER_ERR_BUFFER_TOO_SMALL;
+  if (workspace_bytes < call_bytes(m, M, small)) return LQER_ERR_BUFFER_TOO_SMALL;
   if ((st = check_arch()) != LQER_OK) return st;
   DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
-  void* xcat = static_cast<uint8_t*>(workspace) + align_up(persist_bytes(m), 256);
+  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  void* xcat = wsb + align_up(persist_bytes(m), 256);
   cudaError_t err;
-  if (decode) {
-    err = launch_decode(X, M, m, packed, Y, workspace, s, path == 5);
+  if (small) {
+    if (path != 5 && !project_only && !io.x_bf16 && !io.y_bf16 && decode_cols_fits(m, M)) {
+      err = launch_decode_cols(static_cast<const float*>(X), M, m, packed, static_cast<float*>(Y), workspace, s);
+    } else {
+      const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
+      uint8_t* slice = static_cast<uint8_t*>(xcat);
+      int* tiles = reinterpret_cast<int*>(wsb + kStatusBytes);
+      int* rows = reinterpret_cast<int*>(wsb + pcount_offset(m));
+      err = run_small(&one, &m, 1, &slice, &tiles, &rows, dst, io, Tm, Te, project_only, s);
+    }
   } else {
+    if (io.x_bf16 || io.y_bf16) return LQER_ERR_CONFIG;
     if (path == 1 && M > 65535) return LQER_ERR_SHAPE;
-    uint8_t* wsb = static_cast<uint8_t*>(workspace);
-    err = tc_prologue ? launch_prologue_tc(X, M, m, packed, xcat, Tm, Te, dst,
+    const float* Xf = static_cast<const float*>(X);
+    float* Yf = static_cast<float*>(Y);
+    err = tc_prologue ? launch_prologue_tc(Xf, M, m, packed, xcat, Tm, Te, dst,
                                            reinterpret_cast<double*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M)),
                                            reinterpret_cast<int*>(wsb + pcount_offset(m)), kChainAlone, s)
-                      : launch_prologue(X, M, m, packed, xcat, Tm, Te, dst, s);
+                      : launch_prologue(Xf, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
-      err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, Y, s)
-                        : launch_gemm_tc2_splitk(xcat, M, m, packed, Y,
+      err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, Yf, s)
+                        : launch_gemm_tc2_splitk(xcat, M, m, packed, Yf,
                                                  reinterpret_cast<float*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M) +
                                                                           align_up(prologue_tc_scratch_bytes(m, M), 256)),
                                                  dst, s);
@@ -266,6 +317,46 @@ static int prefill_run(const lqer_call_t* calls, int first, int n_calls, int lim
   }
   if (need != nullptr) *need = head + slices;
   return n;
+}
+// Consecutive small-batch calls from `first` on that may share the two launches of the small-batch path (auto path only):
+// the same M <= kSmallMaxM, the same formats, any shapes, none of them served by the column-owner decode kernel; at most
+// `limit`, only as many as the workspace has slices for, and tile counters for.
+constexpr size_t kGroupRowCountOffset = 256 + 32768 * 4 + 16 * 256 * 8;   // the row-tile counter area at its highest position
+static int small_run(const lqer_call_t* calls, int first, int n_calls, int limit, size_t workspace_bytes,
+                     PackedMeta* metas, size_t* need) {
+  const int M = calls[first].M;
+  const size_t head = align_up(kPersistMaxBytes, 256);
+  size_t slices = 0;
+  int n = 0, tiles = 0;
+  while (first + n < n_calls && n < limit) {
+    PackedMeta m;
+    if (calls[first + n].M != M || lookup(calls[first + n].packed, m) != LQER_OK || decode_cols_fits(m, M)) break;
+    if (n > 0 && !same_formats(metas[0], m)) break;
+    if (tiles + m.n_tiles > 32768) break;
+    const size_t sl = slices + small_slice_bytes(m, M);
+    if (n > 0 && head + sl > workspace_bytes) break;
+    metas[n] = m; slices = sl; tiles += m.n_tiles;
+    ++n;
+  }
+  if (need != nullptr) *need = head + slices;
+  return n;
+}
+static lqer_status_t run_small_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace, cudaStream_t s) {
+  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  uint8_t* slices[16];
+  int* tile_counts[16];
+  int* row_counts[16];
+  size_t off = align_up(kPersistMaxBytes, 256);
+  int tiles = 0;
+  for (int g = 0; g < n; ++g) {
+    slices[g] = wsb + off;
+    off += small_slice_bytes(metas[g], calls[0].M);
+    tile_counts[g] = reinterpret_cast<int*>(wsb + kStatusBytes) + tiles;
+    tiles += metas[g].n_tiles;
+    row_counts[g] = reinterpret_cast<int*>(wsb + kGroupRowCountOffset) + 8 * g;
+  }
+  return run_small(calls, metas, n, slices, tile_counts, row_counts, static_cast<DeviceStatus*>(workspace), IoTypes(), nullptr,
+                   nullptr, false, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
 // The run of decode calls from calls[first] on that may share one launch of the column-owner kernel: one M, one set of
 // formats, each fitting the kernel, at least 32 columns, and a slot for each layer's partial sums of T in the workspace.
@@ -481,7 +572,7 @@ lqer_status_t lqer_call_workspace_bytes(int M, int K, int N, int k, const lqer_c
   if (M <= 0 || M > (1 << 24)) return LQER_ERR_SHAPE;
   PackedMeta m;
   fill_meta(m, K, N, k, *cfg);
-  *bytes = call_bytes(m, M, M <= decode_max_m());
+  *bytes = call_bytes(m, M, M <= kSmallMaxM);
   return LQER_OK;
 }
 
@@ -606,8 +697,8 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     lqer_status_t st = lookup(c.packed, m);
     if (st != LQER_OK) return st;
     const int path = g_path.load();
-    const bool decode = path == 2 || path == 5 || (path == 0 && c.M <= decode_max_m());
-    if (workspace_bytes < call_bytes(m, c.M, decode)) return LQER_ERR_BUFFER_TOO_SMALL;
+    if ((path == 2 || path == 5) && c.M > kSmallMaxM) return LQER_ERR_SHAPE;
+    if (workspace_bytes < call_bytes(m, c.M, takes_small_path(path, c.M))) return LQER_ERR_BUFFER_TOO_SMALL;
   }
   const bool may_group = g_path.load() == 0;   // a forced path runs every call on its own
   // Decode launches that follow one another are independent too (no buffer in common: two sets of slots and counters
@@ -627,13 +718,18 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     // slice for each.
     int n = 1;
     PackedMeta m0, metas[16];
-    bool decode_group = false;
+    bool decode_group = false, small_group = false;
     if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
       if (decode_cols_fits(m0, calls[i].M)) {
         n = decode_run(calls, i, n_calls, decode_cols_max_group(), workspace_bytes, metas, nullptr);
         if (n < 1) n = 1;
         decode_group = n > 1;
-      } else if (calls[i].M > kGemmSplitMaxM) {   // smaller batches run split K, each on its own
+      } else if (calls[i].M <= kSmallMaxM) {
+        const int lim = std::min(gemm_tn_max_layers(), prologue_small_max_layers());
+        n = small_run(calls, i, n_calls, lim, workspace_bytes, metas, nullptr);
+        if (n < 1) n = 1;
+        small_group = n > 1;
+      } else if (calls[i].M > kGemmSplitMaxM) {   // batches in between run split K, each on its own
         n = prefill_run(calls, i, n_calls, gemm_tc2_max_group(), workspace_bytes, metas, nullptr);
         if (n < 1) n = 1;
       }
@@ -675,6 +771,9 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
           return LQER_ERR_CUDA;
         chain_open = fills;
         chain_set = set;
+      } else if (small_group) {
+        chain_open = false;
+        if ((st = run_small_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) return st;
       } else {
         chain_open = false;
         if ((st = run_prefill_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) return st;
@@ -719,6 +818,12 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
         stretch_end = i + decode_stretch(calls, i, n_calls, ~(size_t)0, nullptr, nullptr, &ahead);
         need = std::max(need, align_up(kPersistMaxBytes, 256) + ahead);
       }
+    } else if (c.M <= kSmallMaxM) {
+      PackedMeta metas[16];
+      size_t group_need = 0;
+      n = small_run(calls, i, n_calls, std::min(gemm_tn_max_layers(), prologue_small_max_layers()), ~(size_t)0, metas, &group_need);
+      if (n < 1) n = 1;
+      if (n > 1) need = std::max(need, group_need);
     } else if (c.M > kGemmSplitMaxM) {
       PackedMeta metas[8];
       size_t group_need = 0;

@@ -59,7 +59,7 @@ inline uint32_t meta_checksum(const PackedMeta& m) {
 // followed by per-call scratch: Xcat (bf16 [M, K64 + k_pad]) and the fp64 partial sums of the tensor-core
 // prologue for the GEMM path, or the partial-sum slots of the decode path.
 constexpr int kTCountOffset = 64, kTDoneOffset = 68;
-constexpr int kDecodeMaxCtas = 160;
+constexpr int kDecodeMaxCtas = 160;                  // CTAs of one launch of the column-owner decode kernel, at most
 constexpr int kPrologueRowTiles = 512;               // an arrival and a departure counter each: batches up to 65536 rows
 constexpr int kPrologueMaxCtas = 148;               // CTAs of one tensor-core prologue launch the scratch is sized for (launches use min(this, SMs))
 constexpr int kGemmMaxPairs = 74;                    // CTA pairs of the pair GEMM (one per two SMs)
@@ -71,9 +71,9 @@ __host__ __device__ inline size_t tacc_offset(const PackedMeta& m) {
 __host__ __device__ inline size_t pcount_offset(const PackedMeta& m) {
   return tacc_offset(m) + (size_t)16 * m.k_pad * 8;
 }
-__host__ __device__ inline size_t persist_bytes(const PackedMeta& m) {
-  return pcount_offset(m) + (size_t)kPrologueRowTiles * 8;
-}
+// The head has one size for every layer: a workspace that serves layers of different shapes in turn then never has one
+// layer's scratch (which keeps its last contents) where another layer expects zeroed counters.
+__host__ __device__ inline size_t persist_bytes(const PackedMeta&) { return kPersistMaxBytes; }
 // Split-K form of the pair GEMM for small batches (one row tile, so few tiles): the number of K ranges, the scratch
 // for a batch of M rows, and a bound over all batches up to M_max.
 inline int gemm_splitk_ranges(const PackedMeta& m, int M) {
@@ -115,21 +115,40 @@ inline size_t prologue_tc_scratch_bytes(const PackedMeta& m, int M) {
   if (!prologue_tc_rank_ok(m) || (M + 127) / 128 > kPrologueRowTiles) return 0;
   return (size_t)((M + 127) / 128) * prologue_tc_splits(m, M) * 128 * m.k_pad * 8;
 }
-__host__ __device__ inline int decode_units(const PackedMeta& m) {
-  return m.n_tiles * (m.k_slabs + (m.r_blocks + 1) / 2);
+// Small batches (up to kSmallMaxM rows): the prologue for few rows and the GEMM with the tokens on the MMA's N side.
+// Everything below depends on the shape alone, never on the device or on what else shares a launch.
+constexpr int kSmallMaxM = 128;
+// K ranges per group of 16 rows in the small prologue (each a CTA; the last to arrive adds them up in range order).
+inline int prologue_small_ranges(const PackedMeta& m, int M) {
+  const int rgroups = (M + 15) / 16;
+  int r = 148 / rgroups;
+  if (r > 16) r = 16;
+  if (r > m.K64 / 64) r = m.K64 / 64;             // at least four 16-blocks per range
+  return r < 1 ? 1 : r;
 }
-inline int decode_ctas(const PackedMeta& m, int sm_count) {
-  int g = decode_units(m);
-  if (g > sm_count) g = sm_count;
-  if (g > kDecodeMaxCtas) g = kDecodeMaxCtas;
-  return g;
+inline size_t prologue_small_slot_bytes(const PackedMeta& m, int M) {
+  return (size_t)((M + 15) / 16) * prologue_small_ranges(m, M) * 16 * m.k_pad * 8;
+}
+// K chunks per 128-column tile of the small-batch GEMM, and weight stages (64 K) per chunk: about 148 work items per
+// layer, at least eight stages per chunk.
+inline int small_gemm_chunk_stages(const PackedMeta& m) {
+  int c = (148 + m.n_tiles - 1) / m.n_tiles;
+  int cap = m.k_slabs / 8;
+  if (cap < 1) cap = 1;
+  if (c > cap) c = cap;
+  if (c < 1) c = 1;
+  return (m.k_slabs + c - 1) / c;
+}
+inline int small_gemm_chunks(const PackedMeta& m) {
+  const int cs = small_gemm_chunk_stages(m);
+  return (m.k_slabs + cs - 1) / cs;
+}
+inline size_t small_gemm_partial_bytes(const PackedMeta& m, int M) {
+  const int c = small_gemm_chunks(m);
+  return c > 1 ? (size_t)m.n_tiles * c * M * kTileN * 4 : 0;
 }
 // Scratch of the column-owner decode kernel: fp64 partial sums of T, [16 ranges of K][4 rows][k_pad].
 inline size_t decode_cols_slot_bytes(const PackedMeta& m) { return (size_t)16 * 4 * m.k_pad * 8; }
-inline size_t decode_scratch_bytes(const PackedMeta& m) {
-  const size_t a = (size_t)decode_ctas(m, kDecodeMaxCtas) * 2 * 16 * kTileN * 4, b = decode_cols_slot_bytes(m);
-  return a > b ? a : b;
-}
 
 __host__ __device__ inline int b_tile_bytes(const PackedMeta& m) { return m.r_blocks * kTileN * 17; }
 __host__ __device__ inline size_t xcat_cols(const PackedMeta& m) { return (size_t)m.K64 + (size_t)m.k_pad; }
@@ -330,9 +349,31 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
 int gemm_tc2_max_group();
 cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys,
                                   const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s);
-// M <= 4 goes to the column-owner kernel unless force_split_k (test hook: the split-K kernel serves every M <= 16).
-cudaError_t launch_decode(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
-                          void* workspace, cudaStream_t s, bool force_split_k = false);
+// Small batches (M <= kSmallMaxM).  The prologue quantises X (fp32 or bf16) into Xcat and leaves T_q behind it; up to
+// prologue_small_max_layers() layers with one M and one set of formats per launch.
+struct SmallPrologueLayer {
+  const void* X;
+  const void* packed;
+  const PackedMeta* meta;
+  void* xcat;                 // bf16 [M, K64 + k_pad]
+  double* slots;              // prologue_small_slot_bytes of scratch
+  int* counts;                // one zeroed counter per group of 16 rows
+  int8_t* Tm;                 // optional exports of T_q (may be null)
+  uint8_t* Te;
+};
+int prologue_small_max_layers();
+cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, cudaStream_t s);
+// The GEMM with the tokens on the N side of the MMA; up to gemm_tn_max_layers() layers with one M per launch.
+struct SmallGemmLayer {
+  const void* xcat;
+  const void* packed;
+  const PackedMeta* meta;
+  void* Y;                    // [M, N] fp32 or bf16
+  float* partials;            // small_gemm_partial_bytes of scratch (unused if the tiles have one chunk)
+  int* counters;              // one zeroed counter per 128-column tile
+};
+int gemm_tn_max_layers();
+cudaError_t launch_gemm_tn(const SmallGemmLayer* layers, int n, int M, bool y_bf16, DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);
@@ -355,6 +396,5 @@ inline size_t decode_pre_bytes(const PackedMeta& m, int M) {
 int decode_pre_max_calls();
 cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas, uint8_t* const* outs, int n, int order,
                               cudaStream_t s);
-int decode_max_m();
 
 }  // namespace lqer

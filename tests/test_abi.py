@@ -58,8 +58,9 @@ def test_size_queries_follow_the_format():
     # the tensor-core prologue (at most 148 CTAs x [128, k_pad]), or the decode slots
     xcat = 2048 * (4096 + 32) * 2
     partials = 148 * 128 * 32 * 8
-    assert 256 + xcat <= L.workspace_bytes(2048, 4096, 11008, 32) <= 256 + xcat + partials + 16384
-    assert L.workspace_bytes(1, 4096, 4096, 0) >= 256 + 4096 * 2
+    head = 168192                                     # one size for every layer
+    assert head + xcat <= L.workspace_bytes(2048, 4096, 11008, 32) <= head + xcat + partials + 16384
+    assert L.workspace_bytes(1, 4096, 4096, 0) >= head + 4096 * 2
     assert L.workspace_bytes(1, 4096, 4096, 32) <= 4 << 20
 
 
@@ -128,8 +129,8 @@ def test_workspace_bound_covers_every_smaller_batch():
 def test_static_scratch_limits_follow_the_call_need():
     # the figures the header states for lqer_linear_static at K = N = 4096, rank 32
     fits = lambda M: L.call_workspace_bytes(M, 4096, 4096, 32) <= binding.STATIC_SCRATCH_BYTES
-    assert all(fits(M) for M in (1, 16, 17, 127, 257, 506))
-    assert not fits(128) and not fits(256) and not fits(507)
-    # decode-sized calls fit whatever the shape
-    assert L.call_workspace_bytes(16, 1 << 20, 4096, 256) <= binding.STATIC_SCRATCH_BYTES
+    assert all(fits(M) for M in (1, 16, 17, 86, 257, 487))
+    assert not fits(87) and not fits(128) and not fits(256) and not fits(488)
+    # decode-sized calls fit for every K up to 131072, and whatever N
+    assert L.call_workspace_bytes(16, 131072, 4096, 256) <= binding.STATIC_SCRATCH_BYTES
     assert L.call_workspace_bytes(16, 4096, 1 << 22, 256) <= binding.STATIC_SCRATCH_BYTES

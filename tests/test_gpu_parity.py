@@ -266,8 +266,11 @@ DECODE_SPECS = SMALL_SPECS + MID_SPECS + [
 
 
 @pytest.mark.parametrize("M,path", [(1, binding.PATH_DECODE), (3, binding.PATH_DECODE), (4, binding.PATH_DECODE),
-                                    (1, binding.PATH_DECODE_SPLIT_K), (5, binding.PATH_DECODE), (16, binding.PATH_DECODE)],
-                         ids=["cols_M1", "cols_M3", "cols_M4", "splitk_M1", "splitk_M5", "splitk_M16"])
+                                    (1, binding.PATH_SMALL), (5, binding.PATH_DECODE), (16, binding.PATH_DECODE),
+                                    (23, binding.PATH_AUTO), (64, binding.PATH_AUTO), (100, binding.PATH_AUTO),
+                                    (128, binding.PATH_AUTO)],
+                         ids=["cols_M1", "cols_M3", "cols_M4", "small_M1", "small_M5", "small_M16", "small_M23", "small_M64",
+                              "small_M100", "small_M128"])
 @pytest.mark.parametrize("spec", DECODE_SPECS, ids=lambda s: s.name)
 def test_linear_decode_kernel(spec, M, path):
     W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
@@ -319,11 +322,11 @@ def test_batched_decode_groups_same_shape_calls(M):
                            outlier_frac=spec.outlier_frac, outlier_scale=spec.outlier_scale, seed=spec.seed + i)
         layers.append((sp,) + _random_factor_layer(sp))
     Xs = [_t(gen.make_activations(sp, M=M)) for sp, _, _ in layers]
-    n = max(L.workspace_bytes(M, sp.K, sp.N, sp.k) for sp, _, _ in layers)
-    ws = torch.zeros(n, dtype=torch.uint8, device=DEV)
-    launches = L.launch_count()
     Yb = [torch.full((M, sp.N), float("nan"), dtype=torch.float32, device=DEV) for sp, _, _ in layers]
-    L.linear_batched([(x, lay[2], y) for x, lay, y in zip(Xs, layers, Yb)], ws)
+    calls = L.make_calls([(x, lay[2], y) for x, lay, y in zip(Xs, layers, Yb)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    launches = L.launch_count()
+    L.linear_batched(calls, ws)
     torch.cuda.synchronize()
     assert L.poll_status(ws) == 0
     assert L.launch_count() - launches == 1            # seven layers with one M: one launch
@@ -378,6 +381,43 @@ def test_batched_decode_stretch_quantises_activations_ahead(M):
     assert L.poll_status(small) == 0
     for y2, ys in zip(Y2, singles):
         assert torch.equal(y2, ys)
+    for _, _, Pg in base:
+        Pg.release()
+
+
+@pytest.mark.parametrize("M", [5, 16, 40])
+def test_batched_small_batches_share_two_launches(M):
+    # nine independent calls with one M above the column-owner kernel's range: layers of three shapes (one without a
+    # low-rank part) run as ONE launch of the small prologue and ONE launch of the tokens-on-N GEMM over the work items
+    # of all of them; every layer must give what it gives alone, bit for bit (the K chunks of a tile depend on the
+    # shape alone), and twice in a row (counters are left at zero).
+    shapes = [gen.LayerSpec("sg_a", M=M, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=171),
+              gen.LayerSpec("sg_b", M=M, K=2112, N=264, k=16, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=172),
+              gen.LayerSpec("sg_c", M=M, K=512, N=1032, k=0, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=173)]
+    base = []
+    for sp in shapes:
+        if sp.k:
+            base.append((sp,) + _random_factor_layer(sp))
+        else:
+            W = gen.make_weight(sp)
+            base.append((sp, olqer.prepare_weights(W, None, None), L.prepare_weights(_t(W), None, None)))
+    order = [0, 1, 2, 0, 0, 1, 2, 1, 0]
+    Xs = [_t(gen.make_activations(base[j][0], M=M)) + 0.125 * i for i, j in enumerate(order)]
+    Yb = [torch.full((M, base[j][0].N), float("nan"), dtype=torch.float32, device=DEV) for j in order]
+    calls = L.make_calls([(x, base[j][2], y) for x, j, y in zip(Xs, order, Yb)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    for rep in range(2):
+        launches = L.launch_count()
+        L.linear_batched(calls, ws)
+        torch.cuda.synchronize()
+        assert L.poll_status(ws) == 0
+        assert L.launch_count() - launches == 2
+    ws1 = torch.zeros(max(L.workspace_bytes(M, sp.K, sp.N, sp.k) for sp, _, _ in base), dtype=torch.uint8, device=DEV)
+    for i, (x, j, yb) in enumerate(zip(Xs, order, Yb)):
+        assert torch.equal(L.linear(x, base[j][2], ws1), yb), (i, base[j][0].name)
+    for i in (0, 1, 2):
+        sp, P, _ = base[order[i]]
+        assert worst_ratio(Yb[i].cpu().numpy(), olqer.forward(Xs[i].cpu().numpy(), P)) <= 1.0, sp.name
     for _, _, Pg in base:
         Pg.release()
 
