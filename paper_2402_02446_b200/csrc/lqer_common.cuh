@@ -129,10 +129,10 @@ inline int prologue_small_ranges(const PackedMeta& m, int M) {
 inline size_t prologue_small_slot_bytes(const PackedMeta& m, int M) {
   return (size_t)((M + 15) / 16) * prologue_small_ranges(m, M) * 16 * m.k_pad * 8;
 }
-// K chunks per 128-column tile of the small-batch GEMM, and weight stages (64 K) per chunk: about 148 work items per
-// layer, at least eight stages per chunk.
+// K chunks per 128-column tile of the small-batch GEMM, and weight stages (64 K) per chunk: as many work items per layer
+// as fit 148 CTAs in one round, at least eight stages per chunk.
 inline int small_gemm_chunk_stages(const PackedMeta& m) {
-  int c = (148 + m.n_tiles - 1) / m.n_tiles;
+  int c = 148 / m.n_tiles;
   int cap = m.k_slabs / 8;
   if (cap < 1) cap = 1;
   if (c > cap) c = cap;

@@ -17,7 +17,7 @@
 // Roles per CTA:
 //   warp 0      producer: bulk copies of packed weight tiles (issued before the dependency wait: weights
 //               depend on no earlier kernel) and TMA loads of activation tiles
-//   warp 1      tensor memory allocation, MMA issuer
+//   warp 1, 30  MMA issuers (even / odd stages of an item, an accumulator each); warp 1 also allocates tensor memory
 //   warps 2-5   epilogue (tcgen05.ld, Y or partial sums, the last-arriver reduction)
 //   warps 6-29  converters in six groups; group g converts the stages with index = g (mod 6)
 // Two rings: PK slots hold {activation tile, packed weight tile} and are deep, because the bytes in flight
@@ -34,7 +34,8 @@ constexpr int CV_TILE_BYTES = BMW * BK * 2;   // 16384
 constexpr int CV_SLOTS = 6;
 constexpr int CONVERTER_GROUPS = 6;        // = CV_SLOTS: a group meets one CV slot only, and PK slots in phase order
 constexpr int WARPS_PER_GROUP = 4;
-constexpr int NUM_THREADS = (6 + CONVERTER_GROUPS * WARPS_PER_GROUP) * 32;
+constexpr int ISSUER_B_WARP = 6 + CONVERTER_GROUPS * WARPS_PER_GROUP;   // the second MMA-issuing warp
+constexpr int NUM_THREADS = (ISSUER_B_WARP + 1) * 32;
 constexpr int RANK_PER_STAGE = 32;
 constexpr int MAX_LAYERS = 16;
 
@@ -46,7 +47,7 @@ struct Cfg {
   static constexpr int OFF_BARS = OFF_PK + PK_SLOTS * PK_SLOT_BYTES;
   static constexpr int NUM_BARS = 2 * PK_SLOTS + 2 * CV_SLOTS + 4;
   static constexpr int SMEM_BYTES = OFF_BARS + NUM_BARS * 8 + 64 + 1024;
-  static constexpr int TMEM_COLS = 2 * NT < 32 ? 32 : 2 * NT;
+  static constexpr int TMEM_COLS = 4 * NT < 32 ? 32 : 4 * NT;   // two accumulators per item (one per issuing warp), two items
   static_assert(PK_SLOTS % CONVERTER_GROUPS == 0, "a converter group must meet a PK slot in phase order");
   static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0 && TMEM_COLS <= 512, "tensor memory columns");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -106,6 +107,11 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n .reg .pred p;\n elect.sync _|p, 0xFFFFFFFF;\n selp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 __device__ __forceinline__ uint16_t bf16_rn(float v) {
   uint32_t u = __float_as_uint(v);
@@ -142,7 +148,7 @@ gemm_tn_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constant__
   if (threadIdx.x == 0) {
     for (int s = 0; s < PK_SLOTS; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_free(s), 1); }
     for (int s = 0; s < CV_SLOTS; ++s) { mbar_init(cv_ready(s), WARPS_PER_GROUP); mbar_init(cv_free(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 2); mbar_init(acc_empty(a), 4); }
     abort_flag->abort = 0;
     abort_flag->limit = p.wait_limit;
     fence_barrier_init();
@@ -208,33 +214,44 @@ gemm_tn_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constant__
       }
       if (!waited) flush();
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(BMW, NT);
-      uint32_t it_no = 0, tile_it = 0;
-      bool ok = true;
-      for (int i = cta; i < num_items && ok; i += num_ctas, ++tile_it) {
-        const Item it = item_of(p, i);
-        const Layer& ly = p.L[it.layer];
-        const int acc = tile_it & 1;
-        if (!mbar_wait(acc_empty(acc), ((tile_it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+  } else if (warp == 1 || warp == ISSUER_B_WARP) {
+    // ------------------------------------------------------------------ MMA issuers
+    // An MMA with so few tokens costs the tensor core far more than its arithmetic, and what bounds the kernel is
+    // the rate at which MMAs can be handed over.  So two warps issue: one takes the even stages of an item, the
+    // other the odd ones, each into an accumulator of its own (the epilogue adds the two).  The whole warp runs the
+    // loop, so that descriptors and addresses are warp-uniform values; one elected lane issues.
+    const int which = warp == 1 ? 0 : 1;
+    constexpr uint32_t idesc = make_idesc(BMW, NT);
+    const uint32_t cv0 = smem_u32(cv_base), pk0 = smem_u32(pk_base);
+    uint32_t it_no = 0, tile_it = 0;
+    bool ok = true;
+    for (int i = cta; i < num_items && ok; i += num_ctas, ++tile_it) {
+      const Item it = item_of(p, i);
+      const Layer& ly = p.L[it.layer];
+      const int acc = tile_it & 1;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty(acc), ((tile_it >> 1) & 1) ^ 1, abort_flag)) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + acc * 2 * NT + which * NT;
+      for (int s = it.s_lo; s < it.s_hi; ++s, ++it_no) {
+        if (((s - it.s_lo) & 1) != which) continue;
+        const int cv = it_no % CV_SLOTS, pk = it_no % PK_SLOTS;
+        const uint64_t a_desc = make_desc(cv0 + cv * CV_TILE_BYTES);
+        const uint64_t b_desc = make_desc(pk0 + pk * C::PK_SLOT_BYTES);
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(cv_ready(cv), (it_no / CV_SLOTS) & 1, abort_flag)) != 0;
+        if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * NT;
-        for (int s = it.s_lo; s < it.s_hi; ++s, ++it_no) {
-          const int cv = it_no % CV_SLOTS, pk = it_no % PK_SLOTS;
-          const uint64_t a_desc = make_desc(smem_u32(cv_base + cv * CV_TILE_BYTES));
-          const uint64_t b_desc = make_desc(smem_u32(pk_base + pk * C::PK_SLOT_BYTES));
-          if (!mbar_wait(cv_ready(cv), (it_no / CV_SLOTS) & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const int nk = s < ly.k_slabs ? 4 : min(2, ly.r_blocks - (s - ly.k_slabs) * 2);
-          for (int j = 0; j < nk; ++j)            // +2 in the address field = 32 bytes = 16 K
-            umma_bf16(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (s > it.s_lo || j > 0) ? 1u : 0u);
+        const int nk = s < ly.k_slabs ? 4 : min(2, ly.r_blocks - (s - ly.k_slabs) * 2);
+        if (elect_one()) {
+          for (int j = 0; j < nk; ++j)              // +2 in the address field = 32 bytes = 16 K
+            umma_bf16(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (s > it.s_lo + which || j > 0) ? 1u : 0u);
           umma_commit(cv_free(cv));
           umma_commit(pk_free(pk));
         }
-        if (ok) umma_commit(acc_full(acc));
+        __syncwarp();
       }
+      if (ok && elect_one()) umma_commit(acc_full(acc));   // with no stage of its own (a one-stage item) it arrives at once
+      __syncwarp();
     }
   } else if (warp < 6) {
     // ------------------------------------------------------------------ epilogue
@@ -257,7 +274,14 @@ gemm_tn_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constant__
       for (int c0 = 0; c0 < NT; c0 += 16) {
         if (c0 >= p.M) break;
         uint32_t r[16];
-        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + acc * NT + c0, r);
+        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 2 * NT + c0, r);
+        if (it.s_hi - it.s_lo >= 2) {                // the odd stages' accumulator (empty for a one-stage item)
+          uint32_t r2[16];
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 2 * NT + NT + c0, r2);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+        }
         tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
@@ -283,15 +307,40 @@ gemm_tn_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constant__
         epilogue_barrier();
         if (*last_flag != 0) {
           __threadfence();
-          const float* p0 = ly.partials + ((size_t)it.tile * ly.chunks * p.M) * BMW + col_in_tile;
+          // a warp per token row, a lane per four columns; the chunk loads of two rows are in flight together
+          const int c4 = lane * 4, trow0 = warp - 2;
+          const bool quad_ok = it.tile * BMW + c4 < ly.N;              // N is a multiple of 8: the quad is whole
+          const float* p0 = ly.partials + ((size_t)it.tile * ly.chunks * p.M) * BMW + c4;
           const size_t chunk_stride = (size_t)p.M * BMW;
-#pragma unroll 2
-          for (int token = 0; token < p.M; ++token) {
-            float v = 0.f;
-            for (int c = 0; c < ly.chunks; ++c) v += __ldcg(p0 + (size_t)c * chunk_stride + (size_t)token * BMW);
-            if (col_ok) {
-              if (p.y_bf16) static_cast<uint16_t*>(ly.Y)[(size_t)token * ly.N + col] = bf16_rn(v);
-              else static_cast<float*>(ly.Y)[(size_t)token * ly.N + col] = v;
+          for (int token = trow0; token < p.M; token += 8) {
+            float4 v[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+            for (int cb = 0; cb < ly.chunks; cb += 4) {
+              float4 t[2][4];
+#pragma unroll
+              for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                  t[u][c] = (cb + c < ly.chunks && token + 4 * u < p.M)
+                                ? __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)(cb + c) * chunk_stride + (size_t)(token + 4 * u) * BMW))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {            // chunk order: the same sum whoever computes it
+                  if (cb + c < ly.chunks) { v[u].x += t[u][c].x; v[u].y += t[u][c].y; v[u].z += t[u][c].z; v[u].w += t[u][c].w; }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int tk = token + 4 * u;
+              if (tk < p.M && quad_ok) {
+                const size_t o = (size_t)tk * ly.N + it.tile * BMW + c4;
+                if (p.y_bf16)
+                  *reinterpret_cast<uint2*>(static_cast<uint16_t*>(ly.Y) + o) =
+                      make_uint2(bf16_rn(v[u].x) | ((uint32_t)bf16_rn(v[u].y) << 16), bf16_rn(v[u].z) | ((uint32_t)bf16_rn(v[u].w) << 16));
+                else
+                  *reinterpret_cast<float4*>(static_cast<float*>(ly.Y) + o) = v[u];
+              }
             }
           }
           if (warp == 2 && lane == 0) ly.counters[it.tile] = 0;      // zero again for the next call
@@ -299,7 +348,7 @@ gemm_tn_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constant__
         epilogue_barrier();                         // last_flag may be rewritten only after everyone has read it
       }
     }
-  } else {
+  } else if (warp < ISSUER_B_WARP) {
     // ------------------------------------------------------------------ converters
     const int c = threadIdx.x - 6 * 32;          // 0..767
     const int group = c >> 7, nl = c & 127;      // stage group; weight column of the tile

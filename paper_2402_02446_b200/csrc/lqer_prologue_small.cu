@@ -84,8 +84,17 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
   const int bias = -127 - (p.a_bits - 2) - (p.lr_bits - 2);   // exponent bytes carry +127
 
   // The kernel after this one (the GEMM) may start at once: it only prefetches weights before its own wait.
-  // X and the workspace may still be in use by the kernel before: wait for it.
+  // This CTA's share of A_q depends on no earlier kernel: on its way to L2 while the kernel before drains.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (has_rank) {
+    const int kr_lo = min(kb_lo, kblocks), kr_hi = min(kb_hi, kblocks);
+    const uint8_t* gm = ly.asec + (size_t)kr_lo * k_pad * 16;
+    const uint8_t* ge = a_exp + (size_t)kr_lo * k_pad;
+    const int mant = (kr_hi - kr_lo) * k_pad * 16, ex = (kr_hi - kr_lo) * k_pad;
+    for (int o = tid * 128; o < mant; o += kThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(gm + o));
+    for (int o = tid * 128; o < ex; o += kThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(ge + o));
+  }
+  // X and the workspace may still be in use by the kernel before: wait for it.
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   double acc[TPW][4];
@@ -98,21 +107,35 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
     const int nblk = min(kStepCols / 16, kb_hi - kb0);
     // ---- quantise 16 rows x (nblk * 16) columns: bf16 to Xcat, int8 + exponents to shared memory
     const int quads_per_row = nblk * 4;
-    for (int f0 = 0; f0 < kRows * quads_per_row; f0 += kThreads) {       // whole warps: the block maximum is a shuffle
-      const int f = f0 + tid;
-      const bool live = f < kRows * quads_per_row;
-      const int r = live ? f / quads_per_row : 0, c4 = live ? f % quads_per_row : 0;
-      const int col = kb0 * 16 + c4 * 4, row = row0 + r;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (live && row < M && col < K) v = load_x4(ly.X, (size_t)row * K + col, p.x_bf16);
-      int e;
-      uint32_t m8;
-      uint2 bf;
-      quantize_quad(v, p.a_bits, p.exp_min, p.exp_max, e, m8, bf);
-      if (live) {
-        *reinterpret_cast<uint32_t*>(&s_xq[r * kXqStride + c4 * 4]) = m8;
-        if ((c4 & 3) == 0) s_xe[r][c4 >> 2] = (int8_t)e;
-        if (row < M) *reinterpret_cast<uint2*>(ly.xcat + (size_t)row * ldx + col) = bf;
+    const int n_quads = kRows * quads_per_row;                             // a multiple of 64
+    for (int f0 = 0; f0 < n_quads; f0 += 4 * kThreads) {                  // whole warps: the block maximum is a shuffle
+      // four loads per thread in flight, then the arithmetic: a kernel this short is a chain of memory latencies
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int f = f0 + u * kThreads + tid;
+        const bool live = f < n_quads;
+        const int r = live ? f / quads_per_row : 0, c4 = live ? f % quads_per_row : 0;
+        const int col = kb0 * 16 + c4 * 4, row = row0 + r;
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (live && row < M && col < K) v[u] = load_x4(ly.X, (size_t)row * K + col, p.x_bf16);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int f = f0 + u * kThreads + tid;
+        if (f0 + u * kThreads >= n_quads) break;                           // uniform over the CTA
+        const bool live = f < n_quads;
+        const int r = live ? f / quads_per_row : 0, c4 = live ? f % quads_per_row : 0;
+        const int col = kb0 * 16 + c4 * 4, row = row0 + r;
+        int e;
+        uint32_t m8;
+        uint2 bf;
+        quantize_quad(v[u], p.a_bits, p.exp_min, p.exp_max, e, m8, bf);
+        if (live) {
+          *reinterpret_cast<uint32_t*>(&s_xq[r * kXqStride + c4 * 4]) = m8;
+          if ((c4 & 3) == 0) s_xe[r][c4 >> 2] = (int8_t)e;
+          if (row < M) *reinterpret_cast<uint2*>(ly.xcat + (size_t)row * ldx + col) = bf;
+        }
       }
     }
     __syncthreads();
@@ -122,24 +145,39 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
       const int b_step = NT >= kWarps ? 1 : WPN;
       const int nt0 = NT >= kWarps ? warp : warp % NT;
       const int nreal = min(nblk, kblocks - kb0);
-      for (int b = b_first; b < nreal; b += b_step) {
-        const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s_xq[g * kXqStride + b * 16 + tig * 4]);
-        const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s_xq[(g + 8) * kXqStride + b * 16 + tig * 4]);
-        const int ex0 = s_xe[g][b] + bias, ex1 = s_xe[g + 8][b] + bias;
-        const size_t kb = (size_t)(kb0 + b);
+      // four blocks per round: their A_q words are requested together, then the MMAs run
+      for (int bq = b_first; bq < nreal; bq += 4 * b_step) {
+        uint32_t bw[4][TPW], ew[4][TPW];
 #pragma unroll
-        for (int i = 0; i < TPW; ++i) {
-          const int nt = nt0 + kWarps * i;
-          if (nt < NT) {
-            const uint32_t b0 = __ldg(reinterpret_cast<const uint32_t*>(ly.asec + (kb * k_pad + nt * 8 + g) * 16 + tig * 4));
-            const uint32_t ea2 = __ldg(reinterpret_cast<const uint16_t*>(a_exp + kb * k_pad + nt * 8 + tig * 2));
-            int c[4];
-            mma_s8(c, a0, a1, b0);
-            const int ea_lo = (int)(ea2 & 0xFFu), ea_hi = (int)(ea2 >> 8);
-            acc[i][0] = fma((double)c[0], pow2d(ex0 + ea_lo), acc[i][0]);
-            acc[i][1] = fma((double)c[1], pow2d(ex0 + ea_hi), acc[i][1]);
-            acc[i][2] = fma((double)c[2], pow2d(ex1 + ea_lo), acc[i][2]);
-            acc[i][3] = fma((double)c[3], pow2d(ex1 + ea_hi), acc[i][3]);
+        for (int u = 0; u < 4; ++u) {
+          const int b = bq + u * b_step;
+          const size_t kb = (size_t)(kb0 + (b < nreal ? b : bq));
+#pragma unroll
+          for (int i = 0; i < TPW; ++i) {
+            const int nt = min(nt0 + kWarps * i, NT - 1);
+            bw[u][i] = __ldg(reinterpret_cast<const uint32_t*>(ly.asec + (kb * k_pad + nt * 8 + g) * 16 + tig * 4));
+            ew[u][i] = __ldg(reinterpret_cast<const uint16_t*>(a_exp + kb * k_pad + nt * 8 + tig * 2));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int b = bq + u * b_step;
+          if (b < nreal) {
+            const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s_xq[g * kXqStride + b * 16 + tig * 4]);
+            const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s_xq[(g + 8) * kXqStride + b * 16 + tig * 4]);
+            const int ex0 = s_xe[g][b] + bias, ex1 = s_xe[g + 8][b] + bias;
+#pragma unroll
+            for (int i = 0; i < TPW; ++i) {
+              if (nt0 + kWarps * i < NT) {
+                int c[4];
+                mma_s8(c, a0, a1, bw[u][i]);
+                const int ea_lo = (int)(ew[u][i] & 0xFFu), ea_hi = (int)(ew[u][i] >> 8);
+                acc[i][0] = fma((double)c[0], pow2d(ex0 + ea_lo), acc[i][0]);
+                acc[i][1] = fma((double)c[1], pow2d(ex0 + ea_hi), acc[i][1]);
+                acc[i][2] = fma((double)c[2], pow2d(ex1 + ea_lo), acc[i][2]);
+                acc[i][3] = fma((double)c[3], pow2d(ex1 + ea_hi), acc[i][3]);
+              }
+            }
           }
         }
       }
@@ -189,9 +227,12 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
   const int n_out = kRows * k_pad;                   // a multiple of 32: 16 adjacent lanes hold one block
   for (int o = tid; o < n_out; o += kThreads) {
     const int r = o / k_pad, j = o % k_pad;
+    double part[16];                                 // at most 16 ranges: all loads in flight, then the sum in range order
+#pragma unroll
+    for (int c = 0; c < 16; ++c) part[c] = c < ly.ranges ? __ldcg(slots0 + (size_t)c * n_out + o) : 0.0;
     double t = 0.0;
-#pragma unroll 4
-    for (int c = 0; c < ly.ranges; ++c) t += __ldcg(slots0 + (size_t)c * n_out + o);
+#pragma unroll
+    for (int c = 0; c < 16; ++c) t += part[c];
     double amax = (t != t) ? 0.0 : fabs(t);
 #pragma unroll
     for (int sft = 1; sft < 16; sft <<= 1) amax = fmax(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
