@@ -35,7 +35,6 @@ constexpr int BN = 256;                    // output columns per pair tile
 constexpr int BNH = 128;                   // columns converted by one CTA
 constexpr int BK = 64;
 constexpr int STAGES = 6;
-constexpr int ROUND = 2;                   // ring stages the MMA thread takes per round
 constexpr int A_TILE_BYTES = BM * BK * 2;                     // 16384: activations (TMA, swizzled)
 constexpr int B_TILE_BYTES = BNH * BK * 2;                    // 16384: converted weights (swizzled)
 constexpr int PK_OFFSET = A_TILE_BYTES + B_TILE_BYTES;        // packed weight tile (4608) behind them
@@ -182,7 +181,10 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (lane == 0 && rank == 0) {
+    // The whole warp runs the loop, so that barrier addresses and descriptors are warp-uniform values, and one
+    // elected lane issues: the tensor pipe takes an MMA of this shape every 128 cycles and queues very few, so every
+    // cycle the issuing warp spends between two MMAs beyond that is a cycle the pipe idles.
+    if (rank == 0) {
       int st = 0;
       uint32_t ph = 0, tile_it = 0;
       const uint32_t idesc = make_idesc(2 * BM, BN);
@@ -193,57 +195,34 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
         const int layer = layer_of(p, t);
         const int k_slabs = p.L[layer].k_slabs, r_blocks = p.L[layer].r_blocks, stages_per_tile = p.L[layer].spt;
         const int acc = tile_it & 1;
-        if (!mbar_wait(acc_empty(acc), ((tile_it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty(acc), ((tile_it >> 1) & 1) ^ 1, abort_flag)) != 0;
+        if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int s = 0; s < stages_per_tile;) {
+        for (int s = 0; s < stages_per_tile; ++s) {
           // everything that does not depend on the wait is computed before it
           const uint64_t a_desc = a_desc0 + (uint64_t)(st * (STAGE_BYTES >> 4));
           const uint64_t b_desc = b_desc0 + (uint64_t)(st * (STAGE_BYTES >> 4));
           const uint32_t first = s > 0 ? 1u : 0u;
           const uint32_t free_bar = freed(st);
-          if (s + ROUND <= k_slabs) {
-            // ROUND 64-K stages per round of the issuing thread: the poll of a barrier and the loop cost
-            // about as much as one MMA takes the tensor pipe, so they are paid once per 4 * ROUND MMAs.
-            int sr = st;
-            uint32_t pr = ph;
-#pragma unroll
-            for (int r = 0; r < ROUND; ++r) {
-              if (!mbar_wait(ready(sr), pr, abort_flag)) ok = false;
-              if (++sr == STAGES) { sr = 0; pr ^= 1; }
-            }
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int r = 0; r < ROUND; ++r) {
-              const uint64_t ad = a_desc0 + (uint64_t)(st * (STAGE_BYTES >> 4));
-              const uint64_t bd = b_desc0 + (uint64_t)(st * (STAGE_BYTES >> 4));
-              umma_bf16_pair(d_tmem, ad, bd, idesc, (r > 0 || s > 0) ? 1u : 0u);   // +2 in the address field = 32 bytes = 16 K
-              umma_bf16_pair(d_tmem, ad + 2, bd + 2, idesc, 1u);
-              umma_bf16_pair(d_tmem, ad + 4, bd + 4, idesc, 1u);
-              umma_bf16_pair(d_tmem, ad + 6, bd + 6, idesc, 1u);
-              umma_commit_pair(freed(st));
-              if (++st == STAGES) { st = 0; ph ^= 1; }
-            }
-            s += ROUND;
-            continue;
-          }
-          if (!mbar_wait(ready(st), ph, abort_flag)) { ok = false; break; }
+          const int nk = s < k_slabs ? 4 : min(2, r_blocks - (s - k_slabs) * 2);
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(ready(st), ph, abort_flag)) != 0;
+          if (!ok) break;
           tc_fence_after();
-          if (s < k_slabs) {           // 64 K = four MMAs
-            umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, first);
-            umma_bf16_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
-            umma_bf16_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
-            umma_bf16_pair(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
-          } else {
-            const int nk = min(2, r_blocks - (s - k_slabs) * 2);
-            for (int j = 0; j < nk; ++j) umma_bf16_pair(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, 1u);
+          if (elect_one()) {
+            umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, first);           // +2 in the address field = 32 bytes = 16 K
+            if (nk > 1) umma_bf16_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
+            if (nk > 2) {
+              umma_bf16_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
+              umma_bf16_pair(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+            }
+            umma_commit_pair(free_bar);
           }
-          umma_commit_pair(free_bar);
+          __syncwarp();
           if (++st == STAGES) { st = 0; ph ^= 1; }
-          ++s;
         }
-        if (ok) umma_commit_pair(acc_full(acc));
+        if (ok && elect_one()) umma_commit_pair(acc_full(acc));
+        __syncwarp();
       }
     }
   } else if (warp < 6) {
