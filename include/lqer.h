@@ -63,6 +63,13 @@ typedef struct {
   int w_exp_max;     /* 4-bit shared exponent (16 values, e.g. [-12, 3]) and the activations an 8-bit one */
 } lqer_config_t;
 
+/* Element type of activations at the layer's boundary (Section 2.1: weight-only settings keep 16-bit activations
+ * between layers; the w&a settings quantise them on entry, which the layer does itself either way). */
+typedef enum {
+  LQER_F32 = 0,
+  LQER_BF16 = 1
+} lqer_dtype_t;
+
 /* One call of a batch (Section 4.3: layers are independent). */
 typedef struct {
   const float* X;     /* [M,K] */
@@ -138,7 +145,7 @@ lqer_status_t lqer_project_lowrank(const float* X, int M, const void* packed, in
 /* The layer (Section 3.1 last display, Section 3.2 last display):
  *   Y[M,N] = X_q W_q + q(X_q A_q) B_q,  fp32 accumulation of exactly represented products.
  * M <= 4 runs a fused decode kernel whose CTAs own output columns; M <= 128 a latency-oriented
- * prologue and a tensor-core GEMM that streams the weights once with the tokens on the MMA's N side;
+ * prologue and a tensor-core GEMM that streams the weights once against a 64- or 128-row token tile;
  * larger M the activation prologue and the tensor-core GEMM over 256 x 256 tiles of the concatenated
  * contraction [X_q | T_q] . [W_q ; B_q].
  * lqer_linear uses the default stream. */
@@ -146,6 +153,18 @@ lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y,
                           void* workspace, size_t workspace_bytes);
 lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, float* Y,
                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* The same layer with a choice of element types at its boundary (Section 2.1: the layer sits between 16-bit
+ * activations in the w-only setting and re-quantises them in the w&a setting): X [M,K] of x_dtype, Y [M,N] of
+ * y_dtype, both dense row-major and 16-byte aligned.  bf16 X is quantised to MXINT like fp32 X (every bf16
+ * value is an fp32 value); bf16 Y is the fp32 result rounded to nearest even.  Everything else - packed,
+ * workspace, paths, device-side status - as for lqer_linear_stream; the column-owner decode kernel reads and
+ * writes fp32 only, so 16-bit calls of up to 4 rows take the small-batch kernels.  lqer_linear_batched_ex is
+ * lqer_linear_batched with every call's X and Y of the given types (cast the pointers of lqer_call_t). */
+lqer_status_t lqer_linear_ex(const void* X, lqer_dtype_t x_dtype, int M, const void* packed, void* Y, lqer_dtype_t y_dtype,
+                             void* workspace, size_t workspace_bytes, void* stream);
+lqer_status_t lqer_linear_batched_ex(const lqer_call_t* calls, int n_calls, lqer_dtype_t x_dtype, lqer_dtype_t y_dtype,
+                                     void* workspace, size_t workspace_bytes, void* stream);
 
 /* The same layer for callers that cannot allocate device memory (the paper has no counterpart:
  * this is a property of the library, not of the method).  It is meant for code that runs
@@ -160,8 +179,8 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  *    LQER_STATIC_SCRATCH_BYTES, otherwise LQER_ERR_STATIC_SCRATCH is returned and nothing is launched.  The
  *    need is smaller than lqer_workspace_bytes(M, ...), which covers every batch up to M: it is 2 M (K + k)
  *    bytes for [X_q | T_q] plus the partial sums of the path's K ranges (up to 128 rows: those of the
- *    small-batch GEMM, n_tiles x chunks x M x 512 bytes; up to 256 rows: those of the split-K GEMM).  At
- *    K = N = 4096, rank 32 that admits M <= 86 and 257 <= M <= 487 and refuses the rest; M <= 16 fits for
+ *    small-batch GEMM, ceil(N / 256) x chunks x M x 1024 bytes; up to 256 rows: those of the split-K GEMM).  At
+ *    K = N = 4096, rank 32 that admits M <= 57 and 257 <= M <= 487 and refuses the rest; M <= 16 fits for
  *    every K up to 131072.
  *  - The first call on a device looks up the array's device address (the device must be
  *    current); make that first call before any stream capture begins.
@@ -218,9 +237,9 @@ lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void*
 lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_t* device_status);
 
 /* Force a kernel path for tests: 0 auto, 1 plain CUDA-core reference kernel, 2 small-batch kernels
- * (column-owner kernel for M <= 4, small prologue + tokens-on-N GEMM for M <= 128), 3 tensor-core GEMM behind the
+ * (column-owner kernel for M <= 4, small prologue + small-batch GEMM for M <= 128), 3 tensor-core GEMM behind the
  * activation prologue that runs the projection on int8 mma.sync (at every batch size), 4 tensor-core
- * GEMM with the prologue chosen as in 0, 5 small prologue + tokens-on-N GEMM for every M <= 128, 6 as 4 with the
+ * GEMM with the prologue chosen as in 0, 5 small prologue + small-batch GEMM for every M <= 128, 6 as 4 with the
  * tcgen05 activation prologue at every batch size (ranks up to 64; by default it serves M >= 1024,
  * and paths 1 and 3 never use it).  Host only, process wide. */
 lqer_status_t lqer_set_path(int path);

@@ -96,3 +96,25 @@ def pad_axis(v: np.ndarray, axis: int, multiple: int = BLOCK) -> np.ndarray:
     width = [(0, 0)] * v.ndim
     width[axis] = (0, n_pad - n)
     return np.pad(v, width)
+
+
+def round_bf16(v: np.ndarray) -> np.ndarray:
+    """Nearest bfloat16 value (8 significant bits, round half to even) of each element, as fp64.
+
+    The layer may take its activations and hand over its output in 16 bits (Section 2.1: FP16 activations in
+    the w-only setting); this is the rounding of that boundary, written out from the format's definition:
+    v = f * 2**p with f in [0.5, 1) keeps the eight leading bits of f.  Values inside bfloat16's normal range
+    only (the layer's outputs are); zeros, infinities and NaN pass through.
+    """
+    v = np.asarray(v, dtype=np.float64)
+    f, p = np.frexp(v)
+    with np.errstate(invalid="ignore"):
+        r = np.ldexp(np.rint(f * 256.0), p - 8)
+    return np.where(np.isfinite(v), r, v)
+
+
+def bf16_half_ulp(v: np.ndarray) -> np.ndarray:
+    """Half the spacing of bfloat16 values at each |v|: the most a correctly rounded value differs from v."""
+    v = np.abs(np.asarray(v, dtype=np.float64))
+    _, p = np.frexp(v)
+    return np.where(v > 0.0, np.ldexp(1.0, p - 9), 0.0)

@@ -22,6 +22,8 @@ from .binding import (  # noqa: F401
     project_lowrank,
     new_workspace,
     linear,
+    linear_ex,
+    linear_batched_ex,
     linear_batched,
     batched_workspace_bytes,
     linear_static,

@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
             "lqer_linear": (i, [vp, i, vp, vp, vp, sz]),
             "lqer_linear_stream": (i, [vp, i, vp, vp, vp, sz, vp]),
             "lqer_linear_static": (i, [vp, i, vp, vp, vp]),
+            "lqer_linear_ex": (i, [vp, i, i, vp, vp, i, vp, sz, vp]),
+            "lqer_linear_batched_ex": (i, [C.POINTER(Call), i, i, i, vp, sz, vp]),
             "lqer_linear_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
             "lqer_batched_workspace_bytes": (i, [C.POINTER(Call), i, C.POINTER(sz)]),
             "lqer_linear_host": (i, [vp, i, vp, vp, vp, sz, vp]),
@@ -223,6 +225,20 @@ def linear(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y: torch.Tensor 
     return Y
 
 
+_DTYPES = {torch.float32: 0, torch.bfloat16: 1}
+
+
+def linear_ex(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y: torch.Tensor | None = None,
+              out_dtype: torch.dtype = torch.float32, stream=None):
+    """The layer with fp32 or bf16 activations in and out (the types are taken from X and Y / out_dtype)."""
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, P.N), dtype=out_dtype, device=X.device)
+    _check(lib().lqer_linear_ex(_dev(X), _DTYPES[X.dtype], M, P.ptr, _dev(Y), _DTYPES[Y.dtype], ws.data_ptr(), ws.numel(),
+                                _stream(stream)), "lqer_linear_ex")
+    return Y
+
+
 def linear_static(X: torch.Tensor, P: PackedWeights, Y: torch.Tensor | None = None, stream=None):
     """The layer without a caller-provided workspace: the scratch is a fixed array inside the
     library (STATIC_SCRATCH_BYTES); nothing is allocated by the call (Y must be given for that to
@@ -238,12 +254,12 @@ def linear_static(X: torch.Tensor, P: PackedWeights, Y: torch.Tensor | None = No
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
-def make_calls(items) -> "C.Array":
+def make_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype: torch.dtype = torch.float32) -> "C.Array":
     """items: iterable of (X, PackedWeights, Y) -> a host array of lqer_call_t."""
     items = list(items)
     arr = (Call * len(items))()
     for j, (X, P, Y) in enumerate(items):
-        arr[j] = Call(_dev(X, torch.float32), X.shape[0], P.ptr, _dev(Y, torch.float32))
+        arr[j] = Call(_dev(X, x_dtype), X.shape[0], P.ptr, _dev(Y, y_dtype))
     return arr
 
 
@@ -259,6 +275,12 @@ def linear_batched(calls, ws: torch.Tensor, stream=None) -> None:
     arr = calls if isinstance(calls, C.Array) else make_calls(calls)
     _check(lib().lqer_linear_batched(arr, len(arr), ws.data_ptr(), ws.numel(), _stream(stream)),
            "lqer_linear_batched")
+
+
+def linear_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype: torch.dtype, stream=None) -> None:
+    """linear_batched with every X of x_dtype and every Y of y_dtype (fp32 or bf16); `calls` from make_calls(..., x_dtype, y_dtype)."""
+    _check(lib().lqer_linear_batched_ex(calls, len(calls), _DTYPES[x_dtype], _DTYPES[y_dtype], ws.data_ptr(), ws.numel(),
+                                        _stream(stream)), "lqer_linear_batched_ex")
 
 
 def linear_host(X_host: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y_host: torch.Tensor, stream=None):

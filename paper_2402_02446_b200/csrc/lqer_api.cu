@@ -168,7 +168,7 @@ static size_t small_slice_bytes(const PackedMeta& m, int M) {
   return xcat_bytes(m, M) + align_up(prologue_small_slot_bytes(m, M), 256) + align_up(small_gemm_partial_bytes(m, M), 256);
 }
 // A call of up to kSmallMaxM rows runs the column-owner decode kernel (M <= 4 where the layer fits it) or the small
-// prologue and the GEMM with the tokens on the N side; either finds its scratch behind the head.
+// prologue and the small-batch GEMM; either finds its scratch behind the head.
 static size_t small_bytes(const PackedMeta& m, int M) {
   const size_t a = small_slice_bytes(m, M), b = decode_cols_slot_bytes(m);
   return a > b ? a : b;
@@ -223,7 +223,7 @@ static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, 
     gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g]};
   }
   cudaError_t err = launch_prologue_small(pl, n, M, io.x_bf16, s);
-  if (err == cudaSuccess && !project_only) err = launch_gemm_tn(gl, n, M, io.y_bf16, dst, s);
+  if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_bf16, dst, s);
   return err;
 }
 
@@ -242,7 +242,7 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   const bool small = takes_small_path(path, M);
   if (project_only && !small) path = 3;
   // Paths 1 and 3 keep the SIMT-style prologue at every batch size; the others take the tensor-core one where it fits.
-  const bool tc_prologue = path != 1 && path != 3 && !io.x_bf16 && prologue_tc_fits(m, M, static_cast<const float*>(X), path == 6);
+  const bool tc_prologue = path != 1 && path != 3 && prologue_tc_fits(m, M, X, path == 6);
   if (path == 6) path = 4;
   if (workspace_bytes < call_bytes(m, M, small)) return LQER_ERR_BUFFER_TOO_SMALL;
   if ((st = check_arch()) != LQER_OK) return st;
@@ -261,17 +261,14 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
       err = run_small(&one, &m, 1, &slice, &tiles, &rows, dst, io, Tm, Te, project_only, s);
     }
   } else {
-    if (io.x_bf16 || io.y_bf16) return LQER_ERR_CONFIG;
-    if (path == 1 && M > 65535) return LQER_ERR_SHAPE;
-    const float* Xf = static_cast<const float*>(X);
-    float* Yf = static_cast<float*>(Y);
-    err = tc_prologue ? launch_prologue_tc(Xf, M, m, packed, xcat, Tm, Te, dst,
+    if (path == 1 && (M > 65535 || io.y_bf16)) return LQER_ERR_SHAPE;   // the checking kernel writes fp32 only
+    err = tc_prologue ? launch_prologue_tc(X, io.x_bf16, M, m, packed, xcat, Tm, Te, dst,
                                            reinterpret_cast<double*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M)),
                                            reinterpret_cast<int*>(wsb + pcount_offset(m)), kChainAlone, s)
-                      : launch_prologue(Xf, M, m, packed, xcat, Tm, Te, dst, s);
+                      : launch_prologue(X, io.x_bf16, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
-      err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, Yf, s)
-                        : launch_gemm_tc2_splitk(xcat, M, m, packed, Yf,
+      err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, static_cast<float*>(Y), s)
+                        : launch_gemm_tc2_splitk(xcat, M, m, packed, Y, io.y_bf16,
                                                  reinterpret_cast<float*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M) +
                                                                           align_up(prologue_tc_scratch_bytes(m, M), 256)),
                                                  dst, s);
@@ -322,7 +319,7 @@ static int prefill_run(const lqer_call_t* calls, int first, int n_calls, int lim
 // the same M <= kSmallMaxM, the same formats, any shapes, none of them served by the column-owner decode kernel; at most
 // `limit`, only as many as the workspace has slices for, and tile counters for.
 constexpr size_t kGroupRowCountOffset = 256 + 32768 * 4 + 16 * 256 * 8;   // the row-tile counter area at its highest position
-static int small_run(const lqer_call_t* calls, int first, int n_calls, int limit, size_t workspace_bytes,
+static int small_run(const lqer_call_t* calls, int first, int n_calls, int limit, size_t workspace_bytes, bool cols_ok,
                      PackedMeta* metas, size_t* need) {
   const int M = calls[first].M;
   const size_t head = align_up(kPersistMaxBytes, 256);
@@ -330,7 +327,7 @@ static int small_run(const lqer_call_t* calls, int first, int n_calls, int limit
   int n = 0, tiles = 0;
   while (first + n < n_calls && n < limit) {
     PackedMeta m;
-    if (calls[first + n].M != M || lookup(calls[first + n].packed, m) != LQER_OK || decode_cols_fits(m, M)) break;
+    if (calls[first + n].M != M || lookup(calls[first + n].packed, m) != LQER_OK || (cols_ok && decode_cols_fits(m, M))) break;
     if (n > 0 && !same_formats(metas[0], m)) break;
     if (tiles + m.n_tiles > 32768) break;
     const size_t sl = slices + small_slice_bytes(m, M);
@@ -341,7 +338,8 @@ static int small_run(const lqer_call_t* calls, int first, int n_calls, int limit
   if (need != nullptr) *need = head + slices;
   return n;
 }
-static lqer_status_t run_small_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace, cudaStream_t s) {
+static lqer_status_t run_small_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace, IoTypes io,
+                                     cudaStream_t s) {
   uint8_t* wsb = static_cast<uint8_t*>(workspace);
   uint8_t* slices[16];
   int* tile_counts[16];
@@ -355,7 +353,7 @@ static lqer_status_t run_small_group(const lqer_call_t* calls, int n, const Pack
     tiles += metas[g].n_tiles;
     row_counts[g] = reinterpret_cast<int*>(wsb + kGroupRowCountOffset) + 8 * g;
   }
-  return run_small(calls, metas, n, slices, tile_counts, row_counts, static_cast<DeviceStatus*>(workspace), IoTypes(), nullptr,
+  return run_small(calls, metas, n, slices, tile_counts, row_counts, static_cast<DeviceStatus*>(workspace), io, nullptr,
                    nullptr, false, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
 // The run of decode calls from calls[first] on that may share one launch of the column-owner kernel: one M, one set of
@@ -409,7 +407,7 @@ static int prologue_max_ctas() {
 // n prefill layers with one M: each layer's prologue into its own slice of the workspace, then ONE GEMM launch over
 // the tiles of all of them.
 static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const PackedMeta* metas, void* workspace,
-                                       cudaStream_t s) {
+                                       IoTypes io, cudaStream_t s) {
   const int M = calls[0].M;
   uint8_t* wsb = static_cast<uint8_t*>(workspace);
   DeviceStatus* dst = static_cast<DeviceStatus*>(workspace);
@@ -417,7 +415,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
   for (int g = 0; g < n; ++g) head = std::max(head, align_up(persist_bytes(metas[g]), 256));
   const void* xcats[8];
   const void* packed[8];
-  float* Ys[8];
+  void* Ys[8];
   // The prologues of the group share nothing but the status word: each has its slice of the workspace, and, while the
   // counter pairs last, its own range of them, so that each may overlap the tail of the one before.
   size_t count_base = 0;
@@ -462,7 +460,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
       if (ns == 1 || !squeezed || longest <= 1.35 * (double)total / prologue_max_ctas()) break;
       alone[idx[worst]] = true;
     }
-    const float* Xs[8];
+    const void* Xs[8];
     const void* pk[8];
     void* xc[8];
     double* parts[8];
@@ -490,7 +488,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
       }
       if (cnt == 0) continue;
       const int order = planned == 1 ? kChainAlone : launches == 0 ? kChainFirst : kChainLater;
-      if (launch_prologue_tc_group(Xs, M, ms, pk, xc, parts, counts, sp, cnt, nullptr, nullptr, dst, order, s) != cudaSuccess)
+      if (launch_prologue_tc_group(Xs, io.x_bf16, M, ms, pk, xc, parts, counts, sp, cnt, nullptr, nullptr, dst, order, s) != cudaSuccess)
         return LQER_ERR_CUDA;
       ++launches;
     }
@@ -502,13 +500,13 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
       int* counters = reinterpret_cast<int*>(wsb + count_base) + (own_counters ? (size_t)g * row_tiles * 2 : 0);
       const int order = !own_counters ? kChainAlone : g == 0 ? kChainFirst : kChainLater;
       cudaError_t err = prologue_tc_fits(m, M, X, false)
-                            ? launch_prologue_tc(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
+                            ? launch_prologue_tc(X, io.x_bf16, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
                                                  reinterpret_cast<double*>(xcat + xcat_bytes(m, M)), counters, order, s)
-                            : launch_prologue(X, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
+                            : launch_prologue(X, io.x_bf16, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
       if (err != cudaSuccess) return LQER_ERR_CUDA;
     }
   }
-  return launch_gemm_tc2_group(xcats, packed, Ys, metas, n, M, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+  return launch_gemm_tc2_group(xcats, packed, Ys, io.y_bf16, metas, n, M, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
 
 }  // namespace lqer
@@ -683,8 +681,13 @@ lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y, v
   return lqer_linear_stream(X, M, packed, Y, workspace, workspace_bytes, nullptr);
 }
 
-lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
-                                  void* stream) {
+}  // extern "C"
+
+// The batched entry points: independent calls share launches where the path is left at 0.  With 16-bit activations
+// at the boundary (io) the column-owner decode kernel, which reads and writes fp32, is not used.
+static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
+                                    void* stream, IoTypes io) {
+  const bool cols_ok = !io.x_bf16 && !io.y_bf16;
   if (calls == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
   // validate everything before the first launch
@@ -720,13 +723,13 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
     PackedMeta m0, metas[16];
     bool decode_group = false, small_group = false;
     if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
-      if (decode_cols_fits(m0, calls[i].M)) {
+      if (cols_ok && decode_cols_fits(m0, calls[i].M)) {
         n = decode_run(calls, i, n_calls, decode_cols_max_group(), workspace_bytes, metas, nullptr);
         if (n < 1) n = 1;
         decode_group = n > 1;
       } else if (calls[i].M <= kSmallMaxM) {
-        const int lim = std::min(gemm_tn_max_layers(), prologue_small_max_layers());
-        n = small_run(calls, i, n_calls, lim, workspace_bytes, metas, nullptr);
+        const int lim = std::min(gemm_small_max_layers(), prologue_small_max_layers());
+        n = small_run(calls, i, n_calls, lim, workspace_bytes, cols_ok, metas, nullptr);
         if (n < 1) n = 1;
         small_group = n > 1;
       } else if (calls[i].M > kGemmSplitMaxM) {   // batches in between run split K, each on its own
@@ -773,20 +776,50 @@ lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* w
         chain_set = set;
       } else if (small_group) {
         chain_open = false;
-        if ((st = run_small_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) return st;
+        if ((st = run_small_group(calls + i, n, metas, workspace, io, static_cast<cudaStream_t>(stream))) != LQER_OK) return st;
       } else {
         chain_open = false;
-        if ((st = run_prefill_group(calls + i, n, metas, workspace, static_cast<cudaStream_t>(stream))) != LQER_OK) return st;
+        if ((st = run_prefill_group(calls + i, n, metas, workspace, io, static_cast<cudaStream_t>(stream))) != LQER_OK) return st;
       }
     } else {
       chain_open = false;
-      lqer_status_t st = lqer_linear_stream(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace,
-                                            workspace_bytes, stream);
+      lqer_status_t st = run_linear(calls[i].X, calls[i].M, calls[i].packed, calls[i].Y, workspace, workspace_bytes,
+                                    static_cast<cudaStream_t>(stream), nullptr, nullptr, false, io);
       if (st != LQER_OK) return st;
     }
     i += n;
   }
   return LQER_OK;
+}
+
+static lqer_status_t io_types(lqer_dtype_t x_dtype, lqer_dtype_t y_dtype, IoTypes* io) {
+  if ((x_dtype != LQER_F32 && x_dtype != LQER_BF16) || (y_dtype != LQER_F32 && y_dtype != LQER_BF16)) return LQER_ERR_CONFIG;
+  io->x_bf16 = x_dtype == LQER_BF16;
+  io->y_bf16 = y_dtype == LQER_BF16;
+  return LQER_OK;
+}
+
+extern "C" {
+
+lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+  return linear_batched(calls, n_calls, workspace, workspace_bytes, stream, IoTypes());
+}
+
+lqer_status_t lqer_linear_batched_ex(const lqer_call_t* calls, int n_calls, lqer_dtype_t x_dtype, lqer_dtype_t y_dtype,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+  IoTypes io;
+  lqer_status_t st = io_types(x_dtype, y_dtype, &io);
+  if (st != LQER_OK) return st;
+  return linear_batched(calls, n_calls, workspace, workspace_bytes, stream, io);
+}
+
+lqer_status_t lqer_linear_ex(const void* X, lqer_dtype_t x_dtype, int M, const void* packed, void* Y, lqer_dtype_t y_dtype,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+  IoTypes io;
+  lqer_status_t st = io_types(x_dtype, y_dtype, &io);
+  if (st != LQER_OK) return st;
+  return run_linear(X, M, packed, Y, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), nullptr, nullptr, false, io);
 }
 
 lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes) {
@@ -821,7 +854,7 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
     } else if (c.M <= kSmallMaxM) {
       PackedMeta metas[16];
       size_t group_need = 0;
-      n = small_run(calls, i, n_calls, std::min(gemm_tn_max_layers(), prologue_small_max_layers()), ~(size_t)0, metas, &group_need);
+      n = small_run(calls, i, n_calls, std::min(gemm_small_max_layers(), prologue_small_max_layers()), ~(size_t)0, true, metas, &group_need);
       if (n < 1) n = 1;
       if (n > 1) need = std::max(need, group_need);
     } else if (c.M > kGemmSplitMaxM) {

@@ -129,10 +129,11 @@ inline int prologue_small_ranges(const PackedMeta& m, int M) {
 inline size_t prologue_small_slot_bytes(const PackedMeta& m, int M) {
   return (size_t)((M + 15) / 16) * prologue_small_ranges(m, M) * 16 * m.k_pad * 8;
 }
-// K chunks per 128-column tile of the small-batch GEMM, and weight stages (64 K) per chunk: as many work items per layer
-// as fit 148 CTAs in one round, at least eight stages per chunk.
+// The small-batch GEMM works on tiles of 256 output columns (two packed tiles).  K chunks per tile and weight stages
+// (64 K) per chunk: as many work items per layer as fit 148 CTAs in one round, at least eight stages per chunk.
+inline int small_gemm_col_tiles(const PackedMeta& m) { return (m.n_tiles + 1) / 2; }
 inline int small_gemm_chunk_stages(const PackedMeta& m) {
-  int c = 148 / m.n_tiles;
+  int c = 148 / small_gemm_col_tiles(m);
   int cap = m.k_slabs / 8;
   if (cap < 1) cap = 1;
   if (c > cap) c = cap;
@@ -145,7 +146,7 @@ inline int small_gemm_chunks(const PackedMeta& m) {
 }
 inline size_t small_gemm_partial_bytes(const PackedMeta& m, int M) {
   const int c = small_gemm_chunks(m);
-  return c > 1 ? (size_t)m.n_tiles * c * M * kTileN * 4 : 0;
+  return c > 1 ? (size_t)small_gemm_col_tiles(m) * c * M * 256 * 4 : 0;
 }
 // Scratch of the column-owner decode kernel: fp64 partial sums of T, [16 ranges of K][4 rows][k_pad].
 inline size_t decode_cols_slot_bytes(const PackedMeta& m) { return (size_t)16 * 4 * m.k_pad * 8; }
@@ -318,36 +319,36 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
                               uint8_t* Xe, cudaStream_t s);
 // X -> Xcat[:, 0:K64] (bf16 of the dequantised MXINT8 value) and T_q -> Xcat[:, K64:K64+k_pad];
 // optional int8 / exponent exports of T_q.
-cudaError_t launch_prologue(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
+cudaError_t launch_prologue(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s);
 // The same prologue with the projection on the tcgen05 int8 tensor cores: ranks up to 64, large batches.
-bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch);
+bool prologue_tc_fits(const PackedMeta& m, int M, const void* X, bool any_batch);
 // `partials`: prologue_tc_scratch_bytes(m, M) of scratch; `counters`: zeroed counter pairs of the workspace head,
 // one per row tile.  `order`: kChainAlone, or the place in a run of prologues that share no buffer or counter
 // (each later one overlaps the tail of the one before; the kernel after the run still finds all of them complete).
 enum ChainOrder { kChainAlone = 0, kChainFirst = 1, kChainLater = 2 };
-cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
+cudaError_t launch_prologue_tc(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                int order, cudaStream_t s);
 // The same for up to 8 layers with one M, one k_pad and one set of formats in ONE launch (a CTA per row tile and K range
 // of a layer, found by its index); prologue_tc_group_splits picks the K ranges per row tile so that the CTAs carry
 // about equal work and stay within one per SM.
 bool prologue_tc_group_splits(const PackedMeta* metas, int n, int M, int max_ctas, int* splits);
-cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const PackedMeta* metas, const void* const* packed,
+cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, const PackedMeta* metas, const void* const* packed,
                                      void* const* xcats, double* const* partials, int* const* counters,
                                      const int* splits, int n, int8_t* Tm, uint8_t* Te, DeviceStatus* st, int order,
                                      cudaStream_t s);
 cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                              cudaStream_t s);
-cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
                             DeviceStatus* st, cudaStream_t s);
 // Small batches: the layer's K range cut into gemm_splitk_ranges(m, M) ranges that run as layers of one launch;
 // `partials` holds (ranges - 1) * M * N floats (gemm_splitk_bytes).
-cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
                                    float* partials, DeviceStatus* st, cudaStream_t s);
 // Up to gemm_tc2_max_group() layers with one M in one launch (xcats, packed, Ys, metas: host arrays of n entries).
 int gemm_tc2_max_group();
-cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys,
+cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, void* const* Ys, bool y_bf16,
                                   const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s);
 // Small batches (M <= kSmallMaxM).  The prologue quantises X (fp32 or bf16) into Xcat and leaves T_q behind it; up to
 // prologue_small_max_layers() layers with one M and one set of formats per launch.
@@ -363,17 +364,18 @@ struct SmallPrologueLayer {
 };
 int prologue_small_max_layers();
 cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, cudaStream_t s);
-// The GEMM with the tokens on the N side of the MMA; up to gemm_tn_max_layers() layers with one M per launch.
+// The small-batch GEMM (tokens on the M side of a 64- or 128-row MMA, 256 weight columns on its N side); up to
+// gemm_small_max_layers() layers with one M per launch.
 struct SmallGemmLayer {
   const void* xcat;
   const void* packed;
   const PackedMeta* meta;
   void* Y;                    // [M, N] fp32 or bf16
   float* partials;            // small_gemm_partial_bytes of scratch (unused if the tiles have one chunk)
-  int* counters;              // one zeroed counter per 128-column tile
+  int* counters;              // one zeroed counter per 256-column tile
 };
-int gemm_tn_max_layers();
-cudaError_t launch_gemm_tn(const SmallGemmLayer* layers, int n, int M, bool y_bf16, DeviceStatus* st, cudaStream_t s);
+int gemm_small_max_layers();
+cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y_bf16, DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);

@@ -61,7 +61,7 @@ struct TensorMaps {                        // one activation map per layer of th
 struct Layer {
   const uint8_t* wsec;
   const uint8_t* bsec;
-  float* Y;
+  void* Y;                     // [M, N] fp32, or bf16 where Params::y_bf16 (never for the K ranges of a split layer)
   int N, K64;
   int n_tiles, k_slabs, r_blocks;
   int slab0, slab_stride;      // a layer may be a K range of a real layer (split K): its first weight slab, and the
@@ -77,9 +77,17 @@ struct Params {
   DeviceStatus* status;
   int M, m_tiles;              // row tiles of 256 (the same M for every layer)
   int lr_shift;
+  int y_bf16;                  // Y is bf16 (round to nearest even), else fp32
   long long wait_limit;        // bound of every wait, in clock cycles
   int stall;                   // test hook: the producers withhold the last stage of their last tile, so the waits run out
 };
+
+// Two fp32 bit patterns -> two bf16 (round to nearest even) in one word, the first in the low half.
+__device__ __forceinline__ uint32_t bf16x2_rn(uint32_t lo, uint32_t hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(hi)), "f"(__uint_as_float(lo)));
+  return d;
+}
 
 __device__ __forceinline__ int layer_of(const Params& p, int t) {
   int l = 0;
@@ -239,17 +247,28 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       tc_fence_after();
       const int row = mt * 2 * BM + (int)rank * BM + q * 32 + lane;
       const int ncols = min(BN, Nl - nt * BN);
-      float* yrow = p.L[layer].Y + (size_t)row * Nl + (size_t)nt * BN;
+      const size_t yoff = (size_t)row * Nl + (size_t)nt * BN;
+      float* yrow = static_cast<float*>(p.L[layer].Y) + yoff;
+      uint16_t* yrow16 = static_cast<uint16_t*>(p.L[layer].Y) + yoff;
       for (int c = 0; c < BN; c += 32) {
         if (c >= ncols) break;
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, r);
         tmem_ld_wait();
         if (row < p.M) {
+          if (p.y_bf16) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (c + 4 * j < ncols)
-              *reinterpret_cast<uint4*>(yrow + c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+            for (int j = 0; j < 4; ++j)
+              if (c + 8 * j < ncols)                      // N is a multiple of 8
+                *reinterpret_cast<uint4*>(yrow16 + c + 8 * j) =
+                    make_uint4(bf16x2_rn(r[8 * j], r[8 * j + 1]), bf16x2_rn(r[8 * j + 2], r[8 * j + 3]),
+                               bf16x2_rn(r[8 * j + 4], r[8 * j + 5]), bf16x2_rn(r[8 * j + 6], r[8 * j + 7]));
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (c + 4 * j < ncols)
+                *reinterpret_cast<uint4*>(yrow + c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          }
         }
       }
       tc_fence_before();
@@ -412,11 +431,13 @@ __global__ void __launch_bounds__(256) splitk_sum_kernel(float4* __restrict__ Y,
 
 // Small batches have few tiles; their K range is cut into ranges that run as layers of one launch, the first into Y,
 // the others into scratch that a second kernel adds to Y in a fixed order.
-cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Yv, bool y_bf16,
                                    float* partials, DeviceStatus* st, cudaStream_t s) {
   using namespace tc2;
   const int C = gemm_splitk_ranges(m, M);
-  if (C < 2) return launch_gemm_tc2(xcat, M, m, packed, Y, st, s);
+  // a 16-bit Y cannot collect the ranges' sums: such a layer runs whole
+  if (C < 2 || y_bf16) return launch_gemm_tc2(xcat, M, m, packed, Yv, y_bf16, st, s);
+  float* Y = static_cast<float*>(Yv);
   if ((m.N & 3) != 0) return cudaErrorInvalidValue;
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
@@ -454,6 +475,7 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
   p.status = st;
   p.M = M;
   p.lr_shift = m.lr_bits - 2;
+  p.y_bf16 = 0;
   cudaError_t e = launch_params(tmaps, p, s);
   if (e != cudaSuccess) return e;
   const size_t quads = (size_t)M * m.N / 4;
@@ -464,9 +486,9 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
   return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
+cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
                             DeviceStatus* st, cudaStream_t s) {
-  return launch_gemm_tc2_group(&xcat, &packed, &Y, &m, 1, M, st, s);
+  return launch_gemm_tc2_group(&xcat, &packed, &Y, y_bf16, &m, 1, M, st, s);
 }
 
 int gemm_tc2_max_group() { return tc2::MAX_GROUP; }
@@ -474,7 +496,7 @@ int gemm_tc2_max_group() { return tc2::MAX_GROUP; }
 // n layers with one M (shapes may differ, formats must not) as ONE launch: the tiles of all layers form one list that
 // the CTA pairs walk, so the pairs idle only at the end of the whole list, and set-up and the last epilogue are paid
 // once.  Layers with more K stages per tile come first in the list.
-cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, float* const* Ys,
+cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, void* const* Ys, bool y_bf16,
                                   const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s) {
   using namespace tc2;
   if (n < 1 || n > MAX_GROUP) return cudaErrorInvalidValue;
@@ -520,6 +542,7 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
   p.status = st;
   p.M = M;
   p.lr_shift = metas[0].lr_bits - 2;
+  p.y_bf16 = y_bf16 ? 1 : 0;
   return launch_params(tmaps, p, s);
 }
 

@@ -81,6 +81,7 @@ struct Params {
   long long wait_limit;     // bound of every wait, in clock cycles
   int a_bits, lr_bits, exp_min, exp_max;
   int order;                // ChainOrder: where the wait for the previous kernel sits
+  int x_bf16;               // X is bf16 (a stage of the ring then holds 16 KB), else fp32
   size_t ldx;               // columns of Xcat
 };
 
@@ -292,10 +293,20 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     for (int s = 0; s < n_stages && ok; ++s) {
       const int rs = s % RAW_SLOTS, xs = s % X_SLOTS;
       if (!warp_wait(raw_full(rs), (s / RAW_SLOTS) & 1, abort_flag)) { ok = false; break; }
-      const float4* src = reinterpret_cast<const float4*>(raw_base + rs * RAW_BYTES) + rb * 16 + c4;
       float4 xr[QUADS];
+      if (p.x_bf16) {
+        const uint2* src = reinterpret_cast<const uint2*>(raw_base + rs * RAW_BYTES) + rb * 16 + c4;
 #pragma unroll
-      for (int i = 0; i < QUADS; ++i) xr[i] = src[i * C::ROW_STEP * 16];
+        for (int i = 0; i < QUADS; ++i) {
+          const uint2 v = src[i * C::ROW_STEP * 16];
+          xr[i] = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
+                              __uint_as_float(v.y & 0xFFFF0000u));
+        }
+      } else {
+        const float4* src = reinterpret_cast<const float4*>(raw_base + rs * RAW_BYTES) + rb * 16 + c4;
+#pragma unroll
+        for (int i = 0; i < QUADS; ++i) xr[i] = src[i * C::ROW_STEP * 16];
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(raw_empty(rs));     // the values are in registers: the slot can be refilled
       if (!warp_wait(xq_empty(xs), ((s / X_SLOTS) & 1) ^ 1, abort_flag)) { ok = false; break; }
@@ -392,7 +403,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
       for (int s = 0; s < n_stages; ++s) {
         const int rs = s % RAW_SLOTS;
         if (!parked_wait(raw_empty(rs), ((s / RAW_SLOTS) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(raw_full(rs), RAW_BYTES);       // rows and columns outside X arrive as zeros
+        mbar_expect_tx(raw_full(rs), p.x_bf16 ? RAW_BYTES / 2 : RAW_BYTES);       // rows and columns outside X arrive as zeros
         tma_load_2d(smem_u32(raw_base + rs * RAW_BYTES), tmap_x, (pan_lo * 2 + s) * STAGE_COLS, row0, raw_full(rs));
       }
     }
@@ -510,7 +521,7 @@ static cudaError_t launch_kp(const TensorMaps& tmaps, const GroupParams& gp, int
 }  // namespace ptc
 
 // The tensor-core prologue serves ranks padded to 16, 32 or 64 and batches large enough to give most SMs a CTA.
-bool prologue_tc_fits(const PackedMeta& m, int M, const float* X, bool any_batch) {
+bool prologue_tc_fits(const PackedMeta& m, int M, const void* X, bool any_batch) {
   if (!prologue_tc_rank_ok(m) || (M + 127) / 128 > kPrologueRowTiles) return false;
   if ((reinterpret_cast<uintptr_t>(X) & 15) != 0) return false;
   return any_batch || M >= 1024;
@@ -556,7 +567,7 @@ bool prologue_tc_group_splits(const PackedMeta* metas, int n, int M, int max_cta
 
 // n layers (one M, one k_pad, one set of formats) in ONE launch.  splits[g] K ranges per row tile of layer g; the
 // caller sees to it that the CTAs (row tiles x splits, summed) are at most one per SM.  Tm / Te: for n == 1 only.
-cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const PackedMeta* metas, const void* const* packed,
+cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, const PackedMeta* metas, const void* const* packed,
                                      void* const* xcats, double* const* partials, int* const* counters,
                                      const int* splits, int n, int8_t* Tm, uint8_t* Te, DeviceStatus* st, int order,
                                      cudaStream_t s) {
@@ -575,10 +586,10 @@ cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const Packed
     const PackedMeta& m = metas[g];
     if (m.k_pad != metas[0].k_pad) return cudaErrorInvalidValue;
     const cuuint64_t dims[2] = {(cuuint64_t)m.K, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)m.K * 4};
+    const cuuint64_t strides[1] = {(cuuint64_t)m.K * (x_bf16 ? 2 : 4)};
     const cuuint32_t box[2] = {STAGE_COLS, ROWS};
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&tmaps.m[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(Xs[g]), dims, strides, box, estr,
+    if (enc(&tmaps.m[i], x_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(Xs[g]), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
@@ -595,6 +606,7 @@ cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const Packed
     p.wait_limit = limit;
     p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
     p.order = order;
+    p.x_bf16 = x_bf16 ? 1 : 0;
     p.ldx = xcat_cols(m);
     gp.cta_begin[i] = begin;
     if (i < n) begin += ((M + ROWS - 1) / ROWS) * p.splits;
@@ -607,12 +619,12 @@ cudaError_t launch_prologue_tc_group(const float* const* Xs, int M, const Packed
   }
 }
 
-cudaError_t launch_prologue_tc(const float* X, int M, const PackedMeta& m, const void* packed, void* xcat,
+cudaError_t launch_prologue_tc(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                int order, cudaStream_t s) {
   const int sms = sm_count();
   const int splits = prologue_tc_splits(m, M, sms > 0 && sms < kPrologueMaxCtas ? sms : kPrologueMaxCtas);
-  return launch_prologue_tc_group(&X, M, &m, &packed, &xcat, &partials, &counters, &splits, 1, Tm, Te, st, order, s);
+  return launch_prologue_tc_group(&X, x_bf16, M, &m, &packed, &xcat, &partials, &counters, &splits, 1, Tm, Te, st, order, s);
 }
 
 }  // namespace lqer

@@ -388,7 +388,7 @@ def test_batched_decode_stretch_quantises_activations_ahead(M):
 @pytest.mark.parametrize("M", [5, 16, 40])
 def test_batched_small_batches_share_two_launches(M):
     # nine independent calls with one M above the column-owner kernel's range: layers of three shapes (one without a
-    # low-rank part) run as ONE launch of the small prologue and ONE launch of the tokens-on-N GEMM over the work items
+    # low-rank part) run as ONE launch of the small prologue and ONE launch of the small-batch GEMM over the work items
     # of all of them; every layer must give what it gives alone, bit for bit (the K chunks of a tile depend on the
     # shape alone), and twice in a row (counters are left at zero).
     shapes = [gen.LayerSpec("sg_a", M=M, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=171),

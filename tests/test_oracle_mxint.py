@@ -143,3 +143,24 @@ def test_padding_is_neutral():
     amax = np.abs(b).max(axis=0)
     assert np.array_equal(e[0], np.floor(np.log2(amax)).astype(np.int64))
     assert not m[8:].any()
+
+
+def test_round_bf16_hand_cases_and_library_agreement():
+    # bfloat16 keeps 8 significant bits: the spacing in [1, 2) is 2^-7
+    cases = [(1.0 + 2.0 ** -8, 1.0),                       # exact tie, lower neighbour has the even mantissa
+             (1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -6),       # exact tie, upper neighbour is even
+             (1.0 + 2.0 ** -8 + 2.0 ** -20, 1.0 + 2.0 ** -7),
+             (-0.3, -0.30078125), (3.14159, 3.140625), (255.5, 256.0), (0.0, 0.0), (1e-3, 0.00099945068359375)]
+    for v, want in cases:
+        assert mxint.round_bf16(np.array([v]))[0] == want, v
+    # a correctly rounded value is within half a spacing, and the result is a fixed point
+    g = np.random.default_rng(5)
+    x = g.standard_normal(4000) * np.exp2(g.integers(-20, 20, 4000))
+    r = mxint.round_bf16(x)
+    assert np.all(np.abs(r - x) <= mxint.bf16_half_ulp(x))
+    assert np.array_equal(mxint.round_bf16(r), r)
+    # against a library's conversion (fp32 inputs, so that both start from the same number)
+    torch = pytest.importorskip("torch")
+    x32 = x.astype(np.float32)
+    lib = torch.from_numpy(x32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(mxint.round_bf16(x32), lib)

@@ -66,15 +66,15 @@ def test_static_scratch_rejects_what_does_not_fit():
 
 
 def test_static_scratch_boundary_on_a_4096_layer_and_no_allocation():
-    # K = N = 4096, rank 32: the call's own need decides.  M = 86 is the largest small batch that fits (the partial
-    # sums of the GEMM's K chunks grow with M), M = 87 is the first that is refused, and M = 300 fits again (no
+    # K = N = 4096, rank 32: the call's own need decides.  M = 57 is the largest small batch that fits (the partial
+    # sums of the GEMM's K chunks grow with M), M = 58 is the first that is refused, and M = 300 fits again (no
     # split of K above 256 rows).  The calls that run must not change the amount of device memory in use.
     spec = gen.LayerSpec("static_4096", M=300, K=4096, N=4096, k=32, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=94)
     P = _layer(spec)
     Xall = torch.from_numpy(gen.make_activations(spec)).to(DEV)
     ws = L.new_workspace(spec.M, P)
     refused = binding.STATUS_NAMES.index("LQER_ERR_STATIC_SCRATCH")
-    for M, fits in ((86, True), (87, False), (300, True), (16, True)):
+    for M, fits in ((57, True), (58, False), (300, True), (16, True)):
         assert (L.call_workspace_bytes(M, spec.K, spec.N, spec.k) <= binding.STATIC_SCRATCH_BYTES) == fits
         X = Xall[:M].contiguous()
         Y = torch.full((M, spec.N), float("nan"), dtype=torch.float32, device=DEV)
