@@ -75,12 +75,13 @@ struct Params {
   int M;
   int lr_shift;
   int y_bf16;                  // Y is bf16 (round to nearest even), else fp32
+  int x_rows;                  // rows of an activation tile that TMA fills: M rounded up to 8 (the rest stay zero)
   long long wait_limit;
   int stall;                   // test hook: the producer withholds the last stage of its last item
 };
 
 struct TensorMaps {
-  CUtensorMap m[MAX_LAYERS];   // Xcat of each layer: bf16 [M, K64 + k_pad], box 64 x MT
+  CUtensorMap m[MAX_LAYERS];   // Xcat of each layer: bf16 [M, K64 + k_pad], box 64 x x_rows
 };
 
 struct Item {
@@ -118,6 +119,41 @@ __device__ __forceinline__ void store_y4(void* Y, size_t idx, float4 v, int y_bf
     *reinterpret_cast<float4*>(static_cast<float*>(Y) + idx) = v;
 }
 
+// Y of one 256-column tile = the sum of its chunks' partials, in chunk order (the same sum whoever computes it), by
+// `nthreads` threads (a multiple of 64): a thread per four columns, nthreads / 64 token rows per pass; the chunk loads
+// of four rows are in flight together.
+__device__ __forceinline__ void reduce_tile(const Params& p, const Layer& ly, int tile, int tid, int nthreads) {
+  const int col0 = tile * BN, c4 = (tid & 63) * 4, trow0 = tid >> 6, rstep = nthreads >> 6;
+  const bool quad_ok = col0 + c4 < ly.N;                                   // N is a multiple of 8: the quad is whole
+  const float* p0 = ly.partials + ((size_t)tile * ly.chunks * p.M) * BN + c4;
+  const size_t chunk_stride = (size_t)p.M * BN;
+  for (int t0 = trow0; t0 < p.M; t0 += 4 * rstep) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int cb = 0; cb < ly.chunks; cb += 4) {
+      float4 t[4][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          t[u][c] = (cb + c < ly.chunks && t0 + rstep * u < p.M)
+                        ? __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)(cb + c) * chunk_stride + (size_t)(t0 + rstep * u) * BN))
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (cb + c < ly.chunks) { v[u].x += t[u][c].x; v[u].y += t[u][c].y; v[u].z += t[u][c].z; v[u].w += t[u][c].w; }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int tk = t0 + rstep * u;
+      if (tk < p.M && quad_ok) store_y4(ly.Y, (size_t)tk * ly.N + col0 + c4, v[u], p.y_bf16);
+    }
+  }
+}
+
 template <int MT, int PK_SLOTS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constant__ Params p) {
@@ -129,6 +165,7 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BARS);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
   int* last_flag = reinterpret_cast<int*>(tmem_slot + 1);
+  int* deferred = reinterpret_cast<int*>(tmem_slot + 6);       // item whose chunks the whole CTA adds up at the end, or -1
   volatile WaitState* abort_flag = reinterpret_cast<volatile WaitState*>(tmem_slot + 2);
 
   const uint32_t bar0 = smem_u32(bars);
@@ -150,10 +187,17 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 4); }
     abort_flag->abort = 0;
     abort_flag->limit = p.wait_limit;
+    *deferred = -1;
     fence_barrier_init();
     fence_proxy_async_smem();
   }
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+  // rows of the activation tiles beyond the batch are zero for the whole launch: TMA only ever writes the first x_rows
+  for (int i = threadIdx.x; i < PK_SLOTS * (C::X_TILE_BYTES / 16); i += NUM_THREADS) {
+    const int slot = i / (C::X_TILE_BYTES / 16), o = i % (C::X_TILE_BYTES / 16);
+    if (o * 16 >= p.x_rows * 128) *reinterpret_cast<uint4*>(pk_base + slot * C::PK_SLOT_BYTES + o * 16) = make_uint4(0u, 0u, 0u, 0u);
+  }
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -170,7 +214,7 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
       int npend = 0;
       bool waited = false;
       auto load_x = [&](int slot, int layer, int xcol) {
-        mbar_expect_tx(x_full(slot), C::X_TILE_BYTES);       // rows beyond the batch arrive as zeros
+        mbar_expect_tx(x_full(slot), p.x_rows * 128);        // rows of the box beyond the batch arrive as zeros
         tma_load_2d(smem_u32(pk_base + slot * C::PK_SLOT_BYTES), &tmaps.m[layer], xcol, 0, x_full(slot));
       };
       auto flush = [&]() {
@@ -306,38 +350,14 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
         if (et == 0) *last_flag = (atomicAdd(ly.counters + it.tile, 1) == ly.chunks - 1) ? 1 : 0;
         epilogue_barrier();
         if (*last_flag != 0) {
-          __threadfence();
-          // a thread per four columns, two token rows per pass; the chunk loads of four rows are in flight together
-          const int c4 = (et & 63) * 4, trow0 = et >> 6;
-          const bool quad_ok = col0 + c4 < ly.N;
-          const float* p0 = ly.partials + ((size_t)it.tile * ly.chunks * p.M) * BN + c4;
-          const size_t chunk_stride = (size_t)p.M * BN;
-          for (int t0 = trow0; t0 < p.M; t0 += 8) {
-            float4 v[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int cb = 0; cb < ly.chunks; cb += 4) {
-              float4 t[4][4];
-#pragma unroll
-              for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                  t[u][c] = (cb + c < ly.chunks && t0 + 2 * u < p.M)
-                                ? __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)(cb + c) * chunk_stride + (size_t)(t0 + 2 * u) * BN))
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-              for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int c = 0; c < 4; ++c)                // chunk order: the same sum whoever computes it
-                  if (cb + c < ly.chunks) { v[u].x += t[u][c].x; v[u].y += t[u][c].y; v[u].z += t[u][c].z; v[u].w += t[u][c].w; }
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int tk = t0 + 2 * u;
-              if (tk < p.M && quad_ok) store_y4(ly.Y, (size_t)tk * ly.N + col0 + c4, v[u], p.y_bf16);
-            }
+          if (i + num_ctas >= num_items) {
+            // the CTA's last item: every other role is about to fall idle, so the whole CTA adds the chunks up at the end
+            if (et == 0) *deferred = i;
+          } else {
+            __threadfence();
+            reduce_tile(p, ly, it.tile, et, 128);
+            if (et == 0) ly.counters[it.tile] = 0;    // zero again for the next call
           }
-          if (et == 0) ly.counters[it.tile] = 0;      // zero again for the next call
         }
         epilogue_barrier();                         // last_flag may be rewritten only after everyone has read it
       }
@@ -408,7 +428,13 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
   }
 
   // ------------------------------------------------------------------ teardown
-  __syncthreads();                      // every role is done (or has given up): the flag below is final for this CTA
+  __syncthreads();                      // every role is done (or has given up): the flags below are final for this CTA
+  if (*deferred >= 0 && abort_flag->abort == 0) {
+    const Item it = item_of(p, *deferred);
+    __threadfence();
+    reduce_tile(p, p.L[it.layer], it.tile, threadIdx.x, NUM_THREADS);
+    if (threadIdx.x == 0) p.L[it.layer].counters[it.tile] = 0;     // zero again for the next call
+  }
   if (abort_flag->abort != 0) {
     const long long t0 = clock64();
     while (clock64() - t0 < 400000) { }
@@ -470,6 +496,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   EncodeTiledFn enc = encode_fn();
   if (enc == nullptr) return cudaErrorNotSupported;
   const int MT = M <= 64 ? 64 : 128;
+  const int x_rows = (M + 7) / 8 * 8;
   TensorMaps tmaps;
   Params p;
   int item_begin = 0;
@@ -479,7 +506,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
     if (m.lr_bits != layers[0].meta->lr_bits) return cudaErrorInvalidValue;
     const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
-    const cuuint32_t box[2] = {BK, (cuuint32_t)MT};
+    const cuuint32_t box[2] = {BK, (cuuint32_t)x_rows};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&tmaps.m[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(src.xcat), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -506,6 +533,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   p.M = M;
   p.lr_shift = layers[0].meta->lr_bits - 2;
   p.y_bf16 = y_bf16 ? 1 : 0;
+  p.x_rows = x_rows;
   p.wait_limit = wait_limit_cycles();
   p.stall = take_stall(kFamDecode) ? 1 : 0;
   const int sms = sm_count();
