@@ -205,8 +205,14 @@ lqer_status_t lqer_linear_static(const float* X, int M, const void* packed, floa
  *    prologues into separate slices of the workspace and then ONE GEMM launch over the tiles of
  *    all of them - if the workspace holds lqer_batched_workspace_bytes(calls, n_calls); with a
  *    smaller workspace (at least the largest lqer_workspace_bytes of the calls) fewer calls, or
- *    none, share a launch.
- * Results do not depend on the sharing. */
+ *    none, share a launch;
+ *  - up to 16 consecutive calls with one M <= 128 that the decode kernel does not serve (any shapes,
+ *    one set of formats) run as ONE launch of the small prologue and ONE launch of the small-batch
+ *    GEMM over the work items of all of them, under the same condition on the workspace.
+ * In the first two cases a result does not depend on the sharing, bit for bit.  In the third the
+ * contraction of a tile is cut into fewer K chunks when layers share a launch, so a result may
+ * differ from the single call's in its last bits (both within the layer's tolerance); it is
+ * reproducible for the same sequence of calls. */
 lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes);
 lqer_status_t lqer_linear_batched(const lqer_call_t* calls, int n_calls,
                                   void* workspace, size_t workspace_bytes, void* stream);

@@ -500,6 +500,14 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   TensorMaps tmaps;
   Params p;
   int item_begin = 0;
+  // K chunks per tile.  A layer alone is cut as its shape says (small_gemm_chunks: enough work items for every SM).
+  // Layers that share a launch bring many tiles between them, and every chunk costs a pass of partial sums through
+  // L2, so they are cut less: just enough for about two work items per SM in all, never more than alone (the scratch
+  // is sized for that).  The sums of a tile are then grouped differently, so a layer's result in a shared launch
+  // may differ from its result alone in the last bits; it is the same whenever the same layers share a launch.
+  int total_tiles = 0;
+  for (int i = 0; i < n; ++i) total_tiles += small_gemm_col_tiles(*layers[i].meta);
+  const int group_chunks = (296 + total_tiles - 1) / total_tiles;
   for (int i = 0; i < MAX_LAYERS; ++i) {
     const SmallGemmLayer& src = layers[i < n ? i : 0];
     const PackedMeta& m = *src.meta;
@@ -522,8 +530,10 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
     ly.N = m.N; ly.K64 = m.K64;
     ly.n_tiles = m.n_tiles; ly.k_slabs = m.k_slabs; ly.r_blocks = m.r_blocks;
     ly.spt = m.k_slabs + (m.r_blocks + 1) / 2;
-    ly.chunks = small_gemm_chunks(m);
-    ly.chunk_stages = small_gemm_chunk_stages(m);
+    int want = small_gemm_chunks(m);
+    if (n > 1 && group_chunks < want) want = group_chunks;
+    ly.chunk_stages = (m.k_slabs + want - 1) / want;
+    ly.chunks = (m.k_slabs + ly.chunk_stages - 1) / ly.chunk_stages;
     ly.item_begin = item_begin;
     if (i < n) item_begin += small_gemm_col_tiles(m) * ly.chunks;
   }

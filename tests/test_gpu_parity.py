@@ -389,8 +389,10 @@ def test_batched_decode_stretch_quantises_activations_ahead(M):
 def test_batched_small_batches_share_two_launches(M):
     # nine independent calls with one M above the column-owner kernel's range: layers of three shapes (one without a
     # low-rank part) run as ONE launch of the small prologue and ONE launch of the small-batch GEMM over the work items
-    # of all of them; every layer must give what it gives alone, bit for bit (the K chunks of a tile depend on the
-    # shape alone), and twice in a row (counters are left at zero).
+    # of all of them.  Layers that share a launch are cut into fewer K chunks than alone, so a result may differ from
+    # the single call's in the last bits: every one is held against the oracle, the quantised operands (which do not
+    # depend on the chunks) make the two agree to well within the tolerance, and a second run of the same batch must
+    # reproduce the first bit for bit (counters are left at zero, the grouping is a function of the calls alone).
     shapes = [gen.LayerSpec("sg_a", M=M, K=1024, N=640, k=40, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=171),
               gen.LayerSpec("sg_b", M=M, K=2112, N=264, k=16, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=172),
               gen.LayerSpec("sg_c", M=M, K=512, N=1032, k=0, calib_rows=64, outlier_frac=0.01, outlier_scale=20.0, seed=173)]
@@ -406,18 +408,28 @@ def test_batched_small_batches_share_two_launches(M):
     Yb = [torch.full((M, base[j][0].N), float("nan"), dtype=torch.float32, device=DEV) for j in order]
     calls = L.make_calls([(x, base[j][2], y) for x, j, y in zip(Xs, order, Yb)])
     ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    first = None
     for rep in range(2):
         launches = L.launch_count()
         L.linear_batched(calls, ws)
         torch.cuda.synchronize()
         assert L.poll_status(ws) == 0
         assert L.launch_count() - launches == 2
+        if first is None:
+            first = [y.clone() for y in Yb]
+            for y in Yb:
+                y.fill_(float("nan"))
+        else:
+            for a, b in zip(first, Yb):
+                assert torch.equal(a, b)
     ws1 = torch.zeros(max(L.workspace_bytes(M, sp.K, sp.N, sp.k) for sp, _, _ in base), dtype=torch.uint8, device=DEV)
     for i, (x, j, yb) in enumerate(zip(Xs, order, Yb)):
-        assert torch.equal(L.linear(x, base[j][2], ws1), yb), (i, base[j][0].name)
-    for i in (0, 1, 2):
-        sp, P, _ = base[order[i]]
-        assert worst_ratio(Yb[i].cpu().numpy(), olqer.forward(Xs[i].cpu().numpy(), P)) <= 1.0, sp.name
+        sp, P, Pg = base[j]
+        ref = olqer.forward(x.cpu().numpy(), P)
+        assert worst_ratio(yb.cpu().numpy(), ref) <= 1.0, (i, sp.name)
+        ys = L.linear(x, Pg, ws1)
+        assert worst_ratio(ys.cpu().numpy(), ref) <= 1.0, (i, sp.name)
+        assert float(np.max(np.abs((ys - yb).cpu().numpy().astype(np.float64)) / ref.tol)) <= 0.5, (i, sp.name)
     for _, _, Pg in base:
         Pg.release()
 
