@@ -17,6 +17,7 @@ roofline of the dominant kernel and the CPU oracle timed on a bounded sample.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import hashlib
 import json
 import os
@@ -76,11 +77,14 @@ def layer_flops(M: int, K: int, N: int, k: int) -> float:
     return 2.0 * M * ((K + k) * N + K * k)
 
 
+W_BITS = 4          # mantissa bits of W_q of this run (--w-bits)
+
+
 def layer_weight_bytes(K: int, N: int, k: int) -> float:
-    """Algorithmic bytes of the stored operands: 4-bit + 1 exponent byte per 16 for W_q,
+    """Algorithmic bytes of the stored operands: w_bits + 1 exponent byte per 16 for W_q,
     8-bit + 1 exponent byte per 16 for A_k and B_k (rank padded to a multiple of 16)."""
     k_pad = (k + 15) // 16 * 16
-    return 0.5625 * K * N + 1.0625 * (k * K + k_pad * N)
+    return (W_BITS / 8.0 + 0.0625) * K * N + 1.0625 * (k * K + k_pad * N)
 
 
 def measured_peaks() -> dict:
@@ -376,10 +380,13 @@ def run_ours(args) -> None:
     layers = args.layers
     cfg = L.default_config()
     cfg.a_bits = args.a_bits
+    cfg.w_bits = args.w_bits
     packed, shapes = [], []
     for layer in range(layers):
         for which in range(len(gen.STACK_LINEARS)):
             spec = gen.config_stack(layer, which, M_PREFILL)
+            if args.rank is not None:
+                spec = dataclasses.replace(spec, k=args.rank)
             W = gen.make_weight_device(spec, dev)
             A, B = gen.make_random_factors_device(spec, dev)
             packed.append(L.prepare_weights(W, A, B, cfg))
@@ -569,8 +576,11 @@ def run_ours(args) -> None:
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
             "config": {"workload": (WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]") +
-                                   ("" if args.a_bits == 8 else f" [activations MXINT{args.a_bits}]"),
-                       "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32, "a_bits": args.a_bits,
+                                   ("" if args.a_bits == 8 else f" [activations MXINT{args.a_bits}]") +
+                                   ("" if args.w_bits == 4 else f" [weights MXINT{args.w_bits}]") +
+                                   ("" if args.rank is None else f" [rank {args.rank}]"),
+                       "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32 if args.rank is None else args.rank,
+                       "a_bits": args.a_bits, "w_bits": args.w_bits,
                        "shared_launches": "lqer_linear_batched runs consecutive independent calls together: up to 16 "
                                           "decode calls as one launch that divides the SMs among the layers (their "
                                           "activations quantised ahead by one kernel per 64 calls), up to 8 prefill "
@@ -606,11 +616,15 @@ def main() -> None:
     ap.add_argument("--layers", type=int, default=32, help="decoder layers of the stack (32 = the full workload)")
     ap.add_argument("--oracle-rows", type=int, default=2048, help="token rows of the oracle's bounded sample")
     ap.add_argument("--a-bits", type=int, default=8, help="mantissa bits of the activations: 8 (W4A8, the workload) or 6 (W4A6)")
+    ap.add_argument("--w-bits", type=int, default=4, help="mantissa bits of the weights: 4 (the workload) or 2 (W2A8, Section 4.4)")
+    ap.add_argument("--rank", type=int, default=None, help="rank of the correction of every linear (default 32, the workload)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the decode-layer, prefill-MLP and rank-sweep legs")
     ap.add_argument("--quick-configs", action="store_true", help="rank sweep at M = 1 and 512 only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    global W_BITS
+    W_BITS = args.w_bits
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -52,7 +52,7 @@ typedef enum {
 
 /* Format parameters (Section 3.1: b_l, b_h; Section 4.1: block size, exponent width). */
 typedef struct {
-  int w_bits;        /* mantissa bits of W_q: 4 */
+  int w_bits;        /* mantissa bits of W_q: 4 (default), or 2 (the W2A8 setting of Section 4.4: mantissas -1, 0, 1) */
   int a_bits;        /* mantissa bits of X and of T = X A_k: 3..8, default 8 (W4A8; 6 gives the W4A6 of Section 4.3) */
   int lr_bits;       /* mantissa bits of A_k, B_k: 8 */
   int block;         /* block size along the contraction dimension: 16 */

@@ -79,8 +79,8 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 static lqer_status_t check_config(const lqer_config_t* cfg) {
   if (cfg == nullptr) return LQER_ERR_NULL;
-  // activations (and T) take 3 to 8 mantissa bits (Section 4.3 compares W4A8 and W4A6); weights and factors are fixed
-  if (cfg->w_bits != 4 || cfg->a_bits < 3 || cfg->a_bits > 8 || cfg->lr_bits != 8 || cfg->block != 16) return LQER_ERR_CONFIG;
+  // activations (and T) take 3 to 8 mantissa bits (Section 4.3 compares W4A8 and W4A6); weights 4 or 2 (Section 4.4: W2A8)
+  if ((cfg->w_bits != 4 && cfg->w_bits != 2) || cfg->a_bits < 3 || cfg->a_bits > 8 || cfg->lr_bits != 8 || cfg->block != 16) return LQER_ERR_CONFIG;
   // every dequantised value must be a normal bf16 and every product a normal fp32
   if (cfg->exp_min < -56 || cfg->exp_max > 55 || cfg->exp_min > cfg->exp_max) return LQER_ERR_CONFIG;
   if (cfg->w_exp_min < -56 || cfg->w_exp_max > 55 || cfg->w_exp_min > cfg->w_exp_max) return LQER_ERR_CONFIG;
@@ -108,7 +108,7 @@ static void fill_meta(PackedMeta& m, int K, int N, int k, const lqer_config_t& c
   m.exp_min = c.exp_min; m.exp_max = c.exp_max; m.deterministic = 1;
   m.w_exp_min = c.w_exp_min; m.w_exp_max = c.w_exp_max;
   m.off_w = kHeaderBytes;
-  m.off_b = align_up(m.off_w + (size_t)m.n_tiles * m.k_slabs * kWTileBytes, 256);
+  m.off_b = align_up(m.off_w + (size_t)m.n_tiles * m.k_slabs * w_tile_bytes(m.w_bits), 256);
   m.off_a = align_up(m.off_b + (size_t)m.n_tiles * b_tile_bytes(m), 256);
   m.total_bytes = align_up(m.off_a + (size_t)(K / 16) * m.k_pad * 17, 256);
   m.checksum = meta_checksum(m);

@@ -22,6 +22,10 @@ namespace lqer {
 //   Within a 32-bit word, nibble position p holds k_local = {0,2,4,6,1,3,5,7}[p] of the
 //   word's eight consecutive K, offset-binary (mantissa + 8), so that
 //   (w >> 4i) & 0x000F000F yields the adjacent pair (2i, 2i+1).
+//   With 2-bit mantissas (w_bits == 2) a tile is 2048 bytes of crumbs [n 128][16 B] (one 32-bit word per 16-block:
+//   crumb i of the low half holds k_local = 2i, crumb i of the high half k_local = 2i + 1, offset-binary
+//   (mantissa + 1), so that (w >> 2i) & 0x00030003 yields the adjacent pair (2i, 2i+1)) followed by the same 512
+//   exponent bytes.
 // B section: per n_tile:  mantissas [rb][n 128][16 B int8]  then exps [rb][n 128]
 // A section: mantissas [K/16][k_pad][16 B int8]  then exps [K/16][k_pad]
 constexpr uint32_t kMagic = 0x5245514Cu;  // "LQER"
@@ -31,6 +35,9 @@ constexpr int kTileN = 128;
 constexpr int kSlabK = 64;
 constexpr int kWTileBytes = kTileN * kSlabK / 2 + kTileN * 4;  // 4608
 constexpr int kWTileNibbleBytes = kTileN * kSlabK / 2;          // 4096
+// Bytes of the mantissas of one weight tile, and of the whole tile (mantissas + 512 exponent bytes), by mantissa width.
+__host__ __device__ inline int w_mant_bytes(int w_bits) { return kTileN * kSlabK * w_bits / 8; }   // 4096 (4 bit), 2048 (2 bit)
+__host__ __device__ inline int w_tile_bytes(int w_bits) { return w_mant_bytes(w_bits) + kTileN * 4; }
 constexpr int kStatusBytes = 256;
 
 struct PackedMeta {

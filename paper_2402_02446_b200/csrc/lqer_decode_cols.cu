@@ -621,8 +621,9 @@ static size_t cols_smem_bytes(const PackedMeta& m, int M) {
   return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + 2 * kHoldMax * kWarps * kCg * 8 * kMaxM * 4 +
          (size_t)kMaxM * m.k_pad * 8 * t_subsets(m.k_pad) + kMaxM * 16 * 4 + (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
 }
-// The column-owner kernel serves M <= 4 as long as the quantised X of the whole contraction fits in shared memory.
-bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
+// The column-owner kernel serves M <= 4 (4-bit weights: its dot products run on raw nibbles) as long as the quantised X of
+// the whole contraction fits in shared memory.
+bool decode_cols_fits(const PackedMeta& m, int M) { return m.w_bits == 4 && M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
 
 cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y, void* workspace,
                                cudaStream_t s) {

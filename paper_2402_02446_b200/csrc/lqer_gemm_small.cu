@@ -75,6 +75,7 @@ struct Params {
   int M;
   int lr_shift;
   int y_bf16;                  // Y is bf16 (round to nearest even), else fp32
+  int w_bits;                  // mantissa bits of W_q: 4 or 2 (one value for all layers of a launch)
   int x_rows;                  // rows of an activation tile that TMA fills: M rounded up to 8 (the rest stay zero)
   long long wait_limit;
   int stall;                   // test hook: the producer withholds the last stage of its last item
@@ -226,6 +227,7 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
       int pk = 0;
       uint32_t ph = 0;
       bool ok = true;
+      const uint32_t w_tile = (uint32_t)w_tile_bytes(p.w_bits);
       for (int i = cta; i < num_items && ok; i += num_ctas) {
         const Item it = item_of(p, i);
         const Layer& ly = p.L[it.layer];
@@ -239,9 +241,9 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
           const uint32_t dst = smem_u32(pk_base + pk * C::PK_SLOT_BYTES) + C::X_TILE_BYTES;
           int xcol;
           if (s < ly.k_slabs) {
-            mbar_expect_tx(w_full(pk), n_half * kWTileBytes);
+            mbar_expect_tx(w_full(pk), n_half * w_tile);
             for (int h = 0; h < n_half; ++h)
-              bulk_load(dst + h * kWTileBytes, ly.wsec + ((size_t)(nt0 + h) * ly.k_slabs + s) * kWTileBytes, kWTileBytes, w_full(pk));
+              bulk_load(dst + h * kWTileBytes, ly.wsec + ((size_t)(nt0 + h) * ly.k_slabs + s) * w_tile, w_tile, w_full(pk));
             xcol = s * BK;
           } else {
             const int rs = s - ly.k_slabs;
@@ -396,22 +398,7 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
         const int nchunks = stage < ly.k_slabs ? 8 : 4;
         for (int i = 0; i < nchunks; ++i) *reinterpret_cast<uint4*>(bt + chunk[i]) = make_uint4(0u, 0u, 0u, 0u);
       } else if (stage < ly.k_slabs) {
-        const uint4 wa = *reinterpret_cast<const uint4*>(pkt + nl * 16);
-        const uint4 wb = *reinterpret_cast<const uint4*>(pkt + (kTileN + nl) * 16);
-        const uint32_t eb = *reinterpret_cast<const uint32_t*>(pkt + kWTileNibbleBytes + nl * 4);
-        uint32_t s2, c2;
-        w_scales(eb & 0xFFu, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[0]) = convert_word(wa.x, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[1]) = convert_word(wa.y, s2, c2);
-        w_scales((eb >> 8) & 0xFFu, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[2]) = convert_word(wa.z, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[3]) = convert_word(wa.w, s2, c2);
-        w_scales((eb >> 16) & 0xFFu, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[4]) = convert_word(wb.x, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[5]) = convert_word(wb.y, s2, c2);
-        w_scales(eb >> 24, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[6]) = convert_word(wb.z, s2, c2);
-        *reinterpret_cast<uint4*>(bt + chunk[7]) = convert_word(wb.w, s2, c2);
+        convert_column(pkt, nl, p.w_bits, bt, chunk);
       } else {
         const int nb = min(2, ly.r_blocks - (stage - ly.k_slabs) * 2);
         for (int rb = 0; rb < nb; ++rb) {
@@ -511,7 +498,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   for (int i = 0; i < MAX_LAYERS; ++i) {
     const SmallGemmLayer& src = layers[i < n ? i : 0];
     const PackedMeta& m = *src.meta;
-    if (m.lr_bits != layers[0].meta->lr_bits) return cudaErrorInvalidValue;
+    if (m.lr_bits != layers[0].meta->lr_bits || m.w_bits != layers[0].meta->w_bits) return cudaErrorInvalidValue;
     const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
     const cuuint32_t box[2] = {BK, (cuuint32_t)x_rows};
@@ -544,6 +531,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   p.lr_shift = layers[0].meta->lr_bits - 2;
   p.y_bf16 = y_bf16 ? 1 : 0;
   p.x_rows = x_rows;
+  p.w_bits = layers[0].meta->w_bits;
   p.wait_limit = wait_limit_cycles();
   p.stall = take_stall(kFamDecode) ? 1 : 0;
   const int sms = sm_count();

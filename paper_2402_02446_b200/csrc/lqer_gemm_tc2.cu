@@ -78,6 +78,7 @@ struct Params {
   int M, m_tiles;              // row tiles of 256 (the same M for every layer)
   int lr_shift;
   int y_bf16;                  // Y is bf16 (round to nearest even), else fp32
+  int w_bits;                  // mantissa bits of W_q: 4 or 2 (one value for all layers of a launch)
   long long wait_limit;        // bound of every wait, in clock cycles
   int stall;                   // test hook: the producers withhold the last stage of their last tile, so the waits run out
 };
@@ -148,6 +149,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       int st = 0;
       uint32_t ph = 0;
       bool ok = true;
+      const uint32_t w_tile = (uint32_t)w_tile_bytes(p.w_bits);
       for (int t = pair; t < num_tiles && ok; t += num_pairs) {
         const int layer = layer_of(p, t), tl = t - p.L[layer].tile_begin;
         const int mt = tl % p.m_tiles, nt = tl / p.m_tiles;
@@ -166,11 +168,10 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           if (!mbar_wait<true>(freed(st), ph ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = smem_u32(stage_base + st * STAGE_BYTES);
           if (s < k_slabs) {
-            mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? kWTileBytes : 0));
+            mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? w_tile : 0));
             tma_load_2d(a_dst, tmap_x, (slab0 + s) * BK, row0, loaded(st));
             if (has_w)
-              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * slab_stride + slab0 + s) * kWTileBytes, kWTileBytes,
-                        loaded(st));
+              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * slab_stride + slab0 + s) * w_tile, w_tile, loaded(st));
           } else {
             const int rs = s - k_slabs;
             const int rb0 = rs * 2, nb = min(2, r_blocks - rb0);
@@ -309,22 +310,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       uint8_t* bt = stage_base + st * STAGE_BYTES + A_TILE_BYTES;
       if (s < k_slabs) {
         if (has_w) {
-          const uint4 wa = *reinterpret_cast<const uint4*>(pk + nl * 16);
-          const uint4 wb = *reinterpret_cast<const uint4*>(pk + (kTileN + nl) * 16);
-          const uint32_t eb = *reinterpret_cast<const uint32_t*>(pk + kWTileNibbleBytes + nl * 4);
-          uint32_t s2, c2;
-          w_scales(eb & 0xFFu, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[0]) = convert_word(wa.x, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[1]) = convert_word(wa.y, s2, c2);
-          w_scales((eb >> 8) & 0xFFu, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[2]) = convert_word(wa.z, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[3]) = convert_word(wa.w, s2, c2);
-          w_scales((eb >> 16) & 0xFFu, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[4]) = convert_word(wb.x, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[5]) = convert_word(wb.y, s2, c2);
-          w_scales(eb >> 24, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[6]) = convert_word(wb.z, s2, c2);
-          *reinterpret_cast<uint4*>(bt + chunk[7]) = convert_word(wb.w, s2, c2);
+          convert_column(pk, nl, p.w_bits, bt, chunk);
         } else {                                 // columns beyond N: a zero operand half
 #pragma unroll
           for (int i = 0; i < 8; ++i) *reinterpret_cast<uint4*>(bt + chunk[i]) = make_uint4(0u, 0u, 0u, 0u);
@@ -476,6 +462,7 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
   p.M = M;
   p.lr_shift = m.lr_bits - 2;
   p.y_bf16 = 0;
+  p.w_bits = m.w_bits;
   cudaError_t e = launch_params(tmaps, p, s);
   if (e != cudaSuccess) return e;
   const size_t quads = (size_t)M * m.N / 4;
@@ -516,7 +503,7 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
   for (int slot = 0; slot < MAX_GROUP; ++slot) {
     const int g = order[slot < n ? slot : 0];
     const PackedMeta& m = metas[g];
-    if (m.lr_bits != metas[0].lr_bits) return cudaErrorInvalidValue;
+    if (m.lr_bits != metas[0].lr_bits || m.w_bits != metas[0].w_bits) return cudaErrorInvalidValue;
     const cuuint64_t dims[2] = {(cuuint64_t)xcat_cols(m), (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)xcat_cols(m) * 2};
     const cuuint32_t box[2] = {BK, BM};
@@ -543,6 +530,7 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
   p.M = M;
   p.lr_shift = metas[0].lr_bits - 2;
   p.y_bf16 = y_bf16 ? 1 : 0;
+  p.w_bits = metas[0].w_bits;
   return launch_params(tmaps, p, s);
 }
 

@@ -24,17 +24,28 @@ __global__ void __launch_bounds__(512) pack_w_kernel(const float* __restrict__ W
     amax = fmaxf(amax, abs_ignore_nan(v[i]));
   }
   const int e = block_exponent(amax, m.w_exp_min, m.w_exp_max);
-  uint32_t w[2] = {0u, 0u};
+  uint8_t* tile = wsec + ((size_t)nt * m.k_slabs + ks) * w_tile_bytes(m.w_bits);
+  if (m.w_bits == 2) {
+    // one word per block: even k in the low half, odd k in the high half, offset-binary crumbs
+    uint32_t w = 0u;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const uint32_t nib = (uint32_t)(quant_mantissa(v[i], e, m.w_bits) + 8);
-    w[i >> 3] |= nib << (4 * c_nibble_pos[i & 7]);
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t c = (uint32_t)(quant_mantissa(v[i], e, 2) + 1);
+      w |= c << (2 * (i >> 1) + 16 * (i & 1));
+    }
+    *reinterpret_cast<uint32_t*>(tile + (size_t)nl * 16 + blk * 4) = w;
+  } else {
+    uint32_t w[2] = {0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t nib = (uint32_t)(quant_mantissa(v[i], e, m.w_bits) + 8);
+      w[i >> 3] |= nib << (4 * c_nibble_pos[i & 7]);
+    }
+    const int bp = blk >> 1;
+    uint2* dst = reinterpret_cast<uint2*>(tile + ((size_t)(bp * kTileN + nl) * 16) + (blk & 1) * 8);
+    *dst = make_uint2(w[0], w[1]);
   }
-  uint8_t* tile = wsec + ((size_t)nt * m.k_slabs + ks) * kWTileBytes;
-  const int bp = blk >> 1;
-  uint2* dst = reinterpret_cast<uint2*>(tile + ((size_t)(bp * kTileN + nl) * 16) + (blk & 1) * 8);
-  *dst = make_uint2(w[0], w[1]);
-  tile[kWTileNibbleBytes + nl * 4 + blk] = (uint8_t)(e + 127);
+  tile[w_mant_bytes(m.w_bits) + nl * 4 + blk] = (uint8_t)(e + 127);
 }
 
 // One thread = one (16-block of K, rank column j) of A.
@@ -88,17 +99,24 @@ __global__ void export_w_kernel(PackedMeta m, const uint8_t* __restrict__ wsec, 
   const int n = nt * kTileN + nl;
   const int k0 = ks * kSlabK + blk * 16;
   if (n >= m.N || k0 >= m.K) return;
-  const uint8_t* tile = wsec + ((size_t)nt * m.k_slabs + ks) * kWTileBytes;
-  const uint2 w2 = *reinterpret_cast<const uint2*>(tile + ((size_t)((blk >> 1) * kTileN + nl) * 16) + (blk & 1) * 8);
-  const uint32_t w[2] = {w2.x, w2.y};
+  const uint8_t* tile = wsec + ((size_t)nt * m.k_slabs + ks) * w_tile_bytes(m.w_bits);
   if (Wm != nullptr) {
+    if (m.w_bits == 2) {
+      const uint32_t w = *reinterpret_cast<const uint32_t*>(tile + (size_t)nl * 16 + blk * 4);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int nib = (int)((w[i >> 3] >> (4 * c_nibble_pos[i & 7])) & 0xFu);
-      Wm[(size_t)(k0 + i) * m.N + n] = (int8_t)(nib - 8);
+      for (int i = 0; i < 16; ++i)
+        Wm[(size_t)(k0 + i) * m.N + n] = (int8_t)((int)((w >> (2 * (i >> 1) + 16 * (i & 1))) & 3u) - 1);
+    } else {
+      const uint2 w2 = *reinterpret_cast<const uint2*>(tile + ((size_t)((blk >> 1) * kTileN + nl) * 16) + (blk & 1) * 8);
+      const uint32_t w[2] = {w2.x, w2.y};
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int nib = (int)((w[i >> 3] >> (4 * c_nibble_pos[i & 7])) & 0xFu);
+        Wm[(size_t)(k0 + i) * m.N + n] = (int8_t)(nib - 8);
+      }
     }
   }
-  if (We != nullptr) We[(size_t)(k0 / 16) * m.N + n] = tile[kWTileNibbleBytes + nl * 4 + blk];
+  if (We != nullptr) We[(size_t)(k0 / 16) * m.N + n] = tile[w_mant_bytes(m.w_bits) + nl * 4 + blk];
 }
 
 __global__ void export_a_kernel(PackedMeta m, const uint8_t* __restrict__ asec, int8_t* __restrict__ Am,

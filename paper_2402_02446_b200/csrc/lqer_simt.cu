@@ -22,14 +22,23 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const uint16_t* __restri
   float acc = 0.0f;
   for (int kb = 0; kb < m.K64 / 16; ++kb) {
     const int ks = kb / 4, blk = kb % 4;
-    const uint8_t* tile = wsec + ((size_t)nt * m.k_slabs + ks) * kWTileBytes;
-    const uint2 w2 = *reinterpret_cast<const uint2*>(tile + ((size_t)((blk >> 1) * kTileN + nl) * 16) + (blk & 1) * 8);
-    const uint32_t w[2] = {w2.x, w2.y};
-    const float scale = pow2f((int)tile[kWTileNibbleBytes + nl * 4 + blk] - 127 - (m.w_bits - 2));
+    const uint8_t* tile = wsec + ((size_t)nt * m.k_slabs + ks) * w_tile_bytes(m.w_bits);
+    const float scale = pow2f((int)tile[w_mant_bytes(m.w_bits) + nl * 4 + blk] - 127 - (m.w_bits - 2));
+    if (m.w_bits == 2) {
+      const uint32_t w = *reinterpret_cast<const uint32_t*>(tile + (size_t)nl * 16 + blk * 4);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int mant = (int)((w[i >> 3] >> (4 * pos[i & 7])) & 0xFu) - 8;
-      acc = fmaf(bf16_to_float(x[kb * 16 + i]), (float)mant * scale, acc);
+      for (int i = 0; i < 16; ++i) {
+        const int mant = (int)((w >> (2 * (i >> 1) + 16 * (i & 1))) & 3u) - 1;
+        acc = fmaf(bf16_to_float(x[kb * 16 + i]), (float)mant * scale, acc);
+      }
+    } else {
+      const uint2 w2 = *reinterpret_cast<const uint2*>(tile + ((size_t)((blk >> 1) * kTileN + nl) * 16) + (blk & 1) * 8);
+      const uint32_t w[2] = {w2.x, w2.y};
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int mant = (int)((w[i >> 3] >> (4 * pos[i & 7])) & 0xFu) - 8;
+        acc = fmaf(bf16_to_float(x[kb * 16 + i]), (float)mant * scale, acc);
+      }
     }
   }
   if (m.k > 0) {

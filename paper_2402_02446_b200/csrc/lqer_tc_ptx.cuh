@@ -142,6 +142,66 @@ __device__ __forceinline__ void w_scales(uint32_t eb, uint32_t& s2, uint32_t& c2
   s2 = s | (s << 16);
   c2 = c | (c << 16);
 }
+// The 2-bit format (mantissas -1, 0, 1; value = m * 2^e): sixteen offset-binary crumbs of one block word -> sixteen
+// bf16, exact: 0x4300 | c is the bf16 value 128 + c, and (128 + c) * s - 129 * s rounds nothing away.
+__device__ __forceinline__ void convert_word2(uint32_t w, uint32_t s2, uint32_t c2, uint4& lo, uint4& hi) {
+  lo.x = fma_bf16x2((w & 0x00030003u) | 0x43004300u, s2, c2);
+  lo.y = fma_bf16x2(((w >> 2) & 0x00030003u) | 0x43004300u, s2, c2);
+  lo.z = fma_bf16x2(((w >> 4) & 0x00030003u) | 0x43004300u, s2, c2);
+  lo.w = fma_bf16x2(((w >> 6) & 0x00030003u) | 0x43004300u, s2, c2);
+  hi.x = fma_bf16x2(((w >> 8) & 0x00030003u) | 0x43004300u, s2, c2);
+  hi.y = fma_bf16x2(((w >> 10) & 0x00030003u) | 0x43004300u, s2, c2);
+  hi.z = fma_bf16x2(((w >> 12) & 0x00030003u) | 0x43004300u, s2, c2);
+  hi.w = fma_bf16x2(((w >> 14) & 0x00030003u) | 0x43004300u, s2, c2);
+}
+__device__ __forceinline__ void w_scales2(uint32_t eb, uint32_t& s2, uint32_t& c2) {
+  const uint32_t s = eb << 7;                              // bf16 bits of 2^e, eb = e + 127
+  const uint32_t c = 0x8000u | ((eb + 7u) << 7) | 1u;      // bf16 bits of -129 * 2^e
+  s2 = s | (s << 16);
+  c2 = c | (c << 16);
+}
+// One weight column of a 64-K stage from its packed form (pk: the column's mantissas at mant_off + nl * 16 resp.
+// the two block pairs of the 4-bit layout, exponents at exp_off + nl * 4) into its eight swizzled 16-byte chunks.
+__device__ __forceinline__ void convert_column(const uint8_t* pk, int nl, int w_bits, uint8_t* bt, const uint32_t (&chunk)[8]) {
+  uint32_t s2, c2;
+  if (w_bits == 2) {
+    const uint4 wv = *reinterpret_cast<const uint4*>(pk + nl * 16);
+    const uint32_t eb = *reinterpret_cast<const uint32_t*>(pk + 2048 + nl * 4);
+    uint4 lo, hi;
+    w_scales2(eb & 0xFFu, s2, c2);
+    convert_word2(wv.x, s2, c2, lo, hi);
+    *reinterpret_cast<uint4*>(bt + chunk[0]) = lo;
+    *reinterpret_cast<uint4*>(bt + chunk[1]) = hi;
+    w_scales2((eb >> 8) & 0xFFu, s2, c2);
+    convert_word2(wv.y, s2, c2, lo, hi);
+    *reinterpret_cast<uint4*>(bt + chunk[2]) = lo;
+    *reinterpret_cast<uint4*>(bt + chunk[3]) = hi;
+    w_scales2((eb >> 16) & 0xFFu, s2, c2);
+    convert_word2(wv.z, s2, c2, lo, hi);
+    *reinterpret_cast<uint4*>(bt + chunk[4]) = lo;
+    *reinterpret_cast<uint4*>(bt + chunk[5]) = hi;
+    w_scales2(eb >> 24, s2, c2);
+    convert_word2(wv.w, s2, c2, lo, hi);
+    *reinterpret_cast<uint4*>(bt + chunk[6]) = lo;
+    *reinterpret_cast<uint4*>(bt + chunk[7]) = hi;
+  } else {
+    const uint4 wa = *reinterpret_cast<const uint4*>(pk + nl * 16);
+    const uint4 wb = *reinterpret_cast<const uint4*>(pk + (kTileN + nl) * 16);
+    const uint32_t eb = *reinterpret_cast<const uint32_t*>(pk + kWTileNibbleBytes + nl * 4);
+    w_scales(eb & 0xFFu, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[0]) = convert_word(wa.x, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[1]) = convert_word(wa.y, s2, c2);
+    w_scales((eb >> 8) & 0xFFu, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[2]) = convert_word(wa.z, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[3]) = convert_word(wa.w, s2, c2);
+    w_scales((eb >> 16) & 0xFFu, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[4]) = convert_word(wb.x, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[5]) = convert_word(wb.y, s2, c2);
+    w_scales(eb >> 24, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[6]) = convert_word(wb.z, s2, c2);
+    *reinterpret_cast<uint4*>(bt + chunk[7]) = convert_word(wb.w, s2, c2);
+  }
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xFFFF0000u);   // exact values: truncation loses nothing
 }

@@ -76,6 +76,9 @@ def test_host_side_argument_errors():
     assert lib.lqer_packed_bytes(256, 256, 8, C.byref(cfg), None) == E("LQER_ERR_NULL")
     bad = L.default_config(); bad.w_bits = 3
     assert lib.lqer_packed_bytes(256, 256, 8, C.byref(bad), C.byref(out)) == E("LQER_ERR_CONFIG")
+    two = L.default_config(); two.w_bits = 2           # W2A8 (Section 4.4): 2 bits + 1 exponent byte per 16
+    assert lib.lqer_packed_bytes(4096, 4096, 0, C.byref(two), C.byref(out)) == 0
+    assert 4096 * 4096 * 0.3125 <= out.value <= 4096 * 4096 * 0.3125 + 1024
     bad = L.default_config(); bad.exp_min = -100
     assert lib.lqer_packed_bytes(256, 256, 8, C.byref(bad), C.byref(out)) == E("LQER_ERR_CONFIG")
     bad = L.default_config(); bad.w_exp_max = 56

@@ -120,7 +120,7 @@ def test_approximation_error_and_average_bits():
     assert abs((m + n) * k / (m * n) * 100 - 0.01 * k) < 0.01 * k * 0.05
 
 
-def _exact_forward(Xm, Xe, P, Tm, Te):
+def _exact_forward(Xm, Xe, P, Tm, Te, w_bits=4):
     """Y from integer mantissas in exact rational arithmetic (definition of the MXINT dot, Section 2.2)."""
     M, K = Xm.shape
     Y = [[Fraction(0)] * P.N for _ in range(M)]
@@ -128,7 +128,7 @@ def _exact_forward(Xm, Xe, P, Tm, Te):
         for j in range(P.N):
             acc = Fraction(0)
             for kk in range(K):
-                acc += int(Xm[i, kk]) * int(P.Wm[kk, j]) * Fraction(2) ** (int(Xe[i, kk // 16]) - 6 + int(P.We[kk // 16, j]) - 2)
+                acc += int(Xm[i, kk]) * int(P.Wm[kk, j]) * Fraction(2) ** (int(Xe[i, kk // 16]) - 6 + int(P.We[kk // 16, j]) - (w_bits - 2))
             for r in range(P.k_pad):
                 acc += int(Tm[i, r]) * int(P.Bm[r, j]) * Fraction(2) ** (int(Te[i, r // 16]) - 6 + int(P.Be[r // 16, j]) - 6)
             Y[i][j] = acc
@@ -283,3 +283,28 @@ def test_forward_requantises_t_per_rank_block_hand_worked():
     first, second = 73.0 / 128.0, 48.0
     assert r.Y[0, 0] == first + second and r.Y[0, 1] == second and r.Y[0, 2] == first
     assert not r.Y[0, 3:].any()
+
+
+def test_two_bit_weights_with_a_large_rank():
+    # W2A8 with k = 256 (Section 4.4): the same layer with 2-bit mantissas for W_q.  The full-rank identity, the exact
+    # rational forward pass and the bookkeeping of Appendix D must hold for this width too.
+    spec = gen.LayerSpec("w2", M=5, K=64, N=48, k=32, calib_rows=32, outlier_frac=0.0, n_outliers=2, outlier_scale=20.0, seed=21)
+    W = gen.make_weight(spec)
+    Wm, We = lqer.quantize_weight(W, w_bits=2)
+    assert set(np.unique(Wm)) <= {-1, 0, 1}
+    E = lqer.quantization_error(W, Wm, We, w_bits=2)
+    A, B, _ = lqer.lqer_factors(E, min(spec.K, spec.N), None)             # plain LQER (S = I), full rank
+    assert np.allclose(mxint.dequantize(Wm, We, 2, axis=0) + A @ B, W, rtol=0, atol=1e-10)
+    s = lqer.calibration_scale(gen.make_calibration(spec))
+    A, B, _ = lqer.lqer_factors(E, spec.k, s)
+    P = lqer.prepare_weights(W, A.astype(np.float32), B.astype(np.float32), w_bits=2)
+    X = gen.make_activations(spec)
+    r = lqer.forward(X, P, w_bits=2)
+    exact = _exact_forward(r.Xm, r.Xe, P, r.Tm, r.Te, w_bits=2)
+    assert np.array_equal(np.array([[float(v) for v in row] for row in exact]), r.Y)
+    # a coarser W_q leaves a larger error for the same rank
+    E4 = lqer.quantization_error(W, *lqer.quantize_weight(W, w_bits=4), w_bits=4)
+    assert np.linalg.norm(E) > 2.0 * np.linalg.norm(E4)
+    # 2 + 4/16 bits for W_q alone; with k = 256 on a 13B-shaped layer the factors add about 1.1 bits
+    assert lqer.average_weight_bits(5120, 5120, 0, w_bits=2) == 2.25
+    assert abs(lqer.average_weight_bits(5120, 13824, 256, w_bits=2) - (2.25 + 256 * (5120 + 13824) * 8.25 / (5120 * 13824))) < 1e-12

@@ -54,7 +54,7 @@ def _rand_blocks(seed, n=400, scale_spread=12):
     return v.astype(np.float32)
 
 
-@pytest.mark.parametrize("bits", [4, 6, 8])
+@pytest.mark.parametrize("bits", [2, 4, 6, 8])
 def test_invariants(bits):
     v = _rand_blocks(bits)
     m, e = mxint.quantize(v, bits, axis=1)
