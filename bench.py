@@ -146,7 +146,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ reference arm
-def oracle_sample(rows: int, a_bits: int = 8):
+def oracle_sample(rows: int, a_bits: int = 8, w_bits: int = 4, rank=None):
     """The bounded sample the oracle is timed on: layer 0's q, gate and down linears, `rows` tokens
     of the M=2048 batch.  Returns (callable running the sample once, flops of one run, description)."""
     from oracle import lqer as olqer
@@ -154,14 +154,16 @@ def oracle_sample(rows: int, a_bits: int = 8):
     flops = 0.0
     for which in (0, 4, 6):
         spec = gen.config_stack(0, which, M_PREFILL)
+        if rank is not None:
+            spec = dataclasses.replace(spec, k=rank)
         W = gen.make_weight(spec)
         A, B = gen.make_random_factors(spec)
-        P = olqer.prepare_weights(W, A, B)
+        P = olqer.prepare_weights(W, A, B, w_bits=w_bits)
         X = gen.make_activations(spec, M=rows)
         work.append((X, P, W, A, B))
         flops += layer_flops(rows, spec.K, spec.N, spec.k)
     def run():
-        return [olqer.forward(X, P, a_bits=a_bits) for X, P, _, _, _ in work]
+        return [olqer.forward(X, P, w_bits=w_bits, a_bits=a_bits) for X, P, _, _, _ in work]
     run.work = work
     return run, flops, f"layer 0 q, gate, down linears, {rows} rows of the M={M_PREFILL} batch"
 
@@ -177,11 +179,11 @@ def blas_threads() -> int:
     return os.cpu_count() or 1
 
 
-def time_oracle(steps: int, warmup: int, rows: int, a_bits: int = 8, check=None):
+def time_oracle(steps: int, warmup: int, rows: int, a_bits: int = 8, check=None, w_bits: int = 4, rank=None):
     """TFLOP/s and milliseconds per run of the oracle on its bounded sample.  check(work, results), if given, is
     called with the sample's inputs and the oracle's results of the last run (the GPU arm compares its own
     output on the same inputs with them)."""
-    run, flops, what = oracle_sample(rows, a_bits)
+    run, flops, what = oracle_sample(rows, a_bits, w_bits, rank)
     for _ in range(warmup):
         run()
     t0 = time.perf_counter()
@@ -197,7 +199,7 @@ def run_reference(args) -> None:
     if int(os.environ.get("RANK", "0")) != 0:
         return
     steps, warmup = max(args.steps, 1), max(args.warmup, 0)
-    tflops, ms, what, _ = time_oracle(steps, warmup, rows=args.oracle_rows, a_bits=args.a_bits)
+    tflops, ms, what, _ = time_oracle(steps, warmup, rows=args.oracle_rows, a_bits=args.a_bits, w_bits=args.w_bits, rank=args.rank)
     cores = blas_threads()
     line = {"impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -566,7 +568,8 @@ def run_ours(args) -> None:
                 worst = max(worst, float(np.max(np.abs(Y - ref.Y) / ref.tol)))
                 Pg.release()
             return worst
-        tflops, ms, what, worst = time_oracle(1, 0, rows=args.oracle_rows, a_bits=args.a_bits, check=gpu_against_oracle)
+        tflops, ms, what, worst = time_oracle(1, 0, rows=args.oracle_rows, a_bits=args.a_bits, check=gpu_against_oracle,
+                                              w_bits=args.w_bits, rank=args.rank)
         cpu = {"value": tflops, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": what,
                "seconds": ms / 1e3, "gpu_max_abs_err_over_tol": worst}
 
