@@ -112,6 +112,30 @@ lqer_status_t lqer_call_workspace_bytes(int M, int K, int N, int k, const lqer_c
 lqer_status_t lqer_prepare_weights(const float* W, const float* A, const float* B, int K, int N, int k,
                                    const lqer_config_t* cfg, void* packed, size_t packed_bytes, void* stream);
 
+/* Weight preparation from the weight and a calibration batch alone (Section 3.1: E_q = W - W_q and its rank-k
+ * factors A_k = U_k, B_k = Sigma_k V_k^T; Section 3.2: the SVD is taken of S E_q and A_k = S^-1 U'_k,
+ * B_k = Sigma'_k V'_k^T; Appendix A: S from the calibration samples - mean |X| per channel over the tokens of a
+ * sample, maximum over the samples, normalised by sqrt(min * max)).  All on the GPU: the truncated SVD is a
+ * randomised subspace iteration (k + 16 columns, four rounds, fp64 accumulation), which approaches the optimal
+ * rank-k residual of Section 3.2 from above; the factors are then rounded to fp32, quantised and packed with W
+ * exactly as lqer_prepare_weights does.
+ *  - W [K,N] fp32 (device).  samples: HOST array of n_samples DEVICE pointers, sample i is fp32 [sample_rows[i], K]
+ *    (sample_rows: host array).  n_samples == 0 gives plain LQER (S = I, Section 3.1).
+ *  - omega: the random test matrix, fp32 [N, columns] standard normal (device), columns from
+ *    lqer_factor_sketch_columns; the caller draws it, so the run is reproducible with the caller's generator.
+ *  - A_out [K,k], B_out [k,N] fp32 (device): the factors before quantisation, or NULL.
+ *  - workspace (device, 256-byte aligned): lqer_prepare_workspace_bytes.  Asynchronous on `stream`.
+ *  - lqer_prepare_status (synchronises) reads what only the device could see: 0 fine, 1 a calibration channel is
+ *    identically zero (S not invertible; S = I was used), 2 a sketch lost rank (k larger than the rank of the
+ *    error), 3 the small SVD did not converge. */
+lqer_status_t lqer_factor_sketch_columns(int K, int N, int k, int* columns);
+lqer_status_t lqer_prepare_workspace_bytes(int K, int N, int k, size_t* bytes);
+lqer_status_t lqer_prepare_from_calibration(const float* W, const float* const* samples, const int* sample_rows, int n_samples,
+                                            const float* omega, int K, int N, int k, const lqer_config_t* cfg, void* packed,
+                                            size_t packed_bytes, float* A_out, float* B_out, void* workspace,
+                                            size_t workspace_bytes, void* stream);
+lqer_status_t lqer_prepare_status(const void* workspace, int K, int N, int k, void* stream, int* code);
+
 /* Register a packed buffer that was produced earlier and copied to a new address
  * (save / restore).  Reads the header back from the device: synchronises `stream`.
  * Optional: every entry point that takes `packed` does the same on its own the first

@@ -17,6 +17,8 @@ from .binding import (  # noqa: F401
     set_wait_limit_cycles,
     inject_stall,
     prepare_weights,
+    prepare_from_calibration,
+    factor_sketch_columns,
     export_weights,
     quantize_activations,
     project_lowrank,

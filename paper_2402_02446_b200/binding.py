@@ -69,6 +69,10 @@ def lib() -> C.CDLL:
             "lqer_set_wait_limit_cycles": (i, [C.c_longlong]),
             "lqer_inject_stall": (i, [i]),
             "lqer_prepare_weights": (i, [vp, vp, vp, i, i, i, cfgp, vp, sz, vp]),
+            "lqer_factor_sketch_columns": (i, [i, i, i, C.POINTER(i)]),
+            "lqer_prepare_workspace_bytes": (i, [i, i, i, C.POINTER(sz)]),
+            "lqer_prepare_from_calibration": (i, [vp, C.POINTER(vp), C.POINTER(i), i, vp, i, i, i, cfgp, vp, sz, vp, vp, vp, sz, vp]),
+            "lqer_prepare_status": (i, [vp, i, i, i, vp, C.POINTER(i)]),
             "lqer_attach_packed": (i, [vp, sz, vp]),
             "lqer_release_packed": (i, [vp]),
             "lqer_packed_shape": (i, [vp, C.POINTER(i), C.POINTER(i), C.POINTER(i), C.POINTER(i)]),
@@ -171,6 +175,41 @@ def prepare_weights(W: torch.Tensor, A: torch.Tensor | None, B: torch.Tensor | N
                                       None if k == 0 else _dev(B, torch.float32), K, N, k, C.byref(cfg),
                                       buf.data_ptr(), nbytes, _stream(stream)), "lqer_prepare_weights")
     return PackedWeights(buf, K, N, k, (k + 15) // 16 * 16)
+
+
+def factor_sketch_columns(K: int, N: int, k: int) -> int:
+    out = C.c_int()
+    _check(lib().lqer_factor_sketch_columns(K, N, k, C.byref(out)), "lqer_factor_sketch_columns")
+    return out.value
+
+
+def prepare_from_calibration(W: torch.Tensor, samples, k: int, omega: torch.Tensor | None = None,
+                             cfg: Config | None = None, seed: int = 0, stream=None):
+    """Packed weights from W and calibration samples alone (an empty list gives plain LQER).  Returns
+    (PackedWeights, A [K,k], B [k,N], device status code)."""
+    cfg = cfg or default_config()
+    K, N = W.shape
+    cols = factor_sketch_columns(K, N, k)
+    if omega is None:
+        g = torch.Generator(device=W.device)
+        g.manual_seed(seed)
+        omega = torch.randn((N, cols), generator=g, device=W.device, dtype=torch.float32)
+    nbytes = packed_bytes(K, N, k, cfg)
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    wsb = C.c_size_t()
+    _check(lib().lqer_prepare_workspace_bytes(K, N, k, C.byref(wsb)), "lqer_prepare_workspace_bytes")
+    ws = torch.empty(wsb.value, dtype=torch.uint8, device=W.device)
+    A = torch.empty((K, k), dtype=torch.float32, device=W.device)
+    B = torch.empty((k, N), dtype=torch.float32, device=W.device)
+    samples = list(samples)
+    ptrs = (C.c_void_p * max(len(samples), 1))(*[_dev(x, torch.float32) for x in samples])
+    rows = (C.c_int * max(len(samples), 1))(*[x.shape[0] for x in samples])
+    _check(lib().lqer_prepare_from_calibration(_dev(W, torch.float32), ptrs, rows, len(samples), _dev(omega, torch.float32), K, N, k,
+                                               C.byref(cfg), buf.data_ptr(), nbytes, A.data_ptr(), B.data_ptr(), ws.data_ptr(),
+                                               ws.numel(), _stream(stream)), "lqer_prepare_from_calibration")
+    code = C.c_int()
+    _check(lib().lqer_prepare_status(ws.data_ptr(), K, N, k, _stream(stream), C.byref(code)), "lqer_prepare_status")
+    return PackedWeights(buf, K, N, k, (k + 15) // 16 * 16), A, B, code.value
 
 
 def export_weights(P: PackedWeights, stream=None) -> dict:

@@ -606,6 +606,68 @@ lqer_status_t lqer_prepare_weights(const float* W, const float* A, const float* 
   return LQER_OK;
 }
 
+lqer_status_t lqer_factor_sketch_columns(int K, int N, int k, int* columns) {
+  if (columns == nullptr) return LQER_ERR_NULL;
+  lqer_status_t st = check_shape(K, N, k);
+  if (st != LQER_OK) return st;
+  if (k < 1) return LQER_ERR_SHAPE;
+  *columns = factor_sketch_rank(K, N, k);
+  return LQER_OK;
+}
+
+lqer_status_t lqer_prepare_workspace_bytes(int K, int N, int k, size_t* bytes) {
+  if (bytes == nullptr) return LQER_ERR_NULL;
+  lqer_status_t st = check_shape(K, N, k);
+  if (st != LQER_OK) return st;
+  if (k < 1) return LQER_ERR_SHAPE;
+  *bytes = factor_workspace_bytes(K, N, k, 0);
+  return LQER_OK;
+}
+
+lqer_status_t lqer_prepare_from_calibration(const float* W, const float* const* samples, const int* sample_rows, int n_samples,
+                                            const float* omega, int K, int N, int k, const lqer_config_t* cfg, void* packed,
+                                            size_t packed_bytes, float* A_out, float* B_out, void* workspace,
+                                            size_t workspace_bytes, void* stream) {
+  if (W == nullptr || omega == nullptr || packed == nullptr || workspace == nullptr) return LQER_ERR_NULL;
+  if (n_samples < 0 || n_samples > 4096 || (n_samples > 0 && (samples == nullptr || sample_rows == nullptr))) return LQER_ERR_NULL;
+  lqer_status_t st = check_config(cfg);
+  if (st != LQER_OK) return st;
+  if ((st = check_shape(K, N, k)) != LQER_OK) return st;
+  if (k < 1) return LQER_ERR_SHAPE;
+  for (int i = 0; i < n_samples; ++i) {
+    if (samples[i] == nullptr) return LQER_ERR_NULL;
+    if (sample_rows[i] < 1) return LQER_ERR_SHAPE;
+  }
+  if (!aligned16(W) || !aligned16(omega) || (A_out != nullptr && !aligned16(A_out)) || (B_out != nullptr && !aligned16(B_out)) ||
+      (reinterpret_cast<uintptr_t>(packed) & 255u) != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return LQER_ERR_ALIGN;
+  PackedMeta m;
+  fill_meta(m, K, N, k, *cfg);
+  if (packed_bytes < m.total_bytes || workspace_bytes < factor_workspace_bytes(K, N, k, 0)) return LQER_ERR_BUFFER_TOO_SMALL;
+  if ((st = check_arch()) != LQER_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  float* A = nullptr;
+  float* B = nullptr;
+  if (launch_factorize(W, samples, sample_rows, n_samples, omega, K, N, k, cfg->w_bits, cfg->w_exp_min, cfg->w_exp_max, A_out, B_out,
+                       workspace, nullptr, &A, &B, s) != cudaSuccess)
+    return LQER_ERR_CUDA;
+  return lqer_prepare_weights(W, A, B, K, N, k, cfg, packed, packed_bytes, stream);
+}
+
+lqer_status_t lqer_prepare_status(const void* workspace, int K, int N, int k, void* stream, int* code) {
+  if (workspace == nullptr || code == nullptr) return LQER_ERR_NULL;
+  lqer_status_t st = check_shape(K, N, k);
+  if (st != LQER_OK) return st;
+  if (k < 1) return LQER_ERR_SHAPE;
+  // the status word sits behind the fixed-size pieces of the workspace, in front of the internal A and B
+  auto al = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  const size_t off = factor_workspace_bytes(K, N, k, 0) - al((size_t)K * k * 4) - al((size_t)k * N * 4) - 256;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(code, static_cast<const uint8_t*>(workspace) + off, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return LQER_ERR_CUDA;
+  return cudaStreamSynchronize(s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+}
+
 lqer_status_t lqer_attach_packed(const void* packed, size_t packed_bytes, void* stream) {
   if (packed == nullptr) return LQER_ERR_NULL;
   if (packed_bytes < (size_t)kHeaderBytes) return LQER_ERR_BUFFER_TOO_SMALL;

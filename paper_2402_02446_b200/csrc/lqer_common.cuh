@@ -357,6 +357,13 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
 int gemm_tc2_max_group();
 cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, void* const* Ys, bool y_bf16,
                                   const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s);
+// Factor preparation (Section 3.1 / 3.2, Appendix A): A_k, B_k from W and calibration samples, by randomised subspace
+// iteration with factor_sketch_rank columns; Omega [N, that many] fp32 is the caller's random test matrix.
+int factor_sketch_rank(int K, int N, int k);
+size_t factor_workspace_bytes(int K, int N, int k, int max_calib_rows);
+cudaError_t launch_factorize(const float* W, const float* const* Xs, const int* rows, int n_samples, const float* Omega, int K,
+                             int N, int k, int w_bits, int emin, int emax, float* A, float* B, void* workspace, int** status_dev,
+                             float** A_used, float** B_used, cudaStream_t s);
 // Small batches (M <= kSmallMaxM).  The prologue quantises X (fp32 or bf16) into Xcat and leaves T_q behind it; up to
 // prologue_small_max_layers() layers with one M and one set of formats per launch.
 struct SmallPrologueLayer {
