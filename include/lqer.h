@@ -182,8 +182,7 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * activations in the w-only setting and re-quantises them in the w&a setting): X [M,K] of x_dtype, Y [M,N] of
  * y_dtype, both dense row-major and 16-byte aligned.  bf16 X is quantised to MXINT like fp32 X (every bf16
  * value is an fp32 value); bf16 Y is the fp32 result rounded to nearest even.  Everything else - packed,
- * workspace, paths, device-side status - as for lqer_linear_stream; the column-owner decode kernel reads and
- * writes fp32 only, so 16-bit calls of up to 4 rows take the small-batch kernels.  lqer_linear_batched_ex is
+ * workspace, paths, device-side status - as for lqer_linear_stream.  lqer_linear_batched_ex is
  * lqer_linear_batched with every call's X and Y of the given types (cast the pointers of lqer_call_t). */
 lqer_status_t lqer_linear_ex(const void* X, lqer_dtype_t x_dtype, int M, const void* packed, void* Y, lqer_dtype_t y_dtype,
                              void* workspace, size_t workspace_bytes, void* stream);
@@ -257,6 +256,10 @@ lqer_status_t lqer_linear_host(const float* X_host, int M, const void* packed, f
 lqer_status_t lqer_linear_host_batched_bytes(const lqer_call_t* calls, int n_calls, size_t* bytes);
 lqer_status_t lqer_linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace,
                                        size_t workspace_bytes, void* stream);
+/* The same with host X of x_dtype and host Y of y_dtype (Section 2.1: 16-bit activations between layers): bf16
+ * halves the bytes that cross the host link in that direction.  The workspace size is the same. */
+lqer_status_t lqer_linear_host_batched_ex(const lqer_call_t* calls, int n_calls, lqer_dtype_t x_dtype, lqer_dtype_t y_dtype,
+                                          void* workspace, size_t workspace_bytes, void* stream);
 
 /* Zero the head of a fresh workspace (status area, counters, accumulator; at most 168192 bytes;
  * asynchronous on `stream`).  Call once after allocating the workspace and again after

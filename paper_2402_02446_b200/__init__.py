@@ -31,6 +31,7 @@ from .binding import (  # noqa: F401
     linear_static,
     linear_host,
     linear_host_batched,
+    linear_host_batched_ex,
     linear_host_batched_bytes,
     make_host_calls,
     poll_status,

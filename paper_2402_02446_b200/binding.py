@@ -89,6 +89,7 @@ def lib() -> C.CDLL:
             "lqer_linear_host": (i, [vp, i, vp, vp, vp, sz, vp]),
             "lqer_linear_host_batched_bytes": (i, [C.POINTER(Call), i, C.POINTER(sz)]),
             "lqer_linear_host_batched": (i, [C.POINTER(Call), i, vp, sz, vp]),
+            "lqer_linear_host_batched_ex": (i, [C.POINTER(Call), i, i, i, vp, sz, vp]),
             "lqer_workspace_init": (i, [vp, sz, vp]),
             "lqer_poll_status": (i, [vp, vp, C.POINTER(i)]),
             "lqer_set_path": (i, [i]),
@@ -331,14 +332,14 @@ def linear_host(X_host: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y_host
     return Y_host
 
 
-def make_host_calls(items) -> "C.Array":
-    """items: iterable of (X_cpu, PackedWeights, Y_cpu), contiguous fp32 CPU tensors -> a host array of lqer_call_t."""
+def make_host_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype: torch.dtype = torch.float32) -> "C.Array":
+    """items: iterable of (X_cpu, PackedWeights, Y_cpu), contiguous CPU tensors of the given types -> a host array of lqer_call_t."""
     items = list(items)
     arr = (Call * len(items))()
     for j, (X, P, Y) in enumerate(items):
-        for t in (X, Y):
-            if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
-                raise ValueError("expected contiguous fp32 CPU tensors")
+        for t, dt in ((X, x_dtype), (Y, y_dtype)):
+            if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+                raise ValueError("expected contiguous CPU tensors of the stated types")
         arr[j] = Call(X.data_ptr(), X.shape[0], P.ptr, Y.data_ptr())
     return arr
 
@@ -355,6 +356,12 @@ def linear_host_batched(calls, ws: torch.Tensor, stream=None) -> None:
     arr = calls if isinstance(calls, C.Array) else make_host_calls(calls)
     _check(lib().lqer_linear_host_batched(arr, len(arr), ws.data_ptr(), ws.numel(), _stream(stream)),
            "lqer_linear_host_batched")
+
+
+def linear_host_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype: torch.dtype, stream=None) -> None:
+    """linear_host_batched with host X of x_dtype and host Y of y_dtype; `calls` from make_host_calls(..., x_dtype, y_dtype)."""
+    _check(lib().lqer_linear_host_batched_ex(calls, len(calls), _DTYPES[x_dtype], _DTYPES[y_dtype], ws.data_ptr(), ws.numel(),
+                                             _stream(stream)), "lqer_linear_host_batched_ex")
 
 
 def poll_status(ws: torch.Tensor, stream=None) -> int:

@@ -251,8 +251,8 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   void* xcat = wsb + align_up(persist_bytes(m), 256);
   cudaError_t err;
   if (small) {
-    if (path != 5 && !project_only && !io.x_bf16 && !io.y_bf16 && decode_cols_fits(m, M)) {
-      err = launch_decode_cols(static_cast<const float*>(X), M, m, packed, static_cast<float*>(Y), workspace, s);
+    if (path != 5 && !project_only && decode_cols_fits(m, M)) {
+      err = launch_decode_cols(X, io.x_bf16, M, m, packed, Y, io.y_bf16, workspace, s);
     } else {
       const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
       uint8_t* slice = static_cast<uint8_t*>(xcat);
@@ -745,11 +745,10 @@ lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y, v
 
 }  // extern "C"
 
-// The batched entry points: independent calls share launches where the path is left at 0.  With 16-bit activations
-// at the boundary (io) the column-owner decode kernel, which reads and writes fp32, is not used.
+// The batched entry points: independent calls share launches where the path is left at 0.
 static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
                                     void* stream, IoTypes io) {
-  const bool cols_ok = !io.x_bf16 && !io.y_bf16;
+  const bool cols_ok = true;
   if (calls == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
   // validate everything before the first launch
@@ -820,7 +819,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
             for (int q = 0; q < (int)pm.size(); q += step) {
               const int cnt = std::min(step, (int)pm.size() - q);
               if (launch_decode_pre(calls + i + q, pm.data() + q, outs.data() + q, cnt, q == 0 ? kChainFirst : kChainLater,
-                                    cs) != cudaSuccess)
+                                    io.x_bf16, cs) != cudaSuccess)
                 return LQER_ERR_CUDA;
             }
           }
@@ -832,7 +831,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
         const int set = chain_open ? 1 - chain_set : 0;
         bool fills = false;
         if (launch_decode_cols_group(calls + i, metas, n, workspace, workspace_bytes, chain_open ? kChainLater : kChainFirst,
-                                     set, &fills, ahead ? pres : nullptr, cs) != cudaSuccess)
+                                     set, &fills, ahead ? pres : nullptr, io.x_bf16, io.y_bf16, cs) != cudaSuccess)
           return LQER_ERR_CUDA;
         chain_open = fills;
         chain_set = set;
@@ -1000,8 +999,11 @@ lqer_status_t lqer_linear_host_batched_bytes(const lqer_call_t* calls, int n_cal
   return LQER_OK;
 }
 
-lqer_status_t lqer_linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
-                                       void* stream) {
+}  // extern "C"
+
+static lqer_status_t linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
+                                         void* stream, IoTypes io) {
+  const size_t xe = io.x_bf16 ? 2 : 4, ye = io.y_bf16 ? 2 : 4;   // bytes per element on the host side and in the staging buffers
   if (calls == nullptr || workspace == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
@@ -1037,17 +1039,17 @@ lqer_status_t lqer_linear_host_batched(const lqer_call_t* calls, int n_calls, vo
     lookup(c.packed, m);
     // copy in: the buffer is free once the layer two calls back has run
     ok = (i < 2 || cudaStreamWaitEvent(hp->in, hp->comp_done[b], 0) == cudaSuccess) &&
-         cudaMemcpyAsync(Xd[b], c.X, (size_t)c.M * m.K * 4, cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
+         cudaMemcpyAsync(Xd[b], c.X, (size_t)c.M * m.K * xe, cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
          cudaEventRecord(hp->in_done[b], hp->in) == cudaSuccess &&
          // the layer: after its X has landed and after the Y buffer's previous contents have left
          cudaStreamWaitEvent(s, hp->in_done[b], 0) == cudaSuccess &&
          (i < 2 || cudaStreamWaitEvent(s, hp->out_done[b], 0) == cudaSuccess);
     if (!ok) { result = LQER_ERR_CUDA; break; }
-    result = lqer_linear_stream(Xd[b], c.M, c.packed, Yd[b], workspace, core, stream);
+    result = run_linear(Xd[b], c.M, c.packed, Yd[b], workspace, core, s, nullptr, nullptr, false, io);
     if (result != LQER_OK) break;
     ok = cudaEventRecord(hp->comp_done[b], s) == cudaSuccess &&
          cudaStreamWaitEvent(hp->out, hp->comp_done[b], 0) == cudaSuccess &&
-         cudaMemcpyAsync(c.Y, Yd[b], (size_t)c.M * m.N * 4, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess &&
+         cudaMemcpyAsync(c.Y, Yd[b], (size_t)c.M * m.N * ye, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess &&
          cudaEventRecord(hp->out_done[b], hp->out) == cudaSuccess;
     if (!ok) result = LQER_ERR_CUDA;
   }
@@ -1056,6 +1058,21 @@ lqer_status_t lqer_linear_host_batched(const lqer_call_t* calls, int n_calls, vo
                        cudaStreamSynchronize(hp->out) == cudaSuccess;
   if (result == LQER_OK && !drained) result = LQER_ERR_CUDA;
   return result;
+}
+
+extern "C" {
+
+lqer_status_t lqer_linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+  return linear_host_batched(calls, n_calls, workspace, workspace_bytes, stream, IoTypes());
+}
+
+lqer_status_t lqer_linear_host_batched_ex(const lqer_call_t* calls, int n_calls, lqer_dtype_t x_dtype, lqer_dtype_t y_dtype,
+                                          void* workspace, size_t workspace_bytes, void* stream) {
+  IoTypes io;
+  lqer_status_t st = io_types(x_dtype, y_dtype, &io);
+  if (st != LQER_OK) return st;
+  return linear_host_batched(calls, n_calls, workspace, workspace_bytes, stream, io);
 }
 
 lqer_status_t lqer_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {

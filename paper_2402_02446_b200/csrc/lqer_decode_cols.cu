@@ -52,8 +52,8 @@ constexpr int kTRanges = 16;      // CTAs of a layer that share the work of T = 
 constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
 
 struct Layer {
-  const float* X;
-  float* Y;
+  const void* X;                // [M, K] fp32, or bf16 where Params::x_bf16
+  void* Y;                      // [M, N] fp32, or bf16 where Params::y_bf16
   const uint8_t* packed;
   size_t off_w, off_b, off_a;   // sections of the packed buffer
   int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
@@ -74,6 +74,7 @@ struct Params {
   DeviceStatus* status;
   int M;
   int a_bits, lr_bits, exp_min, exp_max;
+  int x_bf16, y_bf16;           // element types of X and Y (else fp32)
   long long wait_limit;         // bound of the wait for the other CTAs' partial sums, in clock cycles
 };
 
@@ -106,12 +107,12 @@ __host__ __device__ inline int t_subsets(int k_pad) {
   return tiles < kWarps ? kWarps / tiles : 1;
 }
 
-struct Formats { int a_bits, lr_bits, exp_min, exp_max; };
+struct Formats { int a_bits, lr_bits, exp_min, exp_max, x_bf16; };
 
 // X -> MXINT8 for the whole contraction, by all threads of the CTA: per row the mantissas in the byte order the nibbles
 // unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales 2^(e_x - 6) and the dp4a seeds (bits of
 // 1.5 * 2^23, minus 8 * sum(x) of the block).
-__device__ __forceinline__ void quantize_x_rows(const float* X, int M, int K, int K64, const Formats& f, uint8_t* xm,
+__device__ __forceinline__ void quantize_x_rows(const void* X, int M, int K, int K64, const Formats& f, uint8_t* xm,
                                                 float* xsc, int* xof) {
   const int tid = threadIdx.x, KB = K64 / 16;
   const int per_row = K64 / 4, total = M * per_row;             // float4 items: (row, quarter-block)
@@ -122,8 +123,16 @@ __device__ __forceinline__ void quantize_x_rows(const float* X, int M, int K, in
     for (int u = 0; u < U; ++u) {
       const int item = base + u * kThreads + tid;
       const int row = item / per_row, c4 = item % per_row;
-      v[u] = (item < total && c4 * 4 < K) ? __ldg(reinterpret_cast<const float4*>(X + (size_t)row * K + c4 * 4))
-                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (item < total && c4 * 4 < K) {
+        if (f.x_bf16) {                            // 16-bit activations: every bf16 value is an fp32 value
+          const uint2 h = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(X) + (size_t)row * K + c4 * 4));
+          v[u] = make_float4(__uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u), __uint_as_float(h.y << 16),
+                             __uint_as_float(h.y & 0xFFFF0000u));
+        } else {
+          v[u] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(X) + (size_t)row * K + c4 * 4));
+        }
+      }
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -221,7 +230,7 @@ __device__ __forceinline__ void store_tq(double tv, bool valid, int row, int col
 //   [M][K64] mantissas, [M][K64/16] scales, [M][K64/16] dp4a seeds, [kMaxM][16] scales of T_q, [kMaxM][k_pad] T_q.
 constexpr int kPreMaxCalls = 64;
 struct PreCall {
-  const float* X;
+  const void* X;
   const uint8_t* asec;          // A_q section of the packed buffer
   uint8_t* out;
   int M, K, K64, k_pad;
@@ -299,8 +308,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = ly.ctas, cta = (int)blockIdx.x - ly.cta_begin;
-  const float* const X = ly.X;
-  float* const Y = ly.Y;
+  const void* const X = ly.X;
+  void* const Y = ly.Y;
   const uint8_t* const wsec = ly.packed + ly.off_w;
   const uint8_t* const bsec = ly.packed + ly.off_b;
   const uint8_t* const asec = ly.packed + ly.off_a;
@@ -381,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 
   // ---- X -> MXINT8 for the whole contraction: per row the mantissas in the byte order the nibbles
   //      unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales and the offsets 8 * sum(x)
-  const Formats fmt = {p.a_bits, p.lr_bits, p.exp_min, p.exp_max};
+  const Formats fmt = {p.a_bits, p.lr_bits, p.exp_min, p.exp_max, p.x_bf16};
   if (pre) {                                       // quantised X and T_q are there already: straight into shared memory
     const int xb = (int)pre_x_bytes(M, ly.K64), tb = (int)pre_t_bytes(ly.k_pad);
     for (int o = tid * 16; o < xb; o += kThreads * 16)
@@ -603,7 +612,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
             float v = 0.f;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) v += red_now[((h * kWarps + w) * 32 + col) * kMaxM + r];
-            Y[(size_t)r * ly.N + c0 * 8 + col] = v;
+            if (p.y_bf16) {
+              uint32_t u = __float_as_uint(v);               // round to nearest even (NaN / inf keep their class)
+              u = ((u & 0x7F800000u) == 0x7F800000u) ? ((u >> 16) | ((u & 0xFFFFu) ? 0x40u : 0u)) : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+              static_cast<uint16_t*>(Y)[(size_t)r * ly.N + c0 * 8 + col] = (uint16_t)u;
+            } else {
+              static_cast<float*>(Y)[(size_t)r * ly.N + c0 * 8 + col] = v;
+            }
           }
         }
       }
@@ -625,10 +640,10 @@ static size_t cols_smem_bytes(const PackedMeta& m, int M) {
 // the whole contraction fits in shared memory.
 bool decode_cols_fits(const PackedMeta& m, int M) { return m.w_bits == 4 && M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
 
-cudaError_t launch_decode_cols(const float* X, int M, const PackedMeta& m, const void* packed, float* Y, void* workspace,
-                               cudaStream_t s) {
-  const lqer_call_t one = {X, M, packed, Y};
-  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, nullptr, s);
+cudaError_t launch_decode_cols(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+                               void* workspace, cudaStream_t s) {
+  const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
+  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, nullptr, x_bf16, y_bf16, s);
 }
 
 int decode_cols_max_group() { return dcol::kMaxGroup; }
@@ -639,7 +654,7 @@ int decode_cols_max_group() { return dcol::kMaxGroup; }
 // at least one cluster's worth of column groups.
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
                                      size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
-                                     cudaStream_t s) {
+                                     bool x_bf16, bool y_bf16, cudaStream_t s) {
   using namespace dcol;
   static OncePerDevice once;
   static bool one_cta_per_sm = true;               // false if any device could hold two CTAs of the kernel on one SM
@@ -665,6 +680,8 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   p.status = reinterpret_cast<DeviceStatus*>(workspace);
   p.M = M;
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
+  p.x_bf16 = x_bf16 ? 1 : 0;
+  p.y_bf16 = y_bf16 ? 1 : 0;
   p.wait_limit = wait_limit_cycles();
   const int stall = take_stall(kFamDecode) ? 1 : 0;
 
@@ -764,7 +781,7 @@ int decode_pre_max_calls() { return dcol::kPreMaxCalls; }
 // X_q and T_q of n independent decode calls (M <= 4 each, every layer fitting decode_cols_fits), one CTA per call, into
 // outs[i] (decode_pre_bytes each, 256-byte aligned).
 cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas, uint8_t* const* outs, int n, int order,
-                              cudaStream_t s) {
+                              bool x_bf16, cudaStream_t s) {
   using namespace dcol;
   static OncePerDevice once;
   cudaError_t e0 = once.run([] {
@@ -787,7 +804,7 @@ cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas,
     c.asec = static_cast<const uint8_t*>(calls[g].packed) + m.off_a;
     c.out = outs[g];
     c.M = calls[g].M; c.K = m.K; c.K64 = m.K64; c.k_pad = m.k_pad;
-    c.f = Formats{m.a_bits, m.lr_bits, m.exp_min, m.exp_max};
+    c.f = Formats{m.a_bits, m.lr_bits, m.exp_min, m.exp_max, x_bf16 ? 1 : 0};
     if (c.M < 1 || c.M > kMaxM) return cudaErrorInvalidValue;
     if (c.M > 1) single = false;
     const size_t need = pre_x_bytes(c.M, c.K64) + pre_t_bytes(c.k_pad) + 16 +
