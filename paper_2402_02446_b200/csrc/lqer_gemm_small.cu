@@ -214,6 +214,8 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
       int pend_slot[PK_SLOTS], pend_x[PK_SLOTS], pend_layer[PK_SLOTS];
       int npend = 0;
       bool waited = false;
+      // the activation tiles of the stages requested before the wait land on a barrier of their own (x_full, used
+      // once per slot); later ones share the weights' barrier, so that the MMA warp has one barrier to watch
       auto load_x = [&](int slot, int layer, int xcol) {
         mbar_expect_tx(x_full(slot), p.x_rows * 128);        // rows of the box beyond the batch arrive as zeros
         tma_load_2d(smem_u32(pk_base + slot * C::PK_SLOT_BYTES), &tmaps.m[layer], xcol, 0, x_full(slot));
@@ -240,15 +242,16 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
           if (!mbar_wait<true>(pk_free(pk), ph ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t dst = smem_u32(pk_base + pk * C::PK_SLOT_BYTES) + C::X_TILE_BYTES;
           int xcol;
+          const uint32_t x_bytes = waited ? (uint32_t)p.x_rows * 128u : 0u;
           if (s < ly.k_slabs) {
-            mbar_expect_tx(w_full(pk), n_half * w_tile);
+            mbar_expect_tx(w_full(pk), n_half * w_tile + x_bytes);
             for (int h = 0; h < n_half; ++h)
               bulk_load(dst + h * kWTileBytes, ly.wsec + ((size_t)(nt0 + h) * ly.k_slabs + s) * w_tile, w_tile, w_full(pk));
             xcol = s * BK;
           } else {
             const int rs = s - ly.k_slabs;
             const int rb0 = rs * 2, nb = min(2, ly.r_blocks - rb0);
-            mbar_expect_tx(w_full(pk), n_half * nb * (kTileN * 17));
+            mbar_expect_tx(w_full(pk), n_half * nb * (kTileN * 17) + x_bytes);
             for (int h = 0; h < n_half; ++h) {
               const uint8_t* tile = ly.bsec + (size_t)(nt0 + h) * b_tile_stride;
               bulk_load(dst + h * kWTileBytes, tile + (size_t)rb0 * kTileN * 16, nb * kTileN * 16, w_full(pk));
@@ -257,7 +260,7 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
             xcol = ly.K64 + rs * RANK_PER_STAGE;
           }
           if (waited) {
-            load_x(pk, it.layer, xcol);
+            tma_load_2d(smem_u32(pk_base + pk * C::PK_SLOT_BYTES), &tmaps.m[it.layer], xcol, 0, w_full(pk));
           } else {
             pend_slot[npend] = pk; pend_x[npend] = xcol; pend_layer[npend] = it.layer;
             ++npend;
@@ -289,8 +292,10 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
         const uint64_t a_desc = make_desc(pk0 + pk * C::PK_SLOT_BYTES);
         const uint64_t b_desc = make_desc(cv0 + cv * CV_TILE_BYTES);
         const int nk = s < ly.k_slabs ? 4 : min(2, ly.r_blocks - (s - ly.k_slabs) * 2);
+        // a converted tile implies its packed tile had landed, and with it (from the second pass over the ring on) the
+        // activation tile; on the first pass the activation tiles have their own barrier
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(cv_ready(cv), (it_no / CV_SLOTS) & 1, abort_flag) &&
-                                         mbar_wait(x_full(pk), (it_no / PK_SLOTS) & 1, abort_flag)) != 0;
+                                         (it_no >= (uint32_t)PK_SLOTS || mbar_wait(x_full(pk), 0, abort_flag))) != 0;
         if (!ok) break;
         tc_fence_after();
         if (elect_one()) {
@@ -490,11 +495,14 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   // K chunks per tile.  A layer alone is cut as its shape says (small_gemm_chunks: enough work items for every SM).
   // Layers that share a launch bring many tiles between them, and every chunk costs a pass of partial sums through
   // L2, so they are cut less: just enough for about two work items per SM in all, never more than alone (the scratch
-  // is sized for that).  The sums of a tile are then grouped differently, so a layer's result in a shared launch
+  // is sized for that; finer cuts that would even out the last round of items were measured and lose more in
+  // epilogues than they gain).  The sums of a tile are then grouped differently, so a layer's result in a shared launch
   // may differ from its result alone in the last bits; it is the same whenever the same layers share a launch.
+  const int sms = sm_count();
+  if (sms < 1) return cudaErrorInvalidDevice;
   int total_tiles = 0;
   for (int i = 0; i < n; ++i) total_tiles += small_gemm_col_tiles(*layers[i].meta);
-  const int group_chunks = (296 + total_tiles - 1) / total_tiles;
+  const int group_chunks = (2 * 148 + total_tiles - 1) / total_tiles;      // about two work items per SM in all
   for (int i = 0; i < MAX_LAYERS; ++i) {
     const SmallGemmLayer& src = layers[i < n ? i : 0];
     const PackedMeta& m = *src.meta;
@@ -534,8 +542,6 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   p.w_bits = layers[0].meta->w_bits;
   p.wait_limit = wait_limit_cycles();
   p.stall = take_stall(kFamDecode) ? 1 : 0;
-  const int sms = sm_count();
-  if (sms < 1) return cudaErrorInvalidDevice;
   const int ctas = p.num_items < sms ? p.num_items : sms;
   return MT == 64 ? launch_mt<64, 6>(tmaps, p, ctas, s) : launch_mt<128, 3>(tmaps, p, ctas, s);
 }
