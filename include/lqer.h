@@ -91,15 +91,15 @@ lqer_status_t lqer_default_config(lqer_config_t* cfg);
 lqer_status_t lqer_packed_bytes(int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
 
 /* Size in bytes (host out) of the scratch `workspace` lqer_linear* needs for any call of up to
- * M_max rows.  The workspace holds a head that is all zero between calls (status area, the
- * kernels' arrival counters, the decode kernel's fp64 accumulator of X A_k) followed by per-call
- * scratch: the quantised activations [X_q | T_q] (bf16, M rows) with the prologue's fp64
- * partial sums of X A_k, or the decode kernel's partial sums.  One workspace may serve layers
- * of different shapes if it fits the largest. */
+ * M_max rows.  The workspace holds a head of one fixed size that is all zero between calls (status
+ * area, the kernels' arrival counters) followed by per-call scratch: the quantised activations
+ * [X_q | T_q] (bf16, M rows) with the prologue's fp64 partial sums of X A_k and the GEMM's fp32
+ * partial sums of Y where its K range is cut, or the decode kernel's partial sums of X A_k.  One
+ * workspace may serve layers of different shapes in turn if it fits the largest. */
 lqer_status_t lqer_workspace_bytes(int M_max, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);
 
 /* Size in bytes (host out) that one call with exactly M rows uses of its workspace on the path the library
- * picks for it (decode kernels up to 16 rows, prologue + GEMM above): never more than
+ * picks for it (column-owner decode kernel up to 4 rows, small-batch kernels up to 128, prologue + GEMM above): never more than
  * lqer_workspace_bytes(M_max, ...) for any M_max >= M.  This is the figure lqer_linear_static holds against
  * LQER_STATIC_SCRATCH_BYTES. */
 lqer_status_t lqer_call_workspace_bytes(int M, int K, int N, int k, const lqer_config_t* cfg, size_t* bytes);

@@ -59,13 +59,13 @@ inline uint32_t meta_checksum(const PackedMeta& m) {
   return h;
 }
 
-// Workspace layout: a persistent head that is all zero between calls
-//   [0, 256)   status area: DeviceStatus, the decode kernel's two T counters
-//   [256, ..)  per-column-tile arrival counters of the decode kernel, its fp64 T accumulator, then the
-//              per-row-tile arrival counters of the tensor-core prologue
-// followed by per-call scratch: Xcat (bf16 [M, K64 + k_pad]) and the fp64 partial sums of the tensor-core
-// prologue for the GEMM path, or the partial-sum slots of the decode path.
-constexpr int kTCountOffset = 64, kTDoneOffset = 68;
+// Workspace layout: a persistent head of one fixed size (kPersistMaxBytes) that is all zero between calls
+//   [0, 256)   status area: DeviceStatus
+//   [256, ..)  the column-owner decode kernel's counters (two sets of 16 layers), the small-batch GEMM's per-tile
+//              arrival counters (up to 32768 over the layers of a launch), then the counter pairs of the row tiles
+//              (tensor-core prologue) or row groups (small prologue)
+// followed by per-call scratch: Xcat (bf16 [M, K64 + k_pad]) with the fp64 partial sums of the prologue that runs
+// and the fp32 partial sums of the small-batch or split-K GEMM, or the decode kernel's partial sums of T.
 constexpr int kDecodeMaxCtas = 160;                  // CTAs of one launch of the column-owner decode kernel, at most
 constexpr int kPrologueRowTiles = 512;               // an arrival and a departure counter each: batches up to 65536 rows
 constexpr int kPrologueMaxCtas = 148;               // CTAs of one tensor-core prologue launch the scratch is sized for (launches use min(this, SMs))
@@ -122,7 +122,8 @@ inline size_t prologue_tc_scratch_bytes(const PackedMeta& m, int M) {
   if (!prologue_tc_rank_ok(m) || (M + 127) / 128 > kPrologueRowTiles) return 0;
   return (size_t)((M + 127) / 128) * prologue_tc_splits(m, M) * 128 * m.k_pad * 8;
 }
-// Small batches (up to kSmallMaxM rows): the prologue for few rows and the GEMM with the tokens on the MMA's N side.
+// Small batches (up to kSmallMaxM rows): the prologue for few rows and the GEMM with the tokens on the MMA's M side
+// (padded to 64 or 128 rows) and 256 weight columns on its N side.
 // Everything below depends on the shape alone, never on the device or on what else shares a launch.
 constexpr int kSmallMaxM = 128;
 // K ranges per group of 16 rows in the small prologue (each a CTA; the last to arrive adds them up in range order).
