@@ -245,6 +245,73 @@ __device__ __forceinline__ void quantize_quad(const float4 vin, int bits, int em
   bf.y = __byte_perm(__float_as_uint(r[2]), __float_as_uint(r[3]), 0x7632);
 }
 
+// What quantize_block16 needs of the format, computed once per kernel instead of once per block.
+struct QuantConsts {
+  float qmax, qlim;      // 2^(bits-1) - 1, and qmax + 1/2
+  int shift;             // bits - 2
+  int emin, emax;
+};
+__device__ __forceinline__ QuantConsts quant_consts(int bits, int emin, int emax) {
+  QuantConsts c;
+  c.qmax = (float)((1 << (bits - 1)) - 1);
+  c.qlim = c.qmax + 0.5f;
+  c.shift = bits - 2;
+  c.emin = emin; c.emax = emax;
+  return c;
+}
+// The same quantisation with one lane holding a whole 16-block: no shuffles, and the exponent arithmetic is paid once
+// per 16 elements.  m8 = the sixteen int8 mantissas in element order; bf0 / bf1 = the sixteen exact bf16 values.
+__device__ __forceinline__ void quantize_block16(const float (&v)[16], const QuantConsts& c, int& e, uint4& m8, uint4& bf0,
+                                                 uint4& bf1) {
+  // Block maximum and a NaN detector, both as trees (four levels deep instead of fifteen dependent operations).
+  // fmaxf drops a NaN operand, so NaN counts as zero in the maximum; the sum is NaN iff a NaN (or inf - inf) is
+  // among the values, and its order does not matter because only that is asked of it.
+  float mx[8], sm[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { mx[i] = fmaxf(fabsf(v[2 * i]), fabsf(v[2 * i + 1])); sm[i] = v[2 * i] + v[2 * i + 1]; }
+#pragma unroll
+  for (int w = 4; w > 0; w >>= 1)
+#pragma unroll
+    for (int i = 0; i < w; ++i) { mx[i] = fmaxf(mx[i], mx[i + w]); sm[i] += sm[i + w]; }
+  float amax = mx[0];
+  const float sum = sm[0];
+  amax = fmaxf(amax, 0.0f);
+  e = block_exponent(amax, c.emin, c.emax);
+  const float inv_step = pow2f(c.shift - e), step = pow2f(e - c.shift);
+  const float kMagic = 12582912.0f;                   // 1.5 * 2^23, see quantize_quad
+  const float back = -kMagic * step;
+  uint32_t m[4], b[8];
+  if (sum == sum && amax * inv_step < c.qlim) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {                     // four elements at a time: few values alive at once
+      float s4[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) s4[i] = fmaf(v[4 * q + i], inv_step, kMagic);
+      m[q] = __byte_perm(__byte_perm(__float_as_uint(s4[0]), __float_as_uint(s4[1]), 0x0040),
+                         __byte_perm(__float_as_uint(s4[2]), __float_as_uint(s4[3]), 0x0040), 0x5410);
+      b[2 * q] = __byte_perm(__float_as_uint(fmaf(s4[0], step, back)), __float_as_uint(fmaf(s4[1], step, back)), 0x7632);
+      b[2 * q + 1] = __byte_perm(__float_as_uint(fmaf(s4[2], step, back)), __float_as_uint(fmaf(s4[3], step, back)), 0x7632);
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float s4[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float x = (v[4 * q + i] == v[4 * q + i]) ? v[4 * q + i] : 0.0f;
+        s4[i] = fminf(fmaxf(x * inv_step, -c.qmax), c.qmax) + kMagic;
+      }
+      m[q] = __byte_perm(__byte_perm(__float_as_uint(s4[0]), __float_as_uint(s4[1]), 0x0040),
+                         __byte_perm(__float_as_uint(s4[2]), __float_as_uint(s4[3]), 0x0040), 0x5410);
+      b[2 * q] = __byte_perm(__float_as_uint(fmaf(s4[0], step, back)), __float_as_uint(fmaf(s4[1], step, back)), 0x7632);
+      b[2 * q + 1] = __byte_perm(__float_as_uint(fmaf(s4[2], step, back)), __float_as_uint(fmaf(s4[3], step, back)), 0x7632);
+    }
+  }
+  m8 = make_uint4(m[0], m[1], m[2], m[3]);
+  bf0 = make_uint4(b[0], b[1], b[2], b[3]);
+  bf1 = make_uint4(b[4], b[5], b[6], b[7]);
+}
+
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
                : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3]) : "r"(a0), "r"(a1), "r"(b0), "r"(0));

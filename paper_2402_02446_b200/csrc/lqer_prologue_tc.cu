@@ -37,14 +37,14 @@ constexpr int WORK_WARPS = 24;               // scalers + quantisers
 constexpr int NUM_WARPS = WORK_WARPS + 3;
 constexpr int NUM_THREADS = NUM_WARPS * 32;  // 864
 constexpr int MAX_TMEM_SLOTS = 8;
+constexpr unsigned kNapNs = 100;              // sleep between polls of the roles that run ahead of the scalers
 
 template <int KP>
 struct Cfg {
-  static constexpr int SCALER_WARPS = KP > 32 ? 16 : 8;      // four lane quarters x column groups
+  static constexpr int SCALER_WARPS = KP >= 32 ? 16 : 8;     // four lane quarters x column groups
   static constexpr int QUANT_WARPS = WORK_WARPS - SCALER_WARPS;
   static constexpr int CPW = KP / (SCALER_WARPS / 4);        // rank columns per scaler warp
-  static constexpr int ROW_STEP = QUANT_WARPS * 2;           // rows one pass of the quantisers covers
-  static constexpr int QUADS = ROWS / ROW_STEP;              // float4 per quantiser per stage
+  static constexpr int BPL = ROWS / (QUANT_WARPS * 8);       // 16-blocks per quantiser lane and stage (a warp: 8 rows x 4 blocks)
   static constexpr int SLOT_COLS = 2 * KP;                   // accumulator columns per block pair
   static constexpr int TMEM_SLOTS = (512 / SLOT_COLS) < MAX_TMEM_SLOTS ? (512 / SLOT_COLS) : MAX_TMEM_SLOTS;
   static constexpr int TMEM_COLS = 512;
@@ -60,7 +60,7 @@ struct Cfg {
   static constexpr int NUM_BARS = 2 * RAW_SLOTS + 2 * X_SLOTS + 2 * PANELS + 2 * MAX_TMEM_SLOTS;
   static constexpr int SMEM_BYTES = OFF_BARS + NUM_BARS * 8 + 32 + 1024;
   static_assert(CPW % 8 == 0 && CPW <= 16, "scaler registers");
-  static_assert(ROWS % ROW_STEP == 0, "quantiser passes");
+  static_assert(ROWS % (QUANT_WARPS * 8) == 0, "quantiser passes");
   static_assert(PANEL_BYTES % 1024 == 0, "swizzle atoms need 1024-byte bases");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
@@ -94,7 +94,7 @@ struct GroupParams {
   int n;
 };
 struct TensorMaps {
-  CUtensorMap m[kMaxLayers];   // X of each layer: fp32 [M, K], box 64 x 128
+  CUtensorMap m[kMaxLayers];   // X of each layer: [M, K], box 128 bytes (32 fp32 or 64 bf16) x 128 rows, 128-byte swizzle
 };
 
 // int8 x int8 -> int32, both operands K-major, M = m, N = n.
@@ -129,18 +129,21 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t pari
   return ok != 0;
 }
 // Bounded like tc::mbar_wait: gives up after the launch's wait limit or as soon as another role has given up.
-__device__ __forceinline__ bool parked_wait(uint32_t bar, uint32_t parity, volatile WaitState* abort_flag) {
+// nap_ns > 0: the role is ahead of the one it waits for, so it sleeps between polls and leaves the issue slots to
+// the roles that work (a polling warp is eligible every cycle and competes with them).
+__device__ __forceinline__ bool parked_wait(uint32_t bar, uint32_t parity, volatile WaitState* abort_flag, unsigned nap_ns = 0) {
   if (mbar_try_wait_parked(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait_parked(bar, parity)) {
+    if (nap_ns) __nanosleep(nap_ns);
     if (abort_flag->abort != 0) return false;
     if (clock64() - t0 > abort_flag->limit) { abort_flag->abort = 1; return false; }
   }
   return true;
 }
 // A wait whose outcome every lane of the warp shares (the code after it shuffles or touches tensor memory as a warp).
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile WaitState* abort_flag) {
-  return __all_sync(0xFFFFFFFFu, parked_wait(bar, parity, abort_flag)) != 0;
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile WaitState* abort_flag, unsigned nap_ns = 0) {
+  return __all_sync(0xFFFFFFFFu, parked_wait(bar, parity, abort_flag, nap_ns)) != 0;
 }
 
 template <int KP>
@@ -154,7 +157,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
   const Params& p = gp.L[layer];
   const CUtensorMap* const tmap_x = &tmaps.m[layer];
   const int bid = (int)blockIdx.x - gp.cta_begin[layer];          // index within the layer's CTAs
-  constexpr int SW = C::SCALER_WARPS, QW = C::QUANT_WARPS, CPW = C::CPW, QUADS = C::QUADS;
+  constexpr int SW = C::SCALER_WARPS, QW = C::QUANT_WARPS, CPW = C::CPW;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* raw_base = smem;
@@ -238,32 +241,42 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
         const int u = 2 * s + j, slot = u % C::TMEM_SLOTS;
         if (!warp_wait(slot_full(slot), (u / C::TMEM_SLOTS) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        // As few round trips to tensor memory as the registers allow: with 8 columns per warp both blocks of the
+        // slot are loaded together and waited for once, with 16 a block at a time.  The slot is free again as soon
+        // as its last values are in registers, before the arithmetic on them.
+        constexpr int LB = CPW == 8 ? 2 : 1;                              // blocks per round trip
+        const double kMagic = 4503601774854144.0;                         // 2^52 + 2^31
 #pragma unroll
-        for (int blk = 0; blk < 2; ++blk) {
-          const int bi = 2 * j + blk;                                   // block within the stage
-          const int ehi = (int)(int8_t)(e4 >> (8 * bi)) * (1 << 20);
-          const int* hrow = hia + bi * KP + h * CPW;
-          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + slot * C::SLOT_COLS + blk * KP + h * CPW;
-          const double kMagic = 4503601774854144.0;                     // 2^52 + 2^31
+        for (int trip = 0; trip < 2 / LB; ++trip) {
+          uint32_t c[LB][CPW];
 #pragma unroll
-          for (int g8 = 0; g8 < CPW / 8; ++g8) {                        // eight columns at a time keeps the registers few
-            uint32_t c[8];
-            tmem_ld8(taddr + g8 * 8, c);
-            tmem_ld_wait();
-            if (blk == 1 && g8 == CPW / 8 - 1) {                        // the whole slot has been read
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(slot_empty(slot));
-            }
+          for (int lb = 0; lb < LB; ++lb) {
+            const int blk = trip * LB + lb;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + slot * C::SLOT_COLS + blk * KP + h * CPW;
 #pragma unroll
-            for (int g = 0; g < 2; ++g) {
-              const int4 hv = *reinterpret_cast<const int4*>(hrow + g8 * 8 + 4 * g);
-              double* a = acc + g8 * 8 + 4 * g;
+            for (int g8 = 0; g8 < CPW / 8; ++g8) tmem_ld8(taddr + g8 * 8, c[lb] + g8 * 8);
+          }
+          tmem_ld_wait();
+          if (trip == 2 / LB - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(slot_empty(slot));
+          }
+#pragma unroll
+          for (int lb = 0; lb < LB; ++lb) {
+            const int bi = 2 * j + trip * LB + lb;                        // block within the stage
+            const int ehi = (int)(int8_t)(e4 >> (8 * bi)) * (1 << 20);
+            const int* hrow = hia + bi * KP + h * CPW;
+#pragma unroll
+            for (int g = 0; g < CPW / 4; ++g) {
+              const int4 hv = *reinterpret_cast<const int4*>(hrow + 4 * g);
+              double* a = acc + 4 * g;
+              const uint32_t* cc = c[lb] + 4 * g;
               // int32 -> fp64 without the conversion unit: 2^52 + 2^31 + c has the bits (0x43300000, c ^ 2^31)
-              a[0] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 0] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.x + ehi, 0), a[0]);
-              a[1] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 1] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.y + ehi, 0), a[1]);
-              a[2] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 2] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.z + ehi, 0), a[2]);
-              a[3] = fma(__hiloint2double(0x43300000, (int)(c[4 * g + 3] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.w + ehi, 0), a[3]);
+              a[0] = fma(__hiloint2double(0x43300000, (int)(cc[0] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.x + ehi, 0), a[0]);
+              a[1] = fma(__hiloint2double(0x43300000, (int)(cc[1] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.y + ehi, 0), a[1]);
+              a[2] = fma(__hiloint2double(0x43300000, (int)(cc[2] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.z + ehi, 0), a[2]);
+              a[3] = fma(__hiloint2double(0x43300000, (int)(cc[3] ^ 0x80000000u)) - kMagic, __hiloint2double(hv.w + ehi, 0), a[3]);
             }
           }
         }
@@ -279,50 +292,69 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     for (int i = 0; i < CPW; i += 2) *reinterpret_cast<double2*>(dst + i) = make_double2(acc[i], acc[i + 1]);
   } else if (warp < WORK_WARPS) {
     // ------------------------------------------------------------------ quantisers
+    // A lane owns a whole 16-block of a row: lanes 0-7 of a warp take block 0 of eight consecutive rows, lanes 8-15
+    // block 1, and so on, so that every quarter warp reads and writes eight different 16-byte chunks of the swizzled
+    // tiles (no bank conflicts) and the warp stores 8 rows x 128 contiguous bytes of Xcat.
     if (C::REG_SHIFT) asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
-    const int tq = tid - SW * 32;
-    const int c4 = tq & 15, rb = tq >> 4;            // float4 within the 64-column stage; first row (then + ROW_STEP per quad)
-    const int col0 = pan_lo * 2 * STAGE_COLS + c4 * 4;
-    uint16_t* cp = p.xcat + (size_t)(row0 + rb) * p.ldx + col0;
-    const size_t c_step = (size_t)C::ROW_STEP * p.ldx;
-    const int rows_ok = p.M - (row0 + rb);            // quad i is a real row while ROW_STEP * i < rows_ok
-    const uint32_t off_row = (uint32_t)(rb * 128 + (c4 & 3) * 4);
-    int8_t* xe_dst = s_xe + rb * 4 + (c4 >> 2);
-    const bool xe_writer = (c4 & 3) == 0;
+    const int qwarp = warp - SW;
+    const int blk = lane >> 3;                         // 16-block within the 64-column stage
+    const int r0 = qwarp * 8 + (lane & 7);             // first row (then + 8 * QW per pass)
+    const uint32_t swz = (uint32_t)(lane & 7);         // row & 7: the rows of a pass differ by multiples of 8
+    const QuantConsts qc = quant_consts(p.a_bits, p.exp_min, p.exp_max);
+    uint16_t* cp = p.xcat + (size_t)(row0 + r0) * p.ldx + pan_lo * 2 * STAGE_COLS + blk * 16;
+    const size_t c_step = (size_t)(8 * QW) * p.ldx;
+    const int rows_ok = p.M - (row0 + r0);              // pass i is a real row while 8 * QW * i < rows_ok
+    // offsets of the lane's block within a raw slot: fp32 = two half tiles of 32 columns (16 KB each, rows of 128
+    // bytes), the block is four chunks; bf16 = one tile of 64 columns, the block is two chunks
+    const uint32_t raw_off = p.x_bf16 ? (uint32_t)(r0 * 128) : (uint32_t)((blk >> 1) * (RAW_BYTES / 2) + r0 * 128);
+    const uint32_t chunk0 = p.x_bf16 ? (uint32_t)(blk * 2) : (uint32_t)((blk & 1) * 4);
     bool ok = true;
     for (int s = 0; s < n_stages && ok; ++s) {
       const int rs = s % RAW_SLOTS, xs = s % X_SLOTS;
-      if (!warp_wait(raw_full(rs), (s / RAW_SLOTS) & 1, abort_flag)) { ok = false; break; }
-      float4 xr[QUADS];
-      if (p.x_bf16) {
-        const uint2* src = reinterpret_cast<const uint2*>(raw_base + rs * RAW_BYTES) + rb * 16 + c4;
-#pragma unroll
-        for (int i = 0; i < QUADS; ++i) {
-          const uint2 v = src[i * C::ROW_STEP * 16];
-          xr[i] = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
-                              __uint_as_float(v.y & 0xFFFF0000u));
-        }
-      } else {
-        const float4* src = reinterpret_cast<const float4*>(raw_base + rs * RAW_BYTES) + rb * 16 + c4;
-#pragma unroll
-        for (int i = 0; i < QUADS; ++i) xr[i] = src[i * C::ROW_STEP * 16];
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(raw_empty(rs));     // the values are in registers: the slot can be refilled
-      if (!warp_wait(xq_empty(xs), ((s / X_SLOTS) & 1) ^ 1, abort_flag)) { ok = false; break; }
-      const int chunk = (xs & 1) * 4 + (c4 >> 2);    // 16-byte chunk of the 128-byte row
-      uint8_t* xdst = xq_base + (xs >> 1) * XBUF_BYTES + off_row + ((chunk ^ (rb & 7)) << 4);
-      const bool store_ok = col0 + s * STAGE_COLS < p.K64;
+      if (!warp_wait(raw_full(rs), (s / RAW_SLOTS) & 1, abort_flag, kNapNs)) { ok = false; break; }
+      if (!warp_wait(xq_empty(xs), ((s / X_SLOTS) & 1) ^ 1, abort_flag, kNapNs)) { ok = false; break; }
+      const uint8_t* src = raw_base + rs * RAW_BYTES + raw_off;
+      const uint32_t chunk = (uint32_t)((xs & 1) * 4 + blk);     // 16-byte chunk of the 128-byte row of mantissas
+      uint8_t* xdst = xq_base + (xs >> 1) * XBUF_BYTES + r0 * 128 + ((chunk ^ swz) << 4);
+      int8_t* xe_dst = s_xe + (xs * ROWS + r0) * 4 + blk;
+      const bool store_ok = (pan_lo * 2 + s) * STAGE_COLS < p.K64;
       uint16_t* cd = cp + (size_t)s * STAGE_COLS;
 #pragma unroll
-      for (int i = 0; i < QUADS; ++i) {
-        uint32_t m8;
-        uint2 bf;
+      for (int i = 0; i < C::BPL; ++i) {
+        float v[16];
+        const uint8_t* row = src + i * (8 * QW) * 128;
+        if (p.x_bf16) {
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint4 w = *reinterpret_cast<const uint4*>(row + (((chunk0 + j) ^ swz) << 4));
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              v[8 * j + 2 * t] = __uint_as_float(ww[t] << 16);
+              v[8 * j + 2 * t + 1] = __uint_as_float(ww[t] & 0xFFFF0000u);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float4 w = *reinterpret_cast<const float4*>(row + (((chunk0 + j) ^ swz) << 4));
+            v[4 * j] = w.x; v[4 * j + 1] = w.y; v[4 * j + 2] = w.z; v[4 * j + 3] = w.w;
+          }
+        }
+        if (i == C::BPL - 1) {                         // the stage's values are in registers: the slot can be refilled
+          __syncwarp();
+          if (lane == 0) mbar_arrive(raw_empty(rs));
+        }
+        uint4 m8, bf0, bf1;
         int e;
-        quantize_quad(xr[i], p.a_bits, p.exp_min, p.exp_max, e, m8, bf);
-        *reinterpret_cast<uint32_t*>(xdst + i * C::ROW_STEP * 128) = m8;
-        if (xe_writer) xe_dst[(xs * ROWS + C::ROW_STEP * i) * 4] = (int8_t)e;
-        if (store_ok && C::ROW_STEP * i < rows_ok) *reinterpret_cast<uint2*>(cd + i * c_step) = bf;
+        quantize_block16(v, qc, e, m8, bf0, bf1);
+        *reinterpret_cast<uint4*>(xdst + i * (8 * QW) * 128) = m8;
+        xe_dst[i * (8 * QW) * 4] = (int8_t)e;
+        if (store_ok && 8 * QW * i < rows_ok) {
+          uint4* g = reinterpret_cast<uint4*>(cd + i * c_step);
+          g[0] = bf0;
+          g[1] = bf1;
+        }
       }
       fence_proxy_async_smem();                      // generic-proxy writes -> visible to the MMA's async proxy
       __syncwarp();
@@ -352,7 +384,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     load_exps(0);
     for (int pp = 0; pp < n_pan && ok; ++pp) {
       const int pb = pp % PANELS;
-      if (!warp_wait(panel_empty(pb), ((pp / PANELS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+      if (!warp_wait(panel_empty(pb), ((pp / PANELS) & 1) ^ 1, abort_flag, kNapNs)) { ok = false; break; }
       const int b0 = (pan_lo + pp) * 8;
       const uint32_t dst0 = smem_u32(panel_base + pb * C::PANEL_BYTES);
       for (int i = lane; i < 8 * KP; i += 32) {
@@ -380,13 +412,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
       bool ok = true;
       for (int s = 0; s < n_stages && ok; ++s) {
         const int xs = s % X_SLOTS, pp = s >> 1, pb = pp % PANELS;
-        if (!parked_wait(xq_full(xs), (s / X_SLOTS) & 1, abort_flag)) { ok = false; break; }
-        if ((s & 1) == 0 && !parked_wait(panel_full(pb), (pp / PANELS) & 1, abort_flag)) { ok = false; break; }
+        if (!parked_wait(xq_full(xs), (s / X_SLOTS) & 1, abort_flag, kNapNs)) { ok = false; break; }
+        if ((s & 1) == 0 && !parked_wait(panel_full(pb), (pp / PANELS) & 1, abort_flag, kNapNs)) { ok = false; break; }
         const uint64_t a_desc = make_desc(smem_u32(xq_base + (xs >> 1) * XBUF_BYTES));
         const uint64_t b_desc = make_desc(smem_u32(panel_base + pb * C::PANEL_BYTES));
         for (int j = 0; j < 2; ++j) {
           const int u = 2 * s + j, slot = u % C::TMEM_SLOTS;
-          if (!parked_wait(slot_empty(slot), ((u / C::TMEM_SLOTS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          if (!parked_wait(slot_empty(slot), ((u / C::TMEM_SLOTS) & 1) ^ 1, abort_flag, kNapNs)) { ok = false; break; }
           tc_fence_after();
           const int kstep = (s & 1) * 2 + j;           // 32 bytes along the swizzled row: +2 in the address field
           umma_i8(tmem_base + slot * C::SLOT_COLS, a_desc + 2 * kstep, b_desc + 2 * kstep, idesc);
@@ -402,9 +434,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     if (lane == 0) {
       for (int s = 0; s < n_stages; ++s) {
         const int rs = s % RAW_SLOTS;
-        if (!parked_wait(raw_empty(rs), ((s / RAW_SLOTS) & 1) ^ 1, abort_flag)) break;
+        if (!parked_wait(raw_empty(rs), ((s / RAW_SLOTS) & 1) ^ 1, abort_flag, kNapNs)) break;
         mbar_expect_tx(raw_full(rs), p.x_bf16 ? RAW_BYTES / 2 : RAW_BYTES);       // rows and columns outside X arrive as zeros
-        tma_load_2d(smem_u32(raw_base + rs * RAW_BYTES), tmap_x, (pan_lo * 2 + s) * STAGE_COLS, row0, raw_full(rs));
+        const uint32_t dst = smem_u32(raw_base + rs * RAW_BYTES);
+        const int col = (pan_lo * 2 + s) * STAGE_COLS;
+        tma_load_2d(dst, tmap_x, col, row0, raw_full(rs));                         // a box is 128 bytes wide (swizzled rows):
+        if (!p.x_bf16) tma_load_2d(dst + RAW_BYTES / 2, tmap_x, col + STAGE_COLS / 2, row0, raw_full(rs));   // fp32 takes two
       }
     }
   }
@@ -587,10 +622,10 @@ cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, 
     if (m.k_pad != metas[0].k_pad) return cudaErrorInvalidValue;
     const cuuint64_t dims[2] = {(cuuint64_t)m.K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)m.K * (x_bf16 ? 2 : 4)};
-    const cuuint32_t box[2] = {STAGE_COLS, ROWS};
+    const cuuint32_t box[2] = {(cuuint32_t)(x_bf16 ? STAGE_COLS : STAGE_COLS / 2), ROWS};   // 128 bytes wide: one swizzled row
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&tmaps.m[i], x_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(Xs[g]), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
     Params& p = gp.L[i];

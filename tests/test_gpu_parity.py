@@ -130,6 +130,30 @@ def test_project_lowrank_tensor_core_prologue_bit_exact(spec):
     Pg.release()
 
 
+@pytest.mark.parametrize("path", [binding.PATH_AUTO, binding.PATH_TENSOR, binding.PATH_TENSOR_PROLOGUE, binding.PATH_SIMT],
+                         ids=["auto_small", "mma_sync_prologue", "tensor_prologue", "checking_kernel"])
+def test_adversarial_activations_through_every_prologue(path, ratio_log):
+    # zero, tie, clipped-maximum, subnormal, out-of-window, infinite and NaN blocks (the quantisers' slow path) through
+    # each prologue of the layer: X_q feeds T (bit-exact against the oracle) and Y (within the tolerance)
+    spec = gen.LayerSpec("adversarial", M=64, K=256, N=136, k=20, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=61)
+    W, A, B, P, Pg = _prepare(spec)
+    X = _adversarial_x()
+    ref = olqer.forward(X, P)
+    assert np.isfinite(ref.Y).all()
+    ws = L.new_workspace(spec.M, Pg)
+    L.set_path(path)
+    try:
+        Tm, Te = L.project_lowrank(_t(X), Pg, ws)
+        Y = L.linear(_t(X), Pg, ws).cpu().numpy()
+    finally:
+        L.set_path(binding.PATH_AUTO)
+    assert L.poll_status(ws) == 0
+    assert np.array_equal(Tm.cpu().numpy(), ref.Tm)
+    assert np.array_equal(Te.cpu().numpy(), exp_bytes(ref.Te))
+    assert ratio_log(f"adversarial_path{path}", worst_ratio(Y, ref)) <= 1.0
+    Pg.release()
+
+
 @pytest.mark.parametrize("a_bits", [6, 4])
 def test_activation_mantissa_width_option(a_bits):
     # W4A6 (Section 4.3) and a narrower width: X and T = X_q A_q take a_bits mantissa bits, everything else as before.
