@@ -243,14 +243,14 @@ def time_calls(fn, iters: int, warmup: int = 3) -> float:
     return e0.elapsed_time(e1) * 1e3 / iters
 
 
-def one_launch_per_call_us(L, calls, ws, iters: int, io_t=torch.float32) -> float:
+def one_launch_per_call_us(L, calls, ws, iters: int, x_t=torch.float32, y_t=torch.float32) -> float:
     """Microseconds for one pass over `calls` (decode-sized) with every call a launch of its own, in stream order, as a
     decoder must run layers that depend on one another.  The loop over the calls runs inside the library, so the
     figure is the device's, not the Python interpreter's."""
     from paper_2402_02446_b200 import binding
     L.set_path(binding.PATH_DECODE)
     try:
-        return time_calls(lambda i: L.linear_batched_ex(calls, ws, io_t, io_t), iters)
+        return time_calls(lambda i: L.linear_batched_ex(calls, ws, x_t, y_t), iters)
     finally:
         L.set_path(binding.PATH_AUTO)
 
@@ -401,17 +401,25 @@ def run_ours(args) -> None:
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     L.lib().lqer_workspace_init(ws.data_ptr(), ws_bytes, int(torch.cuda.current_stream().cuda_stream))
 
-    io_t = torch.bfloat16 if args.io == "bf16" else torch.float32
-    io_b = 2 if args.io == "bf16" else 4
-    X1 = [gen.make_activations_device(s[3], dev, M=M_DECODE).to(io_t) for s in shapes]
-    X2 = [gen.make_activations_device(s[3], dev, M=M_PREFILL).to(io_t) for s in shapes]
+    # element types at the boundary: X fp32 or bf16; Y fp32, bf16, or re-quantised to MXINT8 (17 bytes per 16 elements)
+    x_t = torch.float32 if args.io == "f32" else torch.bfloat16
+    y_t = torch.float32 if args.io == "f32" else torch.bfloat16 if args.io == "bf16" else L.MXINT8
+    x_b = 4 if args.io == "f32" else 2
+    y_b = 4.0 if args.io == "f32" else 2.0 if args.io == "bf16" else 17.0 / 16.0
+
+    def new_y(M, N, device=dev):
+        if y_t == L.MXINT8:
+            return torch.empty(L.mxint8_bytes(M, N), dtype=torch.uint8, device=device)
+        return torch.empty((M, N), dtype=y_t, device=device)
+
+    X1 = [gen.make_activations_device(s[3], dev, M=M_DECODE).to(x_t) for s in shapes]
+    X2 = [gen.make_activations_device(s[3], dev, M=M_PREFILL).to(x_t) for s in shapes]
     # outputs: one buffer per linear type and M (write-only; each is larger than a tile's reuse window)
-    Y1 = [torch.empty((M_DECODE, N), dtype=io_t, device=dev) for _, N, _, _ in shapes]
-    Y2_by_type = [torch.empty((M_PREFILL, gen.STACK_LINEARS[w][2]), dtype=io_t, device=dev)
-                  for w in range(len(gen.STACK_LINEARS))]
+    Y1 = [new_y(M_DECODE, N) for _, N, _, _ in shapes]
+    Y2_by_type = [new_y(M_PREFILL, gen.STACK_LINEARS[w][2]) for w in range(len(gen.STACK_LINEARS))]
     Y2 = [Y2_by_type[j % len(gen.STACK_LINEARS)] for j in range(n_lin)]
-    decode_calls = L.make_calls(zip(X1, packed, Y1), io_t, io_t)
-    prefill_calls = L.make_calls(zip(X2, packed, Y2), io_t, io_t)
+    decode_calls = L.make_calls(zip(X1, packed, Y1), x_t, y_t)
+    prefill_calls = L.make_calls(zip(X2, packed, Y2), x_t, y_t)
     # room for the shared launches of same-shape neighbours (one Xcat slice per layer of a group)
     ws_bytes = max(ws_bytes, L.batched_workspace_bytes(decode_calls), L.batched_workspace_bytes(prefill_calls))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
@@ -419,15 +427,15 @@ def run_ours(args) -> None:
 
     flops_decode = sum(layer_flops(M_DECODE, K, N, k) for K, N, k, _ in shapes)
     flops_prefill = sum(layer_flops(M_PREFILL, K, N, k) for K, N, k, _ in shapes)
-    bytes_decode = sum(layer_weight_bytes(K, N, k) + float(io_b) * M_DECODE * (K + N) for K, N, k, _ in shapes)
+    bytes_decode = sum(layer_weight_bytes(K, N, k) + (x_b * K + y_b * N) * M_DECODE for K, N, k, _ in shapes)
 
     stream = torch.cuda.current_stream()
 
     def step(mid_event=None):
-        L.linear_batched_ex(decode_calls, ws, io_t, io_t)
+        L.linear_batched_ex(decode_calls, ws, x_t, y_t)
         if mid_event is not None:
             mid_event.record(stream)
-        L.linear_batched_ex(prefill_calls, ws, io_t, io_t)
+        L.linear_batched_ex(prefill_calls, ws, x_t, y_t)
 
     def barrier():
         if dist is not None:
@@ -501,7 +509,7 @@ def run_ours(args) -> None:
                                    "traffic": traffic_of("decode", bytes_decode / c)}
     if "prologue" in fam:
         c, ms = fam["prologue"]
-        pb = sum(float(io_b) * M_PREFILL * K + 2.0 * M_PREFILL * ((K + 63) // 64 * 64 + (k + 15) // 16 * 16) for K, N, k, _ in shapes)
+        pb = sum(float(x_b) * M_PREFILL * K + 2.0 * M_PREFILL * ((K + 63) // 64 * 64 + (k + 15) // 16 * 16) for K, N, k, _ in shapes)
         ach = pb / (ms * 1e-3) / 1e9
         rooflines["hbm_prologue"] = {"bound": "hbm", "kernel": "prologue (activation quantisation + low-rank projection)",
                                      "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
@@ -509,7 +517,7 @@ def run_ours(args) -> None:
                                      "launches": c, "avg_launch_us": ms / c * 1e3, "traffic": traffic_of("prologue", pb / c)}
 
     # ---- the decode leg with every linear a launch of its own (stream order, as layers that depend on one another run)
-    dep_us = one_launch_per_call_us(L, decode_calls, ws, max(2, min(args.steps, 5)), io_t)
+    dep_us = one_launch_per_call_us(L, decode_calls, ws, max(2, min(args.steps, 5)), x_t, y_t)
     (dep_us,) = max_over_ranks([dep_us], dist, dev)
     decode_dependent = {"us_per_linear": dep_us / n_lin, "us_per_decoder_layer": dep_us / layers,
                         "hbm_gbs": bytes_decode / dep_us * 1e-3,
@@ -525,12 +533,12 @@ def run_ours(args) -> None:
     e2e = None
     if not args.no_e2e:
         types = len(gen.STACK_LINEARS)
-        hx1 = [torch.randn((M_DECODE, gen.STACK_LINEARS[w][1])).to(io_t).pin_memory() for w in range(types)]
-        hx2 = [torch.randn((M_PREFILL, gen.STACK_LINEARS[w][1])).to(io_t).pin_memory() for w in range(types)]
-        hy1 = [torch.empty((M_DECODE, gen.STACK_LINEARS[w][2]), dtype=io_t).pin_memory() for w in range(types)]
-        hy2 = [torch.empty((M_PREFILL, gen.STACK_LINEARS[w][2]), dtype=io_t).pin_memory() for w in range(types)]
-        calls1 = L.make_host_calls([(hx1[j % types], packed[j], hy1[j % types]) for j in range(n_lin)], io_t, io_t)
-        calls2 = L.make_host_calls([(hx2[j % types], packed[j], hy2[j % types]) for j in range(n_lin)], io_t, io_t)
+        hx1 = [torch.randn((M_DECODE, gen.STACK_LINEARS[w][1])).to(x_t).pin_memory() for w in range(types)]
+        hx2 = [torch.randn((M_PREFILL, gen.STACK_LINEARS[w][1])).to(x_t).pin_memory() for w in range(types)]
+        hy1 = [new_y(M_DECODE, gen.STACK_LINEARS[w][2], "cpu").pin_memory() for w in range(types)]
+        hy2 = [new_y(M_PREFILL, gen.STACK_LINEARS[w][2], "cpu").pin_memory() for w in range(types)]
+        calls1 = L.make_host_calls([(hx1[j % types], packed[j], hy1[j % types]) for j in range(n_lin)], x_t, y_t)
+        calls2 = L.make_host_calls([(hx2[j % types], packed[j], hy2[j % types]) for j in range(n_lin)], x_t, y_t)
         ws_h = torch.empty(max(L.linear_host_batched_bytes(calls1), L.linear_host_batched_bytes(calls2)),
                            dtype=torch.uint8, device=dev)
         L.lib().lqer_workspace_init(ws_h.data_ptr(), ws_h.numel(), int(stream.cuda_stream))
@@ -538,8 +546,8 @@ def run_ours(args) -> None:
         def e2e_step():
             # every layer's X goes host -> device and its Y device -> host inside the call; the copies of
             # neighbouring layers overlap the layer that is running
-            L.linear_host_batched_ex(calls1, ws_h, io_t, io_t, stream)
-            L.linear_host_batched_ex(calls2, ws_h, io_t, io_t, stream)
+            L.linear_host_batched_ex(calls1, ws_h, x_t, y_t, stream)
+            L.linear_host_batched_ex(calls2, ws_h, x_t, y_t, stream)
 
         e2e_step()
         barrier()
@@ -550,8 +558,8 @@ def run_ours(args) -> None:
         barrier()
         e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
         (e_ms,) = max_over_ranks([e_ms], dist, dev)
-        h2d = sum(io_b * (M_DECODE + M_PREFILL) * K for K, _, _, _ in shapes)
-        d2h = sum(io_b * (M_DECODE + M_PREFILL) * N for _, N, _, _ in shapes)
+        h2d = sum(x_b * (M_DECODE + M_PREFILL) * K for K, _, _, _ in shapes)
+        d2h = int(sum(y_b * (M_DECODE + M_PREFILL) * N for _, N, _, _ in shapes))
         e2e = {"value": world * (flops_decode + flops_prefill) / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                "ms_per_step": e_ms, "steps": e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "api": "lqer_linear_host_batched (224 layers per call, M=1 then M=2048), pinned host X and Y, "
@@ -610,7 +618,7 @@ def run_ours(args) -> None:
             "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
             "config": {"workload": (WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]") +
                                    ("" if args.a_bits == 8 else f" [activations MXINT{args.a_bits}]") +
-                                   ("" if args.w_bits == 4 else f" [weights MXINT{args.w_bits}]") + ("" if args.io == "f32" else " [bf16 X and Y]") +
+                                   ("" if args.w_bits == 4 else f" [weights MXINT{args.w_bits}]") + ("" if args.io == "f32" else " [bf16 X and Y]" if args.io == "bf16" else " [bf16 X, MXINT8 Y]") +
                                    ("" if args.rank is None else f" [rank {args.rank}]"),
                        "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32 if args.rank is None else args.rank,
                        "a_bits": args.a_bits, "w_bits": args.w_bits, "io": args.io,
@@ -651,8 +659,9 @@ def main() -> None:
     ap.add_argument("--a-bits", type=int, default=8, help="mantissa bits of the activations: 8 (W4A8, the workload) or 6 (W4A6)")
     ap.add_argument("--w-bits", type=int, default=4, help="mantissa bits of the weights: 4 (the workload) or 2 (W2A8, Section 4.4)")
     ap.add_argument("--rank", type=int, default=None, help="rank of the correction of every linear (default 32, the workload)")
-    ap.add_argument("--io", choices=["f32", "bf16"], default="f32",
-                    help="element type of X and Y at the layer's boundary: f32 (the workload) or bf16 (16-bit activations, Section 2.1)")
+    ap.add_argument("--io", choices=["f32", "bf16", "bf16-mxint8"], default="f32",
+                    help="element types of X and Y at the layer's boundary: f32 (the workload), bf16 (16-bit activations, "
+                         "Section 2.1), or bf16 X with Y re-quantised to MXINT8 by the epilogue (w&a setting)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the decode-layer, prefill-MLP and rank-sweep legs")
     ap.add_argument("--quick-configs", action="store_true", help="rank sweep at M = 1 and 512 only")

@@ -67,7 +67,8 @@ typedef struct {
  * between layers; the w&a settings quantise them on entry, which the layer does itself either way). */
 typedef enum {
   LQER_F32 = 0,
-  LQER_BF16 = 1
+  LQER_BF16 = 1,
+  LQER_MXINT8 = 2    /* output only: Y re-quantised to the layer's activation format, see lqer_linear_ex */
 } lqer_dtype_t;
 
 /* One call of a batch (Section 4.3: layers are independent). */
@@ -183,7 +184,13 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * y_dtype, both dense row-major and 16-byte aligned.  bf16 X is quantised to MXINT like fp32 X (every bf16
  * value is an fp32 value); bf16 Y is the fp32 result rounded to nearest even.  Everything else - packed,
  * workspace, paths, device-side status - as for lqer_linear_stream.  lqer_linear_batched_ex is
- * lqer_linear_batched with every call's X and Y of the given types (cast the pointers of lqer_call_t). */
+ * lqer_linear_batched with every call's X and Y of the given types (cast the pointers of lqer_call_t).
+ * y_dtype LQER_MXINT8 (Section 2.1, w&a setting: the activations between layers are quantised; Section 4.1:
+ * MXINT, blocks [1,16]): the epilogue quantises Y itself, in blocks of 16 along N (the next layer's K), to the
+ * layer's activation format (a_bits and exponent window of its lqer_config_t), exactly as the next layer's
+ * prologue would quantise the fp32 Y.  Y then points to M*N + M*N/16 bytes: the int8 mantissas [M,N] followed
+ * directly by the exponent bytes [M,N/16] (e + 127); N must be a multiple of 16.  Calls of up to 4 rows take
+ * the small-batch kernels for this output (the column-owner kernel's CTAs do not own whole blocks). */
 lqer_status_t lqer_linear_ex(const void* X, lqer_dtype_t x_dtype, int M, const void* packed, void* Y, lqer_dtype_t y_dtype,
                              void* workspace, size_t workspace_bytes, void* stream);
 lqer_status_t lqer_linear_batched_ex(const lqer_call_t* calls, int n_calls, lqer_dtype_t x_dtype, lqer_dtype_t y_dtype,

@@ -265,17 +265,35 @@ def linear(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y: torch.Tensor 
     return Y
 
 
-_DTYPES = {torch.float32: 0, torch.bfloat16: 1}
+MXINT8 = "mxint8"       # output type: a flat uint8 buffer, int8 mantissas [M, N] then exponent bytes [M, N / 16]
+_DTYPES = {torch.float32: 0, torch.bfloat16: 1, MXINT8: 2}
+
+
+def _tensor_dtype(dt):
+    return torch.uint8 if dt == MXINT8 else dt
+
+
+def mxint8_bytes(M: int, N: int) -> int:
+    return M * N + M * N // 16
+
+
+def split_mxint8(Y: torch.Tensor, M: int, N: int):
+    """Views of an MXINT8 output buffer: (mantissas int8 [M, N], exponent bytes uint8 [M, N / 16])."""
+    return Y[: M * N].view(torch.int8).view(M, N), Y[M * N: M * N + M * N // 16].view(M, N // 16)
 
 
 def linear_ex(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y: torch.Tensor | None = None,
-              out_dtype: torch.dtype = torch.float32, stream=None):
-    """The layer with fp32 or bf16 activations in and out (the types are taken from X and Y / out_dtype)."""
+              out_dtype=torch.float32, stream=None):
+    """The layer with fp32 or bf16 activations in and fp32, bf16 or MXINT8 out (the input type is taken from X, the output
+    type from out_dtype; an MXINT8 Y is a flat uint8 buffer of mxint8_bytes(M, N), see split_mxint8)."""
     M = X.shape[0]
     if Y is None:
-        Y = torch.empty((M, P.N), dtype=out_dtype, device=X.device)
-    _check(lib().lqer_linear_ex(_dev(X), _DTYPES[X.dtype], M, P.ptr, _dev(Y), _DTYPES[Y.dtype], ws.data_ptr(), ws.numel(),
-                                _stream(stream)), "lqer_linear_ex")
+        Y = (torch.empty(mxint8_bytes(M, P.N), dtype=torch.uint8, device=X.device) if out_dtype == MXINT8
+             else torch.empty((M, P.N), dtype=out_dtype, device=X.device))
+    elif out_dtype != MXINT8:
+        out_dtype = Y.dtype
+    _check(lib().lqer_linear_ex(_dev(X), _DTYPES[X.dtype], M, P.ptr, _dev(Y, _tensor_dtype(out_dtype)), _DTYPES[out_dtype],
+                                ws.data_ptr(), ws.numel(), _stream(stream)), "lqer_linear_ex")
     return Y
 
 
@@ -294,12 +312,12 @@ def linear_static(X: torch.Tensor, P: PackedWeights, Y: torch.Tensor | None = No
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
-def make_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype: torch.dtype = torch.float32) -> "C.Array":
+def make_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype=torch.float32) -> "C.Array":
     """items: iterable of (X, PackedWeights, Y) -> a host array of lqer_call_t."""
     items = list(items)
     arr = (Call * len(items))()
     for j, (X, P, Y) in enumerate(items):
-        arr[j] = Call(_dev(X, x_dtype), X.shape[0], P.ptr, _dev(Y, y_dtype))
+        arr[j] = Call(_dev(X, x_dtype), X.shape[0], P.ptr, _dev(Y, _tensor_dtype(y_dtype)))
     return arr
 
 
@@ -317,8 +335,9 @@ def linear_batched(calls, ws: torch.Tensor, stream=None) -> None:
            "lqer_linear_batched")
 
 
-def linear_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype: torch.dtype, stream=None) -> None:
-    """linear_batched with every X of x_dtype and every Y of y_dtype (fp32 or bf16); `calls` from make_calls(..., x_dtype, y_dtype)."""
+def linear_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype, stream=None) -> None:
+    """linear_batched with every X of x_dtype (fp32 or bf16) and every Y of y_dtype (fp32, bf16 or MXINT8); `calls` from
+    make_calls(..., x_dtype, y_dtype)."""
     _check(lib().lqer_linear_batched_ex(calls, len(calls), _DTYPES[x_dtype], _DTYPES[y_dtype], ws.data_ptr(), ws.numel(),
                                         _stream(stream)), "lqer_linear_batched_ex")
 
@@ -332,12 +351,12 @@ def linear_host(X_host: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y_host
     return Y_host
 
 
-def make_host_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype: torch.dtype = torch.float32) -> "C.Array":
+def make_host_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype=torch.float32) -> "C.Array":
     """items: iterable of (X_cpu, PackedWeights, Y_cpu), contiguous CPU tensors of the given types -> a host array of lqer_call_t."""
     items = list(items)
     arr = (Call * len(items))()
     for j, (X, P, Y) in enumerate(items):
-        for t, dt in ((X, x_dtype), (Y, y_dtype)):
+        for t, dt in ((X, x_dtype), (Y, _tensor_dtype(y_dtype))):
             if t.is_cuda or t.dtype != dt or not t.is_contiguous():
                 raise ValueError("expected contiguous CPU tensors of the stated types")
         arr[j] = Call(X.data_ptr(), X.shape[0], P.ptr, Y.data_ptr())
@@ -358,7 +377,7 @@ def linear_host_batched(calls, ws: torch.Tensor, stream=None) -> None:
            "lqer_linear_host_batched")
 
 
-def linear_host_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype: torch.dtype, stream=None) -> None:
+def linear_host_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype, stream=None) -> None:
     """linear_host_batched with host X of x_dtype and host Y of y_dtype; `calls` from make_host_calls(..., x_dtype, y_dtype)."""
     _check(lib().lqer_linear_host_batched_ex(calls, len(calls), _DTYPES[x_dtype], _DTYPES[y_dtype], ws.data_ptr(), ws.numel(),
                                              _stream(stream)), "lqer_linear_host_batched_ex")

@@ -201,7 +201,9 @@ static size_t workspace_total(const PackedMeta& m, int M_max) {
 
 // Element types of X and Y (Section 2.1: the layer sits between 16-bit activations in the w-only setting).
 struct IoTypes {
-  bool x_bf16 = false, y_bf16 = false;
+  bool x_bf16 = false;
+  int y_type = kYF32;          // kYF32, kYBF16 or kYMXINT8
+  bool y_bf16() const { return y_type == kYBF16; }
 };
 
 // n small-batch layers with one M (n == 1: a single call): one launch of the small prologue for all of them, then one
@@ -223,7 +225,7 @@ static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, 
     gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g]};
   }
   cudaError_t err = launch_prologue_small(pl, n, M, io.x_bf16, s);
-  if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_bf16, dst, s);
+  if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, dst, s);
   return err;
 }
 
@@ -237,6 +239,7 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   PackedMeta m;
   lqer_status_t st = lookup(packed, m);
   if (st != LQER_OK) return st;
+  if (io.y_type == kYMXINT8 && m.N % 16 != 0) return LQER_ERR_SHAPE;     // whole 16-blocks of Y along N
   int path = g_path.load();
   if ((path == 2 || path == 5) && M > kSmallMaxM) return LQER_ERR_SHAPE;
   const bool small = takes_small_path(path, M);
@@ -251,8 +254,8 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   void* xcat = wsb + align_up(persist_bytes(m), 256);
   cudaError_t err;
   if (small) {
-    if (path != 5 && !project_only && decode_cols_fits(m, M)) {
-      err = launch_decode_cols(X, io.x_bf16, M, m, packed, Y, io.y_bf16, workspace, s);
+    if (path != 5 && !project_only && io.y_type != kYMXINT8 && decode_cols_fits(m, M)) {
+      err = launch_decode_cols(X, io.x_bf16, M, m, packed, Y, io.y_bf16(), workspace, s);
     } else {
       const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
       uint8_t* slice = static_cast<uint8_t*>(xcat);
@@ -261,14 +264,14 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
       err = run_small(&one, &m, 1, &slice, &tiles, &rows, dst, io, Tm, Te, project_only, s);
     }
   } else {
-    if (path == 1 && (M > 65535 || io.y_bf16)) return LQER_ERR_SHAPE;   // the checking kernel writes fp32 only
+    if (path == 1 && (M > 65535 || io.y_type != kYF32)) return LQER_ERR_SHAPE;   // the checking kernel writes fp32 only
     err = tc_prologue ? launch_prologue_tc(X, io.x_bf16, M, m, packed, xcat, Tm, Te, dst,
                                            reinterpret_cast<double*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M)),
                                            reinterpret_cast<int*>(wsb + pcount_offset(m)), kChainAlone, s)
                       : launch_prologue(X, io.x_bf16, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
       err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, static_cast<float*>(Y), s)
-                        : launch_gemm_tc2_splitk(xcat, M, m, packed, Y, io.y_bf16,
+                        : launch_gemm_tc2_splitk(xcat, M, m, packed, Y, io.y_type,
                                                  reinterpret_cast<float*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M) +
                                                                           align_up(prologue_tc_scratch_bytes(m, M), 256)),
                                                  dst, s);
@@ -506,7 +509,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
       if (err != cudaSuccess) return LQER_ERR_CUDA;
     }
   }
-  return launch_gemm_tc2_group(xcats, packed, Ys, io.y_bf16, metas, n, M, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+  return launch_gemm_tc2_group(xcats, packed, Ys, io.y_type, metas, n, M, dst, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
 }
 
 }  // namespace lqer
@@ -748,7 +751,7 @@ lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y, v
 // The batched entry points: independent calls share launches where the path is left at 0.
 static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
                                     void* stream, IoTypes io) {
-  const bool cols_ok = true;
+  const bool cols_ok = io.y_type != kYMXINT8;    // the column-owner kernel's CTAs do not own whole 16-blocks of Y
   if (calls == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
   // validate everything before the first launch
@@ -762,6 +765,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
     if (st != LQER_OK) return st;
     const int path = g_path.load();
     if ((path == 2 || path == 5) && c.M > kSmallMaxM) return LQER_ERR_SHAPE;
+    if (io.y_type == kYMXINT8 && m.N % 16 != 0) return LQER_ERR_SHAPE;
     if (workspace_bytes < call_bytes(m, c.M, takes_small_path(path, c.M))) return LQER_ERR_BUFFER_TOO_SMALL;
   }
   const bool may_group = g_path.load() == 0;   // a forced path runs every call on its own
@@ -831,7 +835,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
         const int set = chain_open ? 1 - chain_set : 0;
         bool fills = false;
         if (launch_decode_cols_group(calls + i, metas, n, workspace, workspace_bytes, chain_open ? kChainLater : kChainFirst,
-                                     set, &fills, ahead ? pres : nullptr, io.x_bf16, io.y_bf16, cs) != cudaSuccess)
+                                     set, &fills, ahead ? pres : nullptr, io.x_bf16, io.y_bf16(), cs) != cudaSuccess)
           return LQER_ERR_CUDA;
         chain_open = fills;
         chain_set = set;
@@ -854,9 +858,10 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
 }
 
 static lqer_status_t io_types(lqer_dtype_t x_dtype, lqer_dtype_t y_dtype, IoTypes* io) {
-  if ((x_dtype != LQER_F32 && x_dtype != LQER_BF16) || (y_dtype != LQER_F32 && y_dtype != LQER_BF16)) return LQER_ERR_CONFIG;
+  if ((x_dtype != LQER_F32 && x_dtype != LQER_BF16) || (y_dtype != LQER_F32 && y_dtype != LQER_BF16 && y_dtype != LQER_MXINT8))
+    return LQER_ERR_CONFIG;
   io->x_bf16 = x_dtype == LQER_BF16;
-  io->y_bf16 = y_dtype == LQER_BF16;
+  io->y_type = y_dtype == LQER_BF16 ? kYBF16 : y_dtype == LQER_MXINT8 ? kYMXINT8 : kYF32;
   return LQER_OK;
 }
 
@@ -1003,7 +1008,7 @@ lqer_status_t lqer_linear_host_batched_bytes(const lqer_call_t* calls, int n_cal
 
 static lqer_status_t linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
                                          void* stream, IoTypes io) {
-  const size_t xe = io.x_bf16 ? 2 : 4, ye = io.y_bf16 ? 2 : 4;   // bytes per element on the host side and in the staging buffers
+  const size_t xe = io.x_bf16 ? 2 : 4;   // bytes per element of X on the host side and in the staging buffers
   if (calls == nullptr || workspace == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
@@ -1015,6 +1020,7 @@ static lqer_status_t linear_host_batched(const lqer_call_t* calls, int n_calls, 
     PackedMeta m;
     lqer_status_t st = lookup(c.packed, m);
     if (st != LQER_OK) return st;
+    if (io.y_type == kYMXINT8 && m.N % 16 != 0) return LQER_ERR_SHAPE;
     core = std::max(core, workspace_total(m, c.M));
     xb = std::max(xb, align_up((size_t)c.M * m.K * 4, 256));
     yb = std::max(yb, align_up((size_t)c.M * m.N * 4, 256));
@@ -1049,7 +1055,7 @@ static lqer_status_t linear_host_batched(const lqer_call_t* calls, int n_calls, 
     if (result != LQER_OK) break;
     ok = cudaEventRecord(hp->comp_done[b], s) == cudaSuccess &&
          cudaStreamWaitEvent(hp->out, hp->comp_done[b], 0) == cudaSuccess &&
-         cudaMemcpyAsync(c.Y, Yd[b], (size_t)c.M * m.N * ye, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess &&
+         cudaMemcpyAsync(c.Y, Yd[b], y_bytes(io.y_type, (size_t)c.M, (size_t)m.N), cudaMemcpyDeviceToHost, hp->out) == cudaSuccess &&
          cudaEventRecord(hp->out_done[b], hp->out) == cudaSuccess;
     if (!ok) result = LQER_ERR_CUDA;
   }

@@ -415,15 +415,18 @@ cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, 
                                      cudaStream_t s);
 cudaError_t launch_gemm_simt(const void* xcat, int M, const PackedMeta& m, const void* packed, float* Y,
                              cudaStream_t s);
-cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+// y_type: element type of Y (kYF32, kYBF16, kYMXINT8: mantissas [M,N] then exponent bytes [M,N/16], N % 16 == 0).
+constexpr int kYF32 = 0, kYBF16 = 1, kYMXINT8 = 2;
+inline size_t y_bytes(int y_type, size_t M, size_t N) { return y_type == kYMXINT8 ? M * N + M * N / 16 : M * N * (y_type == kYBF16 ? 2 : 4); }
+cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, int y_type,
                             DeviceStatus* st, cudaStream_t s);
 // Small batches: the layer's K range cut into gemm_splitk_ranges(m, M) ranges that run as layers of one launch;
 // `partials` holds (ranges - 1) * M * N floats (gemm_splitk_bytes).
-cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, int y_type,
                                    float* partials, DeviceStatus* st, cudaStream_t s);
 // Up to gemm_tc2_max_group() layers with one M in one launch (xcats, packed, Ys, metas: host arrays of n entries).
 int gemm_tc2_max_group();
-cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, void* const* Ys, bool y_bf16,
+cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, void* const* Ys, int y_type,
                                   const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s);
 // Factor preparation (Section 3.1 / 3.2, Appendix A): A_k, B_k from W and calibration samples, by randomised subspace
 // iteration with factor_sketch_rank columns; Omega [N, that many] fp32 is the caller's random test matrix.
@@ -452,12 +455,12 @@ struct SmallGemmLayer {
   const void* xcat;
   const void* packed;
   const PackedMeta* meta;
-  void* Y;                    // [M, N] fp32 or bf16
+  void* Y;                    // [M, N] fp32 or bf16, or the MXINT8 pair of sections
   float* partials;            // small_gemm_partial_bytes of scratch (unused if the tiles have one chunk)
   int* counters;              // one zeroed counter per 256-column tile
 };
 int gemm_small_max_layers();
-cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y_bf16, DeviceStatus* st, cudaStream_t s);
+cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_decode_cols(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);

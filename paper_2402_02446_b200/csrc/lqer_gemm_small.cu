@@ -58,7 +58,7 @@ struct Cfg {
 struct Layer {
   const uint8_t* wsec;
   const uint8_t* bsec;
-  void* Y;                     // [M, N] fp32 or bf16
+  void* Y;                     // [M, N] fp32 or bf16, or the MXINT8 sections (mantissas [M, N], exponent bytes [M, N / 16])
   float* partials;             // [tile][chunk][M][256] fp32 (tiles with more than one chunk)
   int* counters;               // [tile] arrivals, zero between calls
   int N, K64, n_tiles, k_slabs, r_blocks;
@@ -74,7 +74,8 @@ struct Params {
   DeviceStatus* status;
   int M;
   int lr_shift;
-  int y_bf16;                  // Y is bf16 (round to nearest even), else fp32
+  int y_type;                  // kYF32; kYBF16 (round to nearest even); kYMXINT8 (blocks of 16 along N, format below)
+  int a_bits, exp_min, exp_max;// activation format, for an MXINT8 Y
   int w_bits;                  // mantissa bits of W_q: 4 or 2 (one value for all layers of a launch)
   int x_rows;                  // rows of an activation tile that TMA fills: M rounded up to 8 (the rest stay zero)
   long long wait_limit;
@@ -112,8 +113,8 @@ __device__ __forceinline__ uint32_t bf16_rn(float v) {
   return u >> 16;
 }
 // Four consecutive elements of a row of Y.
-__device__ __forceinline__ void store_y4(void* Y, size_t idx, float4 v, int y_bf16) {
-  if (y_bf16)
+__device__ __forceinline__ void store_y4(void* Y, size_t idx, float4 v, int y_type) {
+  if (y_type == kYBF16)
     *reinterpret_cast<uint2*>(static_cast<uint16_t*>(Y) + idx) =
         make_uint2(bf16_rn(v.x) | (bf16_rn(v.y) << 16), bf16_rn(v.z) | (bf16_rn(v.w) << 16));
   else
@@ -150,7 +151,21 @@ __device__ __forceinline__ void reduce_tile(const Params& p, const Layer& ly, in
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int tk = t0 + rstep * u;
-      if (tk < p.M && quad_ok) store_y4(ly.Y, (size_t)tk * ly.N + col0 + c4, v[u], p.y_bf16);
+      if (p.y_type == kYMXINT8) {
+        // four adjacent lanes hold a 16-block of the row (every lane of the warp takes part in the exchange)
+        uint32_t m8;
+        uint2 unused;
+        int e;
+        quantize_quad(v[u], p.a_bits, p.exp_min, p.exp_max, e, m8, unused);
+        if (tk < p.M && quad_ok) {
+          uint8_t* yq = static_cast<uint8_t*>(ly.Y);
+          const size_t idx = (size_t)tk * ly.N + col0 + c4;
+          *reinterpret_cast<uint32_t*>(yq + idx) = m8;
+          if ((c4 & 15) == 0) yq[(size_t)p.M * ly.N + idx / 16] = (uint8_t)(e + 127);
+        }
+      } else if (tk < p.M && quad_ok) {
+        store_y4(ly.Y, (size_t)tk * ly.N + col0 + c4, v[u], p.y_type);
+      }
     }
   }
 }
@@ -337,12 +352,31 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c0, r);
           tmem_ld_wait();
           if (token < p.M) {
+            if (direct && p.y_type == kYMXINT8) {
+              // a token's 32 columns are two whole 16-blocks of its row
+              const QuantConsts qc = quant_consts(p.a_bits, p.exp_min, p.exp_max);
+              uint8_t* yq = static_cast<uint8_t*>(ly.Y);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                                           __uint_as_float(r[4 * j + 3]));
-              if (!direct) *reinterpret_cast<float4*>(prow + c0 + 4 * j) = v;
-              else if (col0 + c0 + 4 * j < ly.N) store_y4(ly.Y, (size_t)token * ly.N + col0 + c0 + 4 * j, v, p.y_bf16);   // N is a multiple of 8
+              for (int j = 0; j < 2; ++j)
+                if (col0 + c0 + 16 * j < ly.N) {          // N is a multiple of 16 here
+                  float v[16];
+#pragma unroll
+                  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[16 * j + i]);
+                  uint4 m8, b0, b1;
+                  int e;
+                  quantize_block16(v, qc, e, m8, b0, b1);
+                  const size_t idx = (size_t)token * ly.N + col0 + c0 + 16 * j;
+                  *reinterpret_cast<uint4*>(yq + idx) = m8;
+                  yq[(size_t)p.M * ly.N + idx / 16] = (uint8_t)(e + 127);
+                }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                                             __uint_as_float(r[4 * j + 3]));
+                if (!direct) *reinterpret_cast<float4*>(prow + c0 + 4 * j) = v;
+                else if (col0 + c0 + 4 * j < ly.N) store_y4(ly.Y, (size_t)token * ly.N + col0 + c0 + 4 * j, v, p.y_type);   // N is a multiple of 8
+              }
             }
           }
         }
@@ -482,7 +516,7 @@ static cudaError_t launch_mt(const TensorMaps& tmaps, const Params& p, int ctas,
 
 int gemm_small_max_layers() { return sg::MAX_LAYERS; }
 
-cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y_bf16, DeviceStatus* st, cudaStream_t s) {
+cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, DeviceStatus* st, cudaStream_t s) {
   using namespace sg;
   if (n < 1 || n > MAX_LAYERS || M < 1 || M > kSmallMaxM) return cudaErrorInvalidValue;
   EncodeTiledFn enc = encode_fn();
@@ -537,7 +571,8 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, bool y
   p.status = st;
   p.M = M;
   p.lr_shift = layers[0].meta->lr_bits - 2;
-  p.y_bf16 = y_bf16 ? 1 : 0;
+  p.y_type = y_type;
+  p.a_bits = layers[0].meta->a_bits; p.exp_min = layers[0].meta->exp_min; p.exp_max = layers[0].meta->exp_max;
   p.x_rows = x_rows;
   p.w_bits = layers[0].meta->w_bits;
   p.wait_limit = wait_limit_cycles();

@@ -61,7 +61,7 @@ struct TensorMaps {                        // one activation map per layer of th
 struct Layer {
   const uint8_t* wsec;
   const uint8_t* bsec;
-  void* Y;                     // [M, N] fp32, or bf16 where Params::y_bf16 (never for the K ranges of a split layer)
+  void* Y;                     // [M, N] fp32; bf16 or the MXINT8 sections by Params::y_type (never for the K ranges of a split layer)
   int N, K64;
   int n_tiles, k_slabs, r_blocks;
   int slab0, slab_stride;      // a layer may be a K range of a real layer (split K): its first weight slab, and the
@@ -77,7 +77,8 @@ struct Params {
   DeviceStatus* status;
   int M, m_tiles;              // row tiles of 256 (the same M for every layer)
   int lr_shift;
-  int y_bf16;                  // Y is bf16 (round to nearest even), else fp32
+  int y_type;                  // kYF32; kYBF16 (round to nearest even); kYMXINT8 (blocks of 16 along N, format below)
+  int a_bits, exp_min, exp_max;// activation format, for an MXINT8 Y
   int w_bits;                  // mantissa bits of W_q: 4 or 2 (one value for all layers of a launch)
   long long wait_limit;        // bound of every wait, in clock cycles
   int stall;                   // test hook: the producers withhold the last stage of their last tile, so the waits run out
@@ -251,19 +252,36 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       const size_t yoff = (size_t)row * Nl + (size_t)nt * BN;
       float* yrow = static_cast<float*>(p.L[layer].Y) + yoff;
       uint16_t* yrow16 = static_cast<uint16_t*>(p.L[layer].Y) + yoff;
+      // MXINT8 Y: mantissas [M, N], then exponent bytes [M, N / 16]; a thread holds whole 16-blocks of its row
+      uint8_t* yq = static_cast<uint8_t*>(p.L[layer].Y) + yoff;
+      uint8_t* yqe = static_cast<uint8_t*>(p.L[layer].Y) + (size_t)p.M * Nl + ((size_t)row * Nl + (size_t)nt * BN) / 16;
+      const QuantConsts qc = quant_consts(p.a_bits, p.exp_min, p.exp_max);
       for (int c = 0; c < BN; c += 32) {
         if (c >= ncols) break;
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, r);
         tmem_ld_wait();
         if (row < p.M) {
-          if (p.y_bf16) {
+          if (p.y_type == kYBF16) {
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               if (c + 8 * j < ncols)                      // N is a multiple of 8
                 *reinterpret_cast<uint4*>(yrow16 + c + 8 * j) =
                     make_uint4(bf16x2_rn(r[8 * j], r[8 * j + 1]), bf16x2_rn(r[8 * j + 2], r[8 * j + 3]),
                                bf16x2_rn(r[8 * j + 4], r[8 * j + 5]), bf16x2_rn(r[8 * j + 6], r[8 * j + 7]));
+          } else if (p.y_type == kYMXINT8) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              if (c + 16 * j < ncols) {                   // N is a multiple of 16 here
+                float v[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[16 * j + i]);
+                uint4 m8, b0, b1;
+                int e;
+                quantize_block16(v, qc, e, m8, b0, b1);
+                *reinterpret_cast<uint4*>(yq + c + 16 * j) = m8;
+                yqe[(c >> 4) + j] = (uint8_t)(e + 127);
+              }
           } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -417,12 +435,12 @@ __global__ void __launch_bounds__(256) splitk_sum_kernel(float4* __restrict__ Y,
 
 // Small batches have few tiles; their K range is cut into ranges that run as layers of one launch, the first into Y,
 // the others into scratch that a second kernel adds to Y in a fixed order.
-cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Yv, bool y_bf16,
+cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Yv, int y_type,
                                    float* partials, DeviceStatus* st, cudaStream_t s) {
   using namespace tc2;
   const int C = gemm_splitk_ranges(m, M);
-  // a 16-bit Y cannot collect the ranges' sums: such a layer runs whole
-  if (C < 2 || y_bf16) return launch_gemm_tc2(xcat, M, m, packed, Yv, y_bf16, st, s);
+  // only an fp32 Y can collect the ranges' sums: a layer with another output type runs whole
+  if (C < 2 || y_type != kYF32) return launch_gemm_tc2(xcat, M, m, packed, Yv, y_type, st, s);
   float* Y = static_cast<float*>(Yv);
   if ((m.N & 3) != 0) return cudaErrorInvalidValue;
   EncodeTiledFn enc = encode_fn();
@@ -461,7 +479,8 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
   p.status = st;
   p.M = M;
   p.lr_shift = m.lr_bits - 2;
-  p.y_bf16 = 0;
+  p.y_type = kYF32;
+  p.a_bits = m.a_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
   p.w_bits = m.w_bits;
   cudaError_t e = launch_params(tmaps, p, s);
   if (e != cudaSuccess) return e;
@@ -473,9 +492,9 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
   return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+cudaError_t launch_gemm_tc2(const void* xcat, int M, const PackedMeta& m, const void* packed, void* Y, int y_type,
                             DeviceStatus* st, cudaStream_t s) {
-  return launch_gemm_tc2_group(&xcat, &packed, &Y, y_bf16, &m, 1, M, st, s);
+  return launch_gemm_tc2_group(&xcat, &packed, &Y, y_type, &m, 1, M, st, s);
 }
 
 int gemm_tc2_max_group() { return tc2::MAX_GROUP; }
@@ -483,7 +502,7 @@ int gemm_tc2_max_group() { return tc2::MAX_GROUP; }
 // n layers with one M (shapes may differ, formats must not) as ONE launch: the tiles of all layers form one list that
 // the CTA pairs walk, so the pairs idle only at the end of the whole list, and set-up and the last epilogue are paid
 // once.  Layers with more K stages per tile come first in the list.
-cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, void* const* Ys, bool y_bf16,
+cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* packed, void* const* Ys, int y_type,
                                   const PackedMeta* metas, int n, int M, DeviceStatus* st, cudaStream_t s) {
   using namespace tc2;
   if (n < 1 || n > MAX_GROUP) return cudaErrorInvalidValue;
@@ -529,7 +548,8 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
   p.status = st;
   p.M = M;
   p.lr_shift = metas[0].lr_bits - 2;
-  p.y_bf16 = y_bf16 ? 1 : 0;
+  p.y_type = y_type;
+  p.a_bits = metas[0].a_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
   p.w_bits = metas[0].w_bits;
   return launch_params(tmaps, p, s);
 }

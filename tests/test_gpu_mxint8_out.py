@@ -1,0 +1,185 @@
+"""MXINT8 output (Section 2.1, w&a setting: the activations between layers are quantised; Section 4.1: MXINT8,
+blocks [1,16]): with y_dtype LQER_MXINT8 the epilogue quantises Y in blocks of 16 along N, as the next layer's
+prologue would.
+
+Parity against the oracle.  The oracle quantises its fp64 Y, the library its fp32 Y; the two Y differ by at most the
+layer's tolerance, and a quantised code is a decision taken on that value.  So:
+  * every dequantised element lies within tol + half a quantisation step of the oracle's Y (a whole step where the
+    symmetric clamp holds the block's maximum at 2^(b-1) - 1);
+  * a block's shared exponent equals the oracle's unless the block maximum lies within tol of a power of two
+    (then it may be the neighbouring exponent);
+  * where the exponents agree, a mantissa equals the oracle's unless the oracle's scaled value lies within tol of
+    a rounding tie (then it may differ by one).
+The quantiser itself is also checked in the kernel's own precision: the codes are exactly what round-to-nearest-even
+with the block's exponent gives on the fp32 Y the same path writes.
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import lqer_inputs as gen
+import paper_2402_02446_b200 as L
+from paper_2402_02446_b200 import binding
+from oracle import lqer as olqer
+from oracle import mxint
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+E = binding.STATUS_NAMES.index
+
+
+def _t(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def _layer(spec):
+    W = gen.make_weight(spec)
+    if spec.k == 0:
+        return olqer.prepare_weights(W, None, None), L.prepare_weights(_t(W), None, None)
+    A, B = gen.make_random_factors(spec)
+    return olqer.prepare_weights(W, A, B), L.prepare_weights(_t(W), _t(A), _t(B))
+
+
+def _check_against_oracle(Ym, Ye, ref, a_bits=8):
+    """Ym int8 [M, N], Ye exponent bytes [M, N/16] from the library; ref: the oracle's forward result."""
+    M, N = ref.Y.shape
+    e_gpu = Ye.astype(np.int64) - 127
+    om, oe = mxint.quantize(ref.Y, a_bits, axis=1)
+    oe = np.asarray(oe, dtype=np.int64)
+    shift = a_bits - 2
+    step = np.repeat(np.exp2((e_gpu - shift).astype(np.float64)), 16, axis=1)
+    dq = Ym.astype(np.float64) * step
+    # (1) every element within tol + half a step (a whole step where the symmetric clamp holds a block maximum at qmax)
+    qmax = 2 ** (a_bits - 1) - 1
+    room = np.where(np.abs(Ym.astype(np.int64)) == qmax, 1.0, 0.5) * step
+    assert np.all(np.abs(dq - ref.Y) <= ref.tol + room * (1 + 1e-12))
+    # (2) exponents: the oracle's, or the neighbour where the block maximum is within tol of a power of two
+    tol_blk = ref.tol.reshape(M, N // 16, 16).max(axis=2)
+    amax = np.abs(ref.Y).reshape(M, N // 16, 16).max(axis=2)
+    lo = np.floor(np.log2(np.maximum(amax - tol_blk, 2.0 ** -60)))
+    hi = np.floor(np.log2(np.maximum(amax + tol_blk, 2.0 ** -60)))
+    lo, hi = np.clip(lo, -56, 55), np.clip(hi, -56, 55)
+    assert np.all((e_gpu >= lo) & (e_gpu <= hi))
+    # (3) mantissas where the exponents agree: equal, or one apart next to a tie
+    same = np.repeat(e_gpu == oe, 16, axis=1)
+    diff = Ym.astype(np.int64) - om.astype(np.int64)
+    assert np.all(np.abs(diff[same]) <= 1)
+    off = same & (diff != 0)
+    if off.any():
+        scaled = ref.Y[off] / step[off]
+        to_tie = np.abs(np.abs(scaled - np.floor(scaled)) - 0.5)
+        assert np.all(to_tie <= ref.tol[off] / step[off] + 1e-9)
+    return float(np.mean(same)), int(off.sum())
+
+
+def _check_own_precision(Ym, Ye, Y32, a_bits=8):
+    """The codes against the fp32 Y of the same path, in the kernel's precision: exponent from the block's maximum,
+    round to nearest even, symmetric clamp."""
+    M, N = Y32.shape
+    blk = Y32.reshape(M, N // 16, 16).astype(np.float64)
+    amax = np.abs(blk).max(axis=2)
+    e = np.clip(np.floor(np.log2(np.maximum(amax, 2.0 ** -100))), -56, 55)
+    assert np.array_equal(Ye.astype(np.int64) - 127, e.astype(np.int64))
+    q = 2 ** (a_bits - 1) - 1
+    m = np.clip(np.rint(blk / np.exp2(e - (a_bits - 2))[:, :, None]), -q, q)       # rint: half to even
+    assert np.array_equal(Ym.reshape(M, N // 16, 16).astype(np.int64), m.astype(np.int64))
+
+
+SPECS = [gen.LayerSpec("q_a", M=300, K=1024, N=640, k=40, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=401),
+         gen.LayerSpec("q_k0", M=129, K=512, N=400, k=0, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=402),
+         gen.LayerSpec("q_tc", M=1100, K=2112, N=272, k=64, calib_rows=32, outlier_frac=0.005, outlier_scale=50.0,
+                       weight_law="student_t4", seed=403)]
+
+
+@pytest.mark.parametrize("spec", SPECS, ids=lambda s: s.name)
+def test_mxint8_output_every_path(spec):
+    # small-batch kernels (1, 4, 9, 70 rows; the chunks of a tile meet in the last arriver's reduction or the tile is
+    # written directly), the pair GEMM without split K (200) and behind either prologue (the spec's own M)
+    P, Pg = _layer(spec)
+    ws = L.new_workspace(spec.M, Pg)
+    for M in (1, 4, 9, 70, 200, spec.M):
+        if M > spec.M:
+            continue
+        X = gen.make_activations(spec, M=M)
+        ref = olqer.forward(X, P)
+        Yq = L.linear_ex(_t(X), Pg, ws, out_dtype=L.MXINT8)
+        assert L.poll_status(ws) == 0
+        Ym, Ye = L.split_mxint8(Yq, M, spec.N)
+        _check_against_oracle(Ym.cpu().numpy(), Ye.cpu().numpy(), ref)
+        # the same path with an fp32 Y (M <= 4 takes the small-batch kernels for an MXINT8 Y; M <= 256 would cut K for fp32)
+        if M <= 128:
+            L.set_path(binding.PATH_SMALL)
+        try:
+            Y32 = L.linear(_t(X), Pg, ws).cpu().numpy() if not (128 < M <= 256) else None
+        finally:
+            L.set_path(binding.PATH_AUTO)
+        if Y32 is not None:
+            _check_own_precision(Ym.cpu().numpy(), Ye.cpu().numpy(), Y32)
+    Pg.release()
+
+
+def test_mxint8_output_where_the_sums_round():
+    # long K, all terms of one sign: the fp32 sums differ from the oracle's fp64 sums, so codes next to ties and block
+    # maxima next to powers of two may legitimately differ; the three rules above must still hold
+    spec = gen.LayerSpec("q_round", M=40, K=11008, N=256, k=32, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=404)
+    W = np.abs(gen.make_weight(spec))
+    A, B = gen.make_random_factors(spec)
+    P, Pg = olqer.prepare_weights(W, A, B), L.prepare_weights(_t(W), _t(A), _t(B))
+    X = np.abs(gen.make_activations(spec))
+    ref = olqer.forward(X, P)
+    ws = L.new_workspace(spec.M, Pg)
+    Yq = L.linear_ex(_t(X), Pg, ws, out_dtype=L.MXINT8)
+    Ym, Ye = L.split_mxint8(Yq, spec.M, spec.N)
+    same, off = _check_against_oracle(Ym.cpu().numpy(), Ye.cpu().numpy(), ref)
+    assert same > 0.9
+    Pg.release()
+
+
+def test_mxint8_output_of_shared_launches_and_host_buffers():
+    # three prefill layers in one GEMM launch, three small-batch layers in one launch, and the host-buffer entry point
+    specs = [gen.LayerSpec("q_g0", M=300, K=512, N=256, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=411),
+             gen.LayerSpec("q_g1", M=300, K=1024, N=384, k=32, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=412),
+             gen.LayerSpec("q_g2", M=300, K=320, N=512, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=413)]
+    layers = [_layer(s) for s in specs]
+    for M in (300, 24, 3):
+        Xs = [gen.make_activations(s, M=M) for s in specs]
+        refs = [olqer.forward(X, P) for X, (P, _) in zip(Xs, layers)]
+        Yq = [torch.zeros(L.mxint8_bytes(M, s.N), dtype=torch.uint8, device=DEV) for s in specs]
+        Xd = [_t(X) for X in Xs]                          # the calls hold pointers only: keep the tensors alive
+        calls = L.make_calls([(x, Pg, y) for x, (_, Pg), y in zip(Xd, layers, Yq)], torch.float32, L.MXINT8)
+        ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+        before = L.launch_count()
+        L.linear_batched_ex(calls, ws, torch.float32, L.MXINT8)
+        torch.cuda.synchronize()
+        assert L.launch_count() - before <= 4           # shared launches: prologue(s) + one GEMM, not one pair per layer
+        assert L.poll_status(ws) == 0
+        for s, y, ref in zip(specs, Yq, refs):
+            Ym, Ye = L.split_mxint8(y, M, s.N)
+            _check_against_oracle(Ym.cpu().numpy(), Ye.cpu().numpy(), ref)
+        # host buffers
+        Xh = [torch.from_numpy(X).pin_memory() for X in Xs]
+        Yh = [torch.zeros(L.mxint8_bytes(M, s.N), dtype=torch.uint8).pin_memory() for s in specs]
+        hcalls = L.make_host_calls([(x, Pg, y) for x, (_, Pg), y in zip(Xh, layers, Yh)], torch.float32, L.MXINT8)
+        wsh = torch.zeros(L.linear_host_batched_bytes(hcalls), dtype=torch.uint8, device=DEV)
+        L.linear_host_batched_ex(hcalls, wsh, torch.float32, L.MXINT8)
+        for y_dev, y_host in zip(Yq, Yh):
+            assert torch.equal(y_dev.cpu(), y_host)
+    for _, Pg in layers:
+        Pg.release()
+
+
+def test_mxint8_output_is_refused_where_it_cannot_be_written():
+    spec = gen.LayerSpec("q_n8", M=8, K=64, N=136, k=0, calib_rows=32, outlier_frac=0, n_outliers=1, outlier_scale=20.0, seed=421)
+    P, Pg = _layer(spec)                                  # N = 136 is a multiple of 8, not of 16
+    ws = L.new_workspace(spec.M, Pg)
+    X = _t(gen.make_activations(spec))
+    Y = torch.zeros(L.mxint8_bytes(spec.M, 144), dtype=torch.uint8, device=DEV)
+    launches = L.launch_count()
+    st = L.lib().lqer_linear_ex(X.data_ptr(), 0, spec.M, Pg.ptr, Y.data_ptr(), 2, ws.data_ptr(), ws.numel(), None)
+    assert st == E("LQER_ERR_SHAPE")
+    st = L.lib().lqer_linear_ex(X.data_ptr(), 2, spec.M, Pg.ptr, Y.data_ptr(), 0, ws.data_ptr(), ws.numel(), None)
+    assert st == E("LQER_ERR_CONFIG")                     # MXINT8 is an output type only
+    assert L.launch_count() == launches
+    Pg.release()
