@@ -296,6 +296,16 @@ lqer_status_t lqer_set_path(int path);
 lqer_status_t lqer_set_wait_limit_cycles(long long cycles);
 lqer_status_t lqer_inject_stall(int kernel_family);
 
+/* The checked build of the library (liblqer_dbg.so, compiled with -DLQER_DEBUG_BOUNDS; the paper has no counterpart).
+ * Every global store of the inference kernels and every bulk copy of packed weights first checks its byte range
+ * against the extent of the buffer it belongs to; the first violation is written to the status word
+ * (LQER_ERR_BOUNDS; lqer_poll_status) and the access is skipped - nothing traps, nothing out of range is touched.
+ * It stands in for a memory checker where none can be run.  lqer_debug_bounds_shrink (host, process wide) is its test
+ * hook: the declared extent of every Y is made `bytes` smaller for the launches that follow, so that the checks at
+ * the end of Y fire (the stores they guard are skipped; Y is then incomplete); 0 restores.  The ordinary build
+ * returns LQER_ERR_CONFIG. */
+lqer_status_t lqer_debug_bounds_shrink(long long bytes);
+
 /* Number of kernels launched by the library in this process so far (host). */
 unsigned long long lqer_launch_count(void);
 

@@ -12,7 +12,9 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "lib", "liblqer.so")
+# LQER_DEBUG_BOUNDS=1 in the environment selects the checked build of the library (see include/lqer.h).
+DEBUG_BOUNDS = os.environ.get("LQER_DEBUG_BOUNDS", "0") not in ("", "0")
+_LIB_PATH = os.path.join(_HERE, "lib", "liblqer_dbg.so" if DEBUG_BOUNDS else "liblqer.so")
 _lib = None
 
 STATUS_NAMES = ["LQER_OK", "LQER_ERR_NULL", "LQER_ERR_SHAPE", "LQER_ERR_ALIGN", "LQER_ERR_CONFIG",
@@ -68,6 +70,7 @@ def lib() -> C.CDLL:
             "lqer_call_workspace_bytes": (i, [i, i, i, i, cfgp, C.POINTER(sz)]),
             "lqer_set_wait_limit_cycles": (i, [C.c_longlong]),
             "lqer_inject_stall": (i, [i]),
+            "lqer_debug_bounds_shrink": (i, [C.c_longlong]),
             "lqer_prepare_weights": (i, [vp, vp, vp, i, i, i, cfgp, vp, sz, vp]),
             "lqer_factor_sketch_columns": (i, [i, i, i, C.POINTER(i)]),
             "lqer_prepare_workspace_bytes": (i, [i, i, i, C.POINTER(sz)]),
@@ -400,6 +403,12 @@ def set_wait_limit_cycles(cycles: int) -> None:
 def inject_stall(kernel_family: int) -> None:
     """Test hook: the next launch of that kernel family waits for something that never comes (-1 disarms)."""
     _check(lib().lqer_inject_stall(kernel_family), "lqer_inject_stall")
+
+
+def debug_bounds_shrink(nbytes: int) -> None:
+    """Test hook of the checked build: the declared extent of every Y shrinks by nbytes for the launches that follow, so the
+    bounds checks at the end of Y fire (their stores are skipped); 0 restores.  The ordinary build refuses."""
+    _check(lib().lqer_debug_bounds_shrink(nbytes), "lqer_debug_bounds_shrink")
 
 
 def launch_count() -> int:

@@ -35,7 +35,16 @@ def _stale(target: str, deps: list[str]) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+LIB_DEBUG = os.path.join(OUT_DIR, "liblqer_dbg.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    """Compiles the library.  debug_bounds: the checked build (-DLQER_DEBUG_BOUNDS -> lib/liblqer_dbg.so), whose kernels
+    check every global store and weight copy against its buffer's extent and report the first violation through the
+    status word; the binding loads it when LQER_DEBUG_BOUNDS=1 is in the environment."""
+    OBJ_DIR = os.path.join(HERE, "_build_dbg" if debug_bounds else "_build")
+    LIB = LIB_DEBUG if debug_bounds else globals()["LIB"]
+    NVCC_FLAGS = globals()["NVCC_FLAGS"] + (["-DLQER_DEBUG_BOUNDS"] if debug_bounds else [])
     os.makedirs(OUT_DIR, exist_ok=True)
     os.makedirs(OBJ_DIR, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
@@ -69,5 +78,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_all(force: bool = False, verbose: bool = False) -> list[str]:
+    """The library and its checked build."""
+    return [build(force, verbose), build(force, verbose, debug_bounds=True)]
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    for path in build_all(force="--force" in sys.argv, verbose="-v" in sys.argv):
+        print(path)

@@ -47,6 +47,8 @@ static std::atomic<long long> g_wait_limit{4000000000LL};      // about two seco
 static std::atomic<int> g_stall_family{-1};
 
 long long wait_limit_cycles() { return g_wait_limit.load(std::memory_order_relaxed); }
+static std::atomic<size_t> g_y_shrink{0};                      // checked build only: see lqer_debug_bounds_shrink
+size_t debug_y_shrink() { return g_y_shrink.load(std::memory_order_relaxed); }
 
 bool take_stall(int family) {
   int want = family;
@@ -224,7 +226,7 @@ static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, 
                                n == 1 ? Tm : nullptr, n == 1 ? Te : nullptr};
     gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g]};
   }
-  cudaError_t err = launch_prologue_small(pl, n, M, io.x_bf16, s);
+  cudaError_t err = launch_prologue_small(pl, n, M, io.x_bf16, dst, s);
   if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, dst, s);
   return err;
 }
@@ -1097,6 +1099,13 @@ lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_
   if (cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return LQER_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return LQER_ERR_CUDA;
   *device_status = (h.code >= 0 && h.code <= LQER_ERR_BOUNDS) ? (lqer_status_t)h.code : LQER_ERR_CUDA;
+  return LQER_OK;
+}
+
+lqer_status_t lqer_debug_bounds_shrink(long long bytes) {
+  if (!kDebugBounds) return LQER_ERR_CONFIG;          // the ordinary build has no checks to trip
+  if (bytes < 0 || bytes > (1LL << 40)) return LQER_ERR_CONFIG;
+  g_y_shrink.store((size_t)bytes);
   return LQER_OK;
 }
 

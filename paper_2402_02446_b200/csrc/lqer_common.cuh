@@ -331,6 +331,26 @@ __device__ __forceinline__ void report_error(DeviceStatus* st, int code, int whe
   }
 }
 
+// Checked build (-DLQER_DEBUG_BOUNDS; the library is then liblqer_dbg.so): every global store of the inference kernels,
+// and every bulk copy of packed weights, first checks its byte range against the extent of the buffer it goes to
+// (or comes from).  The first violation goes to the status word (LQER_ERR_BOUNDS, the site, offset and extent in
+// 16-byte units) and the access is skipped: nothing traps and nothing out of range is touched.  In the ordinary build
+// the macro is the constant true and the extents in the kernels' parameters are dead.
+#ifdef LQER_DEBUG_BOUNDS
+__device__ __forceinline__ bool in_bounds(DeviceStatus* st, size_t off, size_t len, size_t extent, int site) {
+  if (off + len <= extent) return true;
+  report_error(st, LQER_ERR_BOUNDS, site, (int)(off >> 4), (int)(extent >> 4));
+  return false;
+}
+#define LQER_IN_BOUNDS(st, off, len, extent, site) ::lqer::in_bounds(st, (size_t)(off), (size_t)(len), (size_t)(extent), site)
+constexpr bool kDebugBounds = true;
+#else
+#define LQER_IN_BOUNDS(st, off, len, extent, site) true
+constexpr bool kDebugBounds = false;
+#endif
+// Test hook of the checked build (lqer_debug_bounds_shrink): bytes taken off the declared extent of Y at the next launches.
+size_t debug_y_shrink();
+
 // ----------------------------------------------------------------------------
 // Per-device host state
 // ----------------------------------------------------------------------------
@@ -448,7 +468,7 @@ struct SmallPrologueLayer {
   uint8_t* Te;
 };
 int prologue_small_max_layers();
-cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, cudaStream_t s);
+cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, DeviceStatus* st, cudaStream_t s);
 // The small-batch GEMM (tokens on the M side of a 64- or 128-row MMA, 256 weight columns on its N side); up to
 // gemm_small_max_layers() layers with one M per launch.
 struct SmallGemmLayer {

@@ -34,6 +34,8 @@
 //
 // Launches of one batched call that follow one another share no buffer and need not wait for one
 // another (ChainOrder): a launch fills the SMs as the one before leaves them.
+#include <algorithm>
+
 #include "lqer_common.cuh"
 
 namespace lqer {
@@ -54,6 +56,7 @@ constexpr int kMaxGroup = 16;  // independent layers with one M that may share a
 struct Layer {
   const void* X;                // [M, K] fp32, or bf16 where Params::x_bf16
   void* Y;                      // [M, N] fp32, or bf16 where Params::y_bf16
+  size_t y_extent;              // bytes behind Y, for the checked build
   const uint8_t* packed;
   size_t off_w, off_b, off_a;   // sections of the packed buffer
   int K, N, K64, k_pad, k_slabs, r_blocks, n_cg;
@@ -612,7 +615,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
             float v = 0.f;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) v += red_now[((h * kWarps + w) * 32 + col) * kMaxM + r];
-            if (p.y_bf16) {
+            if (!LQER_IN_BOUNDS(p.status, ((size_t)r * ly.N + c0 * 8 + col) * (p.y_bf16 ? 2 : 4), p.y_bf16 ? 2 : 4, ly.y_extent, 711)) {
+            } else if (p.y_bf16) {
               uint32_t u = __float_as_uint(v);               // round to nearest even (NaN / inf keep their class)
               u = ((u & 0x7F800000u) == 0x7F800000u) ? ((u >> 16) | ((u & 0xFFFFu) ? 0x40u : 0u)) : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
               static_cast<uint16_t*>(Y)[(size_t)r * ly.N + c0 * 8 + col] = (uint16_t)u;
@@ -734,6 +738,8 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
       return cudaErrorInvalidValue;
     Layer& ly = p.L[i];
     ly.X = calls[g].X; ly.Y = calls[g].Y; ly.packed = static_cast<const uint8_t*>(calls[g].packed);
+    ly.y_extent = (size_t)calls[g].M * metas[g].N * (y_bf16 ? 2 : 4);
+    if (kDebugBounds) ly.y_extent -= std::min(ly.y_extent, debug_y_shrink());
     ly.off_w = m.off_w; ly.off_b = m.off_b; ly.off_a = m.off_a;
     ly.K = m.K; ly.N = m.N; ly.K64 = m.K64; ly.k_pad = m.k_pad;
     ly.k_slabs = m.k_slabs; ly.r_blocks = m.r_blocks;

@@ -25,6 +25,8 @@
 // Two rings: PK slots hold {activation tile, two packed weight tiles}, with a barrier for the weights and one for
 // the activations (the converters need only the former, so they work while the prologue still runs); CV slots
 // hold converted weight tiles.
+#include <algorithm>
+
 #include "lqer_tc_ptx.cuh"
 
 namespace lqer {
@@ -61,6 +63,8 @@ struct Layer {
   void* Y;                     // [M, N] fp32 or bf16, or the MXINT8 sections (mantissas [M, N], exponent bytes [M, N / 16])
   float* partials;             // [tile][chunk][M][256] fp32 (tiles with more than one chunk)
   int* counters;               // [tile] arrivals, zero between calls
+  size_t y_extent, partial_extent;   // bytes behind Y and behind partials, for the checked build
+  size_t w_extent, b_extent;         // bytes of the packed W and B sections
   int N, K64, n_tiles, k_slabs, r_blocks;
   int spt;                     // K stages per tile: k_slabs + rank stages
   int chunks, chunk_stages;    // K chunks per tile; weight stages per chunk (the last chunk also takes the rank stages)
@@ -113,7 +117,8 @@ __device__ __forceinline__ uint32_t bf16_rn(float v) {
   return u >> 16;
 }
 // Four consecutive elements of a row of Y.
-__device__ __forceinline__ void store_y4(void* Y, size_t idx, float4 v, int y_type) {
+__device__ __forceinline__ void store_y4(void* Y, size_t idx, float4 v, int y_type, DeviceStatus* st, size_t extent) {
+  if (!LQER_IN_BOUNDS(st, idx * (y_type == kYBF16 ? 2 : 4), y_type == kYBF16 ? 8 : 16, extent, 701)) return;
   if (y_type == kYBF16)
     *reinterpret_cast<uint2*>(static_cast<uint16_t*>(Y) + idx) =
         make_uint2(bf16_rn(v.x) | (bf16_rn(v.y) << 16), bf16_rn(v.z) | (bf16_rn(v.w) << 16));
@@ -157,14 +162,14 @@ __device__ __forceinline__ void reduce_tile(const Params& p, const Layer& ly, in
         uint2 unused;
         int e;
         quantize_quad(v[u], p.a_bits, p.exp_min, p.exp_max, e, m8, unused);
-        if (tk < p.M && quad_ok) {
+        if (tk < p.M && quad_ok && LQER_IN_BOUNDS(p.status, (size_t)p.M * ly.N + ((size_t)tk * ly.N + col0 + c4) / 16, 1, ly.y_extent, 702)) {
           uint8_t* yq = static_cast<uint8_t*>(ly.Y);
           const size_t idx = (size_t)tk * ly.N + col0 + c4;
           *reinterpret_cast<uint32_t*>(yq + idx) = m8;
           if ((c4 & 15) == 0) yq[(size_t)p.M * ly.N + idx / 16] = (uint8_t)(e + 127);
         }
       } else if (tk < p.M && quad_ok) {
-        store_y4(ly.Y, (size_t)tk * ly.N + col0 + c4, v[u], p.y_type);
+        store_y4(ly.Y, (size_t)tk * ly.N + col0 + c4, v[u], p.y_type, p.status, ly.y_extent);
       }
     }
   }
@@ -259,6 +264,7 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
           int xcol;
           const uint32_t x_bytes = waited ? (uint32_t)p.x_rows * 128u : 0u;
           if (s < ly.k_slabs) {
+            if (!LQER_IN_BOUNDS(p.status, ((size_t)(nt0 + n_half - 1) * ly.k_slabs + s) * w_tile, w_tile, ly.w_extent, 705)) { ok = false; break; }
             mbar_expect_tx(w_full(pk), n_half * w_tile + x_bytes);
             for (int h = 0; h < n_half; ++h)
               bulk_load(dst + h * kWTileBytes, ly.wsec + ((size_t)(nt0 + h) * ly.k_slabs + s) * w_tile, w_tile, w_full(pk));
@@ -266,6 +272,8 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
           } else {
             const int rs = s - ly.k_slabs;
             const int rb0 = rs * 2, nb = min(2, ly.r_blocks - rb0);
+            if (!LQER_IN_BOUNDS(p.status, (size_t)(nt0 + n_half - 1) * b_tile_stride + (size_t)ly.r_blocks * kTileN * 16 + rb0 * kTileN,
+                                nb * kTileN, ly.b_extent, 706)) { ok = false; break; }
             mbar_expect_tx(w_full(pk), n_half * nb * (kTileN * 17) + x_bytes);
             for (int h = 0; h < n_half; ++h) {
               const uint8_t* tile = ly.bsec + (size_t)(nt0 + h) * b_tile_stride;
@@ -366,16 +374,21 @@ gemm_small_kernel(const __grid_constant__ TensorMaps tmaps, const __grid_constan
                   int e;
                   quantize_block16(v, qc, e, m8, b0, b1);
                   const size_t idx = (size_t)token * ly.N + col0 + c0 + 16 * j;
-                  *reinterpret_cast<uint4*>(yq + idx) = m8;
-                  yq[(size_t)p.M * ly.N + idx / 16] = (uint8_t)(e + 127);
+                  if (LQER_IN_BOUNDS(p.status, (size_t)p.M * ly.N + idx / 16, 1, ly.y_extent, 703)) {
+                    *reinterpret_cast<uint4*>(yq + idx) = m8;
+                    yq[(size_t)p.M * ly.N + idx / 16] = (uint8_t)(e + 127);
+                  }
                 }
             } else {
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 const float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
                                              __uint_as_float(r[4 * j + 3]));
-                if (!direct) *reinterpret_cast<float4*>(prow + c0 + 4 * j) = v;
-                else if (col0 + c0 + 4 * j < ly.N) store_y4(ly.Y, (size_t)token * ly.N + col0 + c0 + 4 * j, v, p.y_type);   // N is a multiple of 8
+                if (!direct) {
+                  if (LQER_IN_BOUNDS(p.status, (size_t)(prow + c0 + 4 * j - ly.partials) * 4, 16, ly.partial_extent, 704))
+                    *reinterpret_cast<float4*>(prow + c0 + 4 * j) = v;
+                }
+                else if (col0 + c0 + 4 * j < ly.N) store_y4(ly.Y, (size_t)token * ly.N + col0 + c0 + 4 * j, v, p.y_type, p.status, ly.y_extent);   // N is a multiple of 8
               }
             }
           }
@@ -554,6 +567,9 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_
     ly.wsec = base + m.off_w;
     ly.bsec = base + m.off_b;
     ly.Y = src.Y;
+    ly.y_extent = y_bytes(y_type, (size_t)M, (size_t)m.N);
+    if (kDebugBounds) ly.y_extent -= std::min(ly.y_extent, debug_y_shrink());
+    ly.w_extent = m.off_b - m.off_w; ly.b_extent = m.off_a - m.off_b;
     ly.partials = src.partials;
     ly.counters = src.counters;
     ly.N = m.N; ly.K64 = m.K64;
@@ -563,6 +579,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_
     if (n > 1 && group_chunks < want) want = group_chunks;
     ly.chunk_stages = (m.k_slabs + want - 1) / want;
     ly.chunks = (m.k_slabs + ly.chunk_stages - 1) / ly.chunk_stages;
+    ly.partial_extent = ly.chunks > 1 ? (size_t)small_gemm_col_tiles(m) * ly.chunks * M * 256 * 4 : 0;
     ly.item_begin = item_begin;
     if (i < n) item_begin += small_gemm_col_tiles(m) * ly.chunks;
   }

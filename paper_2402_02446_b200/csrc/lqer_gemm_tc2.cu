@@ -24,6 +24,8 @@
 // A launch may serve several layers with one M: their tiles form one list (layers with more K
 // stages per tile first) that the pairs walk round robin, so pairs idle only at the end of the
 // list and set-up and the last epilogue are paid once per launch.
+#include <algorithm>
+
 #include "lqer_tc_ptx.cuh"
 
 namespace lqer {
@@ -62,6 +64,8 @@ struct Layer {
   const uint8_t* wsec;
   const uint8_t* bsec;
   void* Y;                     // [M, N] fp32; bf16 or the MXINT8 sections by Params::y_type (never for the K ranges of a split layer)
+  size_t y_extent;             // bytes of the buffer behind Y, for the checked build
+  size_t w_extent, b_extent;   // bytes of the packed W and B sections
   int N, K64;
   int n_tiles, k_slabs, r_blocks;
   int slab0, slab_stride;      // a layer may be a K range of a real layer (split K): its first weight slab, and the
@@ -169,13 +173,16 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           if (!mbar_wait<true>(freed(st), ph ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = smem_u32(stage_base + st * STAGE_BYTES);
           if (s < k_slabs) {
+            const size_t w_off = ((size_t)my_ntile * slab_stride + slab0 + s) * w_tile;
+            if (has_w && !LQER_IN_BOUNDS(p.status, w_off, w_tile, p.L[layer].w_extent, 605)) { ok = false; break; }
             mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? w_tile : 0));
             tma_load_2d(a_dst, tmap_x, (slab0 + s) * BK, row0, loaded(st));
-            if (has_w)
-              bulk_load(a_dst + PK_OFFSET, wsec + ((size_t)my_ntile * slab_stride + slab0 + s) * w_tile, w_tile, loaded(st));
+            if (has_w) bulk_load(a_dst + PK_OFFSET, wsec + w_off, w_tile, loaded(st));
           } else {
             const int rs = s - k_slabs;
             const int rb0 = rs * 2, nb = min(2, r_blocks - rb0);
+            if (has_w && !LQER_IN_BOUNDS(p.status, (size_t)my_ntile * b_tile_stride + (size_t)r_blocks * kTileN * 16 + rb0 * kTileN,
+                                         nb * kTileN, p.L[layer].b_extent, 606)) { ok = false; break; }
             mbar_expect_tx(loaded(st), A_TILE_BYTES + (has_w ? nb * (kTileN * 17) : 0));
             tma_load_2d(a_dst, tmap_x, K64 + rs * RANK_PER_STAGE, row0, loaded(st));
             if (has_w) {
@@ -265,14 +272,15 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           if (p.y_type == kYBF16) {
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-              if (c + 8 * j < ncols)                      // N is a multiple of 8
+              if (c + 8 * j < ncols && LQER_IN_BOUNDS(p.status, (yoff + c + 8 * j) * 2, 16, p.L[layer].y_extent, 601))   // N is a multiple of 8
                 *reinterpret_cast<uint4*>(yrow16 + c + 8 * j) =
                     make_uint4(bf16x2_rn(r[8 * j], r[8 * j + 1]), bf16x2_rn(r[8 * j + 2], r[8 * j + 3]),
                                bf16x2_rn(r[8 * j + 4], r[8 * j + 5]), bf16x2_rn(r[8 * j + 6], r[8 * j + 7]));
           } else if (p.y_type == kYMXINT8) {
 #pragma unroll
             for (int j = 0; j < 2; ++j)
-              if (c + 16 * j < ncols) {                   // N is a multiple of 16 here
+              if (c + 16 * j < ncols && LQER_IN_BOUNDS(p.status, yoff + c + 16 * j, 16, p.L[layer].y_extent, 602) &&
+                  LQER_IN_BOUNDS(p.status, (size_t)p.M * Nl + yoff / 16 + (c >> 4) + j, 1, p.L[layer].y_extent, 603)) {   // N is a multiple of 16 here
                 float v[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[16 * j + i]);
@@ -285,7 +293,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
           } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              if (c + 4 * j < ncols)
+              if (c + 4 * j < ncols && LQER_IN_BOUNDS(p.status, (yoff + c + 4 * j) * 4, 16, p.L[layer].y_extent, 604))
                 *reinterpret_cast<uint4*>(yrow + c + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
           }
         }
@@ -467,6 +475,8 @@ cudaError_t launch_gemm_tc2_splitk(const void* xcat, int M, const PackedMeta& m,
     ly.wsec = base + m.off_w;
     ly.bsec = base + m.off_b;
     ly.Y = c == 0 ? Y : partials + (size_t)(c - 1) * M * m.N;
+    ly.y_extent = (size_t)M * m.N * 4;
+    ly.w_extent = m.off_b - m.off_w; ly.b_extent = m.off_a - m.off_b;
     ly.N = m.N; ly.K64 = m.K64;
     ly.n_tiles = m.n_tiles; ly.k_slabs = hi - lo;
     ly.r_blocks = c == C - 1 ? m.r_blocks : 0;
@@ -536,6 +546,9 @@ cudaError_t launch_gemm_tc2_group(const void* const* xcats, const void* const* p
     ly.wsec = base + m.off_w;
     ly.bsec = base + m.off_b;
     ly.Y = Ys[g];
+    ly.y_extent = y_bytes(y_type, (size_t)M, (size_t)m.N);
+    if (kDebugBounds) ly.y_extent -= std::min(ly.y_extent, debug_y_shrink());
+    ly.w_extent = m.off_b - m.off_w; ly.b_extent = m.off_a - m.off_b;
     ly.N = m.N; ly.K64 = m.K64;
     ly.n_tiles = m.n_tiles; ly.k_slabs = m.k_slabs; ly.r_blocks = m.r_blocks;
     ly.slab0 = 0; ly.slab_stride = m.k_slabs;

@@ -77,8 +77,10 @@ template <int PB, int TPW>
 __global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(const void* __restrict__ X, int x_bf16, int M, PackedMeta m,
                                                                const uint8_t* __restrict__ asec,
                                                                uint16_t* __restrict__ xcat,
-                                                               int8_t* __restrict__ Tm, uint8_t* __restrict__ Te) {
+                                                               int8_t* __restrict__ Tm, uint8_t* __restrict__ Te,
+                                                               DeviceStatus* status) {
   constexpr int SW = PB * 16;                     // columns per step
+  const size_t xcat_extent = (size_t)M * ((size_t)m.K64 + m.k_pad) * 2;   // bytes behind xcat, for the checked build
   constexpr int F4 = kRows * SW / 4 / kThreads;   // float4 per thread per step (PB / 4)
   __shared__ __align__(16) uint8_t s_xq[kRows * kXqStride];
   __shared__ int8_t s_xe[kRows][32];
@@ -155,7 +157,8 @@ __global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(co
       quantize_quad(xr[i], m.a_bits, m.exp_min, m.exp_max, e, m8, bf);
       *reinterpret_cast<uint32_t*>(&s_xq[r * kXqStride + c4 * 4]) = m8;
       if ((c4 & 3) == 0) s_xe[r][c4 >> 2] = (int8_t)e;
-      if (row < M && col < m.K64) *reinterpret_cast<uint2*>(xcat + (size_t)row * ldx + col) = bf;
+      if (row < M && col < m.K64 && LQER_IN_BOUNDS(status, ((size_t)row * ldx + col) * 2, 8, xcat_extent, 321))
+        *reinterpret_cast<uint2*>(xcat + (size_t)row * ldx + col) = bf;
     }
     // ---- next step's loads fly while this step's MMAs run
     if (s + CS < steps) {
@@ -235,7 +238,7 @@ __global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(co
     const int e = block_exponent(amax, m.exp_min, m.exp_max);
     const int q = quant_mantissa(t, e, m.a_bits);
     const int row = row0 + r;
-    if (row < M) {
+    if (row < M && LQER_IN_BOUNDS(status, ((size_t)row * ldx + m.K64 + j) * 2, 2, xcat_extent, 322)) {
       xcat[(size_t)row * ldx + m.K64 + j] = (uint16_t)bf16_bits_of(q, e - (m.a_bits - 2));
       if (Tm != nullptr) Tm[(size_t)row * m.k_pad + j] = (int8_t)q;
       if (Te != nullptr && (j & 15) == 0) Te[(size_t)row * (m.k_pad / 16) + (j >> 4)] = (uint8_t)(e + 127);
@@ -257,7 +260,7 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
 
 template <int PB, int TPW>
 static cudaError_t launch_prologue_pb(const void* X, bool x_bf16, int M, const PackedMeta& m, const uint8_t* asec, uint16_t* xc,
-                                      int8_t* Tm, uint8_t* Te, cudaStream_t s) {
+                                      int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s) {
   const int groups = (M + kRows - 1) / kRows;
   const int steps = (m.K64 + PB * 16 - 1) / (PB * 16);
   int cs = 1;
@@ -273,17 +276,16 @@ static cudaError_t launch_prologue_pb(const void* X, bool x_bf16, int M, const P
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   LaunchScope scope(kFamPrologue, s);
-  return cudaLaunchKernelEx(&cfg, prologue_kernel<PB, TPW>, X, x_bf16 ? 1 : 0, M, m, asec, xc, Tm, Te);
+  return cudaLaunchKernelEx(&cfg, prologue_kernel<PB, TPW>, X, x_bf16 ? 1 : 0, M, m, asec, xc, Tm, Te, st);
 }
 
 cudaError_t launch_prologue(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s) {
-  (void)st;
   const uint8_t* asec = static_cast<const uint8_t*>(packed) + m.off_a;
   uint16_t* xc = static_cast<uint16_t*>(xcat);
-  if (m.k_pad <= 64) return launch_prologue_pb<16, 1>(X, x_bf16, M, m, asec, xc, Tm, Te, s);
-  if (m.k_pad <= 128) return launch_prologue_pb<8, 2>(X, x_bf16, M, m, asec, xc, Tm, Te, s);
-  return launch_prologue_pb<4, 4>(X, x_bf16, M, m, asec, xc, Tm, Te, s);
+  if (m.k_pad <= 64) return launch_prologue_pb<16, 1>(X, x_bf16, M, m, asec, xc, Tm, Te, st, s);
+  if (m.k_pad <= 128) return launch_prologue_pb<8, 2>(X, x_bf16, M, m, asec, xc, Tm, Te, st, s);
+  return launch_prologue_pb<4, 4>(X, x_bf16, M, m, asec, xc, Tm, Te, st, s);
 }
 
 }  // namespace lqer

@@ -32,6 +32,7 @@ struct Layer {
   int* counts;                // [row group] arrivals, zero between calls
   int8_t* Tm;                 // optional exports of T_q
   uint8_t* Te;
+  size_t xcat_extent, slots_extent;   // bytes behind xcat and slots, for the checked build
   int K, K64, k, k_pad;
   int ranges;                 // K ranges per row group
   int cta_begin;              // first CTA of this layer in the launch
@@ -41,6 +42,7 @@ struct Params {
   Layer L[kMaxLayers];
   int n;                      // layers in this launch
   int M;
+  DeviceStatus* status;
   int x_bf16;                 // X is bf16 (else fp32)
   int a_bits, lr_bits, exp_min, exp_max;
 };
@@ -134,7 +136,8 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
         if (live) {
           *reinterpret_cast<uint32_t*>(&s_xq[r * kXqStride + c4 * 4]) = m8;
           if ((c4 & 3) == 0) s_xe[r][c4 >> 2] = (int8_t)e;
-          if (row < M) *reinterpret_cast<uint2*>(ly.xcat + (size_t)row * ldx + col) = bf;
+          if (row < M && LQER_IN_BOUNDS(p.status, ((size_t)row * ldx + col) * 2, 8, ly.xcat_extent, 311))
+            *reinterpret_cast<uint2*>(ly.xcat + (size_t)row * ldx + col) = bf;
         }
       }
     }
@@ -188,6 +191,7 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
 
   // ---- this CTA's partial sums -> its slot: the warps that share a rank tile add up in warp order
   double* slot = ly.slots + ((size_t)rgroup * ly.ranges + range) * kRows * k_pad;
+  if (!LQER_IN_BOUNDS(p.status, (size_t)(slot - ly.slots) * 8, (size_t)kRows * k_pad * 8, ly.slots_extent, 312)) return;
   if (NT >= kWarps) {
     if (active) {
 #pragma unroll
@@ -239,7 +243,7 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
     const int e = block_exponent(amax, p.exp_min, p.exp_max);
     const int q = quant_mantissa(t, e, p.a_bits);
     const int row = row0 + r;
-    if (row < M) {
+    if (row < M && LQER_IN_BOUNDS(p.status, ((size_t)row * ldx + ly.K64 + j) * 2, 2, ly.xcat_extent, 313)) {
       ly.xcat[(size_t)row * ldx + ly.K64 + j] = (uint16_t)bf16_bits_of(q, e - (p.a_bits - 2));
       if (ly.Tm != nullptr) ly.Tm[(size_t)row * k_pad + j] = (int8_t)q;
       if (ly.Te != nullptr && (j & 15) == 0) ly.Te[(size_t)row * (k_pad / 16) + (j >> 4)] = (uint8_t)(e + 127);
@@ -252,7 +256,7 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
 
 int prologue_small_max_layers() { return psm::kMaxLayers; }
 
-cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, cudaStream_t s) {
+cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, DeviceStatus* st, cudaStream_t s) {
   using namespace psm;
   if (n < 1 || n > kMaxLayers || M < 1) return cudaErrorInvalidValue;
   Params p;
@@ -260,6 +264,7 @@ cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M
   p.M = M;
   p.x_bf16 = x_bf16 ? 1 : 0;
   const PackedMeta& m0 = *layers[0].meta;
+  p.status = st;
   p.a_bits = m0.a_bits; p.lr_bits = m0.lr_bits; p.exp_min = m0.exp_min; p.exp_max = m0.exp_max;
   const int rgroups = (M + kRows - 1) / kRows;
   int begin = 0, max_kpad = 0;
@@ -273,6 +278,8 @@ cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M
     ly.asec = static_cast<const uint8_t*>(src.packed) + m.off_a;
     ly.xcat = static_cast<uint16_t*>(src.xcat);
     ly.slots = src.slots;
+    ly.xcat_extent = (size_t)M * xcat_cols(m) * 2;
+    ly.slots_extent = prologue_small_slot_bytes(m, M);
     ly.counts = src.counts;
     ly.Tm = src.Tm; ly.Te = src.Te;
     ly.K = m.K; ly.K64 = m.K64; ly.k = m.k; ly.k_pad = m.k_pad;

@@ -83,6 +83,7 @@ struct Params {
   int order;                // ChainOrder: where the wait for the previous kernel sits
   int x_bf16;               // X is bf16 (a stage of the ring then holds 16 KB), else fp32
   size_t ldx;               // columns of Xcat
+  size_t xcat_extent, partials_extent;   // bytes behind xcat and partials, for the checked build
 };
 
 // Up to kMaxLayers independent layers with one M, one rank padding and one set of formats may share a launch: a
@@ -288,8 +289,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     }
     // partial sums of this CTA's K range -> global scratch
     double* dst = p.partials + ((size_t)bid * ROWS + row) * KP + h * CPW;
+    if (LQER_IN_BOUNDS(p.status, (size_t)(dst - p.partials) * 8, CPW * 8, p.partials_extent, 302)) {
 #pragma unroll
-    for (int i = 0; i < CPW; i += 2) *reinterpret_cast<double2*>(dst + i) = make_double2(acc[i], acc[i + 1]);
+      for (int i = 0; i < CPW; i += 2) *reinterpret_cast<double2*>(dst + i) = make_double2(acc[i], acc[i + 1]);
+    }
   } else if (warp < WORK_WARPS) {
     // ------------------------------------------------------------------ quantisers
     // A lane owns a whole 16-block of a row: lanes 0-7 of a warp take block 0 of eight consecutive rows, lanes 8-15
@@ -350,7 +353,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
         quantize_block16(v, qc, e, m8, bf0, bf1);
         *reinterpret_cast<uint4*>(xdst + i * (8 * QW) * 128) = m8;
         xe_dst[i * (8 * QW) * 4] = (int8_t)e;
-        if (store_ok && 8 * QW * i < rows_ok) {
+        if (store_ok && 8 * QW * i < rows_ok &&
+            LQER_IN_BOUNDS(p.status, (size_t)(cd + i * c_step - p.xcat) * 2, 32, p.xcat_extent, 301)) {
           uint4* g = reinterpret_cast<uint4*>(cd + i * c_step);
           g[0] = bf0;
           g[1] = bf1;
@@ -500,7 +504,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
       const int qv = quant_mantissa(t, e, p.a_bits);
       const int r = r_lo + o / KP, j = o % KP;
       const int row = row0 + r;
-      if (live && row < p.M) {
+      if (live && row < p.M && LQER_IN_BOUNDS(p.status, ((size_t)row * p.ldx + p.K64 + j) * 2, 2, p.xcat_extent, 303)) {
         p.xcat[(size_t)row * p.ldx + p.K64 + j] = (uint16_t)bf16_bits_of(qv, e - (p.a_bits - 2));
         if (p.Tm != nullptr) p.Tm[(size_t)row * KP + j] = (int8_t)qv;
         if (p.Te != nullptr && (j & 15) == 0) p.Te[(size_t)row * (KP / 16) + (j >> 4)] = (uint8_t)(e + 127);
@@ -643,6 +647,8 @@ cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, 
     p.order = order;
     p.x_bf16 = x_bf16 ? 1 : 0;
     p.ldx = xcat_cols(m);
+    p.xcat_extent = (size_t)M * xcat_cols(m) * 2;
+    p.partials_extent = (size_t)((M + ROWS - 1) / ROWS) * splits[g] * ROWS * m.k_pad * 8;
     gp.cta_begin[i] = begin;
     if (i < n) begin += ((M + ROWS - 1) / ROWS) * p.splits;
   }
