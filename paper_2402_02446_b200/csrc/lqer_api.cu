@@ -69,13 +69,6 @@ int sm_count() {
   return count_of[dev];
 }
 
-// Two packed buffers with the same sections, formats and sizes (their contents may differ).
-static bool same_shape(const PackedMeta& a, const PackedMeta& b) {
-  return a.K == b.K && a.N == b.N && a.k == b.k && a.k_pad == b.k_pad && a.w_bits == b.w_bits && a.a_bits == b.a_bits &&
-         a.lr_bits == b.lr_bits && a.exp_min == b.exp_min && a.exp_max == b.exp_max && a.off_w == b.off_w &&
-         a.off_b == b.off_b && a.off_a == b.off_a;
-}
-
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -284,17 +277,6 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
 // Scratch one layer of a grouped prefill launch needs: its own Xcat and its own prologue partial sums.
 static size_t group_slice_bytes(const PackedMeta& m, int M) {
   return xcat_bytes(m, M) + align_up(prologue_tc_scratch_bytes(m, M), 256);
-}
-// Consecutive calls from `first` on that may share launches with it (auto path only): same M, same shape,
-// at most `limit` of them.
-static int same_shape_run(const lqer_call_t* calls, int first, int n_calls, const PackedMeta& m0, int limit) {
-  int n = 1;
-  while (first + n < n_calls && n < limit) {
-    PackedMeta m1;
-    if (calls[first + n].M != calls[first].M || lookup(calls[first + n].packed, m1) != LQER_OK || !same_shape(m0, m1)) break;
-    ++n;
-  }
-  return n;
 }
 // Consecutive prefill calls from `first` on that may share a GEMM launch with it (auto path only): the same M > 256,
 // the same formats, any shapes; at most `limit`, and only as many as the workspace has slices for.

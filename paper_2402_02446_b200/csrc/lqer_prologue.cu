@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(co
                                                                int8_t* __restrict__ Tm, uint8_t* __restrict__ Te,
                                                                DeviceStatus* status) {
   constexpr int SW = PB * 16;                     // columns per step
-  const size_t xcat_extent = (size_t)M * ((size_t)m.K64 + m.k_pad) * 2;   // bytes behind xcat, for the checked build
+  [[maybe_unused]] const size_t xcat_extent = (size_t)M * ((size_t)m.K64 + m.k_pad) * 2;   // bytes behind xcat, for the checked build
   constexpr int F4 = kRows * SW / 4 / kThreads;   // float4 per thread per step (PB / 4)
   __shared__ __align__(16) uint8_t s_xq[kRows * kXqStride];
   __shared__ int8_t s_xe[kRows][32];

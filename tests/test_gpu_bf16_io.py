@@ -97,7 +97,7 @@ def test_linear_batched_ex_shares_launches_like_fp32():
     for x, (sp, Pg, M), y in zip(Xs, plan, Ys):
         if M > 128:        # large batches: the same tiles, the same arithmetic
             assert torch.equal(L.linear_ex(x, Pg, ws, out_dtype=torch.bfloat16), y), sp.name
-        else:              # small batches that share a launch are cut into fewer K chunks: the oracle is the judge
+        else:              # small batches that share a launch are cut into fewer K chunks: both are compared with the oracle
             assert _check(y, olqer.forward(x.to(torch.float32).cpu().numpy(), Ps), True) <= 1.0
     ref = olqer.forward(Xs[0].to(torch.float32).cpu().numpy(), Pb)
     assert _check(Ys[0], ref, True) <= 1.0
