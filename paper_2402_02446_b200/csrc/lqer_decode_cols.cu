@@ -78,6 +78,7 @@ struct Params {
   int M;
   int a_bits, lr_bits, exp_min, exp_max;
   int x_bf16, y_bf16;           // element types of X and Y (else fp32)
+  int w_bits;                   // mantissa bits of W_q: 4 (nibbles) or 2 (crumbs), one value for all layers of a launch
   long long wait_limit;         // bound of the wait for the other CTAs' partial sums, in clock cycles
 };
 
@@ -110,11 +111,11 @@ __host__ __device__ inline int t_subsets(int k_pad) {
   return tiles < kWarps ? kWarps / tiles : 1;
 }
 
-struct Formats { int a_bits, lr_bits, exp_min, exp_max, x_bf16; };
+struct Formats { int a_bits, lr_bits, exp_min, exp_max, x_bf16, w_bits; };
 
 // X -> MXINT8 for the whole contraction, by all threads of the CTA: per row the mantissas in the byte order the nibbles
 // unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales 2^(e_x - 6) and the dp4a seeds (bits of
-// 1.5 * 2^23, minus 8 * sum(x) of the block).
+// 1.5 * 2^23, minus sum(x) of the block times the offset of the stored weights: 8 for nibbles, 1 for crumbs).
 __device__ __forceinline__ void quantize_x_rows(const void* X, int M, int K, int K64, const Formats& f, uint8_t* xm,
                                                 float* xsc, int* xof) {
   const int tid = threadIdx.x, KB = K64 / 16;
@@ -156,7 +157,7 @@ __device__ __forceinline__ void quantize_x_rows(const void* X, int M, int K, int
         *reinterpret_cast<uint32_t*>(xm + (size_t)row * K64 + c4 * 4) = perm;
         if ((c4 & 3) == 0) {
           xsc[row * KB + (c4 >> 2)] = pow2f(e - (f.a_bits - 2));
-          xof[row * KB + (c4 >> 2)] = kIntMagicBits - 8 * sum;
+          xof[row * KB + (c4 >> 2)] = kIntMagicBits - (f.w_bits == 2 ? 1 : 8) * sum;
         }
       }
     }
@@ -288,7 +289,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_pre_kernel(const __grid_co
 }
 
 // MT: rows the accumulators are compiled for (1 for the single-token call, kMaxM otherwise); M <= MT.
-template <int MT>
+// WB: mantissa bits of W_q the kernel is compiled for: 4 (nibbles) or 2 (crumbs).
+template <int MT, int WB>
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -323,20 +325,22 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   // CTA's range are clamped to its last one and slabs past K to the last slab: such loads stay inside the section
   // and what they return is never used (the sums of those slabs are skipped, those columns are not stored).
   const uint32_t lane_w = (uint32_t)((lane & 7) * 16);
-  const uint32_t lane_e = (uint32_t)(kWTileNibbleBytes + (lane & 7) * 4);
+  constexpr uint32_t w_tile = (uint32_t)(kTileN * kSlabK * WB / 8 + kTileN * 4);   // 4608 bytes with nibbles, 2560 with crumbs
+  constexpr bool crumbs = WB == 2;                                  // then a column of a slab is one 16-byte word group
+  const uint32_t lane_e = (uint32_t)(kTileN * kSlabK * WB / 8 + (lane & 7) * 4);
   struct ColOff { uint32_t w, e; };
   auto col_off = [&](int cg0) -> ColOff {
     const int cg = max(min(cg0 + (lane >> 3), cg_hi - 1), 0);
-    const uint32_t tile = (uint32_t)(cg >> 4) * (uint32_t)ly.k_slabs * (uint32_t)kWTileBytes;
+    const uint32_t tile = (uint32_t)(cg >> 4) * (uint32_t)ly.k_slabs * w_tile;
     ColOff o;
     o.w = tile + (uint32_t)(cg & 15) * 128u + lane_w;
     o.e = tile + (uint32_t)(cg & 15) * 32u + lane_e;
     return o;
   };
   auto fetch = [&](SlabRegs& d, const ColOff& o, int j) {
-    const uint32_t jo = (uint32_t)min(j, ly.k_slabs - 1) * (uint32_t)kWTileBytes;
+    const uint32_t jo = (uint32_t)min(j, ly.k_slabs - 1) * w_tile;
     d.h0 = ld_stream_u128(wsec + (o.w + jo));
-    d.h1 = ld_stream_u128(wsec + (o.w + jo + (uint32_t)(kTileN * 16)));
+    if (!crumbs) d.h1 = ld_stream_u128(wsec + (o.w + jo + (uint32_t)(kTileN * 16)));
     d.e = ld_stream_u32(wsec + (o.e + jo));
   };
 
@@ -393,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 
   // ---- X -> MXINT8 for the whole contraction: per row the mantissas in the byte order the nibbles
   //      unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales and the offsets 8 * sum(x)
-  const Formats fmt = {p.a_bits, p.lr_bits, p.exp_min, p.exp_max, p.x_bf16};
+  const Formats fmt = {p.a_bits, p.lr_bits, p.exp_min, p.exp_max, p.x_bf16, WB};
   if (pre) {                                       // quantised X and T_q are there already: straight into shared memory
     const int xb = (int)pre_x_bytes(M, ly.K64), tb = (int)pre_t_bytes(ly.k_pad);
     for (int o = tid * 16; o < xb; o += kThreads * 16)
@@ -509,17 +513,31 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
         const int j = warp + kWarps * (js + s);
         if (j < ly.k_slabs) {
           const SlabRegs d = regs[s];
-          // nibbles as bytes: k {0,4,1,5}, {2,6,3,7}, {8,12,9,13}, {10,14,11,15} of each block
-          const uint32_t wd[8] = {d.h0.x, d.h0.y, d.h0.z, d.h0.w, d.h1.x, d.h1.y, d.h1.z, d.h1.w};
+          // weights as bytes in the order k {0,4,1,5}, {2,6,3,7}, {8,12,9,13}, {10,14,11,15} of each block
           uint32_t nib[16];
+          if (crumbs) {
+            // a word per block: (w >> 2i) & 0x03030303 holds k {2i, 2i + 8, 2i + 1, 2i + 9}; two byte permutes per pair
+            const uint32_t wd[4] = {d.h0.x, d.h0.y, d.h0.z, d.h0.w};
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            nib[2 * i] = wd[i] & 0x0F0F0F0Fu;
-            nib[2 * i + 1] = (wd[i] >> 4) & 0x0F0F0F0Fu;
+            for (int b = 0; b < 4; ++b) {
+              const uint32_t c0 = wd[b] & 0x03030303u, c1 = (wd[b] >> 2) & 0x03030303u;
+              const uint32_t c2 = (wd[b] >> 4) & 0x03030303u, c3 = (wd[b] >> 6) & 0x03030303u;
+              nib[4 * b] = __byte_perm(c0, c2, 0x6240);
+              nib[4 * b + 1] = __byte_perm(c1, c3, 0x6240);
+              nib[4 * b + 2] = __byte_perm(c0, c2, 0x7351);
+              nib[4 * b + 3] = __byte_perm(c1, c3, 0x7351);
+            }
+          } else {
+            const uint32_t wd[8] = {d.h0.x, d.h0.y, d.h0.z, d.h0.w, d.h1.x, d.h1.y, d.h1.z, d.h1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              nib[2 * i] = wd[i] & 0x0F0F0F0Fu;
+              nib[2 * i + 1] = (wd[i] >> 4) & 0x0F0F0F0Fu;
+            }
           }
-          float sw[4];                                               // 2^(e_w - 2) of the four blocks
+          float sw[4];                                               // 2^(e_w - (w_bits - 2)) of the four blocks
 #pragma unroll
-          for (int b = 0; b < 4; ++b) sw[b] = __uint_as_float((((d.e >> (8 * b)) & 0xFFu) - 2u) << 23);
+          for (int b = 0; b < 4; ++b) sw[b] = __uint_as_float((((d.e >> (8 * b)) & 0xFFu) - (uint32_t)(WB - 2)) << 23);
 #pragma unroll
           for (int r = 0; r < MT; ++r) {
             if (r < M) {
@@ -640,9 +658,9 @@ static size_t cols_smem_bytes(const PackedMeta& m, int M) {
   return (size_t)M * m.K64 + (size_t)M * (m.K64 / 16) * 8 + 2 * kHoldMax * kWarps * kCg * 8 * kMaxM * 4 +
          (size_t)kMaxM * m.k_pad * 8 * t_subsets(m.k_pad) + kMaxM * 16 * 4 + (size_t)kMaxM * (m.k_pad > 0 ? m.k_pad : 16) + 256;
 }
-// The column-owner kernel serves M <= 4 (4-bit weights: its dot products run on raw nibbles) as long as the quantised X of
+// The column-owner kernel serves M <= 4 (its dot products run on the raw nibbles or crumbs) as long as the quantised X of
 // the whole contraction fits in shared memory.
-bool decode_cols_fits(const PackedMeta& m, int M) { return m.w_bits == 4 && M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
+bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
 
 cudaError_t launch_decode_cols(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
                                void* workspace, cudaStream_t s) {
@@ -663,15 +681,16 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   static OncePerDevice once;
   static bool one_cta_per_sm = true;               // false if any device could hold two CTAs of the kernel on one SM
   cudaError_t e0 = once.run([] {
-    cudaError_t e = cudaFuncSetAttribute(decode_cols_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(decode_cols_kernel<kMaxM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
     // chaining launches relies on one CTA per SM (registers): a launch on every SM then leaves room for no other
-    int o1 = 2, o4 = 2;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o1, decode_cols_kernel<1>, kThreads, 0) != cudaSuccess) o1 = 2;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o4, decode_cols_kernel<kMaxM>, kThreads, 0) != cudaSuccess) o4 = 2;
-    if (!(o1 == 1 && o4 == 1)) one_cta_per_sm = false;
+    const void* kernels[4] = {reinterpret_cast<const void*>(decode_cols_kernel<1, 4>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 4>),
+                              reinterpret_cast<const void*>(decode_cols_kernel<1, 2>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 2>)};
+    for (const void* k : kernels) {
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return e;
+      int o = 2;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, k, kThreads, 0) != cudaSuccess) o = 2;
+      if (o != 1) one_cta_per_sm = false;
+    }
     return cudaSuccess;
   });
   if (e0 != cudaSuccess) return e0;
@@ -685,6 +704,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   p.M = M;
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
   p.x_bf16 = x_bf16 ? 1 : 0;
+  p.w_bits = metas[0].w_bits;
   p.y_bf16 = y_bf16 ? 1 : 0;
   p.wait_limit = wait_limit_cycles();
   const int stall = take_stall(kFamDecode) ? 1 : 0;
@@ -779,7 +799,9 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   cfg.numAttrs = 1;
   if (fills_gpu != nullptr) *fills_gpu = one_cta_per_sm && begin == sm_count;
   LaunchScope scope(kFamDecode, s);
-  return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM>, p);
+  if (p.w_bits == 2)
+    return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 2>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 2>, p);
+  return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 4>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 4>, p);
 }
 
 int decode_pre_max_calls() { return dcol::kPreMaxCalls; }
@@ -810,7 +832,7 @@ cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas,
     c.asec = static_cast<const uint8_t*>(calls[g].packed) + m.off_a;
     c.out = outs[g];
     c.M = calls[g].M; c.K = m.K; c.K64 = m.K64; c.k_pad = m.k_pad;
-    c.f = Formats{m.a_bits, m.lr_bits, m.exp_min, m.exp_max, x_bf16 ? 1 : 0};
+    c.f = Formats{m.a_bits, m.lr_bits, m.exp_min, m.exp_max, x_bf16 ? 1 : 0, m.w_bits};
     if (c.M < 1 || c.M > kMaxM) return cudaErrorInvalidValue;
     if (c.M > 1) single = false;
     const size_t need = pre_x_bytes(c.M, c.K64) + pre_t_bytes(c.k_pad) + 16 +

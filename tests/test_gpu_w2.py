@@ -113,3 +113,33 @@ def test_two_bit_full_size_sampled_rows(ratio_log):
         y1 = L.linear(_t(X[:M]), Pg, ws).cpu().numpy()
         assert worst_ratio(y1, r1) <= 1.0, M
     Pg.release()
+
+
+@pytest.mark.parametrize("M", [1, 3])
+def test_two_bit_batched_decode_shares_launches(M):
+    # the column-owner decode kernel on crumbs: a stretch of independent calls shares launches (activations quantised
+    # ahead by one kernel), and every result equals the single call's bit for bit and the oracle's within the tolerance
+    specs = [gen.LayerSpec("w2_dec_a", M=M, K=1024, N=640, k=40, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=411),
+             gen.LayerSpec("w2_dec_b", M=M, K=2112, N=264, k=72, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=412)]
+    layers = []
+    for s in specs:
+        W = gen.make_weight(s)
+        A, B = gen.make_random_factors(s)
+        layers.append((olqer.prepare_weights(W, A, B, w_bits=2), L.prepare_weights(_t(W), _t(A), _t(B), _cfg())))
+    order = [0, 1] * 10                                   # 20 calls: more than one launch of 16
+    Xs = [gen.make_activations(specs[i], M=M) + 0.125 * j for j, i in enumerate(order)]
+    Xd = [_t(X) for X in Xs]
+    Yb = [torch.full((M, specs[i].N), float("nan"), dtype=torch.float32, device=DEV) for i in order]
+    calls = L.make_calls([(x, layers[i][1], y) for x, i, y in zip(Xd, order, Yb)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    before = L.launch_count()
+    L.linear_batched(calls, ws)
+    torch.cuda.synchronize()
+    assert L.launch_count() - before == 3                 # activations ahead + two decode launches (16 + 4 layers)
+    assert L.poll_status(ws) == 0
+    for x, X, i, y in zip(Xd, Xs, order, Yb):
+        single = L.linear(x, layers[i][1], ws)
+        assert torch.equal(single, y)
+        assert worst_ratio(y.cpu().numpy(), olqer.forward(X, layers[i][0], w_bits=2)) <= 1.0
+    for _, Pg in layers:
+        Pg.release()
