@@ -77,6 +77,29 @@ def test_linear_ex_every_path(spec, x_bf16, y_bf16, ratio_log):
     Pg.release()
 
 
+@pytest.mark.parametrize("x_bf16", [True, False], ids=["bf16_x", "f32_x"])
+def test_tensor_core_prologue_on_ragged_shapes(x_bf16):
+    # the tensor-core prologue forced on shapes it does not meet by itself: K = 80 (the second 64-column stage is mostly
+    # outside X and its TMA boxes read zeros there), 37 and 300 rows (row tiles mostly outside X), ranks 5 and 40
+    for spec in (gen.LayerSpec("rag_a", M=37, K=80, N=136, k=5, calib_rows=32, outlier_frac=0, n_outliers=2, outlier_scale=20.0, seed=321),
+                 gen.LayerSpec("rag_b", M=300, K=1104, N=264, k=40, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=322)):
+        P, Pg = _layer(spec)
+        ws = L.new_workspace(spec.M, Pg)
+        Xf, Xb = _bf16_inputs(spec, spec.M)
+        ref = olqer.forward(Xf, P)
+        X = Xb if x_bf16 else _t(Xf)
+        L.set_path(binding.PATH_TENSOR_PROLOGUE)
+        try:
+            Y = L.linear_ex(X, Pg, ws, out_dtype=torch.float32)
+            Tm, Te = L.project_lowrank(_t(Xf), Pg, ws)
+        finally:
+            L.set_path(binding.PATH_AUTO)
+        assert L.poll_status(ws) == 0
+        assert np.array_equal(Tm.cpu().numpy(), ref.Tm) and np.array_equal(Te.cpu().numpy(), mxint.exponent_bytes(ref.Te))
+        assert _check(Y, ref, False) <= 1.0, spec.name
+        Pg.release()
+
+
 def test_linear_batched_ex_shares_launches_like_fp32():
     # four prefill calls (M = 1100: one prologue launch, one GEMM launch) and five small-batch calls (M = 9: two launches)
     # with bf16 in and out
