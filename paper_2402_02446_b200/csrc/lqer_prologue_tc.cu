@@ -8,12 +8,12 @@
 // in a fixed order.
 //   scalers      read the int32 block products from tensor memory, scale each by 2^(e_x + e_a)
 //                and sum in fp64 (exact for any realistic exponent spread)
-//   quantisers   take fp32 X from a shared-memory ring that TMA fills, write the exact bf16
-//                values m * 2^(e-6) to Xcat, the int8 mantissas to shared memory in the K-major
+//   quantisers   take X (fp32 or bf16) from a shared-memory ring that TMA fills, a whole 16-block per lane, write
+//                the exact bf16 values m * 2^(e-6) to Xcat, the int8 mantissas to shared memory in the K-major
 //                128-byte-swizzled layout the MMA reads, and the block exponents beside them
 //   panel warp   A_q panels: 16-byte asynchronous copies into a block-diagonal operand
 //   issuer warp  one lane issues tcgen05.mma kind::i8 (M=128, N=2*k_pad, K=32)
-//   TMA warp     one lane keeps the fp32 ring full (128 rows x 64 columns per stage)
+//   TMA warp     one lane keeps the ring of X full (128 rows x 64 columns per stage, in 128-byte-wide swizzled boxes)
 // Each 16-block needs its own integer product, because its scale differs from its neighbour's.
 // The int8 MMA contracts 32 values, so the B operand of a block pair is laid out as
 //     rows 0..k_pad-1:        [A_b | 0]        rows k_pad..2 k_pad-1:  [0 | A_{b+1}]
@@ -48,9 +48,13 @@ struct Cfg {
   static constexpr int SLOT_COLS = 2 * KP;                   // accumulator columns per block pair
   static constexpr int TMEM_SLOTS = (512 / SLOT_COLS) < MAX_TMEM_SLOTS ? (512 / SLOT_COLS) : MAX_TMEM_SLOTS;
   static constexpr int TMEM_COLS = 512;
-  // With 8 scaler and 16 quantiser warps (whole warpgroups each) the quantisers hand 8 registers per thread to the
-  // scalers: 8 x 88 + 16 x 64 + 3 x 72 registers per lane = the 27 x 72 the CTA was launched with.
-  static constexpr bool REG_SHIFT = SCALER_WARPS == 8;
+  // The quantisers hand registers to the scalers (whole warpgroups each; the CTA was launched with 27 x 72 per lane):
+  // 8 x 88 + 16 x 64 + 3 x 72 with 8 scaler warps (k_pad 16), 16 x 80 + 8 x 56 + 3 x 72 with 16 scaler warps of 16
+  // columns (k_pad 64).  At k_pad 32 (16 scaler warps of 8 columns) nobody is short of registers and the shift only
+  // slowed the quantisers.
+  static constexpr bool REG_SHIFT = CPW == 16 || SCALER_WARPS == 8;
+  static constexpr int SCALER_REGS = SCALER_WARPS == 8 ? 88 : 80;
+  static constexpr int QUANT_REGS = SCALER_WARPS == 8 ? 64 : 56;
   static constexpr int PANEL_BYTES = 2 * KP * 128;           // 2 k_pad rows x 128 bytes
   static constexpr int OFF_XQ = RAW_SLOTS * RAW_BYTES;
   static constexpr int OFF_PANEL = OFF_XQ + (X_SLOTS / 2) * XBUF_BYTES;
@@ -222,7 +226,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
 
   if (warp < SW) {
     // ------------------------------------------------------------------ scalers
-    if (C::REG_SHIFT) asm volatile("setmaxnreg.inc.sync.aligned.u32 88;" ::: "memory");   // registers the quantisers gave up
+    if (C::REG_SHIFT) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::SCALER_REGS) : "memory");   // registers the quantisers gave up
     const int q = warp & 3, h = warp >> 2;
     const int row = q * 32 + lane;
     double acc[CPW];
@@ -298,7 +302,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     // A lane owns a whole 16-block of a row: lanes 0-7 of a warp take block 0 of eight consecutive rows, lanes 8-15
     // block 1, and so on, so that every quarter warp reads and writes eight different 16-byte chunks of the swizzled
     // tiles (no bank conflicts) and the warp stores 8 rows x 128 contiguous bytes of Xcat.
-    if (C::REG_SHIFT) asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
+    if (C::REG_SHIFT) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::QUANT_REGS) : "memory");
     const int qwarp = warp - SW;
     const int blk = lane >> 3;                         // 16-block within the 64-column stage
     const int r0 = qwarp * 8 + (lane & 7);             // first row (then + 8 * QW per pass)
