@@ -331,9 +331,7 @@ gemm_tc2_kernel(const __grid_constant__ TensorMaps tmaps, const Params p) {
       if (tile >= num_tiles) break;
       const int st = it % STAGES;
       const uint32_t ph = (uint32_t)((it / STAGES) & 1);
-      // sleeping poll: a converter group has five stages' time to spare, and 24 warps that poll in a tight loop cost
-      // power the tensor cores could use (the step runs at the power cap)
-      if (!mbar_wait<true>(loaded(st), ph, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(loaded(st), ph, abort_flag)) { ok = false; break; }
       const uint8_t* pk = stage_base + st * STAGE_BYTES + PK_OFFSET;
       uint8_t* bt = stage_base + st * STAGE_BYTES + A_TILE_BYTES;
       if (s < k_slabs) {
