@@ -116,8 +116,8 @@ def test_missing_library_fails_loudly(monkeypatch):
 
 
 def test_workspace_bound_covers_every_smaller_batch():
-    # lqer_workspace_bytes(M_max) must fit the call with any M <= M_max, whichever path that call takes: decode
-    # kernels (M <= 16), split-K GEMM (M <= 256), the tensor-core prologue's partial sums (row tiles x K ranges,
+    # lqer_workspace_bytes(M_max) must fit the call with any M <= M_max, whichever path that call takes: the
+    # small-batch kernels (M <= 128), the split-K GEMM (M <= 256), the tensor-core prologue's partial sums (row tiles x K ranges,
     # which grows past one CTA per SM once there are more than 148 row tiles)
     Ms = [1, 4, 16, 17, 64, 127, 128, 129, 255, 256, 257, 300, 511, 512, 1023, 1024, 2048, 4096, 18944, 19072,
           32768, 65536]

@@ -279,7 +279,7 @@ def test_linear_tensor_core_kernel(spec, path):
     Pg.release()
 
 
-# ---------------------------------------------------------------------------- decode kernel (M <= 16)
+# ---------------------------------------------------------------------------- decode and small-batch kernels (M <= 128)
 DECODE_SPECS = SMALL_SPECS + MID_SPECS + [
     gen.LayerSpec("dec_many_tiles", M=16, K=64, N=2048, k=24, calib_rows=32, outlier_frac=0.0, n_outliers=1,
                   outlier_scale=20.0, seed=41),      # few units per column tile: CTAs span several tiles
@@ -492,7 +492,7 @@ def test_linear_decode_full_size(M, ratio_log):
     X = gen.make_activations(spec)
     ref = olqer.forward(X, P)
     ws = L.new_workspace(M, Pg)
-    Y = L.linear(_t(X), Pg, ws).cpu().numpy()          # automatic path selection: decode for M <= 16
+    Y = L.linear(_t(X), Pg, ws).cpu().numpy()          # automatic path selection: the column-owner kernel (M <= 4) or the small-batch kernels
     assert L.poll_status(ws) == 0
     assert ratio_log(spec.name, worst_ratio(Y, ref)) <= 1.0
     Pg.release()
