@@ -402,18 +402,26 @@ def run_ours(args) -> None:
     L.lib().lqer_workspace_init(ws.data_ptr(), ws_bytes, int(torch.cuda.current_stream().cuda_stream))
 
     # element types at the boundary: X fp32 or bf16; Y fp32, bf16, or re-quantised to MXINT8 (17 bytes per 16 elements)
-    x_t = torch.float32 if args.io == "f32" else torch.bfloat16
+    x_t = torch.float32 if args.io == "f32" else L.MXINT8 if args.io == "mxint8" else torch.bfloat16
     y_t = torch.float32 if args.io == "f32" else torch.bfloat16 if args.io == "bf16" else L.MXINT8
-    x_b = 4 if args.io == "f32" else 2
+    x_b = 4.0 if args.io == "f32" else 17.0 / 16.0 if args.io == "mxint8" else 2.0
     y_b = 4.0 if args.io == "f32" else 2.0 if args.io == "bf16" else 17.0 / 16.0
+
+    def as_x(Xf):
+        """An fp32 activation tensor in the element type of the run (MXINT8: quantised by the library's own routine)."""
+        if x_t == L.MXINT8:
+            Xm, Xe = L.quantize_activations(Xf if Xf.is_cuda else Xf.to(dev), cfg)
+            buf = L.to_mxint8(Xm, Xe)
+            return buf if Xf.is_cuda else buf.cpu()
+        return Xf.to(x_t)
 
     def new_y(M, N, device=dev):
         if y_t == L.MXINT8:
             return torch.empty(L.mxint8_bytes(M, N), dtype=torch.uint8, device=device)
         return torch.empty((M, N), dtype=y_t, device=device)
 
-    X1 = [gen.make_activations_device(s[3], dev, M=M_DECODE).to(x_t) for s in shapes]
-    X2 = [gen.make_activations_device(s[3], dev, M=M_PREFILL).to(x_t) for s in shapes]
+    X1 = [as_x(gen.make_activations_device(s[3], dev, M=M_DECODE)) for s in shapes]
+    X2 = [as_x(gen.make_activations_device(s[3], dev, M=M_PREFILL)) for s in shapes]
     # outputs: one buffer per linear type and M (write-only; each is larger than a tile's reuse window)
     Y1 = [new_y(M_DECODE, N) for _, N, _, _ in shapes]
     Y2_by_type = [new_y(M_PREFILL, gen.STACK_LINEARS[w][2]) for w in range(len(gen.STACK_LINEARS))]
@@ -533,8 +541,8 @@ def run_ours(args) -> None:
     e2e = None
     if not args.no_e2e:
         types = len(gen.STACK_LINEARS)
-        hx1 = [torch.randn((M_DECODE, gen.STACK_LINEARS[w][1])).to(x_t).pin_memory() for w in range(types)]
-        hx2 = [torch.randn((M_PREFILL, gen.STACK_LINEARS[w][1])).to(x_t).pin_memory() for w in range(types)]
+        hx1 = [as_x(torch.randn((M_DECODE, gen.STACK_LINEARS[w][1]))).pin_memory() for w in range(types)]
+        hx2 = [as_x(torch.randn((M_PREFILL, gen.STACK_LINEARS[w][1]))).pin_memory() for w in range(types)]
         hy1 = [new_y(M_DECODE, gen.STACK_LINEARS[w][2], "cpu").pin_memory() for w in range(types)]
         hy2 = [new_y(M_PREFILL, gen.STACK_LINEARS[w][2], "cpu").pin_memory() for w in range(types)]
         calls1 = L.make_host_calls([(hx1[j % types], packed[j], hy1[j % types]) for j in range(n_lin)], x_t, y_t)
@@ -558,7 +566,7 @@ def run_ours(args) -> None:
         barrier()
         e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
         (e_ms,) = max_over_ranks([e_ms], dist, dev)
-        h2d = sum(x_b * (M_DECODE + M_PREFILL) * K for K, _, _, _ in shapes)
+        h2d = int(sum(x_b * (M_DECODE + M_PREFILL) * K for K, _, _, _ in shapes))
         d2h = int(sum(y_b * (M_DECODE + M_PREFILL) * N for _, N, _, _ in shapes))
         e2e = {"value": world * (flops_decode + flops_prefill) / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                "ms_per_step": e_ms, "steps": e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -618,7 +626,7 @@ def run_ours(args) -> None:
             "vs_baseline": None, "dtype": "bf16 operands (exact MXINT values), fp32 accumulate", "data": "synthetic",
             "config": {"workload": (WORKLOAD if layers == 32 else WORKLOAD + f" [reduced to {layers} layers]") +
                                    ("" if args.a_bits == 8 else f" [activations MXINT{args.a_bits}]") +
-                                   ("" if args.w_bits == 4 else f" [weights MXINT{args.w_bits}]") + ("" if args.io == "f32" else " [bf16 X and Y]" if args.io == "bf16" else " [bf16 X, MXINT8 Y]") +
+                                   ("" if args.w_bits == 4 else f" [weights MXINT{args.w_bits}]") + ("" if args.io == "f32" else " [bf16 X and Y]" if args.io == "bf16" else " [bf16 X, MXINT8 Y]" if args.io == "bf16-mxint8" else " [MXINT8 X and Y]") +
                                    ("" if args.rank is None else f" [rank {args.rank}]"),
                        "linears": n_lin, "M_decode": M_DECODE, "M_prefill": M_PREFILL, "rank": 32 if args.rank is None else args.rank,
                        "a_bits": args.a_bits, "w_bits": args.w_bits, "io": args.io,
@@ -659,9 +667,10 @@ def main() -> None:
     ap.add_argument("--a-bits", type=int, default=8, help="mantissa bits of the activations: 8 (W4A8, the workload) or 6 (W4A6)")
     ap.add_argument("--w-bits", type=int, default=4, help="mantissa bits of the weights: 4 (the workload) or 2 (W2A8, Section 4.4)")
     ap.add_argument("--rank", type=int, default=None, help="rank of the correction of every linear (default 32, the workload)")
-    ap.add_argument("--io", choices=["f32", "bf16", "bf16-mxint8"], default="f32",
+    ap.add_argument("--io", choices=["f32", "bf16", "bf16-mxint8", "mxint8"], default="f32",
                     help="element types of X and Y at the layer's boundary: f32 (the workload), bf16 (16-bit activations, "
-                         "Section 2.1), or bf16 X with Y re-quantised to MXINT8 by the epilogue (w&a setting)")
+                         "Section 2.1), bf16 X with Y re-quantised to MXINT8 by the epilogue, or MXINT8 both ways (w&a setting: "
+                         "17 bytes per 16 activations)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the decode-layer, prefill-MLP and rank-sweep legs")
     ap.add_argument("--quick-configs", action="store_true", help="rank sweep at M = 1 and 512 only")

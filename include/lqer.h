@@ -68,7 +68,7 @@ typedef struct {
 typedef enum {
   LQER_F32 = 0,
   LQER_BF16 = 1,
-  LQER_MXINT8 = 2    /* output only: Y re-quantised to the layer's activation format, see lqer_linear_ex */
+  LQER_MXINT8 = 2    /* MXINT activations in the layer's format: int8 mantissas, then exponent bytes; see lqer_linear_ex */
 } lqer_dtype_t;
 
 /* One call of a batch (Section 4.3: layers are independent). */
@@ -190,7 +190,12 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * layer's activation format (a_bits and exponent window of its lqer_config_t), exactly as the next layer's
  * prologue would quantise the fp32 Y.  Y then points to M*N + M*N/16 bytes: the int8 mantissas [M,N] followed
  * directly by the exponent bytes [M,N/16] (e + 127); N must be a multiple of 16.  Calls of up to 4 rows take
- * the small-batch kernels for this output (the column-owner kernel's CTAs do not own whole blocks). */
+ * the small-batch kernels for this output (the column-owner kernel's CTAs do not own whole blocks).
+ * x_dtype LQER_MXINT8: X is given in the same layout - mantissas [M,K], then exponent bytes [M,K/16], M*K + M*K/16
+ * bytes - with the mantissa width and exponent window of the layer's lqer_config_t (what a previous layer's MXINT8
+ * output holds if it has the same format).  It is taken at its value: a block that a quantiser would have produced
+ * passes through unchanged, any other block is renormalised without changing its values, so the layer computes
+ * exactly what it computes on the fp32 tensor of those values - without reading 4 bytes per element. */
 lqer_status_t lqer_linear_ex(const void* X, lqer_dtype_t x_dtype, int M, const void* packed, void* Y, lqer_dtype_t y_dtype,
                              void* workspace, size_t workspace_bytes, void* stream);
 lqer_status_t lqer_linear_batched_ex(const lqer_call_t* calls, int n_calls, lqer_dtype_t x_dtype, lqer_dtype_t y_dtype,

@@ -286,18 +286,29 @@ def split_mxint8(Y: torch.Tensor, M: int, N: int):
 
 
 def linear_ex(X: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y: torch.Tensor | None = None,
-              out_dtype=torch.float32, stream=None):
-    """The layer with fp32 or bf16 activations in and fp32, bf16 or MXINT8 out (the input type is taken from X, the output
-    type from out_dtype; an MXINT8 Y is a flat uint8 buffer of mxint8_bytes(M, N), see split_mxint8)."""
-    M = X.shape[0]
+              out_dtype=torch.float32, stream=None, M: int | None = None):
+    """The layer with fp32, bf16 or MXINT8 activations in and fp32, bf16 or MXINT8 out.  The input type is taken from X
+    (a flat uint8 tensor is an MXINT8 X of M rows: give M), the output type from out_dtype; an MXINT8 Y is a flat uint8
+    buffer of mxint8_bytes(M, N), see split_mxint8."""
+    x_dtype = MXINT8 if X.dtype == torch.uint8 else X.dtype
+    if x_dtype == MXINT8:
+        if M is None or X.numel() != mxint8_bytes(M, P.K):
+            raise ValueError("an MXINT8 X is a flat uint8 tensor of mxint8_bytes(M, K); pass M")
+    else:
+        M = X.shape[0]
     if Y is None:
         Y = (torch.empty(mxint8_bytes(M, P.N), dtype=torch.uint8, device=X.device) if out_dtype == MXINT8
              else torch.empty((M, P.N), dtype=out_dtype, device=X.device))
     elif out_dtype != MXINT8:
         out_dtype = Y.dtype
-    _check(lib().lqer_linear_ex(_dev(X), _DTYPES[X.dtype], M, P.ptr, _dev(Y, _tensor_dtype(out_dtype)), _DTYPES[out_dtype],
+    _check(lib().lqer_linear_ex(_dev(X), _DTYPES[x_dtype], M, P.ptr, _dev(Y, _tensor_dtype(out_dtype)), _DTYPES[out_dtype],
                                 ws.data_ptr(), ws.numel(), _stream(stream)), "lqer_linear_ex")
     return Y
+
+
+def to_mxint8(Xm: torch.Tensor, Xe: torch.Tensor) -> torch.Tensor:
+    """The flat MXINT8 buffer of mantissas Xm int8 [M, K] and exponent bytes Xe uint8 [M, K / 16]."""
+    return torch.cat([Xm.contiguous().view(torch.uint8).flatten(), Xe.contiguous().flatten()])
 
 
 def linear_static(X: torch.Tensor, P: PackedWeights, Y: torch.Tensor | None = None, stream=None):
@@ -315,12 +326,22 @@ def linear_static(X: torch.Tensor, P: PackedWeights, Y: torch.Tensor | None = No
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
-def make_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype=torch.float32) -> "C.Array":
+def _rows(X: torch.Tensor, P: "PackedWeights", x_dtype) -> int:
+    """Rows of an activation tensor: its first dimension, or, for a flat MXINT8 buffer, what its size says."""
+    if x_dtype != MXINT8:
+        return X.shape[0]
+    M, rest = divmod(X.numel() * 16, 17 * P.K)
+    if rest:
+        raise ValueError("an MXINT8 X holds mxint8_bytes(M, K) bytes")
+    return M
+
+
+def make_calls(items, x_dtype=torch.float32, y_dtype=torch.float32) -> "C.Array":
     """items: iterable of (X, PackedWeights, Y) -> a host array of lqer_call_t."""
     items = list(items)
     arr = (Call * len(items))()
     for j, (X, P, Y) in enumerate(items):
-        arr[j] = Call(_dev(X, x_dtype), X.shape[0], P.ptr, _dev(Y, _tensor_dtype(y_dtype)))
+        arr[j] = Call(_dev(X, _tensor_dtype(x_dtype)), _rows(X, P, x_dtype), P.ptr, _dev(Y, _tensor_dtype(y_dtype)))
     return arr
 
 
@@ -338,7 +359,7 @@ def linear_batched(calls, ws: torch.Tensor, stream=None) -> None:
            "lqer_linear_batched")
 
 
-def linear_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype, stream=None) -> None:
+def linear_batched_ex(calls, ws: torch.Tensor, x_dtype, y_dtype, stream=None) -> None:
     """linear_batched with every X of x_dtype (fp32 or bf16) and every Y of y_dtype (fp32, bf16 or MXINT8); `calls` from
     make_calls(..., x_dtype, y_dtype)."""
     _check(lib().lqer_linear_batched_ex(calls, len(calls), _DTYPES[x_dtype], _DTYPES[y_dtype], ws.data_ptr(), ws.numel(),
@@ -354,15 +375,15 @@ def linear_host(X_host: torch.Tensor, P: PackedWeights, ws: torch.Tensor, Y_host
     return Y_host
 
 
-def make_host_calls(items, x_dtype: torch.dtype = torch.float32, y_dtype=torch.float32) -> "C.Array":
+def make_host_calls(items, x_dtype=torch.float32, y_dtype=torch.float32) -> "C.Array":
     """items: iterable of (X_cpu, PackedWeights, Y_cpu), contiguous CPU tensors of the given types -> a host array of lqer_call_t."""
     items = list(items)
     arr = (Call * len(items))()
     for j, (X, P, Y) in enumerate(items):
-        for t, dt in ((X, x_dtype), (Y, _tensor_dtype(y_dtype))):
+        for t, dt in ((X, _tensor_dtype(x_dtype)), (Y, _tensor_dtype(y_dtype))):
             if t.is_cuda or t.dtype != dt or not t.is_contiguous():
                 raise ValueError("expected contiguous CPU tensors of the stated types")
-        arr[j] = Call(X.data_ptr(), X.shape[0], P.ptr, Y.data_ptr())
+        arr[j] = Call(X.data_ptr(), _rows(X, P, x_dtype), P.ptr, Y.data_ptr())
     return arr
 
 
@@ -380,7 +401,7 @@ def linear_host_batched(calls, ws: torch.Tensor, stream=None) -> None:
            "lqer_linear_host_batched")
 
 
-def linear_host_batched_ex(calls, ws: torch.Tensor, x_dtype: torch.dtype, y_dtype, stream=None) -> None:
+def linear_host_batched_ex(calls, ws: torch.Tensor, x_dtype, y_dtype, stream=None) -> None:
     """linear_host_batched with host X of x_dtype and host Y of y_dtype; `calls` from make_host_calls(..., x_dtype, y_dtype)."""
     _check(lib().lqer_linear_host_batched_ex(calls, len(calls), _DTYPES[x_dtype], _DTYPES[y_dtype], ws.data_ptr(), ws.numel(),
                                              _stream(stream)), "lqer_linear_host_batched_ex")

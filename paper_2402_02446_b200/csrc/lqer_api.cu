@@ -196,7 +196,7 @@ static size_t workspace_total(const PackedMeta& m, int M_max) {
 
 // Element types of X and Y (Section 2.1: the layer sits between 16-bit activations in the w-only setting).
 struct IoTypes {
-  bool x_bf16 = false;
+  int x_type = kXF32;          // kXF32, kXBF16 or kXMXINT8
   int y_type = kYF32;          // kYF32, kYBF16 or kYMXINT8
   bool y_bf16() const { return y_type == kYBF16; }
 };
@@ -219,7 +219,7 @@ static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, 
                                n == 1 ? Tm : nullptr, n == 1 ? Te : nullptr};
     gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g]};
   }
-  cudaError_t err = launch_prologue_small(pl, n, M, io.x_bf16, dst, s);
+  cudaError_t err = launch_prologue_small(pl, n, M, io.x_type, dst, s);
   if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, dst, s);
   return err;
 }
@@ -250,7 +250,7 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   cudaError_t err;
   if (small) {
     if (path != 5 && !project_only && io.y_type != kYMXINT8 && decode_cols_fits(m, M)) {
-      err = launch_decode_cols(X, io.x_bf16, M, m, packed, Y, io.y_bf16(), workspace, s);
+      err = launch_decode_cols(X, io.x_type, M, m, packed, Y, io.y_bf16(), workspace, s);
     } else {
       const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
       uint8_t* slice = static_cast<uint8_t*>(xcat);
@@ -260,10 +260,10 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
     }
   } else {
     if (path == 1 && (M > 65535 || io.y_type != kYF32)) return LQER_ERR_SHAPE;   // the checking kernel writes fp32 only
-    err = tc_prologue ? launch_prologue_tc(X, io.x_bf16, M, m, packed, xcat, Tm, Te, dst,
+    err = tc_prologue ? launch_prologue_tc(X, io.x_type, M, m, packed, xcat, Tm, Te, dst,
                                            reinterpret_cast<double*>(static_cast<uint8_t*>(xcat) + xcat_bytes(m, M)),
                                            reinterpret_cast<int*>(wsb + pcount_offset(m)), kChainAlone, s)
-                      : launch_prologue(X, io.x_bf16, M, m, packed, xcat, Tm, Te, dst, s);
+                      : launch_prologue(X, io.x_type, M, m, packed, xcat, Tm, Te, dst, s);
     if (err == cudaSuccess && !project_only)
       err = (path == 1) ? launch_gemm_simt(xcat, M, m, packed, static_cast<float*>(Y), s)
                         : launch_gemm_tc2_splitk(xcat, M, m, packed, Y, io.y_type,
@@ -475,7 +475,7 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
       }
       if (cnt == 0) continue;
       const int order = planned == 1 ? kChainAlone : launches == 0 ? kChainFirst : kChainLater;
-      if (launch_prologue_tc_group(Xs, io.x_bf16, M, ms, pk, xc, parts, counts, sp, cnt, nullptr, nullptr, dst, order, s) != cudaSuccess)
+      if (launch_prologue_tc_group(Xs, io.x_type, M, ms, pk, xc, parts, counts, sp, cnt, nullptr, nullptr, dst, order, s) != cudaSuccess)
         return LQER_ERR_CUDA;
       ++launches;
     }
@@ -487,9 +487,9 @@ static lqer_status_t run_prefill_group(const lqer_call_t* calls, int n, const Pa
       int* counters = reinterpret_cast<int*>(wsb + count_base) + (own_counters ? (size_t)g * row_tiles * 2 : 0);
       const int order = !own_counters ? kChainAlone : g == 0 ? kChainFirst : kChainLater;
       cudaError_t err = prologue_tc_fits(m, M, X, false)
-                            ? launch_prologue_tc(X, io.x_bf16, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
+                            ? launch_prologue_tc(X, io.x_type, M, m, calls[g].packed, xcat, nullptr, nullptr, dst,
                                                  reinterpret_cast<double*>(xcat + xcat_bytes(m, M)), counters, order, s)
-                            : launch_prologue(X, io.x_bf16, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
+                            : launch_prologue(X, io.x_type, M, m, calls[g].packed, xcat, nullptr, nullptr, dst, s);
       if (err != cudaSuccess) return LQER_ERR_CUDA;
     }
   }
@@ -807,7 +807,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
             for (int q = 0; q < (int)pm.size(); q += step) {
               const int cnt = std::min(step, (int)pm.size() - q);
               if (launch_decode_pre(calls + i + q, pm.data() + q, outs.data() + q, cnt, q == 0 ? kChainFirst : kChainLater,
-                                    io.x_bf16, cs) != cudaSuccess)
+                                    io.x_type, cs) != cudaSuccess)
                 return LQER_ERR_CUDA;
             }
           }
@@ -819,7 +819,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
         const int set = chain_open ? 1 - chain_set : 0;
         bool fills = false;
         if (launch_decode_cols_group(calls + i, metas, n, workspace, workspace_bytes, chain_open ? kChainLater : kChainFirst,
-                                     set, &fills, ahead ? pres : nullptr, io.x_bf16, io.y_bf16(), cs) != cudaSuccess)
+                                     set, &fills, ahead ? pres : nullptr, io.x_type, io.y_bf16(), cs) != cudaSuccess)
           return LQER_ERR_CUDA;
         chain_open = fills;
         chain_set = set;
@@ -842,9 +842,10 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
 }
 
 static lqer_status_t io_types(lqer_dtype_t x_dtype, lqer_dtype_t y_dtype, IoTypes* io) {
-  if ((x_dtype != LQER_F32 && x_dtype != LQER_BF16) || (y_dtype != LQER_F32 && y_dtype != LQER_BF16 && y_dtype != LQER_MXINT8))
+  if ((x_dtype != LQER_F32 && x_dtype != LQER_BF16 && x_dtype != LQER_MXINT8) ||
+      (y_dtype != LQER_F32 && y_dtype != LQER_BF16 && y_dtype != LQER_MXINT8))
     return LQER_ERR_CONFIG;
-  io->x_bf16 = x_dtype == LQER_BF16;
+  io->x_type = x_dtype == LQER_BF16 ? kXBF16 : x_dtype == LQER_MXINT8 ? kXMXINT8 : kXF32;
   io->y_type = y_dtype == LQER_BF16 ? kYBF16 : y_dtype == LQER_MXINT8 ? kYMXINT8 : kYF32;
   return LQER_OK;
 }
@@ -992,7 +993,6 @@ lqer_status_t lqer_linear_host_batched_bytes(const lqer_call_t* calls, int n_cal
 
 static lqer_status_t linear_host_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
                                          void* stream, IoTypes io) {
-  const size_t xe = io.x_bf16 ? 2 : 4;   // bytes per element of X on the host side and in the staging buffers
   if (calls == nullptr || workspace == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LQER_ERR_ALIGN;
@@ -1029,7 +1029,7 @@ static lqer_status_t linear_host_batched(const lqer_call_t* calls, int n_calls, 
     lookup(c.packed, m);
     // copy in: the buffer is free once the layer two calls back has run
     ok = (i < 2 || cudaStreamWaitEvent(hp->in, hp->comp_done[b], 0) == cudaSuccess) &&
-         cudaMemcpyAsync(Xd[b], c.X, (size_t)c.M * m.K * xe, cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
+         cudaMemcpyAsync(Xd[b], c.X, x_bytes(io.x_type, (size_t)c.M, (size_t)m.K), cudaMemcpyHostToDevice, hp->in) == cudaSuccess &&
          cudaEventRecord(hp->in_done[b], hp->in) == cudaSuccess &&
          // the layer: after its X has landed and after the Y buffer's previous contents have left
          cudaStreamWaitEvent(s, hp->in_done[b], 0) == cudaSuccess &&

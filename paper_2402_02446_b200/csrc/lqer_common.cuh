@@ -245,6 +245,41 @@ __device__ __forceinline__ void quantize_quad(const float4 vin, int bits, int em
   bf.y = __byte_perm(__float_as_uint(r[2]), __float_as_uint(r[3]), 0x7632);
 }
 
+// Element type of X at the layer's boundary: fp32, bf16, or MXINT (int8 mantissas [M, K] followed by the exponent bytes
+// [M, K / 16], the layout the MXINT8 output has).  An MXINT X is taken at its value: the loaders below turn a block's
+// mantissas into the fp32 values m * 2^(e - (bits - 2)) (exact), and the ordinary quantisers then see numbers that
+// are fixed points of the quantisation (or, for a block that is not normalised, the same values renormalised).
+constexpr int kXF32 = 0, kXBF16 = 1, kXMXINT8 = 2;
+inline size_t x_bytes(int x_type, size_t M, size_t K) { return x_type == kXMXINT8 ? M * K + M * K / 16 : M * K * (x_type == kXBF16 ? 2 : 4); }
+// Four mantissas (one word, element order) of a block with exponent byte eb -> their values.
+__device__ __forceinline__ float4 mxint_quad_values(uint32_t m8, uint32_t eb, int bits, int emin, int emax) {
+  const int e = min(max((int)eb - 127, emin), emax);
+  const float step = pow2f(e - (bits - 2));
+  const float back = -12583040.0f * step;                   // -(1.5 * 2^23 + 128) * step
+  const uint32_t u = m8 ^ 0x80808080u;                       // two's complement -> offset binary
+  // the bytes (u_i, 0x00, 0x40, 0x4B) are the float 1.5 * 2^23 + u_i: one byte permute converts, one fma scales (exact)
+  return make_float4(fmaf(__uint_as_float(__byte_perm(u, 0x4B400000u, 0x7640)), step, back),
+                     fmaf(__uint_as_float(__byte_perm(u, 0x4B400000u, 0x7641)), step, back),
+                     fmaf(__uint_as_float(__byte_perm(u, 0x4B400000u, 0x7642)), step, back),
+                     fmaf(__uint_as_float(__byte_perm(u, 0x4B400000u, 0x7643)), step, back));
+}
+// Four consecutive elements of row `row` from column `col` (a multiple of 4) of X [M, K] in any of the three types.
+__device__ __forceinline__ float4 load_x_quad(const void* X, int x_type, int M, int K, int row, int col, int bits, int emin, int emax) {
+  const size_t idx = (size_t)row * K + col;
+  if (x_type == kXBF16) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(X) + idx));
+    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
+                       __uint_as_float(v.y & 0xFFFF0000u));
+  }
+  if (x_type == kXMXINT8) {
+    const uint8_t* xb = static_cast<const uint8_t*>(X);
+    const uint32_t m8 = __ldg(reinterpret_cast<const uint32_t*>(xb + idx));
+    const uint32_t eb = __ldg(xb + (size_t)M * K + (size_t)row * (K / 16) + (col >> 4));
+    return mxint_quad_values(m8, eb, bits, emin, emax);
+  }
+  return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(X) + idx));
+}
+
 // What quantize_block16 needs of the format, computed once per kernel instead of once per block.
 struct QuantConsts {
   float qmax, qlim;      // 2^(bits-1) - 1, and qmax + 1/2
@@ -414,7 +449,7 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
                               uint8_t* Xe, cudaStream_t s);
 // X -> Xcat[:, 0:K64] (bf16 of the dequantised MXINT8 value) and T_q -> Xcat[:, K64:K64+k_pad];
 // optional int8 / exponent exports of T_q.
-cudaError_t launch_prologue(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
+cudaError_t launch_prologue(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* xcat,
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s);
 // The same prologue with the projection on the tcgen05 int8 tensor cores: ranks up to 64, large batches.
 bool prologue_tc_fits(const PackedMeta& m, int M, const void* X, bool any_batch);
@@ -422,14 +457,14 @@ bool prologue_tc_fits(const PackedMeta& m, int M, const void* X, bool any_batch)
 // one per row tile.  `order`: kChainAlone, or the place in a run of prologues that share no buffer or counter
 // (each later one overlaps the tail of the one before; the kernel after the run still finds all of them complete).
 enum ChainOrder { kChainAlone = 0, kChainFirst = 1, kChainLater = 2 };
-cudaError_t launch_prologue_tc(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
+cudaError_t launch_prologue_tc(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                int order, cudaStream_t s);
 // The same for up to 8 layers with one M, one k_pad and one set of formats in ONE launch (a CTA per row tile and K range
 // of a layer, found by its index); prologue_tc_group_splits picks the K ranges per row tile so that the CTAs carry
 // about equal work and stay within one per SM.
 bool prologue_tc_group_splits(const PackedMeta* metas, int n, int M, int max_ctas, int* splits);
-cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, const PackedMeta* metas, const void* const* packed,
+cudaError_t launch_prologue_tc_group(const void* const* Xs, int x_type, int M, const PackedMeta* metas, const void* const* packed,
                                      void* const* xcats, double* const* partials, int* const* counters,
                                      const int* splits, int n, int8_t* Tm, uint8_t* Te, DeviceStatus* st, int order,
                                      cudaStream_t s);
@@ -468,7 +503,7 @@ struct SmallPrologueLayer {
   uint8_t* Te;
 };
 int prologue_small_max_layers();
-cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, DeviceStatus* st, cudaStream_t s);
+cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, int x_type, DeviceStatus* st, cudaStream_t s);
 // The small-batch GEMM (tokens on the M side of a 64- or 128-row MMA, 256 weight columns on its N side); up to
 // gemm_small_max_layers() layers with one M per launch.
 struct SmallGemmLayer {
@@ -481,7 +516,7 @@ struct SmallGemmLayer {
 };
 int gemm_small_max_layers();
 cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, DeviceStatus* st, cudaStream_t s);
-cudaError_t launch_decode_cols(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);
 // Up to decode_cols_max_group() independent layers with one M (all fitting decode_cols_fits, N >= 32) in one launch.
@@ -492,7 +527,7 @@ bool decode_cols_fits(const PackedMeta& m, int M);
 int decode_cols_max_group();
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
                                      size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
-                                     bool x_bf16, bool y_bf16, cudaStream_t s);
+                                     int x_type, bool y_bf16, cudaStream_t s);
 // The quantised activations and T_q of up to decode_pre_max_calls() independent decode calls, computed ahead (one CTA
 // per call) into outs[i] (decode_pre_bytes each, 256-byte aligned); launch_decode_cols_group takes them as `pres` and
 // then has no X to quantise, no T to compute and nothing to exchange.  `order` as above.
@@ -502,6 +537,6 @@ inline size_t decode_pre_bytes(const PackedMeta& m, int M) {
 }
 int decode_pre_max_calls();
 cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas, uint8_t* const* outs, int n, int order,
-                              bool x_bf16, cudaStream_t s);
+                              int x_type, cudaStream_t s);
 
 }  // namespace lqer

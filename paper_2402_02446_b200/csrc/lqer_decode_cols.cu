@@ -54,7 +54,7 @@ constexpr int kTRanges = 16;      // CTAs of a layer that share the work of T = 
 constexpr int kMaxGroup = 16;  // independent layers with one M that may share a launch
 
 struct Layer {
-  const void* X;                // [M, K] fp32, or bf16 where Params::x_bf16
+  const void* X;                // [M, K] of Params::x_type
   void* Y;                      // [M, N] fp32, or bf16 where Params::y_bf16
   size_t y_extent;              // bytes behind Y, for the checked build
   const uint8_t* packed;
@@ -77,7 +77,7 @@ struct Params {
   DeviceStatus* status;
   int M;
   int a_bits, lr_bits, exp_min, exp_max;
-  int x_bf16, y_bf16;           // element types of X and Y (else fp32)
+  int x_type, y_bf16;           // X: kXF32, kXBF16 or kXMXINT8; Y: bf16, else fp32
   int w_bits;                   // mantissa bits of W_q: 4 (nibbles) or 2 (crumbs), one value for all layers of a launch
   long long wait_limit;         // bound of the wait for the other CTAs' partial sums, in clock cycles
 };
@@ -111,7 +111,7 @@ __host__ __device__ inline int t_subsets(int k_pad) {
   return tiles < kWarps ? kWarps / tiles : 1;
 }
 
-struct Formats { int a_bits, lr_bits, exp_min, exp_max, x_bf16, w_bits; };
+struct Formats { int a_bits, lr_bits, exp_min, exp_max, x_type, w_bits; };
 
 // X -> MXINT8 for the whole contraction, by all threads of the CTA: per row the mantissas in the byte order the nibbles
 // unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales 2^(e_x - 6) and the dp4a seeds (bits of
@@ -128,15 +128,7 @@ __device__ __forceinline__ void quantize_x_rows(const void* X, int M, int K, int
       const int item = base + u * kThreads + tid;
       const int row = item / per_row, c4 = item % per_row;
       v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (item < total && c4 * 4 < K) {
-        if (f.x_bf16) {                            // 16-bit activations: every bf16 value is an fp32 value
-          const uint2 h = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(X) + (size_t)row * K + c4 * 4));
-          v[u] = make_float4(__uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u), __uint_as_float(h.y << 16),
-                             __uint_as_float(h.y & 0xFFFF0000u));
-        } else {
-          v[u] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(X) + (size_t)row * K + c4 * 4));
-        }
-      }
+      if (item < total && c4 * 4 < K) v[u] = load_x_quad(X, f.x_type, M, K, row, c4 * 4, f.a_bits, f.exp_min, f.exp_max);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -397,7 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 
   // ---- X -> MXINT8 for the whole contraction: per row the mantissas in the byte order the nibbles
   //      unpack to ({0,4,1,5}, {2,6,3,7} within each 8), the block scales and the offsets 8 * sum(x)
-  const Formats fmt = {p.a_bits, p.lr_bits, p.exp_min, p.exp_max, p.x_bf16, WB};
+  const Formats fmt = {p.a_bits, p.lr_bits, p.exp_min, p.exp_max, p.x_type, WB};
   if (pre) {                                       // quantised X and T_q are there already: straight into shared memory
     const int xb = (int)pre_x_bytes(M, ly.K64), tb = (int)pre_t_bytes(ly.k_pad);
     for (int o = tid * 16; o < xb; o += kThreads * 16)
@@ -662,10 +654,10 @@ static size_t cols_smem_bytes(const PackedMeta& m, int M) {
 // the whole contraction fits in shared memory.
 bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
 
-cudaError_t launch_decode_cols(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
                                void* workspace, cudaStream_t s) {
   const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
-  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, nullptr, x_bf16, y_bf16, s);
+  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, nullptr, x_type, y_bf16, s);
 }
 
 int decode_cols_max_group() { return dcol::kMaxGroup; }
@@ -676,7 +668,7 @@ int decode_cols_max_group() { return dcol::kMaxGroup; }
 // at least one cluster's worth of column groups.
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
                                      size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
-                                     bool x_bf16, bool y_bf16, cudaStream_t s) {
+                                     int x_type, bool y_bf16, cudaStream_t s) {
   using namespace dcol;
   static OncePerDevice once;
   static bool one_cta_per_sm = true;               // false if any device could hold two CTAs of the kernel on one SM
@@ -703,7 +695,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   p.status = reinterpret_cast<DeviceStatus*>(workspace);
   p.M = M;
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
-  p.x_bf16 = x_bf16 ? 1 : 0;
+  p.x_type = x_type;
   p.w_bits = metas[0].w_bits;
   p.y_bf16 = y_bf16 ? 1 : 0;
   p.wait_limit = wait_limit_cycles();
@@ -809,7 +801,7 @@ int decode_pre_max_calls() { return dcol::kPreMaxCalls; }
 // X_q and T_q of n independent decode calls (M <= 4 each, every layer fitting decode_cols_fits), one CTA per call, into
 // outs[i] (decode_pre_bytes each, 256-byte aligned).
 cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas, uint8_t* const* outs, int n, int order,
-                              bool x_bf16, cudaStream_t s) {
+                              int x_type, cudaStream_t s) {
   using namespace dcol;
   static OncePerDevice once;
   cudaError_t e0 = once.run([] {
@@ -832,7 +824,7 @@ cudaError_t launch_decode_pre(const lqer_call_t* calls, const PackedMeta* metas,
     c.asec = static_cast<const uint8_t*>(calls[g].packed) + m.off_a;
     c.out = outs[g];
     c.M = calls[g].M; c.K = m.K; c.K64 = m.K64; c.k_pad = m.k_pad;
-    c.f = Formats{m.a_bits, m.lr_bits, m.exp_min, m.exp_max, x_bf16 ? 1 : 0, m.w_bits};
+    c.f = Formats{m.a_bits, m.lr_bits, m.exp_min, m.exp_max, x_type, m.w_bits};
     if (c.M < 1 || c.M > kMaxM) return cudaErrorInvalidValue;
     if (c.M > 1) single = false;
     const size_t need = pre_x_bytes(c.M, c.K64) + pre_t_bytes(c.k_pad) + 16 +

@@ -74,7 +74,7 @@ __device__ __forceinline__ double ld_dsmem_f64(const double* local, uint32_t cta
 // takes the K steps s = r, r + CS, ...; the partial T sums meet through distributed shared memory.
 // TPW = rank tiles one warp can own (1 for ranks up to 64): fewer accumulators, more CTAs per SM.
 template <int PB, int TPW>
-__global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(const void* __restrict__ X, int x_bf16, int M, PackedMeta m,
+__global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(const void* __restrict__ X, int x_type, int M, PackedMeta m,
                                                                const uint8_t* __restrict__ asec,
                                                                uint16_t* __restrict__ xcat,
                                                                int8_t* __restrict__ Tm, uint8_t* __restrict__ Te,
@@ -113,15 +113,7 @@ __global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : 2) prologue_kernel(co
       const int r = f / (SW / 4), c4 = f % (SW / 4);
       const int col = s * SW + c4 * 4, row = row0 + r;
       xr[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (row < M && col < m.K) {
-        if (x_bf16) {
-          const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(X) + (size_t)row * m.K + col));
-          xr[i] = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
-                              __uint_as_float(v.y & 0xFFFF0000u));
-        } else {
-          xr[i] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(X) + (size_t)row * m.K + col));
-        }
-      }
+      if (row < M && col < m.K) xr[i] = load_x_quad(X, x_type, M, m.K, row, col, m.a_bits, m.exp_min, m.exp_max);
     }
   };
   auto load_panel = [&](int s, int buf) {
@@ -259,7 +251,7 @@ cudaError_t launch_quantize_x(const float* X, int M, int K, int bits, int emin, 
 }
 
 template <int PB, int TPW>
-static cudaError_t launch_prologue_pb(const void* X, bool x_bf16, int M, const PackedMeta& m, const uint8_t* asec, uint16_t* xc,
+static cudaError_t launch_prologue_pb(const void* X, int x_type, int M, const PackedMeta& m, const uint8_t* asec, uint16_t* xc,
                                       int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s) {
   const int groups = (M + kRows - 1) / kRows;
   const int steps = (m.K64 + PB * 16 - 1) / (PB * 16);
@@ -276,16 +268,16 @@ static cudaError_t launch_prologue_pb(const void* X, bool x_bf16, int M, const P
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   LaunchScope scope(kFamPrologue, s);
-  return cudaLaunchKernelEx(&cfg, prologue_kernel<PB, TPW>, X, x_bf16 ? 1 : 0, M, m, asec, xc, Tm, Te, st);
+  return cudaLaunchKernelEx(&cfg, prologue_kernel<PB, TPW>, X, x_type, M, m, asec, xc, Tm, Te, st);
 }
 
-cudaError_t launch_prologue(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
+cudaError_t launch_prologue(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* xcat,
                             int8_t* Tm, uint8_t* Te, DeviceStatus* st, cudaStream_t s) {
   const uint8_t* asec = static_cast<const uint8_t*>(packed) + m.off_a;
   uint16_t* xc = static_cast<uint16_t*>(xcat);
-  if (m.k_pad <= 64) return launch_prologue_pb<16, 1>(X, x_bf16, M, m, asec, xc, Tm, Te, st, s);
-  if (m.k_pad <= 128) return launch_prologue_pb<8, 2>(X, x_bf16, M, m, asec, xc, Tm, Te, st, s);
-  return launch_prologue_pb<4, 4>(X, x_bf16, M, m, asec, xc, Tm, Te, st, s);
+  if (m.k_pad <= 64) return launch_prologue_pb<16, 1>(X, x_type, M, m, asec, xc, Tm, Te, st, s);
+  if (m.k_pad <= 128) return launch_prologue_pb<8, 2>(X, x_type, M, m, asec, xc, Tm, Te, st, s);
+  return launch_prologue_pb<4, 4>(X, x_type, M, m, asec, xc, Tm, Te, st, s);
 }
 
 }  // namespace lqer

@@ -43,18 +43,9 @@ struct Params {
   int n;                      // layers in this launch
   int M;
   DeviceStatus* status;
-  int x_bf16;                 // X is bf16 (else fp32)
+  int x_type;                 // kXF32, kXBF16 or kXMXINT8
   int a_bits, lr_bits, exp_min, exp_max;
 };
-
-__device__ __forceinline__ float4 load_x4(const void* X, size_t idx, int x_bf16) {
-  if (x_bf16) {
-    const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(X) + idx));
-    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
-                       __uint_as_float(v.y & 0xFFFF0000u));
-  }
-  return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(X) + idx));
-}
 
 // TPW: rank tiles (8 columns) a warp owns: 1 for ranks up to 64, 2 up to 128, 4 up to 256.
 template <int TPW>
@@ -120,7 +111,7 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
         const int r = live ? f / quads_per_row : 0, c4 = live ? f % quads_per_row : 0;
         const int col = kb0 * 16 + c4 * 4, row = row0 + r;
         v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (live && row < M && col < K) v[u] = load_x4(ly.X, (size_t)row * K + col, p.x_bf16);
+        if (live && row < M && col < K) v[u] = load_x_quad(ly.X, p.x_type, M, K, row, col, p.a_bits, p.exp_min, p.exp_max);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -256,13 +247,13 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
 
 int prologue_small_max_layers() { return psm::kMaxLayers; }
 
-cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, bool x_bf16, DeviceStatus* st, cudaStream_t s) {
+cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, int x_type, DeviceStatus* st, cudaStream_t s) {
   using namespace psm;
   if (n < 1 || n > kMaxLayers || M < 1) return cudaErrorInvalidValue;
   Params p;
   p.n = n;
   p.M = M;
-  p.x_bf16 = x_bf16 ? 1 : 0;
+  p.x_type = x_type;
   const PackedMeta& m0 = *layers[0].meta;
   p.status = st;
   p.a_bits = m0.a_bits; p.lr_bits = m0.lr_bits; p.exp_min = m0.exp_min; p.exp_max = m0.exp_max;

@@ -85,7 +85,8 @@ struct Params {
   long long wait_limit;     // bound of every wait, in clock cycles
   int a_bits, lr_bits, exp_min, exp_max;
   int order;                // ChainOrder: where the wait for the previous kernel sits
-  int x_bf16;               // X is bf16 (a stage of the ring then holds 16 KB), else fp32
+  int x_type;               // kXF32 (a stage of the ring holds 32 KB), kXBF16 (16 KB) or kXMXINT8 (8 KB of mantissas)
+  const uint8_t* x_exp;     // MXINT X: its exponent bytes [M, K / 16]
   size_t ldx;               // columns of Xcat
   size_t xcat_extent, partials_extent;   // bytes behind xcat and partials, for the checked build
 };
@@ -313,8 +314,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
     const int rows_ok = p.M - (row0 + r0);              // pass i is a real row while 8 * QW * i < rows_ok
     // offsets of the lane's block within a raw slot: fp32 = two half tiles of 32 columns (16 KB each, rows of 128
     // bytes), the block is four chunks; bf16 = one tile of 64 columns, the block is two chunks
-    const uint32_t raw_off = p.x_bf16 ? (uint32_t)(r0 * 128) : (uint32_t)((blk >> 1) * (RAW_BYTES / 2) + r0 * 128);
-    const uint32_t chunk0 = p.x_bf16 ? (uint32_t)(blk * 2) : (uint32_t)((blk & 1) * 4);
+    // an MXINT X: the tile is 128 rows of 64 mantissa bytes (64-byte swizzle: chunk ^ (row / 2 mod 4)), the block one chunk
+    const uint32_t raw_off = p.x_type == kXMXINT8 ? (uint32_t)(r0 * 64)
+                             : p.x_type == kXBF16 ? (uint32_t)(r0 * 128) : (uint32_t)((blk >> 1) * (RAW_BYTES / 2) + r0 * 128);
+    const uint32_t chunk0 = p.x_type == kXBF16 ? (uint32_t)(blk * 2) : (uint32_t)((blk & 1) * 4);
+    const uint32_t swz64 = (uint32_t)((lane >> 1) & 3);   // (row >> 1) & 3: the rows of a pass differ by multiples of 8
+    const int kb_row = p.K / 16;
     bool ok = true;
     for (int s = 0; s < n_stages && ok; ++s) {
       const int rs = s % RAW_SLOTS, xs = s % X_SLOTS;
@@ -330,7 +335,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
       for (int i = 0; i < C::BPL; ++i) {
         float v[16];
         const uint8_t* row = src + i * (8 * QW) * 128;
-        if (p.x_bf16) {
+        if (p.x_type == kXMXINT8) {
+          const uint4 w = *reinterpret_cast<const uint4*>(src + i * (8 * QW) * 64 + ((blk ^ swz64) << 4));
+          const int grow = row0 + r0 + i * (8 * QW), kb = (pan_lo * 2 + s) * 4 + blk;
+          const uint32_t eb = (grow < p.M && kb < kb_row) ? (uint32_t)__ldg(p.x_exp + (size_t)grow * kb_row + kb) : 127u;
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const float4 q = mxint_quad_values(ww[t], eb, p.a_bits, p.exp_min, p.exp_max);
+            v[4 * t] = q.x; v[4 * t + 1] = q.y; v[4 * t + 2] = q.z; v[4 * t + 3] = q.w;
+          }
+        } else if (p.x_type == kXBF16) {
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             const uint4 w = *reinterpret_cast<const uint4*>(row + (((chunk0 + j) ^ swz) << 4));
@@ -443,11 +458,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
       for (int s = 0; s < n_stages; ++s) {
         const int rs = s % RAW_SLOTS;
         if (!parked_wait(raw_empty(rs), ((s / RAW_SLOTS) & 1) ^ 1, abort_flag, kNapNs)) break;
-        mbar_expect_tx(raw_full(rs), p.x_bf16 ? RAW_BYTES / 2 : RAW_BYTES);       // rows and columns outside X arrive as zeros
+        mbar_expect_tx(raw_full(rs), p.x_type == kXMXINT8 ? RAW_BYTES / 4 : p.x_type == kXBF16 ? RAW_BYTES / 2 : RAW_BYTES);   // rows and columns outside X arrive as zeros
         const uint32_t dst = smem_u32(raw_base + rs * RAW_BYTES);
         const int col = (pan_lo * 2 + s) * STAGE_COLS;
         tma_load_2d(dst, tmap_x, col, row0, raw_full(rs));                         // a box is 128 bytes wide (swizzled rows):
-        if (!p.x_bf16) tma_load_2d(dst + RAW_BYTES / 2, tmap_x, col + STAGE_COLS / 2, row0, raw_full(rs));   // fp32 takes two
+        if (p.x_type == kXF32) tma_load_2d(dst + RAW_BYTES / 2, tmap_x, col + STAGE_COLS / 2, row0, raw_full(rs));   // fp32 takes two
       }
     }
   }
@@ -610,7 +625,7 @@ bool prologue_tc_group_splits(const PackedMeta* metas, int n, int M, int max_cta
 
 // n layers (one M, one k_pad, one set of formats) in ONE launch.  splits[g] K ranges per row tile of layer g; the
 // caller sees to it that the CTAs (row tiles x splits, summed) are at most one per SM.  Tm / Te: for n == 1 only.
-cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, const PackedMeta* metas, const void* const* packed,
+cudaError_t launch_prologue_tc_group(const void* const* Xs, int x_type, int M, const PackedMeta* metas, const void* const* packed,
                                      void* const* xcats, double* const* partials, int* const* counters,
                                      const int* splits, int n, int8_t* Tm, uint8_t* Te, DeviceStatus* st, int order,
                                      cudaStream_t s) {
@@ -629,12 +644,15 @@ cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, 
     const PackedMeta& m = metas[g];
     if (m.k_pad != metas[0].k_pad) return cudaErrorInvalidValue;
     const cuuint64_t dims[2] = {(cuuint64_t)m.K, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)m.K * (x_bf16 ? 2 : 4)};
-    const cuuint32_t box[2] = {(cuuint32_t)(x_bf16 ? STAGE_COLS : STAGE_COLS / 2), ROWS};   // 128 bytes wide: one swizzled row
+    const cuuint64_t strides[1] = {(cuuint64_t)m.K * (x_type == kXMXINT8 ? 1 : x_type == kXBF16 ? 2 : 4)};
+    // a box is one swizzled row wide: 128 bytes of fp32 (half a stage) or bf16, 64 bytes of MXINT mantissas
+    const cuuint32_t box[2] = {(cuuint32_t)(x_type == kXF32 ? STAGE_COLS / 2 : STAGE_COLS), ROWS};
+    const CUtensorMapDataType x_dt = x_type == kXMXINT8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                     : x_type == kXBF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&tmaps.m[i], x_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(Xs[g]), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    if (enc(&tmaps.m[i], x_dt, 2, const_cast<void*>(Xs[g]), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, x_type == kXMXINT8 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
     Params& p = gp.L[i];
     p.asec = static_cast<const uint8_t*>(packed[g]) + m.off_a;
@@ -649,7 +667,8 @@ cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, 
     p.wait_limit = limit;
     p.a_bits = m.a_bits; p.lr_bits = m.lr_bits; p.exp_min = m.exp_min; p.exp_max = m.exp_max;
     p.order = order;
-    p.x_bf16 = x_bf16 ? 1 : 0;
+    p.x_type = x_type;
+    p.x_exp = static_cast<const uint8_t*>(Xs[g]) + (size_t)M * m.K;
     p.ldx = xcat_cols(m);
     p.xcat_extent = (size_t)M * xcat_cols(m) * 2;
     p.partials_extent = (size_t)((M + ROWS - 1) / ROWS) * splits[g] * ROWS * m.k_pad * 8;
@@ -664,12 +683,12 @@ cudaError_t launch_prologue_tc_group(const void* const* Xs, bool x_bf16, int M, 
   }
 }
 
-cudaError_t launch_prologue_tc(const void* X, bool x_bf16, int M, const PackedMeta& m, const void* packed, void* xcat,
+cudaError_t launch_prologue_tc(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* xcat,
                                int8_t* Tm, uint8_t* Te, DeviceStatus* st, double* partials, int* counters,
                                int order, cudaStream_t s) {
   const int sms = sm_count();
   const int splits = prologue_tc_splits(m, M, sms > 0 && sms < kPrologueMaxCtas ? sms : kPrologueMaxCtas);
-  return launch_prologue_tc_group(&X, x_bf16, M, &m, &packed, &xcat, &partials, &counters, &splits, 1, Tm, Te, st, order, s);
+  return launch_prologue_tc_group(&X, x_type, M, &m, &packed, &xcat, &partials, &counters, &splits, 1, Tm, Te, st, order, s);
 }
 
 }  // namespace lqer

@@ -179,7 +179,112 @@ def test_mxint8_output_is_refused_where_it_cannot_be_written():
     launches = L.launch_count()
     st = L.lib().lqer_linear_ex(X.data_ptr(), 0, spec.M, Pg.ptr, Y.data_ptr(), 2, ws.data_ptr(), ws.numel(), None)
     assert st == E("LQER_ERR_SHAPE")
-    st = L.lib().lqer_linear_ex(X.data_ptr(), 2, spec.M, Pg.ptr, Y.data_ptr(), 0, ws.data_ptr(), ws.numel(), None)
-    assert st == E("LQER_ERR_CONFIG")                     # MXINT8 is an output type only
+    st = L.lib().lqer_linear_ex(X.data_ptr(), 7, spec.M, Pg.ptr, Y.data_ptr(), 0, ws.data_ptr(), ws.numel(), None)
+    assert st == E("LQER_ERR_CONFIG")                     # no such element type
     assert L.launch_count() == launches
+    Pg.release()
+
+
+# ---------------------------------------------------------------------------- MXINT8 input
+# X given as mantissas + exponent bytes (the layout of the MXINT8 output): the layer takes it at its value, so it must
+# compute exactly what it computes on the fp32 tensor of those values - compared bit for bit with the library's own
+# fp32-input result (same path, same X_q) and, through that input, with the oracle.
+
+
+def _mx_buffer(Xm, Xe):
+    return L.to_mxint8(_t(Xm), _t(mxint.exponent_bytes(Xe)))
+
+
+@pytest.mark.parametrize("spec", SPECS + [gen.LayerSpec("q_ragged", M=300, K=80, N=144, k=5, calib_rows=32, outlier_frac=0, n_outliers=2,
+                                                        outlier_scale=20.0, seed=431)], ids=lambda s: s.name)
+def test_mxint8_input_every_path(spec):
+    P, Pg = _layer(spec)
+    ws = L.new_workspace(spec.M, Pg)
+    for M in (1, 4, 9, 70, 200, spec.M):
+        if M > spec.M:
+            continue
+        X = gen.make_activations(spec, M=M)
+        Xm, Xe = mxint.quantize(X, 8, axis=1)                     # what a previous layer's MXINT8 output would hold
+        Xq = _mx_buffer(Xm, Xe)
+        ref = olqer.forward(X, P)                                  # the oracle quantises X itself: the same X_q
+        assert np.array_equal(ref.Xm, Xm)
+        for path in (binding.PATH_AUTO, binding.PATH_TENSOR_PROLOGUE, binding.PATH_TENSOR):
+            if path != binding.PATH_AUTO and M < 70:
+                continue
+            L.set_path(path)
+            try:
+                Y = L.linear_ex(Xq, Pg, ws, M=M)
+                Yf = L.linear(_t(X), Pg, ws)
+            finally:
+                L.set_path(binding.PATH_AUTO)
+            assert L.poll_status(ws) == 0
+            assert torch.equal(Y, Yf), (M, path)
+            assert float(np.max(np.abs(Y.cpu().numpy().astype(np.float64) - ref.Y) / ref.tol)) <= 1.0, (M, path)
+    Pg.release()
+
+
+def test_mxint8_input_blocks_that_are_not_normalised():
+    # mantissas a quantiser would not have produced (small ones under a large exponent, -128, all-zero blocks under
+    # any exponent): the layer must compute on their values, i.e. what it computes on the fp32 tensor of these values
+    spec = gen.LayerSpec("q_raw", M=40, K=512, N=256, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=432)
+    P, Pg = _layer(spec)
+    g = np.random.default_rng(432)
+    Xm = g.integers(-20, 21, size=(spec.M, spec.K)).astype(np.int8)
+    Xm[:, ::37] = -128
+    Xm[3, 16:48] = 0
+    Xe = g.integers(-8, 9, size=(spec.M, spec.K // 16)).astype(np.int64)
+    X = mxint.dequantize(Xm, Xe, 8, axis=1).astype(np.float32)     # exact: at most 8 significant bits
+    ref = olqer.forward(X, P)
+    ws = L.new_workspace(spec.M, Pg)
+    for M in (2, spec.M):
+        Y = L.linear_ex(L.to_mxint8(_t(Xm[:M]), _t(mxint.exponent_bytes(Xe[:M]))), Pg, ws, M=M)
+        assert L.poll_status(ws) == 0
+        assert torch.equal(Y, L.linear(_t(X[:M]), Pg, ws))
+        assert float(np.max(np.abs(Y.cpu().numpy().astype(np.float64) - ref.Y[:M]) / ref.tol[:M])) <= 1.0
+    Pg.release()
+
+
+def test_mxint8_chain_of_two_layers_equals_the_fp32_hand_over():
+    # layer 1 writes MXINT8, layer 2 reads it: bit for bit what layer 2 gives on layer 1's fp32 output, because the
+    # hand-over quantisation is the one layer 2's prologue would have done itself
+    s1 = gen.LayerSpec("q_c1", M=300, K=512, N=1024, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=441)
+    s2 = gen.LayerSpec("q_c2", M=300, K=1024, N=384, k=32, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=442)
+    (_, Pg1), (_, Pg2) = _layer(s1), _layer(s2)
+    for M in (1, 3, 24, 300):
+        X = _t(gen.make_activations(s1, M=M))
+        ws = L.new_workspace(M, Pg1 if L.workspace_bytes(M, s1.K, s1.N, s1.k) > L.workspace_bytes(M, s2.K, s2.N, s2.k) else Pg2)
+        Y1 = L.linear(X, Pg1, ws)
+        Y2 = L.linear(Y1, Pg2, ws)
+        H = L.linear_ex(X, Pg1, ws, out_dtype=L.MXINT8)            # the hand-over buffer: 17 bytes per 16 activations
+        Y2q = L.linear_ex(H, Pg2, ws, M=M)
+        assert L.poll_status(ws) == 0
+        assert torch.equal(Y2q, Y2), M
+    Pg1.release()
+    Pg2.release()
+
+
+def test_mxint8_input_of_shared_launches_and_host_buffers():
+    spec = gen.LayerSpec("q_in_b", M=1, K=1024, N=640, k=40, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=451)
+    P, Pg = _layer(spec)
+    for M, n in ((1, 20), (24, 3), (300, 3)):
+        Xs = [gen.make_activations(spec, M=M) + 0.125 * j for j in range(n)]
+        Xq = [_mx_buffer(*mxint.quantize(X, 8, axis=1)) for X in Xs]
+        Ys = [torch.zeros((M, spec.N), dtype=torch.float32, device=DEV) for _ in Xs]
+        calls = L.make_calls([(x, Pg, y) for x, y in zip(Xq, Ys)], L.MXINT8, torch.float32)
+        ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+        L.linear_batched_ex(calls, ws, L.MXINT8, torch.float32)
+        torch.cuda.synchronize()
+        assert L.poll_status(ws) == 0
+        for X, y in zip(Xs, Ys):
+            ref = olqer.forward(X, P)
+            assert float(np.max(np.abs(y.cpu().numpy().astype(np.float64) - ref.Y) / ref.tol)) <= 1.0
+            if M != 24:        # (small-batch groups cut K into fewer chunks than single calls: compared with the oracle only)
+                assert torch.equal(y, L.linear(_t(X), Pg, ws))
+        Xh = [x.cpu().pin_memory() for x in Xq]
+        Yh = [torch.zeros((M, spec.N), dtype=torch.float32).pin_memory() for _ in Xs]
+        hcalls = L.make_host_calls([(x, Pg, y) for x, y in zip(Xh, Yh)], L.MXINT8, torch.float32)
+        wsh = torch.zeros(L.linear_host_batched_bytes(hcalls), dtype=torch.uint8, device=DEV)
+        L.linear_host_batched_ex(hcalls, wsh, L.MXINT8, torch.float32)
+        for X, yh in zip(Xs, Yh):
+            assert torch.equal(yh, L.linear(_t(X), Pg, wsh).cpu())
     Pg.release()
