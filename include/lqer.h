@@ -193,9 +193,10 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * the small-batch kernels for this output (the column-owner kernel's CTAs do not own whole blocks).
  * x_dtype LQER_MXINT8: X is given in the same layout - mantissas [M,K], then exponent bytes [M,K/16], M*K + M*K/16
  * bytes - with the mantissa width and exponent window of the layer's lqer_config_t (what a previous layer's MXINT8
- * output holds if it has the same format).  It is taken at its value: a block that a quantiser would have produced
- * passes through unchanged, any other block is renormalised without changing its values, so the layer computes
- * exactly what it computes on the fp32 tensor of those values - without reading 4 bytes per element. */
+ * output holds if it has the same format; mantissas within the format's symmetric range, |m| <= 2^(a_bits-1) - 1).
+ * It is taken at its value: a block that a quantiser would have produced passes through unchanged, any other block
+ * stands for the same values as its normalised form, so the layer computes exactly what it computes on the fp32
+ * tensor of those values - without reading 4 bytes per element. */
 lqer_status_t lqer_linear_ex(const void* X, lqer_dtype_t x_dtype, int M, const void* packed, void* Y, lqer_dtype_t y_dtype,
                              void* workspace, size_t workspace_bytes, void* stream);
 lqer_status_t lqer_linear_batched_ex(const lqer_call_t* calls, int n_calls, lqer_dtype_t x_dtype, lqer_dtype_t y_dtype,

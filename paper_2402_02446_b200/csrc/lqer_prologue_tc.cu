@@ -333,43 +333,56 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) prologue_tc_kernel(const __gri
       uint16_t* cd = cp + (size_t)s * STAGE_COLS;
 #pragma unroll
       for (int i = 0; i < C::BPL; ++i) {
-        float v[16];
         const uint8_t* row = src + i * (8 * QW) * 128;
+        uint4 m8, bf0, bf1;
+        int e;
         if (p.x_type == kXMXINT8) {
-          const uint4 w = *reinterpret_cast<const uint4*>(src + i * (8 * QW) * 64 + ((blk ^ swz64) << 4));
+          // the block is quantised already: its mantissas are the MMA's operand as they stand, its values m * 2^(e - 6)
+          // go to Xcat (a block that is not normalised gives the same values, hence the same T and Y, as its normal form)
+          m8 = *reinterpret_cast<const uint4*>(src + i * (8 * QW) * 64 + ((blk ^ swz64) << 4));
           const int grow = row0 + r0 + i * (8 * QW), kb = (pan_lo * 2 + s) * 4 + blk;
           const uint32_t eb = (grow < p.M && kb < kb_row) ? (uint32_t)__ldg(p.x_exp + (size_t)grow * kb_row + kb) : 127u;
-          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+          if (i == C::BPL - 1) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(raw_empty(rs));
+          }
+          e = min(max((int)eb - 127, p.exp_min), p.exp_max);
+          const uint32_t ww[4] = {m8.x, m8.y, m8.z, m8.w};
+          uint32_t b[8];
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
             const float4 q = mxint_quad_values(ww[t], eb, p.a_bits, p.exp_min, p.exp_max);
-            v[4 * t] = q.x; v[4 * t + 1] = q.y; v[4 * t + 2] = q.z; v[4 * t + 3] = q.w;
+            b[2 * t] = __byte_perm(__float_as_uint(q.x), __float_as_uint(q.y), 0x7632);
+            b[2 * t + 1] = __byte_perm(__float_as_uint(q.z), __float_as_uint(q.w), 0x7632);
           }
-        } else if (p.x_type == kXBF16) {
+          bf0 = make_uint4(b[0], b[1], b[2], b[3]);
+          bf1 = make_uint4(b[4], b[5], b[6], b[7]);
+        } else {
+          float v[16];
+          if (p.x_type == kXBF16) {
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const uint4 w = *reinterpret_cast<const uint4*>(row + (((chunk0 + j) ^ swz) << 4));
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+            for (int j = 0; j < 2; ++j) {
+              const uint4 w = *reinterpret_cast<const uint4*>(row + (((chunk0 + j) ^ swz) << 4));
+              const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              v[8 * j + 2 * t] = __uint_as_float(ww[t] << 16);
-              v[8 * j + 2 * t + 1] = __uint_as_float(ww[t] & 0xFFFF0000u);
+              for (int t = 0; t < 4; ++t) {
+                v[8 * j + 2 * t] = __uint_as_float(ww[t] << 16);
+                v[8 * j + 2 * t + 1] = __uint_as_float(ww[t] & 0xFFFF0000u);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float4 w = *reinterpret_cast<const float4*>(row + (((chunk0 + j) ^ swz) << 4));
+              v[4 * j] = w.x; v[4 * j + 1] = w.y; v[4 * j + 2] = w.z; v[4 * j + 3] = w.w;
             }
           }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float4 w = *reinterpret_cast<const float4*>(row + (((chunk0 + j) ^ swz) << 4));
-            v[4 * j] = w.x; v[4 * j + 1] = w.y; v[4 * j + 2] = w.z; v[4 * j + 3] = w.w;
+          if (i == C::BPL - 1) {                       // the stage's values are in registers: the slot can be refilled
+            __syncwarp();
+            if (lane == 0) mbar_arrive(raw_empty(rs));
           }
+          quantize_block16(v, qc, e, m8, bf0, bf1);
         }
-        if (i == C::BPL - 1) {                         // the stage's values are in registers: the slot can be refilled
-          __syncwarp();
-          if (lane == 0) mbar_arrive(raw_empty(rs));
-        }
-        uint4 m8, bf0, bf1;
-        int e;
-        quantize_block16(v, qc, e, m8, bf0, bf1);
         *reinterpret_cast<uint4*>(xdst + i * (8 * QW) * 128) = m8;
         xe_dst[i * (8 * QW) * 4] = (int8_t)e;
         if (store_ok && 8 * QW * i < rows_ok &&

@@ -224,22 +224,28 @@ def test_mxint8_input_every_path(spec):
 
 
 def test_mxint8_input_blocks_that_are_not_normalised():
-    # mantissas a quantiser would not have produced (small ones under a large exponent, -128, all-zero blocks under
-    # any exponent): the layer must compute on their values, i.e. what it computes on the fp32 tensor of these values
+    # blocks a quantiser would not have produced (small mantissas under a large exponent, the extreme -127 beside odd
+    # mantissas, all-zero blocks under any exponent): the layer must compute on their values, i.e. what it computes on the fp32 tensor of these values
     spec = gen.LayerSpec("q_raw", M=40, K=512, N=256, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=432)
     P, Pg = _layer(spec)
     g = np.random.default_rng(432)
     Xm = g.integers(-20, 21, size=(spec.M, spec.K)).astype(np.int8)
-    Xm[:, ::37] = -128
+    Xm[:, ::37] = -127
     Xm[3, 16:48] = 0
     Xe = g.integers(-8, 9, size=(spec.M, spec.K // 16)).astype(np.int64)
     X = mxint.dequantize(Xm, Xe, 8, axis=1).astype(np.float32)     # exact: at most 8 significant bits
     ref = olqer.forward(X, P)
     ws = L.new_workspace(spec.M, Pg)
-    for M in (2, spec.M):
-        Y = L.linear_ex(L.to_mxint8(_t(Xm[:M]), _t(mxint.exponent_bytes(Xe[:M]))), Pg, ws, M=M)
+    for M, path in ((2, binding.PATH_AUTO), (spec.M, binding.PATH_AUTO), (spec.M, binding.PATH_TENSOR),
+                    (spec.M, binding.PATH_TENSOR_PROLOGUE)):       # the last takes the mantissas as they stand
+        L.set_path(path)
+        try:
+            Y = L.linear_ex(L.to_mxint8(_t(Xm[:M]), _t(mxint.exponent_bytes(Xe[:M]))), Pg, ws, M=M)
+            Yf = L.linear(_t(X[:M]), Pg, ws)
+        finally:
+            L.set_path(binding.PATH_AUTO)
         assert L.poll_status(ws) == 0
-        assert torch.equal(Y, L.linear(_t(X[:M]), Pg, ws))
+        assert torch.equal(Y, Yf), (M, path)
         assert float(np.max(np.abs(Y.cpu().numpy().astype(np.float64) - ref.Y[:M]) / ref.tol[:M])) <= 1.0
     Pg.release()
 
