@@ -189,8 +189,7 @@ lqer_status_t lqer_linear_stream(const float* X, int M, const void* packed, floa
  * MXINT, blocks [1,16]): the epilogue quantises Y itself, in blocks of 16 along N (the next layer's K), to the
  * layer's activation format (a_bits and exponent window of its lqer_config_t), exactly as the next layer's
  * prologue would quantise the fp32 Y.  Y then points to M*N + M*N/16 bytes: the int8 mantissas [M,N] followed
- * directly by the exponent bytes [M,N/16] (e + 127); N must be a multiple of 16.  Calls of up to 4 rows take
- * the small-batch kernels for this output (the column-owner kernel's CTAs do not own whole blocks).
+ * directly by the exponent bytes [M,N/16] (e + 127); N must be a multiple of 16.
  * x_dtype LQER_MXINT8: X is given in the same layout - mantissas [M,K], then exponent bytes [M,K/16], M*K + M*K/16
  * bytes - with the mantissa width and exponent window of the layer's lqer_config_t (what a previous layer's MXINT8
  * output holds if it has the same format; mantissas within the format's symmetric range, |m| <= 2^(a_bits-1) - 1).

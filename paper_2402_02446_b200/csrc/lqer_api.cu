@@ -198,7 +198,6 @@ static size_t workspace_total(const PackedMeta& m, int M_max) {
 struct IoTypes {
   int x_type = kXF32;          // kXF32, kXBF16 or kXMXINT8
   int y_type = kYF32;          // kYF32, kYBF16 or kYMXINT8
-  bool y_bf16() const { return y_type == kYBF16; }
 };
 
 // n small-batch layers with one M (n == 1: a single call): one launch of the small prologue for all of them, then one
@@ -249,8 +248,8 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   void* xcat = wsb + align_up(persist_bytes(m), 256);
   cudaError_t err;
   if (small) {
-    if (path != 5 && !project_only && io.y_type != kYMXINT8 && decode_cols_fits(m, M)) {
-      err = launch_decode_cols(X, io.x_type, M, m, packed, Y, io.y_bf16(), workspace, s);
+    if (path != 5 && !project_only && decode_cols_fits(m, M)) {
+      err = launch_decode_cols(X, io.x_type, M, m, packed, Y, io.y_type, workspace, s);
     } else {
       const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
       uint8_t* slice = static_cast<uint8_t*>(xcat);
@@ -735,7 +734,7 @@ lqer_status_t lqer_linear(const float* X, int M, const void* packed, float* Y, v
 // The batched entry points: independent calls share launches where the path is left at 0.
 static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void* workspace, size_t workspace_bytes,
                                     void* stream, IoTypes io) {
-  const bool cols_ok = io.y_type != kYMXINT8;    // the column-owner kernel's CTAs do not own whole 16-blocks of Y
+  const bool cols_ok = true;
   if (calls == nullptr) return LQER_ERR_NULL;
   if (n_calls < 0) return LQER_ERR_SHAPE;
   // validate everything before the first launch
@@ -819,7 +818,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
         const int set = chain_open ? 1 - chain_set : 0;
         bool fills = false;
         if (launch_decode_cols_group(calls + i, metas, n, workspace, workspace_bytes, chain_open ? kChainLater : kChainFirst,
-                                     set, &fills, ahead ? pres : nullptr, io.x_type, io.y_bf16(), cs) != cudaSuccess)
+                                     set, &fills, ahead ? pres : nullptr, io.x_type, io.y_type, cs) != cudaSuccess)
           return LQER_ERR_CUDA;
         chain_open = fills;
         chain_set = set;

@@ -516,7 +516,7 @@ struct SmallGemmLayer {
 };
 int gemm_small_max_layers();
 cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, DeviceStatus* st, cudaStream_t s);
-cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, int y_type,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);
 // Up to decode_cols_max_group() independent layers with one M (all fitting decode_cols_fits, N >= 32) in one launch.
@@ -527,7 +527,7 @@ bool decode_cols_fits(const PackedMeta& m, int M);
 int decode_cols_max_group();
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
                                      size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
-                                     int x_type, bool y_bf16, cudaStream_t s);
+                                     int x_type, int y_type, cudaStream_t s);
 // The quantised activations and T_q of up to decode_pre_max_calls() independent decode calls, computed ahead (one CTA
 // per call) into outs[i] (decode_pre_bytes each, 256-byte aligned); launch_decode_cols_group takes them as `pres` and
 // then has no X to quantise, no T to compute and nothing to exchange.  `order` as above.

@@ -55,7 +55,7 @@ constexpr int kMaxGroup = 16;  // independent layers with one M that may share a
 
 struct Layer {
   const void* X;                // [M, K] of Params::x_type
-  void* Y;                      // [M, N] fp32, or bf16 where Params::y_bf16
+  void* Y;                      // [M, N] of Params::y_type (MXINT8: mantissas [M, N], then exponent bytes [M, N / 16])
   size_t y_extent;              // bytes behind Y, for the checked build
   const uint8_t* packed;
   size_t off_w, off_b, off_a;   // sections of the packed buffer
@@ -77,7 +77,7 @@ struct Params {
   DeviceStatus* status;
   int M;
   int a_bits, lr_bits, exp_min, exp_max;
-  int x_type, y_bf16;           // X: kXF32, kXBF16 or kXMXINT8; Y: bf16, else fp32
+  int x_type, y_type;           // X: kXF32, kXBF16 or kXMXINT8; Y: kYF32, kYBF16 or kYMXINT8
   int w_bits;                   // mantissa bits of W_q: 4 (nibbles) or 2 (crumbs), one value for all layers of a launch
   long long wait_limit;         // bound of the wait for the other CTAs' partial sums, in clock cycles
 };
@@ -310,7 +310,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const uint8_t* const wsec = ly.packed + ly.off_w;
   const uint8_t* const bsec = ly.packed + ly.off_b;
   const uint8_t* const asec = ly.packed + ly.off_a;
-  const int cg_lo = cta * ly.n_cg / G, cg_hi = (cta + 1) * ly.n_cg / G;
+  // a CTA's columns: a range of groups of 8; for an MXINT8 Y a range of pairs of groups, so that it owns whole 16-blocks
+  const int cgu = p.y_type == kYMXINT8 ? 2 : 1;
+  const int cg_lo = cgu * (cta * (ly.n_cg / cgu) / G), cg_hi = cgu * ((cta + 1) * (ly.n_cg / cgu) / G);
 
   // This lane's column of a round (the 32 columns from column group cg0 on) and slab j: global -> registers.  Byte
   // offsets into the W section are kept per round (32 bits: the section is far below 4 GB).  Column groups past the
@@ -612,7 +614,41 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 #pragma unroll
     for (int r = 0; r < MT; ++r) red_now[((n_held * kWarps + warp) * 32 + lane) * kMaxM + r] = acc[r];
     __syncthreads();
-    if (tid < 32 * kMaxM) {
+    if (p.y_type == kYMXINT8) {
+      // a warp per token, a lane per column of the round: the two 16-blocks of the round are the two halves of the
+      // warp, their maxima a butterfly over 16 lanes; the CTA's range holds whole blocks (see cg_lo)
+      if (tid < 32 * kMaxM) {
+        const int r = warp, col = lane;
+        if (r < M) {
+#pragma unroll
+          for (int h = 0; h < kHold; ++h) {
+            if (h <= n_held) {
+              int c0 = cg0;
+#pragma unroll
+              for (int q = 0; q < kHold - 1; ++q)
+                if (q == h && h < n_held) c0 = held_cg0[q];
+              const bool live = c0 + (col >> 3) < cg_hi;
+              float v = 0.f;
+              if (live) {
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) v += red_now[((h * kWarps + w) * 32 + col) * kMaxM + r];
+              }
+              float amax = abs_ignore_nan(v);
+#pragma unroll
+              for (int sft = 1; sft < 16; sft <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, sft));
+              const int e = block_exponent(amax, p.exp_min, p.exp_max);
+              const int q8 = quant_mantissa(v, e, p.a_bits);
+              const size_t idx = (size_t)r * ly.N + c0 * 8 + col;
+              uint8_t* yq = static_cast<uint8_t*>(Y);
+              if (live && LQER_IN_BOUNDS(p.status, (size_t)M * ly.N + idx / 16, 1, ly.y_extent, 712)) {
+                yq[idx] = (uint8_t)(int8_t)q8;
+                if ((col & 15) == 0) yq[(size_t)M * ly.N + idx / 16] = (uint8_t)(e + 127);
+              }
+            }
+          }
+        }
+      }
+    } else if (tid < 32 * kMaxM) {
       const int col = tid >> 2, r = tid & 3;
 #pragma unroll
       for (int h = 0; h < kHold; ++h) {
@@ -625,8 +661,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
             float v = 0.f;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) v += red_now[((h * kWarps + w) * 32 + col) * kMaxM + r];
-            if (!LQER_IN_BOUNDS(p.status, ((size_t)r * ly.N + c0 * 8 + col) * (p.y_bf16 ? 2 : 4), p.y_bf16 ? 2 : 4, ly.y_extent, 711)) {
-            } else if (p.y_bf16) {
+            const bool y16 = p.y_type == kYBF16;
+            if (!LQER_IN_BOUNDS(p.status, ((size_t)r * ly.N + c0 * 8 + col) * (y16 ? 2 : 4), y16 ? 2 : 4, ly.y_extent, 711)) {
+            } else if (y16) {
               uint32_t u = __float_as_uint(v);               // round to nearest even (NaN / inf keep their class)
               u = ((u & 0x7F800000u) == 0x7F800000u) ? ((u >> 16) | ((u & 0xFFFFu) ? 0x40u : 0u)) : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
               static_cast<uint16_t*>(Y)[(size_t)r * ly.N + c0 * 8 + col] = (uint16_t)u;
@@ -654,10 +691,10 @@ static size_t cols_smem_bytes(const PackedMeta& m, int M) {
 // the whole contraction fits in shared memory.
 bool decode_cols_fits(const PackedMeta& m, int M) { return M <= dcol::kMaxM && cols_smem_bytes(m, M) <= 200 * 1024; }
 
-cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, bool y_bf16,
+cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, int y_type,
                                void* workspace, cudaStream_t s) {
   const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
-  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, nullptr, x_type, y_bf16, s);
+  return launch_decode_cols_group(&one, &m, 1, workspace, 0, kChainAlone, 0, nullptr, nullptr, x_type, y_type, s);
 }
 
 int decode_cols_max_group() { return dcol::kMaxGroup; }
@@ -668,7 +705,7 @@ int decode_cols_max_group() { return dcol::kMaxGroup; }
 // at least one cluster's worth of column groups.
 cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta* metas, int n, void* workspace,
                                      size_t workspace_bytes, int order, int set, bool* fills_gpu, const uint8_t* const* pres,
-                                     int x_type, bool y_bf16, cudaStream_t s) {
+                                     int x_type, int y_type, cudaStream_t s) {
   using namespace dcol;
   static OncePerDevice once;
   static bool one_cta_per_sm = true;               // false if any device could hold two CTAs of the kernel on one SM
@@ -697,7 +734,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   p.a_bits = metas[0].a_bits; p.lr_bits = metas[0].lr_bits; p.exp_min = metas[0].exp_min; p.exp_max = metas[0].exp_max;
   p.x_type = x_type;
   p.w_bits = metas[0].w_bits;
-  p.y_bf16 = y_bf16 ? 1 : 0;
+  p.y_type = y_type;
   p.wait_limit = wait_limit_cycles();
   const int stall = take_stall(kFamDecode) ? 1 : 0;
 
@@ -750,7 +787,7 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
       return cudaErrorInvalidValue;
     Layer& ly = p.L[i];
     ly.X = calls[g].X; ly.Y = calls[g].Y; ly.packed = static_cast<const uint8_t*>(calls[g].packed);
-    ly.y_extent = (size_t)calls[g].M * metas[g].N * (y_bf16 ? 2 : 4);
+    ly.y_extent = y_bytes(y_type, (size_t)calls[g].M, (size_t)metas[g].N);
     if (kDebugBounds) ly.y_extent -= std::min(ly.y_extent, debug_y_shrink());
     ly.off_w = m.off_w; ly.off_b = m.off_b; ly.off_a = m.off_a;
     ly.K = m.K; ly.N = m.N; ly.K64 = m.K64; ly.k_pad = m.k_pad;

@@ -95,8 +95,8 @@ SPECS = [gen.LayerSpec("q_a", M=300, K=1024, N=640, k=40, calib_rows=32, outlier
 
 @pytest.mark.parametrize("spec", SPECS, ids=lambda s: s.name)
 def test_mxint8_output_every_path(spec):
-    # small-batch kernels (1, 4, 9, 70 rows; the chunks of a tile meet in the last arriver's reduction or the tile is
-    # written directly), the pair GEMM without split K (200) and behind either prologue (the spec's own M)
+    # the column-owner decode kernel (1, 4 rows), the small-batch kernels (9, 70 rows; the chunks of a tile meet in the
+    # last arriver's reduction or the tile is written directly), the pair GEMM without split K (200) and behind either prologue (the spec's own M)
     P, Pg = _layer(spec)
     ws = L.new_workspace(spec.M, Pg)
     for M in (1, 4, 9, 70, 200, spec.M):
@@ -108,13 +108,8 @@ def test_mxint8_output_every_path(spec):
         assert L.poll_status(ws) == 0
         Ym, Ye = L.split_mxint8(Yq, M, spec.N)
         _check_against_oracle(Ym.cpu().numpy(), Ye.cpu().numpy(), ref)
-        # the same path with an fp32 Y (M <= 4 takes the small-batch kernels for an MXINT8 Y; M <= 256 would cut K for fp32)
-        if M <= 128:
-            L.set_path(binding.PATH_SMALL)
-        try:
-            Y32 = L.linear(_t(X), Pg, ws).cpu().numpy() if not (128 < M <= 256) else None
-        finally:
-            L.set_path(binding.PATH_AUTO)
+        # the same path with an fp32 Y (for 128 < M <= 256 the fp32 call would cut K, which an MXINT8 Y does not)
+        Y32 = L.linear(_t(X), Pg, ws).cpu().numpy() if not (128 < M <= 256) else None
         if Y32 is not None:
             _check_own_precision(Ym.cpu().numpy(), Ye.cpu().numpy(), Y32)
     Pg.release()
