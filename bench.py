@@ -42,8 +42,8 @@ M_DECODE, M_PREFILL = 1, 2048
 
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # from an ncu capture) per shape, valid only for the kernel sources whose hash is given.
-TRAFFIC = {"sources_sha256": "50984f2c583415ea", "bytes_per_launch": 731.9e6,
-           "note": "640.4 MB measured on one launch of the seven linears of a decoder layer, scaled to the eight linears "
+TRAFFIC = {"sources_sha256": "50984f2c583415ea", "bytes_per_launch": 737.0e6,
+           "note": "644.9 MB measured on one launch of the seven linears of a decoder layer, scaled to the eight linears "
                    "of a bench launch (profiles/gemm_tc2_kernel_7b_layer.md)"}
 DOMINANT_SOURCES = ["paper_2402_02446_b200/csrc/lqer_gemm_tc2.cu", "paper_2402_02446_b200/csrc/lqer_tc_ptx.cuh"]
 
@@ -60,9 +60,9 @@ def sources_hash(sources=None) -> str:
 # grows in proportion to the bytes a launch streams), valid for the sources whose hash is given.
 TRAFFIC_RATIO = {
     "decode": {"sources": ["paper_2402_02446_b200/csrc/lqer_decode_cols.cu", "paper_2402_02446_b200/csrc/lqer_common.cuh"],
-               "sha256": "836139e65421d3ce", "ratio": 254.8 / 250.5, "note": "profiles/decode_cols_kernel_7b_layer.md"},
+               "sha256": "03758cf6c3b093d7", "ratio": 254.6 / 250.5, "note": "profiles/decode_cols_kernel_7b_layer.md"},
     "prologue": {"sources": ["paper_2402_02446_b200/csrc/lqer_prologue_tc.cu", "paper_2402_02446_b200/csrc/lqer_common.cuh"],
-                 "sha256": "6d901cfda86ae781", "ratio": 411.5 / 438.2, "note": "profiles/prologue_tc_kernel_7b_layer.md"},
+                 "sha256": "18c279e7932709df", "ratio": 411.4 / 438.2, "note": "profiles/prologue_tc_kernel_7b_layer.md"},
 }
 
 

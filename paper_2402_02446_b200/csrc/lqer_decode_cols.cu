@@ -281,8 +281,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_pre_kernel(const __grid_co
 }
 
 // MT: rows the accumulators are compiled for (1 for the single-token call, kMaxM otherwise); M <= MT.
-// WB: mantissa bits of W_q the kernel is compiled for: 4 (nibbles) or 2 (crumbs).
-template <int MT, int WB>
+// WB: mantissa bits of W_q the kernel is compiled for: 4 (nibbles) or 2 (crumbs).  YQ: Y is MXINT8.
+template <int MT, int WB, bool YQ>
 __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
   const uint8_t* const bsec = ly.packed + ly.off_b;
   const uint8_t* const asec = ly.packed + ly.off_a;
   // a CTA's columns: a range of groups of 8; for an MXINT8 Y a range of pairs of groups, so that it owns whole 16-blocks
-  const int cgu = p.y_type == kYMXINT8 ? 2 : 1;
+  constexpr int cgu = YQ ? 2 : 1;
   const int cg_lo = cgu * (cta * (ly.n_cg / cgu) / G), cg_hi = cgu * ((cta + 1) * (ly.n_cg / cgu) / G);
 
   // This lane's column of a round (the 32 columns from column group cg0 on) and slab j: global -> registers.  Byte
@@ -614,7 +614,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
 #pragma unroll
     for (int r = 0; r < MT; ++r) red_now[((n_held * kWarps + warp) * 32 + lane) * kMaxM + r] = acc[r];
     __syncthreads();
-    if (p.y_type == kYMXINT8) {
+    if constexpr (YQ) {
       // a warp per token, a lane per column of the round: the two 16-blocks of the round are the two halves of the
       // warp, their maxima a butterfly over 16 lanes; the CTA's range holds whole blocks (see cg_lo)
       if (tid < 32 * kMaxM) {
@@ -711,8 +711,10 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   static bool one_cta_per_sm = true;               // false if any device could hold two CTAs of the kernel on one SM
   cudaError_t e0 = once.run([] {
     // chaining launches relies on one CTA per SM (registers): a launch on every SM then leaves room for no other
-    const void* kernels[4] = {reinterpret_cast<const void*>(decode_cols_kernel<1, 4>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 4>),
-                              reinterpret_cast<const void*>(decode_cols_kernel<1, 2>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 2>)};
+    const void* kernels[8] = {reinterpret_cast<const void*>(decode_cols_kernel<1, 4, false>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 4, false>),
+                              reinterpret_cast<const void*>(decode_cols_kernel<1, 2, false>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 2, false>),
+                              reinterpret_cast<const void*>(decode_cols_kernel<1, 4, true>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 4, true>),
+                              reinterpret_cast<const void*>(decode_cols_kernel<1, 2, true>), reinterpret_cast<const void*>(decode_cols_kernel<kMaxM, 2, true>)};
     for (const void* k : kernels) {
       cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
       if (e != cudaSuccess) return e;
@@ -828,9 +830,13 @@ cudaError_t launch_decode_cols_group(const lqer_call_t* calls, const PackedMeta*
   cfg.numAttrs = 1;
   if (fills_gpu != nullptr) *fills_gpu = one_cta_per_sm && begin == sm_count;
   LaunchScope scope(kFamDecode, s);
-  if (p.w_bits == 2)
-    return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 2>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 2>, p);
-  return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 4>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 4>, p);
+  const bool yq = y_type == kYMXINT8;
+  if (p.w_bits == 2) {
+    if (yq) return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 2, true>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 2, true>, p);
+    return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 2, false>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 2, false>, p);
+  }
+  if (yq) return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 4, true>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 4, true>, p);
+  return M == 1 ? cudaLaunchKernelEx(&cfg, decode_cols_kernel<1, 4, false>, p) : cudaLaunchKernelEx(&cfg, decode_cols_kernel<kMaxM, 4, false>, p);
 }
 
 int decode_pre_max_calls() { return dcol::kPreMaxCalls; }
