@@ -289,3 +289,26 @@ def test_mxint8_input_of_shared_launches_and_host_buffers():
         for X, yh in zip(Xs, Yh):
             assert torch.equal(yh, L.linear(_t(X), Pg, wsh).cpu())
     Pg.release()
+
+
+def test_mxint8_both_ways_with_two_bit_weights():
+    # W2A8 (Section 4.4) with the quantised hand-over on both sides: the decode kernel on crumbs (1 and 3 rows), the
+    # small-batch kernels (40) and the pair GEMM (300)
+    spec = gen.LayerSpec("q_w2", M=300, K=1024, N=640, k=72, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=461)
+    cfg = L.default_config()
+    cfg.w_bits = 2
+    W = gen.make_weight(spec)
+    A, B = gen.make_random_factors(spec)
+    P = olqer.prepare_weights(W, A, B, w_bits=2)
+    Pg = L.prepare_weights(_t(W), _t(A), _t(B), cfg)
+    ws = L.new_workspace(spec.M, Pg)
+    for M in (1, 3, 40, spec.M):
+        X = gen.make_activations(spec, M=M)
+        ref = olqer.forward(X, P, w_bits=2)
+        Xq = _mx_buffer(*mxint.quantize(X, 8, axis=1))
+        Yq = L.linear_ex(Xq, Pg, ws, out_dtype=L.MXINT8, M=M)
+        assert L.poll_status(ws) == 0
+        Ym, Ye = L.split_mxint8(Yq, M, spec.N)
+        _check_against_oracle(Ym.cpu().numpy(), Ye.cpu().numpy(), ref)
+        _check_own_precision(Ym.cpu().numpy(), Ye.cpu().numpy(), L.linear(_t(X), Pg, ws).cpu().numpy())
+    Pg.release()
