@@ -27,7 +27,7 @@ def test_small_parity_cases_pass_under_the_checked_build():
     # every path of the layer on the small specs: prepare, both prologues, both GEMMs, the decode kernels, shared
     # launches, bf16 and MXINT8 boundaries; each test polls the status word, so a bounds report fails it
     r = _run(["-m", "pytest", "-x", "-q", "-m", "gpu",
-              "tests/test_gpu_parity.py", "tests/test_gpu_bf16_io.py", "tests/test_gpu_mxint8_out.py", "tests/test_gpu_w2.py",
+              "tests/test_gpu_parity.py", "tests/test_gpu_bf16_io.py", "tests/test_gpu_mxint8_io.py", "tests/test_gpu_w2.py",
               "-k", "not full and not stack and not sweep and not round"])
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
     assert " passed" in r.stdout

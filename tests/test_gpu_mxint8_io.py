@@ -1,6 +1,6 @@
-"""MXINT8 output (Section 2.1, w&a setting: the activations between layers are quantised; Section 4.1: MXINT8,
-blocks [1,16]): with y_dtype LQER_MXINT8 the epilogue quantises Y in blocks of 16 along N, as the next layer's
-prologue would.
+"""MXINT8 activations at the layer's boundary (Section 2.1, w&a setting: the activations between layers are quantised;
+Section 4.1: MXINT8, blocks [1,16]).  Output: with y_dtype LQER_MXINT8 the epilogue quantises Y in blocks of 16 along N,
+as the next layer's prologue would.  Input (second half of the file): X given in the same layout is taken at its value.
 
 Parity against the oracle.  The oracle quantises its fp64 Y, the library its fp32 Y; the two Y differ by at most the
 layer's tolerance, and a quantised code is a decision taken on that value.  So:
