@@ -529,9 +529,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_cols_kernel(const __grid_c
               nib[2 * i + 1] = (wd[i] >> 4) & 0x0F0F0F0Fu;
             }
           }
-          float sw[4];                                               // 2^(e_w - (w_bits - 2)) of the four blocks
-#pragma unroll
-          for (int b = 0; b < 4; ++b) sw[b] = __uint_as_float((((d.e >> (8 * b)) & 0xFFu) - (uint32_t)(WB - 2)) << 23);
+          // 2^(e_w - (w_bits - 2)) of the four blocks: the four exponent bytes lose the mantissa's binary point at once,
+          // then a byte permute brings a byte to the top of a word and a shift by one puts it into the exponent field
+          float sw[4];
+          const uint32_t e4w = d.e - (uint32_t)(WB - 2) * 0x01010101u;
+          sw[0] = __uint_as_float(__byte_perm(e4w, 0u, 0x0444) >> 1);
+          sw[1] = __uint_as_float(__byte_perm(e4w, 0u, 0x1444) >> 1);
+          sw[2] = __uint_as_float(__byte_perm(e4w, 0u, 0x2444) >> 1);
+          sw[3] = __uint_as_float((e4w >> 1) & 0x7F800000u);
 #pragma unroll
           for (int r = 0; r < MT; ++r) {
             if (r < M) {
