@@ -21,7 +21,7 @@ STATUS_NAMES = ["LQER_OK", "LQER_ERR_NULL", "LQER_ERR_SHAPE", "LQER_ERR_ALIGN", 
                 "LQER_ERR_BUFFER_TOO_SMALL", "LQER_ERR_BAD_PACKED", "LQER_ERR_ARCH", "LQER_ERR_CUDA",
                 "LQER_ERR_TIMEOUT", "LQER_ERR_BOUNDS", "LQER_ERR_STATIC_SCRATCH"]
 
-PATH_AUTO, PATH_SIMT, PATH_DECODE, PATH_TENSOR, PATH_TENSOR_PAIR, PATH_SMALL, PATH_TENSOR_PROLOGUE = 0, 1, 2, 3, 4, 5, 6
+PATH_AUTO, PATH_SIMT, PATH_DECODE, PATH_TENSOR, PATH_TENSOR_PAIR, PATH_SMALL, PATH_TENSOR_PROLOGUE, PATH_SMALL_TMEM = 0, 1, 2, 3, 4, 5, 6, 7
 
 
 class LqerError(RuntimeError):

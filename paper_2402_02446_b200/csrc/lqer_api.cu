@@ -176,7 +176,7 @@ static size_t call_bytes(const PackedMeta& m, int M, bool small) {
 }
 // Whether a call with M rows takes the small-batch kernels under the current path setting.
 static bool takes_small_path(int path, int M) {
-  return (path == 0 || path == 2 || path == 5) && M <= kSmallMaxM;
+  return (path == 0 || path == 2 || path == 5 || path == 7) && M <= kSmallMaxM;
 }
 // The same for a registered packed buffer, on the path lqer_linear_stream takes for M rows right now.
 lqer_status_t call_workspace_bytes(const void* packed, int M, size_t* bytes) {
@@ -219,7 +219,7 @@ static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, 
     gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g]};
   }
   cudaError_t err = launch_prologue_small(pl, n, M, io.x_type, dst, s);
-  if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, dst, s);
+  if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, g_path.load() == 7, dst, s);
   return err;
 }
 
@@ -235,7 +235,7 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   if (st != LQER_OK) return st;
   if (io.y_type == kYMXINT8 && m.N % 16 != 0) return LQER_ERR_SHAPE;     // whole 16-blocks of Y along N
   int path = g_path.load();
-  if ((path == 2 || path == 5) && M > kSmallMaxM) return LQER_ERR_SHAPE;
+  if ((path == 2 || path == 5 || path == 7) && M > kSmallMaxM) return LQER_ERR_SHAPE;
   const bool small = takes_small_path(path, M);
   if (project_only && !small) path = 3;
   // Paths 1 and 3 keep the SIMT-style prologue at every batch size; the others take the tensor-core one where it fits.
@@ -248,7 +248,7 @@ static lqer_status_t run_linear(const void* X, int M, const void* packed, void* 
   void* xcat = wsb + align_up(persist_bytes(m), 256);
   cudaError_t err;
   if (small) {
-    if (path != 5 && !project_only && decode_cols_fits(m, M)) {
+    if (path != 5 && path != 7 && !project_only && decode_cols_fits(m, M)) {
       err = launch_decode_cols(X, io.x_type, M, m, packed, Y, io.y_type, workspace, s);
     } else {
       const lqer_call_t one = {static_cast<const float*>(X), M, packed, static_cast<float*>(Y)};
@@ -747,7 +747,7 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
     lqer_status_t st = lookup(c.packed, m);
     if (st != LQER_OK) return st;
     const int path = g_path.load();
-    if ((path == 2 || path == 5) && c.M > kSmallMaxM) return LQER_ERR_SHAPE;
+    if ((path == 2 || path == 5 || path == 7) && c.M > kSmallMaxM) return LQER_ERR_SHAPE;
     if (io.y_type == kYMXINT8 && m.N % 16 != 0) return LQER_ERR_SHAPE;
     if (workspace_bytes < call_bytes(m, c.M, takes_small_path(path, c.M))) return LQER_ERR_BUFFER_TOO_SMALL;
   }
@@ -1103,7 +1103,7 @@ lqer_status_t lqer_inject_stall(int kernel_family) {
 }
 
 lqer_status_t lqer_set_path(int path) {
-  if (path < 0 || path > 6) return LQER_ERR_CONFIG;
+  if (path < 0 || path > 7) return LQER_ERR_CONFIG;
   g_path.store(path);
   return LQER_OK;
 }

@@ -515,7 +515,10 @@ struct SmallGemmLayer {
   int* counters;              // one zeroed counter per 256-column tile
 };
 int gemm_small_max_layers();
-cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, DeviceStatus* st, cudaStream_t s);
+// tensor_memory_form: keep the tcgen05 kernel also where the register-operand kernel (up to 16 rows, 4-bit weights)
+// would take the launch.
+cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, bool tensor_memory_form, DeviceStatus* st,
+                              cudaStream_t s);
 cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, int y_type,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);

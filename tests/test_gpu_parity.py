@@ -290,11 +290,13 @@ DECODE_SPECS = SMALL_SPECS + MID_SPECS + [
 
 
 @pytest.mark.parametrize("M,path", [(1, binding.PATH_DECODE), (3, binding.PATH_DECODE), (4, binding.PATH_DECODE),
-                                    (1, binding.PATH_SMALL), (5, binding.PATH_DECODE), (16, binding.PATH_DECODE),
+                                    (1, binding.PATH_SMALL), (2, binding.PATH_SMALL), (5, binding.PATH_DECODE),
+                                    (8, binding.PATH_SMALL), (9, binding.PATH_AUTO), (16, binding.PATH_DECODE),
+                                    (1, binding.PATH_SMALL_TMEM), (16, binding.PATH_SMALL_TMEM),
                                     (23, binding.PATH_AUTO), (64, binding.PATH_AUTO), (100, binding.PATH_AUTO),
                                     (128, binding.PATH_AUTO)],
-                         ids=["cols_M1", "cols_M3", "cols_M4", "small_M1", "small_M5", "small_M16", "small_M23", "small_M64",
-                              "small_M100", "small_M128"])
+                         ids=["cols_M1", "cols_M3", "cols_M4", "mma_M1", "mma_M2", "mma_M5", "mma_M8", "mma_M9", "mma_M16",
+                              "small_M1", "small_M16", "small_M23", "small_M64", "small_M100", "small_M128"])
 @pytest.mark.parametrize("spec", DECODE_SPECS, ids=lambda s: s.name)
 def test_linear_decode_kernel(spec, M, path):
     W, A, B, P, Pg = _prepare(spec, "jacobi" if spec.K <= 320 else "subspace")
