@@ -159,8 +159,13 @@ static lqer_status_t check_arch() {
 
 static size_t xcat_bytes(const PackedMeta& m, int M) { return align_up((size_t)M * xcat_cols(m) * 2, 256); }
 // Scratch of one small-batch call behind the head: Xcat, the prologue's partial sums of T, the GEMM's partial sums of Y.
+// The activations of a small-batch call: Xcat, or (register-operand GEMM) the fragment order of 16 rows.
+static size_t small_xcat_bytes(const PackedMeta& m, int M) {
+  const size_t a = xcat_bytes(m, M), b = small_takes_mma(m, M) ? align_up(frag_bytes(m), 256) : 0;
+  return a > b ? a : b;
+}
 static size_t small_slice_bytes(const PackedMeta& m, int M) {
-  return xcat_bytes(m, M) + align_up(prologue_small_slot_bytes(m, M), 256) + align_up(small_gemm_partial_bytes(m, M), 256);
+  return small_xcat_bytes(m, M) + align_up(prologue_small_slot_bytes(m, M), 256) + align_up(small_gemm_partial_bytes(m, M), 256);
 }
 // A call of up to kSmallMaxM rows runs the column-owner decode kernel (M <= 4 where the layer fits it) or the small
 // prologue and the small-batch GEMM; either finds its scratch behind the head.
@@ -212,14 +217,25 @@ static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, 
   for (int g = 0; g < n; ++g) {
     const PackedMeta& m = metas[g];
     uint8_t* xcat = slices[g];
-    uint8_t* slots = xcat + xcat_bytes(m, M);
+    uint8_t* slots = xcat + small_xcat_bytes(m, M);
     uint8_t* partials = slots + align_up(prologue_small_slot_bytes(m, M), 256);
+    int* flags = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(dst) + kFlagAreaOffset) + 2 * g;
     pl[g] = SmallPrologueLayer{calls[g].X, calls[g].packed, &metas[g], xcat, reinterpret_cast<double*>(slots), row_counts[g],
-                               n == 1 ? Tm : nullptr, n == 1 ? Te : nullptr};
-    gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g]};
+                               n == 1 ? Tm : nullptr, n == 1 ? Te : nullptr, flags};
+    gl[g] = SmallGemmLayer{xcat, calls[g].packed, &metas[g], calls[g].Y, reinterpret_cast<float*>(partials), tile_counts[g], flags};
   }
-  cudaError_t err = launch_prologue_small(pl, n, M, io.x_type, dst, s);
-  if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, g_path.load() == 7, dst, s);
+  // a number for the flags of this pair of launches that no earlier pair on any workspace used (never zero)
+  static std::atomic<unsigned> epochs{0};
+  const int epoch = (int)(epochs.fetch_add(1) & 0x3FFFFFFFu) + 1;
+  // the register-operand GEMM reads the activations in fragment order and follows the prologue's flags
+  // (a call on its own is a chain of latencies that the tensor-memory kernel gets through sooner: measured 23.6 against
+  // 26.6 us on a 4096 x 4096 layer; the register-operand kernel serves launches that several layers share, and single
+  // calls where a small-batch path is forced)
+  const int path = g_path.load();
+  const bool tmem_form = path == 7 || (path == 0 && n == 1);
+  const bool frag = !project_only && !tmem_form && small_takes_mma(metas[0], M);
+  cudaError_t err = launch_prologue_small(pl, n, M, io.x_type, frag, epoch, dst, s);
+  if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, tmem_form, epoch, dst, s);
   return err;
 }
 

@@ -496,14 +496,30 @@ struct SmallPrologueLayer {
   const void* X;
   const void* packed;
   const PackedMeta* meta;
-  void* xcat;                 // bf16 [M, K64 + k_pad]
+  void* xcat;                 // bf16 [M, K64 + k_pad], or the fragment order below
   double* slots;              // prologue_small_slot_bytes of scratch
-  int* counts;                // one zeroed counter per group of 16 rows
+  int* counts;                // one zeroed counter per group of 16 rows (eight ints; in fragment order counts[kCountXq] too)
   int8_t* Tm;                 // optional exports of T_q (may be null)
   uint8_t* Te;
+  int* flags;                 // fragment order: the layer's two flags (below)
 };
 int prologue_small_max_layers();
-cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, int x_type, DeviceStatus* st, cudaStream_t s);
+// Fragment order of [X_q | T_q] for up to 16 rows, as the register-operand GEMM reads it (frag_order = true; M <= 16):
+// eight planes q of [slab][256 bytes], a slab being 64 columns of X_q (k_slabs of them) or 64 rank indices of T_q
+// (frag_rank_slabs of them, zero beyond k_pad).  The element of row r at column c of slab s lies in plane
+// q = (c % 32) / 4 at byte  s * 256 + (2 (r % 8) + c / 32) * 16 + ((c % 4) / 2 * 2 + r / 8) * 4 + (c % 2) * 2:
+// 16 bytes = the four registers of one mma.sync A fragment.  Rows beyond M are written as zeros.  The prologue also
+// raises two flags for the GEMM that follows it (`flags`, two ints of the layer in the workspace's status area from
+// kFlagAreaOffset on, used by nothing else): flags[0] takes the launch's `epoch` once every CTA's share of X_q is in
+// place (the CTAs count themselves in at counts[kCountXq]; the last one sets it back to zero), flags[1] once T_q is.
+// An epoch is a number that no earlier launch on this workspace used, so a flag left by the call before never
+// passes for this call's, and the flags need no reset.
+constexpr int kCountXq = 1;
+constexpr int kFlagAreaOffset = 64;                 // status area bytes [64, 64 + 16 layers * 8)
+inline int frag_rank_slabs(const PackedMeta& m) { return (m.k_pad + 63) / 64; }
+inline size_t frag_bytes(const PackedMeta& m) { return (size_t)8 * (m.k_slabs + frag_rank_slabs(m)) * 256; }
+cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, int x_type, bool frag_order, int epoch,
+                                  DeviceStatus* st, cudaStream_t s);
 // The small-batch GEMM (tokens on the M side of a 64- or 128-row MMA, 256 weight columns on its N side); up to
 // gemm_small_max_layers() layers with one M per launch.
 struct SmallGemmLayer {
@@ -513,12 +529,16 @@ struct SmallGemmLayer {
   void* Y;                    // [M, N] fp32 or bf16, or the MXINT8 pair of sections
   float* partials;            // small_gemm_partial_bytes of scratch (unused if the tiles have one chunk)
   int* counters;              // one zeroed counter per 256-column tile
+  int* flags;                 // register-operand kernel: the layer's two flags, as the small prologue raises them
 };
+// Whether a small-batch call of M rows on these weights takes the register-operand GEMM (and with it the fragment order
+// of the activations) unless the tensor-memory kernel is forced.
+inline bool small_takes_mma(const PackedMeta& m, int M) { return M <= 16 && m.w_bits == 4; }
 int gemm_small_max_layers();
 // tensor_memory_form: keep the tcgen05 kernel also where the register-operand kernel (up to 16 rows, 4-bit weights)
 // would take the launch.
-cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, bool tensor_memory_form, DeviceStatus* st,
-                              cudaStream_t s);
+cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, bool tensor_memory_form, int epoch,
+                              DeviceStatus* st, cudaStream_t s);
 cudaError_t launch_decode_cols(const void* X, int x_type, int M, const PackedMeta& m, const void* packed, void* Y, int y_type,
                                void* workspace, cudaStream_t s);
 bool decode_cols_fits(const PackedMeta& m, int M);

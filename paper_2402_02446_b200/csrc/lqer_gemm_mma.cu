@@ -14,15 +14,25 @@
 //     [128 j + 32 t, 128 j + 32 t + 32)
 // of step j - exactly the 16 bytes the packed tile stores contiguously for one column and block pair.  MMA number q
 // (0..7) of the step takes the lane's K 4 q .. 4 q + 3: two bf16 pairs, the halves of a converted nibble word.  The
-// activations are laid out to match when a sub-chunk of Xcat (up to 2048 K) is copied into shared memory: a record of
-// 512 bytes holds, for lane l, the A fragment of one MMA in register order - token rows l / 4 and l / 4 + 8 (zeros
-// beyond the batch) at the lane's K 4 q, 4 q + 1, then at 4 q + 2, 4 q + 3 - so one conflict-free 16-byte load per lane
-// lands in the four consecutive registers the instruction wants and serves four column octets.
+// activations arrive in that order already: the small prologue writes [X_q | T_q] of its (up to) 16 rows as eight
+// planes of [slab][256 bytes], 16 bytes per (row pair, block pair) = the A fragment of one MMA in register order (token
+// rows l / 4 and l / 4 + 8 at the lane's K 4 q, 4 q + 1, then at 4 q + 2, 4 q + 3), so a sub-chunk of 16 slabs is
+// eight bulk copies into shared memory, a lane's fragment is one conflict-free 16-byte load that lands in the four
+// consecutive registers the instruction wants, and it serves four column octets.
 //
 // Work items are those of the tcgen05 form: (layer, 256-column tile, K chunk), chunks fixed by the shapes of the
 // launch; a chunk's partial goes to scratch and the CTA whose partial arrives last adds the chunks in chunk order.
-// A CTA has eight warps of 32 columns each; two CTAs share an SM, so that one streams while the other copies
-// activations or adds up.  Nothing waits for another CTA, and there is no spin in this kernel.
+// A CTA has eight warps of 32 columns each; two CTAs share an SM.  The activations of the next sub-chunk are copied
+// while the current one is multiplied (two buffers, one mbarrier each).
+//
+// The kernel does not wait for the prologue as a whole.  The prologue raises a flag per layer when X_q is in place
+// and another when T_q is (which takes it several times longer); an item waits for the first before its first copy and
+// for the second before the rank term, its last sub-chunk, so the weight stream runs while T is still being formed.
+// Both waits are bounded polls of one thread.  The prologue was launched before this kernel and all its CTAs are
+// resident or done by the time this one starts (the launch order of programmatic dependent launches), so it never
+// depends on this kernel's progress.  The flags are raised only after the prologue's own wait for the kernels before
+// it, so whatever this kernel writes after seeing a flag cannot collide with them.  A flag holds the launch's epoch, a
+// number no earlier launch on the workspace used: the flag the call before left behind never passes for this call's.
 #include "lqer_gemm_small.cuh"
 #include "lqer_tc_ptx.cuh"
 
@@ -31,13 +41,13 @@ namespace mg {
 using namespace sg;
 
 constexpr int THREADS = 256;
-constexpr int WARPS = THREADS / 32;
-constexpr int SUB_SLABS = 32;                       // slabs of 64 K whose activations are in shared memory at a time
-constexpr int STEP_BYTES = 8 * 512;                 // a step's eight records: the A fragments of its eight MMAs
-constexpr int X_BYTES = (SUB_SLABS / 2) * STEP_BYTES;                // 64 KB
-constexpr int SMEM_BYTES = X_BYTES + 16;
+constexpr int SUB_SLABS = 16;                       // slabs of 64 K per activation buffer
+constexpr int PLANE_BYTES = SUB_SLABS * 256;        // a buffer's share of one of the eight planes
+constexpr int BUF_BYTES = 8 * PLANE_BYTES;          // 32 KB
+constexpr int OFF_BARS = 2 * BUF_BYTES;
+constexpr int SMEM_BYTES = OFF_BARS + 64;
 constexpr int STAGE_ROW_BYTES = BN * 4 + 32;        // a token row of a finished tile, padded
-static_assert(16 * STAGE_ROW_BYTES <= X_BYTES, "a finished tile is staged in the activation buffer");
+static_assert(16 * STAGE_ROW_BYTES <= BUF_BYTES, "a finished tile is staged in the first activation buffer");
 
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {
   uint4 v;
@@ -118,9 +128,10 @@ __device__ __forceinline__ void compute_w_oct(float (&acc)[4], const WOct& f, co
 }
 
 // One octet's share of a step of the rank term: 128 rank indices, of which the lane takes two 16-blocks of B_q (rb0,
-// rb0 + 1) for its column.  bt: the packed B tile of the warp's 128-column half; nl: the lane's column in it.
+// rb0 + 1) for its column.  bt: the packed B tile of the warp's 128-column half; nl: the lane's column in it; a: the
+// step's eight A fragments.
 __device__ __forceinline__ void compute_r_oct(float (&acc)[4], const uint8_t* bt, int r_blocks, int rb0, int nl, int lr_shift,
-                                              const uint8_t* xs, int lane) {
+                                              const uint4 (&a)[8]) {
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
     const int rb = rb0 + u;
@@ -133,44 +144,9 @@ __device__ __forceinline__ void compute_r_oct(float (&acc)[4], const uint8_t* bt
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int m = 2 * u + h;
-      const uint4 a0 = *reinterpret_cast<const uint4*>(xs + (2 * m) * 512 + lane * 16);
-      const uint4 a1 = *reinterpret_cast<const uint4*>(xs + (2 * m + 1) * 512 + lane * 16);
       const uint4 b = tc::convert_i8x8(h ? w.z : w.x, h ? w.w : w.y, sc);
-      mma_bf16(acc, a0, b.x, b.y);
-      mma_bf16(acc, a1, b.z, b.w);
-    }
-  }
-}
-
-// Columns [c_lo, c_hi) of Xcat (a multiple of 8 each) into the records of shared memory, zeros beyond c_hi and beyond
-// the batch.  A lane reads 8 K of its rows g and g + 8 and writes the A fragments of the two MMAs that take them.
-__device__ __forceinline__ void fill_x(uint8_t* xs, const uint16_t* xcat, int xcat_cols, int M, int c_lo, int c_hi, int warp, int lane) {
-  constexpr int kBatch = 8;                      // loads of this many passes are in flight together (the copy is bound by latency)
-  const int steps = (c_hi - c_lo + 127) / 128;
-  const int g = lane >> 2, t = lane & 3;
-  const uint16_t* r_lo = xcat + (size_t)g * xcat_cols;
-  const uint16_t* r_hi = xcat + (size_t)(g + 8) * xcat_cols;
-  const bool lo_ok = g < M, hi_ok = g + 8 < M;
-  for (int pr0 = warp; pr0 < steps * 4; pr0 += WARPS * kBatch) {
-    uint4 lo[kBatch], hi[kBatch];
-#pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      const int pr = pr0 + u * WARPS;
-      const int col = c_lo + 128 * (pr >> 2) + 32 * t + 8 * (pr & 3);
-      lo[u] = hi[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (pr < steps * 4 && col < c_hi) {
-        if (lo_ok) lo[u] = __ldcg(reinterpret_cast<const uint4*>(r_lo + col));
-        if (hi_ok) hi[u] = __ldcg(reinterpret_cast<const uint4*>(r_hi + col));
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      const int pr = pr0 + u * WARPS;
-      if (pr < steps * 4) {
-        uint8_t* rec = xs + ((pr >> 2) * 8 + 2 * (pr & 3)) * 512 + lane * 16;
-        *reinterpret_cast<uint4*>(rec) = make_uint4(lo[u].x, hi[u].x, lo[u].y, hi[u].y);
-        *reinterpret_cast<uint4*>(rec + 512) = make_uint4(lo[u].z, hi[u].z, lo[u].w, hi[u].w);
-      }
+      mma_bf16(acc, a[2 * m], b.x, b.y);
+      mma_bf16(acc, a[2 * m + 1], b.z, b.w);
     }
   }
 }
@@ -179,26 +155,52 @@ __device__ __forceinline__ void fill_x(uint8_t* xs, const uint16_t* xcat, int xc
 // index, so that the threads which later read one block each meet no bank twice.
 __device__ __forceinline__ int stage_unit(int u) { return (u & ~3) | ((u & 3) ^ ((u >> 3) & 3)); }
 
+// Bounded poll (one thread) until a flag of the prologue holds this call's epoch.
+__device__ __forceinline__ bool poll_flag(const int* flag, int epoch, volatile tc::WaitState* ws) {
+  const long long t0 = clock64();
+  for (;;) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v == epoch) return true;
+    __nanosleep(100);
+    if (ws->abort != 0) return false;
+    if (clock64() - t0 > ws->limit) { ws->abort = 1; return false; }
+  }
+}
+
 __global__ void __launch_bounds__(THREADS, 2)
 gemm_mma_kernel(const __grid_constant__ Params p) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  uint8_t* xs = smem;
-  int* last_flag = reinterpret_cast<int*>(smem + X_BYTES);
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BARS);
+  int* last_flag = reinterpret_cast<int*>(smem + OFF_BARS + 16);
+  volatile tc::WaitState* ws = reinterpret_cast<volatile tc::WaitState*>(smem + OFF_BARS + 32);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
   const int h = warp >> 2;                       // which 128-column packed tile of the 256-column item
   const int nl = 32 * (warp & 3) + g;            // the lane's column of octet 0 in that tile
   const int eb0 = 2 * (t & 1);
+  const uint32_t a_off = (uint32_t)((t >> 1) * 256 + (2 * g + (t & 1)) * 16);   // the lane's fragment within a step of a plane
   const ConvConsts kc = conv_consts();
+  if (tid == 0) {
+    tc::mbar_init(tc::smem_u32(bars), 1);
+    tc::mbar_init(tc::smem_u32(bars + 1), 1);
+    ws->abort = 0;
+    ws->limit = p.wait_limit;
+    tc::fence_barrier_init();
+  }
   tc::pdl_launch_dependents();                   // the next kernel may set up (it waits for this one before it touches memory)
-  bool waited = false;
+  uint32_t copies = 0;                           // activation copies issued so far (the same in every thread): buffer = copies & 1
+  bool ok = true;
 
-  for (int i = blockIdx.x; i < p.num_items; i += gridDim.x) {
+  for (int i = blockIdx.x; i < p.num_items && ok; i += gridDim.x) {
     const Item it = item_of(p, i);
     const Layer& ly = p.L[it.layer];
     const int w_lo = it.s_lo, w_hi = min(it.s_hi, ly.k_slabs);
     const bool has_rank = it.s_hi > ly.k_slabs && ly.r_blocks > 0;
+    const int n_w = (w_hi - w_lo + SUB_SLABS - 1) / SUB_SLABS;
+    const int n_sub = n_w + (has_rank ? 1 : 0);
+    const int r_slabs = (ly.r_blocks + 3) / 4;
     const int nt = 2 * it.tile + h;
     const bool warp_live = nt < ly.n_tiles;
     const uint8_t* tile_row = ly.wsec + (size_t)(warp_live ? nt : 0) * ly.k_slabs * kWTileBytes;
@@ -211,7 +213,6 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) acc[o][q] = 0.f;
 
-    // packed weights depend on no earlier kernel: the first step is requested before the wait for the prologue
     WOct f[4];                                   // the step's weights; an octet's registers are refilled for the next step as soon as it is done
     // The lane's slab of the step that starts at slab s is s + t / 2.  Where that is beyond the chunk (the second half of
     // an odd last step, or the step after the last) the lane reads the chunk's last slab instead: its activations in
@@ -222,46 +223,91 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
       if (!LQER_IN_BOUNDS(p.status, (size_t)(tile_row - ly.wsec) + (size_t)slab * kWTileBytes, kWTileBytes, ly.w_extent, 721)) slab = w_lo;
       return slab;
     };
-    if (warp_live && w_lo < w_hi) {
+    // Sub-chunk n of the item: up to SUB_SLABS slabs of X_q, or (the last one of a tile's last chunk) the slabs of T_q.
+    auto sub_lo = [&](int n) { return n < n_w ? w_lo + n * SUB_SLABS : ly.k_slabs; };
+    auto sub_len = [&](int n) { return n < n_w ? min(SUB_SLABS, w_hi - (w_lo + n * SUB_SLABS)) : r_slabs; };
+    // Thread 0: waits for what sub-chunk n needs of the prologue, then requests its eight planes into buffer `copies & 1`.
+    auto request = [&](int n) {
+      const int want = p.stall != 0 ? ~p.epoch : p.epoch;   // test hook: a value the flags never take
+      if (n == 0 || n >= n_w) {
+        if (!poll_flag(ly.flags + (n < n_w ? 0 : 1), want, ws)) return;
+        asm volatile("fence.proxy.async.global;" ::: "memory");       // what the flag vouches for, before the copies read it
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // this buffer's earlier readers, before the copies overwrite it
+      const int len = sub_len(n);
+      const uint32_t bar = tc::smem_u32(bars + (copies & 1));
+      const uint32_t dst = tc::smem_u32(smem + (copies & 1) * BUF_BYTES);
+      const uint8_t* src = ly.xfrag + (size_t)sub_lo(n) * 256;
+      tc::mbar_expect_tx(bar, 8u * len * 256u);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) tc::bulk_load(dst + q * PLANE_BYTES, src + (size_t)q * ly.plane, len * 256, bar);
+    };
+    // Every thread: an odd sub-chunk ends in half a step; the slab after its last one reads as zeros.
+    auto zero_tail = [&](int n) {
+      const int len = sub_len(n);
+      if ((len & 1) && tid < 128)
+        *reinterpret_cast<uint4*>(smem + (copies & 1) * BUF_BYTES + (tid >> 4) * PLANE_BYTES + len * 256 + (tid & 15) * 16) = make_uint4(0u, 0u, 0u, 0u);
+    };
+
+    __syncthreads();                             // the item before has left both buffers (and the staged tile)
+    if (tid == 0) request(0);
+    zero_tail(0);
+    ++copies;
+    // the first step's weights (after the request, whose fence would otherwise sit behind these loads)
+    if (warp_live) {
       const size_t off = (size_t)slab_of(w_lo) * kWTileBytes;
 #pragma unroll
       for (int o = 0; o < 4; ++o) load_w_oct(f[o], wp + off + o * 128, ep + off + o * 32);
+      if (has_rank) {
+        // the rank term comes last and is short: its weights are asked into L2 now, so that it does not wait for DRAM then
+        const uint8_t* bt = ly.bsec + (size_t)nt * ly.r_blocks * kTileN * 17;
+        if (g < 4)                                 // lane (g, t): the 128-byte line of octet g in rank blocks t, t + 4, ...
+          for (int rb = t; rb < ly.r_blocks; rb += 4)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(bt + ((size_t)rb * kTileN + 32 * (warp & 3) + 8 * g) * 16));
+        if (lane < ly.r_blocks) asm volatile("prefetch.global.L2 [%0];" ::"l"(bt + (size_t)ly.r_blocks * kTileN * 16 + lane * kTileN));
+      }
     }
-    if (!waited) { tc::pdl_wait(); waited = true; }
 
-    for (int sub = w_lo; sub < w_hi; sub += SUB_SLABS) {
-      const int sub_hi = min(sub + SUB_SLABS, w_hi);
-      __syncthreads();                           // the records of the sub-chunk before have been read
-      fill_x(xs, ly.xcat, ly.xcat_cols, p.M, sub * kSlabK, sub_hi * kSlabK, warp, lane);
-      __syncthreads();
+    for (int n = 0; n < n_sub; ++n) {
+      __syncthreads();                           // sub-chunk n - 1 has been read: its buffer is free; zeroed tails are visible
+      if (n + 1 < n_sub) {
+        if (tid == 0) request(n + 1);
+        zero_tail(n + 1);
+        ++copies;
+      }
+      const uint32_t mine = copies - (n + 1 < n_sub ? 2u : 1u);           // the copy that carries sub-chunk n
+      ok = tc::mbar_wait<true>(tc::smem_u32(bars + (mine & 1)), (mine >> 1) & 1, ws);
+      if (__syncthreads_or(ok ? 0 : 1)) { ok = false; break; }
+      const uint8_t* buf = smem + (mine & 1) * BUF_BYTES + a_off;
       if (warp_live) {
+        const int lo = sub_lo(n), len = sub_len(n);
+        if (n < n_w) {
 #pragma unroll 1
-        for (int s = sub; s < sub_hi; s += 2) {
-          const size_t off = (size_t)slab_of(s + 2) * kWTileBytes;
-          const uint8_t* step = xs + ((s - sub) >> 1) * STEP_BYTES + lane * 16;
-          uint4 a[8];                            // the step's A fragments, read once for the four octets
+          for (int j = 0; 2 * j < len; ++j) {
+            const size_t off = (size_t)slab_of(lo + 2 * j + 2) * kWTileBytes;
+            uint4 a[8];                          // the step's A fragments, read once for the four octets
 #pragma unroll
-          for (int q = 0; q < 8; ++q) a[q] = *reinterpret_cast<const uint4*>(step + q * 512);
+            for (int q = 0; q < 8; ++q) a[q] = *reinterpret_cast<const uint4*>(buf + q * PLANE_BYTES + j * 512);
 #pragma unroll
-          for (int o = 0; o < 4; ++o) {
-            compute_w_oct(acc[o], f[o], a, eb0, kc);
-            load_w_oct(f[o], wp + off + o * 128, ep + off + o * 32);
+            for (int o = 0; o < 4; ++o) {
+              compute_w_oct(acc[o], f[o], a, eb0, kc);
+              load_w_oct(f[o], wp + off + o * 128, ep + off + o * 32);
+            }
+          }
+        } else {
+          const uint8_t* bt = ly.bsec + (size_t)nt * ly.r_blocks * kTileN * 17;
+          for (int j = 0; 2 * j < len; ++j) {
+            uint4 a[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) a[q] = *reinterpret_cast<const uint4*>(buf + q * PLANE_BYTES + j * 512);
+#pragma unroll
+            for (int o = 0; o < 4; ++o) compute_r_oct(acc[o], bt, ly.r_blocks, 8 * j + 2 * t, nl + 8 * o, p.lr_shift, a);
           }
         }
       }
     }
-    if (has_rank) {
-      __syncthreads();
-      fill_x(xs, ly.xcat, ly.xcat_cols, p.M, ly.K64, ly.K64 + 16 * ly.r_blocks, warp, lane);
-      __syncthreads();
-      if (warp_live) {
-        const uint8_t* bt = ly.bsec + (size_t)nt * ly.r_blocks * kTileN * 17;
-        for (int j = 0; j * 8 < ly.r_blocks; ++j)
-#pragma unroll
-          for (int o = 0; o < 4; ++o)
-            compute_r_oct(acc[o], bt, ly.r_blocks, 8 * j + 2 * t, nl + 8 * o, p.lr_shift, xs + j * STEP_BYTES, lane);
-      }
-    }
+    if (!ok) break;
+    uint8_t* xs = smem;                          // the first buffer doubles as the staging area of a finished tile
 
     // ------------------------------------------------------------------ the item's result
     // lane (g, t) holds rows g and g + 8 of columns 32 warp + 8 o + 2 t, + 1
@@ -331,6 +377,15 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
               store_y4(ly.Y, idx + 4 * q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]), p.y_type, p.status, ly.y_extent);
         }
       }
+    }
+  }
+  // ------------------------------------------------------------------ leaving
+  __syncthreads();
+  if (tid == 0) {
+    if (!ok || ws->abort != 0) {
+      const long long t0 = clock64();
+      while (clock64() - t0 < 400000) { }          // a copy requested before the give-up lands well within this
+      report_error(p.status, LQER_ERR_TIMEOUT, 720, blockIdx.x);
     }
   }
 }

@@ -417,11 +417,12 @@ static cudaError_t launch_mt(const TensorMaps& tmaps, const Params& p, int ctas,
 
 int gemm_small_max_layers() { return sg::MAX_LAYERS; }
 
-cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, bool tensor_memory_form, DeviceStatus* st, cudaStream_t s) {
+cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, bool tensor_memory_form, int epoch,
+                              DeviceStatus* st, cudaStream_t s) {
   using namespace sg;
   if (n < 1 || n > MAX_LAYERS || M < 1 || M > kSmallMaxM) return cudaErrorInvalidValue;
   // up to 16 tokens on 4-bit weights: the register-operand kernel, unless the caller asks for this file's
-  const bool use_mma = !tensor_memory_form && M <= kMmaMaxM && layers[0].meta->w_bits == 4;
+  const bool use_mma = !tensor_memory_form && small_takes_mma(*layers[0].meta, M);
   EncodeTiledFn enc = use_mma ? nullptr : encode_fn();
   if (enc == nullptr && !use_mma) return cudaErrorNotSupported;
   const int MT = M <= 64 ? 64 : 128;
@@ -439,7 +440,24 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_
   if (sms < 1) return cudaErrorInvalidDevice;
   int total_tiles = 0;
   for (int i = 0; i < n; ++i) total_tiles += small_gemm_col_tiles(*layers[i].meta);
-  const int group_chunks = (2 * 148 + total_tiles - 1) / total_tiles;      // about two work items per SM in all
+  int group_chunks = (2 * 148 + total_tiles - 1) / total_tiles;            // about two work items per SM in all
+  if (use_mma && n > 1) {
+    // The register-operand kernel runs two CTAs per SM, an item each at a time, and an item costs about ten slabs' worth
+    // of time beside its own slabs (activation copy, rank term, partial sums): the cut that makes (rounds of items over
+    // 2 x 148 CTAs) x (slabs per item + 10) smallest, a function of the shapes alone like the rule above.
+    long best = -1;
+    for (int c = 1; c <= 16; ++c) {
+      long items = 0, len = 0;
+      for (int i = 0; i < n; ++i) {
+        const PackedMeta& m = *layers[i].meta;
+        const int ci = std::min(c, small_gemm_chunks(m));
+        items += (long)small_gemm_col_tiles(m) * ci;
+        len = std::max(len, (long)(m.k_slabs + ci - 1) / ci);
+      }
+      const long cost = ((items + 2 * 148 - 1) / (2 * 148)) * (len + 10);
+      if (best < 0 || cost < best) { best = cost; group_chunks = c; }
+    }
+  }
   for (int i = 0; i < MAX_LAYERS; ++i) {
     const SmallGemmLayer& src = layers[i < n ? i : 0];
     const PackedMeta& m = *src.meta;
@@ -457,8 +475,9 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_
     Layer& ly = p.L[i];
     ly.wsec = base + m.off_w;
     ly.bsec = base + m.off_b;
-    ly.xcat = static_cast<const uint16_t*>(src.xcat);
-    ly.xcat_cols = xcat_cols(m);
+    ly.xfrag = static_cast<const uint8_t*>(src.xcat);
+    ly.flags = src.flags;
+    ly.plane = (m.k_slabs + frag_rank_slabs(m)) * 256;
     ly.Y = src.Y;
     ly.y_extent = y_bytes(y_type, (size_t)M, (size_t)m.N);
     if (kDebugBounds) ly.y_extent -= std::min(ly.y_extent, debug_y_shrink());
@@ -486,11 +505,9 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_
   p.x_rows = x_rows;
   p.w_bits = layers[0].meta->w_bits;
   p.wait_limit = wait_limit_cycles();
-  if (use_mma) {
-    p.stall = 0;
-    return launch_gemm_mma(p, s);
-  }
+  p.epoch = epoch;
   p.stall = take_stall(kFamDecode) ? 1 : 0;
+  if (use_mma) return launch_gemm_mma(p, s);
   const int ctas = p.num_items < sms ? p.num_items : sms;
   return MT == 64 ? launch_mt<64, 6>(tmaps, p, ctas, s) : launch_mt<128, 3>(tmaps, p, ctas, s);
 }

@@ -13,13 +13,15 @@ constexpr int MAX_LAYERS = 16;
 struct Layer {
   const uint8_t* wsec;
   const uint8_t* bsec;
-  const uint16_t* xcat;        // [M, xcat_cols] bf16: X_q, then T_q from column K64 on
+  const uint8_t* xfrag;        // register-operand kernel: [X_q | T_q] in fragment order (eight planes of `plane` bytes)
+  const int* flags;            // ... and the prologue's two flags for this layer (X_q in place, T_q in place)
   void* Y;                     // [M, N] fp32 or bf16, or the MXINT8 sections (mantissas [M, N], exponent bytes [M, N / 16])
   float* partials;             // [tile][chunk][M][256] fp32 (tiles with more than one chunk)
   int* counters;               // [tile] arrivals, zero between calls
   size_t y_extent, partial_extent;   // bytes behind Y and behind partials, for the checked build
   size_t w_extent, b_extent;         // bytes of the packed W and B sections
-  int N, K64, n_tiles, k_slabs, r_blocks, xcat_cols;
+  int N, K64, n_tiles, k_slabs, r_blocks;
+  int plane;                   // bytes of a plane
   int spt;                     // K stages per tile: k_slabs + rank stages
   int chunks, chunk_stages;    // K chunks per tile; weight stages per chunk (the last chunk also takes the rank stages)
   int item_begin;              // first item of this layer in the launch's list
@@ -37,6 +39,7 @@ struct Params {
   int w_bits;                  // mantissa bits of W_q: 4 or 2 (one value for all layers of a launch)
   int x_rows;                  // rows of an activation tile that TMA fills: M rounded up to 8 (the rest stay zero)
   long long wait_limit;
+  int epoch;                   // register-operand kernel: the value the prologue's flags take in this call
   int stall;                   // test hook: the producer withholds the last stage of its last item
 };
 

@@ -30,6 +30,7 @@ struct Layer {
   uint16_t* xcat;             // [M, K64 + k_pad] bf16
   double* slots;              // [row group][range][16][k_pad] partial sums of T
   int* counts;                // [row group] arrivals, zero between calls
+  int* flags;                 // fragment order: X_q ready, T_q ready (each takes the launch's epoch)
   int8_t* Tm;                 // optional exports of T_q
   uint8_t* Te;
   size_t xcat_extent, slots_extent;   // bytes behind xcat and slots, for the checked build
@@ -45,7 +46,15 @@ struct Params {
   DeviceStatus* status;
   int x_type;                 // kXF32, kXBF16 or kXMXINT8
   int a_bits, lr_bits, exp_min, exp_max;
+  int frag;                   // Xcat in the fragment order of the register-operand GEMM (M <= 16), with its flags
+  int epoch;                  // value the flags take in this launch
 };
+
+// Byte offset of (row, column c of slab s) in the fragment order; plane: bytes of one plane.
+__device__ __forceinline__ size_t frag_offset(int row, int slab, int c, size_t plane) {
+  return (size_t)((c & 31) >> 2) * plane + (size_t)slab * 256 + (2 * (row & 7) + (c >> 5)) * 16 + (((c & 3) >> 1) * 2 + (row >> 3)) * 4 +
+         (c & 1) * 2;
+}
 
 // TPW: rank tiles (8 columns) a warp owns: 1 for ranks up to 64, 2 up to 128, 4 up to 256.
 template <int TPW>
@@ -73,6 +82,7 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
   const int NT = k_pad / 8;                              // 8-column rank tiles
   const int WPN = NT >= kWarps ? 1 : kWarps / NT;        // warps that share one rank tile (they split the blocks)
   const bool has_rank = ly.k > 0;
+  const size_t plane = (size_t)(ly.K64 / 64 + (k_pad + 63) / 64) * 256;      // fragment order: bytes of one plane
   const bool active = has_rank && (NT >= kWarps || warp < NT * WPN);
   const int bias = -127 - (p.a_bits - 2) - (p.lr_bits - 2);   // exponent bytes carry +127
 
@@ -127,12 +137,27 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
         if (live) {
           *reinterpret_cast<uint32_t*>(&s_xq[r * kXqStride + c4 * 4]) = m8;
           if ((c4 & 3) == 0) s_xe[r][c4 >> 2] = (int8_t)e;
-          if (row < M && LQER_IN_BOUNDS(p.status, ((size_t)row * ldx + col) * 2, 8, ly.xcat_extent, 311))
+          if (p.frag) {
+            // four consecutive K of a row: the two pairs of one A fragment, 8 bytes apart (rows beyond M are zeros)
+            const size_t o = frag_offset(r, col >> 6, col & 63, plane);
+            if (LQER_IN_BOUNDS(p.status, o, 12, ly.xcat_extent, 311)) {
+              uint8_t* dst = reinterpret_cast<uint8_t*>(ly.xcat) + o;
+              *reinterpret_cast<uint32_t*>(dst) = bf.x;
+              *reinterpret_cast<uint32_t*>(dst + 8) = bf.y;
+            }
+          } else if (row < M && LQER_IN_BOUNDS(p.status, ((size_t)row * ldx + col) * 2, 8, ly.xcat_extent, 311))
             *reinterpret_cast<uint2*>(ly.xcat + (size_t)row * ldx + col) = bf;
         }
       }
     }
+    const bool last_step = kb0 + kStepCols / 16 >= kb_hi;
+    if (p.frag && last_step) __threadfence();          // this CTA's share of X_q before its arrival
     __syncthreads();
+    if (p.frag && last_step && tid == 0 && atomicAdd(ly.counts + kCountXq, 1) == ly.ranges - 1) {
+      ly.counts[kCountXq] = 0;                         // zero again for the next call
+      __threadfence();                                 // every CTA's share before the flag
+      atomicExch(ly.flags, p.epoch);
+    }
     // ---- partial T over these blocks (blocks beyond K are padding: zero mantissas, no A_q rows)
     if (active) {
       const int b_first = NT >= kWarps ? 0 : warp / NT;
@@ -234,11 +259,28 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
     const int e = block_exponent(amax, p.exp_min, p.exp_max);
     const int q = quant_mantissa(t, e, p.a_bits);
     const int row = row0 + r;
-    if (row < M && LQER_IN_BOUNDS(p.status, ((size_t)row * ldx + ly.K64 + j) * 2, 2, ly.xcat_extent, 313)) {
-      ly.xcat[(size_t)row * ldx + ly.K64 + j] = (uint16_t)bf16_bits_of(q, e - (p.a_bits - 2));
+    if (p.frag) {
+      const size_t off = frag_offset(r, ly.K64 / 64 + (j >> 6), j & 63, plane);
+      if (LQER_IN_BOUNDS(p.status, off, 2, ly.xcat_extent, 313))
+        *reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(ly.xcat) + off) = row < M ? (uint16_t)bf16_bits_of(q, e - (p.a_bits - 2)) : (uint16_t)0;
+    }
+    if (row < M && (p.frag || LQER_IN_BOUNDS(p.status, ((size_t)row * ldx + ly.K64 + j) * 2, 2, ly.xcat_extent, 313))) {
+      if (!p.frag) ly.xcat[(size_t)row * ldx + ly.K64 + j] = (uint16_t)bf16_bits_of(q, e - (p.a_bits - 2));
       if (ly.Tm != nullptr) ly.Tm[(size_t)row * k_pad + j] = (int8_t)q;
       if (ly.Te != nullptr && (j & 15) == 0) ly.Te[(size_t)row * (k_pad / 16) + (j >> 4)] = (uint8_t)(e + 127);
     }
+  }
+  if (p.frag) {
+    // rank indices between k_pad and the end of the last rank slab: zeros (the GEMM multiplies them with zero weights)
+    const int pad = ((k_pad + 63) / 64) * 64 - k_pad;
+    for (int o = tid; o < kRows * pad; o += kThreads) {
+      const int r = o / pad, j = k_pad + o % pad;
+      const size_t off = frag_offset(r, ly.K64 / 64 + (j >> 6), j & 63, plane);
+      if (LQER_IN_BOUNDS(p.status, off, 2, ly.xcat_extent, 314)) *reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(ly.xcat) + off) = 0;
+    }
+    __threadfence();                                 // T_q before its flag
+    __syncthreads();
+    if (tid == 0) atomicExch(ly.flags + 1, p.epoch);
   }
   if (tid == 0) ly.counts[rgroup] = 0;               // zero again for the next call
 }
@@ -247,10 +289,13 @@ __global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_c
 
 int prologue_small_max_layers() { return psm::kMaxLayers; }
 
-cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, int x_type, DeviceStatus* st, cudaStream_t s) {
+cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, int x_type, bool frag_order, int epoch,
+                                  DeviceStatus* st, cudaStream_t s) {
   using namespace psm;
-  if (n < 1 || n > kMaxLayers || M < 1) return cudaErrorInvalidValue;
+  if (n < 1 || n > kMaxLayers || M < 1 || (frag_order && M > 16)) return cudaErrorInvalidValue;
   Params p;
+  p.frag = frag_order ? 1 : 0;
+  p.epoch = epoch;
   p.n = n;
   p.M = M;
   p.x_type = x_type;
@@ -269,9 +314,10 @@ cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M
     ly.asec = static_cast<const uint8_t*>(src.packed) + m.off_a;
     ly.xcat = static_cast<uint16_t*>(src.xcat);
     ly.slots = src.slots;
-    ly.xcat_extent = (size_t)M * xcat_cols(m) * 2;
+    ly.xcat_extent = frag_order ? frag_bytes(m) : (size_t)M * xcat_cols(m) * 2;
     ly.slots_extent = prologue_small_slot_bytes(m, M);
     ly.counts = src.counts;
+    ly.flags = src.flags;
     ly.Tm = src.Tm; ly.Te = src.Te;
     ly.K = m.K; ly.K64 = m.K64; ly.k = m.k; ly.k_pad = m.k_pad;
     ly.ranges = prologue_small_ranges(m, M);

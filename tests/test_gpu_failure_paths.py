@@ -37,7 +37,8 @@ def _layer(spec):
 CASES = [
     # (name, family, forced path, M, K, N, k)
     ("decode_cols_T_exchange", FAM_DECODE, binding.PATH_AUTO, 2, 2112, 264, 72),   # 132 K blocks x 3 rank tiles: T is exchanged
-    ("small_gemm_ring", FAM_DECODE, binding.PATH_AUTO, 40, 1024, 640, 40),
+    ("small_gemm_ring", FAM_DECODE, binding.PATH_AUTO, 9, 1024, 640, 40),
+    ("small_mma_flags", FAM_DECODE, binding.PATH_SMALL, 9, 1024, 640, 40),      # the polls of the prologue's flags
     ("prologue_tc_row_tile", FAM_PROLOGUE, binding.PATH_TENSOR_PROLOGUE, 300, 1024, 640, 32),
     ("gemm_pair_ring", FAM_GEMM, binding.PATH_AUTO, 300, 1024, 640, 40),
 ]

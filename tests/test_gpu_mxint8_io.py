@@ -138,7 +138,7 @@ def test_mxint8_output_of_shared_launches_and_host_buffers():
              gen.LayerSpec("q_g1", M=300, K=1024, N=384, k=32, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=412),
              gen.LayerSpec("q_g2", M=300, K=320, N=512, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=413)]
     layers = [_layer(s) for s in specs]
-    for M in (300, 24, 3):
+    for M in (300, 24, 12, 3):
         Xs = [gen.make_activations(s, M=M) for s in specs]
         refs = [olqer.forward(X, P) for X, (P, _) in zip(Xs, layers)]
         Yq = [torch.zeros(L.mxint8_bytes(M, s.N), dtype=torch.uint8, device=DEV) for s in specs]

@@ -291,7 +291,7 @@ DECODE_SPECS = SMALL_SPECS + MID_SPECS + [
 
 @pytest.mark.parametrize("M,path", [(1, binding.PATH_DECODE), (3, binding.PATH_DECODE), (4, binding.PATH_DECODE),
                                     (1, binding.PATH_SMALL), (2, binding.PATH_SMALL), (5, binding.PATH_DECODE),
-                                    (8, binding.PATH_SMALL), (9, binding.PATH_AUTO), (16, binding.PATH_DECODE),
+                                    (8, binding.PATH_SMALL), (9, binding.PATH_SMALL), (16, binding.PATH_DECODE),
                                     (1, binding.PATH_SMALL_TMEM), (16, binding.PATH_SMALL_TMEM),
                                     (23, binding.PATH_AUTO), (64, binding.PATH_AUTO), (100, binding.PATH_AUTO),
                                     (128, binding.PATH_AUTO)],
@@ -411,7 +411,7 @@ def test_batched_decode_stretch_quantises_activations_ahead(M):
         Pg.release()
 
 
-@pytest.mark.parametrize("M", [5, 16, 40])
+@pytest.mark.parametrize("M", [5, 8, 16, 40])
 def test_batched_small_batches_share_two_launches(M):
     # nine independent calls with one M above the column-owner kernel's range: layers of three shapes (one without a
     # low-rank part) run as ONE launch of the small prologue and ONE launch of the small-batch GEMM over the work items
