@@ -230,9 +230,9 @@ static cudaError_t run_small(const lqer_call_t* calls, const PackedMeta* metas, 
   // the register-operand GEMM reads the activations in fragment order and follows the prologue's flags
   // (a call on its own is a chain of latencies that the tensor-memory kernel gets through sooner: measured 23.6 against
   // 26.6 us on a 4096 x 4096 layer; the register-operand kernel serves launches that several layers share, and single
-  // calls where a small-batch path is forced)
+  // calls where path 5 is forced)
   const int path = g_path.load();
-  const bool tmem_form = path == 7 || (path == 0 && n == 1);
+  const bool tmem_form = path == 7 || ((path == 0 || path == 2) && n == 1);
   const bool frag = !project_only && !tmem_form && small_takes_mma(metas[0], M);
   cudaError_t err = launch_prologue_small(pl, n, M, io.x_type, frag, epoch, dst, s);
   if (err == cudaSuccess && !project_only) err = launch_gemm_small(gl, n, M, io.y_type, tmem_form, epoch, dst, s);
@@ -357,6 +357,18 @@ static lqer_status_t run_small_group(const lqer_call_t* calls, int n, const Pack
   }
   return run_small(calls, metas, n, slices, tile_counts, row_counts, static_cast<DeviceStatus*>(workspace), io, nullptr,
                    nullptr, false, s) == cudaSuccess ? LQER_OK : LQER_ERR_CUDA;
+}
+// Three or four rows in many layers at once: the register-operand GEMM's launches take less per layer than the
+// column-owner kernel's (measured on 4096 x 4096 layers: from 6 layers on at 4 rows, 5.7 against 6.9 us, and from 12 on
+// at 3 rows, 4.4 against 4.6 us; with fewer layers the column-owner kernel's shorter chain wins).  The length of such
+// a run from calls[first] on, or 0.
+static int many_small_rows(const lqer_call_t* calls, int first, int n_calls, size_t workspace_bytes, const PackedMeta& m0,
+                           PackedMeta* metas, size_t* need) {
+  const int M = calls[first].M;
+  if (M < 3 || !decode_cols_fits(m0, M) || !small_takes_mma(m0, M)) return 0;
+  const int lim = std::min(gemm_small_max_layers(), prologue_small_max_layers());
+  const int n = small_run(calls, first, n_calls, lim, workspace_bytes, false, metas, need);
+  return n >= (M == 4 ? 6 : 12) ? n : 0;
 }
 // The run of decode calls from calls[first] on that may share one launch of the column-owner kernel: one M, one set of
 // formats, each fitting the kernel, at least 32 columns, and a slot for each layer's partial sums of T in the workspace.
@@ -787,7 +799,11 @@ static lqer_status_t linear_batched(const lqer_call_t* calls, int n_calls, void*
     PackedMeta m0, metas[16];
     bool decode_group = false, small_group = false;
     if (may_group && lookup(calls[i].packed, m0) == LQER_OK) {
-      if (cols_ok && decode_cols_fits(m0, calls[i].M)) {
+      const int many = cols_ok ? many_small_rows(calls, i, n_calls, workspace_bytes, m0, metas, nullptr) : 0;
+      if (many > 0) {
+        n = many;
+        small_group = true;
+      } else if (cols_ok && decode_cols_fits(m0, calls[i].M)) {
         n = decode_run(calls, i, n_calls, decode_cols_max_group(), workspace_bytes, metas, nullptr);
         if (n < 1) n = 1;
         decode_group = n > 1;
@@ -906,8 +922,14 @@ lqer_status_t lqer_batched_workspace_bytes(const lqer_call_t* calls, int n_calls
     const lqer_call_t& c = calls[i];
     PackedMeta m;
     lookup(c.packed, m);
+    PackedMeta many_metas[16];
+    size_t many_need = 0;
+    const int many = many_small_rows(calls, i, n_calls, ~(size_t)0, m, many_metas, &many_need);
     int n = 1;
-    if (decode_cols_fits(m, c.M)) {
+    if (many > 0) {
+      n = many;
+      need = std::max(need, many_need);
+    } else if (decode_cols_fits(m, c.M)) {
       PackedMeta metas[16];
       size_t group_need = 0, ahead = 0;
       n = decode_run(calls, i, n_calls, decode_cols_max_group(), ~(size_t)0, metas, &group_need);
