@@ -28,6 +28,7 @@ def test_small_parity_cases_pass_under_the_checked_build():
     # launches, bf16 and MXINT8 boundaries; each test polls the status word, so a bounds report fails it
     r = _run(["-m", "pytest", "-x", "-q", "-m", "gpu",
               "tests/test_gpu_parity.py", "tests/test_gpu_bf16_io.py", "tests/test_gpu_mxint8_io.py", "tests/test_gpu_w2.py",
+              "tests/test_gpu_small_mma.py",
               "-k", "not full and not stack and not sweep and not round"])
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
     assert " passed" in r.stdout
@@ -43,12 +44,13 @@ def test_a_short_extent_is_reported_and_nothing_beyond_it_is_written():
         E = binding.STATUS_NAMES.index
         dev = "cuda:0"
         t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
-        for M, path in ((3, binding.PATH_AUTO), (40, binding.PATH_AUTO), (300, binding.PATH_AUTO)):
+        for M, path in ((3, binding.PATH_AUTO), (9, binding.PATH_SMALL), (40, binding.PATH_AUTO), (300, binding.PATH_AUTO)):
             spec = gen.LayerSpec("short", M=M, K=512, N=384, k=16, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=501)
             W = gen.make_weight(spec); A, B = gen.make_random_factors(spec)
             Pg = L.prepare_weights(t(W), t(A), t(B))
             X = t(gen.make_activations(spec))
             ws = L.new_workspace(M, Pg)
+            L.set_path(path)
             Y_good = L.linear(X, Pg, ws).clone()
             assert L.poll_status(ws) == 0
             cut = 4 * 100                                   # the last hundred floats of Y are declared out of range
@@ -65,6 +67,7 @@ def test_a_short_extent_is_reported_and_nothing_beyond_it_is_written():
             assert torch.equal(flat[:-128], good[:-128])    # everything clear of the cut was written as usual
             assert L.lib().lqer_workspace_init(ws.data_ptr(), ws.numel(), None) == 0
             assert torch.equal(L.linear(X, Pg, ws), Y_good) and L.poll_status(ws) == 0
+            L.set_path(binding.PATH_AUTO)
             Pg.release()
         print("checked-build-ok")
     """)
