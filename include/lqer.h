@@ -285,7 +285,7 @@ lqer_status_t lqer_poll_status(const void* workspace, void* stream, lqer_status_
  * (column-owner kernel for M <= 4, small prologue + small-batch GEMM for M <= 128), 3 tensor-core GEMM behind the
  * activation prologue that runs the projection on int8 mma.sync (at every batch size), 4 tensor-core
  * GEMM with the prologue chosen as in 0, 5 small prologue + small-batch GEMM for every M <= 128 (the register-operand
- * kernel up to 16 rows on 4-bit weights - which paths 0 and 2 use only where several calls share its launches - and
+ * kernel up to 16 rows - which paths 0 and 2 use only where several calls share its launches - and
  * the tensor-memory kernel otherwise), 6 as 4 with the
  * tcgen05 activation prologue at every batch size (ranks up to 64; by default it serves M >= 1024,
  * and paths 1 and 3 never use it), 7 as 5 with the tensor-memory kernel at every M <= 128.  Host only, process wide. */

@@ -365,7 +365,7 @@ static lqer_status_t run_small_group(const lqer_call_t* calls, int n, const Pack
 static int many_small_rows(const lqer_call_t* calls, int first, int n_calls, size_t workspace_bytes, const PackedMeta& m0,
                            PackedMeta* metas, size_t* need) {
   const int M = calls[first].M;
-  if (M < 3 || !decode_cols_fits(m0, M) || !small_takes_mma(m0, M)) return 0;
+  if (M < 3 || m0.w_bits != 4 || !decode_cols_fits(m0, M) || !small_takes_mma(m0, M)) return 0;     // measured on 4-bit weights only
   const int lim = std::min(gemm_small_max_layers(), prologue_small_max_layers());
   const int n = small_run(calls, first, n_calls, lim, workspace_bytes, false, metas, need);
   return n >= (M == 4 ? 6 : 12) ? n : 0;

@@ -533,9 +533,9 @@ struct SmallGemmLayer {
 };
 // Whether a small-batch call of M rows on these weights takes the register-operand GEMM (and with it the fragment order
 // of the activations) unless the tensor-memory kernel is forced.
-inline bool small_takes_mma(const PackedMeta& m, int M) { return M <= 16 && m.w_bits == 4; }
+inline bool small_takes_mma(const PackedMeta& m, int M) { return M <= 16 && (m.w_bits == 4 || m.w_bits == 2); }
 int gemm_small_max_layers();
-// tensor_memory_form: keep the tcgen05 kernel also where the register-operand kernel (up to 16 rows, 4-bit weights)
+// tensor_memory_form: keep the tcgen05 kernel also where the register-operand kernel (up to 16 rows)
 // would take the launch.
 cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_type, bool tensor_memory_form, int epoch,
                               DeviceStatus* st, cudaStream_t s);

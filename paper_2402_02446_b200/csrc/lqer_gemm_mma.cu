@@ -4,7 +4,7 @@
 // The tcgen05 form of the small-batch GEMM converts every packed weight tile to bf16 in shared memory (32 KB written
 // and read again per 9 KB of packed weights), and that traffic, not DRAM, sets its pace.  Here the weights never
 // touch shared memory: a lane loads 16 bytes of one column straight from the packed tile into registers, turns its
-// nibbles into the exact bf16 values m * 2^e there (one fma.rn.bf16x2 per pair) and feeds them to
+// nibbles (or crumbs, with 2-bit weights) into the exact bf16 values m * 2^e there (one fma.rn.bf16x2 per pair) and feeds them to
 //     D[16 tokens, 8 columns] += A[16, 16 K] . B[16 K, 8]           (mma.sync m16n8k16, bf16 -> fp32)
 // as the B fragment.  The products are exact and the sums are fp32, as in the tensor-memory kernels.
 //
@@ -82,11 +82,13 @@ __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
   return d;
 }
 struct ConvConsts {
-  uint32_t mask, magic;        // 0x000F000F, 0x43004300
+  uint32_t mask, magic;        // 0x000F000F (nibbles) or 0x00030003 (crumbs), 0x43004300
 };
+template <int WB>
 __device__ __forceinline__ ConvConsts conv_consts() {
   ConvConsts k;
-  asm volatile("mov.b32 %0, 0x000F000F;" : "=r"(k.mask));     // opaque to the compiler, so that they stay in registers
+  if (WB == 4) asm volatile("mov.b32 %0, 0x000F000F;" : "=r"(k.mask));     // opaque to the compiler, so that they stay in registers
+  else asm volatile("mov.b32 %0, 0x00030003;" : "=r"(k.mask));
   asm volatile("mov.b32 %0, 0x43004300;" : "=r"(k.magic));
   return k;
 }
@@ -100,28 +102,58 @@ __device__ __forceinline__ uint4 convert_nibbles(uint32_t w, uint32_t s2, uint32
   o.w = tc::fma_bf16x2(and_or(w >> 12, k.mask, k.magic), s2, c2);
   return o;
 }
+// The 2-bit format (mantissas -1, 0, 1; value m * 2^e): crumbs 4 j .. 4 j + 3 of the low and of the high half of a block
+// word (K 8 j .. 8 j + 7 of the block's sixteen) -> eight bf16, exact: (128 + c) * s - 129 * s rounds nothing away.
+__device__ __forceinline__ uint4 convert_crumbs(uint32_t w, int j, uint32_t s2, uint32_t c2, const ConvConsts& k) {
+  uint4 o;
+  o.x = tc::fma_bf16x2(and_or(w >> (8 * j), k.mask, k.magic), s2, c2);
+  o.y = tc::fma_bf16x2(and_or(w >> (8 * j + 2), k.mask, k.magic), s2, c2);
+  o.z = tc::fma_bf16x2(and_or(w >> (8 * j + 4), k.mask, k.magic), s2, c2);
+  o.w = tc::fma_bf16x2(and_or(w >> (8 * j + 6), k.mask, k.magic), s2, c2);
+  return o;
+}
+// bf16 pairs (2^e, 2^e) and (-129 * 2^e, -129 * 2^e) of an exponent byte of word e4: bits eb << 7 and 0x8000 | (eb + 7) << 7 | 1.
+__device__ __forceinline__ void w_scale_pair2(uint32_t e4, int byte, uint32_t& s2, uint32_t& c2) {
+  const uint32_t eb = __byte_perm(e4, 0u, 0x4440u + byte);
+  s2 = eb * 0x00800080u;
+  c2 = eb * 0x00800080u + 0x83818381u;
+}
 
-// A lane's weights of one step in one column octet: 32 nibbles (one block pair) of its column, and the slab's four
-// exponent bytes of that column.
+// A lane's weights of one step in one column octet: one block pair (32 K) of its column - 16 bytes of nibbles, or 8
+// bytes of crumbs in w.x, w.y - and the slab's four exponent bytes of that column.
 struct WOct {
   uint4 w;
   uint32_t e;
 };
-// wp / ep: the lane's column in the packed tile of the lane's slab (nibbles of its block pair; exponent word).
+// wp / ep: the lane's column in the packed tile of the lane's slab (mantissas of its block pair; exponent word).
+template <int WB>
 __device__ __forceinline__ void load_w_oct(WOct& f, const uint8_t* wp, const uint8_t* ep) {
-  f.w = ld_stream16(wp);
+  if (WB == 4) {
+    f.w = ld_stream16(wp);
+  } else {
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(f.w.x), "=r"(f.w.y) : "l"(wp));
+  }
   f.e = ld_stream4(ep);
 }
 
 // One octet's share of a step of weight slabs: eight MMAs.  a: the step's eight A fragments; eb0: index of the first
 // exponent byte of the lane's block pair in an exponent word.
+template <int WB>
 __device__ __forceinline__ void compute_w_oct(float (&acc)[4], const WOct& f, const uint4 (&a)[8], int eb0, const ConvConsts& k) {
   uint32_t s2, c2;
 #pragma unroll
   for (int m = 0; m < 4; ++m) {
-    if ((m & 1) == 0) w_scale_pair(f.e, eb0 + (m >> 1), s2, c2);
-    const uint32_t word = m == 0 ? f.w.x : m == 1 ? f.w.y : m == 2 ? f.w.z : f.w.w;
-    const uint4 b = convert_nibbles(word, s2, c2, k);
+    if ((m & 1) == 0) {
+      if (WB == 4) w_scale_pair(f.e, eb0 + (m >> 1), s2, c2);
+      else w_scale_pair2(f.e, eb0 + (m >> 1), s2, c2);
+    }
+    uint4 b;
+    if (WB == 4) {
+      const uint32_t word = m == 0 ? f.w.x : m == 1 ? f.w.y : m == 2 ? f.w.z : f.w.w;
+      b = convert_nibbles(word, s2, c2, k);
+    } else {
+      b = convert_crumbs(m < 2 ? f.w.x : f.w.y, m & 1, s2, c2, k);
+    }
     mma_bf16(acc, a[2 * m], b.x, b.y);
     mma_bf16(acc, a[2 * m + 1], b.z, b.w);
   }
@@ -168,8 +200,11 @@ __device__ __forceinline__ bool poll_flag(const int* flag, int epoch, volatile t
   }
 }
 
+template <int WB>
 __global__ void __launch_bounds__(THREADS, 2)
 gemm_mma_kernel(const __grid_constant__ Params p) {
+  constexpr int kTile = WB == 4 ? kWTileBytes : 2048 + kTileN * 4;   // bytes of a packed weight tile
+  constexpr int kMant = WB == 4 ? kWTileNibbleBytes : 2048;          // of which mantissas
   extern __shared__ __align__(128) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BARS);
   int* last_flag = reinterpret_cast<int*>(smem + OFF_BARS + 16);
@@ -181,7 +216,7 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
   const int nl = 32 * (warp & 3) + g;            // the lane's column of octet 0 in that tile
   const int eb0 = 2 * (t & 1);
   const uint32_t a_off = (uint32_t)((t >> 1) * 256 + (2 * g + (t & 1)) * 16);   // the lane's fragment within a step of a plane
-  const ConvConsts kc = conv_consts();
+  const ConvConsts kc = conv_consts<WB>();
   if (tid == 0) {
     tc::mbar_init(tc::smem_u32(bars), 1);
     tc::mbar_init(tc::smem_u32(bars + 1), 1);
@@ -203,9 +238,9 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
     const int r_slabs = (ly.r_blocks + 3) / 4;
     const int nt = 2 * it.tile + h;
     const bool warp_live = nt < ly.n_tiles;
-    const uint8_t* tile_row = ly.wsec + (size_t)(warp_live ? nt : 0) * ly.k_slabs * kWTileBytes;
-    const uint8_t* wp = tile_row + (t & 1) * 2048 + nl * 16;
-    const uint8_t* ep = tile_row + kWTileNibbleBytes + nl * 4;
+    const uint8_t* tile_row = ly.wsec + (size_t)(warp_live ? nt : 0) * ly.k_slabs * kTile;
+    const uint8_t* wp = WB == 4 ? tile_row + (t & 1) * 2048 + nl * 16 : tile_row + nl * 16 + (t & 1) * 8;
+    const uint8_t* ep = tile_row + kMant + nl * 4;
 
     float acc[4][4];
 #pragma unroll
@@ -220,7 +255,7 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
     // In the checked build a slab beyond the buffer is reported and slab w_lo read in its place.
     auto slab_of = [&](int s) {
       int slab = min(s + (t >> 1), w_hi - 1);
-      if (!LQER_IN_BOUNDS(p.status, (size_t)(tile_row - ly.wsec) + (size_t)slab * kWTileBytes, kWTileBytes, ly.w_extent, 721)) slab = w_lo;
+      if (!LQER_IN_BOUNDS(p.status, (size_t)(tile_row - ly.wsec) + (size_t)slab * kTile, kTile, ly.w_extent, 721)) slab = w_lo;
       return slab;
     };
     // Sub-chunk n of the item: up to SUB_SLABS slabs of X_q, or (the last one of a tile's last chunk) the slabs of T_q.
@@ -255,9 +290,9 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
     ++copies;
     // the first step's weights (after the request, whose fence would otherwise sit behind these loads)
     if (warp_live) {
-      const size_t off = (size_t)slab_of(w_lo) * kWTileBytes;
+      const size_t off = (size_t)slab_of(w_lo) * kTile;
 #pragma unroll
-      for (int o = 0; o < 4; ++o) load_w_oct(f[o], wp + off + o * 128, ep + off + o * 32);
+      for (int o = 0; o < 4; ++o) load_w_oct<WB>(f[o], wp + off + o * 128, ep + off + o * 32);
       if (has_rank) {
         // the rank term comes last and is short: its weights are asked into L2 now, so that it does not wait for DRAM then
         const uint8_t* bt = ly.bsec + (size_t)nt * ly.r_blocks * kTileN * 17;
@@ -284,14 +319,14 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
         if (n < n_w) {
 #pragma unroll 1
           for (int j = 0; 2 * j < len; ++j) {
-            const size_t off = (size_t)slab_of(lo + 2 * j + 2) * kWTileBytes;
+            const size_t off = (size_t)slab_of(lo + 2 * j + 2) * kTile;
             uint4 a[8];                          // the step's A fragments, read once for the four octets
 #pragma unroll
             for (int q = 0; q < 8; ++q) a[q] = *reinterpret_cast<const uint4*>(buf + q * PLANE_BYTES + j * 512);
 #pragma unroll
             for (int o = 0; o < 4; ++o) {
-              compute_w_oct(acc[o], f[o], a, eb0, kc);
-              load_w_oct(f[o], wp + off + o * 128, ep + off + o * 32);
+              compute_w_oct<WB>(acc[o], f[o], a, eb0, kc);
+              load_w_oct<WB>(f[o], wp + off + o * 128, ep + off + o * 32);
             }
           }
         } else {
@@ -390,10 +425,11 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
   }
 }
 
+template <int WB>
 static cudaError_t launch(const Params& p, int ctas, cudaStream_t s) {
   static OncePerDevice once;
   cudaError_t e = once.run([] {
-    return cudaFuncSetAttribute(gemm_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    return cudaFuncSetAttribute(gemm_mma_kernel<WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   });
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -407,17 +443,17 @@ static cudaError_t launch(const Params& p, int ctas, cudaStream_t s) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   LaunchScope scope(kFamDecode, s);
-  return cudaLaunchKernelEx(&cfg, gemm_mma_kernel, p);
+  return cudaLaunchKernelEx(&cfg, gemm_mma_kernel<WB>, p);
 }
 
 }  // namespace mg
 
 cudaError_t launch_gemm_mma(const sg::Params& p, cudaStream_t s) {
-  if (p.M < 1 || p.M > kMmaMaxM || p.w_bits != 4) return cudaErrorInvalidValue;
+  if (p.M < 1 || p.M > kMmaMaxM || (p.w_bits != 4 && p.w_bits != 2)) return cudaErrorInvalidValue;
   const int sms = sm_count();
   if (sms < 1) return cudaErrorInvalidDevice;
   const int ctas = p.num_items < 2 * sms ? p.num_items : 2 * sms;
-  return mg::launch(p, ctas, s);
+  return p.w_bits == 4 ? mg::launch<4>(p, ctas, s) : mg::launch<2>(p, ctas, s);
 }
 
 }  // namespace lqer

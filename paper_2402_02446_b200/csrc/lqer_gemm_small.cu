@@ -421,7 +421,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_
                               DeviceStatus* st, cudaStream_t s) {
   using namespace sg;
   if (n < 1 || n > MAX_LAYERS || M < 1 || M > kSmallMaxM) return cudaErrorInvalidValue;
-  // up to 16 tokens on 4-bit weights: the register-operand kernel, unless the caller asks for this file's
+  // up to 16 tokens: the register-operand kernel, unless the caller asks for this file's
   const bool use_mma = !tensor_memory_form && small_takes_mma(*layers[0].meta, M);
   EncodeTiledFn enc = use_mma ? nullptr : encode_fn();
   if (enc == nullptr && !use_mma) return cudaErrorNotSupported;

@@ -129,7 +129,7 @@ __device__ __forceinline__ void reduce_tile(const Params& p, const Layer& ly, in
 
 }  // namespace sg
 
-// The register-operand form of the small-batch GEMM for up to kMmaMaxM tokens and 4-bit weights (lqer_gemm_mma.cu).
+// The register-operand form of the small-batch GEMM for up to kMmaMaxM tokens (lqer_gemm_mma.cu).
 constexpr int kMmaMaxM = 16;
 cudaError_t launch_gemm_mma(const sg::Params& p, cudaStream_t s);
 

@@ -61,9 +61,10 @@ def test_two_bit_weights_pack_and_layer(spec, ratio_log):
     if spec.k:
         assert np.array_equal(ex["Bm"].cpu().numpy(), P.Bm) and np.array_equal(ex["Am"].cpu().numpy(), P.Am)
     ws = L.new_workspace(spec.M, Pg)
-    # every path: the checking kernel, the small-batch kernels (1 .. 100 rows), the large-batch GEMM with either prologue
+    # every path: the checking kernel, the small-batch kernels (1 .. 100 rows; path 5 at up to 16 rows: the register-operand
+    # GEMM on crumbs), the large-batch GEMM with either prologue
     for M, path in ((spec.M, binding.PATH_SIMT), (1, binding.PATH_AUTO), (4, binding.PATH_AUTO), (9, binding.PATH_AUTO),
-                    (100, binding.PATH_AUTO), (spec.M, binding.PATH_TENSOR), (spec.M, binding.PATH_TENSOR_PAIR),
+                    (9, binding.PATH_SMALL), (16, binding.PATH_SMALL), (100, binding.PATH_AUTO), (spec.M, binding.PATH_TENSOR), (spec.M, binding.PATH_TENSOR_PAIR),
                     (spec.M, binding.PATH_AUTO)):
         if M > spec.M:
             continue
@@ -140,6 +141,41 @@ def test_two_bit_batched_decode_shares_launches(M):
     for x, X, i, y in zip(Xd, Xs, order, Yb):
         single = L.linear(x, layers[i][1], ws)
         assert torch.equal(single, y)
+        assert worst_ratio(y.cpu().numpy(), olqer.forward(X, layers[i][0], w_bits=2)) <= 1.0
+    for _, Pg in layers:
+        Pg.release()
+
+
+@pytest.mark.parametrize("M", [6, 16])
+def test_two_bit_small_batches_share_launches(M):
+    # twelve independent calls above the column-owner kernel's range: one launch of the small prologue and one of the
+    # register-operand GEMM (crumbs converted in registers), every result within the tolerance of the oracle's and
+    # the second run of the batch equal to the first bit for bit
+    specs = [gen.LayerSpec("w2_sm_a", M=M, K=1024, N=640, k=40, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=421),
+             gen.LayerSpec("w2_sm_b", M=M, K=2112, N=264, k=72, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=422)]
+    layers = []
+    for s in specs:
+        W = gen.make_weight(s)
+        A, B = gen.make_random_factors(s)
+        layers.append((olqer.prepare_weights(W, A, B, w_bits=2), L.prepare_weights(_t(W), _t(A), _t(B), _cfg())))
+    order = [0, 1] * 6
+    Xs = [gen.make_activations(specs[i], M=M) + 0.125 * j for j, i in enumerate(order)]
+    Xd = [_t(X) for X in Xs]
+    Yb = [torch.full((M, specs[i].N), float("nan"), dtype=torch.float32, device=DEV) for i in order]
+    calls = L.make_calls([(x, layers[i][1], y) for x, i, y in zip(Xd, order, Yb)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    first = None
+    for rep in range(2):
+        before = L.launch_count()
+        L.linear_batched(calls, ws)
+        torch.cuda.synchronize()
+        assert L.launch_count() - before == 2
+        assert L.poll_status(ws) == 0
+        if first is None:
+            first = [y.clone() for y in Yb]
+        else:
+            assert all(torch.equal(a, b) for a, b in zip(first, Yb))
+    for X, i, y in zip(Xs, order, Yb):
         assert worst_ratio(y.cpu().numpy(), olqer.forward(X, layers[i][0], w_bits=2)) <= 1.0
     for _, Pg in layers:
         Pg.release()
