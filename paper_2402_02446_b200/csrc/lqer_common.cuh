@@ -513,9 +513,10 @@ int prologue_small_max_layers();
 // kFlagAreaOffset on, used by nothing else): flags[0] takes the launch's `epoch` once every CTA's share of X_q is in
 // place (the CTAs count themselves in at counts[kCountXq]; the last one sets it back to zero), flags[1] once T_q is.
 // An epoch is a number that no earlier launch on this workspace used, so a flag left by the call before never
-// passes for this call's, and the flags need no reset.
+// passes for this call's, whenever the two overlap; the GEMM's last CTA clears the flags when it leaves (a counter
+// behind them counts its CTAs out), which is what a replayed graph, whose epoch repeats, relies on.
 constexpr int kCountXq = 1;
-constexpr int kFlagAreaOffset = 64;                 // status area bytes [64, 64 + 16 layers * 8)
+constexpr int kFlagAreaOffset = 64;                 // status area bytes [64, 64 + 16 layers * 8), then the exit counter
 inline int frag_rank_slabs(const PackedMeta& m) { return (m.k_pad + 63) / 64; }
 inline size_t frag_bytes(const PackedMeta& m) { return (size_t)8 * (m.k_slabs + frag_rank_slabs(m)) * 256; }
 cudaError_t launch_prologue_small(const SmallPrologueLayer* layers, int n, int M, int x_type, bool frag_order, int epoch,

@@ -32,7 +32,9 @@
 // resident or done by the time this one starts (the launch order of programmatic dependent launches), so it never
 // depends on this kernel's progress.  The flags are raised only after the prologue's own wait for the kernels before
 // it, so whatever this kernel writes after seeing a flag cannot collide with them.  A flag holds the launch's epoch, a
-// number no earlier launch on the workspace used: the flag the call before left behind never passes for this call's.
+// number no earlier launch on the workspace used: the flag the call before left behind never passes for this call's,
+// even while that call's last CTAs are still running.  The last CTA to leave clears the flags all the same, so that a
+// captured graph, whose replays repeat the epoch, starts from cleared flags too.
 #include "lqer_gemm_small.cuh"
 #include "lqer_tc_ptx.cuh"
 
@@ -421,6 +423,14 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
       const long long t0 = clock64();
       while (clock64() - t0 < 400000) { }          // a copy requested before the give-up lands well within this
       report_error(p.status, LQER_ERR_TIMEOUT, 720, blockIdx.x);
+    } else {
+      // The last CTA to leave clears the flags.  Epochs already keep a later launch from taking them for its own; a
+      // replay of a captured graph, though, repeats its epoch, and must find the flags as the first run found them.
+      __threadfence();
+      if (atomicAdd(p.exit_count, 1) == (int)gridDim.x - 1) {
+        for (int l = 0; l < p.n; ++l) { p.L[l].flags[0] = 0; p.L[l].flags[1] = 0; }
+        *p.exit_count = 0;
+      }
     }
   }
 }

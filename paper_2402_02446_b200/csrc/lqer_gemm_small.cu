@@ -506,6 +506,7 @@ cudaError_t launch_gemm_small(const SmallGemmLayer* layers, int n, int M, int y_
   p.w_bits = layers[0].meta->w_bits;
   p.wait_limit = wait_limit_cycles();
   p.epoch = epoch;
+  p.exit_count = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(st) + kFlagAreaOffset + 2 * MAX_LAYERS * 4);
   p.stall = take_stall(kFamDecode) ? 1 : 0;
   if (use_mma) return launch_gemm_mma(p, s);
   const int ctas = p.num_items < sms ? p.num_items : sms;

@@ -14,7 +14,7 @@ struct Layer {
   const uint8_t* wsec;
   const uint8_t* bsec;
   const uint8_t* xfrag;        // register-operand kernel: [X_q | T_q] in fragment order (eight planes of `plane` bytes)
-  const int* flags;            // ... and the prologue's two flags for this layer (X_q in place, T_q in place)
+  int* flags;                  // ... and the prologue's two flags for this layer (X_q in place, T_q in place)
   void* Y;                     // [M, N] fp32 or bf16, or the MXINT8 sections (mantissas [M, N], exponent bytes [M, N / 16])
   float* partials;             // [tile][chunk][M][256] fp32 (tiles with more than one chunk)
   int* counters;               // [tile] arrivals, zero between calls
@@ -40,6 +40,7 @@ struct Params {
   int x_rows;                  // rows of an activation tile that TMA fills: M rounded up to 8 (the rest stay zero)
   long long wait_limit;
   int epoch;                   // register-operand kernel: the value the prologue's flags take in this call
+  int* exit_count;             // ... and a zeroed counter of the CTAs that have left (the last one clears the flags)
   int stall;                   // test hook: the producer withholds the last stage of its last item
 };
 

@@ -83,3 +83,34 @@ def test_forced_single_call_equals_itself_and_the_oracle_on_a_long_layer():
     assert worst_ratio(Y1.cpu().numpy(), ref) <= 1.0
     assert torch.equal(Y1, Y2)
     Pg.release()
+
+
+def test_replays_of_a_captured_graph_follow_their_inputs():
+    # a captured batch repeats its launch parameters, the epoch of the prologue's flags among them: every replay must
+    # still wait for its own prologue, so a replay on new activations gives the new results
+    spec = gen.LayerSpec("mma_graph", M=9, K=1024, N=640, k=40, calib_rows=32, outlier_frac=0.01, outlier_scale=20.0, seed=703)
+    P, Pg = _layer(spec)
+    n = 8
+    Xd = [torch.zeros((9, spec.K), dtype=torch.float32, device=DEV) for _ in range(n)]
+    Ys = [torch.zeros((9, spec.N), dtype=torch.float32, device=DEV) for _ in range(n)]
+    calls = L.make_calls([(x, Pg, y) for x, y in zip(Xd, Ys)])
+    ws = torch.zeros(L.batched_workspace_bytes(calls), dtype=torch.uint8, device=DEV)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        L.linear_batched(calls, ws, stream=s)              # first use of the kernels outside the capture
+    s.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        L.linear_batched(calls, ws, stream=torch.cuda.current_stream())
+    for rep in range(3):
+        Xs = [gen.make_activations(spec, M=9) * (1.0 + rep) + 0.25 * i for i in range(n)]
+        for x, X in zip(Xd, Xs):
+            x.copy_(_t(X))
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        assert L.poll_status(ws) == 0
+        for X, y in zip(Xs, Ys):
+            assert worst_ratio(y.cpu().numpy(), olqer.forward(X, P)) <= 1.0, rep
+    Pg.release()
