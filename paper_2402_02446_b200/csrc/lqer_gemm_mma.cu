@@ -263,21 +263,32 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
     // Sub-chunk n of the item: up to SUB_SLABS slabs of X_q, or (the last one of a tile's last chunk) the slabs of T_q.
     auto sub_lo = [&](int n) { return n < n_w ? w_lo + n * SUB_SLABS : ly.k_slabs; };
     auto sub_len = [&](int n) { return n < n_w ? min(SUB_SLABS, w_hi - (w_lo + n * SUB_SLABS)) : r_slabs; };
-    // Thread 0: waits for what sub-chunk n needs of the prologue, then requests its eight planes into buffer `copies & 1`.
-    auto request = [&](int n) {
+    // Thread 0: waits for what sub-chunk n needs of the prologue, then requests its eight planes as copy number `copy`
+    // (buffer copy & 1).  With `ahead` (the request is made a sub-chunk early) a T_q that is not there yet is not waited
+    // for: the request is put off (returns false) and made again when its turn comes, so that a short chunk's weight
+    // loop runs while T is still being formed.
+    auto request = [&](int n, uint32_t copy, bool ahead) -> bool {
       const int want = p.stall != 0 ? ~p.epoch : p.epoch;   // test hook: a value the flags never take
       if (n == 0 || n >= n_w) {
-        if (!poll_flag(ly.flags + (n < n_w ? 0 : 1), want, ws)) return;
+        const int* flag = ly.flags + (n < n_w ? 0 : 1);
+        if (ahead) {
+          int v;
+          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+          if (v != want) return false;
+        } else if (!poll_flag(flag, want, ws)) {
+          return true;                                       // given up: nothing is requested, every wait runs out
+        }
         asm volatile("fence.proxy.async.global;" ::: "memory");       // what the flag vouches for, before the copies read it
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // this buffer's earlier readers, before the copies overwrite it
       const int len = sub_len(n);
-      const uint32_t bar = tc::smem_u32(bars + (copies & 1));
-      const uint32_t dst = tc::smem_u32(smem + (copies & 1) * BUF_BYTES);
+      const uint32_t bar = tc::smem_u32(bars + (copy & 1));
+      const uint32_t dst = tc::smem_u32(smem + (copy & 1) * BUF_BYTES);
       const uint8_t* src = ly.xfrag + (size_t)sub_lo(n) * 256;
       tc::mbar_expect_tx(bar, 8u * len * 256u);
 #pragma unroll
       for (int q = 0; q < 8; ++q) tc::bulk_load(dst + q * PLANE_BYTES, src + (size_t)q * ly.plane, len * 256, bar);
+      return true;
     };
     // Every thread: an odd sub-chunk ends in half a step; the slab after its last one reads as zeros.
     auto zero_tail = [&](int n) {
@@ -287,9 +298,10 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
     };
 
     __syncthreads();                             // the item before has left both buffers (and the staged tile)
-    if (tid == 0) request(0);
+    if (tid == 0) request(0, copies, false);
     zero_tail(0);
     ++copies;
+    bool put_off = false;                        // thread 0: the request of the next sub-chunk was put off
     // the first step's weights (after the request, whose fence would otherwise sit behind these loads)
     if (warp_live) {
       const size_t off = (size_t)slab_of(w_lo) * kTile;
@@ -307,8 +319,12 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
 
     for (int n = 0; n < n_sub; ++n) {
       __syncthreads();                           // sub-chunk n - 1 has been read: its buffer is free; zeroed tails are visible
+      if (tid == 0 && put_off) {                 // this sub-chunk's own request, put off a round ago
+        request(n, copies - 1, false);
+        put_off = false;
+      }
       if (n + 1 < n_sub) {
-        if (tid == 0) request(n + 1);
+        if (tid == 0) put_off = !request(n + 1, copies, true);
         zero_tail(n + 1);
         ++copies;
       }
