@@ -58,7 +58,7 @@ __device__ __forceinline__ size_t frag_offset(int row, int slab, int c, size_t p
 
 // TPW: rank tiles (8 columns) a warp owns: 1 for ranks up to 64, 2 up to 128, 4 up to 256.
 template <int TPW>
-__global__ void __launch_bounds__(kThreads) prologue_small_kernel(const __grid_constant__ Params p) {
+__global__ void __launch_bounds__(kThreads, TPW == 1 ? 3 : TPW == 2 ? 2 : 1) prologue_small_kernel(const __grid_constant__ Params p) {
   __shared__ __align__(16) uint8_t s_xq[kRows * kXqStride];
   __shared__ int8_t s_xe[kRows][kStepCols / 16];
   __shared__ double s_part[kWarps][kRows * 8];        // warps that share a rank tile meet here (TPW == 1)
