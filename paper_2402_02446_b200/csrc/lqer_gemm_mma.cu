@@ -392,7 +392,7 @@ gemm_mma_kernel(const __grid_constant__ Params p) {
       }
     } else {
       // the only chunk: through shared memory, so that a thread ends up with a whole 16-block of a row
-      __syncthreads();                                // the activation records have been read
+      __syncthreads();                                // the activation buffers have been read
       if (warp_live) {
 #pragma unroll
         for (int o = 0; o < 4; ++o) {
